@@ -1,0 +1,372 @@
+/*
+ * TWEO / FP8 per-tensor linear path -- CPU ORACLE.
+ *
+ * This file is TEST INFRASTRUCTURE, not product code.  It is a plain, slow,
+ * scalar restatement of what the hot path computes, written from the paper's
+ * definitions so that a reader can check it against them by eye:
+ *
+ *   - the TWEO regulariser (paper Eq. 3) and its derivative (paper Eq. 2 times
+ *     Eq. 3, differentiated with respect to each activation),
+ *   - per-tensor FP8 scaling and casting (paper Sec. 4.2: one scale for the
+ *     whole tensor, E4M3 forward / E5M2 gradients; E4M3 range +-448 from the
+ *     paper's introduction) with the OCP FP8 code tables,
+ *   - the three linear-layer contractions on the quantised operands,
+ *   - symmetric AbsMax b-bit quantisation (paper Eq. 4).
+ *
+ * Floating point is FP64 unless the step is *defined* in FP32 (the scale, the
+ * scaled value that gets rounded to FP8).  There is no blocking, no SIMD, no
+ * BLAS, no reordering: sums run in index order.  OpenMP only splits outer
+ * rows between threads, which changes no value.
+ *
+ * It shares no code, header, table or constant generator with the CUDA path
+ * and neither includes the other.  Only tests, the smoke check and the
+ * benchmark's CPU-baseline leg may link or load this.
+ *
+ * Pins (see the CPU tests): every function below is pinned to something
+ * outside itself -- printed values from the paper, closed forms, brute force,
+ * finite differences, or an independent library routine.  Nothing here is
+ * "parity unpinned".
+ */
+#include <float.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_E4M3 0
+#define ORACLE_E5M2 1
+
+/* ------------------------------------------------------------------ bf16 */
+
+/* bf16 is the upper half of an IEEE binary32; widening is exact. */
+static float bf16_bits_to_f32(uint16_t b) {
+  uint32_t u = ((uint32_t)b) << 16;
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return f;
+}
+
+float oracle_bf16_to_f32(uint16_t b) { return bf16_bits_to_f32(b); }
+
+/* Round a double to bf16 (8 significant bits, binary32 exponent range),
+ * round-to-nearest, ties to even, in ONE rounding from the double.
+ * Overflow goes to infinity as IEEE prescribes; NaN maps to 0x7FC0|sign. */
+uint16_t oracle_f64_to_bf16(double v) {
+  if (isnan(v)) return (uint16_t)(signbit(v) ? 0xFFC0 : 0x7FC0);
+  uint16_t sign = signbit(v) ? 0x8000 : 0;
+  double a = fabs(v);
+  if (a == 0.0) return sign;
+  if (isinf(a)) return (uint16_t)(sign | 0x7F80);
+  int ex;
+  (void)frexp(a, &ex);      /* a = f * 2^ex, f in [0.5,1)            */
+  int E = ex - 1;           /* a = m * 2^E,  m in [1,2)              */
+  const int MBITS = 7, BIAS = 127, EMIN = -126;
+  if (E < EMIN) {           /* subnormal: spacing 2^(EMIN-MBITS)     */
+    double q = ldexp(a, -(EMIN - MBITS));
+    double r = nearbyint(q); /* default rounding mode = ties-to-even */
+    return (uint16_t)(sign | (uint16_t)r); /* r==128 carries into e=1 */
+  }
+  double q = ldexp(a, -(E - MBITS)); /* in [128,256) */
+  double r = nearbyint(q);
+  if (r == 256.0) { r = 128.0; E += 1; }
+  if (E > 127) return (uint16_t)(sign | 0x7F80);
+  return (uint16_t)(sign | ((uint16_t)(E + BIAS) << MBITS) | ((uint16_t)r - 128));
+}
+
+void oracle_f64_array_to_bf16(const double* v, int64_t n, uint16_t* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = oracle_f64_to_bf16(v[i]);
+}
+
+/* ------------------------------------------------------------ FP8 tables */
+
+/* OCP FP8 value of one code.  E4M3: 1 sign, 4 exponent (bias 7), 3 mantissa,
+ * no infinities, the single NaN pattern is exponent=15 & mantissa=7; largest
+ * finite value is 1.75 * 2^8 = 448 (the range the paper quotes).
+ * E5M2: 1 sign, 5 exponent (bias 15), 2 mantissa, IEEE-style inf/NaN;
+ * largest finite value is 1.75 * 2^15 = 57344. */
+double oracle_fp8_decode(uint8_t code, int fmt) {
+  int s = code >> 7;
+  double sign = s ? -1.0 : 1.0;
+  if (fmt == ORACLE_E4M3) {
+    int e = (code >> 3) & 15, m = code & 7;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) return sign * ldexp((double)m, -9);
+    return sign * ldexp(1.0 + m / 8.0, e - 7);
+  } else {
+    int e = (code >> 2) & 31, m = code & 3;
+    if (e == 31) return m == 0 ? sign * INFINITY : NAN;
+    if (e == 0) return sign * ldexp((double)m, -16);
+    return sign * ldexp(1.0 + m / 4.0, e - 15);
+  }
+}
+
+double oracle_fp8_max(int fmt) { return fmt == ORACLE_E4M3 ? 448.0 : 57344.0; }
+static uint8_t fp8_max_code(int fmt) { return fmt == ORACLE_E4M3 ? 0x7E : 0x7B; }
+
+/* Encoder A (arithmetic).  Saturating round-to-nearest-even of a binary32
+ * value: NaN -> sign|0x7F; |v| >= max finite (infinity included) -> sign|max
+ * code; otherwise the nearest representable value, ties to the even code;
+ * zero and values that round to zero keep their sign. */
+uint8_t oracle_fp8_encode(float v, int fmt) {
+  uint8_t sign = signbit(v) ? 0x80 : 0x00;
+  if (isnan(v)) return (uint8_t)(sign | 0x7F);
+  double a = fabs((double)v);
+  if (a >= oracle_fp8_max(fmt)) return (uint8_t)(sign | fp8_max_code(fmt));
+  if (a == 0.0) return sign;
+  const int MBITS = fmt == ORACLE_E4M3 ? 3 : 2;
+  const int BIAS = fmt == ORACLE_E4M3 ? 7 : 15;
+  const int EMIN = 1 - BIAS;
+  int ex;
+  (void)frexp(a, &ex);
+  int E = ex - 1; /* a = m * 2^E with m in [1,2) */
+  if (E < EMIN) {
+    /* subnormal grid: multiples of 2^(EMIN-MBITS); a carry to 2^MBITS is the
+     * smallest normal number, whose code is exactly that integer. */
+    double r = nearbyint(ldexp(a, -(EMIN - MBITS)));
+    return (uint8_t)(sign | (uint8_t)r);
+  }
+  double r = nearbyint(ldexp(a, -(E - MBITS))); /* in [2^MBITS, 2^(MBITS+1)] */
+  if (r == (double)(2 << MBITS)) { r = (double)(1 << MBITS); E += 1; }
+  return (uint8_t)(sign | ((uint8_t)(E + BIAS) << MBITS) | ((uint8_t)r - (1 << MBITS)));
+}
+
+/* Encoder B (brute force).  Same contract, no exponent arithmetic: look at
+ * every non-negative finite code, keep the closest decoded value, and on an
+ * exact tie keep the code whose last bit is 0.  Used only to cross-check A. */
+uint8_t oracle_fp8_encode_search(float v, int fmt) {
+  uint8_t sign = signbit(v) ? 0x80 : 0x00;
+  if (isnan(v)) return (uint8_t)(sign | 0x7F);
+  double a = fabs((double)v);
+  if (a >= oracle_fp8_max(fmt)) return (uint8_t)(sign | fp8_max_code(fmt));
+  int best = 0;
+  double best_d = INFINITY;
+  for (int c = 0; c <= fp8_max_code(fmt); ++c) {
+    double d = fabs(oracle_fp8_decode((uint8_t)c, fmt) - a); /* exact in FP64 */
+    if (d < best_d || (d == best_d && (c & 1) == 0)) { best_d = d; best = c; }
+  }
+  return (uint8_t)(sign | best);
+}
+
+/* Element-wise application of encoder A (which = 0) or B (which = 1). */
+void oracle_fp8_encode_array(const float* v, int64_t n, int fmt, int which, uint8_t* out) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < n; ++i)
+    out[i] = which ? oracle_fp8_encode_search(v[i], fmt) : oracle_fp8_encode(v[i], fmt);
+}
+
+/* ------------------------------------------------- amax / scale / quantize */
+
+/* amax = max_i |x_i| over the whole tensor (one scale per tensor, Sec. 4.2).
+ * NaN elements are skipped (fmax semantics); infinities count. */
+float oracle_amax_bf16(const uint16_t* x, int64_t n) {
+  float amax = 0.0f;
+  for (int64_t i = 0; i < n; ++i) {
+    float a = fabsf(bf16_bits_to_f32(x[i]));
+    if (a > amax) amax = a; /* false for NaN */
+  }
+  return amax;
+}
+
+/* scale = fl32(FP8MAX / amax) so that the largest element lands on the
+ * format's largest finite value; scale_inv = fl32(1 / scale).  Degenerate
+ * tensors (amax = 0, or non-finite) get scale 1; a quotient that overflows
+ * binary32 is clamped to FLT_MAX. */
+void oracle_scale_from_amax(float amax, int fmt, float* scale, float* scale_inv) {
+  float s = 1.0f;
+  if (amax > 0.0f && isfinite(amax)) {
+    volatile float q = (float)oracle_fp8_max(fmt) / amax; /* one fp32 division */
+    s = q;
+    if (isinf(s)) s = FLT_MAX;
+  }
+  volatile float inv = 1.0f / s;
+  *scale = s;
+  *scale_inv = inv;
+}
+
+/* q_i = encode( fl32( x_i * scale ) ): one binary32 multiply (round to
+ * nearest even, not fused with anything), then one saturating RNE to FP8.
+ * sat_count (optional) = number of elements whose scaled magnitude exceeds
+ * the largest finite FP8 value, i.e. that the saturation actually clips. */
+void oracle_quantize_bf16(const uint16_t* x, int64_t n, int fmt, float scale,
+                          uint8_t* q, uint64_t* sat_count) {
+  uint64_t sat = 0;
+  const float fmax = (float)oracle_fp8_max(fmt);
+  for (int64_t i = 0; i < n; ++i) {
+    volatile float v = bf16_bits_to_f32(x[i]) * scale;
+    q[i] = oracle_fp8_encode(v, fmt);
+    if (fabsf(v) > fmax) ++sat; /* false for NaN */
+  }
+  if (sat_count) *sat_count = sat;
+}
+
+/* ------------------------------------------------------------------ GEMMs */
+/* All three take the FP8 codes, decode them, and sum in FP64 in index order,
+ * then apply the two dequantisation factors.  Storage (row-major):
+ *   xq  [M, K]   activations          (ldx  elements between rows)
+ *   wq  [N, K]   weights, one row per output feature
+ *   dyq [M, N]   output gradients
+ * Products of two FP8 values are small dyadic rationals, so for the
+ * contraction lengths used here the FP64 sums are exact. */
+
+static void fill_table(double* t, int fmt) {
+  for (int c = 0; c < 256; ++c) t[c] = oracle_fp8_decode((uint8_t)c, fmt);
+}
+
+/* forward: Y[i,j] = (sum_k X[i,k] W[j,k]) * sx_inv * sw_inv */
+void oracle_gemm_fwd(const uint8_t* xq, int64_t ldx, int fmt_x,
+                     const uint8_t* wq, int64_t ldw, int fmt_w,
+                     double sx_inv, double sw_inv,
+                     int64_t M, int64_t N, int64_t K, double* y, int64_t ldy) {
+  double tx[256], tw[256];
+  fill_table(tx, fmt_x);
+  fill_table(tw, fmt_w);
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t j = 0; j < N; ++j) {
+      double acc = 0.0;
+      for (int64_t k = 0; k < K; ++k) acc += tx[xq[i * ldx + k]] * tw[wq[j * ldw + k]];
+      y[i * ldy + j] = acc * sx_inv * sw_inv;
+    }
+}
+
+/* data gradient: dX[i,k] = (sum_n dY[i,n] W[n,k]) * sdy_inv * sw_inv */
+void oracle_gemm_dgrad(const uint8_t* dyq, int64_t lddy, int fmt_dy,
+                       const uint8_t* wq, int64_t ldw, int fmt_w,
+                       double sdy_inv, double sw_inv,
+                       int64_t M, int64_t N, int64_t K, double* dx, int64_t lddx) {
+  double tdy[256], tw[256];
+  fill_table(tdy, fmt_dy);
+  fill_table(tw, fmt_w);
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t k = 0; k < K; ++k) {
+      double acc = 0.0;
+      for (int64_t n = 0; n < N; ++n) acc += tdy[dyq[i * lddy + n]] * tw[wq[n * ldw + k]];
+      dx[i * lddx + k] = acc * sdy_inv * sw_inv;
+    }
+}
+
+/* weight gradient: dW[n,k] = (sum_m dY[m,n] X[m,k]) * sx_inv * sdy_inv */
+void oracle_gemm_wgrad(const uint8_t* xq, int64_t ldx, int fmt_x,
+                       const uint8_t* dyq, int64_t lddy, int fmt_dy,
+                       double sx_inv, double sdy_inv,
+                       int64_t M, int64_t N, int64_t K, double* dw, int64_t lddw) {
+  double tx[256], tdy[256];
+  fill_table(tx, fmt_x);
+  fill_table(tdy, fmt_dy);
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < N; ++n)
+    for (int64_t k = 0; k < K; ++k) {
+      double acc = 0.0;
+      for (int64_t m = 0; m < M; ++m) acc += tdy[dyq[m * lddy + n]] * tx[xq[m * ldx + k]];
+      dw[n * lddw + k] = acc * sx_inv * sdy_inv;
+    }
+}
+
+/* The same three definitions evaluated only at a list of output positions
+ * (rows[t], cols[t]); used where a full FP64 product would take hours. */
+void oracle_gemm_fwd_at(const uint8_t* xq, int64_t ldx, int fmt_x,
+                        const uint8_t* wq, int64_t ldw, int fmt_w,
+                        double sx_inv, double sw_inv, int64_t K,
+                        const int64_t* rows, const int64_t* cols, int64_t npts, double* out) {
+  double tx[256], tw[256];
+  fill_table(tx, fmt_x);
+  fill_table(tw, fmt_w);
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < npts; ++t) {
+    int64_t i = rows[t], j = cols[t];
+    double acc = 0.0;
+    for (int64_t k = 0; k < K; ++k) acc += tx[xq[i * ldx + k]] * tw[wq[j * ldw + k]];
+    out[t] = acc * sx_inv * sw_inv;
+  }
+}
+
+void oracle_gemm_dgrad_at(const uint8_t* dyq, int64_t lddy, int fmt_dy,
+                          const uint8_t* wq, int64_t ldw, int fmt_w,
+                          double sdy_inv, double sw_inv, int64_t N,
+                          const int64_t* rows, const int64_t* cols, int64_t npts, double* out) {
+  double tdy[256], tw[256];
+  fill_table(tdy, fmt_dy);
+  fill_table(tw, fmt_w);
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < npts; ++t) {
+    int64_t i = rows[t], k = cols[t];
+    double acc = 0.0;
+    for (int64_t n = 0; n < N; ++n) acc += tdy[dyq[i * lddy + n]] * tw[wq[n * ldw + k]];
+    out[t] = acc * sdy_inv * sw_inv;
+  }
+}
+
+void oracle_gemm_wgrad_at(const uint8_t* xq, int64_t ldx, int fmt_x,
+                          const uint8_t* dyq, int64_t lddy, int fmt_dy,
+                          double sx_inv, double sdy_inv, int64_t M,
+                          const int64_t* rows, const int64_t* cols, int64_t npts, double* out) {
+  double tx[256], tdy[256];
+  fill_table(tx, fmt_x);
+  fill_table(tdy, fmt_dy);
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < npts; ++t) {
+    int64_t n = rows[t], k = cols[t];
+    double acc = 0.0;
+    for (int64_t m = 0; m < M; ++m) acc += tdy[dyq[m * lddy + n]] * tx[xq[m * ldx + k]];
+    out[t] = acc * sx_inv * sdy_inv;
+  }
+}
+
+/* ------------------------------------------------------------------- TWEO */
+
+/* Eq. 3 for one block output: the mean over all n elements of
+ * (|a_i| / (tau + eps))^p.  eps is added to tau, as printed. */
+double oracle_tweo_loss_block(const uint16_t* a, int64_t n, double tau, double eps, double p) {
+  const double d = tau + eps;
+  double sum = 0.0;
+  for (int64_t i = 0; i < n; ++i) {
+    double r = fabs((double)bf16_bits_to_f32(a[i])) / d;
+    sum += pow(r, p);
+  }
+  return n > 0 ? sum / (double)n : 0.0;
+}
+
+/* Derivative of  c * (1/n) sum_i (|a_i|/(tau+eps))^p  with respect to a_i:
+ *   g_i = c * p * sign(a_i) * |a_i|^(p-1) / (n * (tau+eps)^p),   g_i = 0 at a_i = 0.
+ * The caller folds lambda(t) (Eq. 2), the 1/L of Eq. 3 and any upstream
+ * gradient into the single coefficient c. */
+void oracle_tweo_grad_block(const uint16_t* a, int64_t n, double tau, double eps, double p,
+                            double c, double* g) {
+  const double d = tau + eps;
+  const double k = c * p / ((double)n * pow(d, p));
+  for (int64_t i = 0; i < n; ++i) {
+    double v = (double)bf16_bits_to_f32(a[i]);
+    if (v == 0.0 || isnan(v)) { g[i] = v == 0.0 ? 0.0 : NAN; continue; }
+    double s = v > 0.0 ? 1.0 : -1.0;
+    g[i] = k * s * pow(fabs(v), p - 1.0);
+  }
+}
+
+/* ------------------------------------------------- Eq. 4, integer AbsMax */
+
+/* s = max|X| + eps;  X_q = round(X / s * Q_b), Q_b = 2^(b-1) - 1, ties to
+ * even, clamped to [-Q_b, Q_b] (the clamp only acts when a static s is
+ * smaller than the tensor's own maximum).  Returns Q_b. */
+int oracle_absmax_qmax(int bits) { return (1 << (bits - 1)) - 1; }
+
+void oracle_absmax_quantize(const double* x, int64_t n, int bits, double s, int32_t* xq) {
+  const double Q = (double)oracle_absmax_qmax(bits);
+  for (int64_t i = 0; i < n; ++i) {
+    double r = nearbyint(x[i] / s * Q);
+    if (r > Q) r = Q;
+    if (r < -Q) r = -Q;
+    xq[i] = (int32_t)r;
+  }
+}
+
+void oracle_absmax_dequantize(const int32_t* xq, int64_t n, int bits, double s, double* x) {
+  const double Q = (double)oracle_absmax_qmax(bits);
+  for (int64_t i = 0; i < n; ++i) x[i] = (double)xq[i] / Q * s;
+}
+
+double oracle_absmax_scale(const double* x, int64_t n, double eps) {
+  double m = 0.0;
+  for (int64_t i = 0; i < n; ++i) if (fabs(x[i]) > m) m = fabs(x[i]);
+  return m + eps;
+}

@@ -1,0 +1,295 @@
+"""ctypes front end of the CPU oracle (``tweo_oracle.c``).
+
+TEST INFRASTRUCTURE.  Only tests, the smoke check and the benchmark's CPU
+baseline leg may import this module.  It performs no arithmetic of the method
+itself: every function marshals numpy arrays into the C routines, which are
+the plain restatement of the paper's definitions (Eq. 2-4, Sec. 4.2).  It does
+not import, and is not imported by, the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+E4M3 = 0
+E5M2 = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "tweo_oracle.c")
+_LIB = os.path.join(_HERE, "libtweo_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain -O2, no fast-math, no contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-std=c11", "-O2", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
+             "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _p(arr, ctype):
+    return arr.ctypes.data_as(C.POINTER(ctype))
+
+
+def lib():
+    global _lib
+    with _lock:
+        if _lib is None:
+            L = C.CDLL(build())
+            L.oracle_bf16_to_f32.restype = C.c_float
+            L.oracle_bf16_to_f32.argtypes = [C.c_uint16]
+            L.oracle_f64_to_bf16.restype = C.c_uint16
+            L.oracle_f64_to_bf16.argtypes = [C.c_double]
+            L.oracle_f64_array_to_bf16.restype = None
+            L.oracle_f64_array_to_bf16.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+            L.oracle_fp8_encode_array.restype = None
+            L.oracle_fp8_encode_array.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_void_p]
+            L.oracle_fp8_decode.restype = C.c_double
+            L.oracle_fp8_decode.argtypes = [C.c_uint8, C.c_int]
+            L.oracle_fp8_max.restype = C.c_double
+            L.oracle_fp8_max.argtypes = [C.c_int]
+            for name in ("oracle_fp8_encode", "oracle_fp8_encode_search"):
+                f = getattr(L, name)
+                f.restype = C.c_uint8
+                f.argtypes = [C.c_float, C.c_int]
+            L.oracle_amax_bf16.restype = C.c_float
+            L.oracle_amax_bf16.argtypes = [C.c_void_p, C.c_int64]
+            L.oracle_scale_from_amax.restype = None
+            L.oracle_scale_from_amax.argtypes = [C.c_float, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_float)]
+            L.oracle_quantize_bf16.restype = None
+            L.oracle_quantize_bf16.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_float, C.c_void_p,
+                                               C.POINTER(C.c_uint64)]
+            for name in ("oracle_gemm_fwd", "oracle_gemm_dgrad", "oracle_gemm_wgrad"):
+                f = getattr(L, name)
+                f.restype = None
+                f.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_int64, C.c_int,
+                              C.c_double, C.c_double, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int64]
+            for name in ("oracle_gemm_fwd_at", "oracle_gemm_dgrad_at", "oracle_gemm_wgrad_at"):
+                f = getattr(L, name)
+                f.restype = None
+                f.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_int64, C.c_int,
+                              C.c_double, C.c_double, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
+            L.oracle_tweo_loss_block.restype = C.c_double
+            L.oracle_tweo_loss_block.argtypes = [C.c_void_p, C.c_int64, C.c_double, C.c_double, C.c_double]
+            L.oracle_tweo_grad_block.restype = None
+            L.oracle_tweo_grad_block.argtypes = [C.c_void_p, C.c_int64, C.c_double, C.c_double, C.c_double,
+                                                 C.c_double, C.c_void_p]
+            L.oracle_absmax_qmax.restype = C.c_int
+            L.oracle_absmax_qmax.argtypes = [C.c_int]
+            L.oracle_absmax_quantize.restype = None
+            L.oracle_absmax_quantize.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_double, C.c_void_p]
+            L.oracle_absmax_dequantize.restype = None
+            L.oracle_absmax_dequantize.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_double, C.c_void_p]
+            L.oracle_absmax_scale.restype = C.c_double
+            L.oracle_absmax_scale.argtypes = [C.c_void_p, C.c_int64, C.c_double]
+            _lib = L
+    return _lib
+
+
+def _u16(x):
+    x = np.ascontiguousarray(x)
+    assert x.dtype == np.uint16, "bf16 tensors are passed as their uint16 bit patterns"
+    return x
+
+
+def _u8(x, ndim=None):
+    x = np.ascontiguousarray(x)
+    assert x.dtype == np.uint8
+    if ndim is not None:
+        assert x.ndim == ndim
+    return x
+
+
+# ---------------------------------------------------------------- scalars
+def bf16_to_f32(bits: int) -> float:
+    return float(lib().oracle_bf16_to_f32(int(bits)))
+
+
+def f64_to_bf16(v: float) -> int:
+    return int(lib().oracle_f64_to_bf16(float(v)))
+
+
+def f64_array_to_bf16(v) -> np.ndarray:
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    out = np.empty(v.shape, dtype=np.uint16)
+    lib().oracle_f64_array_to_bf16(v.ctypes.data, v.size, out.ctypes.data)
+    return out
+
+
+def fp8_decode(code: int, fmt: int) -> float:
+    return float(lib().oracle_fp8_decode(int(code), fmt))
+
+
+def fp8_decode_table(fmt: int) -> np.ndarray:
+    return np.array([fp8_decode(c, fmt) for c in range(256)], dtype=np.float64)
+
+
+def fp8_max(fmt: int) -> float:
+    return float(lib().oracle_fp8_max(fmt))
+
+
+def fp8_encode(v, fmt: int) -> int:
+    return int(lib().oracle_fp8_encode(np.float32(v), fmt))
+
+
+def fp8_encode_search(v, fmt: int) -> int:
+    return int(lib().oracle_fp8_encode_search(np.float32(v), fmt))
+
+
+def fp8_encode_array(v, fmt: int, search: bool = False) -> np.ndarray:
+    v = np.ascontiguousarray(v, dtype=np.float32)
+    out = np.empty(v.shape, dtype=np.uint8)
+    lib().oracle_fp8_encode_array(v.ctypes.data, v.size, fmt, 1 if search else 0, out.ctypes.data)
+    return out
+
+
+# ---------------------------------------------------------------- tensors
+def amax_bf16(x_bits) -> np.float32:
+    x = _u16(x_bits)
+    return np.float32(lib().oracle_amax_bf16(x.ctypes.data, x.size))
+
+
+def scale_from_amax(amax, fmt: int):
+    s, si = C.c_float(), C.c_float()
+    lib().oracle_scale_from_amax(np.float32(amax), fmt, C.byref(s), C.byref(si))
+    return np.float32(s.value), np.float32(si.value)
+
+
+def quantize_bf16(x_bits, fmt: int, scale):
+    """Returns (codes uint8 with x's shape, sat_count)."""
+    x = _u16(x_bits)
+    q = np.empty(x.shape, dtype=np.uint8)
+    sat = C.c_uint64(0)
+    lib().oracle_quantize_bf16(x.ctypes.data, x.size, fmt, np.float32(scale), q.ctypes.data, C.byref(sat))
+    return q, int(sat.value)
+
+
+def quantize_per_tensor_current(x_bits, fmt: int):
+    """amax -> scale -> cast; returns dict(amax, scale, scale_inv, q, sat_count)."""
+    amax = amax_bf16(x_bits)
+    scale, scale_inv = scale_from_amax(amax, fmt)
+    q, sat = quantize_bf16(x_bits, fmt, scale)
+    return dict(amax=amax, scale=scale, scale_inv=scale_inv, q=q, sat_count=sat)
+
+
+def gemm_fwd(xq, fmt_x, wq, fmt_w, sx_inv, sw_inv) -> np.ndarray:
+    xq, wq = _u8(xq, 2), _u8(wq, 2)
+    M, K = xq.shape
+    N, K2 = wq.shape
+    assert K == K2
+    y = np.empty((M, N), dtype=np.float64)
+    lib().oracle_gemm_fwd(xq.ctypes.data, K, fmt_x, wq.ctypes.data, K, fmt_w, float(sx_inv), float(sw_inv),
+                          M, N, K, y.ctypes.data, N)
+    return y
+
+
+def gemm_dgrad(dyq, fmt_dy, wq, fmt_w, sdy_inv, sw_inv) -> np.ndarray:
+    dyq, wq = _u8(dyq, 2), _u8(wq, 2)
+    M, N = dyq.shape
+    N2, K = wq.shape
+    assert N == N2
+    dx = np.empty((M, K), dtype=np.float64)
+    lib().oracle_gemm_dgrad(dyq.ctypes.data, N, fmt_dy, wq.ctypes.data, K, fmt_w, float(sdy_inv), float(sw_inv),
+                            M, N, K, dx.ctypes.data, K)
+    return dx
+
+
+def gemm_wgrad(xq, fmt_x, dyq, fmt_dy, sx_inv, sdy_inv) -> np.ndarray:
+    xq, dyq = _u8(xq, 2), _u8(dyq, 2)
+    M, K = xq.shape
+    M2, N = dyq.shape
+    assert M == M2
+    dw = np.empty((N, K), dtype=np.float64)
+    lib().oracle_gemm_wgrad(xq.ctypes.data, K, fmt_x, dyq.ctypes.data, N, fmt_dy, float(sx_inv), float(sdy_inv),
+                            M, N, K, dw.ctypes.data, K)
+    return dw
+
+
+def _pts(rows, cols):
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    assert rows.shape == cols.shape and rows.ndim == 1
+    return rows, cols
+
+
+def gemm_fwd_at(xq, fmt_x, wq, fmt_w, sx_inv, sw_inv, rows, cols) -> np.ndarray:
+    xq, wq = _u8(xq, 2), _u8(wq, 2)
+    rows, cols = _pts(rows, cols)
+    out = np.empty(rows.size, dtype=np.float64)
+    lib().oracle_gemm_fwd_at(xq.ctypes.data, xq.shape[1], fmt_x, wq.ctypes.data, wq.shape[1], fmt_w,
+                             float(sx_inv), float(sw_inv), xq.shape[1], rows.ctypes.data, cols.ctypes.data,
+                             rows.size, out.ctypes.data)
+    return out
+
+
+def gemm_dgrad_at(dyq, fmt_dy, wq, fmt_w, sdy_inv, sw_inv, rows, cols) -> np.ndarray:
+    dyq, wq = _u8(dyq, 2), _u8(wq, 2)
+    rows, cols = _pts(rows, cols)
+    out = np.empty(rows.size, dtype=np.float64)
+    lib().oracle_gemm_dgrad_at(dyq.ctypes.data, dyq.shape[1], fmt_dy, wq.ctypes.data, wq.shape[1], fmt_w,
+                               float(sdy_inv), float(sw_inv), dyq.shape[1], rows.ctypes.data, cols.ctypes.data,
+                               rows.size, out.ctypes.data)
+    return out
+
+
+def gemm_wgrad_at(xq, fmt_x, dyq, fmt_dy, sx_inv, sdy_inv, rows, cols) -> np.ndarray:
+    xq, dyq = _u8(xq, 2), _u8(dyq, 2)
+    rows, cols = _pts(rows, cols)
+    out = np.empty(rows.size, dtype=np.float64)
+    lib().oracle_gemm_wgrad_at(xq.ctypes.data, xq.shape[1], fmt_x, dyq.ctypes.data, dyq.shape[1], fmt_dy,
+                               float(sx_inv), float(sdy_inv), xq.shape[0], rows.ctypes.data, cols.ctypes.data,
+                               rows.size, out.ctypes.data)
+    return out
+
+
+def tweo_loss_block(a_bits, tau, eps, p) -> float:
+    a = _u16(a_bits)
+    return float(lib().oracle_tweo_loss_block(a.ctypes.data, a.size, float(tau), float(eps), float(p)))
+
+
+def tweo_loss(blocks, tau, eps, p):
+    """Eq. 3 over a list of block outputs: returns (L_TWEO, per-block means)."""
+    per = [tweo_loss_block(a, tau, eps, p) for a in blocks]
+    total = 0.0
+    for v in per:
+        total += v
+    return total / len(per), per
+
+
+def tweo_grad_block(a_bits, tau, eps, p, c) -> np.ndarray:
+    a = _u16(a_bits)
+    g = np.empty(a.shape, dtype=np.float64)
+    lib().oracle_tweo_grad_block(a.ctypes.data, a.size, float(tau), float(eps), float(p), float(c), g.ctypes.data)
+    return g
+
+
+def absmax_qmax(bits: int) -> int:
+    return int(lib().oracle_absmax_qmax(bits))
+
+
+def absmax_scale(x, eps) -> float:
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    return float(lib().oracle_absmax_scale(x.ctypes.data, x.size, float(eps)))
+
+
+def absmax_quantize(x, bits: int, s: float) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    q = np.empty(x.shape, dtype=np.int32)
+    lib().oracle_absmax_quantize(x.ctypes.data, x.size, bits, float(s), q.ctypes.data)
+    return q
+
+
+def absmax_dequantize(xq, bits: int, s: float) -> np.ndarray:
+    xq = np.ascontiguousarray(xq, dtype=np.int32)
+    x = np.empty(xq.shape, dtype=np.float64)
+    lib().oracle_absmax_dequantize(xq.ctypes.data, xq.size, bits, float(s), x.ctypes.data)
+    return x
