@@ -1,0 +1,224 @@
+/*
+ * tweo.h -- C ABI of the B200 (sm_100a) library for FP8 per-tensor-scaled
+ * linear layers and the TWEO activation penalty.
+ *
+ * What the calls compute follows the TWEO paper (arXiv 2511.23225):
+ *   - Sec. 3.3, Eq. 2-3: the penalty  L_TWEO = (1/L) sum_l mean((|A^(l)|/(tau+eps))^p)
+ *     on every transformer block output A^(l), weighted by lambda(t);
+ *   - Sec. 4.2: every linear layer runs in FP8 with ONE scale per tensor,
+ *     E4M3 for activations and weights, E5M2 for gradients (the HYBRID recipe),
+ *     scales derived from the tensor's absolute maximum;
+ *   - Sec. 4.3, Eq. 4 and the "W8(T)A8(T)" discussion: inference with static
+ *     per-tensor scales for weights and activations.
+ *
+ * Conventions (all calls)
+ *   - Every function returns a tweo_status_t and never throws or exits.
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, valid until
+ *     the work enqueued by the call has finished.  Scalars the device produces
+ *     (amax, scale, scale_inv, loss) are DEVICE pointers too, so calls can be
+ *     chained on a stream without a host synchronisation.  Hyper-parameters are
+ *     passed by value.  `stream` is a cudaStream_t passed as void*.
+ *   - Calls only enqueue work on `stream`; they do not synchronise and do not
+ *     allocate device memory.  Scratch memory, where needed, is passed in as
+ *     (ws, ws_bytes); size it with tweo_workspace_bytes().  A workspace must be
+ *     zero-filled once before its first use (tweo_workspace_init); every call
+ *     leaves it ready for the next one.  Two calls that overlap on the GPU must
+ *     not share a workspace.
+ *   - Tensors are row-major.  bf16 tensors are passed as uint16_t bit patterns,
+ *     FP8 tensors as uint8_t codes (OCP FP8: E4M3 has no infinity, NaN = 0x7F /
+ *     0xFF, max finite 448; E5M2 is IEEE-like, max finite 57344).
+ *   - Leading dimensions (ld*) are in ELEMENTS.  All tensor bases must be
+ *     16-byte aligned and every row must start 16-byte aligned (ld * element
+ *     size is a multiple of 16), otherwise TWEO_ERR_ALIGNMENT.
+ *   - Weights are stored one row per output feature: W is [N rows, K columns],
+ *     K contiguous (the layout of a framework's Linear.weight).
+ *   - Device-side waits are bounded; if one expires the kernel records it and
+ *     returns, and tweo_read_device_status() reports TWEO_ERR_TIMEOUT.
+ */
+#ifndef TWEO_H_
+#define TWEO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Exported symbols (the library is built with hidden default visibility). */
+#if defined(__GNUC__)
+#define TWEO_API __attribute__((visibility("default")))
+#else
+#define TWEO_API
+#endif
+
+typedef int32_t tweo_status_t;
+enum {
+  TWEO_OK = 0,
+  TWEO_ERR_INVALID_ARG = 1,        /* NULL where a pointer is required, negative size, bad enum */
+  TWEO_ERR_UNSUPPORTED_SHAPE = 2,  /* a dimension the kernels cannot tile (see each call)         */
+  TWEO_ERR_ALIGNMENT = 3,          /* base pointer or row pitch not 16-byte aligned               */
+  TWEO_ERR_WORKSPACE_TOO_SMALL = 4,
+  TWEO_ERR_CUDA = 5,               /* a CUDA runtime/driver call failed; see tweo_last_cuda_error */
+  TWEO_ERR_TIMEOUT = 6             /* a bounded device-side wait expired                          */
+};
+
+typedef enum { TWEO_E4M3 = 0, TWEO_E5M2 = 1 } tweo_fp8_t;
+typedef enum { TWEO_SCALE_CURRENT = 0, TWEO_SCALE_GIVEN = 1 } tweo_scale_mode_t;
+typedef enum { TWEO_BF16 = 0, TWEO_F32 = 1, TWEO_FP8_E4M3 = 2 } tweo_dtype_t;
+typedef enum {
+  TWEO_OP_QUANTIZE = 0,
+  TWEO_OP_LINEAR_FWD = 1,
+  TWEO_OP_LINEAR_DGRAD = 2,
+  TWEO_OP_LINEAR_WGRAD = 3,
+  TWEO_OP_LOSS = 4,
+  TWEO_OP_W8A8 = 5
+} tweo_op_t;
+
+/* Upper bound on the number of block outputs one tweo_loss_fwd_bwd call takes. */
+#define TWEO_MAX_BLOCKS 128
+
+/*
+ * Optional fused outputs of a GEMM epilogue (Sec. 4.2: with delayed scaling the
+ * next layer's scale is known before the GEMM runs, so the cast of the output
+ * can ride on the epilogue instead of costing two more passes over it).
+ * All three act on the bf16-ROUNDED output values, so that the fused result is
+ * bit-identical to running tweo_quantize_per_tensor(GIVEN) on the stored output.
+ *   out_amax : device float*, receives max |y| over the whole output, or NULL.
+ *   out_q    : device uint8*, receives sat_rne_fp8(fl32(y * *q_scale)), or NULL;
+ *              row pitch ldq elements (multiple of 16), format q_fmt.
+ *   q_scale  : device const float*, required when out_q != NULL.
+ */
+typedef struct tweo_epilogue_t {
+  float* out_amax;
+  uint8_t* out_q;
+  int64_t ldq;
+  int32_t q_fmt; /* tweo_fp8_t */
+  const float* q_scale;
+} tweo_epilogue_t;
+
+/*
+ * tweo_quantize_per_tensor -- amax, scale and FP8 cast of one bf16 tensor
+ * (Sec. 4.2: one scaling factor for the entire tensor; E4M3 range +-448).
+ *   x [n] bf16 in.  q [n] uint8 out (same element order).  n >= 0; n == 0 yields
+ *   amax 0, scale 1 (CURRENT) and writes nothing to q.
+ *   mode CURRENT: amax = max|x_i|; scale = fl32(FP8MAX/amax) (1 if amax is 0 or
+ *     not finite; clamped to FLT_MAX on overflow); *scale, *scale_inv, *amax are
+ *     written; q_i = sat_rne_fp8(fl32(x_i * scale)).
+ *   mode GIVEN: *scale is read (delayed or static scaling), one pass; *amax of x
+ *     is still written (it feeds the next step's scale); *scale_inv is written.
+ *   Rounding: one binary32 multiply, then round-to-nearest-even to FP8 with
+ *     saturation to +-FP8MAX; NaN -> 0x7F (no sign).  amax skips NaN.
+ *   sat_count: device uint32*, or NULL; receives the number of elements with
+ *     |fl32(x_i * scale)| > FP8MAX.
+ *   No workspace is needed (ws may be NULL).
+ */
+TWEO_API tweo_status_t tweo_quantize_per_tensor(const uint16_t* x, int64_t n, int32_t fmt, int32_t mode,
+                                       float* scale, float* scale_inv, float* amax, uint8_t* q,
+                                       uint32_t* sat_count, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * tweo_fp8_linear_fwd -- forward GEMM of an FP8 linear layer (Sec. 4.2):
+ *   Y[M,N] = (Xq[M,K] . Wq[N,K]^T) * (*sx_inv) * (*sw_inv), fp32 accumulation on
+ *   the tensor cores, result rounded once to bf16.
+ *   xq [M,K] codes (fmt_x), wq [N,K] codes (fmt_w), y [M,N] bf16.
+ *   Shapes: M >= 1 (ragged M is zero-filled by the loader); N % 16 == 0,
+ *   K % 16 == 0.  epi may be NULL.
+ */
+TWEO_API tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const uint8_t* wq, int64_t ldw,
+                                  const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy,
+                                  int64_t M, int64_t N, int64_t K, int32_t fmt_x, int32_t fmt_w,
+                                  const tweo_epilogue_t* epi, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * tweo_fp8_linear_bwd_dgrad -- data gradient (Sec. 4.2, gradients in E5M2):
+ *   dX[M,K] = (dYq[M,N] . Wq[N,K]) * (*sdy_inv) * (*sw_inv) -> bf16; the
+ *   contraction runs over N.  wq is the same buffer the forward call used.
+ *   Shapes: N % 16 == 0, K % 16 == 0.  epi may be NULL.
+ */
+TWEO_API tweo_status_t tweo_fp8_linear_bwd_dgrad(const uint8_t* dyq, int64_t lddy, int32_t fmt_dy,
+                                        const uint8_t* wq, int64_t ldw, int32_t fmt_w,
+                                        const float* sdy_inv, const float* sw_inv, uint16_t* dx,
+                                        int64_t lddx, int64_t M, int64_t N, int64_t K,
+                                        const tweo_epilogue_t* epi, void* ws, size_t ws_bytes,
+                                        void* stream);
+
+/*
+ * tweo_fp8_linear_bwd_wgrad -- weight gradient (Sec. 4.2):
+ *   dW[N,K] = (dYq[M,N]^T . Xq[M,K]) * (*sx_inv) * (*sdy_inv); the contraction
+ *   runs over the tokens M.  dw has the layout of W.  dw_dtype TWEO_BF16
+ *   (uint16_t*) or TWEO_F32 (float*); accumulate != 0 adds into dw instead of
+ *   overwriting it (F32 only).  Shapes: N % 16 == 0, K % 16 == 0, any M >= 1.
+ */
+TWEO_API tweo_status_t tweo_fp8_linear_bwd_wgrad(const uint8_t* xq, int64_t ldx, int32_t fmt_x,
+                                        const uint8_t* dyq, int64_t lddy, int32_t fmt_dy,
+                                        const float* sx_inv, const float* sdy_inv, void* dw,
+                                        int64_t lddw, int32_t dw_dtype, int32_t accumulate,
+                                        int64_t M, int64_t N, int64_t K, void* ws, size_t ws_bytes,
+                                        void* stream);
+
+/*
+ * tweo_loss_fwd_bwd -- TWEO penalty and its gradient in one pass (Eq. 3, and
+ * the derivative of Eq. 2's lambda(t) * L_TWEO term):
+ *   loss_l = (1/n) sum_i (|a_i| / (tau+eps))^p,          l = 0..L-1
+ *   *loss  = (1/L) sum_l loss_l                           (= L_TWEO)
+ *   g_i    = grad_coeff * p * sign(a_i) |a_i|^(p-1) / (n (tau+eps)^p),  g = 0 at a = 0
+ *   a: HOST array of L device pointers, each a bf16 tensor of n_per_tensor
+ *      elements (a block output [batch, seq, hidden] flattened; the mean runs
+ *      over all of them).  1 <= L <= TWEO_MAX_BLOCKS.
+ *   grad_coeff folds lambda(t), the 1/L of Eq. 3 and any upstream gradient.
+ *   loss: device float* out.  loss_per_block: device float[L] out, or NULL.
+ *   grad: HOST array of L device pointers (bf16 or float according to
+ *      grad_dtype), or NULL for loss only.  grad[l] may alias a[l] only if
+ *      grad_dtype is bf16 (in-place).
+ *   p = 4 (the paper's setting) runs a fast path; other p > 1 a generic one.
+ *   Needs a workspace (TWEO_OP_LOSS); the sum is reduced in a fixed order, so
+ *   results are bit-reproducible run to run.
+ */
+TWEO_API tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, int64_t n_per_tensor, float tau,
+                                float eps, float p, float grad_coeff, float* loss,
+                                float* loss_per_block, void* const* grad, int32_t grad_dtype, void* ws,
+                                size_t ws_bytes, void* stream);
+
+/*
+ * tweo_w8a8_static_gemm -- inference linear with static per-tensor scales for
+ * both operands (Sec. 4.3: AbsMax static quantisation, W8(T)A8(T)), in the E4M3
+ * flavour: Y[M,N] = (Xq . Wq^T) * (1 / *sx) * (*sw_inv) -> bf16.
+ *   x: activations [M,K]; x_dtype TWEO_BF16 (cast inside with the static scale
+ *      *sx, saturating; needs a workspace for the codes) or TWEO_FP8_E4M3
+ *      (already cast by the caller with *sx).
+ *   sx: device const float*, the calibrated activation scale (FP8MAX / amax_cal).
+ *   wq [N,K] E4M3 codes, sw_inv device const float*.
+ *   Shapes: N % 16 == 0, K % 16 == 0, any M >= 1 (small M takes a
+ *   weight-streaming split-K path).
+ */
+TWEO_API tweo_status_t tweo_w8a8_static_gemm(const void* x, int32_t x_dtype, int64_t ldx, const float* sx,
+                                    const uint8_t* wq, int64_t ldw, const float* sw_inv, uint16_t* y,
+                                    int64_t ldy, int64_t M, int64_t N, int64_t K, void* ws,
+                                    size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------- helpers */
+
+/* Bytes of workspace `op` needs for the given problem (n for QUANTIZE / LOSS is
+ * passed in M, with N = number of tensors for LOSS; unused dims may be 0). */
+TWEO_API size_t tweo_workspace_bytes(int32_t op, int64_t M, int64_t N, int64_t K);
+
+/* Zero-fills a workspace (enqueued on stream); call once after allocating it. */
+TWEO_API tweo_status_t tweo_workspace_init(void* ws, size_t ws_bytes, void* stream);
+
+/* Synchronises `stream`, then returns TWEO_ERR_TIMEOUT if any kernel since the
+ * last call recorded an expired wait (and clears the record), TWEO_ERR_CUDA if
+ * the stream reports an error, else TWEO_OK. */
+TWEO_API tweo_status_t tweo_read_device_status(void* stream);
+
+TWEO_API const char* tweo_status_string(tweo_status_t s);
+TWEO_API const char* tweo_last_cuda_error(void); /* text of the last failing CUDA call in this thread */
+TWEO_API int32_t tweo_version(void);             /* major * 10000 + minor * 100 + patch */
+
+/* Number of kernel launches this library has enqueued since it was loaded. */
+TWEO_API uint64_t tweo_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TWEO_H_ */

@@ -104,12 +104,13 @@ double oracle_fp8_max(int fmt) { return fmt == ORACLE_E4M3 ? 448.0 : 57344.0; }
 static uint8_t fp8_max_code(int fmt) { return fmt == ORACLE_E4M3 ? 0x7E : 0x7B; }
 
 /* Encoder A (arithmetic).  Saturating round-to-nearest-even of a binary32
- * value: NaN -> sign|0x7F; |v| >= max finite (infinity included) -> sign|max
+ * value: NaN -> 0x7F (a NaN carries no sign: IEEE 754 leaves the sign of a NaN
+ * product unspecified, so none is propagated); |v| >= max finite (infinity included) -> sign|max
  * code; otherwise the nearest representable value, ties to the even code;
  * zero and values that round to zero keep their sign. */
 uint8_t oracle_fp8_encode(float v, int fmt) {
+  if (isnan(v)) return 0x7F;
   uint8_t sign = signbit(v) ? 0x80 : 0x00;
-  if (isnan(v)) return (uint8_t)(sign | 0x7F);
   double a = fabs((double)v);
   if (a >= oracle_fp8_max(fmt)) return (uint8_t)(sign | fp8_max_code(fmt));
   if (a == 0.0) return sign;
@@ -134,8 +135,8 @@ uint8_t oracle_fp8_encode(float v, int fmt) {
  * every non-negative finite code, keep the closest decoded value, and on an
  * exact tie keep the code whose last bit is 0.  Used only to cross-check A. */
 uint8_t oracle_fp8_encode_search(float v, int fmt) {
+  if (isnan(v)) return 0x7F;
   uint8_t sign = signbit(v) ? 0x80 : 0x00;
-  if (isnan(v)) return (uint8_t)(sign | 0x7F);
   double a = fabs((double)v);
   if (a >= oracle_fp8_max(fmt)) return (uint8_t)(sign | fp8_max_code(fmt));
   int best = 0;

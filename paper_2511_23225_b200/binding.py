@@ -1,0 +1,292 @@
+"""Thin ctypes binding over the C ABI in ``include/tweo.h``.
+
+Argument marshalling only: every function takes torch CUDA tensors (used for
+device memory and streams, nothing else), checks dtypes, and forwards raw
+device pointers and the current CUDA stream to the library entry point of the
+same name.  There is no CPU path: a missing library or a non-CUDA tensor raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+E4M3, E5M2 = 0, 1
+SCALE_CURRENT, SCALE_GIVEN = 0, 1
+BF16, F32, FP8_E4M3 = 0, 1, 2
+OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_DGRAD, OP_LINEAR_WGRAD, OP_LOSS, OP_W8A8 = range(6)
+MAX_BLOCKS = 128
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtweo_b200.so")
+
+EXPORTS = [
+    "tweo_quantize_per_tensor", "tweo_fp8_linear_fwd", "tweo_fp8_linear_bwd_dgrad",
+    "tweo_fp8_linear_bwd_wgrad", "tweo_loss_fwd_bwd", "tweo_w8a8_static_gemm",
+    "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
+    "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
+]
+
+
+class TweoError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        L = lib()
+        msg = L.tweo_status_string(status).decode()
+        if status == 5:
+            msg += ": " + L.tweo_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} (status {status})")
+        self.status = status
+
+
+class _Epilogue(C.Structure):
+    _fields_ = [("out_amax", C.c_void_p), ("out_q", C.c_void_p), ("ldq", C.c_int64),
+                ("q_fmt", C.c_int32), ("q_scale", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2511_23225_b200.build` "
+                "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
+        L.tweo_quantize_per_tensor.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.tweo_fp8_linear_fwd.argtypes = [vp, i64, vp, i64, vp, vp, vp, i64, i64, i64, i64, i32, i32,
+                                          C.POINTER(_Epilogue), vp, sz, vp]
+        L.tweo_fp8_linear_bwd_dgrad.argtypes = [vp, i64, i32, vp, i64, i32, vp, vp, vp, i64, i64, i64, i64,
+                                                C.POINTER(_Epilogue), vp, sz, vp]
+        L.tweo_fp8_linear_bwd_wgrad.argtypes = [vp, i64, i32, vp, i64, i32, vp, vp, vp, i64, i32, i32,
+                                                i64, i64, i64, vp, sz, vp]
+        L.tweo_loss_fwd_bwd.argtypes = [C.POINTER(vp), i32, i64, f32, f32, f32, f32, vp, vp, C.POINTER(vp), i32,
+                                        vp, sz, vp]
+        L.tweo_w8a8_static_gemm.argtypes = [vp, i32, i64, vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, sz, vp]
+        L.tweo_workspace_bytes.argtypes = [i32, i64, i64, i64]
+        L.tweo_workspace_bytes.restype = sz
+        L.tweo_workspace_init.argtypes = [vp, sz, vp]
+        L.tweo_read_device_status.argtypes = [vp]
+        L.tweo_status_string.argtypes = [i32]
+        L.tweo_status_string.restype = C.c_char_p
+        L.tweo_last_cuda_error.restype = C.c_char_p
+        L.tweo_version.restype = i32
+        L.tweo_launch_count.restype = C.c_uint64
+        for name in EXPORTS:
+            f = getattr(L, name)
+            if f.restype is C.c_int:  # default -> status
+                f.restype = i32
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise TweoError(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype=None, name="tensor") -> int:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor (no CPU fallback exists)")
+    if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):
+        raise TypeError(f"{name} has dtype {t.dtype}, expected {dtype}")
+    return t.data_ptr()
+
+
+def _rows(t: torch.Tensor, name: str):
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError(f"{name} must be 2-D with contiguous rows")
+    return t.stride(0)
+
+
+U8 = (torch.uint8, torch.float8_e4m3fn, torch.float8_e5m2)
+
+
+def launch_count() -> int:
+    return int(lib().tweo_launch_count())
+
+
+def version() -> int:
+    return int(lib().tweo_version())
+
+
+def workspace_bytes(op: int, M: int = 0, N: int = 0, K: int = 0) -> int:
+    return int(lib().tweo_workspace_bytes(op, M, N, K))
+
+
+def new_workspace(op: int, M: int = 0, N: int = 0, K: int = 0, device="cuda") -> torch.Tensor:
+    """Allocates (torch) and zero-fills (library call) a workspace for `op`."""
+    n = max(256, workspace_bytes(op, M, N, K))
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    _check(lib().tweo_workspace_init(ws.data_ptr(), n, _stream()), "tweo_workspace_init")
+    return ws
+
+
+def read_device_status() -> int:
+    return int(lib().tweo_read_device_status(_stream()))
+
+
+@dataclass
+class Quantized:
+    q: torch.Tensor          # uint8 codes, same shape as the input
+    scale: torch.Tensor      # float32 [1]
+    scale_inv: torch.Tensor  # float32 [1]
+    amax: torch.Tensor       # float32 [1]
+    sat_count: torch.Tensor | None
+    fmt: int
+
+
+def quantize_per_tensor(x: torch.Tensor, fmt: int = E4M3, mode: int = SCALE_CURRENT,
+                        scale: torch.Tensor | None = None, count_saturated: bool = False,
+                        out: Quantized | None = None) -> Quantized:
+    """tweo_quantize_per_tensor: amax -> scale -> FP8 codes of a bf16 tensor."""
+    xp = _dev(x, torch.bfloat16, "x")
+    if not x.is_contiguous():
+        raise ValueError("x must be contiguous")
+    if out is None:
+        q = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+        scalars = torch.empty(4, dtype=torch.float32, device=x.device)
+        if mode == SCALE_GIVEN:
+            if scale is None:
+                raise ValueError("GIVEN mode needs a scale tensor")
+            s = scale
+        else:
+            s = scalars[0:1]
+        out = Quantized(q, s, scalars[1:2], scalars[2:3],
+                        torch.empty(1, dtype=torch.int32, device=x.device) if count_saturated else None, fmt)
+    sat = out.sat_count.data_ptr() if out.sat_count is not None else None
+    _check(lib().tweo_quantize_per_tensor(xp, x.numel(), fmt, mode, _dev(out.scale, torch.float32, "scale"),
+                                          out.scale_inv.data_ptr(), out.amax.data_ptr(), out.q.data_ptr(), sat,
+                                          None, 0, _stream()), "tweo_quantize_per_tensor")
+    return out
+
+
+def _epilogue(amax, q, q_fmt, q_scale):
+    if amax is None and q is None:
+        return None
+    e = _Epilogue()
+    e.out_amax = _dev(amax, torch.float32, "out_amax") if amax is not None else None
+    if q is not None:
+        e.out_q = _dev(q, U8, "out_q")
+        e.ldq = _rows(q, "out_q")
+        e.q_fmt = q_fmt
+        e.q_scale = _dev(q_scale, torch.float32, "q_scale")
+    return C.byref(e)
+
+
+def fp8_linear_fwd(xq, wq, sx_inv, sw_inv, fmt_x=E4M3, fmt_w=E4M3, y=None, out_amax=None, out_q=None,
+                   q_fmt=E4M3, q_scale=None) -> torch.Tensor:
+    """tweo_fp8_linear_fwd: Y[M,N] = Xq[M,K] . Wq[N,K]^T * sx_inv * sw_inv -> bf16."""
+    M, K = xq.shape
+    N, K2 = wq.shape
+    if K != K2:
+        raise ValueError("inner dimensions differ")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=xq.device)
+    _check(lib().tweo_fp8_linear_fwd(_dev(xq, U8, "xq"), _rows(xq, "xq"), _dev(wq, U8, "wq"), _rows(wq, "wq"),
+                                     _dev(sx_inv, torch.float32), _dev(sw_inv, torch.float32),
+                                     _dev(y, torch.bfloat16, "y"), _rows(y, "y"), M, N, K, fmt_x, fmt_w,
+                                     _epilogue(out_amax, out_q, q_fmt, q_scale), None, 0, _stream()),
+           "tweo_fp8_linear_fwd")
+    return y
+
+
+def fp8_linear_bwd_dgrad(dyq, wq, sdy_inv, sw_inv, fmt_dy=E5M2, fmt_w=E4M3, dx=None, out_amax=None, out_q=None,
+                         q_fmt=E5M2, q_scale=None) -> torch.Tensor:
+    """tweo_fp8_linear_bwd_dgrad: dX[M,K] = dYq[M,N] . Wq[N,K] * sdy_inv * sw_inv -> bf16."""
+    M, N = dyq.shape
+    N2, K = wq.shape
+    if N != N2:
+        raise ValueError("inner dimensions differ")
+    if dx is None:
+        dx = torch.empty((M, K), dtype=torch.bfloat16, device=dyq.device)
+    _check(lib().tweo_fp8_linear_bwd_dgrad(_dev(dyq, U8, "dyq"), _rows(dyq, "dyq"), fmt_dy, _dev(wq, U8, "wq"),
+                                           _rows(wq, "wq"), fmt_w, _dev(sdy_inv, torch.float32),
+                                           _dev(sw_inv, torch.float32), _dev(dx, torch.bfloat16, "dx"),
+                                           _rows(dx, "dx"), M, N, K, _epilogue(out_amax, out_q, q_fmt, q_scale),
+                                           None, 0, _stream()), "tweo_fp8_linear_bwd_dgrad")
+    return dx
+
+
+def fp8_linear_bwd_wgrad(xq, dyq, sx_inv, sdy_inv, fmt_x=E4M3, fmt_dy=E5M2, dw=None, dw_dtype=BF16,
+                         accumulate=False) -> torch.Tensor:
+    """tweo_fp8_linear_bwd_wgrad: dW[N,K] = dYq[M,N]^T . Xq[M,K] * sx_inv * sdy_inv."""
+    M, K = xq.shape
+    M2, N = dyq.shape
+    if M != M2:
+        raise ValueError("token dimensions differ")
+    tdt = torch.bfloat16 if dw_dtype == BF16 else torch.float32
+    if dw is None:
+        if accumulate:
+            raise ValueError("accumulate needs an existing dw")
+        dw = torch.empty((N, K), dtype=tdt, device=xq.device)
+    _check(lib().tweo_fp8_linear_bwd_wgrad(_dev(xq, U8, "xq"), _rows(xq, "xq"), fmt_x, _dev(dyq, U8, "dyq"),
+                                           _rows(dyq, "dyq"), fmt_dy, _dev(sx_inv, torch.float32),
+                                           _dev(sdy_inv, torch.float32), _dev(dw, tdt, "dw"), _rows(dw, "dw"),
+                                           dw_dtype, 1 if accumulate else 0, M, N, K, None, 0, _stream()),
+           "tweo_fp8_linear_bwd_wgrad")
+    return dw
+
+
+def loss_fwd_bwd(blocks, tau=3.0, eps=1e-6, p=4.0, grad_coeff=1.0, want_grad=True, grad_dtype=BF16,
+                 grads=None, ws=None, per_block=True):
+    """tweo_loss_fwd_bwd over a list of bf16 block outputs of equal size.
+    Returns (loss [1] float32, per-block [L] float32 or None, list of grads or None)."""
+    Lb = len(blocks)
+    n = blocks[0].numel()
+    dev = blocks[0].device
+    a_arr = (C.c_void_p * Lb)()
+    for i, b in enumerate(blocks):
+        if b.numel() != n or not b.is_contiguous():
+            raise ValueError("block outputs must be contiguous and of equal size")
+        a_arr[i] = _dev(b, torch.bfloat16, "block output")
+    g_arr = None
+    if want_grad:
+        gdt = torch.bfloat16 if grad_dtype == BF16 else torch.float32
+        if grads is None:
+            grads = [torch.empty(b.shape, dtype=gdt, device=dev) for b in blocks]
+        g_arr = (C.c_void_p * Lb)()
+        for i, g in enumerate(grads):
+            g_arr[i] = _dev(g, gdt, "grad")
+    else:
+        grads = None
+    if ws is None:
+        ws = new_workspace(OP_LOSS, n, Lb)
+    loss = torch.empty(1, dtype=torch.float32, device=dev)
+    pb = torch.empty(Lb, dtype=torch.float32, device=dev) if per_block else None
+    _check(lib().tweo_loss_fwd_bwd(a_arr, Lb, n, tau, eps, p, grad_coeff, loss.data_ptr(),
+                                   pb.data_ptr() if pb is not None else None, g_arr, grad_dtype, ws.data_ptr(),
+                                   ws.numel(), _stream()), "tweo_loss_fwd_bwd")
+    return loss, pb, grads
+
+
+def w8a8_static_gemm(x, sx, wq, sw_inv, y=None, ws=None) -> torch.Tensor:
+    """tweo_w8a8_static_gemm: static per-tensor W8A8 linear, bf16 or E4M3-coded activations."""
+    M, K = x.shape
+    N, K2 = wq.shape
+    if K != K2:
+        raise ValueError("inner dimensions differ")
+    if x.dtype == torch.bfloat16:
+        xdt = BF16
+    elif x.dtype in U8:
+        xdt = FP8_E4M3
+    else:
+        raise TypeError("x must be bf16 or uint8 E4M3 codes")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    if ws is None:
+        ws = new_workspace(OP_W8A8, M, N, K)
+    _check(lib().tweo_w8a8_static_gemm(_dev(x, None, "x"), xdt, _rows(x, "x"), _dev(sx, torch.float32, "sx"),
+                                       _dev(wq, U8, "wq"), _rows(wq, "wq"), _dev(sw_inv, torch.float32),
+                                       _dev(y, torch.bfloat16, "y"), _rows(y, "y"), M, N, K, ws.data_ptr(),
+                                       ws.numel(), _stream()), "tweo_w8a8_static_gemm")
+    return y

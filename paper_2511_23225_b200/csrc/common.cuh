@@ -1,0 +1,90 @@
+// Shared host/device helpers of the CUDA library (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tweo.h"
+
+namespace tweo_detail {
+
+// Number of SMs the persistent kernels size their grids for (queried once per device).
+int sm_count();
+
+// Book-keeping shared by all translation units.
+void count_launch(int n = 1);
+tweo_status_t cuda_fail(cudaError_t e, const char* what);  // records text, returns TWEO_ERR_CUDA
+tweo_status_t check_launch(const char* what);              // cudaGetLastError after a launch
+
+// Device status word (bounded waits that expired); lives with the GEMM kernels.
+tweo_status_t read_and_clear_device_status(cudaStream_t stream);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace tweo_detail
+
+#define TWEO_CUDA_TRY(expr)                                              \
+  do {                                                                   \
+    cudaError_t _e = (expr);                                             \
+    if (_e != cudaSuccess) return tweo_detail::cuda_fail(_e, #expr);     \
+  } while (0)
+
+#ifdef __CUDACC__
+namespace tweo_detail {
+
+constexpr float kE4M3Max = 448.0f;
+constexpr float kE5M2Max = 57344.0f;
+
+__device__ __forceinline__ float fp8_max(int fmt) { return fmt == TWEO_E4M3 ? kE4M3Max : kE5M2Max; }
+
+// Two binary32 values -> two FP8 codes (round-to-nearest-even, saturating to the
+// largest finite value); `lo` lands in bits 0-7, `hi` in bits 8-15.
+template <int FMT>
+__device__ __forceinline__ uint32_t cvt_fp8x2(float lo, float hi) {
+  uint16_t r;
+  if (FMT == TWEO_E4M3)
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  else
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  uint32_t out = r;
+  // NaN in -> NaN code 0x7F (no sign: a NaN product's sign is unspecified), whatever the converter picks.
+  if (lo != lo) out = (out & 0xFF00u) | 0x7Fu;
+  if (hi != hi) out = (out & 0x00FFu) | 0x7F00u;
+  return out;
+}
+
+__device__ __forceinline__ float bf16lo_to_f32(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi_to_f32(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// binary32 -> bf16 bits, round-to-nearest-even.
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
+  uint16_t r;
+  asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(f));
+  return r;
+}
+// packs bf16(lo) | bf16(hi) << 16
+__device__ __forceinline__ uint32_t f32x2_to_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// per-tensor scale from amax: fl32(FP8MAX / amax); 1 for amax == 0 or non-finite;
+// clamped to FLT_MAX when the quotient overflows.
+__device__ __forceinline__ float scale_from_amax(float amax, int fmt) {
+  float s = 1.0f;
+  if (amax > 0.0f && amax < __int_as_float(0x7F800000)) {
+    s = __fdiv_rn(fp8_max(fmt), amax);
+    if (s > 3.402823466e38f) s = 3.402823466e38f;
+  }
+  return s;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  return v;
+}
+
+}  // namespace tweo_detail
+#endif  // __CUDACC__

@@ -1,0 +1,619 @@
+// FP8 x FP8 -> fp32 GEMMs of the linear layer (forward, data gradient, weight gradient)
+// on the sm_100a tensor cores: tcgen05.mma kind::f8f6f4, operands staged in shared memory
+// by TMA (128-byte swizzle), accumulators in tensor memory, epilogue through tcgen05.ld.
+//
+// One kernel serves all three products.  It computes D[Md,Nd] = A . B over a contraction
+// of length Kc, where each operand is either
+//   "K-major"  : stored [rows = Md or Nd, Kc] with the contraction contiguous, or
+//   "MN-major" : stored [Kc, rows] with the output dimension contiguous.
+//     forward  Y  = Xq  . Wq^T : A = Xq  [M,K]  K-major , B = Wq [N,K]  K-major , Kc = K
+//     dgrad    dX = dYq . Wq   : A = dYq [M,N]  K-major , B = Wq [N,K]  MN-major, Kc = N
+//     wgrad    dW = dYq^T . Xq : A = dYq [M,N]  MN-major, B = Xq [M,K]  MN-major, Kc = M
+//   so no operand is ever transposed in memory: the major-ness bits of the instruction
+//   descriptor and the shared-memory descriptors absorb the layout.
+//
+// CTA = 192 threads: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the
+// MMAs (one thread), warps 2-5 are the epilogue (each reads its own 32-lane quarter of
+// tensor memory).  The kernel is persistent (grid = #SMs, static tile striding) with a
+// ring of shared-memory stages and two accumulators in tensor memory, so the epilogue of
+// tile i overlaps the main loop of tile i+1.  Every mbarrier wait is bounded: on expiry
+// the CTA records TWEO_ERR_TIMEOUT in a device status word, drains and exits.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <mutex>
+
+#include "common.cuh"
+
+namespace {
+
+using namespace tweo_detail;
+
+constexpr int BM = 128;      // rows of D per tile = tcgen05 M (lanes of tensor memory)
+constexpr int BK = 128;      // contraction bytes per stage = one 128-byte swizzle span
+constexpr int UMMA_K = 32;   // contraction per instruction for 8-bit operands
+constexpr int kThreads = 192;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+
+__device__ unsigned int g_device_status = 0;
+
+struct GemmParams {
+  void* d;
+  int64_t ldd;
+  int32_t Md, Nd, Kc;
+  int32_t tiles_m, tiles_n, k_blocks;
+  const float* sa_inv;
+  const float* sb_inv;
+  int32_t out_f32;     // 0: bf16 out, 1: fp32 out
+  int32_t accumulate;  // fp32 out only
+  float* out_amax;
+  uint8_t* out_q;
+  int64_t ldq;
+  int32_t q_fmt;
+  const float* q_scale;
+  uint32_t idesc;
+};
+
+// ----------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait: false if the CTA is aborting or the limit expired (then it raises abort).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = globaltimer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 0x3FFu) == 0) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(&g_device_status, (unsigned int)TWEO_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] . B[smem]
+__device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// mbarrier arrives once all MMAs issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 consecutive 32-bit columns: thread i gets row (lane base + i), columns c..c+31
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Fields (bit positions):
+//   [0,14)  start address >> 4        [16,30) leading-dimension byte offset >> 4
+//   [32,46) stride byte offset >> 4   [46,48) descriptor version = 1 (sm_100)
+//   [61,64) swizzle mode, 2 = 128 B
+// K-major tile: rows of 128 contraction bytes, 8-row groups 1024 B apart (stride offset);
+//   the leading offset is unused for swizzled K-major layouts.
+// MN-major tile: rows are contraction indices holding 128 contiguous bytes of the output
+//   dimension; 8-row groups 1024 B apart (stride offset); further 128-wide slabs of the
+//   output dimension `slab_bytes` apart (leading offset).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)(1024u >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+// ----------------------------------------------------------------- epilogue helpers
+template <int FMT>
+__device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d) {
+  return cvt_fp8x2<FMT>(a, b) | (cvt_fp8x2<FMT>(c, d) << 16);
+}
+
+// ----------------------------------------------------------------- the kernel
+template <int BN, bool A_MN, bool B_MN, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                const GemmParams p) {
+  constexpr uint32_t A_BYTES = BM * BK;
+  constexpr uint32_t B_BYTES = BN * BK;
+  constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr uint32_t TMEM_COLS = 2 * BN >= 512 ? 512 : (2 * BN >= 256 ? 256 : (2 * BN >= 128 ? 128 : 64));
+  static_assert(BN % 16 == 0 && BN >= 16 && BN <= 256, "tcgen05 N for M = 128");
+  static_assert(!B_MN || BN % 128 == 0, "MN-major B tiles come in 128-wide slabs");
+
+  extern __shared__ uint8_t smem_dyn[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  // bars: [0,STAGES) full, [STAGES,2*STAGES) empty, then tmem_full[2], tmem_empty[2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 4);  // one arrival per epilogue warp
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int num_tiles = p.tiles_m * p.tiles_n;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        const int m0 = (tile % p.tiles_m) * BM;
+        const int n0 = (tile / p.tiles_m) * BN;
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t fb = full_bar(stage);
+          mbar_expect_tx(fb, STAGE_BYTES);
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+          const int k0 = kb * BK;
+          if (A_MN) tma_load_2d(sa, &tmap_a, m0, k0, fb);
+          else tma_load_2d(sa, &tmap_a, k0, m0, fb);
+          if (B_MN) {
+#pragma unroll
+            for (int j = 0; j < BN / 128; ++j) tma_load_2d(sb + j * (BK * 128), &tmap_b, n0 + j * 128, k0, fb);
+          } else {
+            tma_load_2d(sb, &tmap_b, k0, n0, fb);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      // Do not leave while copies may still be landing in this CTA's shared memory:
+      // wait (bounded) for the last fill of every stage.  On the normal path these
+      // phases completed long ago.
+      if (!ok) {
+        for (int s = 0; s < STAGES; ++s) {
+          const uint64_t t0 = globaltimer_ns();
+          while (!mbar_try_wait(full_bar(s), 0) && !mbar_try_wait(full_bar(s), 1)) {
+            if (globaltimer_ns() - t0 > 100000000ull) break;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // K-major: step 32 bytes inside the swizzle span; MN-major: step 32 rows of 128 B
+            const uint64_t adesc = make_smem_desc(sa + (A_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
+            const uint64_t bdesc = make_smem_desc(sb + (B_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
+            umma_f8(d_tmem, adesc, bdesc, p.idesc, (uint32_t)((kb | k) != 0));
+          }
+          umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(tfull_bar(acc));      // accumulator complete -> epilogue
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;  // tensor-memory lanes [32*quarter, 32*quarter+32) belong to this warp
+    const float alpha = __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
+    const float qs = p.out_q ? __ldg(p.q_scale) : 0.0f;
+    float run_amax = 0.0f;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+      const int m0 = (tile % p.tiles_m) * BM;
+      const int n0 = (tile / p.tiles_m) * BN;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+      const bool row_ok = row < p.Md;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        const int col0 = n0 + c * 32;
+        if (col0 >= p.Nd) break;  // uniform across the warp
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
+        tmem_ld_wait();
+        if (!row_ok) continue;
+        if (p.out_f32) {
+          float* drow = reinterpret_cast<float*>(p.d) + (int64_t)row * p.ldd + col0;
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            if (col0 + j < p.Nd) {
+              float4 v = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
+                                     __uint_as_float(r[j + 2]) * alpha, __uint_as_float(r[j + 3]) * alpha);
+              float4* dst = reinterpret_cast<float4*>(drow + j);
+              if (p.accumulate) {
+                float4 o = *dst;
+                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+              }
+              *dst = v;
+            }
+          }
+        } else {
+          uint16_t* drow = reinterpret_cast<uint16_t*>(p.d) + (int64_t)row * p.ldd + col0;
+          uint32_t packed[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            packed[j] = f32x2_to_bf16x2(__fmul_rn(__uint_as_float(r[2 * j]), alpha),
+                                        __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha));
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (col0 + 8 * j < p.Nd)
+              *reinterpret_cast<uint4*>(drow + 8 * j) =
+                  make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+          if (p.out_amax || p.out_q) {
+            // fused amax / cast act on the bf16-rounded values just stored
+            uint32_t q[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              float v[4] = {bf16lo_to_f32(packed[2 * j]), bf16hi_to_f32(packed[2 * j]),
+                            bf16lo_to_f32(packed[2 * j + 1]), bf16hi_to_f32(packed[2 * j + 1])};
+              if (col0 + 4 * j < p.Nd) {
+                run_amax = fmaxf(run_amax, fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))));
+              }
+              if (p.out_q) {
+                if (p.q_fmt == TWEO_E4M3)
+                  q[j] = quant4<TWEO_E4M3>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
+                                           __fmul_rn(v[3], qs));
+                else
+                  q[j] = quant4<TWEO_E5M2>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
+                                           __fmul_rn(v[3], qs));
+              }
+            }
+            if (p.out_q) {
+              uint8_t* qrow = p.out_q + (int64_t)row * p.ldq + col0;
+              if (col0 < p.Nd) *reinterpret_cast<uint4*>(qrow) = make_uint4(q[0], q[1], q[2], q[3]);
+              if (col0 + 16 < p.Nd) *reinterpret_cast<uint4*>(qrow + 16) = make_uint4(q[4], q[5], q[6], q[7]);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+    if (p.out_amax) {
+      run_amax = warp_max(run_amax);
+      if (lane == 0 && run_amax > 0.0f)
+        atomicMax(reinterpret_cast<unsigned int*>(p.out_amax), __float_as_uint(run_amax));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+__global__ void zero_float_kernel(float* p) { *p = 0.0f; }
+
+// ----------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// 2-D uint8 tensor [outer, inner] (inner contiguous, row pitch ld bytes), boxes of
+// {128 bytes, box_outer rows}, 128-byte swizzle, out-of-bounds reads return zero.
+bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld, int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)ld};
+  cuuint32_t box[2] = {128u, (cuuint32_t)box_outer};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+uint32_t make_idesc(int fmt_a, int fmt_b, bool a_mn, bool b_mn, int n) {
+  // [4,6) accumulator format (1 = fp32)   [7,10) A format   [10,13) B format (0 = E4M3, 1 = E5M2)
+  // [15] A major (1 = MN)   [16] B major   [17,23) N >> 3   [24,29) M >> 4
+  uint32_t d = 0;
+  d |= 1u << 4;
+  d |= (uint32_t)(fmt_a == TWEO_E5M2 ? 1 : 0) << 7;
+  d |= (uint32_t)(fmt_b == TWEO_E5M2 ? 1 : 0) << 10;
+  d |= (uint32_t)(a_mn ? 1 : 0) << 15;
+  d |= (uint32_t)(b_mn ? 1 : 0) << 16;
+  d |= (uint32_t)(n >> 3) << 17;
+  d |= (uint32_t)(BM >> 4) << 24;
+  return d;
+}
+
+template <int BN, bool A_MN, bool B_MN, int STAGES>
+tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p, cudaStream_t st) {
+  constexpr size_t smem = (size_t)STAGES * (BM * BK + BN * BK) + 1024 + 256;
+  auto kern = gemm_fp8_kernel<BN, A_MN, B_MN, STAGES>;
+  static bool attr_done = false;  // per instantiation
+  if (!attr_done) {
+    TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_done = true;
+  }
+  p.tiles_m = (p.Md + BM - 1) / BM;
+  p.tiles_n = (p.Nd + BN - 1) / BN;
+  p.k_blocks = (p.Kc + BK - 1) / BK;
+  const int tiles = p.tiles_m * p.tiles_n;
+  int grid = sm_count();
+  if (grid > tiles) grid = tiles;
+  kern<<<grid, kThreads, smem, st>>>(ma, mb, p);
+  count_launch();
+  return check_launch("gemm_fp8_kernel");
+}
+
+struct Operand {
+  const uint8_t* ptr;
+  int64_t ld;
+  int fmt;
+  bool mn_major;  // stored [Kc, rows] (true) or [rows, Kc] (false)
+};
+
+// D[Md,Nd] = A . B, see the header comment for how the three linear products map here.
+tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t Nd, int64_t Kc, GemmParams p,
+                       cudaStream_t st) {
+  if (Md < 1 || Nd < 1 || Kc < 1) return TWEO_ERR_INVALID_ARG;
+  if (Md > INT32_MAX || Nd > INT32_MAX || Kc > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(A.ptr) || !aligned16(B.ptr) || !aligned16(p.d) || (A.ld & 15) || (B.ld & 15))
+    return TWEO_ERR_ALIGNMENT;
+  if ((p.ldd * (p.out_f32 ? 4 : 2)) & 15) return TWEO_ERR_ALIGNMENT;
+  p.Md = (int32_t)Md;
+  p.Nd = (int32_t)Nd;
+  p.Kc = (int32_t)Kc;
+  const int BN = Nd > 128 ? 256 : 128;
+  p.idesc = make_idesc(A.fmt, B.fmt, A.mn_major, B.mn_major, BN);
+
+  CUtensorMap ma, mb;
+  bool ok;
+  if (A.mn_major) ok = make_map(&ma, A.ptr, Md, Kc, A.ld, BK);   // [Kc, Md]: box 128 (Md) x BK rows
+  else ok = make_map(&ma, A.ptr, Kc, Md, A.ld, BM);              // [Md, Kc]: box 128 (Kc) x BM rows
+  if (B.mn_major) ok = ok && make_map(&mb, B.ptr, Nd, Kc, B.ld, BK);
+  else ok = ok && make_map(&mb, B.ptr, Kc, Nd, B.ld, BN);
+  if (!ok) {
+    cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return TWEO_ERR_CUDA;
+  }
+  if (p.out_amax) {
+    zero_float_kernel<<<1, 1, 0, st>>>(p.out_amax);
+    count_launch();
+  }
+#define TWEO_DISPATCH(AMN, BMN)                                                        \
+  (BN == 256 ? launch_cfg<256, AMN, BMN, 4>(ma, mb, p, st) : launch_cfg<128, AMN, BMN, 6>(ma, mb, p, st))
+  if (!A.mn_major && !B.mn_major) return TWEO_DISPATCH(false, false);
+  if (!A.mn_major && B.mn_major) return TWEO_DISPATCH(false, true);
+  if (A.mn_major && B.mn_major) return TWEO_DISPATCH(true, true);
+  return TWEO_ERR_INVALID_ARG;
+#undef TWEO_DISPATCH
+}
+
+bool fmt_ok(int f) { return f == TWEO_E4M3 || f == TWEO_E5M2; }
+
+tweo_status_t fill_epilogue(GemmParams& p, const tweo_epilogue_t* epi) {
+  p.out_amax = nullptr;
+  p.out_q = nullptr;
+  p.ldq = 0;
+  p.q_fmt = TWEO_E4M3;
+  p.q_scale = nullptr;
+  if (!epi) return TWEO_OK;
+  p.out_amax = epi->out_amax;
+  if (epi->out_q) {
+    if (!epi->q_scale || !fmt_ok(epi->q_fmt)) return TWEO_ERR_INVALID_ARG;
+    if (!aligned16(epi->out_q) || (epi->ldq & 15)) return TWEO_ERR_ALIGNMENT;
+    p.out_q = epi->out_q;
+    p.ldq = epi->ldq;
+    p.q_fmt = epi->q_fmt;
+    p.q_scale = epi->q_scale;
+  }
+  return TWEO_OK;
+}
+
+}  // namespace
+
+namespace tweo_detail {
+
+tweo_status_t read_and_clear_device_status(cudaStream_t stream) {
+  TWEO_CUDA_TRY(cudaStreamSynchronize(stream));
+  unsigned int v = 0, zero = 0;
+  TWEO_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_device_status, sizeof v));
+  if (v != 0) TWEO_CUDA_TRY(cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero));
+  return v == 0 ? TWEO_OK : (tweo_status_t)v;
+}
+
+// Used by the static W8A8 entry point: forward product on already-cast activations.
+tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
+                             const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
+                             int64_t N, int64_t K, const tweo_epilogue_t* epi, cudaStream_t st) {
+  GemmParams p{};
+  p.d = y;
+  p.ldd = ldy;
+  p.sa_inv = sx_inv;
+  p.sb_inv = sw_inv;
+  tweo_status_t s = fill_epilogue(p, epi);
+  if (s != TWEO_OK) return s;
+  return run_gemm(Operand{xq, ldx, fmt_x, false}, Operand{wq, ldw, fmt_w, false}, M, N, K, p, st);
+}
+
+}  // namespace tweo_detail
+
+extern "C" {
+
+tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const uint8_t* wq, int64_t ldw,
+                                  const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
+                                  int64_t N, int64_t K, int32_t fmt_x, int32_t fmt_w, const tweo_epilogue_t* epi,
+                                  void* ws, size_t ws_bytes, void* stream) {
+  (void)ws;
+  (void)ws_bytes;
+  if (!xq || !wq || !sx_inv || !sw_inv || !y || !fmt_ok(fmt_x) || !fmt_ok(fmt_w)) return TWEO_ERR_INVALID_ARG;
+  if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
+  if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  return tweo_detail::gemm_fwd_codes(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, y, ldy, M, N, K, epi,
+                                     (cudaStream_t)stream);
+}
+
+tweo_status_t tweo_fp8_linear_bwd_dgrad(const uint8_t* dyq, int64_t lddy, int32_t fmt_dy, const uint8_t* wq,
+                                        int64_t ldw, int32_t fmt_w, const float* sdy_inv, const float* sw_inv,
+                                        uint16_t* dx, int64_t lddx, int64_t M, int64_t N, int64_t K,
+                                        const tweo_epilogue_t* epi, void* ws, size_t ws_bytes, void* stream) {
+  (void)ws;
+  (void)ws_bytes;
+  if (!dyq || !wq || !sdy_inv || !sw_inv || !dx || !fmt_ok(fmt_dy) || !fmt_ok(fmt_w)) return TWEO_ERR_INVALID_ARG;
+  if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
+  if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  GemmParams p{};
+  p.d = dx;
+  p.ldd = lddx;
+  p.sa_inv = sdy_inv;
+  p.sb_inv = sw_inv;
+  tweo_status_t s = fill_epilogue(p, epi);
+  if (s != TWEO_OK) return s;
+  // dX[M,K] = dYq[M,N] . Wq[N,K]: contraction over N; Wq is stored [N(contraction), K(out)] = MN-major
+  return run_gemm(Operand{dyq, lddy, fmt_dy, false}, Operand{wq, ldw, fmt_w, true}, M, K, N, p,
+                  (cudaStream_t)stream);
+}
+
+tweo_status_t tweo_fp8_linear_bwd_wgrad(const uint8_t* xq, int64_t ldx, int32_t fmt_x, const uint8_t* dyq,
+                                        int64_t lddy, int32_t fmt_dy, const float* sx_inv, const float* sdy_inv,
+                                        void* dw, int64_t lddw, int32_t dw_dtype, int32_t accumulate, int64_t M,
+                                        int64_t N, int64_t K, void* ws, size_t ws_bytes, void* stream) {
+  (void)ws;
+  (void)ws_bytes;
+  if (!xq || !dyq || !sx_inv || !sdy_inv || !dw || !fmt_ok(fmt_x) || !fmt_ok(fmt_dy)) return TWEO_ERR_INVALID_ARG;
+  if (dw_dtype != TWEO_BF16 && dw_dtype != TWEO_F32) return TWEO_ERR_INVALID_ARG;
+  if (accumulate && dw_dtype != TWEO_F32) return TWEO_ERR_INVALID_ARG;
+  if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
+  if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  GemmParams p{};
+  p.d = dw;
+  p.ldd = lddw;
+  p.sa_inv = sdy_inv;
+  p.sb_inv = sx_inv;
+  p.out_f32 = dw_dtype == TWEO_F32;
+  p.accumulate = accumulate ? 1 : 0;
+  fill_epilogue(p, nullptr);
+  // dW[N,K] = dYq[M,N]^T . Xq[M,K]: contraction over M; both operands stored [M(contraction), out]
+  return run_gemm(Operand{dyq, lddy, fmt_dy, true}, Operand{xq, ldx, fmt_x, true}, N, K, M, p,
+                  (cudaStream_t)stream);
+}
+
+}  // extern "C"

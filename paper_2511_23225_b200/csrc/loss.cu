@@ -1,0 +1,274 @@
+// TWEO penalty (Eq. 3) and its gradient in one streaming pass over each block output.
+//
+// HBM-bound: 2 B read + 2 B (bf16 grad) or 4 B (fp32 grad) written per element, ~8 flop.
+// One launch covers all L block outputs: grid = (blocks per tensor, L).  Each thread
+// streams 16-byte vectors (8 bf16) with four independent loads in flight, accumulates
+// sum |a|^p per vector in binary32 and across vectors in binary64, the CTA reduces with
+// shuffles and writes ONE partial sum to the workspace; the last CTA to finish (ticket
+// counter) adds the partials in a fixed order, so the result does not depend on
+// scheduling.  The ticket counter is left at zero for the next call.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace tweo_detail {
+
+constexpr int kLossThreads = 256;
+constexpr int kLossUnroll = 4;  // 16-byte vectors in flight per thread
+
+int loss_blocks_per_tensor(int64_t n, int L) {
+  if (L < 1) L = 1;
+  int64_t vec = n / 8;
+  int64_t want = (vec + (int64_t)kLossThreads * kLossUnroll - 1) / ((int64_t)kLossThreads * kLossUnroll);
+  int64_t cap = ((int64_t)sm_count() * 8 + L - 1) / L;  // about 8 resident CTAs per SM overall
+  if (cap < 1) cap = 1;
+  if (want > cap) want = cap;
+  if (want < 1) want = 1;
+  return (int)want;
+}
+
+}  // namespace tweo_detail
+
+namespace {
+
+using namespace tweo_detail;
+
+struct LossPtrs {
+  const uint16_t* a[TWEO_MAX_BLOCKS];
+  void* g[TWEO_MAX_BLOCKS];
+};
+
+struct LossArgs {
+  int64_t n;        // elements per tensor
+  int L;
+  float p;
+  float k_grad;     // fl32( grad_coeff * p / (n * (tau+eps)^p) ), rounded once on the host
+  double inv_norm;  // 1 / (n * (tau+eps)^p)
+  float* loss;
+  float* loss_per_block;  // or nullptr
+  double* partials;       // [L][gridDim.x]
+  unsigned int* ticket;
+};
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+// |a|^4 and k*a^3 for a pair of bf16 packed in one word.  a*a is exact in binary32
+// (8-bit significands), a^3 too (24 bits); a^4 and k*a^3 round once each.
+template <bool FAST, bool GRAD, bool GRAD_F32>
+__device__ __forceinline__ void process_vec(const uint4 v, float k, float p, float& vsum, uint4* gout_bf16,
+                                            float4* gout_f32) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  float g[8];
+  float t[8];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    float a0 = bf16lo_to_f32(w[j]), a1 = bf16hi_to_f32(w[j]);
+    if (FAST) {
+      float s0 = a0 * a0, s1 = a1 * a1;
+      t[2 * j] = s0 * s0;
+      t[2 * j + 1] = s1 * s1;
+      if (GRAD) {
+        g[2 * j] = __fmul_rn(k, s0 * a0);
+        g[2 * j + 1] = __fmul_rn(k, s1 * a1);
+      }
+    } else {
+      // generic exponent: binary64 pow keeps the 1e-5 budget for any p > 1
+      double m0 = fabs((double)a0), m1 = fabs((double)a1);
+      t[2 * j] = (float)pow(m0, (double)p);
+      t[2 * j + 1] = (float)pow(m1, (double)p);
+      if (GRAD) {
+        g[2 * j] = a0 == 0.0f ? 0.0f : (float)((double)k * copysign(pow(m0, (double)p - 1.0), (double)a0));
+        g[2 * j + 1] = a1 == 0.0f ? 0.0f : (float)((double)k * copysign(pow(m1, (double)p - 1.0), (double)a1));
+      }
+    }
+  }
+  vsum = ((t[0] + t[1]) + (t[2] + t[3])) + ((t[4] + t[5]) + (t[6] + t[7]));
+  if (GRAD) {
+    if (GRAD_F32) {
+      gout_f32[0] = make_float4(g[0], g[1], g[2], g[3]);
+      gout_f32[1] = make_float4(g[4], g[5], g[6], g[7]);
+    } else {
+      *gout_bf16 = make_uint4(f32x2_to_bf16x2(g[0], g[1]), f32x2_to_bf16x2(g[2], g[3]),
+                              f32x2_to_bf16x2(g[4], g[5]), f32x2_to_bf16x2(g[6], g[7]));
+    }
+  }
+}
+
+template <bool FAST, bool GRAD, bool GRAD_F32>
+__global__ void __launch_bounds__(kLossThreads)
+tweo_loss_kernel(const __grid_constant__ LossPtrs ptrs, const LossArgs args) {
+  const int l = blockIdx.y;
+  const uint16_t* __restrict__ a = ptrs.a[l];
+  void* gptr = ptrs.g[l];
+  const int64_t nvec = args.n >> 3;
+  const uint4* av = reinterpret_cast<const uint4*>(a);
+  const int64_t stride = (int64_t)gridDim.x * kLossThreads * kLossUnroll;
+  double acc = 0.0;
+
+  for (int64_t base = (int64_t)blockIdx.x * kLossThreads * kLossUnroll + threadIdx.x; base < nvec; base += stride) {
+    uint4 v[kLossUnroll];
+#pragma unroll
+    for (int u = 0; u < kLossUnroll; ++u) {
+      int64_t i = base + (int64_t)u * kLossThreads;
+      v[u] = i < nvec ? __ldcs(av + i) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < kLossUnroll; ++u) {
+      int64_t i = base + (int64_t)u * kLossThreads;
+      if (i < nvec) {
+        float vsum;
+        uint4 gb;
+        float4 gf[2];
+        process_vec<FAST, GRAD, GRAD_F32>(v[u], args.k_grad, args.p, vsum, &gb, gf);
+        acc += (double)vsum;
+        if (GRAD) {
+          if (GRAD_F32) {
+            float4* go = reinterpret_cast<float4*>(gptr) + 2 * i;
+            __stcs(go, gf[0]);
+            __stcs(go + 1, gf[1]);
+          } else {
+            __stcs(reinterpret_cast<uint4*>(gptr) + i, gb);
+          }
+        }
+      }
+    }
+  }
+  // ragged tail (n % 8 elements), handled by the first threads of CTA 0 of this tensor
+  if (blockIdx.x == 0) {
+    int64_t i = (nvec << 3) + threadIdx.x;
+    if (threadIdx.x < 8 && i < args.n) {
+      float af = __uint_as_float((uint32_t)a[i] << 16);
+      float t, g;
+      if (FAST) {
+        float s = af * af;
+        t = s * s;
+        g = __fmul_rn(args.k_grad, s * af);
+      } else {
+        double m = fabs((double)af);
+        t = (float)pow(m, (double)args.p);
+        g = af == 0.0f ? 0.0f : (float)((double)args.k_grad * copysign(pow(m, (double)args.p - 1.0), (double)af));
+      }
+      acc += (double)t;
+      if (GRAD) {
+        if (GRAD_F32) reinterpret_cast<float*>(gptr)[i] = g;
+        else reinterpret_cast<uint16_t*>(gptr)[i] = (uint16_t)f32_to_bf16_bits(g);
+      }
+    }
+  }
+
+  // CTA reduction in a fixed order
+  __shared__ double warp_part[kLossThreads / 32];
+  __shared__ bool is_last;
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+#pragma unroll
+    for (int w = 0; w < kLossThreads / 32; ++w) s += warp_part[w];
+    args.partials[(size_t)l * gridDim.x + blockIdx.x] = s;
+    __threadfence();
+    unsigned int total = gridDim.x * gridDim.y;
+    unsigned int t = atomicAdd(args.ticket, 1u);
+    is_last = (t == total - 1);
+  }
+  __syncthreads();
+  if (!is_last) return;
+
+  // Last CTA: per-tensor sums in index order of the partials (strided by thread, then a
+  // fixed tree), then the mean over the L tensors.
+  __threadfence();
+  __shared__ double block_loss[TWEO_MAX_BLOCKS];
+  for (int t = 0; t < args.L; ++t) {
+    double s = 0.0;
+    for (unsigned int b = threadIdx.x; b < gridDim.x; b += kLossThreads)
+      s += __ldcg(&args.partials[(size_t)t * gridDim.x + b]);
+    s = warp_sum(s);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double tot = 0.0;
+#pragma unroll
+      for (int w = 0; w < kLossThreads / 32; ++w) tot += warp_part[w];
+      block_loss[t] = tot * args.inv_norm;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double sum = 0.0;
+    for (int t = 0; t < args.L; ++t) {
+      sum += block_loss[t];
+      if (args.loss_per_block) args.loss_per_block[t] = (float)block_loss[t];
+    }
+    *args.loss = (float)(sum / (double)args.L);
+    *args.ticket = 0u;  // ready for the next call
+  }
+}
+
+template <bool FAST, bool GRAD, bool GRAD_F32>
+void launch(dim3 grid, cudaStream_t st, const LossPtrs& ptrs, const LossArgs& args) {
+  tweo_loss_kernel<FAST, GRAD, GRAD_F32><<<grid, kLossThreads, 0, st>>>(ptrs, args);
+}
+
+}  // namespace
+
+extern "C" tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, int64_t n_per_tensor, float tau,
+                                           float eps, float p, float grad_coeff, float* loss,
+                                           float* loss_per_block, void* const* grad, int32_t grad_dtype,
+                                           void* ws, size_t ws_bytes, void* stream) {
+  if (!a || !loss || L < 1 || L > TWEO_MAX_BLOCKS || n_per_tensor < 0) return TWEO_ERR_INVALID_ARG;
+  if (!(p > 1.0f) || !(tau + eps > 0.0f)) return TWEO_ERR_INVALID_ARG;
+  if (grad && grad_dtype != TWEO_BF16 && grad_dtype != TWEO_F32) return TWEO_ERR_INVALID_ARG;
+  const size_t need = tweo_workspace_bytes(TWEO_OP_LOSS, n_per_tensor, L, 0);
+  if (!ws || ws_bytes < need) return TWEO_ERR_WORKSPACE_TOO_SMALL;
+  if (!aligned16(ws)) return TWEO_ERR_ALIGNMENT;
+
+  LossPtrs ptrs;
+  for (int l = 0; l < L; ++l) {
+    if (!a[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
+    if (!aligned16(a[l])) return TWEO_ERR_ALIGNMENT;
+    ptrs.a[l] = a[l];
+    ptrs.g[l] = nullptr;
+    if (grad) {
+      if (!grad[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
+      if (!aligned16(grad[l])) return TWEO_ERR_ALIGNMENT;
+      if (grad_dtype == TWEO_F32 && grad[l] == (const void*)a[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
+      ptrs.g[l] = grad[l];
+    }
+  }
+
+  LossArgs args;
+  args.n = n_per_tensor;
+  args.L = L;
+  args.p = p;
+  const double d = (double)tau + (double)eps;
+  const double norm = (double)n_per_tensor * pow(d, (double)p);
+  args.inv_norm = n_per_tensor > 0 ? 1.0 / norm : 0.0;
+  args.k_grad = n_per_tensor > 0 ? (float)((double)grad_coeff * (double)p / norm) : 0.0f;
+  args.loss = loss;
+  args.loss_per_block = loss_per_block;
+  args.ticket = reinterpret_cast<unsigned int*>(ws);
+  args.partials = reinterpret_cast<double*>(reinterpret_cast<char*>(ws) + 256);
+
+  dim3 grid((unsigned)tweo_detail::loss_blocks_per_tensor(n_per_tensor, L), (unsigned)L);
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool fast = (p == 4.0f);
+  const bool has_grad = grad != nullptr;
+  const bool f32 = grad_dtype == TWEO_F32;
+  if (fast) {
+    if (!has_grad) launch<true, false, false>(grid, st, ptrs, args);
+    else if (f32) launch<true, true, true>(grid, st, ptrs, args);
+    else launch<true, true, false>(grid, st, ptrs, args);
+  } else {
+    if (!has_grad) launch<false, false, false>(grid, st, ptrs, args);
+    else if (f32) launch<false, true, true>(grid, st, ptrs, args);
+    else launch<false, true, false>(grid, st, ptrs, args);
+  }
+  tweo_detail::count_launch();
+  return tweo_detail::check_launch("tweo_loss_kernel");
+}

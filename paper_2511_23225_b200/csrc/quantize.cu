@@ -1,0 +1,186 @@
+// Per-tensor amax, scale and FP8 cast of a bf16 tensor (one scale for the whole tensor).
+//
+// HBM-bound streaming kernels.  CURRENT scaling is two passes (amax, then cast: 2+2+1 B
+// per element; the second read comes from L2 when the tensor fits there), GIVEN scaling
+// is one pass (2+1 B per element) that still reports the tensor's amax.  Loads are
+// 2 x 16 bytes per thread (16 bf16), stores 16 bytes (16 codes).  amax is the integer
+// maximum of the sign-stripped bf16 bit patterns (exact, order-independent; NaN
+// patterns are skipped), reduced by shuffles and one atomicMax per CTA.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace {
+
+using namespace tweo_detail;
+
+constexpr int kThreads = 256;
+
+// Largest |x| of a packed pair of bf16, as raw 15-bit-exponent+mantissa patterns, NaN -> 0.
+__device__ __forceinline__ uint32_t absmax_bits(uint32_t m, uint32_t w) {
+  uint32_t lo = w & 0x7FFFu, hi = (w >> 16) & 0x7FFFu;
+  lo = lo > 0x7F80u ? 0u : lo;
+  hi = hi > 0x7F80u ? 0u : hi;
+  return max(m, max(lo, hi));
+}
+
+__device__ __forceinline__ void cta_amax_to_global(uint32_t m, float* amax) {
+  __shared__ uint32_t part[kThreads / 32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int w = 1; w < kThreads / 32; ++w) m = max(m, part[w]);
+    // non-negative binary32 values order like their bit patterns
+    if (m) atomicMax(reinterpret_cast<unsigned int*>(amax), m << 16);
+  }
+}
+
+__global__ void init_kernel(float* amax, uint32_t* sat_count, const float* scale_in, float* scale_inv) {
+  *amax = 0.0f;
+  if (sat_count) *sat_count = 0u;
+  if (scale_in) *scale_inv = __fdiv_rn(1.0f, *scale_in);
+}
+
+__global__ void __launch_bounds__(kThreads) amax_kernel(const uint16_t* x, int64_t n, float* amax) {
+  const int64_t nvec = n >> 3;
+  const uint4* xv = reinterpret_cast<const uint4*>(x);
+  const int64_t stride = (int64_t)gridDim.x * kThreads * 4;
+  uint32_t m = 0;
+  for (int64_t base = (int64_t)blockIdx.x * kThreads * 4 + threadIdx.x; base < nvec; base += stride) {
+    uint4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      int64_t i = base + (int64_t)u * kThreads;
+      v[u] = i < nvec ? __ldg(xv + i) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      m = absmax_bits(m, v[u].x);
+      m = absmax_bits(m, v[u].y);
+      m = absmax_bits(m, v[u].z);
+      m = absmax_bits(m, v[u].w);
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x < 8) {
+    int64_t i = (nvec << 3) + threadIdx.x;
+    if (i < n) m = absmax_bits(m, (uint32_t)x[i]);
+  }
+  cta_amax_to_global(m, amax);
+}
+
+// 16 elements: two 16-byte loads -> one 16-byte store.
+template <int FMT>
+__device__ __forceinline__ uint4 cast16(const uint4 a, const uint4 b, float scale, uint32_t& sat, uint32_t& m,
+                                        bool want_amax) {
+  const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+  uint32_t c[8];
+  const float fmax = FMT == TWEO_E4M3 ? kE4M3Max : kE5M2Max;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    float lo = __fmul_rn(bf16lo_to_f32(w[j]), scale);
+    float hi = __fmul_rn(bf16hi_to_f32(w[j]), scale);
+    sat += (fabsf(lo) > fmax) + (fabsf(hi) > fmax);
+    c[j] = cvt_fp8x2<FMT>(lo, hi);
+    if (want_amax) m = absmax_bits(m, w[j]);
+  }
+  return make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16));
+}
+
+// CURRENT mode reads *amax (finished by the previous kernel) and derives the scale;
+// GIVEN mode reads *scale and accumulates amax while casting.
+template <int FMT, bool GIVEN>
+__global__ void __launch_bounds__(kThreads)
+cast_kernel(const uint16_t* x, int64_t n, float* scale, float* scale_inv, float* amax, uint8_t* q,
+            uint32_t* sat_count) {
+  float s;
+  if (GIVEN) {
+    s = *scale;
+  } else {
+    s = scale_from_amax(*amax, FMT);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      *scale = s;
+      *scale_inv = __fdiv_rn(1.0f, s);
+    }
+  }
+  const int64_t n16 = n >> 4;
+  const uint4* xv = reinterpret_cast<const uint4*>(x);
+  uint4* qv = reinterpret_cast<uint4*>(q);
+  const int64_t stride = (int64_t)gridDim.x * kThreads * 2;
+  uint32_t sat = 0, m = 0;
+  for (int64_t base = (int64_t)blockIdx.x * kThreads * 2 + threadIdx.x; base < n16; base += stride) {
+    uint4 v[2][2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      int64_t i = base + (int64_t)u * kThreads;
+      if (i < n16) {
+        v[u][0] = __ldcs(xv + 2 * i);
+        v[u][1] = __ldcs(xv + 2 * i + 1);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      int64_t i = base + (int64_t)u * kThreads;
+      if (i < n16) __stcs(qv + i, cast16<FMT>(v[u][0], v[u][1], s, sat, m, GIVEN));
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x < 16) {  // ragged tail: n % 16 elements
+    int64_t i = (n16 << 4) + threadIdx.x;
+    if (i < n) {
+      uint32_t w = x[i];
+      float v = __fmul_rn(bf16lo_to_f32(w), s);
+      sat += fabsf(v) > (FMT == TWEO_E4M3 ? kE4M3Max : kE5M2Max);
+      q[i] = (uint8_t)(cvt_fp8x2<FMT>(v, 0.0f) & 0xFFu);
+      if (GIVEN) m = absmax_bits(m, w);
+    }
+  }
+  if (sat_count) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sat += __shfl_xor_sync(0xFFFFFFFFu, sat, o);
+    if ((threadIdx.x & 31) == 0 && sat) atomicAdd(sat_count, sat);
+  }
+  if (GIVEN) cta_amax_to_global(m, amax);
+}
+
+int grid_for(int64_t work_items, int per_cta, int ctas_per_sm) {
+  int64_t want = (work_items + per_cta - 1) / per_cta;
+  int64_t cap = (int64_t)sm_count() * ctas_per_sm;
+  if (want > cap) want = cap;
+  if (want < 1) want = 1;
+  return (int)want;
+}
+
+}  // namespace
+
+extern "C" tweo_status_t tweo_quantize_per_tensor(const uint16_t* x, int64_t n, int32_t fmt, int32_t mode,
+                                                  float* scale, float* scale_inv, float* amax, uint8_t* q,
+                                                  uint32_t* sat_count, void* ws, size_t ws_bytes, void* stream) {
+  (void)ws;
+  (void)ws_bytes;
+  if (n < 0 || !scale || !scale_inv || !amax) return TWEO_ERR_INVALID_ARG;
+  if (n > 0 && (!x || !q)) return TWEO_ERR_INVALID_ARG;
+  if (fmt != TWEO_E4M3 && fmt != TWEO_E5M2) return TWEO_ERR_INVALID_ARG;
+  if (mode != TWEO_SCALE_CURRENT && mode != TWEO_SCALE_GIVEN) return TWEO_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(q)) return TWEO_ERR_ALIGNMENT;
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool given = mode == TWEO_SCALE_GIVEN;
+
+  init_kernel<<<1, 1, 0, st>>>(amax, sat_count, given ? scale : nullptr, scale_inv);
+  count_launch();
+  if (!given) {
+    amax_kernel<<<grid_for(n >> 3, kThreads * 4, 8), kThreads, 0, st>>>(x, n, amax);
+    count_launch();
+  }
+  const int grid = grid_for(n >> 4, kThreads * 2, 8);
+  if (fmt == TWEO_E4M3) {
+    if (given) cast_kernel<TWEO_E4M3, true><<<grid, kThreads, 0, st>>>(x, n, scale, scale_inv, amax, q, sat_count);
+    else cast_kernel<TWEO_E4M3, false><<<grid, kThreads, 0, st>>>(x, n, scale, scale_inv, amax, q, sat_count);
+  } else {
+    if (given) cast_kernel<TWEO_E5M2, true><<<grid, kThreads, 0, st>>>(x, n, scale, scale_inv, amax, q, sat_count);
+    else cast_kernel<TWEO_E5M2, false><<<grid, kThreads, 0, st>>>(x, n, scale, scale_inv, amax, q, sat_count);
+  }
+  count_launch();
+  return check_launch("tweo_quantize_per_tensor");
+}

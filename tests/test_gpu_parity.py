@@ -1,0 +1,340 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle.
+
+Bars: bit-exact for FP8 codes, amax, scale, scale_inv and saturation counts;
+relative Frobenius error <= 1e-2 for FP8 GEMM outputs against the FP64 product
+of the same quantised operands (bf16 rounding alone gives ~2^-9/sqrt(3) ~ 1.1e-3);
+relative error <= 1e-5 for the TWEO loss and the fp32 gradient.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tweo_oracle as orc
+from paper_2511_23225_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+E4M3, E5M2 = 0, 1
+GEMM_TOL = 1e-2
+TWEO_TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def tw():
+    from paper_2511_23225_b200 import binding
+    binding.lib()
+    return binding
+
+
+def to_gpu_bf16(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def bf16_to_bits(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def f32_bits(t: torch.Tensor) -> int:
+    return int(t.view(torch.int32).cpu().item()) & 0xFFFFFFFF
+
+
+def np_f32_bits(v) -> int:
+    return int(np.float32(v).view(np.uint32))
+
+
+def rel_fro(got: np.ndarray, ref: np.ndarray) -> float:
+    return float(np.linalg.norm(got.astype(np.float64) - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+# ------------------------------------------------------------------ quantize
+QUANT_CASES = [
+    ("cfg1_X", lambda: synth.linear_inputs(1, 0)[0]),
+    ("cfg1_W", lambda: synth.linear_inputs(1, 0)[1]),
+    ("grad_small", lambda: synth.normal_bf16(7, (333, 77), 1e-3)),          # ragged: 25641 elements
+    ("tiny", lambda: synth.normal_bf16(8, (5,), 1.0)),
+    ("cfg2_fc1_X_rows", lambda: synth.linear_inputs(2, 2, M=2048)[0]),      # outlier channel x500, many tiles
+    ("student_t", lambda: synth.normal_plus_student_t_bf16(9, (1024, 2048))),
+]
+
+
+@pytest.mark.parametrize("fmt", [E4M3, E5M2])
+@pytest.mark.parametrize("name,make", QUANT_CASES, ids=[c[0] for c in QUANT_CASES])
+def test_quantize_current_bit_exact(tw, fmt, name, make):
+    bits = make()
+    ref = orc.quantize_per_tensor_current(bits, fmt)
+    out = tw.quantize_per_tensor(to_gpu_bf16(bits), fmt, tw.SCALE_CURRENT, count_saturated=True)
+    torch.cuda.synchronize()
+    assert f32_bits(out.amax) == np_f32_bits(ref["amax"])
+    assert f32_bits(out.scale) == np_f32_bits(ref["scale"])
+    assert f32_bits(out.scale_inv) == np_f32_bits(ref["scale_inv"])
+    assert np.array_equal(out.q.cpu().numpy(), ref["q"])
+    assert int(out.sat_count.item()) == ref["sat_count"]
+
+
+@pytest.mark.parametrize("fmt", [E4M3, E5M2])
+def test_quantize_given_scale_saturates_and_reports_amax(tw, fmt):
+    bits = synth.normal_with_extreme_outliers_bf16(12, (700, 129))
+    # a static scale calibrated for |x| <= 6: the planted outliers must clip to +-max
+    scale = np.float32(orc.fp8_max(fmt) / 6.0)
+    q_ref, sat_ref = orc.quantize_bf16(bits, fmt, scale)
+    s = torch.tensor([scale], dtype=torch.float32, device="cuda")
+    out = tw.quantize_per_tensor(to_gpu_bf16(bits), fmt, tw.SCALE_GIVEN, scale=s, count_saturated=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.q.cpu().numpy(), q_ref)
+    assert int(out.sat_count.item()) == sat_ref and sat_ref > 0
+    assert f32_bits(out.amax) == np_f32_bits(orc.amax_bf16(bits))
+    assert f32_bits(out.scale_inv) == np_f32_bits(np.float32(1.0) / scale)
+
+
+def test_quantize_degenerate_inputs(tw):
+    z = torch.zeros(4096, dtype=torch.bfloat16, device="cuda")
+    out = tw.quantize_per_tensor(z, E4M3)
+    torch.cuda.synchronize()
+    assert out.amax.item() == 0.0 and out.scale.item() == 1.0 and not out.q.any()
+    e = torch.zeros(0, dtype=torch.bfloat16, device="cuda")
+    out = tw.quantize_per_tensor(e, E5M2)
+    torch.cuda.synchronize()
+    assert out.amax.item() == 0.0 and out.scale.item() == 1.0
+    # NaN is skipped by amax and maps to the NaN code; infinities saturate (codec parity on non-finite inputs)
+    bits = synth.normal_bf16(13, (64,), 1.0)
+    bits[3], bits[9] = 0x7FC0, 0xFFC0
+    ref = orc.quantize_per_tensor_current(bits, E4M3)
+    out = tw.quantize_per_tensor(to_gpu_bf16(bits), E4M3)
+    torch.cuda.synchronize()
+    assert f32_bits(out.amax) == np_f32_bits(ref["amax"])
+    assert np.array_equal(out.q.cpu().numpy(), ref["q"])
+
+
+def test_quantize_all_bf16_patterns_both_formats(tw):
+    """Every finite bf16 value through the GPU cast equals the oracle's code (scale 1 and an odd scale)."""
+    bits = np.arange(1 << 16, dtype=np.uint16)
+    f = synth.bf16_bits_to_f32(bits)
+    bits = bits[np.isfinite(f)]
+    for fmt in (E4M3, E5M2):
+        for sc in (1.0, 0.37109375, 173.25):
+            s = torch.tensor([sc], dtype=torch.float32, device="cuda")
+            out = tw.quantize_per_tensor(to_gpu_bf16(bits), fmt, tw.SCALE_GIVEN, scale=s)
+            torch.cuda.synchronize()
+            q_ref, _ = orc.quantize_bf16(bits, fmt, np.float32(sc))
+            assert np.array_equal(out.q.cpu().numpy(), q_ref)
+
+
+# ------------------------------------------------------------------ TWEO
+def _tweo_case(tw, blocks_bits, p, grad_dtype, c=0.01 / 12):
+    tau, eps = 3.0, 1e-6
+    blocks = [to_gpu_bf16(b) for b in blocks_bits]
+    loss, per, grads = tw.loss_fwd_bwd(blocks, tau, eps, p, c, True, grad_dtype)
+    torch.cuda.synchronize()
+    # the binding passes tau/eps/p/c as binary32; give the oracle the same values
+    tau32, eps32, p32, c32 = (float(np.float32(v)) for v in (tau, eps, p, c))
+    ref_total, ref_per = orc.tweo_loss(blocks_bits, tau32, eps32, p32)
+    assert abs(loss.item() - ref_total) <= TWEO_TOL * abs(ref_total)
+    for got, want in zip(per.cpu().numpy(), ref_per):
+        assert abs(got - want) <= TWEO_TOL * abs(want)
+    for b, g in zip(blocks_bits, grads):
+        ref = orc.tweo_grad_block(b, tau32, eps32, p32, c32)
+        if grad_dtype == tw.F32:
+            got = g.cpu().numpy().astype(np.float64)
+            assert rel_fro(got, ref) <= TWEO_TOL
+            assert np.all(np.abs(got - ref) <= TWEO_TOL * np.abs(ref) + 1e-38)
+        else:
+            # bf16 output = the fp32 value rounded once more: equal to the oracle's bf16 rounding except
+            # within one fp32 ulp of a rounding boundary, where it may be the neighbouring bf16 value
+            got_bits = bf16_to_bits(g)
+            ref_bits = orc.f64_array_to_bf16(ref)
+            got = synth.bf16_bits_to_f32(got_bits).astype(np.float64)
+            assert np.all(np.abs(got - ref) <= np.abs(ref) * 2.0 ** -8 * (1 + 1e-5) + 1e-38)
+            differ = (got_bits != ref_bits) & ~((got == 0) & (ref == 0))
+            assert differ.mean() < 1e-3
+            assert rel_fro(got, ref) <= 2.0 ** -8
+    return loss
+
+
+@pytest.mark.parametrize("grad_dtype", [0, 1], ids=["bf16grad", "f32grad"])
+def test_tweo_cfg1_block_output(tw, grad_dtype):
+    a = synth.block_output(1)
+    loss = _tweo_case(tw, [a], 4.0, grad_dtype)
+    assert loss.item() > 1e7   # extreme outliers dominate: (2000/3)^4 * 1e-3
+
+
+@pytest.mark.parametrize("grad_dtype", [0, 1], ids=["bf16grad", "f32grad"])
+def test_tweo_multi_block_ragged(tw, grad_dtype):
+    blocks = [synth.normal_with_outlier_channels_bf16(50 + i, (1237, 131)) for i in range(3)]  # 162047 elements each
+    _tweo_case(tw, blocks, 4.0, grad_dtype)
+
+
+@pytest.mark.parametrize("p", [2.0, 3.0, 2.5])
+def test_tweo_generic_exponent(tw, p):
+    blocks = [synth.normal_bf16(60 + i, (301, 97)) for i in range(2)]
+    _tweo_case(tw, blocks, p, 1)
+
+
+def test_tweo_loss_only_in_place_and_reproducible(tw):
+    bits = synth.block_output(2, M=1024)
+    a = to_gpu_bf16(bits)
+    ws = tw.new_workspace(tw.OP_LOSS, a.numel(), 1)
+    l1, _, g1 = tw.loss_fwd_bwd([a], ws=ws)
+    l0, _, none = tw.loss_fwd_bwd([a], want_grad=False, ws=ws)
+    l2, _, g2 = tw.loss_fwd_bwd([a], ws=ws)
+    torch.cuda.synchronize()
+    assert none is None
+    assert f32_bits(l1) == f32_bits(l0) == f32_bits(l2)       # fixed reduction order
+    assert torch.equal(g1[0].view(torch.int16), g2[0].view(torch.int16))
+    inplace = a.clone()
+    tw.loss_fwd_bwd([inplace], grads=[inplace], ws=ws)      # bf16 gradient may overwrite its input
+    torch.cuda.synchronize()
+    assert torch.equal(inplace.view(torch.int16), g1[0].view(torch.int16))
+    z = torch.zeros(4096, dtype=torch.bfloat16, device="cuda")
+    lz, _, gz = tw.loss_fwd_bwd([z])
+    torch.cuda.synchronize()
+    assert lz.item() == 0.0 and not gz[0].any()
+
+
+# ------------------------------------------------------------------ GEMMs
+def quantized_operands(x_bits, w_bits, dy_bits, fmt_g=E5M2):
+    qx = orc.quantize_per_tensor_current(x_bits, E4M3)
+    qw = orc.quantize_per_tensor_current(w_bits, E4M3)
+    qd = orc.quantize_per_tensor_current(dy_bits, fmt_g)
+    return qx, qw, qd
+
+
+def dev_scalar(v):
+    return torch.tensor([float(v)], dtype=torch.float32, device="cuda")
+
+
+def run_three(tw, qx, qw, qd, fmt_g, dw_f32=False):
+    xq, wq, dyq = (torch.from_numpy(q["q"]).cuda() for q in (qx, qw, qd))
+    sx, sw, sd = (dev_scalar(q["scale_inv"]) for q in (qx, qw, qd))
+    y = tw.fp8_linear_fwd(xq, wq, sx, sw)
+    dx = tw.fp8_linear_bwd_dgrad(dyq, wq, sd, sw, fmt_dy=fmt_g)
+    dw = tw.fp8_linear_bwd_wgrad(xq, dyq, sx, sd, fmt_dy=fmt_g, dw_dtype=tw.F32 if dw_f32 else tw.BF16)
+    torch.cuda.synchronize()
+    assert tw.read_device_status() == 0
+    return y, dx, dw
+
+
+GEMM_SHAPES = [
+    # (name, M, K, N, maker)
+    ("cfg1", 512, 256, 1024),
+    ("one_tile", 128, 128, 256),
+    ("ragged_all", 300, 400, 272),     # ragged M, K not a multiple of 128, N not a multiple of 256
+    ("narrow_n", 200, 256, 128),       # BN = 128 path
+    ("m1", 1, 512, 512),
+    ("m16", 16, 512, 768),
+]
+
+
+@pytest.mark.parametrize("fmt_g", [E5M2, E4M3], ids=["e5m2grad", "e4m3grad"])
+@pytest.mark.parametrize("name,M,K,N", GEMM_SHAPES, ids=[s[0] for s in GEMM_SHAPES])
+def test_gemms_small_full_compare(tw, name, M, K, N, fmt_g):
+    if name == "cfg1":
+        x, w, dy = synth.linear_inputs(1, 0)
+    else:
+        x = synth.normal_with_outlier_channels_bf16(70, (M, K))
+        w = synth.normal_bf16(71, (N, K), 0.02)
+        dy = synth.normal_bf16(72, (M, N), 1e-3)
+    qx, qw, qd = quantized_operands(x, w, dy, fmt_g)
+    y, dx, dw = run_three(tw, qx, qw, qd, fmt_g)
+    y_ref = orc.gemm_fwd(qx["q"], E4M3, qw["q"], E4M3, qx["scale_inv"], qw["scale_inv"])
+    dx_ref = orc.gemm_dgrad(qd["q"], fmt_g, qw["q"], E4M3, qd["scale_inv"], qw["scale_inv"])
+    dw_ref = orc.gemm_wgrad(qx["q"], E4M3, qd["q"], fmt_g, qx["scale_inv"], qd["scale_inv"])
+    for got, ref, what in ((y, y_ref, "fwd"), (dx, dx_ref, "dgrad"), (dw, dw_ref, "wgrad")):
+        err = rel_fro(got.float().cpu().numpy(), ref)
+        assert err <= GEMM_TOL, f"{what} {name}: rel err {err}"
+        # element-wise: bf16 rounding of the exact value, plus fp32 accumulation noise
+        g = got.float().cpu().numpy().astype(np.float64)
+        scale = np.max(np.abs(ref)) + 1e-300
+        assert np.max(np.abs(g - ref) - np.abs(ref) * 2.0 ** -8) <= 1e-4 * scale, what
+
+
+def test_wgrad_fp32_output_and_accumulate(tw):
+    x = synth.normal_bf16(80, (640, 256))
+    w = synth.normal_bf16(81, (384, 256), 0.02)
+    dy = synth.normal_bf16(82, (640, 384), 1e-3)
+    qx, qw, qd = quantized_operands(x, w, dy)
+    _, _, dw = run_three(tw, qx, qw, qd, E5M2, dw_f32=True)
+    ref = orc.gemm_wgrad(qx["q"], E4M3, qd["q"], E5M2, qx["scale_inv"], qd["scale_inv"])
+    assert rel_fro(dw.cpu().numpy(), ref) <= 1e-5
+    xq, dyq = torch.from_numpy(qx["q"]).cuda(), torch.from_numpy(qd["q"]).cuda()
+    tw.fp8_linear_bwd_wgrad(xq, dyq, dev_scalar(qx["scale_inv"]), dev_scalar(qd["scale_inv"]), dw=dw,
+                            dw_dtype=tw.F32, accumulate=True)
+    torch.cuda.synchronize()
+    assert rel_fro(dw.cpu().numpy(), 2 * ref) <= 1e-5
+
+
+def test_fused_epilogue_equals_unfused_bit_for_bit(tw):
+    x, w, _ = synth.linear_inputs(4, 1, M=384)          # llama 'o' projection rows: heavy-tailed input
+    qx = orc.quantize_per_tensor_current(x, E4M3)
+    qw = orc.quantize_per_tensor_current(w, E4M3)
+    xq, wq = torch.from_numpy(qx["q"]).cuda(), torch.from_numpy(qw["q"]).cuda()
+    sx, sw = dev_scalar(qx["scale_inv"]), dev_scalar(qw["scale_inv"])
+    M, N = xq.shape[0], wq.shape[0]
+    y_plain = tw.fp8_linear_fwd(xq, wq, sx, sw)
+    next_scale = dev_scalar(448.0 / 40.0)               # a delayed scale: some outputs will saturate
+    amax = torch.empty(1, dtype=torch.float32, device="cuda")
+    yq = torch.empty((M, N), dtype=torch.uint8, device="cuda")
+    y_fused = tw.fp8_linear_fwd(xq, wq, sx, sw, out_amax=amax, out_q=yq, q_fmt=E4M3, q_scale=next_scale)
+    torch.cuda.synchronize()
+    assert torch.equal(y_plain.view(torch.int16), y_fused.view(torch.int16))
+    y_bits = bf16_to_bits(y_fused)
+    # oracle applied to the GPU's own bf16 output
+    assert f32_bits(amax) == np_f32_bits(orc.amax_bf16(y_bits))
+    q_ref, _ = orc.quantize_bf16(y_bits, E4M3, np.float32(next_scale.item()))
+    assert np.array_equal(yq.cpu().numpy(), q_ref)
+    # and to the library's own unfused route
+    s = next_scale.clone()
+    unf = tw.quantize_per_tensor(y_fused, E4M3, tw.SCALE_GIVEN, scale=s)
+    torch.cuda.synchronize()
+    assert torch.equal(unf.q, yq) and f32_bits(unf.amax) == f32_bits(amax)
+
+
+def sample_points(g, rows, cols, n_rows=4, n_pts=2048):
+    r_full = g.choice(rows, size=min(n_rows, rows), replace=False)
+    rr = np.repeat(r_full, cols)
+    cc = np.tile(np.arange(cols), len(r_full))
+    pr, pc = g.integers(0, rows, n_pts), g.integers(0, cols, n_pts)
+    return np.concatenate([rr, pr]), np.concatenate([cc, pc])
+
+
+@pytest.mark.parametrize("cfg,lin,M", [(2, 0, None), (2, 3, None), (4, 4, 4096), (3, 2, 50432 // 8)],
+                         ids=["cfg2_qkv", "cfg2_fc2", "cfg4_down_rows", "cfg3_fc1_rows"])
+def test_gemms_benchmark_shapes_sampled(tw, cfg, lin, M):
+    """Full-width linears of the benchmark configs; the oracle evaluates whole rows plus scattered points."""
+    x, w, dy = synth.linear_inputs(cfg, lin, M=M)
+    qx, qw, qd = quantized_operands(x, w, dy)
+    y, dx, dw = run_three(tw, qx, qw, qd, E5M2)
+    g = np.random.Generator(np.random.PCG64(99))
+    Mx, K = qx["q"].shape
+    N = qw["q"].shape[0]
+    r, c = sample_points(g, Mx, N)
+    ref = orc.gemm_fwd_at(qx["q"], E4M3, qw["q"], E4M3, qx["scale_inv"], qw["scale_inv"], r, c)
+    assert rel_fro(y.float().cpu().numpy()[r, c], ref) <= GEMM_TOL
+    r, c = sample_points(g, Mx, K)
+    ref = orc.gemm_dgrad_at(qd["q"], E5M2, qw["q"], E4M3, qd["scale_inv"], qw["scale_inv"], r, c)
+    assert rel_fro(dx.float().cpu().numpy()[r, c], ref) <= GEMM_TOL
+    r, c = sample_points(g, N, K, n_rows=2, n_pts=1024)
+    ref = orc.gemm_wgrad_at(qx["q"], E4M3, qd["q"], E5M2, qx["scale_inv"], qd["scale_inv"], r, c)
+    assert rel_fro(dw.float().cpu().numpy()[r, c], ref) <= GEMM_TOL
+
+
+# ------------------------------------------------------------------ static W8A8
+@pytest.mark.parametrize("M", [1, 16, 128, 1024])
+def test_w8a8_static_gemm(tw, M):
+    K, N = 4096, 4096
+    w = synth.w8a8_weight(K, N)
+    qw = orc.quantize_per_tensor_current(w, E4M3)
+    # calibration: amax over seeded batches (fewer rows here than the benchmark uses; same recipe)
+    amax_cal = max(float(orc.amax_bf16(synth.w8a8_calibration_batch(K, i, rows=64))) for i in range(4))
+    sx = np.float32(448.0) / np.float32(amax_cal)
+    x = synth.w8a8_activation(M, K)
+    xq_ref, _ = orc.quantize_bf16(x, E4M3, sx)
+    sx_inv = np.float32(1.0) / sx
+    g = np.random.Generator(np.random.PCG64(5))
+    r, c = sample_points(g, M, N, n_rows=2, n_pts=1024)
+    ref = orc.gemm_fwd_at(xq_ref, E4M3, qw["q"], E4M3, sx_inv, qw["scale_inv"], r, c)
+    wq = torch.from_numpy(qw["q"]).cuda()
+    y = tw.w8a8_static_gemm(to_gpu_bf16(x), dev_scalar(sx), wq, dev_scalar(qw["scale_inv"]))
+    y2 = tw.w8a8_static_gemm(torch.from_numpy(xq_ref).cuda(), dev_scalar(sx), wq, dev_scalar(qw["scale_inv"]))
+    torch.cuda.synchronize()
+    assert rel_fro(y.float().cpu().numpy()[r, c], ref) <= GEMM_TOL
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))   # cast inside == pre-cast codes
