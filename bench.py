@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the FP8 per-tensor linear + TWEO-loss hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg1|cfg3|cfg4] [--impl reference]
+
+One step = per linear of the block: per-tensor FP8 casts of X, W (E4M3) and dY
+(E5M2) with current scaling, forward / dgrad / wgrad GEMMs; then the TWEO loss
+and gradient on the block output.  Prints ONE JSON line (rank 0).
+
+  value        FP8 linear fwd+bwd TFLOP/s over the whole step (casts and the TWEO
+               pass included in the time, 6*M*K*N flop per linear), inputs resident
+               in HBM, CUDA-event timed, max over ranks, summed over ranks (weak
+               scaling: every rank runs its own token shard, no data-path collective).
+  e2e          same metric with the step's inputs copied from pinned host memory and
+               the loss read back inside the timed region.
+  roofline     dominant kernel family (largest share of the instrumented step time),
+               algorithmic flops or bytes / CUDA-event duration, against the measured
+               peak in MEASURED_PEAKS.json (fallback stated if absent).
+  cpu_baseline the CPU oracle, as it stands, timed on a bounded sample (N=1, rank 0).
+
+`--impl reference` times the CPU oracle alone (there is no reference code for this
+paper; the oracle is the reference arm).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fp8_linear_fwd_bwd_tflops_with_tweo_loss"
+UNIT = "TFLOP/s"
+FP8_DATASHEET_TFLOPS = 4500.0
+FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, FALLBACK_BF16_SUSTAINED = 6650.0, 1590.0, 1400.0
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=FALLBACK_HBM_GBS, bf16=FALLBACK_BF16_TFLOPS, bf16_sustained=FALLBACK_BF16_SUSTAINED,
+                source="fallback")
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def oracle_sample_step(cfg_idx: int, rows: int):
+    """Runs the oracle over the first `rows` tokens of every linear of the config (full K, N;
+    the weight-gradient contraction runs over those rows only) plus the TWEO term on the same
+    rows.  Returns (flops, seconds)."""
+    import numpy as np
+    from oracle import tweo_oracle as orc
+    from paper_2511_23225_b200 import synth
+    cfg = synth.CONFIGS[cfg_idx]
+    inputs = [synth.linear_inputs(cfg_idx, i, M=rows) for i in range(len(cfg.linears))]
+    a = synth.block_output(cfg_idx, 0, M=rows)
+    orc.lib()
+    t0 = time.perf_counter()
+    flops = 0
+    for (x, w, dy) in inputs:
+        qx = orc.quantize_per_tensor_current(x, orc.E4M3)
+        qw = orc.quantize_per_tensor_current(w, orc.E4M3)
+        qd = orc.quantize_per_tensor_current(dy, orc.E5M2)
+        orc.gemm_fwd(qx["q"], orc.E4M3, qw["q"], orc.E4M3, qx["scale_inv"], qw["scale_inv"])
+        orc.gemm_dgrad(qd["q"], orc.E5M2, qw["q"], orc.E4M3, qd["scale_inv"], qw["scale_inv"])
+        orc.gemm_wgrad(qx["q"], orc.E4M3, qd["q"], orc.E5M2, qx["scale_inv"], qd["scale_inv"])
+        flops += 6 * x.shape[0] * x.shape[1] * w.shape[0]
+    orc.tweo_loss_block(a, 3.0, 1e-6, 4.0)
+    orc.tweo_grad_block(a, 3.0, 1e-6, 4.0, 0.01)
+    return flops, time.perf_counter() - t0
+
+
+def cpu_threads() -> int:
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env and env.isdigit():
+        return int(env)
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    cfg_idx = int(args.workload[3:])
+    rows = args.ref_rows
+    for _ in range(args.warmup):
+        oracle_sample_step(cfg_idx, min(rows, 32))
+    times, flops = [], 0
+    for _ in range(args.steps):
+        f, t = oracle_sample_step(cfg_idx, rows)
+        flops, _ = f, times.append(t)
+    tot = sum(times)
+    val = flops * len(times) / tot / 1e12
+    sample = f"first {rows} tokens of every linear (full K,N) + TWEO on {rows} rows, per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * tot / len(times), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(cfg_idx), "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def workload_name(cfg_idx: int) -> str:
+    from paper_2511_23225_b200 import synth
+    return f"cfg{cfg_idx}:{synth.CONFIGS[cfg_idx].name}"
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
+        }
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or getattr(
+            nv, "nvmlDeviceGetCurrentClocksThrottleReasons", None)
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                if get_reasons:
+                    r = get_reasons(self.h)
+                    for bit, name in names.items():
+                        if r & bit:
+                            self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.nv:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread:
+            self._stop.set()
+            self._thread.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- CUDA arm
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2511_23225_b200 import binding as tw
+    from paper_2511_23225_b200.workload import BlockStep
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    tw.lib()  # fail loudly if the library is missing
+    cfg_idx = int(args.workload[3:])
+    peaks = load_peaks()
+
+    bs = BlockStep(cfg_idx)
+    bs.make_host_inputs()
+    bs.upload()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        bs.step()
+    barrier()
+    if tw.read_device_status() != 0:
+        raise SystemExit("device status reports an expired wait")
+
+    # ---- timed region: K steps, inputs resident in HBM
+    sampler = ClockSampler(local)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = tw.launch_count()
+    barrier()
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        bs.step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    launches = tw.launch_count() - launches0
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * bs.flops_per_step / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: pinned host inputs -> device, step, loss back to host, every step
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    host_loss = torch.empty(1, dtype=torch.float32).pin_memory()
+    for _ in range(2):
+        bs.upload()
+        bs.step()
+        host_loss.copy_(bs.loss, non_blocking=True)
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        bs.upload()
+        bs.step()
+        host_loss.copy_(bs.loss, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * bs.flops_per_step / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    loss_value = float(host_loss.item())
+
+    # ---- instrumented steps: CUDA events around every library call, per kernel family
+    fam = {"quantize": [0.0, 0, 0.0], "gemm": [0.0, 0, 0.0], "tweo_loss": [0.0, 0, 0.0]}  # ms, calls, work
+    inst_steps = max(1, min(args.steps, 30))
+    pairs = []
+
+    def timed(name, work, fn):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        pairs.append((name, work, a, b))
+
+    for _ in range(inst_steps):
+        for lb in bs.linears:
+            n_el = lb.x.numel() + lb.w.numel() + lb.dy.numel()
+            timed("quantize", 5.0 * n_el, lambda: bs.quantize_all(lb))          # 2 + 2 + 1 bytes per element
+            timed("gemm", float(lb.flops), lambda: bs.gemms(lb))
+        n_a = sum(t.numel() for t in bs.a)
+        timed("tweo_loss", 4.0 * n_a, bs.tweo)                                    # 2 read + 2 written
+    torch.cuda.synchronize()
+    for name, work, a, b in pairs:
+        fam[name][0] += a.elapsed_time(b)
+        fam[name][1] += 1
+        fam[name][2] += work
+    total_inst = sum(v[0] for v in fam.values())
+    kernels = {}
+    for name, (tms, calls, work) in fam.items():
+        rate = work / (tms * 1e-3) if tms > 0 else 0.0
+        kernels[name] = {"share": tms / total_inst, "ms_per_step": tms / inst_steps,
+                         "achieved": rate / 1e12 if name == "gemm" else rate / 1e9,
+                         "unit": "TFLOP/s" if name == "gemm" else "GB/s"}
+    dom = max(fam, key=lambda k: fam[k][0])
+    fp8_peak = 2.0 * peaks["bf16_sustained"]  # FP8 dense = 2x bf16 (nominal ratio) on the sustained bf16 figure
+    if dom == "gemm":
+        roof = {"bound": "tensor", "achieved": kernels["gemm"]["achieved"], "peak": fp8_peak, "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": kernels[dom]["achieved"], "peak": peaks["hbm"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof["kernel"] = dom
+    roof["peak_source"] = ("of measured" if peaks["source"] == "measured" else "of fallback") + \
+        (" (2 x sustained bf16)" if dom == "gemm" else " (copy bandwidth)")
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "fp8_e4m3xe5m2_fp32acc", "data": "synthetic",
+            "config": {"workload": workload_name(cfg_idx), "tokens_per_gpu": bs.M,
+                       "linears": [f"{l.name}:{l.K}x{l.N}" for l in bs.cfg.linears], "tweo_blocks": bs.n_blocks,
+                       "parallelism": f"replicas x{world} (token shards, no data-path collective)",
+                       "l2": f"working set {bs.working_set_bytes() / 1e6:.0f} MB per step > 126 MB L2, no flush"},
+            "pct_of_fp8_datasheet_peak": 100.0 * value / world / FP8_DATASHEET_TFLOPS,
+            "pct_of_fp8_measured_peak": 100.0 * value / world / fp8_peak,
+            "gemm_only_tflops": world * kernels["gemm"]["achieved"],
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bs.h2d_bytes(), "d2h_bytes_per_step": 4,
+                    "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": roof,
+            "kernels": kernels,
+            "tweo_loss": loss_value,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            f, t = oracle_sample_step(cfg_idx, args.cpu_rows)
+            line["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                    "sample": f"first {args.cpu_rows} of {bs.M} tokens of every linear (full K,N) "
+                                              f"+ TWEO on {args.cpu_rows} rows; {t:.1f} s"}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--cpu-rows", type=int, default=4096)
+    ap.add_argument("--ref-rows", type=int, default=128)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps > 50:
+            args.steps = 50  # each step is a bounded CPU sample; keep the run to a few minutes
+        return run_reference(args)
+    return run_cuda(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
