@@ -181,6 +181,36 @@ TWEO_API tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, in
                                 size_t ws_bytes, void* stream);
 
 /*
+ * tweo_loss_fwd_bwd_static -- tweo_loss_fwd_bwd without a workspace argument.
+ * (The paper has no counterpart to this call; it exists for deployment reasons only.)
+ *
+ * Some programs that embed this library may not allocate GPU memory at the point where
+ * they call it: an inference or training server that hands all device memory to its own
+ * pool at start-up and forbids later cudaMalloc calls, a plug-in running inside a host
+ * application that owns the allocator, or a control loop that cannot tolerate the latency
+ * or the possible failure of an allocation.  For them the scratch memory of the loss
+ * kernel (its per-CTA partial sums and its ticket counter) is a fixed 33024-byte array
+ * compiled into the library; every GPU that loads the library holds it until the process
+ * exits.  Inputs and outputs are still the caller's.  Arguments, results and numerics are
+ * those of tweo_loss_fwd_bwd (same kernel, same reduction order).
+ *
+ *   Limit: L * (CTAs per tensor) must not exceed 4096 partial sums; beyond that the call
+ *     returns TWEO_ERR_WORKSPACE_TOO_SMALL and does nothing (on a 148-SM B200 the kernel
+ *     uses at most 1184 + L CTAs, so every L <= TWEO_MAX_BLOCKS fits).
+ *   The call performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *   First call on a device: looks up the array's device address (once per device, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   The array is shared by every call in the process and keeps the last call's contents;
+ *     the call clears the part that must start at zero.  Two such calls that overlap on
+ *     the GPU (different streams, or different threads) race on it: serialise them, or
+ *     use tweo_loss_fwd_bwd with separate workspaces.
+ */
+TWEO_API tweo_status_t tweo_loss_fwd_bwd_static(const uint16_t* const* a, int32_t L, int64_t n_per_tensor,
+                                                float tau, float eps, float p, float grad_coeff, float* loss,
+                                                float* loss_per_block, void* const* grad, int32_t grad_dtype,
+                                                void* stream);
+
+/*
  * tweo_w8a8_static_gemm -- inference linear with static per-tensor scales for
  * both operands (Sec. 4.3: AbsMax static quantisation, W8(T)A8(T)), in the E4M3
  * flavour: Y[M,N] = (Xq . Wq^T) * (1 / *sx) * (*sw_inv) -> bf16.

@@ -24,7 +24,7 @@ LIB_PATH = os.path.join(_HERE, "libtweo_b200.so")
 
 EXPORTS = [
     "tweo_quantize_per_tensor", "tweo_fp8_linear_fwd", "tweo_fp8_linear_bwd_dgrad",
-    "tweo_fp8_linear_bwd_wgrad", "tweo_loss_fwd_bwd", "tweo_w8a8_static_gemm",
+    "tweo_fp8_linear_bwd_wgrad", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
 ]
@@ -67,6 +67,8 @@ def lib() -> C.CDLL:
                                                 i64, i64, i64, vp, sz, vp]
         L.tweo_loss_fwd_bwd.argtypes = [C.POINTER(vp), i32, i64, f32, f32, f32, f32, vp, vp, C.POINTER(vp), i32,
                                         vp, sz, vp]
+        L.tweo_loss_fwd_bwd_static.argtypes = [C.POINTER(vp), i32, i64, f32, f32, f32, f32, vp, vp, C.POINTER(vp),
+                                               i32, vp]
         L.tweo_w8a8_static_gemm.argtypes = [vp, i32, i64, vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, sz, vp]
         L.tweo_workspace_bytes.argtypes = [i32, i64, i64, i64]
         L.tweo_workspace_bytes.restype = sz
@@ -267,6 +269,41 @@ def loss_fwd_bwd(blocks, tau=3.0, eps=1e-6, p=4.0, grad_coeff=1.0, want_grad=Tru
                                    pb.data_ptr() if pb is not None else None, g_arr, grad_dtype, ws.data_ptr(),
                                    ws.numel(), _stream()), "tweo_loss_fwd_bwd")
     return loss, pb, grads
+
+
+def loss_fwd_bwd_static(blocks, tau=3.0, eps=1e-6, p=4.0, grad_coeff=1.0, want_grad=True, grad_dtype=BF16,
+                        grads=None, loss=None, per_block_out=None):
+    """tweo_loss_fwd_bwd_static: the TWEO loss and gradient for callers that may not allocate
+    device memory when they call.  The library's built-in scratch array replaces the workspace;
+    pass `grads`, `loss` and `per_block_out` to keep this wrapper from allocating as well.
+    Calls that overlap on the GPU share that array and race: issue them on one stream."""
+    Lb = len(blocks)
+    n = blocks[0].numel()
+    dev = blocks[0].device
+    a_arr = (C.c_void_p * Lb)()
+    for i, b in enumerate(blocks):
+        if b.numel() != n or not b.is_contiguous():
+            raise ValueError("block outputs must be contiguous and of equal size")
+        a_arr[i] = _dev(b, torch.bfloat16, "block output")
+    g_arr = None
+    if want_grad:
+        gdt = torch.bfloat16 if grad_dtype == BF16 else torch.float32
+        if grads is None:
+            grads = [torch.empty(b.shape, dtype=gdt, device=dev) for b in blocks]
+        g_arr = (C.c_void_p * Lb)()
+        for i, g in enumerate(grads):
+            g_arr[i] = _dev(g, gdt, "grad")
+    else:
+        grads = None
+    if loss is None:
+        loss = torch.empty(1, dtype=torch.float32, device=dev)
+    if per_block_out is None:
+        per_block_out = torch.empty(Lb, dtype=torch.float32, device=dev)
+    _check(lib().tweo_loss_fwd_bwd_static(a_arr, Lb, n, tau, eps, p, grad_coeff,
+                                          _dev(loss, torch.float32, "loss"),
+                                          _dev(per_block_out, torch.float32, "per_block_out"), g_arr, grad_dtype,
+                                          _stream()), "tweo_loss_fwd_bwd_static")
+    return loss, per_block_out, grads
 
 
 def w8a8_static_gemm(x, sx, wq, sw_inv, y=None, ws=None) -> torch.Tensor:

@@ -9,6 +9,8 @@
 // scheduling.  The ticket counter is left at zero for the next call.
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace tweo_detail {
@@ -271,4 +273,104 @@ extern "C" tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, 
   }
   tweo_detail::count_launch();
   return tweo_detail::check_launch("tweo_loss_kernel");
+}
+
+// ---------------------------------------------------------------------------------------
+// Variant of the entry point above for callers that cannot allocate device memory.
+//
+// The partial sums and the ticket counter live in a fixed array inside the library image
+// instead of a caller-provided workspace.  Every GPU that loads the library holds these
+// 33 KB until the process exits.  The kernel is the one above, unchanged.
+namespace {
+
+constexpr size_t kStaticPartials = 4096;                                   // partial sums that fit
+constexpr size_t kStaticScratchBytes = 256 + sizeof(double) * kStaticPartials;  // 33024 bytes
+
+static __device__ __align__(256) unsigned char g_loss_static_scratch[kStaticScratchBytes];
+
+// In host code the array's name is only a handle for the runtime, not a device address:
+// the real address is looked up once per device, with that device current.
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {nullptr};
+std::mutex g_static_scratch_mutex;
+
+tweo_status_t static_scratch_for_current_device(void** out) {
+  int dev = -1;
+  TWEO_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return TWEO_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (!g_static_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    TWEO_CUDA_TRY(cudaGetSymbolAddress((void**)&ptr, g_loss_static_scratch));
+    if (!ptr) return TWEO_ERR_CUDA;
+    g_static_scratch_addr[dev] = ptr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return TWEO_OK;
+}
+
+}  // namespace
+
+extern "C" tweo_status_t tweo_loss_fwd_bwd_static(const uint16_t* const* a, int32_t L, int64_t n_per_tensor,
+                                                  float tau, float eps, float p, float grad_coeff, float* loss,
+                                                  float* loss_per_block, void* const* grad, int32_t grad_dtype,
+                                                  void* stream) {
+  if (!a || !loss || L < 1 || L > TWEO_MAX_BLOCKS || n_per_tensor < 0) return TWEO_ERR_INVALID_ARG;
+  if (!(p > 1.0f) || !(tau + eps > 0.0f)) return TWEO_ERR_INVALID_ARG;
+  if (grad && grad_dtype != TWEO_BF16 && grad_dtype != TWEO_F32) return TWEO_ERR_INVALID_ARG;
+  const int blocks = tweo_detail::loss_blocks_per_tensor(n_per_tensor, L);
+  if ((size_t)blocks * (size_t)L > kStaticPartials) {
+    // more partial sums than the built-in scratch holds: use tweo_loss_fwd_bwd with a workspace
+    return TWEO_ERR_WORKSPACE_TOO_SMALL;
+  }
+
+  LossPtrs ptrs;
+  for (int l = 0; l < L; ++l) {
+    if (!a[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
+    if (!aligned16(a[l])) return TWEO_ERR_ALIGNMENT;
+    ptrs.a[l] = a[l];
+    ptrs.g[l] = nullptr;
+    if (grad) {
+      if (!grad[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
+      if (!aligned16(grad[l])) return TWEO_ERR_ALIGNMENT;
+      if (grad_dtype == TWEO_F32 && grad[l] == (const void*)a[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
+      ptrs.g[l] = grad[l];
+    }
+  }
+
+  void* scratch = nullptr;
+  tweo_status_t s = static_scratch_for_current_device(&scratch);
+  if (s != TWEO_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  // The array keeps whatever the previous call left; the ticket counter must start at zero.
+  TWEO_CUDA_TRY(cudaMemsetAsync(scratch, 0, 256, st));
+
+  LossArgs args;
+  args.n = n_per_tensor;
+  args.L = L;
+  args.p = p;
+  const double d = (double)tau + (double)eps;
+  const double norm = (double)n_per_tensor * pow(d, (double)p);
+  args.inv_norm = n_per_tensor > 0 ? 1.0 / norm : 0.0;
+  args.k_grad = n_per_tensor > 0 ? (float)((double)grad_coeff * (double)p / norm) : 0.0f;
+  args.loss = loss;
+  args.loss_per_block = loss_per_block;
+  args.ticket = reinterpret_cast<unsigned int*>(scratch);
+  args.partials = reinterpret_cast<double*>(reinterpret_cast<char*>(scratch) + 256);
+
+  dim3 grid((unsigned)blocks, (unsigned)L);
+  const bool fast = (p == 4.0f);
+  const bool has_grad = grad != nullptr;
+  const bool f32 = grad_dtype == TWEO_F32;
+  if (fast) {
+    if (!has_grad) launch<true, false, false>(grid, st, ptrs, args);
+    else if (f32) launch<true, true, true>(grid, st, ptrs, args);
+    else launch<true, true, false>(grid, st, ptrs, args);
+  } else {
+    if (!has_grad) launch<false, false, false>(grid, st, ptrs, args);
+    else if (f32) launch<false, true, true>(grid, st, ptrs, args);
+    else launch<false, true, false>(grid, st, ptrs, args);
+  }
+  tweo_detail::count_launch();
+  return tweo_detail::check_launch("tweo_loss_kernel (static scratch)");
 }
