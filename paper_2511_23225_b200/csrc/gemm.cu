@@ -14,7 +14,9 @@
 //
 // CTA = 192 threads: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the
 // MMAs (one thread), warps 2-5 are the epilogue (each reads its own 32-lane quarter of
-// tensor memory).  The kernel is persistent (grid = #SMs, static tile striding) with a
+// tensor memory, converts, stages 32 rows x 128 bytes in swizzled shared memory and hands
+// them to a TMA store, so global writes are full lines and ragged edges are clipped by
+// the hardware).  The kernel is persistent (grid = #SMs, static tile striding) with a
 // ring of shared-memory stages and two accumulators in tensor memory, so the epilogue of
 // tile i overlaps the main loop of tile i+1.  Every mbarrier wait is bounded: on expiry
 // the CTA records TWEO_ERR_TIMEOUT in a device status word, drains and exits.
@@ -108,6 +110,29 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// shared -> global tile store (bulk async group); out-of-range rows / columns are clipped
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(src)
+               : "memory");
+}
+// same, but adds the tile to what global memory holds (fp32 accumulate)
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t src) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -176,10 +201,10 @@ __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d) {
 }
 
 // ----------------------------------------------------------------- the kernel
-template <int BN, bool A_MN, bool B_MN, int STAGES>
+template <int BN, bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                const GemmParams p) {
+                const __grid_constant__ CUtensorMap tmap_d, const GemmParams p) {
   constexpr uint32_t A_BYTES = BM * BK;
   constexpr uint32_t B_BYTES = BN * BK;
   constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
@@ -189,7 +214,11 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  // epilogue staging: per epilogue warp two buffers of 32 rows x 128 bytes (128-byte swizzle)
+  constexpr uint32_t EPI_BUF = 32 * 128;
+  constexpr uint32_t EPI_BYTES = 4 * 2 * EPI_BUF;
+  uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES);
   // bars: [0,STAGES) full, [STAGES,2*STAGES) empty, then tmem_full[2], tmem_empty[2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -300,6 +329,11 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     const int quarter = warp & 3;  // tensor-memory lanes [32*quarter, 32*quarter+32) belong to this warp
     const float alpha = __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
     const float qs = p.out_q ? __ldg(p.q_scale) : 0.0f;
+    constexpr int CH = OUT_F32 ? 32 : 64;  // output columns per 128-byte staging row
+    const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
+    const uint32_t row_off = (uint32_t)lane * 128u;
+    const uint32_t swz = (uint32_t)(lane & 7);
+    uint32_t it = 0;
     float run_amax = 0.0f;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -309,69 +343,77 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const int n0 = (tile / p.tiles_m) * BN;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int row = m0 + quarter * 32 + lane;
+      const int row0 = m0 + quarter * 32;
+      const int row = row0 + lane;
       const bool row_ok = row < p.Md;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int col0 = n0 + c * 32;
+      for (int c = 0; c < BN / CH; ++c) {
+        const int col0 = n0 + c * CH;
         if (col0 >= p.Nd) break;  // uniform across the warp
-        uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
+        uint32_t r[CH];
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c * CH);
+        tmem_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+        if (!OUT_F32) tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[CH - 32]));
         tmem_ld_wait();
-        if (!row_ok) continue;
-        if (p.out_f32) {
-          float* drow = reinterpret_cast<float*>(p.d) + (int64_t)row * p.ldd + col0;
+        if (row0 >= p.Md) continue;  // whole warp past the ragged edge (uniform)
+        const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
+        // the store issued two chunks ago must have finished reading this buffer
+        if (lane == 0) bulk_wait_read<1>();
+        __syncwarp();
+        if (OUT_F32) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            if (col0 + j < p.Nd) {
-              float4 v = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
-                                     __uint_as_float(r[j + 2]) * alpha, __uint_as_float(r[j + 3]) * alpha);
-              float4* dst = reinterpret_cast<float4*>(drow + j);
-              if (p.accumulate) {
-                float4 o = *dst;
-                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-              }
-              *dst = v;
-            }
-          }
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j]), alpha)),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 1]), alpha)),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 2]), alpha)),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 3]), alpha)));
         } else {
-          uint16_t* drow = reinterpret_cast<uint16_t*>(p.d) + (int64_t)row * p.ldd + col0;
-          uint32_t packed[16];
+          uint32_t packed[CH / 2];
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
+          for (int j = 0; j < CH / 2; ++j)
             packed[j] = f32x2_to_bf16x2(__fmul_rn(__uint_as_float(r[2 * j]), alpha),
                                         __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha));
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            if (col0 + 8 * j < p.Nd)
-              *reinterpret_cast<uint4*>(drow + 8 * j) =
-                  make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
-          if (p.out_amax || p.out_q) {
-            // fused amax / cast act on the bf16-rounded values just stored
-            uint32_t q[8];
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1],
+                         packed[4 * j + 2], packed[4 * j + 3]);
+          if ((p.out_amax || p.out_q) && row_ok) {
+            // fused amax / cast act on the bf16-rounded values just staged
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              float v[4] = {bf16lo_to_f32(packed[2 * j]), bf16hi_to_f32(packed[2 * j]),
-                            bf16lo_to_f32(packed[2 * j + 1]), bf16hi_to_f32(packed[2 * j + 1])};
-              if (col0 + 4 * j < p.Nd) {
-                run_amax = fmaxf(run_amax, fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))));
+            for (int h = 0; h < 2; ++h) {  // two groups of 32 columns
+              uint32_t q[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const uint32_t w0 = packed[16 * h + 2 * j], w1 = packed[16 * h + 2 * j + 1];
+                float v[4] = {bf16lo_to_f32(w0), bf16hi_to_f32(w0), bf16lo_to_f32(w1), bf16hi_to_f32(w1)};
+                if (col0 + 32 * h + 4 * j < p.Nd)
+                  run_amax = fmaxf(run_amax, fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))));
+                if (p.out_q) {
+                  if (p.q_fmt == TWEO_E4M3)
+                    q[j] = quant4<TWEO_E4M3>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
+                                             __fmul_rn(v[3], qs));
+                  else
+                    q[j] = quant4<TWEO_E5M2>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
+                                             __fmul_rn(v[3], qs));
+                }
               }
               if (p.out_q) {
-                if (p.q_fmt == TWEO_E4M3)
-                  q[j] = quant4<TWEO_E4M3>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
-                                           __fmul_rn(v[3], qs));
-                else
-                  q[j] = quant4<TWEO_E5M2>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
-                                           __fmul_rn(v[3], qs));
+                uint8_t* qrow = p.out_q + (int64_t)row * p.ldq + col0 + 32 * h;
+                if (col0 + 32 * h < p.Nd) *reinterpret_cast<uint4*>(qrow) = make_uint4(q[0], q[1], q[2], q[3]);
+                if (col0 + 32 * h + 16 < p.Nd) *reinterpret_cast<uint4*>(qrow + 16) = make_uint4(q[4], q[5], q[6], q[7]);
               }
-            }
-            if (p.out_q) {
-              uint8_t* qrow = p.out_q + (int64_t)row * p.ldq + col0;
-              if (col0 < p.Nd) *reinterpret_cast<uint4*>(qrow) = make_uint4(q[0], q[1], q[2], q[3]);
-              if (col0 + 16 < p.Nd) *reinterpret_cast<uint4*>(qrow + 16) = make_uint4(q[4], q[5], q[6], q[7]);
             }
           }
         }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          if (OUT_F32 && p.accumulate) tma_reduce_add_2d(&tmap_d, col0, row0, buf);
+          else tma_store_2d(&tmap_d, col0, row0, buf);
+          bulk_commit();
+        }
+        ++it;
       }
       tc_fence_before();
       __syncwarp();
@@ -379,6 +421,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
+    if (lane == 0) bulk_wait_all();  // staged tiles must have left shared memory before the CTA exits
     if (p.out_amax) {
       run_amax = warp_max(run_amax);
       if (lane == 0 && run_amax > 0.0f)
@@ -429,6 +472,21 @@ bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, 
   return r == CUDA_SUCCESS;
 }
 
+// 2-D output tensor [rows, cols] of bf16 or fp32, boxes of {128 bytes, 32 rows}, 128-byte swizzle.
+bool make_out_map(CUtensorMap* map, void* base, int64_t cols, int64_t rows, int64_t ld, bool f32) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t esz = f32 ? 4 : 2;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * esz};
+  cuuint32_t box[2] = {(cuuint32_t)(128 / esz), 32u};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 uint32_t make_idesc(int fmt_a, int fmt_b, bool a_mn, bool b_mn, int n) {
   // [4,6) accumulator format (1 = fp32)   [7,10) A format   [10,13) B format (0 = E4M3, 1 = E5M2)
   // [15] A major (1 = MN)   [16] B major   [17,23) N >> 3   [24,29) M >> 4
@@ -443,10 +501,11 @@ uint32_t make_idesc(int fmt_a, int fmt_b, bool a_mn, bool b_mn, int n) {
   return d;
 }
 
-template <int BN, bool A_MN, bool B_MN, int STAGES>
-tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p, cudaStream_t st) {
-  constexpr size_t smem = (size_t)STAGES * (BM * BK + BN * BK) + 1024 + 256;
-  auto kern = gemm_fp8_kernel<BN, A_MN, B_MN, STAGES>;
+template <int BN, bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
+tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, GemmParams& p,
+                         cudaStream_t st) {
+  constexpr size_t smem = (size_t)STAGES * (BM * BK + BN * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
+  auto kern = gemm_fp8_kernel<BN, A_MN, B_MN, STAGES, OUT_F32>;
   static bool attr_done = false;  // per instantiation
   if (!attr_done) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -458,7 +517,7 @@ tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, GemmParam
   const int tiles = p.tiles_m * p.tiles_n;
   int grid = sm_count();
   if (grid > tiles) grid = tiles;
-  kern<<<grid, kThreads, smem, st>>>(ma, mb, p);
+  kern<<<grid, kThreads, smem, st>>>(ma, mb, md, p);
   count_launch();
   return check_launch("gemm_fp8_kernel");
 }
@@ -484,8 +543,12 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
   const int BN = Nd > 128 ? 256 : 128;
   p.idesc = make_idesc(A.fmt, B.fmt, A.mn_major, B.mn_major, BN);
 
-  CUtensorMap ma, mb;
-  bool ok;
+  CUtensorMap ma, mb, md;
+  bool ok = make_out_map(&md, p.d, Nd, Md, p.ldd, p.out_f32 != 0);
+  if (!ok) {
+    cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled (output)");
+    return TWEO_ERR_CUDA;
+  }
   if (A.mn_major) ok = make_map(&ma, A.ptr, Md, Kc, A.ld, BK);   // [Kc, Md]: box 128 (Md) x BK rows
   else ok = make_map(&ma, A.ptr, Kc, Md, A.ld, BM);              // [Md, Kc]: box 128 (Kc) x BM rows
   if (B.mn_major) ok = ok && make_map(&mb, B.ptr, Nd, Kc, B.ld, BK);
@@ -498,8 +561,11 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
     zero_float_kernel<<<1, 1, 0, st>>>(p.out_amax);
     count_launch();
   }
-#define TWEO_DISPATCH(AMN, BMN)                                                        \
-  (BN == 256 ? launch_cfg<256, AMN, BMN, 4>(ma, mb, p, st) : launch_cfg<128, AMN, BMN, 6>(ma, mb, p, st))
+#define TWEO_DISPATCH(AMN, BMN)                                                                   \
+  (p.out_f32 ? (BN == 256 ? launch_cfg<256, AMN, BMN, 4, true>(ma, mb, md, p, st)                 \
+                          : launch_cfg<128, AMN, BMN, 6, true>(ma, mb, md, p, st))                \
+             : (BN == 256 ? launch_cfg<256, AMN, BMN, 4, false>(ma, mb, md, p, st)                \
+                          : launch_cfg<128, AMN, BMN, 6, false>(ma, mb, md, p, st)))
   if (!A.mn_major && !B.mn_major) return TWEO_DISPATCH(false, false);
   if (!A.mn_major && B.mn_major) return TWEO_DISPATCH(false, true);
   if (A.mn_major && B.mn_major) return TWEO_DISPATCH(true, true);
