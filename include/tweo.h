@@ -124,6 +124,11 @@ TWEO_API tweo_status_t tweo_quantize_per_tensor(const uint16_t* x, int64_t n, in
  *   xq [M,K] codes (fmt_x), wq [N,K] codes (fmt_w), y [M,N] bf16.
  *   Shapes: M >= 1 (ragged M is zero-filled by the loader); N % 16 == 0,
  *   K % 16 == 0.  epi may be NULL.
+ *   ws is optional for the three linear calls (NULL, 0 is valid).  With a zero-
+ *   initialised workspace of tweo_workspace_bytes(TWEO_OP_LINEAR_*) bytes the
+ *   kernel may split tiles along the contraction when whole tiles would leave SMs
+ *   idle (few output tiles, long contraction); partial sums are added in a fixed
+ *   order, so results stay bit-reproducible.
  */
 TWEO_API tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const uint8_t* wq, int64_t ldw,
                                   const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy,

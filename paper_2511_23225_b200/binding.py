@@ -185,8 +185,12 @@ def _epilogue(amax, q, q_fmt, q_scale):
     return C.byref(e)
 
 
+def _ws(ws):
+    return (None, 0) if ws is None else (_dev(ws, torch.uint8, "ws"), ws.numel())
+
+
 def fp8_linear_fwd(xq, wq, sx_inv, sw_inv, fmt_x=E4M3, fmt_w=E4M3, y=None, out_amax=None, out_q=None,
-                   q_fmt=E4M3, q_scale=None) -> torch.Tensor:
+                   q_fmt=E4M3, q_scale=None, ws=None) -> torch.Tensor:
     """tweo_fp8_linear_fwd: Y[M,N] = Xq[M,K] . Wq[N,K]^T * sx_inv * sw_inv -> bf16."""
     M, K = xq.shape
     N, K2 = wq.shape
@@ -197,13 +201,13 @@ def fp8_linear_fwd(xq, wq, sx_inv, sw_inv, fmt_x=E4M3, fmt_w=E4M3, y=None, out_a
     _check(lib().tweo_fp8_linear_fwd(_dev(xq, U8, "xq"), _rows(xq, "xq"), _dev(wq, U8, "wq"), _rows(wq, "wq"),
                                      _dev(sx_inv, torch.float32), _dev(sw_inv, torch.float32),
                                      _dev(y, torch.bfloat16, "y"), _rows(y, "y"), M, N, K, fmt_x, fmt_w,
-                                     _epilogue(out_amax, out_q, q_fmt, q_scale), None, 0, _stream()),
+                                     _epilogue(out_amax, out_q, q_fmt, q_scale), *_ws(ws), _stream()),
            "tweo_fp8_linear_fwd")
     return y
 
 
 def fp8_linear_bwd_dgrad(dyq, wq, sdy_inv, sw_inv, fmt_dy=E5M2, fmt_w=E4M3, dx=None, out_amax=None, out_q=None,
-                         q_fmt=E5M2, q_scale=None) -> torch.Tensor:
+                         q_fmt=E5M2, q_scale=None, ws=None) -> torch.Tensor:
     """tweo_fp8_linear_bwd_dgrad: dX[M,K] = dYq[M,N] . Wq[N,K] * sdy_inv * sw_inv -> bf16."""
     M, N = dyq.shape
     N2, K = wq.shape
@@ -215,12 +219,12 @@ def fp8_linear_bwd_dgrad(dyq, wq, sdy_inv, sw_inv, fmt_dy=E5M2, fmt_w=E4M3, dx=N
                                            _rows(wq, "wq"), fmt_w, _dev(sdy_inv, torch.float32),
                                            _dev(sw_inv, torch.float32), _dev(dx, torch.bfloat16, "dx"),
                                            _rows(dx, "dx"), M, N, K, _epilogue(out_amax, out_q, q_fmt, q_scale),
-                                           None, 0, _stream()), "tweo_fp8_linear_bwd_dgrad")
+                                           *_ws(ws), _stream()), "tweo_fp8_linear_bwd_dgrad")
     return dx
 
 
 def fp8_linear_bwd_wgrad(xq, dyq, sx_inv, sdy_inv, fmt_x=E4M3, fmt_dy=E5M2, dw=None, dw_dtype=BF16,
-                         accumulate=False) -> torch.Tensor:
+                         accumulate=False, ws=None) -> torch.Tensor:
     """tweo_fp8_linear_bwd_wgrad: dW[N,K] = dYq[M,N]^T . Xq[M,K] * sx_inv * sdy_inv."""
     M, K = xq.shape
     M2, N = dyq.shape
@@ -234,7 +238,7 @@ def fp8_linear_bwd_wgrad(xq, dyq, sx_inv, sdy_inv, fmt_x=E4M3, fmt_dy=E5M2, dw=N
     _check(lib().tweo_fp8_linear_bwd_wgrad(_dev(xq, U8, "xq"), _rows(xq, "xq"), fmt_x, _dev(dyq, U8, "dyq"),
                                            _rows(dyq, "dyq"), fmt_dy, _dev(sx_inv, torch.float32),
                                            _dev(sdy_inv, torch.float32), _dev(dw, tdt, "dw"), _rows(dw, "dw"),
-                                           dw_dtype, 1 if accumulate else 0, M, N, K, None, 0, _stream()),
+                                           dw_dtype, 1 if accumulate else 0, M, N, K, *_ws(ws), _stream()),
            "tweo_fp8_linear_bwd_wgrad")
     return dw
 

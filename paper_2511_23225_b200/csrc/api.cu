@@ -64,18 +64,23 @@ int32_t tweo_version(void) { return 100; }
 uint64_t tweo_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 size_t tweo_workspace_bytes(int32_t op, int64_t M, int64_t N, int64_t K) {
+  const size_t sms = (size_t)tweo_detail::sm_count();
+  const size_t stream_k_bytes = sms * 128 * 256 * sizeof(float) + ((sms * 16 + 255) & ~(size_t)255) + 256;
   switch (op) {
     case TWEO_OP_LOSS: {
       int L = (int)(N < 1 ? 1 : N);
       return 256 + sizeof(double) * (size_t)L * (size_t)tweo_detail::loss_blocks_per_tensor(M, L);
     }
+    case TWEO_OP_LINEAR_FWD:
+    case TWEO_OP_LINEAR_DGRAD:
+    case TWEO_OP_LINEAR_WGRAD:
+      // optional: lets the GEMM split tiles along the contraction (one 128x256 fp32 slot per SM + flags)
+      return stream_k_bytes;
     case TWEO_OP_W8A8: {
-      // codes of the activations (bf16 input is cast inside) + split-K partial sums for small M
+      // scalars + codes of the activations (a bf16 input is cast inside) + the GEMM's stream-K area
       size_t codes = (size_t)(M < 0 ? 0 : M) * (size_t)(K < 0 ? 0 : K);
       codes = (codes + 255) & ~(size_t)255;
-      size_t partial = 0;
-      if (M > 0 && M <= 64) partial = (size_t)64 * (size_t)N * sizeof(float) * 16 + 4096;
-      return 256 + codes + partial;
+      return 256 + codes + stream_k_bytes;
     }
     default:
       return 0;

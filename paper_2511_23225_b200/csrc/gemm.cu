@@ -18,11 +18,24 @@
 // them to a TMA store, so global writes are full lines and ragged edges are clipped by
 // the hardware).  The kernel is persistent (grid = #SMs, static tile striding) with a
 // ring of shared-memory stages and two accumulators in tensor memory, so the epilogue of
-// tile i overlaps the main loop of tile i+1.  Every mbarrier wait is bounded: on expiry
-// the CTA records TWEO_ERR_TIMEOUT in a device status word, drains and exits.
+// tile i overlaps the main loop of tile i+1.
+//
+// Scheduling.  Tiles are dealt round-robin to the CTAs.  When that would leave SMs idle
+// (fewer tiles than SMs, or a ragged last wave) and the contraction is long, the last
+// tiles are instead cut along the contraction ("stream-K"): their (tile, k-block) units
+// are split evenly over all CTAs.  A CTA whose share starts in the middle of a tile writes
+// its raw fp32 accumulator to a workspace slot and raises a flag; the CTA that owns the
+// tile's first k-block adds the other shares in CTA order (fixed order => reproducible)
+// and runs the epilogue.  Such a share is always the FIRST thing a CTA does and an owner's
+// wait is the LAST step of its stream-K work, so waits cannot form a cycle.
+//
+// Every wait (mbarrier or flag) is bounded: on expiry the CTA records TWEO_ERR_TIMEOUT in
+// a device status word, drains and exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <atomic>
+#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -54,7 +67,55 @@ struct GemmParams {
   int32_t q_fmt;
   const float* q_scale;
   uint32_t idesc;
+  // stream-K: tiles [0, sk_tiles) are split along the contraction, the rest dealt whole
+  int32_t sk_tiles;
+  float* sk_partials;   // [grid][BM*BN] raw accumulators of shares that do not own their tile
+  uint32_t* sk_flags;   // [grid][4] per epilogue warp: == epoch once the share is written
+  uint32_t epoch;
 };
+
+// The work list of one CTA, identical in the three roles (producer, MMA, epilogue).
+struct Sched {
+  int64_t u, u_end;   // stream-K units (tile * k_blocks + k-block) still to do
+  int dp_tile, num_tiles, k_blocks, grid;
+  __device__ Sched(const GemmParams& p, int cta, int grid_)
+      : dp_tile(p.sk_tiles + cta), num_tiles(p.tiles_m * p.tiles_n), k_blocks(p.k_blocks), grid(grid_) {
+    const int64_t total = (int64_t)p.sk_tiles * p.k_blocks;
+    u = total * cta / grid_;
+    u_end = total * (cta + 1) / grid_;
+  }
+  // first unit of CTA j's stream-K share
+  __device__ static int64_t share_begin(const GemmParams& p, int j, int grid_) {
+    return (int64_t)p.sk_tiles * p.k_blocks * j / grid_;
+  }
+  __device__ bool next(int& tile, int& kb0, int& kb1) {
+    if (u < u_end) {
+      tile = (int)(u / k_blocks);
+      kb0 = (int)(u - (int64_t)tile * k_blocks);
+      const int64_t len = min((int64_t)(k_blocks - kb0), u_end - u);
+      kb1 = kb0 + (int)len;
+      u += len;
+      return true;
+    }
+    if (dp_tile < num_tiles) {
+      tile = dp_tile;
+      kb0 = 0;
+      kb1 = k_blocks;
+      dp_tile += grid;
+      return true;
+    }
+    return false;
+  }
+};
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* ptr) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_u32(uint32_t* ptr, uint32_t v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
+}
 
 // ----------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -250,18 +311,18 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int num_tiles = p.tiles_m * p.tiles_n;
-
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+      Sched sched(p, blockIdx.x, gridDim.x);
+      int tile, kb0, kb1;
+      while (ok && sched.next(tile, kb0, kb1)) {
         const int m0 = (tile % p.tiles_m) * BM;
         const int n0 = (tile / p.tiles_m) * BN;
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t fb = full_bar(stage);
           mbar_expect_tx(fb, STAGE_BYTES);
@@ -299,11 +360,13 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+      Sched sched(p, blockIdx.x, gridDim.x);
+      int tile, kb0, kb1;
+      while (ok && sched.next(tile, kb0, kb1)) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
@@ -313,7 +376,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             // K-major: step 32 bytes inside the swizzle span; MN-major: step 32 rows of 128 B
             const uint64_t adesc = make_smem_desc(sa + (A_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
             const uint64_t bdesc = make_smem_desc(sb + (B_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
-            umma_f8(d_tmem, adesc, bdesc, p.idesc, (uint32_t)((kb | k) != 0));
+            umma_f8(d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != kb0 || k != 0));
           }
           umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -338,11 +401,62 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+    Sched sched(p, blockIdx.x, gridDim.x);
+    int tile, kb0, kb1;
+    while (ok && sched.next(tile, kb0, kb1)) {
       const int m0 = (tile % p.tiles_m) * BM;
       const int n0 = (tile / p.tiles_m) * BN;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
+      const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
+      if (kb0 > 0) {
+        // A share that does not own its tile: park the raw accumulator, raise the flag.
+        float* slot = p.sk_partials + (size_t)blockIdx.x * (BM * BN);
+#pragma unroll 1
+        for (int g = 0; g < BN / 32; ++g) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + tlane + (uint32_t)(acc * BN + g * 32), r);
+          tmem_ld_wait();
+          float* dst = slot + ((g * 4 + quarter) * 32) * 32 + lane;
+#pragma unroll
+          for (int k = 0; k < 32; ++k) __stcg(dst + k * 32, __uint_as_float(r[k]));
+        }
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) st_release_u32(p.sk_flags + blockIdx.x * 4 + quarter, p.epoch);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+        continue;
+      }
+      int n_contrib = 0;
+      if (kb1 < p.k_blocks) {
+        // Owner of a tile whose later k-blocks went to the following CTAs: wait for them.
+        const int64_t tile_end = (int64_t)(tile + 1) * p.k_blocks;
+        for (int j = blockIdx.x + 1; j < (int)gridDim.x && Sched::share_begin(p, j, gridDim.x) < tile_end; ++j) {
+          const uint32_t* flag = p.sk_flags + j * 4 + quarter;
+          if (ld_acquire_u32(flag) != p.epoch) {
+            const uint64_t t0 = globaltimer_ns();
+            for (uint32_t spin = 1; ld_acquire_u32(flag) != p.epoch; ++spin) {
+              if ((spin & 0xFFu) == 0) {
+                if (*abort_flag) { ok = false; break; }
+                if (globaltimer_ns() - t0 > kWaitLimitNs) {
+                  *abort_flag = 1;
+                  atomicExch(&g_device_status, (unsigned int)TWEO_ERR_TIMEOUT);
+                  ok = false;
+                  break;
+                }
+              }
+            }
+          }
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          ++n_contrib;
+        }
+        if (!ok) break;
+      }
       const int row0 = m0 + quarter * 32;
       const int row = row0 + lane;
       const bool row_ok = row < p.Md;
@@ -351,10 +465,20 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         const int col0 = n0 + c * CH;
         if (col0 >= p.Nd) break;  // uniform across the warp
         uint32_t r[CH];
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c * CH);
+        const uint32_t taddr = tmem_base + tlane + (uint32_t)(acc * BN + c * CH);
         tmem_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
         if (!OUT_F32) tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[CH - 32]));
         tmem_ld_wait();
+        for (int jc = 0; jc < n_contrib; ++jc) {  // add the other shares, in CTA order
+          const float* part = p.sk_partials + (size_t)(blockIdx.x + 1 + jc) * (BM * BN);
+#pragma unroll
+          for (int h = 0; h < CH / 32; ++h) {
+            const float* src = part + (((c * (CH / 32) + h) * 4 + quarter) * 32) * 32 + lane;
+#pragma unroll
+            for (int k = 0; k < 32; ++k)
+              r[h * 32 + k] = __float_as_uint(__uint_as_float(r[h * 32 + k]) + __ldcg(src + k * 32));
+          }
+        }
         if (row0 >= p.Md) continue;  // whole warp past the ragged edge (uniform)
         const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
         // the store issued two chunks ago must have finished reading this buffer
@@ -437,6 +561,294 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   }
 }
 
+
+// ----------------------------------------------------------------- CTA-pair kernel
+// Two CTAs of a cluster (adjacent SMs) compute one 256 x 256 tile with tcgen05
+// cta_group::2 instructions: each CTA stages its own 128 rows of A and only HALF of the
+// B tile (128 of the 256 output columns), the pair's tensor cores read both halves, and
+// each CTA's tensor memory receives the accumulator of its own 128 rows.  Per SM this
+// moves 32 KB of operands per 128-deep contraction block instead of 48 KB, which is what
+// lifts the kernel off the shared-memory fill limit.  Roles per CTA are those of the
+// single-CTA kernel; only CTA 0 (the leader) issues MMAs.  Barriers:
+//   full[s]    leader only : leader's producer arrives (+ expected bytes of BOTH CTAs' loads)
+//   empty[s]   each CTA    : leader's MMA thread commits to its own and to the peer's
+//   tfull[a]   each CTA    : same, once a tile's accumulator is complete
+//   tempty[a]  leader only : 4 epilogue warps of each CTA arrive (the peer's remotely)
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1,
+                                                 uint32_t leader_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(leader_bar)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_f8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives (at the given cluster-window address) once all MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint32_t cluster_bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar)
+               : "memory");
+}
+
+template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                     const __grid_constant__ CUtensorMap tmap_d, const GemmParams p) {
+  constexpr int BN = 256;                 // tile columns of the pair
+  constexpr uint32_t A_BYTES = BM * BK;   // this CTA's 128 rows of A
+  constexpr uint32_t B_BYTES = 128 * BK;  // this CTA's 128 of the 256 columns of B
+  constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr uint32_t TMEM_COLS = 512;
+
+  extern __shared__ uint8_t smem_dyn[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  constexpr uint32_t EPI_BUF = 32 * 128;
+  constexpr uint32_t EPI_BYTES = 4 * 2 * EPI_BUF;
+  uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 8);  // four epilogue warps of each CTA of the pair
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // both CTAs' barriers are initialised before anyone signals across
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int num_tiles = p.tiles_m * p.tiles_n;
+  const int pair = blockIdx.x >> 1;
+  const int num_pairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+        const int m0 = (tile % p.tiles_m) * (2 * BM) + (int)rank * BM;  // this CTA's rows
+        const int n0 = (tile / p.tiles_m) * BN + (int)rank * 128;       // this CTA's half of B
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
+          const uint32_t fb = map_to_cta(full_bar(stage), 0);
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+          const int k0 = kb * BK;
+          if (A_MN) tma_load_2d_pair(sa, &tmap_a, m0, k0, fb);
+          else tma_load_2d_pair(sa, &tmap_a, k0, m0, fb);
+          if (B_MN) tma_load_2d_pair(sb, &tmap_b, n0, k0, fb);
+          else tma_load_2d_pair(sb, &tmap_b, k0, n0, fb);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && leader) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t adesc = make_smem_desc(sa + (A_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
+            const uint64_t bdesc = make_smem_desc(sb + (B_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
+            umma_f8_pair(d_tmem, adesc, bdesc, p.idesc, (uint32_t)((kb | k) != 0));
+          }
+          umma_commit_pair(map_to_cta(empty_bar(stage), 0));  // frees the stage in both CTAs
+          umma_commit_pair(map_to_cta(empty_bar(stage), 1));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit_pair(map_to_cta(tfull_bar(acc), 0));      // accumulator complete, both CTAs
+        umma_commit_pair(map_to_cta(tfull_bar(acc), 1));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    const int quarter = warp & 3;
+    const float alpha = __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
+    const float qs = p.out_q ? __ldg(p.q_scale) : 0.0f;
+    constexpr int CH = OUT_F32 ? 32 : 64;
+    const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
+    const uint32_t row_off = (uint32_t)lane * 128u;
+    const uint32_t swz = (uint32_t)(lane & 7);
+    const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
+    uint32_t it = 0;
+    float run_amax = 0.0f;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+      const int m0 = (tile % p.tiles_m) * (2 * BM) + (int)rank * BM;
+      const int n0 = (tile / p.tiles_m) * BN;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row0 = m0 + quarter * 32;
+      const int row = row0 + lane;
+      const bool row_ok = row < p.Md;
+#pragma unroll 1
+      for (int c = 0; c < BN / CH; ++c) {
+        const int col0 = n0 + c * CH;
+        if (col0 >= p.Nd) break;
+        uint32_t r[CH];
+        const uint32_t taddr = tmem_base + tlane + (uint32_t)(acc * BN + c * CH);
+        tmem_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+        if (!OUT_F32) tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[CH - 32]));
+        tmem_ld_wait();
+        if (row0 >= p.Md) continue;
+        const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
+        if (lane == 0) bulk_wait_read<1>();
+        __syncwarp();
+        if (OUT_F32) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j]), alpha)),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 1]), alpha)),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 2]), alpha)),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 3]), alpha)));
+        } else {
+          uint32_t packed[CH / 2];
+#pragma unroll
+          for (int j = 0; j < CH / 2; ++j)
+            packed[j] = f32x2_to_bf16x2(__fmul_rn(__uint_as_float(r[2 * j]), alpha),
+                                        __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha));
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1],
+                         packed[4 * j + 2], packed[4 * j + 3]);
+          if ((p.out_amax || p.out_q) && row_ok) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              uint32_t q[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const uint32_t w0 = packed[16 * h + 2 * j], w1 = packed[16 * h + 2 * j + 1];
+                float v[4] = {bf16lo_to_f32(w0), bf16hi_to_f32(w0), bf16lo_to_f32(w1), bf16hi_to_f32(w1)};
+                if (col0 + 32 * h + 4 * j < p.Nd)
+                  run_amax = fmaxf(run_amax, fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))));
+                if (p.out_q) {
+                  if (p.q_fmt == TWEO_E4M3)
+                    q[j] = quant4<TWEO_E4M3>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
+                                             __fmul_rn(v[3], qs));
+                  else
+                    q[j] = quant4<TWEO_E5M2>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
+                                             __fmul_rn(v[3], qs));
+                }
+              }
+              if (p.out_q) {
+                uint8_t* qrow = p.out_q + (int64_t)row * p.ldq + col0 + 32 * h;
+                if (col0 + 32 * h < p.Nd) *reinterpret_cast<uint4*>(qrow) = make_uint4(q[0], q[1], q[2], q[3]);
+                if (col0 + 32 * h + 16 < p.Nd) *reinterpret_cast<uint4*>(qrow + 16) = make_uint4(q[4], q[5], q[6], q[7]);
+              }
+            }
+          }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          if (OUT_F32 && p.accumulate) tma_reduce_add_2d(&tmap_d, col0, row0, buf);
+          else tma_store_2d(&tmap_d, col0, row0, buf);
+          bulk_commit();
+        }
+        ++it;
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's barrier
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+    if (lane == 0) bulk_wait_all();
+    if (p.out_amax) {
+      run_amax = warp_max(run_amax);
+      if (lane == 0 && run_amax > 0.0f)
+        atomicMax(reinterpret_cast<unsigned int*>(p.out_amax), __float_as_uint(run_amax));
+    }
+  }
+
+  // Neither CTA may leave (or free tensor memory) while the other can still signal its
+  // barriers or have MMAs reading its shared memory.
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
 __global__ void zero_float_kernel(float* p) { *p = 0.0f; }
 
 // ----------------------------------------------------------------- host side
@@ -487,7 +899,7 @@ bool make_out_map(CUtensorMap* map, void* base, int64_t cols, int64_t rows, int6
   return r == CUDA_SUCCESS;
 }
 
-uint32_t make_idesc(int fmt_a, int fmt_b, bool a_mn, bool b_mn, int n) {
+uint32_t make_idesc(int fmt_a, int fmt_b, bool a_mn, bool b_mn, int n, int m = BM) {
   // [4,6) accumulator format (1 = fp32)   [7,10) A format   [10,13) B format (0 = E4M3, 1 = E5M2)
   // [15] A major (1 = MN)   [16] B major   [17,23) N >> 3   [24,29) M >> 4
   uint32_t d = 0;
@@ -497,13 +909,17 @@ uint32_t make_idesc(int fmt_a, int fmt_b, bool a_mn, bool b_mn, int n) {
   d |= (uint32_t)(a_mn ? 1 : 0) << 15;
   d |= (uint32_t)(b_mn ? 1 : 0) << 16;
   d |= (uint32_t)(n >> 3) << 17;
-  d |= (uint32_t)(BM >> 4) << 24;
+  d |= (uint32_t)(m >> 4) << 24;
   return d;
 }
 
+std::atomic<uint32_t> g_sk_epoch{0};
+// TWEO_GEMM_NO_PAIR=1 in the environment keeps every GEMM on the single-CTA kernel (A/B timing).
+const bool g_disable_pair = [] { const char* e = getenv("TWEO_GEMM_NO_PAIR"); return e && e[0] == '1'; }();
+
 template <int BN, bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
 tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, GemmParams& p,
-                         cudaStream_t st) {
+                         void* ws, size_t ws_bytes, cudaStream_t st) {
   constexpr size_t smem = (size_t)STAGES * (BM * BK + BN * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
   auto kern = gemm_fp8_kernel<BN, A_MN, B_MN, STAGES, OUT_F32>;
   static bool attr_done = false;  // per instantiation
@@ -515,11 +931,65 @@ tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
   p.tiles_n = (p.Nd + BN - 1) / BN;
   p.k_blocks = (p.Kc + BK - 1) / BK;
   const int tiles = p.tiles_m * p.tiles_n;
-  int grid = sm_count();
-  if (grid > tiles) grid = tiles;
+  const int sms = sm_count();
+  int grid = sms < tiles ? sms : tiles;
+  p.sk_tiles = 0;
+  p.sk_partials = nullptr;
+  p.sk_flags = nullptr;
+  p.epoch = 0;
+  // Stream-K when whole-tile dealing would idle more than ~15 % of the SM-time and the
+  // contraction is long enough to pay for the fix-up (a 128 x BN fp32 round trip through L2).
+  const size_t sk_need = (size_t)sms * BM * BN * sizeof(float) + (size_t)sms * 16 + 256;
+  const int waves = (tiles + sms - 1) / sms;
+  if (ws && ws_bytes >= sk_need && aligned16(ws) && p.k_blocks >= 12 &&
+      (double)tiles < 0.85 * (double)waves * sms) {
+    const int full = tiles / sms;
+    p.sk_tiles = full == 0 ? tiles : tiles - (full - 1) * sms;
+    grid = sms;
+    if ((int64_t)p.sk_tiles * p.k_blocks < grid) grid = (int)((int64_t)p.sk_tiles * p.k_blocks);
+    p.sk_flags = reinterpret_cast<uint32_t*>(ws);
+    p.sk_partials = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + (((size_t)sms * 16 + 255) & ~(size_t)255));
+    p.epoch = g_sk_epoch.fetch_add(1, std::memory_order_relaxed) + 1;
+  }
   kern<<<grid, kThreads, smem, st>>>(ma, mb, md, p);
   count_launch();
   return check_launch("gemm_fp8_kernel");
+}
+
+template <bool A_MN, bool B_MN, bool OUT_F32>
+tweo_status_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, GemmParams& p,
+                          cudaStream_t st) {
+  constexpr int STAGES = 6;
+  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
+  auto kern = gemm_fp8_pair_kernel<A_MN, B_MN, STAGES, OUT_F32>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 0));
+    attr_done = true;
+  }
+  p.tiles_m = (p.Md + 2 * BM - 1) / (2 * BM);
+  p.tiles_n = (p.Nd + 255) / 256;
+  p.k_blocks = (p.Kc + BK - 1) / BK;
+  p.sk_tiles = 0;
+  const int tiles = p.tiles_m * p.tiles_n;
+  int pairs = sm_count() / 2;
+  if (pairs > tiles) pairs = tiles;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, p));
+  count_launch();
+  return check_launch("gemm_fp8_pair_kernel");
 }
 
 struct Operand {
@@ -531,7 +1001,7 @@ struct Operand {
 
 // D[Md,Nd] = A . B, see the header comment for how the three linear products map here.
 tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t Nd, int64_t Kc, GemmParams p,
-                       cudaStream_t st) {
+                       void* ws, size_t ws_bytes, cudaStream_t st) {
   if (Md < 1 || Nd < 1 || Kc < 1) return TWEO_ERR_INVALID_ARG;
   if (Md > INT32_MAX || Nd > INT32_MAX || Kc > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
   if (!aligned16(A.ptr) || !aligned16(B.ptr) || !aligned16(p.d) || (A.ld & 15) || (B.ld & 15))
@@ -541,7 +1011,10 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
   p.Nd = (int32_t)Nd;
   p.Kc = (int32_t)Kc;
   const int BN = Nd > 128 ? 256 : 128;
-  p.idesc = make_idesc(A.fmt, B.fmt, A.mn_major, B.mn_major, BN);
+  // CTA pairs (256 x 256 tiles) whenever the output has more than one 128-row block and is wide enough
+  const bool use_pair = Md > 128 && Nd > 128 && !g_disable_pair;
+  p.idesc = use_pair ? make_idesc(A.fmt, B.fmt, A.mn_major, B.mn_major, 256, 256)
+                     : make_idesc(A.fmt, B.fmt, A.mn_major, B.mn_major, BN);
 
   CUtensorMap ma, mb, md;
   bool ok = make_out_map(&md, p.d, Nd, Md, p.ldd, p.out_f32 != 0);
@@ -552,7 +1025,7 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
   if (A.mn_major) ok = make_map(&ma, A.ptr, Md, Kc, A.ld, BK);   // [Kc, Md]: box 128 (Md) x BK rows
   else ok = make_map(&ma, A.ptr, Kc, Md, A.ld, BM);              // [Md, Kc]: box 128 (Kc) x BM rows
   if (B.mn_major) ok = ok && make_map(&mb, B.ptr, Nd, Kc, B.ld, BK);
-  else ok = ok && make_map(&mb, B.ptr, Kc, Nd, B.ld, BN);
+  else ok = ok && make_map(&mb, B.ptr, Kc, Nd, B.ld, use_pair ? 128 : BN);  // a pair CTA loads half of B
   if (!ok) {
     cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
     return TWEO_ERR_CUDA;
@@ -561,11 +1034,19 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
     zero_float_kernel<<<1, 1, 0, st>>>(p.out_amax);
     count_launch();
   }
+  if (use_pair) {
+#define TWEO_PAIR(AMN, BMN) (p.out_f32 ? launch_pair<AMN, BMN, true>(ma, mb, md, p, st) : launch_pair<AMN, BMN, false>(ma, mb, md, p, st))
+    if (!A.mn_major && !B.mn_major) return TWEO_PAIR(false, false);
+    if (!A.mn_major && B.mn_major) return TWEO_PAIR(false, true);
+    if (A.mn_major && B.mn_major) return TWEO_PAIR(true, true);
+    return TWEO_ERR_INVALID_ARG;
+#undef TWEO_PAIR
+  }
 #define TWEO_DISPATCH(AMN, BMN)                                                                   \
-  (p.out_f32 ? (BN == 256 ? launch_cfg<256, AMN, BMN, 4, true>(ma, mb, md, p, st)                 \
-                          : launch_cfg<128, AMN, BMN, 6, true>(ma, mb, md, p, st))                \
-             : (BN == 256 ? launch_cfg<256, AMN, BMN, 4, false>(ma, mb, md, p, st)                \
-                          : launch_cfg<128, AMN, BMN, 6, false>(ma, mb, md, p, st)))
+  (p.out_f32 ? (BN == 256 ? launch_cfg<256, AMN, BMN, 4, true>(ma, mb, md, p, ws, ws_bytes, st)                 \
+                          : launch_cfg<128, AMN, BMN, 6, true>(ma, mb, md, p, ws, ws_bytes, st))                \
+             : (BN == 256 ? launch_cfg<256, AMN, BMN, 4, false>(ma, mb, md, p, ws, ws_bytes, st)                \
+                          : launch_cfg<128, AMN, BMN, 6, false>(ma, mb, md, p, ws, ws_bytes, st)))
   if (!A.mn_major && !B.mn_major) return TWEO_DISPATCH(false, false);
   if (!A.mn_major && B.mn_major) return TWEO_DISPATCH(false, true);
   if (A.mn_major && B.mn_major) return TWEO_DISPATCH(true, true);
@@ -609,7 +1090,8 @@ tweo_status_t read_and_clear_device_status(cudaStream_t stream) {
 // Used by the static W8A8 entry point: forward product on already-cast activations.
 tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
                              const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
-                             int64_t N, int64_t K, const tweo_epilogue_t* epi, cudaStream_t st) {
+                             int64_t N, int64_t K, const tweo_epilogue_t* epi, void* ws, size_t ws_bytes,
+                             cudaStream_t st) {
   GemmParams p{};
   p.d = y;
   p.ldd = ldy;
@@ -617,7 +1099,7 @@ tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const ui
   p.sb_inv = sw_inv;
   tweo_status_t s = fill_epilogue(p, epi);
   if (s != TWEO_OK) return s;
-  return run_gemm(Operand{xq, ldx, fmt_x, false}, Operand{wq, ldw, fmt_w, false}, M, N, K, p, st);
+  return run_gemm(Operand{xq, ldx, fmt_x, false}, Operand{wq, ldw, fmt_w, false}, M, N, K, p, ws, ws_bytes, st);
 }
 
 }  // namespace tweo_detail
@@ -628,21 +1110,17 @@ tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const uint8_t*
                                   const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
                                   int64_t N, int64_t K, int32_t fmt_x, int32_t fmt_w, const tweo_epilogue_t* epi,
                                   void* ws, size_t ws_bytes, void* stream) {
-  (void)ws;
-  (void)ws_bytes;
   if (!xq || !wq || !sx_inv || !sw_inv || !y || !fmt_ok(fmt_x) || !fmt_ok(fmt_w)) return TWEO_ERR_INVALID_ARG;
   if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
   if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
-  return tweo_detail::gemm_fwd_codes(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, y, ldy, M, N, K, epi,
-                                     (cudaStream_t)stream);
+  return tweo_detail::gemm_fwd_codes(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, y, ldy, M, N, K, epi, ws,
+                                     ws_bytes, (cudaStream_t)stream);
 }
 
 tweo_status_t tweo_fp8_linear_bwd_dgrad(const uint8_t* dyq, int64_t lddy, int32_t fmt_dy, const uint8_t* wq,
                                         int64_t ldw, int32_t fmt_w, const float* sdy_inv, const float* sw_inv,
                                         uint16_t* dx, int64_t lddx, int64_t M, int64_t N, int64_t K,
                                         const tweo_epilogue_t* epi, void* ws, size_t ws_bytes, void* stream) {
-  (void)ws;
-  (void)ws_bytes;
   if (!dyq || !wq || !sdy_inv || !sw_inv || !dx || !fmt_ok(fmt_dy) || !fmt_ok(fmt_w)) return TWEO_ERR_INVALID_ARG;
   if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
   if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
@@ -654,7 +1132,7 @@ tweo_status_t tweo_fp8_linear_bwd_dgrad(const uint8_t* dyq, int64_t lddy, int32_
   tweo_status_t s = fill_epilogue(p, epi);
   if (s != TWEO_OK) return s;
   // dX[M,K] = dYq[M,N] . Wq[N,K]: contraction over N; Wq is stored [N(contraction), K(out)] = MN-major
-  return run_gemm(Operand{dyq, lddy, fmt_dy, false}, Operand{wq, ldw, fmt_w, true}, M, K, N, p,
+  return run_gemm(Operand{dyq, lddy, fmt_dy, false}, Operand{wq, ldw, fmt_w, true}, M, K, N, p, ws, ws_bytes,
                   (cudaStream_t)stream);
 }
 
@@ -662,8 +1140,6 @@ tweo_status_t tweo_fp8_linear_bwd_wgrad(const uint8_t* xq, int64_t ldx, int32_t 
                                         int64_t lddy, int32_t fmt_dy, const float* sx_inv, const float* sdy_inv,
                                         void* dw, int64_t lddw, int32_t dw_dtype, int32_t accumulate, int64_t M,
                                         int64_t N, int64_t K, void* ws, size_t ws_bytes, void* stream) {
-  (void)ws;
-  (void)ws_bytes;
   if (!xq || !dyq || !sx_inv || !sdy_inv || !dw || !fmt_ok(fmt_x) || !fmt_ok(fmt_dy)) return TWEO_ERR_INVALID_ARG;
   if (dw_dtype != TWEO_BF16 && dw_dtype != TWEO_F32) return TWEO_ERR_INVALID_ARG;
   if (accumulate && dw_dtype != TWEO_F32) return TWEO_ERR_INVALID_ARG;
@@ -678,7 +1154,7 @@ tweo_status_t tweo_fp8_linear_bwd_wgrad(const uint8_t* xq, int64_t ldx, int32_t 
   p.accumulate = accumulate ? 1 : 0;
   fill_epilogue(p, nullptr);
   // dW[N,K] = dYq[M,N]^T . Xq[M,K]: contraction over M; both operands stored [M(contraction), out]
-  return run_gemm(Operand{dyq, lddy, fmt_dy, true}, Operand{xq, ldx, fmt_x, true}, N, K, M, p,
+  return run_gemm(Operand{dyq, lddy, fmt_dy, true}, Operand{xq, ldx, fmt_x, true}, N, K, M, p, ws, ws_bytes,
                   (cudaStream_t)stream);
 }
 

@@ -57,6 +57,7 @@ class BlockStep:
         self.a = [torch.empty((self.M, self.cfg.d), dtype=torch.bfloat16, device=device) for _ in range(self.n_blocks)]
         self.ga = [torch.empty_like(t) for t in self.a]
         self.loss_ws = tw.new_workspace(tw.OP_LOSS, n, self.n_blocks, device=device)
+        self.gemm_ws = None
         self.loss = None
         self.host = None
         self.tau, self.eps, self.p, self.lam = 3.0, 1e-6, 4.0, 0.01
@@ -99,9 +100,11 @@ class BlockStep:
         tw.quantize_per_tensor(lb.dy, self.grad_fmt, tw.SCALE_CURRENT, out=lb.qdy)
 
     def gemms(self, lb: LinearBuffers):
-        tw.fp8_linear_fwd(lb.qx.q, lb.qw.q, lb.qx.scale_inv, lb.qw.scale_inv, y=lb.y)
-        tw.fp8_linear_bwd_dgrad(lb.qdy.q, lb.qw.q, lb.qdy.scale_inv, lb.qw.scale_inv, fmt_dy=self.grad_fmt, dx=lb.dx)
-        tw.fp8_linear_bwd_wgrad(lb.qx.q, lb.qdy.q, lb.qx.scale_inv, lb.qdy.scale_inv, fmt_dy=self.grad_fmt, dw=lb.dw)
+        tw.fp8_linear_fwd(lb.qx.q, lb.qw.q, lb.qx.scale_inv, lb.qw.scale_inv, y=lb.y, ws=self.gemm_ws)
+        tw.fp8_linear_bwd_dgrad(lb.qdy.q, lb.qw.q, lb.qdy.scale_inv, lb.qw.scale_inv, fmt_dy=self.grad_fmt, dx=lb.dx,
+                                ws=self.gemm_ws)
+        tw.fp8_linear_bwd_wgrad(lb.qx.q, lb.qdy.q, lb.qx.scale_inv, lb.qdy.scale_inv, fmt_dy=self.grad_fmt, dw=lb.dw,
+                                ws=self.gemm_ws)
 
     def tweo(self):
         c = self.lam / self.n_blocks

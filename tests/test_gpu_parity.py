@@ -202,12 +202,12 @@ def dev_scalar(v):
     return torch.tensor([float(v)], dtype=torch.float32, device="cuda")
 
 
-def run_three(tw, qx, qw, qd, fmt_g, dw_f32=False):
+def run_three(tw, qx, qw, qd, fmt_g, dw_f32=False, ws=None):
     xq, wq, dyq = (torch.from_numpy(q["q"]).cuda() for q in (qx, qw, qd))
     sx, sw, sd = (dev_scalar(q["scale_inv"]) for q in (qx, qw, qd))
-    y = tw.fp8_linear_fwd(xq, wq, sx, sw)
-    dx = tw.fp8_linear_bwd_dgrad(dyq, wq, sd, sw, fmt_dy=fmt_g)
-    dw = tw.fp8_linear_bwd_wgrad(xq, dyq, sx, sd, fmt_dy=fmt_g, dw_dtype=tw.F32 if dw_f32 else tw.BF16)
+    y = tw.fp8_linear_fwd(xq, wq, sx, sw, ws=ws)
+    dx = tw.fp8_linear_bwd_dgrad(dyq, wq, sd, sw, fmt_dy=fmt_g, ws=ws)
+    dw = tw.fp8_linear_bwd_wgrad(xq, dyq, sx, sd, fmt_dy=fmt_g, dw_dtype=tw.F32 if dw_f32 else tw.BF16, ws=ws)
     torch.cuda.synchronize()
     assert tw.read_device_status() == 0
     return y, dx, dw
@@ -245,6 +245,43 @@ def test_gemms_small_full_compare(tw, name, M, K, N, fmt_g):
         g = got.float().cpu().numpy().astype(np.float64)
         scale = np.max(np.abs(ref)) + 1e-300
         assert np.max(np.abs(g - ref) - np.abs(ref) * 2.0 ** -8) <= 1e-4 * scale, what
+
+
+SPLIT_SHAPES = [
+    # few output tiles, long contraction: the kernel splits tiles along the contraction
+    ("wgrad_long_m", 6144, 256, 384),     # wgrad: 3 x 1 tiles, 48 k-blocks
+    ("fwd_long_k", 256, 4096, 512),       # fwd: 2 x 2 tiles, 32 k-blocks; dgrad: 2 x 16 tiles
+    ("ragged", 3000, 1616, 272),          # ragged everywhere, 190 tiles > 148 SMs for dgrad (partial wave)
+]
+
+
+@pytest.mark.parametrize("dw_f32", [False, True], ids=["bf16dw", "f32dw"])
+@pytest.mark.parametrize("name,M,K,N", SPLIT_SHAPES, ids=[s[0] for s in SPLIT_SHAPES])
+def test_gemms_split_along_contraction(tw, name, M, K, N, dw_f32):
+    x = synth.normal_with_outlier_channels_bf16(90, (M, K))
+    w = synth.normal_bf16(91, (N, K), 0.02)
+    dy = synth.normal_bf16(92, (M, N), 1e-3)
+    qx, qw, qd = quantized_operands(x, w, dy)
+    ws = tw.new_workspace(tw.OP_LINEAR_WGRAD)
+    y, dx, dw = run_three(tw, qx, qw, qd, E5M2, dw_f32=dw_f32, ws=ws)
+    y2, dx2, dw2 = run_three(tw, qx, qw, qd, E5M2, dw_f32=dw_f32, ws=ws)        # same workspace again
+    y0, dx0, dw0 = run_three(tw, qx, qw, qd, E5M2, dw_f32=dw_f32, ws=None)      # whole tiles only
+    g = np.random.Generator(np.random.PCG64(7))
+    for got, again, plain, what, (rows, cols) in ((y, y2, y0, "fwd", (M, N)), (dx, dx2, dx0, "dgrad", (M, K)),
+                                                  (dw, dw2, dw0, "wgrad", (N, K))):
+        assert torch.equal(got.view(torch.int32 if got.dtype == torch.float32 else torch.int16),
+                           again.view(torch.int32 if got.dtype == torch.float32 else torch.int16)), what
+        r, c = sample_points(g, rows, cols, n_rows=3, n_pts=3000)
+        if what == "fwd":
+            ref = orc.gemm_fwd_at(qx["q"], E4M3, qw["q"], E4M3, qx["scale_inv"], qw["scale_inv"], r, c)
+        elif what == "dgrad":
+            ref = orc.gemm_dgrad_at(qd["q"], E5M2, qw["q"], E4M3, qd["scale_inv"], qw["scale_inv"], r, c)
+        else:
+            ref = orc.gemm_wgrad_at(qx["q"], E4M3, qd["q"], E5M2, qx["scale_inv"], qd["scale_inv"], r, c)
+        tol = 1e-5 if got.dtype == torch.float32 else GEMM_TOL
+        assert rel_fro(got.float().cpu().numpy()[r, c], ref) <= tol, what
+        # split and unsplit runs agree to fp32 summation order
+        assert rel_fro(got.float().cpu().numpy(), plain.float().cpu().numpy().astype(np.float64)) <= 1e-3, what
 
 
 def test_wgrad_fp32_output_and_accumulate(tw):
@@ -288,7 +325,7 @@ def test_fused_epilogue_equals_unfused_bit_for_bit(tw):
     assert torch.equal(unf.q, yq) and f32_bits(unf.amax) == f32_bits(amax)
 
 
-def sample_points(g, rows, cols, n_rows=4, n_pts=2048):
+def sample_points(g, rows, cols, n_rows=4, n_pts=2048):  # noqa: E302
     r_full = g.choice(rows, size=min(n_rows, rows), replace=False)
     rr = np.repeat(r_full, cols)
     cc = np.tile(np.arange(cols), len(r_full))
