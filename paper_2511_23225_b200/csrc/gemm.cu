@@ -57,6 +57,7 @@ struct GemmParams {
   int64_t ldd;
   int32_t Md, Nd, Kc;
   int32_t tiles_m, tiles_n, k_blocks;
+  int32_t raster_g;    // tiles are numbered in bands of raster_g tile rows (see tile_coords)
   const float* sa_inv;
   const float* sb_inv;
   int32_t out_f32;     // 0: bf16 out, 1: fp32 out
@@ -73,6 +74,21 @@ struct GemmParams {
   uint32_t* sk_flags;   // [grid][4] per epilogue warp: == epoch once the share is written
   uint32_t epoch;
 };
+
+// Tile index -> tile coordinates.  Tiles are numbered band by band: a band is raster_g tile
+// rows high and is walked column by column, so the tiles in flight at any time cover a
+// compact block (about raster_g rows x workers/raster_g columns) and the rows of A and the
+// columns of B they share are re-read from L2 while they are still hot, instead of every wave
+// sweeping all of A.
+__device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& tm, int& tn) {
+  const int per_band = p.raster_g * p.tiles_n;
+  const int band = tile / per_band;
+  const int first = band * p.raster_g;
+  const int rows = min(p.raster_g, p.tiles_m - first);
+  const int in = tile - band * per_band;
+  tn = in / rows;
+  tm = first + in - tn * rows;
+}
 
 // The work list of one CTA, identical in the three roles (producer, MMA, epilogue).
 struct Sched {
@@ -320,8 +336,10 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       Sched sched(p, blockIdx.x, gridDim.x);
       int tile, kb0, kb1;
       while (ok && sched.next(tile, kb0, kb1)) {
-        const int m0 = (tile % p.tiles_m) * BM;
-        const int n0 = (tile / p.tiles_m) * BN;
+        int tm, tn;
+        tile_coords(p, tile, tm, tn);
+        const int m0 = tm * BM;
+        const int n0 = tn * BN;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t fb = full_bar(stage);
@@ -404,8 +422,10 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     Sched sched(p, blockIdx.x, gridDim.x);
     int tile, kb0, kb1;
     while (ok && sched.next(tile, kb0, kb1)) {
-      const int m0 = (tile % p.tiles_m) * BM;
-      const int n0 = (tile / p.tiles_m) * BN;
+      int tm, tn;
+      tile_coords(p, tile, tm, tn);
+      const int m0 = tm * BM;
+      const int n0 = tn * BN;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
@@ -683,8 +703,10 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-        const int m0 = (tile % p.tiles_m) * (2 * BM) + (int)rank * BM;  // this CTA's rows
-        const int n0 = (tile / p.tiles_m) * BN + (int)rank * 128;       // this CTA's half of B
+        int tm, tn;
+        tile_coords(p, tile, tm, tn);
+        const int m0 = tm * (2 * BM) + (int)rank * BM;  // this CTA's rows
+        const int n0 = tn * BN + (int)rank * 128;       // this CTA's half of B
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
@@ -750,8 +772,10 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-      const int m0 = (tile % p.tiles_m) * (2 * BM) + (int)rank * BM;
-      const int n0 = (tile / p.tiles_m) * BN;
+      int tm, tn;
+      tile_coords(p, tile, tm, tn);
+      const int m0 = tm * (2 * BM) + (int)rank * BM;
+      const int n0 = tn * BN;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int row0 = m0 + quarter * 32;
@@ -917,6 +941,15 @@ std::atomic<uint32_t> g_sk_epoch{0};
 // TWEO_GEMM_NO_PAIR=1 in the environment keeps every GEMM on the single-CTA kernel (A/B timing).
 const bool g_disable_pair = [] { const char* e = getenv("TWEO_GEMM_NO_PAIR"); return e && e[0] == '1'; }();
 
+// Band height of the tile numbering: the `workers` tiles in flight cover about g x workers/g
+// tiles, so g near sqrt(workers) keeps the rows of A and the columns of B they touch smallest.
+int raster_band(int tiles_m, int workers) {
+  int g = 1;
+  while ((g + 1) * (g + 1) <= workers) ++g;
+  if (g > tiles_m) g = tiles_m;
+  return g < 1 ? 1 : g;
+}
+
 template <int BN, bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
 tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, GemmParams& p,
                          void* ws, size_t ws_bytes, cudaStream_t st) {
@@ -933,6 +966,7 @@ tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
   const int tiles = p.tiles_m * p.tiles_n;
   const int sms = sm_count();
   int grid = sms < tiles ? sms : tiles;
+  p.raster_g = raster_band(p.tiles_m, sms);
   p.sk_tiles = 0;
   p.sk_partials = nullptr;
   p.sk_flags = nullptr;
@@ -974,6 +1008,7 @@ tweo_status_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CU
   p.sk_tiles = 0;
   const int tiles = p.tiles_m * p.tiles_n;
   int pairs = sm_count() / 2;
+  p.raster_g = raster_band(p.tiles_m, pairs);
   if (pairs > tiles) pairs = tiles;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs));
