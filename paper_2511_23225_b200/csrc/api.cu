@@ -65,7 +65,7 @@ uint64_t tweo_launch_count(void) { return g_launches.load(std::memory_order_rela
 
 size_t tweo_workspace_bytes(int32_t op, int64_t M, int64_t N, int64_t K) {
   const size_t sms = (size_t)tweo_detail::sm_count();
-  const size_t stream_k_bytes = sms * 128 * 256 * sizeof(float) + ((sms * 16 + 255) & ~(size_t)255) + 256;
+  const size_t stream_k_bytes = 12288 + sms * 256 * 1024;  // flags, ticket counters, 256 KB of parked fp32 sums per SM
   switch (op) {
     case TWEO_OP_LOSS: {
       int L = (int)(N < 1 ? 1 : N);
@@ -74,7 +74,7 @@ size_t tweo_workspace_bytes(int32_t op, int64_t M, int64_t N, int64_t K) {
     case TWEO_OP_LINEAR_FWD:
     case TWEO_OP_LINEAR_DGRAD:
     case TWEO_OP_LINEAR_WGRAD:
-      // optional: lets the GEMM split tiles along the contraction (one 128x256 fp32 slot per SM + flags)
+      // optional: lets the GEMM split tiles along the contraction (parked fp32 accumulators + flags)
       return stream_k_bytes;
     case TWEO_OP_W8A8: {
       // scalars + codes of the activations (a bf16 input is cast inside) + the GEMM's stream-K area

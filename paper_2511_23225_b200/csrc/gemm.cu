@@ -72,8 +72,17 @@ struct GemmParams {
   int32_t sk_tiles;
   float* sk_partials;   // [grid][BM*BN] raw accumulators of shares that do not own their tile
   uint32_t* sk_flags;   // [grid][4] per epilogue warp: == epoch once the share is written
+  uint32_t* sk_counters;  // CTA-pair kernel: [sk_tiles][2][4] tickets per (tile, CTA of the pair, epilogue warp)
   uint32_t epoch;
 };
+
+// Workspace layout of the linear calls (bytes from the workspace base):
+//   [0, 4096)       flags of the single-CTA kernel's split tiles (4 words per CTA)
+//   [4096, 12288)   ticket counters of the CTA-pair kernel's split tiles (8 words per tile)
+//   [12288, ...)    parked fp32 accumulators: 256 KB per SM
+constexpr size_t kWsCountersOffset = 4096;
+constexpr size_t kWsPartialsOffset = 12288;
+constexpr size_t kWsPartialBytesPerSm = 256 * 1024;
 
 // Tile index -> tile coordinates.  Tiles are numbered band by band: a band is raster_g tile
 // rows high and is walked column by column, so the tiles in flight at any time cover a
@@ -643,10 +652,134 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t cluster_bar) {
                : "memory");
 }
 
+// A share of the pair kernel that covers only part of a split tile.  Parks this warp's
+// 32 x 256 block of the raw accumulator in the workspace ([column][row], so every store is
+// one full line), hands the accumulator back to the MMA warp and takes a ticket; the warp
+// that draws the last ticket of the tile adds the parked blocks of ALL shares in share order
+// (= ascending k, whoever arrived last, so the sum does not depend on timing) and stores the
+// result.  Nobody waits for anybody.  Kept out of line: it is rare and register-hungry.
+constexpr size_t kPairCtaFloats = 128 * 256;   // one CTA's half of a parked 256 x 256 accumulator
+constexpr size_t kPairWarpFloats = 32 * 256;   // one epilogue warp's block of it
+
+template <bool OUT_F32>
+__device__ __noinline__ float pair_partial_share(const GemmParams& p, const CUtensorMap* tmap_d, int tile, int kb0,
+                                                int pair, int num_pairs, int rank, int wslot,
+                                                uint32_t tacc, uint32_t tempty_leader, float alpha, float qs,
+                                                uint32_t epi_base, uint32_t it, int lane, int row0, int n0) {
+  constexpr int CH = OUT_F32 ? 32 : 64;
+  constexpr uint32_t EPI_BUF = 32 * 128;
+  float run_amax = 0.0f;
+  float* slot = p.sk_partials + ((size_t)(pair * 2 + (kb0 > 0 ? 0 : 1)) * 2 + rank) * kPairCtaFloats +
+                (size_t)wslot * kPairWarpFloats;
+#pragma unroll 1
+  for (int g = 0; g < 8; ++g) {
+    uint32_t r[32];
+    tmem_ld32(tacc + (uint32_t)(g * 32), r);
+    tmem_ld_wait();
+    float* dst = slot + g * 1024 + lane;
+#pragma unroll
+    for (int k = 0; k < 32; ++k) __stcg(dst + k * 32, __uint_as_float(r[k]));
+  }
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive_cluster(tempty_leader);
+  // which pairs hold a share of this tile (they are consecutive)
+  const int64_t t_begin = (int64_t)tile * p.k_blocks, t_end = t_begin + p.k_blocks;
+  int j_first = pair;
+  while (j_first > 0 && Sched::share_begin(p, j_first, num_pairs) > t_begin) --j_first;
+  int j_last = pair;
+  while (j_last + 1 < num_pairs && Sched::share_begin(p, j_last + 1, num_pairs) < t_end) ++j_last;
+  const int n_shares = j_last - j_first + 1;
+  __threadfence();
+  __syncwarp();
+  uint32_t ticket = 0;
+  uint32_t* counter = p.sk_counters + ((size_t)tile * 2 + rank) * 4 + wslot;
+  if (lane == 0) ticket = atomicAdd(counter, 1u);
+  ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+  if (ticket + 1 != (uint32_t)n_shares) return 0.0f;  // not the last share of this tile: done
+  __threadfence();
+  if (lane == 0) *counter = 0u;  // ready for the next launch
+  const uint32_t row_off = (uint32_t)lane * 128u;
+  const uint32_t swz = (uint32_t)(lane & 7);
+  const int row = row0 + lane;
+#pragma unroll 1
+  for (int c = 0; c < 256 / CH; ++c) {
+    const int col0 = n0 + c * CH;
+    if (col0 >= p.Nd || row0 >= p.Md) break;  // uniform across the warp
+    uint32_t r[CH];
+#pragma unroll 1
+    for (int sidx = 0; sidx < n_shares; ++sidx) {
+      const int j = j_first + sidx;
+      const int sel = Sched::share_begin(p, j, num_pairs) > t_begin ? 0 : 1;
+      const float* src = p.sk_partials + ((size_t)(j * 2 + sel) * 2 + rank) * kPairCtaFloats +
+                         (size_t)wslot * kPairWarpFloats + (size_t)(c * CH) * 32 + lane;
+      if (sidx == 0) {
+#pragma unroll
+        for (int k = 0; k < CH; ++k) r[k] = __float_as_uint(__ldcg(src + k * 32));
+      } else {
+#pragma unroll
+        for (int k = 0; k < CH; ++k) r[k] = __float_as_uint(__uint_as_float(r[k]) + __ldcg(src + k * 32));
+      }
+    }
+    const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
+    ++it;
+    if (lane == 0) bulk_wait_read<1>();
+    __syncwarp();
+    if (OUT_F32) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4),
+                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j]), alpha)),
+                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 1]), alpha)),
+                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 2]), alpha)),
+                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 3]), alpha)));
+    } else {
+      uint32_t packed[CH / 2];
+#pragma unroll
+      for (int j = 0; j < CH / 2; ++j)
+        packed[j] = f32x2_to_bf16x2(__fmul_rn(__uint_as_float(r[2 * j]), alpha),
+                                    __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha));
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1], packed[4 * j + 2],
+                     packed[4 * j + 3]);
+      if ((p.out_amax || p.out_q) && row < p.Md) {
+#pragma unroll 1
+        for (int j = 0; j < CH / 4; ++j) {  // groups of four columns
+          const uint32_t w0 = packed[2 * j], w1 = packed[2 * j + 1];
+          float v[4] = {bf16lo_to_f32(w0), bf16hi_to_f32(w0), bf16lo_to_f32(w1), bf16hi_to_f32(w1)};
+          if (col0 + 4 * j < p.Nd) {
+            run_amax = fmaxf(run_amax, fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))));
+            if (p.out_q) {
+              const uint32_t q = p.q_fmt == TWEO_E4M3
+                                     ? quant4<TWEO_E4M3>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs),
+                                                         __fmul_rn(v[2], qs), __fmul_rn(v[3], qs))
+                                     : quant4<TWEO_E5M2>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs),
+                                                         __fmul_rn(v[2], qs), __fmul_rn(v[3], qs));
+              *reinterpret_cast<uint32_t*>(p.out_q + (int64_t)row * p.ldq + col0 + 4 * j) = q;
+            }
+          }
+        }
+      }
+    }
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+      if (OUT_F32 && p.accumulate) tma_reduce_add_2d(tmap_d, col0, row0, buf);
+      else tma_store_2d(tmap_d, col0, row0, buf);
+      bulk_commit();
+    }
+  }
+  // the caller's buffer rotation does not know how many chunks were stored here
+  if (lane == 0) bulk_wait_read<0>();
+  __syncwarp();
+  return run_amax;
+}
+
 template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                     const __grid_constant__ CUtensorMap tmap_d, const GemmParams p) {
+                     const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ GemmParams p) {
   constexpr int BN = 256;                 // tile columns of the pair
   constexpr uint32_t A_BYTES = BM * BK;   // this CTA's 128 rows of A
   constexpr uint32_t B_BYTES = 128 * BK;  // this CTA's 128 of the 256 columns of B
@@ -692,7 +825,6 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int num_tiles = p.tiles_m * p.tiles_n;
   const int pair = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;
 
@@ -702,12 +834,14 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+      Sched sched(p, pair, num_pairs);
+      int tile, kb0, kb1;
+      while (ok && sched.next(tile, kb0, kb1)) {
         int tm, tn;
         tile_coords(p, tile, tm, tn);
         const int m0 = tm * (2 * BM) + (int)rank * BM;  // this CTA's rows
         const int n0 = tn * BN + (int)rank * 128;       // this CTA's half of B
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
           const uint32_t fb = map_to_cta(full_bar(stage), 0);
@@ -730,11 +864,13 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+      Sched sched(p, pair, num_pairs);
+      int tile, kb0, kb1;
+      while (ok && sched.next(tile, kb0, kb1)) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
@@ -743,7 +879,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint64_t adesc = make_smem_desc(sa + (A_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
             const uint64_t bdesc = make_smem_desc(sb + (B_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
-            umma_f8_pair(d_tmem, adesc, bdesc, p.idesc, (uint32_t)((kb | k) != 0));
+            umma_f8_pair(d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != kb0 || k != 0));
           }
           umma_commit_pair(map_to_cta(empty_bar(stage), 0));  // frees the stage in both CTAs
           umma_commit_pair(map_to_cta(empty_bar(stage), 1));
@@ -771,7 +907,9 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+    Sched sched(p, pair, num_pairs);
+    int tile, kb0, kb1;
+    while (ok && sched.next(tile, kb0, kb1)) {
       int tm, tn;
       tile_coords(p, tile, tm, tn);
       const int m0 = tm * (2 * BM) + (int)rank * BM;
@@ -781,6 +919,18 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       const int row0 = m0 + quarter * 32;
       const int row = row0 + lane;
       const bool row_ok = row < p.Md;
+      if (kb0 != 0 || kb1 != p.k_blocks) {
+        // part of a split tile: park the accumulator; the last share to arrive stores the tile
+        const float part_amax = pair_partial_share<OUT_F32>(
+            p, &tmap_d, tile, kb0, pair, num_pairs, (int)rank, warp - 2,
+            tmem_base + tlane + (uint32_t)(acc * BN), map_to_cta(tempty_bar(acc), 0), alpha, qs, epi_base, it, lane,
+            row0, n0);
+        it += BN / CH;  // keeps the staging-buffer rotation in step whether or not this warp stored
+        run_amax = fmaxf(run_amax, part_amax);
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+        continue;
+      }
 #pragma unroll 1
       for (int c = 0; c < BN / CH; ++c) {
         const int col0 = n0 + c * CH;
@@ -970,10 +1120,11 @@ tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
   p.sk_tiles = 0;
   p.sk_partials = nullptr;
   p.sk_flags = nullptr;
+  p.sk_counters = nullptr;
   p.epoch = 0;
   // Stream-K when whole-tile dealing would idle more than ~15 % of the SM-time and the
   // contraction is long enough to pay for the fix-up (a 128 x BN fp32 round trip through L2).
-  const size_t sk_need = (size_t)sms * BM * BN * sizeof(float) + (size_t)sms * 16 + 256;
+  const size_t sk_need = kWsPartialsOffset + (size_t)sms * kWsPartialBytesPerSm;
   const int waves = (tiles + sms - 1) / sms;
   if (ws && ws_bytes >= sk_need && aligned16(ws) && p.k_blocks >= 12 &&
       (double)tiles < 0.85 * (double)waves * sms) {
@@ -982,7 +1133,7 @@ tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
     grid = sms;
     if ((int64_t)p.sk_tiles * p.k_blocks < grid) grid = (int)((int64_t)p.sk_tiles * p.k_blocks);
     p.sk_flags = reinterpret_cast<uint32_t*>(ws);
-    p.sk_partials = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + (((size_t)sms * 16 + 255) & ~(size_t)255));
+    p.sk_partials = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + kWsPartialsOffset);
     p.epoch = g_sk_epoch.fetch_add(1, std::memory_order_relaxed) + 1;
   }
   kern<<<grid, kThreads, smem, st>>>(ma, mb, md, p);
@@ -990,9 +1141,23 @@ tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
   return check_launch("gemm_fp8_kernel");
 }
 
+// How many of the `tiles` the pair kernel splits along the contraction (0 = none).  Whole tiles
+// are dealt round-robin; what does not fill the last wave is split so that every pair gets the
+// same number of k-blocks.  Parking and re-adding 256 x 256 fp32 accumulators costs each SM
+// tens of microseconds' worth of L2 traffic spread over the GPU (measured: about 25 000 cycles
+// per pair), so the split only pays when the idle time it removes is clearly larger.
+int pair_split_tiles(int tiles, int workers, int k_blocks) {
+  const int rem = tiles % workers;
+  if (rem == 0) return 0;
+  const double idle_clks = (double)(workers - rem) / workers * k_blocks * 512.0;  // per pair, if not split
+  if (idle_clks < 40000.0) return 0;
+  if ((int64_t)rem * k_blocks < (int64_t)8 * workers) return 0;                  // shares of at least 8 k-blocks
+  return rem;
+}
+
 template <bool A_MN, bool B_MN, bool OUT_F32>
 tweo_status_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, GemmParams& p,
-                          cudaStream_t st) {
+                          void* ws, size_t ws_bytes, cudaStream_t st) {
   constexpr int STAGES = 6;
   constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
   auto kern = gemm_fp8_pair_kernel<A_MN, B_MN, STAGES, OUT_F32>;
@@ -1006,10 +1171,22 @@ tweo_status_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CU
   p.tiles_n = (p.Nd + 255) / 256;
   p.k_blocks = (p.Kc + BK - 1) / BK;
   p.sk_tiles = 0;
+  p.sk_partials = nullptr;
+  p.sk_flags = nullptr;
+  p.sk_counters = nullptr;
+  p.epoch = 0;
   const int tiles = p.tiles_m * p.tiles_n;
-  int pairs = sm_count() / 2;
+  const int sms = sm_count();
+  int pairs = sms / 2;
   p.raster_g = raster_band(p.tiles_m, pairs);
-  if (pairs > tiles) pairs = tiles;
+  if (ws && ws_bytes >= kWsPartialsOffset + (size_t)sms * kWsPartialBytesPerSm && aligned16(ws)) {
+    p.sk_tiles = pair_split_tiles(tiles, pairs, p.k_blocks);
+    if (p.sk_tiles > 0) {
+      p.sk_counters = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + kWsCountersOffset);
+      p.sk_partials = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + kWsPartialsOffset);
+    }
+  }
+  if (p.sk_tiles == 0 && pairs > tiles) pairs = tiles;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs));
   cfg.blockDim = dim3(kThreads);
@@ -1070,7 +1247,7 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
     count_launch();
   }
   if (use_pair) {
-#define TWEO_PAIR(AMN, BMN) (p.out_f32 ? launch_pair<AMN, BMN, true>(ma, mb, md, p, st) : launch_pair<AMN, BMN, false>(ma, mb, md, p, st))
+#define TWEO_PAIR(AMN, BMN) (p.out_f32 ? launch_pair<AMN, BMN, true>(ma, mb, md, p, ws, ws_bytes, st) : launch_pair<AMN, BMN, false>(ma, mb, md, p, ws, ws_bytes, st))
     if (!A.mn_major && !B.mn_major) return TWEO_PAIR(false, false);
     if (!A.mn_major && B.mn_major) return TWEO_PAIR(false, true);
     if (A.mn_major && B.mn_major) return TWEO_PAIR(true, true);

@@ -252,6 +252,8 @@ SPLIT_SHAPES = [
     ("wgrad_long_m", 6144, 256, 384),     # wgrad: 3 x 1 tiles, 48 k-blocks
     ("fwd_long_k", 256, 4096, 512),       # fwd: 2 x 2 tiles, 32 k-blocks; dgrad: 2 x 16 tiles
     ("ragged", 3000, 1616, 272),          # ragged everywhere, 190 tiles > 148 SMs for dgrad (partial wave)
+    ("wgrad_very_long_m", 16384, 512, 768),   # wgrad: 3 x 2 tiles of 256 x 256, 128 k-blocks: the CTA-pair kernel splits
+    ("wgrad_ragged_long", 20000, 400, 528),   # the same with ragged edges in every dimension (157 k-blocks)
 ]
 
 
