@@ -111,11 +111,45 @@ typedef struct tweo_epilogue_t {
  *     saturation to +-FP8MAX; NaN -> 0x7F (no sign).  amax skips NaN.
  *   sat_count: device uint32*, or NULL; receives the number of elements with
  *     |fl32(x_i * scale)| > FP8MAX.
- *   No workspace is needed (ws may be NULL).
+ *   Workspace: optional.  With ws == NULL the call runs as separate kernels (reset, amax,
+ *     cast).  With a workspace of tweo_workspace_bytes(TWEO_OP_QUANTIZE) bytes (any
+ *     contents) a CURRENT-scaling call without sat_count runs as two kernels: per-CTA
+ *     maxima go to workspace slots and every CTA of the cast reduces them itself, so
+ *     there is no reset kernel and no atomic.  Results are identical bit for bit.
  */
 TWEO_API tweo_status_t tweo_quantize_per_tensor(const uint16_t* x, int64_t n, int32_t fmt, int32_t mode,
                                        float* scale, float* scale_inv, float* amax, uint8_t* q,
                                        uint32_t* sat_count, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * tweo_quantize_per_tensor_batch -- tweo_quantize_per_tensor for up to
+ * TWEO_MAX_QUANT_BATCH tensors in one pair of kernels (Sec. 4.2: a linear layer casts its
+ * activation, its weight and, in the backward pass, its output gradient, each with its
+ * own per-tensor scale; casting them together saves launches, which dominate for small
+ * tensors).  Every tensor is treated exactly as tweo_quantize_per_tensor would treat it
+ * (own amax, own scale, own format and mode; results bit-identical).
+ *   descs: HOST array of `count` descriptors (read during the call, not kept).
+ *   ws: tweo_workspace_bytes(TWEO_OP_QUANTIZE) bytes, any contents.  The tensors with
+ *     CURRENT scaling and no sat_count share one amax kernel and one cast kernel per FP8
+ *     format; GIVEN-scale tensors and those with a sat_count (and all of them when ws is
+ *     NULL or too small) are launched one by one as tweo_quantize_per_tensor does.
+ *   Errors: TWEO_ERR_INVALID_ARG (count out of range, NULL pointers, bad enums),
+ *     TWEO_ERR_ALIGNMENT.
+ */
+#define TWEO_MAX_QUANT_BATCH 8
+typedef struct tweo_quant_desc_t {
+  const uint16_t* x;   /* bf16 [n], device */
+  int64_t n;
+  int32_t fmt;         /* tweo_fp8_t */
+  int32_t mode;        /* tweo_scale_mode_t */
+  float* scale;        /* device; out (CURRENT) or in (GIVEN) */
+  float* scale_inv;    /* device out */
+  float* amax;         /* device out */
+  uint8_t* q;          /* uint8 [n], device out */
+  uint32_t* sat_count; /* device out, or NULL */
+} tweo_quant_desc_t;
+TWEO_API tweo_status_t tweo_quantize_per_tensor_batch(const tweo_quant_desc_t* descs, int32_t count, void* ws,
+                                             size_t ws_bytes, void* stream);
 
 /*
  * tweo_fp8_linear_fwd -- forward GEMM of an FP8 linear layer (Sec. 4.2):

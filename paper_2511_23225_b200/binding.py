@@ -23,7 +23,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtweo_b200.so")
 
 EXPORTS = [
-    "tweo_quantize_per_tensor", "tweo_fp8_linear_fwd", "tweo_fp8_linear_bwd_dgrad",
+    "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_bwd_dgrad",
     "tweo_fp8_linear_bwd_wgrad", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
@@ -38,6 +38,15 @@ class TweoError(RuntimeError):
             msg += ": " + L.tweo_last_cuda_error().decode()
         super().__init__(f"{where}: {msg} (status {status})")
         self.status = status
+
+
+class _QuantDesc(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("n", C.c_int64), ("fmt", C.c_int32), ("mode", C.c_int32),
+                ("scale", C.c_void_p), ("scale_inv", C.c_void_p), ("amax", C.c_void_p), ("q", C.c_void_p),
+                ("sat_count", C.c_void_p)]
+
+
+MAX_QUANT_BATCH = 8
 
 
 class _Epilogue(C.Structure):
@@ -59,6 +68,7 @@ def lib() -> C.CDLL:
         L = C.CDLL(LIB_PATH)
         vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
         L.tweo_quantize_per_tensor.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.tweo_quantize_per_tensor_batch.argtypes = [C.POINTER(_QuantDesc), i32, vp, sz, vp]
         L.tweo_fp8_linear_fwd.argtypes = [vp, i64, vp, i64, vp, vp, vp, i64, i64, i64, i64, i32, i32,
                                           C.POINTER(_Epilogue), vp, sz, vp]
         L.tweo_fp8_linear_bwd_dgrad.argtypes = [vp, i64, i32, vp, i64, i32, vp, vp, vp, i64, i64, i64, i64,
@@ -149,8 +159,9 @@ class Quantized:
 
 def quantize_per_tensor(x: torch.Tensor, fmt: int = E4M3, mode: int = SCALE_CURRENT,
                         scale: torch.Tensor | None = None, count_saturated: bool = False,
-                        out: Quantized | None = None) -> Quantized:
-    """tweo_quantize_per_tensor: amax -> scale -> FP8 codes of a bf16 tensor."""
+                        out: Quantized | None = None, ws: torch.Tensor | None = None) -> Quantized:
+    """tweo_quantize_per_tensor: amax -> scale -> FP8 codes of a bf16 tensor.
+    With a workspace (new_workspace(OP_QUANTIZE)) current scaling runs as two kernels, not three."""
     xp = _dev(x, torch.bfloat16, "x")
     if not x.is_contiguous():
         raise ValueError("x must be contiguous")
@@ -168,8 +179,36 @@ def quantize_per_tensor(x: torch.Tensor, fmt: int = E4M3, mode: int = SCALE_CURR
     sat = out.sat_count.data_ptr() if out.sat_count is not None else None
     _check(lib().tweo_quantize_per_tensor(xp, x.numel(), fmt, mode, _dev(out.scale, torch.float32, "scale"),
                                           out.scale_inv.data_ptr(), out.amax.data_ptr(), out.q.data_ptr(), sat,
-                                          None, 0, _stream()), "tweo_quantize_per_tensor")
+                                          *_ws(ws), _stream()), "tweo_quantize_per_tensor")
     return out
+
+
+def quantize_per_tensor_batch(xs, outs, modes=None, ws: torch.Tensor | None = None):
+    """tweo_quantize_per_tensor_batch: casts up to MAX_QUANT_BATCH bf16 tensors in one kernel, each
+    with its own per-tensor scale.  `outs` are Quantized records (their fmt and, for GIVEN mode, their
+    scale are read); `modes` defaults to CURRENT for all."""
+    n = len(xs)
+    if n != len(outs) or not 1 <= n <= MAX_QUANT_BATCH:
+        raise ValueError("need 1..MAX_QUANT_BATCH tensors with one output record each")
+    if ws is None:
+        ws = new_workspace(OP_QUANTIZE)
+    descs = (_QuantDesc * n)()
+    for i, (x, o) in enumerate(zip(xs, outs)):
+        if not x.is_contiguous():
+            raise ValueError("x must be contiguous")
+        d = descs[i]
+        d.x = _dev(x, torch.bfloat16, "x")
+        d.n = x.numel()
+        d.fmt = o.fmt
+        d.mode = SCALE_CURRENT if modes is None else modes[i]
+        d.scale = _dev(o.scale, torch.float32, "scale")
+        d.scale_inv = _dev(o.scale_inv, torch.float32, "scale_inv")
+        d.amax = _dev(o.amax, torch.float32, "amax")
+        d.q = _dev(o.q, U8, "q")
+        d.sat_count = o.sat_count.data_ptr() if o.sat_count is not None else None
+    _check(lib().tweo_quantize_per_tensor_batch(descs, n, ws.data_ptr(), ws.numel(), _stream()),
+           "tweo_quantize_per_tensor_batch")
+    return outs
 
 
 def _epilogue(amax, q, q_fmt, q_scale):

@@ -37,6 +37,7 @@ tweo_status_t check_launch(const char* what) {
   return TWEO_OK;
 }
 
+size_t quantize_workspace_bytes();
 // Blocks per tensor of the loss kernel; also fixes the workspace size.
 int loss_blocks_per_tensor(int64_t n, int L);
 
@@ -67,6 +68,8 @@ size_t tweo_workspace_bytes(int32_t op, int64_t M, int64_t N, int64_t K) {
   const size_t sms = (size_t)tweo_detail::sm_count();
   const size_t stream_k_bytes = 12288 + sms * 256 * 1024;  // flags, ticket counters, 256 KB of parked fp32 sums per SM
   switch (op) {
+    case TWEO_OP_QUANTIZE:
+      return tweo_detail::quantize_workspace_bytes();  // optional: selects the batched form of the cast
     case TWEO_OP_LOSS: {
       int L = (int)(N < 1 ? 1 : N);
       return 256 + sizeof(double) * (size_t)L * (size_t)tweo_detail::loss_blocks_per_tensor(M, L);

@@ -18,6 +18,7 @@ tweo_status_t check_launch(const char* what);              // cudaGetLastError a
 
 // Device status word (bounded waits that expired); lives with the GEMM kernels.
 tweo_status_t read_and_clear_device_status(cudaStream_t stream);
+unsigned int* device_status_word();  // its device address on the current device (nullptr on failure)
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

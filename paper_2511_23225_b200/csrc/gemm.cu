@@ -1299,6 +1299,22 @@ tweo_status_t read_and_clear_device_status(cudaStream_t stream) {
   return v == 0 ? TWEO_OK : (tweo_status_t)v;
 }
 
+// Device address of the status word on the current device, for kernels in other files whose
+// bounded waits report through it (nullptr if the lookup fails).
+unsigned int* device_status_word() {
+  static unsigned int* cached[64] = {nullptr};
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cached[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_device_status) != cudaSuccess) return nullptr;
+    cached[dev] = static_cast<unsigned int*>(ptr);
+  }
+  return cached[dev];
+}
+
 // Used by the static W8A8 entry point: forward product on already-cast activations.
 tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
                              const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,

@@ -6,7 +6,16 @@
 // 2 x 16 bytes per thread (16 bf16), stores 16 bytes (16 codes).  amax is the integer
 // maximum of the sign-stripped bf16 bit patterns (exact, order-independent; NaN
 // patterns are skipped), reduced by shuffles and one atomicMax per CTA.
+//
+// Two launch forms.  Without a workspace: a reset kernel, the amax kernel and the cast kernel.
+// With a workspace: two kernels for up to TWEO_MAX_QUANT_BATCH tensors at once -- one reduces
+// every tensor's amax into the workspace, the other casts every tensor with the scale derived
+// from it, and its last CTA writes the scalars out and leaves the workspace zeroed for the
+// next call (so no reset kernel).  A linear layer's three casts (X, W, dY) then cost two
+// launches instead of nine, which matters because the tensors of a transformer block are
+// small enough for launch cost to rival streaming time.
 #include <cuda_bf16.h>
+#include <cuda_runtime.h>
 
 #include "common.cuh"
 
@@ -144,6 +153,158 @@ cast_kernel(const uint16_t* x, int64_t n, float* scale, float* scale_inv, float*
   if (GIVEN) cta_amax_to_global(m, amax);
 }
 
+// ---------------------------------------------------------------------------------------
+// Batched form with a workspace (CURRENT scaling): no reset kernel and no atomics.
+//   kernel 1: every CTA writes the maximum of its share of each tensor to its own workspace
+//             slot (so the workspace needs no particular contents on entry);
+//   kernel 2 (one launch per FP8 format present): every CTA first reduces the slots of a
+//             tensor to its amax (a few KB from L2), derives the scale and casts its share;
+//             CTA 0 writes amax, scale and scale_inv.
+struct QTensor {
+  const uint16_t* x;
+  uint8_t* q;
+  int64_t n;
+  float* scale;
+  float* scale_inv;
+  float* amax;
+  int32_t fmt;
+  int32_t pad;
+};
+struct QBatch {
+  QTensor t[TWEO_MAX_QUANT_BATCH];
+  int32_t count;
+  int32_t amax_grid;  // CTAs of kernel 1 = slots per tensor
+};
+constexpr int kMaxAmaxGrid = 2048;  // slots per tensor in the workspace
+
+__device__ __forceinline__ uint32_t cta_max(uint32_t m, uint32_t* part) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  __syncthreads();  // part[] may still be read from the previous use
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = m;
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) m = max(m, part[w]);
+  return m;
+}
+
+__global__ void __launch_bounds__(kThreads) amax_batch_kernel(const __grid_constant__ QBatch b, uint32_t* slots) {
+  __shared__ uint32_t part[kThreads / 32];
+#pragma unroll 1
+  for (int ti = 0; ti < b.count; ++ti) {
+    const int64_t n = b.t[ti].n;
+    const int64_t nvec = n >> 3;
+    const uint16_t* x = b.t[ti].x;
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    const int64_t stride = (int64_t)gridDim.x * kThreads * 4;
+    uint32_t m = 0;
+    for (int64_t base = (int64_t)blockIdx.x * kThreads * 4 + threadIdx.x; base < nvec; base += stride) {
+      uint4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        int64_t i = base + (int64_t)u * kThreads;
+        v[u] = i < nvec ? __ldg(xv + i) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        m = absmax_bits(m, v[u].x);
+        m = absmax_bits(m, v[u].y);
+        m = absmax_bits(m, v[u].z);
+        m = absmax_bits(m, v[u].w);
+      }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 8) {
+      int64_t i = (nvec << 3) + threadIdx.x;
+      if (i < n) m = absmax_bits(m, (uint32_t)x[i]);
+    }
+    m = cta_max(m, part);
+    if (threadIdx.x == 0) slots[ti * kMaxAmaxGrid + blockIdx.x] = m;
+  }
+}
+
+template <int FMT>
+__global__ void __launch_bounds__(kThreads) cast_batch_kernel(const __grid_constant__ QBatch b, const uint32_t* slots) {
+  __shared__ uint32_t part[kThreads / 32];
+#pragma unroll 1
+  for (int ti = 0; ti < b.count; ++ti) {
+    if (b.t[ti].fmt != FMT) continue;
+    uint32_t m = 0;
+    for (int k = threadIdx.x; k < b.amax_grid; k += kThreads) m = max(m, __ldcg(slots + ti * kMaxAmaxGrid + k));
+    m = cta_max(m, part);
+    const float amax = __uint_as_float(m << 16);  // non-negative bf16 pattern -> binary32
+    const float s = scale_from_amax(amax, FMT);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      *b.t[ti].amax = amax;
+      *b.t[ti].scale = s;
+      *b.t[ti].scale_inv = __fdiv_rn(1.0f, s);
+    }
+    const int64_t n = b.t[ti].n;
+    const int64_t n16 = n >> 4;
+    const uint16_t* x = b.t[ti].x;
+    uint8_t* q = b.t[ti].q;
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    uint4* qv = reinterpret_cast<uint4*>(q);
+    const int64_t stride = (int64_t)gridDim.x * kThreads * 2;
+    uint32_t sat = 0, mm = 0;
+    for (int64_t base = (int64_t)blockIdx.x * kThreads * 2 + threadIdx.x; base < n16; base += stride) {
+      uint4 v[2][2];
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        int64_t i = base + (int64_t)u * kThreads;
+        if (i < n16) {
+          v[u][0] = __ldcs(xv + 2 * i);
+          v[u][1] = __ldcs(xv + 2 * i + 1);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        int64_t i = base + (int64_t)u * kThreads;
+        if (i < n16) __stcs(qv + i, cast16<FMT>(v[u][0], v[u][1], s, sat, mm, false));
+      }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 16) {  // ragged tail: n % 16 elements
+      int64_t i = (n16 << 4) + threadIdx.x;
+      if (i < n) {
+        float v = __fmul_rn(bf16lo_to_f32((uint32_t)x[i]), s);
+        q[i] = (uint8_t)(cvt_fp8x2<FMT>(v, 0.0f) & 0xFFu);
+      }
+    }
+  }
+}
+
+int grid_for(int64_t work_items, int per_cta, int ctas_per_sm);
+
+// Launches the batched form for descs[idx[0..count)] (all CURRENT scaling, no saturation count).
+tweo_status_t launch_batch(const tweo_quant_desc_t* descs, const int* idx, int count, void* ws, cudaStream_t st) {
+  QBatch b;
+  b.count = count;
+  int64_t vec8 = 0, vec16[2] = {0, 0};
+  for (int i = 0; i < count; ++i) {
+    const tweo_quant_desc_t& d = descs[idx[i]];
+    b.t[i] = QTensor{d.x, d.q, d.n, d.scale, d.scale_inv, d.amax, d.fmt, 0};
+    vec8 += d.n >> 3;
+    vec16[d.fmt] += d.n >> 4;
+  }
+  b.amax_grid = grid_for(vec8, kThreads * 4, 8);
+  if (b.amax_grid > kMaxAmaxGrid) b.amax_grid = kMaxAmaxGrid;
+  uint32_t* slots = reinterpret_cast<uint32_t*>(ws);
+  amax_batch_kernel<<<b.amax_grid, kThreads, 0, st>>>(b, slots);
+  count_launch();
+  bool has[2] = {false, false};
+  for (int i = 0; i < count; ++i) has[b.t[i].fmt] = true;
+  if (has[TWEO_E4M3]) {
+    cast_batch_kernel<TWEO_E4M3><<<grid_for(vec16[TWEO_E4M3], kThreads * 2, 8), kThreads, 0, st>>>(b, slots);
+    count_launch();
+  }
+  if (has[TWEO_E5M2]) {
+    cast_batch_kernel<TWEO_E5M2><<<grid_for(vec16[TWEO_E5M2], kThreads * 2, 8), kThreads, 0, st>>>(b, slots);
+    count_launch();
+  }
+  return check_launch("quantize batch kernels");
+}
+
+constexpr size_t kBatchWsBytes = (size_t)TWEO_MAX_QUANT_BATCH * kMaxAmaxGrid * sizeof(uint32_t);  // 64 KB
+
 int grid_for(int64_t work_items, int per_cta, int ctas_per_sm) {
   int64_t want = (work_items + per_cta - 1) / per_cta;
   int64_t cap = (int64_t)sm_count() * ctas_per_sm;
@@ -152,35 +313,75 @@ int grid_for(int64_t work_items, int per_cta, int ctas_per_sm) {
   return (int)want;
 }
 
+tweo_status_t check_desc(const tweo_quant_desc_t& d) {
+  if (d.n < 0 || !d.scale || !d.scale_inv || !d.amax) return TWEO_ERR_INVALID_ARG;
+  if (d.n > 0 && (!d.x || !d.q)) return TWEO_ERR_INVALID_ARG;
+  if (d.fmt != TWEO_E4M3 && d.fmt != TWEO_E5M2) return TWEO_ERR_INVALID_ARG;
+  if (d.mode != TWEO_SCALE_CURRENT && d.mode != TWEO_SCALE_GIVEN) return TWEO_ERR_INVALID_ARG;
+  if (!aligned16(d.x) || !aligned16(d.q)) return TWEO_ERR_ALIGNMENT;
+  return TWEO_OK;
+}
+
+// One tensor as separate kernels: reset, amax (CURRENT only), cast.
+tweo_status_t launch_single(const tweo_quant_desc_t& d, cudaStream_t st) {
+  const bool given = d.mode == TWEO_SCALE_GIVEN;
+  init_kernel<<<1, 1, 0, st>>>(d.amax, d.sat_count, given ? d.scale : nullptr, d.scale_inv);
+  count_launch();
+  if (!given) {
+    amax_kernel<<<grid_for(d.n >> 3, kThreads * 4, 8), kThreads, 0, st>>>(d.x, d.n, d.amax);
+    count_launch();
+  }
+  const int grid = grid_for(d.n >> 4, kThreads * 2, 8);
+  if (d.fmt == TWEO_E4M3) {
+    if (given) cast_kernel<TWEO_E4M3, true><<<grid, kThreads, 0, st>>>(d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count);
+    else cast_kernel<TWEO_E4M3, false><<<grid, kThreads, 0, st>>>(d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count);
+  } else {
+    if (given) cast_kernel<TWEO_E5M2, true><<<grid, kThreads, 0, st>>>(d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count);
+    else cast_kernel<TWEO_E5M2, false><<<grid, kThreads, 0, st>>>(d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count);
+  }
+  count_launch();
+  return check_launch("tweo_quantize_per_tensor");
+}
+
+// Tensors with CURRENT scaling and no saturation count go through the batched kernels when a
+// workspace is there; the others (GIVEN scale: one pass anyway; saturation count: needs a zeroed
+// counter) are launched one by one.
+tweo_status_t quantize_many(const tweo_quant_desc_t* descs, int count, void* ws, size_t ws_bytes, cudaStream_t st) {
+  for (int i = 0; i < count; ++i) {
+    tweo_status_t s = check_desc(descs[i]);
+    if (s != TWEO_OK) return s;
+  }
+  const bool have_ws = ws && ws_bytes >= kBatchWsBytes && aligned16(ws);
+  int idx[TWEO_MAX_QUANT_BATCH];
+  int nb = 0;
+  for (int i = 0; i < count; ++i) {
+    if (have_ws && descs[i].mode == TWEO_SCALE_CURRENT && !descs[i].sat_count) {
+      idx[nb++] = i;
+    } else {
+      tweo_status_t s = launch_single(descs[i], st);
+      if (s != TWEO_OK) return s;
+    }
+  }
+  if (nb > 0) return launch_batch(descs, idx, nb, ws, st);
+  return TWEO_OK;
+}
+
 }  // namespace
+
+namespace tweo_detail {
+size_t quantize_workspace_bytes() { return kBatchWsBytes; }
+}
 
 extern "C" tweo_status_t tweo_quantize_per_tensor(const uint16_t* x, int64_t n, int32_t fmt, int32_t mode,
                                                   float* scale, float* scale_inv, float* amax, uint8_t* q,
                                                   uint32_t* sat_count, void* ws, size_t ws_bytes, void* stream) {
-  (void)ws;
-  (void)ws_bytes;
-  if (n < 0 || !scale || !scale_inv || !amax) return TWEO_ERR_INVALID_ARG;
-  if (n > 0 && (!x || !q)) return TWEO_ERR_INVALID_ARG;
-  if (fmt != TWEO_E4M3 && fmt != TWEO_E5M2) return TWEO_ERR_INVALID_ARG;
-  if (mode != TWEO_SCALE_CURRENT && mode != TWEO_SCALE_GIVEN) return TWEO_ERR_INVALID_ARG;
-  if (!aligned16(x) || !aligned16(q)) return TWEO_ERR_ALIGNMENT;
-  cudaStream_t st = (cudaStream_t)stream;
-  const bool given = mode == TWEO_SCALE_GIVEN;
+  tweo_quant_desc_t d{x, n, fmt, mode, scale, scale_inv, amax, q, sat_count};
+  return quantize_many(&d, 1, ws, ws_bytes, (cudaStream_t)stream);
+}
 
-  init_kernel<<<1, 1, 0, st>>>(amax, sat_count, given ? scale : nullptr, scale_inv);
-  count_launch();
-  if (!given) {
-    amax_kernel<<<grid_for(n >> 3, kThreads * 4, 8), kThreads, 0, st>>>(x, n, amax);
-    count_launch();
-  }
-  const int grid = grid_for(n >> 4, kThreads * 2, 8);
-  if (fmt == TWEO_E4M3) {
-    if (given) cast_kernel<TWEO_E4M3, true><<<grid, kThreads, 0, st>>>(x, n, scale, scale_inv, amax, q, sat_count);
-    else cast_kernel<TWEO_E4M3, false><<<grid, kThreads, 0, st>>>(x, n, scale, scale_inv, amax, q, sat_count);
-  } else {
-    if (given) cast_kernel<TWEO_E5M2, true><<<grid, kThreads, 0, st>>>(x, n, scale, scale_inv, amax, q, sat_count);
-    else cast_kernel<TWEO_E5M2, false><<<grid, kThreads, 0, st>>>(x, n, scale, scale_inv, amax, q, sat_count);
-  }
-  count_launch();
-  return check_launch("tweo_quantize_per_tensor");
+extern "C" tweo_status_t tweo_quantize_per_tensor_batch(const tweo_quant_desc_t* descs, int32_t count, void* ws,
+                                                        size_t ws_bytes, void* stream) {
+  if (!descs || count < 1 || count > TWEO_MAX_QUANT_BATCH) return TWEO_ERR_INVALID_ARG;
+  if (ws && !aligned16(ws)) return TWEO_ERR_ALIGNMENT;
+  return quantize_many(descs, count, ws, ws_bytes, (cudaStream_t)stream);
 }

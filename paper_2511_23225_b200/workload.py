@@ -30,9 +30,9 @@ class LinearBuffers:
         self.w = torch.empty((N, K), dtype=bf, device=device)
         self.dy = torch.empty((M, N), dtype=bf, device=device)
         sc = torch.zeros(12, dtype=f32, device=device)
-        mk = lambda t, i: tw.Quantized(torch.empty(t.shape, dtype=u8, device=device), sc[i:i + 1],
-                                       sc[i + 1:i + 2], sc[i + 2:i + 3], None, 0)
-        self.qx, self.qw, self.qdy = mk(self.x, 0), mk(self.w, 3), mk(self.dy, 6)
+        mk = lambda t, i, fmt: tw.Quantized(torch.empty(t.shape, dtype=u8, device=device), sc[i:i + 1],
+                                            sc[i + 1:i + 2], sc[i + 2:i + 3], None, fmt)
+        self.qx, self.qw, self.qdy = mk(self.x, 0, tw.E4M3), mk(self.w, 3, tw.E4M3), mk(self.dy, 6, tw.E5M2)
         self.y = torch.empty((M, N), dtype=bf, device=device)
         self.dx = torch.empty((M, K), dtype=bf, device=device)
         self.dw = torch.empty((N, K), dtype=bf, device=device)
@@ -57,7 +57,10 @@ class BlockStep:
         self.a = [torch.empty((self.M, self.cfg.d), dtype=torch.bfloat16, device=device) for _ in range(self.n_blocks)]
         self.ga = [torch.empty_like(t) for t in self.a]
         self.loss_ws = tw.new_workspace(tw.OP_LOSS, n, self.n_blocks, device=device)
-        self.gemm_ws = None
+        self.quant_ws = tw.new_workspace(tw.OP_QUANTIZE, device=device)
+        self.gemm_ws = tw.new_workspace(tw.OP_LINEAR_WGRAD, device=device)
+        for lb in self.linears:
+            lb.qdy.fmt = grad_fmt
         self.loss = None
         self.host = None
         self.tau, self.eps, self.p, self.lam = 3.0, 1e-6, 4.0, 0.01
@@ -95,9 +98,8 @@ class BlockStep:
 
     # ---- the step
     def quantize_all(self, lb: LinearBuffers):
-        tw.quantize_per_tensor(lb.x, tw.E4M3, tw.SCALE_CURRENT, out=lb.qx)
-        tw.quantize_per_tensor(lb.w, tw.E4M3, tw.SCALE_CURRENT, out=lb.qw)
-        tw.quantize_per_tensor(lb.dy, self.grad_fmt, tw.SCALE_CURRENT, out=lb.qdy)
+        # X, W (E4M3) and dY (E5M2), each with its own per-tensor scale, in one launch
+        tw.quantize_per_tensor_batch([lb.x, lb.w, lb.dy], [lb.qx, lb.qw, lb.qdy], ws=self.quant_ws)
 
     def gemms(self, lb: LinearBuffers):
         tw.fp8_linear_fwd(lb.qx.q, lb.qw.q, lb.qx.scale_inv, lb.qw.scale_inv, y=lb.y, ws=self.gemm_ws)

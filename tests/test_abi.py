@@ -28,11 +28,12 @@ def test_host_side_helpers_without_a_gpu():
     assert L.tweo_version() >= 100
     assert L.tweo_status_string(0) == b"ok"
     assert b"align" in L.tweo_status_string(3)
-    assert L.tweo_workspace_bytes(binding.OP_QUANTIZE, 1 << 20, 0, 0) == 0
+    assert L.tweo_workspace_bytes(binding.OP_QUANTIZE, 1 << 20, 0, 0) == 65536
     assert L.tweo_workspace_bytes(binding.OP_LOSS, 1 << 20, 12, 0) >= 256 + 8 * 12
     # argument validation happens on the host, before any CUDA call
     assert L.tweo_loss_fwd_bwd(None, 1, 8, 3.0, 1e-6, 4.0, 1.0, None, None, None, 0, None, 0, None) == 1
     assert L.tweo_quantize_per_tensor(None, -1, 0, 0, None, None, None, None, None, None, 0, None) == 1
+    assert L.tweo_quantize_per_tensor_batch(None, 1, None, 0, None) == 1
     assert L.tweo_fp8_linear_fwd(None, 0, None, 0, None, None, None, 0, 1, 1, 1, 0, 0, None, None, 0, None) == 1
 
 

@@ -57,13 +57,16 @@ QUANT_CASES = [
 ]
 
 
+@pytest.mark.parametrize("one_kernel", [False, True], ids=["no_ws", "ws"])
 @pytest.mark.parametrize("fmt", [E4M3, E5M2])
 @pytest.mark.parametrize("name,make", QUANT_CASES, ids=[c[0] for c in QUANT_CASES])
-def test_quantize_current_bit_exact(tw, fmt, name, make):
+def test_quantize_current_bit_exact(tw, fmt, name, make, one_kernel):
     bits = make()
     ref = orc.quantize_per_tensor_current(bits, fmt)
-    out = tw.quantize_per_tensor(to_gpu_bf16(bits), fmt, tw.SCALE_CURRENT, count_saturated=True)
+    ws = tw.new_workspace(tw.OP_QUANTIZE) if one_kernel else None
+    out = tw.quantize_per_tensor(to_gpu_bf16(bits), fmt, tw.SCALE_CURRENT, count_saturated=True, ws=ws)
     torch.cuda.synchronize()
+
     assert f32_bits(out.amax) == np_f32_bits(ref["amax"])
     assert f32_bits(out.scale) == np_f32_bits(ref["scale"])
     assert f32_bits(out.scale_inv) == np_f32_bits(ref["scale_inv"])
@@ -71,14 +74,16 @@ def test_quantize_current_bit_exact(tw, fmt, name, make):
     assert int(out.sat_count.item()) == ref["sat_count"]
 
 
+@pytest.mark.parametrize("one_kernel", [False, True], ids=["no_ws", "ws"])
 @pytest.mark.parametrize("fmt", [E4M3, E5M2])
-def test_quantize_given_scale_saturates_and_reports_amax(tw, fmt):
+def test_quantize_given_scale_saturates_and_reports_amax(tw, fmt, one_kernel):
     bits = synth.normal_with_extreme_outliers_bf16(12, (700, 129))
     # a static scale calibrated for |x| <= 6: the planted outliers must clip to +-max
     scale = np.float32(orc.fp8_max(fmt) / 6.0)
     q_ref, sat_ref = orc.quantize_bf16(bits, fmt, scale)
     s = torch.tensor([scale], dtype=torch.float32, device="cuda")
-    out = tw.quantize_per_tensor(to_gpu_bf16(bits), fmt, tw.SCALE_GIVEN, scale=s, count_saturated=True)
+    ws = tw.new_workspace(tw.OP_QUANTIZE) if one_kernel else None
+    out = tw.quantize_per_tensor(to_gpu_bf16(bits), fmt, tw.SCALE_GIVEN, scale=s, count_saturated=True, ws=ws)
     torch.cuda.synchronize()
     assert np.array_equal(out.q.cpu().numpy(), q_ref)
     assert int(out.sat_count.item()) == sat_ref and sat_ref > 0
@@ -103,6 +108,44 @@ def test_quantize_degenerate_inputs(tw):
     torch.cuda.synchronize()
     assert f32_bits(out.amax) == np_f32_bits(ref["amax"])
     assert np.array_equal(out.q.cpu().numpy(), ref["q"])
+
+
+def test_quantize_batch_matches_oracle_per_tensor(tw):
+    """X, W (E4M3, current scaling), dY (E5M2, current) and a static-scale activation in ONE launch:
+    every tensor gets exactly what its own per-tensor call gives; twice on the same workspace."""
+    x, w, dy = synth.linear_inputs(2, 1, M=1536)                   # outlier channel x500 in X
+    a = synth.normal_with_extreme_outliers_bf16(15, (333, 77))     # ragged size, saturates under the static scale
+    e = np.zeros((0,), dtype=np.uint16)                            # an empty tensor in the batch
+    bits = [x, w, dy, a, e]
+    fmts = [E4M3, E4M3, E5M2, E4M3, E5M2]
+    modes = [tw.SCALE_CURRENT, tw.SCALE_CURRENT, tw.SCALE_CURRENT, tw.SCALE_GIVEN, tw.SCALE_CURRENT]
+    static = np.float32(448.0 / 6.0)
+    ws = tw.new_workspace(tw.OP_QUANTIZE)
+    ws.fill_(0xA5)                                                 # its contents must not matter
+    xs = [to_gpu_bf16(b) for b in bits]
+    for _ in range(2):
+        outs = []
+        for b, f, m in zip(xs, fmts, modes):
+            sc = torch.zeros(4, dtype=torch.float32, device="cuda")
+            if m == tw.SCALE_GIVEN:
+                sc[0] = float(static)
+            outs.append(tw.Quantized(torch.empty(b.shape, dtype=torch.uint8, device="cuda"), sc[0:1], sc[1:2], sc[2:3],
+                                     torch.full((1,), 77, dtype=torch.int32, device="cuda"), f))
+        tw.quantize_per_tensor_batch(xs, outs, modes, ws=ws)
+        torch.cuda.synchronize()
+        for b, f, m, o in zip(bits, fmts, modes, outs):
+            if m == tw.SCALE_GIVEN:
+                q_ref, sat_ref = orc.quantize_bf16(b, f, static)
+                assert sat_ref > 0
+                ref = {"q": q_ref, "sat_count": sat_ref, "amax": orc.amax_bf16(b), "scale": static,
+                       "scale_inv": np.float32(1.0) / static}
+            else:
+                ref = orc.quantize_per_tensor_current(b, f)
+            assert np.array_equal(o.q.cpu().numpy(), ref["q"])
+            assert f32_bits(o.amax) == np_f32_bits(ref["amax"])
+            assert f32_bits(o.scale) == np_f32_bits(ref["scale"])
+            assert f32_bits(o.scale_inv) == np_f32_bits(ref["scale_inv"])
+            assert int(o.sat_count.item()) == ref["sat_count"]
 
 
 def test_quantize_all_bf16_patterns_both_formats(tw):
