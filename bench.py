@@ -13,9 +13,11 @@ and gradient on the block output.  Prints ONE JSON line (rank 0).
                scaling: every rank runs its own token shard, no data-path collective).
   e2e          same metric with the step's inputs copied from pinned host memory and
                the loss read back inside the timed region.
-  roofline     dominant kernel family (largest share of the instrumented step time),
-               algorithmic flops or bytes / CUDA-event duration, against the measured
-               peak in MEASURED_PEAKS.json (fallback stated if absent).
+  roofline     dominant kernel family (largest share of the step): its launches of one
+               step replayed alone from a CUDA graph between two events; algorithmic
+               flops or bytes / that duration, against the measured peak in
+               MEASURED_PEAKS.json (fallback stated if absent).
+  other_workloads  short runs of the other training configs (N=1), same measurements.
   cpu_baseline the CPU oracle, as it stands, timed on a bounded sample (N=1, rank 0).
 
 `--impl reference` times the CPU oracle alone (there is no reference code for this
@@ -175,11 +177,127 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- CUDA arm
+def _graph_of(torch, stream, fn):
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(g, stream=stream):
+            fn()
+    torch.cuda.synchronize()
+    return g
+
+
+def _time_replays(torch, graph, reps):
+    """ms per replay, CUDA events on the current stream around `reps` back-to-back replays."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    graph.replay()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def family_breakdown(torch, tw, bs, side, reps):
+    """Times each kernel family of the step on its own: the family's launches of one step are
+    captured into a CUDA graph and replayed back to back between two events (so no host gaps
+    and no other family's kernels inside the timed region)."""
+    def all_quantize():
+        for lb in bs.linears:
+            bs.quantize_all(lb)
+
+    def all_gemms():
+        for lb in bs.linears:
+            bs.gemms(lb)
+
+    n_el = sum(lb.x.numel() + lb.w.numel() + lb.dy.numel() for lb in bs.linears)
+    n_a = sum(t.numel() for t in bs.a)
+    fams = {
+        "quantize": (all_quantize, 5.0 * n_el, "GB/s"),           # 2 + 2 read, 1 written per element
+        "gemm": (all_gemms, float(bs.flops_per_step), "TFLOP/s"),
+        "tweo_loss": (bs.tweo, 4.0 * n_a, "GB/s"),                # 2 read + 2 written per element
+    }
+    out = {}
+    for name, (fn, work, unit) in fams.items():
+        c0 = tw.launch_count()
+        g = _graph_of(torch, side, fn)
+        launches = tw.launch_count() - c0
+        ms = _time_replays(torch, g, reps)
+        rate = work / (ms * 1e-3)
+        out[name] = {"ms_per_step": ms, "launches_per_step": int(launches), "avg_launch_us": 1e3 * ms / max(1, launches),
+                     "achieved": rate / 1e12 if unit == "TFLOP/s" else rate / 1e9, "unit": unit}
+    tot = sum(v["ms_per_step"] for v in out.values())
+    for v in out.values():
+        v["share"] = v["ms_per_step"] / tot
+    return out
+
+
+def measure_workload(torch, tw, cfg_idx, steps, warmup, world, barrier, want_e2e, e2e_steps, local):
+    from paper_2511_23225_b200.workload import BlockStep
+    bs = BlockStep(cfg_idx)
+    bs.make_host_inputs()
+    bs.upload()
+    torch.cuda.synchronize()
+    for _ in range(max(3, warmup)):
+        bs.step()
+    barrier()
+    if tw.read_device_status() != 0:
+        raise SystemExit("device status reports an expired wait")
+
+    # The step is a few dozen short kernels; issued one by one from Python the host is the bottleneck,
+    # so the launch sequence is captured once into a CUDA graph and replayed (same kernels, same order).
+    host_loss = torch.empty(1, dtype=torch.float32).pin_memory()
+    side = torch.cuda.Stream()
+    c0 = tw.launch_count()
+    step_graph = _graph_of(torch, side, bs.step)
+    launches_per_step = tw.launch_count() - c0
+    for _ in range(3):
+        step_graph.replay()
+    barrier()
+
+    # ---- timed region: K steps, inputs resident in HBM
+    sampler = ClockSampler(local)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    e0.record()
+    for _ in range(steps):
+        step_graph.replay()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    if tw.read_device_status() != 0:
+        raise SystemExit("device status reports an expired wait")
+    res = {"bs": bs, "ms_per_step": ms / steps, "launches_per_step": int(launches_per_step), "clocks": clocks}
+
+    # ---- end to end: pinned host inputs -> device, step, loss back to host, every step
+    if want_e2e:
+        def e2e():
+            bs.upload()
+            bs.step()
+            host_loss.copy_(bs.loss, non_blocking=True)
+        e2e_graph = _graph_of(torch, side, e2e)
+        for _ in range(2):
+            e2e_graph.replay()
+        barrier()
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_graph.replay()
+            torch.cuda.current_stream().synchronize()   # the host reads the loss every step
+        e1.record()
+        barrier()
+        res["e2e_ms_per_step"] = e0.elapsed_time(e1) / e2e_steps
+        res["loss"] = float(host_loss.item())
+    res["kernels"] = family_breakdown(torch, tw, bs, side, max(5, min(steps, 50)))
+    return res
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
     from paper_2511_23225_b200 import binding as tw
-    from paper_2511_23225_b200.workload import BlockStep
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -193,162 +311,99 @@ def run_cuda(args):
     cfg_idx = int(args.workload[3:])
     peaks = load_peaks()
 
-    bs = BlockStep(cfg_idx)
-    bs.make_host_inputs()
-    bs.upload()
-    torch.cuda.synchronize()
-
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(3, args.warmup)):
-        bs.step()
-    barrier()
-    if tw.read_device_status() != 0:
-        raise SystemExit("device status reports an expired wait")
+    def max_over_ranks(v):
+        if world > 1:
+            t = torch.tensor([v], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return v
 
-    # The step is ~50 short kernels; issued one by one from Python the host is the bottleneck, so the
-    # launch sequence is captured once into a CUDA graph and replayed (same kernels, same order).
-    host_loss = torch.empty(1, dtype=torch.float32).pin_memory()
-    side = torch.cuda.Stream()
-    step_graph, e2e_graph = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
-    use_graph = not args.eager
-    launches_per_step = None
-    if use_graph:
-        with torch.cuda.stream(side):
-            c0 = tw.launch_count()
-            with torch.cuda.graph(step_graph, stream=side):
-                bs.step()
-            launches_per_step = tw.launch_count() - c0
-            with torch.cuda.graph(e2e_graph, stream=side):
-                bs.upload()
-                bs.step()
-                host_loss.copy_(bs.loss, non_blocking=True)
-        torch.cuda.synchronize()
-        run_step, run_e2e = step_graph.replay, e2e_graph.replay
-        for _ in range(3):
-            run_step()
-    else:
-        def run_e2e():
-            bs.upload()
-            bs.step()
-            host_loss.copy_(bs.loss, non_blocking=True)
-        run_step = bs.step
-    barrier()
-
-    # ---- timed region: K steps, inputs resident in HBM
-    sampler = ClockSampler(local)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = tw.launch_count()
-    barrier()
-    sampler.start()
-    e0.record()
-    for _ in range(args.steps):
-        run_step()
-    e1.record()
-    barrier()
-    clocks = sampler.stop()
-    ms = e0.elapsed_time(e1)
-    launches = launches_per_step * args.steps if use_graph else tw.launch_count() - launches0
-    if tw.read_device_status() != 0:
-        raise SystemExit("device status reports an expired wait")
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    ms_per_step = ms / args.steps
-    value = world * bs.flops_per_step / (ms_per_step * 1e-3) / 1e12
-
-    # ---- end to end: pinned host inputs -> device, step, loss back to host, every step
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    for _ in range(2):
-        run_e2e()
-    barrier()
-    e0.record()
-    for _ in range(e2e_steps):
-        run_e2e()
-        torch.cuda.current_stream().synchronize()   # the host reads the loss every step
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * bs.flops_per_step / (e2e_ms / e2e_steps * 1e-3) / 1e12
-    loss_value = float(host_loss.item())
+    r = measure_workload(torch, tw, cfg_idx, args.steps, args.warmup, world, barrier, True, e2e_steps, local)
+    bs = r["bs"]
+    ms_per_step = max_over_ranks(r["ms_per_step"])
+    e2e_ms = max_over_ranks(r["e2e_ms_per_step"])
+    value = world * bs.flops_per_step / (ms_per_step * 1e-3) / 1e12
+    e2e_value = world * bs.flops_per_step / (e2e_ms * 1e-3) / 1e12
+    kernels = r["kernels"]
 
-    # ---- instrumented steps: CUDA events around every library call, per kernel family
-    fam = {"quantize": [0.0, 0, 0.0], "gemm": [0.0, 0, 0.0], "tweo_loss": [0.0, 0, 0.0]}  # ms, calls, work
-    inst_steps = max(1, min(args.steps, 30))
-    pairs = []
-
-    def timed(name, work, fn):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        fn()
-        b.record()
-        pairs.append((name, work, a, b))
-
-    for _ in range(inst_steps):
-        for lb in bs.linears:
-            n_el = lb.x.numel() + lb.w.numel() + lb.dy.numel()
-            timed("quantize", 5.0 * n_el, lambda: bs.quantize_all(lb))          # 2 + 2 + 1 bytes per element
-            timed("gemm", float(lb.flops), lambda: bs.gemms(lb))
-        n_a = sum(t.numel() for t in bs.a)
-        timed("tweo_loss", 4.0 * n_a, bs.tweo)                                    # 2 read + 2 written
-    torch.cuda.synchronize()
-    for name, work, a, b in pairs:
-        fam[name][0] += a.elapsed_time(b)
-        fam[name][1] += 1
-        fam[name][2] += work
-    total_inst = sum(v[0] for v in fam.values())
-    kernels = {}
-    for name, (tms, calls, work) in fam.items():
-        rate = work / (tms * 1e-3) if tms > 0 else 0.0
-        kernels[name] = {"share": tms / total_inst, "ms_per_step": tms / inst_steps,
-                         "achieved": rate / 1e12 if name == "gemm" else rate / 1e9,
-                         "unit": "TFLOP/s" if name == "gemm" else "GB/s"}
-    dom = max(fam, key=lambda k: fam[k][0])
-    fp8_peak = 2.0 * peaks["bf16_sustained"]  # FP8 dense = 2x bf16 (nominal ratio) on the sustained bf16 figure
+    # Roofline of the dominant kernel family.  FP8 dense peak = 2 x the measured bf16 figure (nominal
+    # ratio); the burst figure, because the family is timed alone in short replays.
+    dom = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    fp8_burst, fp8_sustained = 2.0 * peaks["bf16"], 2.0 * peaks["bf16_sustained"]
+    of = "of measured" if peaks["source"] == "measured" else "of fallback"
     if dom == "gemm":
-        roof = {"bound": "tensor", "achieved": kernels["gemm"]["achieved"], "peak": fp8_peak, "unit": "TFLOP/s"}
+        roof = {"bound": "tensor", "achieved": kernels["gemm"]["achieved"], "peak": fp8_burst, "unit": "TFLOP/s",
+                "peak_source": of + " (2 x burst bf16)"}
     else:
-        roof = {"bound": "hbm", "achieved": kernels[dom]["achieved"], "peak": peaks["hbm"], "unit": "GB/s"}
+        roof = {"bound": "hbm", "achieved": kernels[dom]["achieved"], "peak": peaks["hbm"], "unit": "GB/s",
+                "peak_source": of + " (copy bandwidth)"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = None
     roof["kernel"] = dom
-    roof["peak_source"] = ("of measured" if peaks["source"] == "measured" else "of fallback") + \
-        (" (2 x sustained bf16)" if dom == "gemm" else " (copy bandwidth)")
+    roof["avg_launch_us"] = kernels[dom]["avg_launch_us"]
+
+    workload_cfg = {"workload": workload_name(cfg_idx), "tokens_per_gpu": bs.M,
+                    "linears": [f"{l.name}:{l.K}x{l.N}" for l in bs.cfg.linears], "tweo_blocks": bs.n_blocks,
+                    "parallelism": f"replicas x{world} (token shards, no data-path collective)",
+                    "l2": f"working set {bs.working_set_bytes() / 1e6:.0f} MB per step > 126 MB L2, no flush",
+                    "launch": "cuda graph replay of one captured step"}
+    h2d = bs.h2d_bytes()
+    loss_value = r["loss"]
+    main_clocks = r["clocks"]
+    launches_per_step = r["launches_per_step"]
+    del bs, r
+    torch.cuda.empty_cache()
+
+    # ---- the other training configurations, short runs (context for the large shapes)
+    others = {}
+    if world == 1 and args.also:
+        for name in args.also.split(","):
+            name = name.strip()
+            if not name or name == args.workload:
+                continue
+            o = measure_workload(torch, tw, int(name[3:]), args.also_steps, 3, 1, barrier, False, 0, local)
+            obs = o["bs"]
+            k = o["kernels"]
+            others[name] = {
+                "workload": workload_name(int(name[3:])), "steps": args.also_steps, "ms_per_step": o["ms_per_step"],
+                "value": obs.flops_per_step / (o["ms_per_step"] * 1e-3) / 1e12, "unit": UNIT,
+                "gemm_tflops": k["gemm"]["achieved"], "gemm_frac_of_fp8_burst_peak": k["gemm"]["achieved"] / fp8_burst,
+                "gemm_pct_of_fp8_datasheet_peak": 100.0 * k["gemm"]["achieved"] / FP8_DATASHEET_TFLOPS,
+                "quantize_gbs": k["quantize"]["achieved"], "tweo_loss_gbs": k["tweo_loss"]["achieved"],
+                "shares": {n: v["share"] for n, v in k.items()}, "clocks": o["clocks"]}
+            del obs, o
+            torch.cuda.empty_cache()
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp8_e4m3xe5m2_fp32acc", "data": "synthetic",
-            "config": {"workload": workload_name(cfg_idx), "tokens_per_gpu": bs.M,
-                       "linears": [f"{l.name}:{l.K}x{l.N}" for l in bs.cfg.linears], "tweo_blocks": bs.n_blocks,
-                       "parallelism": f"replicas x{world} (token shards, no data-path collective)",
-                       "l2": f"working set {bs.working_set_bytes() / 1e6:.0f} MB per step > 126 MB L2, no flush",
-                       "launch": "cuda graph replay of one captured step" if use_graph else "eager"},
+            "config": workload_cfg,
             "pct_of_fp8_datasheet_peak": 100.0 * value / world / FP8_DATASHEET_TFLOPS,
-            "pct_of_fp8_measured_peak": 100.0 * value / world / fp8_peak,
+            "pct_of_fp8_measured_peak": 100.0 * value / world / fp8_sustained,
             "gemm_only_tflops": world * kernels["gemm"]["achieved"],
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bs.h2d_bytes(), "d2h_bytes_per_step": 4,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4,
                     "steps": e2e_steps},
-            "gpu_launches": int(launches),
-            "clocks": clocks,
+            "gpu_launches": int(launches_per_step * args.steps),
+            "clocks": main_clocks,
             "roofline": roof,
             "kernels": kernels,
             "tweo_loss": loss_value,
         }
+        if others:
+            line["other_workloads"] = others
         if world == 1 and not args.no_cpu_baseline:
             f, t = oracle_sample_step(cfg_idx, args.cpu_rows)
             line["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-                                    "sample": f"first {args.cpu_rows} of {bs.M} tokens of every linear (full K,N) "
-                                              f"+ TWEO on {args.cpu_rows} rows; {t:.1f} s"}
+                                    "sample": f"first {args.cpu_rows} of {workload_cfg['tokens_per_gpu']} tokens of every "
+                                              f"linear (full K,N) + TWEO on {args.cpu_rows} rows; {t:.1f} s"}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -366,7 +421,8 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=4096)
     ap.add_argument("--ref-rows", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--eager", action="store_true", help="issue every call from Python instead of replaying a CUDA graph")
+    ap.add_argument("--also", default="cfg4", help="comma-separated other configs to run briefly (N=1 only); '' for none")
+    ap.add_argument("--also-steps", type=int, default=20)
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps > 50:
