@@ -1,0 +1,105 @@
+// Definitions shared by the FP8 GEMM kernels: tile constants, the kernel parameter block, the
+// workspace layout, the tile numbering and the work scheduler (whole tiles + tiles split along
+// the contraction).  Not part of the public ABI.
+#pragma once
+
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace tweo_detail {
+
+constexpr int BM = 128;      // rows of D per CTA tile = tcgen05 M per CTA (lanes of tensor memory)
+constexpr int BK = 128;      // contraction bytes per stage = one 128-byte swizzle span
+constexpr int UMMA_K = 32;   // contraction per instruction for 8-bit operands
+constexpr int kThreads = 192;
+
+struct GemmParams {
+  void* d;
+  int64_t ldd;
+  int32_t Md, Nd, Kc;
+  int32_t tiles_m, tiles_n, k_blocks;
+  int32_t raster_g;    // tiles are numbered in bands of raster_g tile rows (see tile_coords)
+  const float* sa_inv;
+  const float* sb_inv;
+  int32_t out_f32;     // 0: bf16 out, 1: fp32 out
+  int32_t accumulate;  // fp32 out only
+  float* out_amax;
+  uint8_t* out_q;
+  int64_t ldq;
+  int32_t q_fmt;
+  const float* q_scale;
+  uint32_t idesc;
+  // stream-K: tiles [0, sk_tiles) are split along the contraction, the rest dealt whole
+  int32_t sk_tiles;
+  float* sk_partials;   // [grid][BM*BN] raw accumulators of shares that do not own their tile
+  uint32_t* sk_flags;   // [grid][4] per epilogue warp: == epoch once the share is written
+  uint32_t* sk_counters;  // CTA-pair kernel: [sk_tiles][2][4] tickets per (tile, CTA of the pair, epilogue warp)
+  uint32_t epoch;
+};
+
+// Workspace layout of the linear calls (bytes from the workspace base):
+//   [0, 4096)       flags of the single-CTA kernel's split tiles (4 words per CTA)
+//   [4096, 12288)   ticket counters of the CTA-pair kernel's split tiles (8 words per tile)
+//   [12288, ...)    parked fp32 accumulators: 256 KB per SM
+constexpr size_t kWsCountersOffset = 4096;
+constexpr size_t kWsPartialsOffset = 12288;
+constexpr size_t kWsPartialBytesPerSm = 256 * 1024;
+
+// Tile index -> tile coordinates.  Tiles are numbered band by band: a band is raster_g tile
+// rows high and is walked column by column, so the tiles in flight at any time cover a
+// compact block (about raster_g rows x workers/raster_g columns) and the rows of A and the
+// columns of B they share are re-read from L2 while they are still hot, instead of every wave
+// sweeping all of A.
+__device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& tm, int& tn) {
+  const int per_band = p.raster_g * p.tiles_n;
+  const int band = tile / per_band;
+  const int first = band * p.raster_g;
+  const int rows = min(p.raster_g, p.tiles_m - first);
+  const int in = tile - band * per_band;
+  tn = in / rows;
+  tm = first + in - tn * rows;
+}
+
+// The work list of one CTA, identical in the three roles (producer, MMA, epilogue).
+struct Sched {
+  int64_t u, u_end;   // stream-K units (tile * k_blocks + k-block) still to do
+  int dp_tile, num_tiles, k_blocks, grid;
+  __device__ Sched(const GemmParams& p, int cta, int grid_)
+      : dp_tile(p.sk_tiles + cta), num_tiles(p.tiles_m * p.tiles_n), k_blocks(p.k_blocks), grid(grid_) {
+    const int64_t total = (int64_t)p.sk_tiles * p.k_blocks;
+    u = total * cta / grid_;
+    u_end = total * (cta + 1) / grid_;
+  }
+  // first unit of CTA j's stream-K share
+  __device__ static int64_t share_begin(const GemmParams& p, int j, int grid_) {
+    return (int64_t)p.sk_tiles * p.k_blocks * j / grid_;
+  }
+  __device__ bool next(int& tile, int& kb0, int& kb1) {
+    if (u < u_end) {
+      tile = (int)(u / k_blocks);
+      kb0 = (int)(u - (int64_t)tile * k_blocks);
+      const int64_t len = min((int64_t)(k_blocks - kb0), u_end - u);
+      kb1 = kb0 + (int)len;
+      u += len;
+      return true;
+    }
+    if (dp_tile < num_tiles) {
+      tile = dp_tile;
+      kb0 = 0;
+      kb1 = k_blocks;
+      dp_tile += grid;
+      return true;
+    }
+    return false;
+  }
+};
+
+// ----------------------------------------------------------------- epilogue helpers
+template <int FMT>
+__device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d) {
+  return cvt_fp8x2<FMT>(a, b) | (cvt_fp8x2<FMT>(c, d) << 16);
+}
+
+
+}  // namespace tweo_detail

@@ -1,0 +1,394 @@
+// CTA-pair FP8 GEMM kernel (included by the translation units that instantiate it).
+// Two CTAs of a cluster (adjacent SMs) compute one 256 x 256 tile with tcgen05
+// cta_group::2 instructions: each CTA stages its own 128 rows of A and only HALF of the
+// B tile (128 of the 256 output columns), the pair's tensor cores read both halves, and
+// each CTA's tensor memory receives the accumulator of its own 128 rows.  Per SM this
+// moves 32 KB of operands per 128-deep contraction block instead of 48 KB, which is what
+// lifts the kernel off the shared-memory fill limit.  Roles per CTA are those of the
+// single-CTA kernel; only CTA 0 (the leader) issues MMAs.  Barriers:
+//   full[s]    leader only : leader's producer arrives (+ expected bytes of BOTH CTAs' loads)
+//   empty[s]   each CTA    : leader's MMA thread commits to its own and to the peer's
+//   tfull[a]   each CTA    : same, once a tile's accumulator is complete
+//   tempty[a]  leader only : 4 epilogue warps of each CTA arrive (the peer's remotely)
+#pragma once
+
+#include <cuda.h>
+
+#include "gemm_common.cuh"
+#include "tc_ptx.cuh"
+
+namespace tweo_detail {
+
+// A share of the pair kernel that covers only part of a split tile.  Parks this warp's
+// 32 x 256 block of the raw accumulator in the workspace ([column][row], so every store is
+// one full line), hands the accumulator back to the MMA warp and takes a ticket; the warp
+// that draws the last ticket of the tile adds the parked blocks of ALL shares in share order
+// (= ascending k, whoever arrived last, so the sum does not depend on timing) and stores the
+// result.  Nobody waits for anybody.  Kept out of line: it is rare and register-hungry.
+constexpr size_t kPairCtaFloats = 128 * 256;   // one CTA's half of a parked 256 x 256 accumulator
+constexpr size_t kPairWarpFloats = 32 * 256;   // one epilogue warp's block of it
+
+template <bool OUT_F32>
+__device__ __noinline__ float pair_partial_share(const GemmParams& p, const CUtensorMap* tmap_d, int tile, int kb0,
+                                                int pair, int num_pairs, int rank, int wslot,
+                                                uint32_t tacc, uint32_t tempty_leader, float alpha, float qs,
+                                                uint32_t epi_base, uint32_t it, int lane, int row0, int n0) {
+  constexpr int CH = OUT_F32 ? 32 : 64;
+  constexpr uint32_t EPI_BUF = 32 * 128;
+  float run_amax = 0.0f;
+  float* slot = p.sk_partials + ((size_t)(pair * 2 + (kb0 > 0 ? 0 : 1)) * 2 + rank) * kPairCtaFloats +
+                (size_t)wslot * kPairWarpFloats;
+#pragma unroll 1
+  for (int g = 0; g < 8; ++g) {
+    uint32_t r[32];
+    tmem_ld32(tacc + (uint32_t)(g * 32), r);
+    tmem_ld_wait();
+    float* dst = slot + g * 1024 + lane;
+#pragma unroll
+    for (int k = 0; k < 32; ++k) __stcg(dst + k * 32, __uint_as_float(r[k]));
+  }
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive_cluster(tempty_leader);
+  // which pairs hold a share of this tile (they are consecutive)
+  const int64_t t_begin = (int64_t)tile * p.k_blocks, t_end = t_begin + p.k_blocks;
+  int j_first = pair;
+  while (j_first > 0 && Sched::share_begin(p, j_first, num_pairs) > t_begin) --j_first;
+  int j_last = pair;
+  while (j_last + 1 < num_pairs && Sched::share_begin(p, j_last + 1, num_pairs) < t_end) ++j_last;
+  const int n_shares = j_last - j_first + 1;
+  __threadfence();
+  __syncwarp();
+  uint32_t ticket = 0;
+  uint32_t* counter = p.sk_counters + ((size_t)tile * 2 + rank) * 4 + wslot;
+  if (lane == 0) ticket = atomicAdd(counter, 1u);
+  ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+  if (ticket + 1 != (uint32_t)n_shares) return 0.0f;  // not the last share of this tile: done
+  __threadfence();
+  if (lane == 0) *counter = 0u;  // ready for the next launch
+  const uint32_t row_off = (uint32_t)lane * 128u;
+  const uint32_t swz = (uint32_t)(lane & 7);
+  const int row = row0 + lane;
+#pragma unroll 1
+  for (int c = 0; c < 256 / CH; ++c) {
+    const int col0 = n0 + c * CH;
+    if (col0 >= p.Nd || row0 >= p.Md) break;  // uniform across the warp
+    uint32_t r[CH];
+#pragma unroll 1
+    for (int sidx = 0; sidx < n_shares; ++sidx) {
+      const int j = j_first + sidx;
+      const int sel = Sched::share_begin(p, j, num_pairs) > t_begin ? 0 : 1;
+      const float* src = p.sk_partials + ((size_t)(j * 2 + sel) * 2 + rank) * kPairCtaFloats +
+                         (size_t)wslot * kPairWarpFloats + (size_t)(c * CH) * 32 + lane;
+      if (sidx == 0) {
+#pragma unroll
+        for (int k = 0; k < CH; ++k) r[k] = __float_as_uint(__ldcg(src + k * 32));
+      } else {
+#pragma unroll
+        for (int k = 0; k < CH; ++k) r[k] = __float_as_uint(__uint_as_float(r[k]) + __ldcg(src + k * 32));
+      }
+    }
+    const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
+    ++it;
+    if (lane == 0) bulk_wait_read<1>();
+    __syncwarp();
+    if (OUT_F32) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4),
+                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j]), alpha)),
+                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 1]), alpha)),
+                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 2]), alpha)),
+                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 3]), alpha)));
+    } else {
+      uint32_t packed[CH / 2];
+#pragma unroll
+      for (int j = 0; j < CH / 2; ++j)
+        packed[j] = f32x2_to_bf16x2(__fmul_rn(__uint_as_float(r[2 * j]), alpha),
+                                    __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha));
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1], packed[4 * j + 2],
+                     packed[4 * j + 3]);
+      if ((p.out_amax || p.out_q) && row < p.Md) {
+#pragma unroll 1
+        for (int j = 0; j < CH / 4; ++j) {  // groups of four columns
+          const uint32_t w0 = packed[2 * j], w1 = packed[2 * j + 1];
+          float v[4] = {bf16lo_to_f32(w0), bf16hi_to_f32(w0), bf16lo_to_f32(w1), bf16hi_to_f32(w1)};
+          if (col0 + 4 * j < p.Nd) {
+            run_amax = fmaxf(run_amax, fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))));
+            if (p.out_q) {
+              const uint32_t q = p.q_fmt == TWEO_E4M3
+                                     ? quant4<TWEO_E4M3>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs),
+                                                         __fmul_rn(v[2], qs), __fmul_rn(v[3], qs))
+                                     : quant4<TWEO_E5M2>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs),
+                                                         __fmul_rn(v[2], qs), __fmul_rn(v[3], qs));
+              *reinterpret_cast<uint32_t*>(p.out_q + (int64_t)row * p.ldq + col0 + 4 * j) = q;
+            }
+          }
+        }
+      }
+    }
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+      if (OUT_F32 && p.accumulate) tma_reduce_add_2d(tmap_d, col0, row0, buf);
+      else tma_store_2d(tmap_d, col0, row0, buf);
+      bulk_commit();
+    }
+  }
+  // the caller's buffer rotation does not know how many chunks were stored here
+  if (lane == 0) bulk_wait_read<0>();
+  __syncwarp();
+  return run_amax;
+}
+
+template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                     const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ GemmParams p) {
+  constexpr int BN = 256;                 // tile columns of the pair
+  constexpr uint32_t A_BYTES = BM * BK;   // this CTA's 128 rows of A
+  constexpr uint32_t B_BYTES = 128 * BK;  // this CTA's 128 of the 256 columns of B
+  constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr uint32_t TMEM_COLS = 512;
+
+  extern __shared__ uint8_t smem_dyn[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  constexpr uint32_t EPI_BUF = 32 * 128;
+  constexpr uint32_t EPI_BYTES = 4 * 2 * EPI_BUF;
+  uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 8);  // four epilogue warps of each CTA of the pair
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // both CTAs' barriers are initialised before anyone signals across
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int pair = blockIdx.x >> 1;
+  const int num_pairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      Sched sched(p, pair, num_pairs);
+      int tile, kb0, kb1;
+      while (ok && sched.next(tile, kb0, kb1)) {
+        int tm, tn;
+        tile_coords(p, tile, tm, tn);
+        const int m0 = tm * (2 * BM) + (int)rank * BM;  // this CTA's rows
+        const int n0 = tn * BN + (int)rank * 128;       // this CTA's half of B
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
+          const uint32_t fb = map_to_cta(full_bar(stage), 0);
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+          const int k0 = kb * BK;
+          if (A_MN) tma_load_2d_pair(sa, &tmap_a, m0, k0, fb);
+          else tma_load_2d_pair(sa, &tmap_a, k0, m0, fb);
+          if (B_MN) tma_load_2d_pair(sb, &tmap_b, n0, k0, fb);
+          else tma_load_2d_pair(sb, &tmap_b, k0, n0, fb);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && leader) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      Sched sched(p, pair, num_pairs);
+      int tile, kb0, kb1;
+      while (ok && sched.next(tile, kb0, kb1)) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t adesc = make_smem_desc(sa + (A_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
+            const uint64_t bdesc = make_smem_desc(sb + (B_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
+            umma_f8_pair(d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != kb0 || k != 0));
+          }
+          umma_commit_pair(map_to_cta(empty_bar(stage), 0));  // frees the stage in both CTAs
+          umma_commit_pair(map_to_cta(empty_bar(stage), 1));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit_pair(map_to_cta(tfull_bar(acc), 0));      // accumulator complete, both CTAs
+        umma_commit_pair(map_to_cta(tfull_bar(acc), 1));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    const int quarter = warp & 3;
+    const float alpha = __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
+    const float qs = p.out_q ? __ldg(p.q_scale) : 0.0f;
+    constexpr int CH = OUT_F32 ? 32 : 64;
+    const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
+    const uint32_t row_off = (uint32_t)lane * 128u;
+    const uint32_t swz = (uint32_t)(lane & 7);
+    const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
+    uint32_t it = 0;
+    float run_amax = 0.0f;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    Sched sched(p, pair, num_pairs);
+    int tile, kb0, kb1;
+    while (ok && sched.next(tile, kb0, kb1)) {
+      int tm, tn;
+      tile_coords(p, tile, tm, tn);
+      const int m0 = tm * (2 * BM) + (int)rank * BM;
+      const int n0 = tn * BN;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row0 = m0 + quarter * 32;
+      const int row = row0 + lane;
+      const bool row_ok = row < p.Md;
+      if (kb0 != 0 || kb1 != p.k_blocks) {
+        // part of a split tile: park the accumulator; the last share to arrive stores the tile
+        const float part_amax = pair_partial_share<OUT_F32>(
+            p, &tmap_d, tile, kb0, pair, num_pairs, (int)rank, warp - 2,
+            tmem_base + tlane + (uint32_t)(acc * BN), map_to_cta(tempty_bar(acc), 0), alpha, qs, epi_base, it, lane,
+            row0, n0);
+        it += BN / CH;  // keeps the staging-buffer rotation in step whether or not this warp stored
+        run_amax = fmaxf(run_amax, part_amax);
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+        continue;
+      }
+#pragma unroll 1
+      for (int c = 0; c < BN / CH; ++c) {
+        const int col0 = n0 + c * CH;
+        if (col0 >= p.Nd) break;
+        uint32_t r[CH];
+        const uint32_t taddr = tmem_base + tlane + (uint32_t)(acc * BN + c * CH);
+        tmem_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+        if (!OUT_F32) tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[CH - 32]));
+        tmem_ld_wait();
+        if (row0 >= p.Md) continue;
+        const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
+        if (lane == 0) bulk_wait_read<1>();
+        __syncwarp();
+        if (OUT_F32) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j]), alpha)),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 1]), alpha)),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 2]), alpha)),
+                         __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 3]), alpha)));
+        } else {
+          uint32_t packed[CH / 2];
+#pragma unroll
+          for (int j = 0; j < CH / 2; ++j)
+            packed[j] = f32x2_to_bf16x2(__fmul_rn(__uint_as_float(r[2 * j]), alpha),
+                                        __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha));
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1],
+                         packed[4 * j + 2], packed[4 * j + 3]);
+          if ((p.out_amax || p.out_q) && row_ok) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              uint32_t q[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const uint32_t w0 = packed[16 * h + 2 * j], w1 = packed[16 * h + 2 * j + 1];
+                float v[4] = {bf16lo_to_f32(w0), bf16hi_to_f32(w0), bf16lo_to_f32(w1), bf16hi_to_f32(w1)};
+                if (col0 + 32 * h + 4 * j < p.Nd)
+                  run_amax = fmaxf(run_amax, fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))));
+                if (p.out_q) {
+                  if (p.q_fmt == TWEO_E4M3)
+                    q[j] = quant4<TWEO_E4M3>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
+                                             __fmul_rn(v[3], qs));
+                  else
+                    q[j] = quant4<TWEO_E5M2>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
+                                             __fmul_rn(v[3], qs));
+                }
+              }
+              if (p.out_q) {
+                uint8_t* qrow = p.out_q + (int64_t)row * p.ldq + col0 + 32 * h;
+                if (col0 + 32 * h < p.Nd) *reinterpret_cast<uint4*>(qrow) = make_uint4(q[0], q[1], q[2], q[3]);
+                if (col0 + 32 * h + 16 < p.Nd) *reinterpret_cast<uint4*>(qrow + 16) = make_uint4(q[4], q[5], q[6], q[7]);
+              }
+            }
+          }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          if (OUT_F32 && p.accumulate) tma_reduce_add_2d(&tmap_d, col0, row0, buf);
+          else tma_store_2d(&tmap_d, col0, row0, buf);
+          bulk_commit();
+        }
+        ++it;
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's barrier
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+    if (lane == 0) bulk_wait_all();
+    if (p.out_amax) {
+      run_amax = warp_max(run_amax);
+      if (lane == 0 && run_amax > 0.0f)
+        atomicMax(reinterpret_cast<unsigned int*>(p.out_amax), __float_as_uint(run_amax));
+    }
+  }
+
+  // Neither CTA may leave (or free tensor memory) while the other can still signal its
+  // barriers or have MMAs reading its shared memory.
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
+
+}  // namespace tweo_detail
