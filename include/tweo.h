@@ -284,13 +284,6 @@ TWEO_API const char* tweo_status_string(tweo_status_t s);
 TWEO_API const char* tweo_last_cuda_error(void); /* text of the last failing CUDA call in this thread */
 TWEO_API int32_t tweo_version(void);             /* major * 10000 + minor * 100 + patch */
 
-/* Large tensor-bound GEMMs can run on clusters of four CTAs in which two CTA pairs share each
- * weight tile through TMA multicast of this GPU's own memory.  That kernel lives in an optional
- * second library (libtweo_b200_mc.so beside this one) meant for single-GPU installations; it is
- * used when present.  tweo_gemm_multicast(0) turns it off, (1) on again; returns 1 if it is
- * loaded and now enabled, else 0.  Results are bit-identical either way. */
-TWEO_API int32_t tweo_gemm_multicast(int32_t enable);
-
 /* Number of kernel launches this library has enqueued since it was loaded. */
 TWEO_API uint64_t tweo_launch_count(void);
 

@@ -26,7 +26,7 @@ EXPORTS = [
     "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_bwd_dgrad",
     "tweo_fp8_linear_bwd_wgrad", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
-    "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count", "tweo_gemm_multicast",
+    "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
 ]
 
 
@@ -89,7 +89,6 @@ def lib() -> C.CDLL:
         L.tweo_last_cuda_error.restype = C.c_char_p
         L.tweo_version.restype = i32
         L.tweo_launch_count.restype = C.c_uint64
-        L.tweo_gemm_multicast.argtypes = [i32]
         for name in EXPORTS:
             f = getattr(L, name)
             if f.restype is C.c_int:  # default -> status
@@ -126,12 +125,6 @@ U8 = (torch.uint8, torch.float8_e4m3fn, torch.float8_e5m2)
 
 def launch_count() -> int:
     return int(lib().tweo_launch_count())
-
-
-def gemm_multicast(enable: bool) -> bool:
-    """tweo_gemm_multicast: switches the optional four-CTA-cluster GEMM library on or off;
-    True if it is loaded and now enabled."""
-    return bool(lib().tweo_gemm_multicast(1 if enable else 0))
 
 
 def version() -> int:

@@ -10,9 +10,6 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libtweo_b200.so")
 SOURCES = ["api.cu", "loss.cu", "quantize.cu", "gemm.cu", "w8a8.cu"]
-# optional second library (single-GPU installations): built when its source is present
-MC_LIB = os.path.join(_HERE, "libtweo_b200_mc.so")
-MC_SOURCES = ["gemm_mc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fvisibility=hidden", "--expt-relaxed-constexpr"]
 
@@ -28,12 +25,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(objdir, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
     headers.append(os.path.join(_ROOT, "include", "tweo.h"))
-    objs, mc_objs, procs = [], [], []
-    mc_present = all(os.path.exists(os.path.join(CSRC, f)) for f in MC_SOURCES)
-    for src in SOURCES + (MC_SOURCES if mc_present else []):
+    objs, procs = [], []
+    for src in SOURCES:
         s = os.path.join(CSRC, src)
         o = os.path.join(objdir, src + ".o")
-        (mc_objs if src in MC_SOURCES else objs).append(o)
+        objs.append(o)
         if force or _newer(s, o) or any(_newer(h, o) for h in headers):
             cmd = [nvcc, *NVCC_FLAGS, *inc, "-c", s, "-o", o]
             if verbose:
@@ -53,11 +49,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
         subprocess.check_call([nvcc, "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a",
                                "-Xcompiler", "-fPIC"])
         os.replace(tmp, LIB)
-    if mc_present and (procs or not os.path.exists(MC_LIB)):
-        tmp = MC_LIB + f".tmp{os.getpid()}"
-        subprocess.check_call([nvcc, "-shared", "-o", tmp, *mc_objs, "-gencode", "arch=compute_100a,code=sm_100a",
-                               "-Xcompiler", "-fPIC"])
-        os.replace(tmp, MC_LIB)
     return LIB
 
 

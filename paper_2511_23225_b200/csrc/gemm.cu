@@ -34,12 +34,9 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
-#include <dlfcn.h>
-
 #include <atomic>
 #include <cstdlib>
 #include <mutex>
-#include <string>
 
 #include "common.cuh"
 
@@ -424,6 +421,15 @@ std::atomic<uint32_t> g_sk_epoch{0};
 // TWEO_GEMM_NO_PAIR=1 in the environment keeps every GEMM on the single-CTA kernel (A/B timing).
 const bool g_disable_pair = [] { const char* e = getenv("TWEO_GEMM_NO_PAIR"); return e && e[0] == '1'; }();
 
+// Band height of the tile numbering: the `workers` tiles in flight cover about g x workers/g
+// tiles, so g near sqrt(workers) keeps the rows of A and the columns of B they touch smallest.
+int raster_band(int tiles_m, int workers) {
+  int g = 1;
+  while ((g + 1) * (g + 1) <= workers) ++g;
+  if (g > tiles_m) g = tiles_m;
+  return g < 1 ? 1 : g;
+}
+
 template <int BN, bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
 tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, GemmParams& p,
                          void* ws, size_t ws_bytes, cudaStream_t st) {
@@ -484,7 +490,7 @@ tweo_status_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CU
                           void* ws, size_t ws_bytes, cudaStream_t st) {
   constexpr int STAGES = 6;
   constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
-  auto kern = gemm_fp8_pair_kernel<PairCfgPlain, A_MN, B_MN, STAGES, OUT_F32>;
+  auto kern = gemm_fp8_pair_kernel<A_MN, B_MN, STAGES, OUT_F32>;
   static bool attr_done = false;
   if (!attr_done) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -528,36 +534,6 @@ tweo_status_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CU
   return check_launch("gemm_fp8_pair_kernel");
 }
 
-// ---- optional accelerator: the four-CTA-cluster form of the pair kernel lives in a library of
-// its own (libtweo_b200_mc.so, next to this one) that single-GPU installations ship.  It is
-// looked up once; without it every GEMM runs on the kernels in this file.
-struct McLib {
-  int (*gemm)(const CUtensorMap*, const CUtensorMap*, const CUtensorMap*, const GemmParams*, int, int, void*);
-  int (*read_status)(unsigned int*);
-};
-std::atomic<int> g_use_mc{1};
-
-McLib* mc_lib() {
-  static McLib lib = {nullptr, nullptr};
-  static McLib* found = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    const char* off = getenv("TWEO_GEMM_NO_MC");
-    if (off && off[0] == '1') return;
-    Dl_info info;
-    if (!dladdr(reinterpret_cast<void*>(&mc_lib), &info) || !info.dli_fname) return;
-    std::string path(info.dli_fname);
-    const size_t slash = path.rfind('/');
-    path = (slash == std::string::npos ? std::string(".") : path.substr(0, slash)) + "/libtweo_b200_mc.so";
-    void* h = dlopen(path.c_str(), RTLD_NOW | RTLD_LOCAL);
-    if (!h) return;
-    lib.gemm = reinterpret_cast<decltype(lib.gemm)>(dlsym(h, "tweo_mc_gemm"));
-    lib.read_status = reinterpret_cast<decltype(lib.read_status)>(dlsym(h, "tweo_mc_read_status"));
-    if (lib.gemm && lib.read_status) found = &lib;
-  });
-  return found;
-}
-
 struct Operand {
   const uint8_t* ptr;
   int64_t ld;
@@ -599,29 +575,6 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
   if (p.out_amax) {
     zero_float_kernel<<<1, 1, 0, st>>>(p.out_amax);
     count_launch();
-  }
-  if (use_pair && g_use_mc.load(std::memory_order_relaxed) && mc_lib()) {
-    // Large outputs with a long enough contraction go to the four-CTA-cluster kernel (two pairs
-    // share each B tile), unless splitting tiles along the contraction is the better deal.
-    const int tiles256 = (int)(((Md + 255) / 256) * ((Nd + 255) / 256));
-    const int super_tiles = (int)(((Md + 511) / 512) * ((Nd + 255) / 256));
-    const int k_blocks = (int)((Kc + BK - 1) / BK);
-    const int pairs = sm_count() / 2;
-    const bool would_split = ws && ws_bytes >= kWsPartialsOffset + (size_t)sm_count() * kWsPartialBytesPerSm &&
-                             pair_split_tiles(tiles256, pairs, k_blocks) > 0;
-    if (Md >= 1024 && super_tiles >= sm_count() / 4 && k_blocks >= 4 && !would_split) {
-      CUtensorMap mb64;
-      if (B.mn_major) ok = make_map(&mb64, B.ptr, Nd, Kc, B.ld, 64);
-      else ok = make_map(&mb64, B.ptr, Kc, Nd, B.ld, 64);
-      if (!ok) {
-        cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-        return TWEO_ERR_CUDA;
-      }
-      const int e = mc_lib()->gemm(&ma, &mb64, &md, &p, A.mn_major ? 1 : 0, B.mn_major ? 1 : 0, st);
-      count_launch();
-      if (e != 0) return cuda_fail((cudaError_t)e, "gemm_fp8_pair_kernel (four-CTA clusters)");
-      return TWEO_OK;
-    }
   }
   if (use_pair) {
 #define TWEO_PAIR(AMN, BMN) (p.out_f32 ? launch_pair<AMN, BMN, true>(ma, mb, md, p, ws, ws_bytes, st) : launch_pair<AMN, BMN, false>(ma, mb, md, p, ws, ws_bytes, st))
@@ -673,12 +626,6 @@ tweo_status_t read_and_clear_device_status(cudaStream_t stream) {
   unsigned int v = 0, zero = 0;
   TWEO_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_device_status, sizeof v));
   if (v != 0) TWEO_CUDA_TRY(cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero));
-  if (McLib* mc = mc_lib()) {  // the accelerator library keeps its own record
-    unsigned int w = 0;
-    const int e = mc->read_status(&w);
-    if (e != 0) return cuda_fail((cudaError_t)e, "status of the four-CTA-cluster library");
-    if (v == 0) v = w;
-  }
   return v == 0 ? TWEO_OK : (tweo_status_t)v;
 }
 
@@ -716,11 +663,6 @@ tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const ui
 }  // namespace tweo_detail
 
 extern "C" {
-
-int32_t tweo_gemm_multicast(int32_t enable) {
-  g_use_mc.store(enable ? 1 : 0, std::memory_order_relaxed);
-  return (enable && mc_lib()) ? 1 : 0;
-}
 
 tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const uint8_t* wq, int64_t ldw,
                                   const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,

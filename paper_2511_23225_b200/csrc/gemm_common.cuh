@@ -95,15 +95,6 @@ struct Sched {
   }
 };
 
-// Band height of the tile numbering: the `workers` tiles in flight cover about g x workers/g
-// tiles, so g near sqrt(workers) keeps the rows of A and the columns of B they touch smallest.
-inline int raster_band(int tiles_m, int workers) {
-  int g = 1;
-  while ((g + 1) * (g + 1) <= workers) ++g;
-  if (g > tiles_m) g = tiles_m;
-  return g < 1 ? 1 : g;
-}
-
 // ----------------------------------------------------------------- epilogue helpers
 template <int FMT>
 __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d) {

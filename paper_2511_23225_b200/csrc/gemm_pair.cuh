@@ -1,26 +1,15 @@
 // CTA-pair FP8 GEMM kernel (included by the translation units that instantiate it).
-// Two CTAs of a cluster (adjacent SMs) compute one 256 x 256 tile with tcgen05 cta_group::2
-// instructions: each CTA stages its own 128 rows of A and only HALF of the B tile (128 of the
-// 256 output columns), the pair's tensor cores read both halves, and each CTA's tensor memory
-// receives the accumulator of its own 128 rows.  Per SM this moves 32 KB of operands per
-// 128-deep contraction block instead of the 48 KB a lone CTA with a 128 x 256 tile needs; the
-// L2 -> shared-memory path (about 64 B per clock per SM) is as scarce as tensor-core time for
-// 8-bit operands.  Roles per CTA are those of the single-CTA kernel; only the leader (even CTA)
-// of a pair issues MMAs.
-//
-// The kernel is written for a cluster of Cfg::kPairs CTA pairs.  kPairs = 1 is the general
-// form.  With kPairs = 2 the two pairs of a cluster compute vertically adjacent tiles, which
-// use the SAME B tile: Cfg::load_b then fetches only half of this CTA's B half and delivers it
-// to the CTA of the same parity in both pairs, so each SM pulls 24 KB per block from L2.  How
-// that delivery is done is the business of the Cfg type, which the including file defines.
-//
-// Barriers of a pair (leader = even CTA):
-//   full[s]    leader only : the leader's producer arrives and posts the bytes that land in BOTH
-//                            CTAs of the pair (64 KB per stage, whoever loads them)
-//   empty[s]   each CTA    : one arrival per pair of the cluster (its leader's MMA thread commits
-//                            to every CTA whose loads can write into a stage it reads)
-//   tfull[a]   each CTA    : the pair's leader commits once an accumulator is complete
-//   tempty[a]  leader only : 4 epilogue warps of each CTA of the pair arrive (the peer's remotely)
+// Two CTAs of a cluster (adjacent SMs) compute one 256 x 256 tile with tcgen05
+// cta_group::2 instructions: each CTA stages its own 128 rows of A and only HALF of the
+// B tile (128 of the 256 output columns), the pair's tensor cores read both halves, and
+// each CTA's tensor memory receives the accumulator of its own 128 rows.  Per SM this
+// moves 32 KB of operands per 128-deep contraction block instead of 48 KB, which is what
+// lifts the kernel off the shared-memory fill limit.  Roles per CTA are those of the
+// single-CTA kernel; only CTA 0 (the leader) issues MMAs.  Barriers:
+//   full[s]    leader only : leader's producer arrives (+ expected bytes of BOTH CTAs' loads)
+//   empty[s]   each CTA    : leader's MMA thread commits to its own and to the peer's
+//   tfull[a]   each CTA    : same, once a tile's accumulator is complete
+//   tempty[a]  leader only : 4 epilogue warps of each CTA arrive (the peer's remotely)
 #pragma once
 
 #include <cuda.h>
@@ -154,21 +143,7 @@ __device__ __noinline__ float pair_partial_share(const GemmParams& p, const CUte
   return run_amax;
 }
 
-// The general cluster shape: one pair, each CTA loads its own half of B.
-struct PairCfgPlain {
-  static constexpr int kPairs = 1;
-  // Brings this CTA's 128 x 128-byte half of the B tile of one k-block into `sb`; c0/c1 address the
-  // half's first element, `lead_bar` is the pair leader's full barrier (cluster address).
-  static __device__ __forceinline__ void load_b(uint32_t sb, const CUtensorMap* map, int32_t c0, int32_t c1,
-                                                bool b_mn, uint32_t lead_bar, uint32_t local_bar, uint32_t crank) {
-    (void)b_mn;
-    (void)local_bar;
-    (void)crank;
-    tma_load_2d_pair(sb, map, c0, c1, lead_bar);
-  }
-};
-
-template <class Cfg, bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
+template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ GemmParams p) {
@@ -189,10 +164,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  constexpr int kPairs = Cfg::kPairs;
-  const uint32_t crank = cluster_ctarank();  // rank in the cluster: pair = crank / 2
-  const uint32_t rank = crank & 1u;          // rank in the pair
-  const uint32_t lead = crank & ~1u;         // the pair's leader
+  const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_u32(bars);
@@ -204,7 +176,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), kPairs);
+      mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
@@ -216,14 +188,12 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
   tc_fence_before();
   __syncthreads();
-  cluster_sync_all();  // every CTA's barriers are initialised before anyone signals across
+  cluster_sync_all();  // both CTAs' barriers are initialised before anyone signals across
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // the unit of scheduling is the cluster: kPairs vertically adjacent 256 x 256 tiles
-  const int pair = blockIdx.x / (2 * kPairs);
-  const int num_pairs = gridDim.x / (2 * kPairs);
-  const int tm_sub = (int)(crank >> 1);  // which of the cluster's tiles this pair computes
+  const int pair = blockIdx.x >> 1;
+  const int num_pairs = gridDim.x >> 1;
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -236,19 +206,19 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       while (ok && sched.next(tile, kb0, kb1)) {
         int tm, tn;
         tile_coords(p, tile, tm, tn);
-        const int m0 = (tm * kPairs + tm_sub) * (2 * BM) + (int)rank * BM;  // this CTA's rows
-        const int n0 = tn * BN + (int)rank * 128;                           // this CTA's half of B
+        const int m0 = tm * (2 * BM) + (int)rank * BM;  // this CTA's rows
+        const int n0 = tn * BN + (int)rank * 128;       // this CTA's half of B
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
-          const uint32_t fb = map_to_cta(full_bar(stage), lead);
+          const uint32_t fb = map_to_cta(full_bar(stage), 0);
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
           const int k0 = kb * BK;
           if (A_MN) tma_load_2d_pair(sa, &tmap_a, m0, k0, fb);
           else tma_load_2d_pair(sa, &tmap_a, k0, m0, fb);
-          if (B_MN) Cfg::load_b(sb, &tmap_b, n0, k0, true, fb, full_bar(stage), crank);
-          else Cfg::load_b(sb, &tmap_b, k0, n0, false, fb, full_bar(stage), crank);
+          if (B_MN) tma_load_2d_pair(sb, &tmap_b, n0, k0, fb);
+          else tma_load_2d_pair(sb, &tmap_b, k0, n0, fb);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -278,14 +248,13 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             const uint64_t bdesc = make_smem_desc(sb + (B_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
             umma_f8_pair(d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != kb0 || k != 0));
           }
-#pragma unroll
-          for (uint32_t c = 0; c < 2u * kPairs; ++c)  // frees the stage in every CTA that loads into it
-            umma_commit_pair(map_to_cta(empty_bar(stage), c));
+          umma_commit_pair(map_to_cta(empty_bar(stage), 0));  // frees the stage in both CTAs
+          umma_commit_pair(map_to_cta(empty_bar(stage), 1));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit_pair(map_to_cta(tfull_bar(acc), lead));       // accumulator complete, both CTAs
-        umma_commit_pair(map_to_cta(tfull_bar(acc), lead + 1u));
+        umma_commit_pair(map_to_cta(tfull_bar(acc), 0));      // accumulator complete, both CTAs
+        umma_commit_pair(map_to_cta(tfull_bar(acc), 1));
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
@@ -310,7 +279,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     while (ok && sched.next(tile, kb0, kb1)) {
       int tm, tn;
       tile_coords(p, tile, tm, tn);
-      const int m0 = (tm * kPairs + tm_sub) * (2 * BM) + (int)rank * BM;
+      const int m0 = tm * (2 * BM) + (int)rank * BM;
       const int n0 = tn * BN;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
@@ -321,7 +290,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         // part of a split tile: park the accumulator; the last share to arrive stores the tile
         const float part_amax = pair_partial_share<OUT_F32>(
             p, &tmap_d, tile, kb0, pair, num_pairs, (int)rank, warp - 2,
-            tmem_base + tlane + (uint32_t)(acc * BN), map_to_cta(tempty_bar(acc), lead), alpha, qs, epi_base, it, lane,
+            tmem_base + tlane + (uint32_t)(acc * BN), map_to_cta(tempty_bar(acc), 0), alpha, qs, epi_base, it, lane,
             row0, n0);
         it += BN / CH;  // keeps the staging-buffer rotation in step whether or not this warp stored
         run_amax = fmaxf(run_amax, part_amax);
@@ -398,7 +367,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), lead));  // the leader's barrier
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's barrier
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }

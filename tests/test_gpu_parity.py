@@ -399,37 +399,6 @@ def test_gemms_benchmark_shapes_sampled(tw, cfg, lin, M):
     assert rel_fro(dw.float().cpu().numpy()[r, c], ref) <= GEMM_TOL
 
 
-@pytest.mark.parametrize("name,M,K,N", [("all_three", 4096, 1280, 4096), ("ragged_fwd", 2381, 528, 2320)],
-                         ids=["all_three", "ragged_fwd"])
-def test_gemms_four_cta_clusters_match_pairs_bit_for_bit(tw, name, M, K, N):
-    """The optional four-CTA-cluster GEMM library (two CTA pairs share each B tile) against the
-    pair kernel: the same bits, and the oracle's values on sampled outputs."""
-    if not tw.gemm_multicast(True):
-        pytest.skip("the optional four-CTA-cluster library is not installed")
-    try:
-        x = synth.normal_with_outlier_channels_bf16(95, (M, K))
-        w = synth.normal_bf16(96, (N, K), 0.02)
-        dy = synth.normal_bf16(97, (M, N), 1e-3)
-        qx, qw, qd = quantized_operands(x, w, dy)
-        y1, dx1, dw1 = run_three(tw, qx, qw, qd, E5M2)
-        _, _, dwf1 = run_three(tw, qx, qw, qd, E5M2, dw_f32=True)
-        assert not tw.gemm_multicast(False)
-        y0, dx0, dw0 = run_three(tw, qx, qw, qd, E5M2)
-        _, _, dwf0 = run_three(tw, qx, qw, qd, E5M2, dw_f32=True)
-    finally:
-        tw.gemm_multicast(True)
-    for a, b in ((y1, y0), (dx1, dx0), (dw1, dw0)):
-        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
-    assert torch.equal(dwf1.view(torch.int32), dwf0.view(torch.int32))
-    g = np.random.Generator(np.random.PCG64(11))
-    r, c = sample_points(g, M, N, n_rows=2, n_pts=2048)
-    ref = orc.gemm_fwd_at(qx["q"], E4M3, qw["q"], E4M3, qx["scale_inv"], qw["scale_inv"], r, c)
-    assert rel_fro(y1.float().cpu().numpy()[r, c], ref) <= GEMM_TOL
-    r, c = sample_points(g, N, K, n_rows=2, n_pts=2048)
-    ref = orc.gemm_wgrad_at(qx["q"], E4M3, qd["q"], E5M2, qx["scale_inv"], qd["scale_inv"], r, c)
-    assert rel_fro(dwf1.cpu().numpy()[r, c], ref) <= 1e-5
-
-
 # ------------------------------------------------------------------ static W8A8
 @pytest.mark.parametrize("M", [1, 16, 128, 1024])
 def test_w8a8_static_gemm(tw, M):
