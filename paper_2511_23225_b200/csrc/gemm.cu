@@ -42,6 +42,7 @@
 
 #include "gemm_common.cuh"
 #include "gemm_pair.cuh"
+#include "gemm_skinny.cuh"
 #include "tc_ptx.cuh"
 
 namespace {
@@ -419,6 +420,8 @@ uint32_t make_idesc(int fmt_a, int fmt_b, bool a_mn, bool b_mn, int n, int m = B
 
 std::atomic<uint32_t> g_sk_epoch{0};
 // TWEO_GEMM_NO_PAIR=1 in the environment keeps every GEMM on the single-CTA kernel (A/B timing).
+// TWEO_GEMM_NO_SKINNY=1 sends small-M forward products through the general kernels (A/B timing).
+const bool g_disable_skinny = [] { const char* e = getenv("TWEO_GEMM_NO_SKINNY"); return e && e[0] == '1'; }();
 const bool g_disable_pair = [] { const char* e = getenv("TWEO_GEMM_NO_PAIR"); return e && e[0] == '1'; }();
 
 // Band height of the tile numbering: the `workers` tiles in flight cover about g x workers/g
@@ -596,6 +599,56 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
 #undef TWEO_DISPATCH
 }
 
+// Forward product for M <= 128 (see gemm_skinny.cuh): W is streamed once, K is sliced over CTAs.
+tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
+                         const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M, int64_t N,
+                         int64_t K, void* ws, size_t ws_bytes, cudaStream_t st) {
+  if (N > INT32_MAX || K > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(xq) || !aligned16(wq) || (ldx & 15) || (ldw & 15)) return TWEO_ERR_ALIGNMENT;
+  SkinnyParams p{};
+  p.y = y;
+  p.ldy = ldy;
+  p.M = (int32_t)M;
+  p.N = (int32_t)N;
+  p.Mpad = (int32_t)((M + 15) / 16 * 16);
+  p.k_blocks = (int32_t)((K + BK - 1) / BK);
+  p.stage_bytes = (uint32_t)((BM * BK + p.Mpad * 128 + 1023) / 1024 * 1024);
+  p.stages = (int32_t)((100 * 1024) / p.stage_bytes);
+  if (p.stages > kSkinnyMaxStages) p.stages = kSkinnyMaxStages;
+  p.tmem_cols = p.Mpad <= 32 ? 32u : (p.Mpad <= 64 ? 64u : 128u);
+  p.idesc = make_idesc(fmt_w, fmt_x, false, false, p.Mpad, BM);
+  p.sx_inv = sx_inv;
+  p.sw_inv = sw_inv;
+  const int sms = sm_count();
+  const int slabs = (int)((N + 127) / 128);
+  p.slices = 1;
+  if (ws && aligned16(ws) && ws_bytes >= kWsPartialsOffset + (size_t)sms * kWsPartialBytesPerSm && slabs <= 512) {
+    int s = (2 * sms) / slabs;                       // two CTAs per SM
+    if (s > p.k_blocks / 4) s = p.k_blocks / 4;      // at least four k-blocks per slice
+    while (s > 1 && (size_t)slabs * s * p.Mpad * 128 * sizeof(float) > (size_t)sms * kWsPartialBytesPerSm) --s;
+    if (s > 1) {
+      p.slices = s;
+      p.counters = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + kWsCountersOffset);
+      p.partials = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + kWsPartialsOffset);
+    }
+  }
+  CUtensorMap mw, mx;
+  if (!make_map(&mw, wq, K, N, ldw, BM) || !make_map(&mx, xq, K, M, ldx, p.Mpad)) {
+    cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return TWEO_ERR_CUDA;
+  }
+  const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
+  static bool attr_done = false;
+  if (!attr_done) {
+    TWEO_CUDA_TRY(cudaFuncSetAttribute(gemm_fp8_skinny_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)(kSkinnyMaxStages * 16384 + 4096)));
+    attr_done = true;
+  }
+  gemm_fp8_skinny_kernel<<<slabs * p.slices, kThreads, smem, st>>>(mw, mx, p);
+  count_launch();
+  return check_launch("gemm_fp8_skinny_kernel");
+}
+
 bool fmt_ok(int f) { return f == TWEO_E4M3 || f == TWEO_E5M2; }
 
 tweo_status_t fill_epilogue(GemmParams& p, const tweo_epilogue_t* epi) {
@@ -650,6 +703,9 @@ tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const ui
                              const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
                              int64_t N, int64_t K, const tweo_epilogue_t* epi, void* ws, size_t ws_bytes,
                              cudaStream_t st) {
+  const bool fused = epi && (epi->out_amax || epi->out_q);
+  if (M <= 128 && !fused && !g_disable_skinny)  // few tokens: stream W once, tokens on the MMA's N side
+    return run_skinny(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, y, ldy, M, N, K, ws, ws_bytes, st);
   GemmParams p{};
   p.d = y;
   p.ldd = ldy;

@@ -399,6 +399,31 @@ def test_gemms_benchmark_shapes_sampled(tw, cfg, lin, M):
     assert rel_fro(dw.float().cpu().numpy()[r, c], ref) <= GEMM_TOL
 
 
+@pytest.mark.parametrize("M,K,N", [(37, 2064, 272), (128, 1024, 384), (5, 4096, 1040)],
+                         ids=["ragged_m37", "m128", "m5_long_k"])
+@pytest.mark.parametrize("with_ws", [False, True], ids=["whole_k", "sliced_k"])
+def test_forward_few_tokens_streams_w(tw, M, K, N, with_ws):
+    """M <= 128 takes the weight-streaming kernel (W rows on the MMA's M side); with a workspace K is
+    sliced over CTAs and the slices are added in a fixed order: same bits on every run."""
+    x = synth.normal_with_outlier_channels_bf16(101, (M, K))
+    w = synth.normal_bf16(102, (N, K), 0.02)
+    qx = orc.quantize_per_tensor_current(x, E4M3)
+    qw = orc.quantize_per_tensor_current(w, E4M3)
+    xq, wq = torch.from_numpy(qx["q"]).cuda(), torch.from_numpy(qw["q"]).cuda()
+    sx, sw = dev_scalar(qx["scale_inv"]), dev_scalar(qw["scale_inv"])
+    ws = tw.new_workspace(tw.OP_LINEAR_FWD) if with_ws else None
+    y = tw.fp8_linear_fwd(xq, wq, sx, sw, ws=ws)
+    y2 = tw.fp8_linear_fwd(xq, wq, sx, sw, ws=ws)
+    torch.cuda.synchronize()
+    assert tw.read_device_status() == 0
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
+    ref = orc.gemm_fwd(qx["q"], E4M3, qw["q"], E4M3, qx["scale_inv"], qw["scale_inv"])
+    got = y.float().cpu().numpy().astype(np.float64)
+    assert rel_fro(got, ref) <= GEMM_TOL
+    scale = np.max(np.abs(ref)) + 1e-300
+    assert np.max(np.abs(got - ref) - np.abs(ref) * 2.0 ** -8) <= 1e-4 * scale
+
+
 # ------------------------------------------------------------------ static W8A8
 @pytest.mark.parametrize("M", [1, 16, 128, 1024])
 def test_w8a8_static_gemm(tw, M):
