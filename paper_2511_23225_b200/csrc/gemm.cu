@@ -613,7 +613,7 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   p.Mpad = (int32_t)((M + 15) / 16 * 16);
   p.k_blocks = (int32_t)((K + BK - 1) / BK);
   p.stage_bytes = (uint32_t)((BM * BK + p.Mpad * 128 + 1023) / 1024 * 1024);
-  p.stages = (int32_t)((100 * 1024) / p.stage_bytes);
+  p.stages = (int32_t)((200 * 1024) / p.stage_bytes);
   if (p.stages > kSkinnyMaxStages) p.stages = kSkinnyMaxStages;
   p.tmem_cols = p.Mpad <= 32 ? 32u : (p.Mpad <= 64 ? 64u : 128u);
   p.idesc = make_idesc(fmt_w, fmt_x, false, false, p.Mpad, BM);
@@ -623,8 +623,10 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   const int slabs = (int)((N + 127) / 128);
   p.slices = 1;
   if (ws && aligned16(ws) && ws_bytes >= kWsPartialsOffset + (size_t)sms * kWsPartialBytesPerSm && slabs <= 512) {
-    int s = (2 * sms) / slabs;                       // two CTAs per SM
+    int s = sms / slabs;                             // one CTA per SM
     if (s > p.k_blocks / 4) s = p.k_blocks / 4;      // at least four k-blocks per slice
+    // parking partial sums pays for a few tokens, or for a very long K
+    if (p.Mpad > 32) s = (p.k_blocks >= 64 && s >= 2) ? 2 : 1;
     while (s > 1 && (size_t)slabs * s * p.Mpad * 128 * sizeof(float) > (size_t)sms * kWsPartialBytesPerSm) --s;
     if (s > 1) {
       p.slices = s;
@@ -641,7 +643,7 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   static bool attr_done = false;
   if (!attr_done) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(gemm_fp8_skinny_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)(kSkinnyMaxStages * 16384 + 4096)));
+                                       (int)(200 * 1024 + 1024 + 256)));
     attr_done = true;
   }
   gemm_fp8_skinny_kernel<<<slabs * p.slices, kThreads, smem, st>>>(mw, mx, p);

@@ -3,14 +3,14 @@
 // the kernel is organised around that: the operands are swapped -- 128 rows of W are the
 // MMA's M dimension, the (padded) tokens its N dimension -- so the accumulator is only
 // 128 x Mpad and nothing but W moves in bulk.  Each CTA takes one 128-row slab of W and one
-// slice of K; slabs x slices is chosen to put two CTAs on every SM, each with its own ring of
-// TMA stages, which keeps about 100 KB of loads in flight per SM.
+// slice of K; slabs x slices is chosen to give every SM one CTA with a deep ring of TMA stages
+// (up to 200 KB of loads in flight per SM).
 //
 // CTA = 192 threads: warp 0 issues TMA loads (W slab 128 x 128 B and X 'Mpad' x 128 B per
 // k-block, 128-byte swizzle, rows beyond M zero-filled), warp 1 owns tensor memory and issues
 // tcgen05.mma kind::f8f6f4 128 x Mpad x 32, warps 2-5 read the accumulator (lane = row of W =
 // output column) and write Y.  With K sliced, every CTA parks its fp32 partial sums in the
-// workspace ([token][128 columns], a few KB), takes a ticket per (slab, warp), and the warp
+// workspace ([column][token], a few KB), takes a ticket per (slab, warp), and the warp
 // that draws the last ticket adds the slices in slice order and stores -- nobody waits, and
 // the sum does not depend on timing.  All mbarrier waits are bounded.
 #pragma once
@@ -22,7 +22,7 @@
 
 namespace tweo_detail {
 
-constexpr int kSkinnyMaxStages = 8;
+constexpr int kSkinnyMaxStages = 11;
 
 struct SkinnyParams {
   uint16_t* y;
@@ -36,7 +36,7 @@ struct SkinnyParams {
   uint32_t idesc;
   const float* sx_inv;
   const float* sw_inv;
-  float* partials;         // [slab][slice][Mpad][128] fp32, used when slices > 1
+  float* partials;         // [slab][slice][128 columns][Mpad] fp32, used when slices > 1
   uint32_t* counters;      // [slab][4] tickets, zero between launches
 };
 
@@ -51,7 +51,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "memory");
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                        const __grid_constant__ SkinnyParams p) {
   extern __shared__ uint8_t smem_dyn[];
@@ -147,14 +147,18 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
           }
         }
       } else {
-        // park the partial sums: [token][128 columns], 32 lanes write 128 contiguous bytes
-        float* mine = p.partials + ((size_t)(slab * p.slices + slice) * p.Mpad) * 128 + quarter * 32 + lane;
+        // park the partial sums: [column][token], a lane writes its column's tokens contiguously
+        const size_t unit_floats = (size_t)128 * p.Mpad;
+        float* mine = p.partials + (size_t)(slab * p.slices + slice) * unit_floats + (size_t)(quarter * 32 + lane) * p.Mpad;
         for (int c = 0; c < p.Mpad; c += 16) {
           uint32_t r[16];
           tmem_ld16(tacc + (uint32_t)c, r);
           tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 16; ++j) __stcg(mine + (size_t)(c + j) * 128, __uint_as_float(r[j]));
+          for (int j = 0; j < 16; j += 4)
+            __stcg(reinterpret_cast<float4*>(mine + c + j),
+                   make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                               __uint_as_float(r[j + 3])));
         }
         __threadfence();
         __syncwarp();
@@ -165,22 +169,41 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
         if (ticket + 1 == (uint32_t)p.slices) {  // the last slice of this slab: add all slices in order
           __threadfence();
           if (lane == 0) *counter = 0u;  // ready for the next launch
-          const float* base = p.partials + ((size_t)slab * p.slices * p.Mpad) * 128 + quarter * 32 + lane;
-          const size_t slice_stride = (size_t)p.Mpad * 128;
-          for (int m = 0; m < p.M; m += 8) {
-            float acc[8];
+          const float* base = p.partials + (size_t)slab * p.slices * unit_floats + (size_t)(quarter * 32 + lane) * p.Mpad;
+          // 16 tokens of this column at a time, the loads of eight slices in flight together
+          // (32 independent 16-byte loads); the additions still run in slice order
+          for (int m = 0; m < p.M; m += 16) {
+            float4 acc[4];
+#pragma unroll 1
+            for (int s0 = 0; s0 < p.slices; s0 += 8) {
+              float4 v[8][4];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
-            for (int s = 0; s < p.slices; ++s) {
+              for (int t = 0; t < 8; ++t) {
+                const float4* src = reinterpret_cast<const float4*>(base + (size_t)(s0 + t) * unit_floats + m);
 #pragma unroll
-              for (int j = 0; j < 8; ++j)  // rows up to Mpad exist in the workspace (zeros beyond M)
-                acc[j] = s == 0 ? __ldcg(base + s * slice_stride + (size_t)(m + j) * 128)
-                                : acc[j] + __ldcg(base + s * slice_stride + (size_t)(m + j) * 128);
+                for (int j = 0; j < 4; ++j) v[t][j] = (s0 + t < p.slices) ? __ldcg(src + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+              }
+#pragma unroll
+              for (int t = 0; t < 8; ++t) {
+                if (s0 + t < p.slices) {
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    if (s0 + t == 0) acc[j] = v[t][j];
+                    else acc[j] = make_float4(acc[j].x + v[t][j].x, acc[j].y + v[t][j].y, acc[j].z + v[t][j].z,
+                                              acc[j].w + v[t][j].w);
+                  }
+                }
+              }
             }
             if (col < p.N) {
 #pragma unroll
-              for (int j = 0; j < 8; ++j)
-                if (m + j < p.M) p.y[(int64_t)(m + j) * p.ldy + col] = (uint16_t)f32_to_bf16_bits(__fmul_rn(acc[j], alpha));
+              for (int j = 0; j < 4; ++j) {
+                const float a4[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (m + 4 * j + e < p.M)
+                    p.y[(int64_t)(m + 4 * j + e) * p.ldy + col] = (uint16_t)f32_to_bf16_bits(__fmul_rn(a4[e], alpha));
+              }
             }
           }
         }
