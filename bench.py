@@ -294,6 +294,35 @@ def measure_workload(torch, tw, cfg_idx, steps, warmup, world, barrier, want_e2e
     return res
 
 
+def w8a8_sweep(torch, tw, peaks, reps=10):
+    """Config 5: the static per-tensor W8A8 linear at LLaMA-7B shapes, E4M3 codes in (the cast of bf16
+    activations is the GIVEN-scale cast timed elsewhere).  Each call is replayed `reps` times from a CUDA
+    graph between two events.  M <= 128 is bound by streaming W (bytes / time against the HBM copy
+    peak; in this back-to-back replay W may partly sit in the 126 MB L2), larger M by the tensor pipe."""
+    side = torch.cuda.Stream()
+    one = torch.ones(1, dtype=torch.float32, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(5)
+    rows = []
+    for K, N in ((4096, 4096), (4096, 11008), (11008, 4096)):
+        wq = torch.randint(0, 256, (N, K), dtype=torch.uint8, device="cuda", generator=g) & 0xBF  # finite codes
+        for M in (1, 16, 128, 1024, 8192):
+            xq = torch.randint(0, 256, (M, K), dtype=torch.uint8, device="cuda", generator=g) & 0xBF
+            y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            ws = tw.new_workspace(tw.OP_W8A8, M, N, K)
+            fn = lambda: [tw.w8a8_static_gemm(xq, one, wq, one, y=y, ws=ws) for _ in range(reps)]
+            fn()
+            torch.cuda.synchronize()
+            us = 1e3 * _time_replays(torch, _graph_of(torch, side, fn), 5) / reps
+            flops, nbytes = 2.0 * M * K * N, float(M * K + K * N + 2 * M * N)
+            hbm_us, tc_us = nbytes / peaks["hbm"] / 1e3, flops / (2.0 * peaks["bf16"]) / 1e6
+            rows.append({"M": M, "K": K, "N": N, "us": us, "tflops": flops / us / 1e6, "gbs": nbytes / us / 1e3,
+                         "bound": "hbm" if hbm_us > tc_us else "tensor", "frac_of_roofline": max(hbm_us, tc_us) / us})
+            del xq, y, ws
+        del wq
+        torch.cuda.empty_cache()
+    return rows
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -380,6 +409,12 @@ def run_cuda(args):
             del obs, o
             torch.cuda.empty_cache()
 
+    w8a8 = None
+    if world == 1 and not args.no_w8a8:
+        w8a8 = w8a8_sweep(torch, tw, peaks)
+        if tw.read_device_status() != 0:
+            raise SystemExit("device status reports an expired wait")
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -399,6 +434,8 @@ def run_cuda(args):
         }
         if others:
             line["other_workloads"] = others
+        if w8a8:
+            line["cfg5_w8a8_static_gemm"] = w8a8
         if world == 1 and not args.no_cpu_baseline:
             f, t = oracle_sample_step(cfg_idx, args.cpu_rows)
             line["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
@@ -423,6 +460,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--also", default="cfg4", help="comma-separated other configs to run briefly (N=1 only); '' for none")
     ap.add_argument("--also-steps", type=int, default=20)
+    ap.add_argument("--no-w8a8", action="store_true", help="skip the config 5 inference GEMM sweep")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps > 50:
