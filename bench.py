@@ -326,6 +326,23 @@ def w8a8_sweep(torch, tw, peaks, reps=10):
     return rows
 
 
+def max_over_ranks(value: float, device) -> float:
+    """The slowest rank's time decides: MAX-allreduce of one float (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        t = torch.tensor([value], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+    return value
+
+
+def whole_job_value(flops_per_rank_step: float, ms_per_step: float, world: int) -> float:
+    """Weak scaling: every rank runs its own token shard, so the job's rate is the sum over ranks of the
+    per-rank work divided by the slowest rank's time."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -348,20 +365,13 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(v):
-        if world > 1:
-            t = torch.tensor([v], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return v
-
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     r = measure_workload(torch, tw, cfg_idx, args.steps, args.warmup, world, barrier, True, e2e_steps, local)
     bs = r["bs"]
-    ms_per_step = max_over_ranks(r["ms_per_step"])
-    e2e_ms = max_over_ranks(r["e2e_ms_per_step"])
-    value = world * bs.flops_per_step / (ms_per_step * 1e-3) / 1e12
-    e2e_value = world * bs.flops_per_step / (e2e_ms * 1e-3) / 1e12
+    ms_per_step = max_over_ranks(r["ms_per_step"], "cuda")
+    e2e_ms = max_over_ranks(r["e2e_ms_per_step"], "cuda")
+    value = whole_job_value(bs.flops_per_step, ms_per_step, world)
+    e2e_value = whole_job_value(bs.flops_per_step, e2e_ms, world)
     kernels = r["kernels"]
 
     # Roofline of the dominant kernel family.  FP8 dense peak = 2 x the measured bf16 figure (nominal
