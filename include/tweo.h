@@ -197,6 +197,24 @@ TWEO_API tweo_status_t tweo_fp8_linear_bwd_wgrad(const uint8_t* xq, int64_t ldx,
                                         void* stream);
 
 /*
+ * tweo_fp8_linear_bwd -- both gradients of a linear layer in one call (Sec. 4.2): exactly
+ *   tweo_fp8_linear_bwd_dgrad (dX, bf16) followed by tweo_fp8_linear_bwd_wgrad (dW, bf16,
+ *   overwrite), without fused epilogue outputs; results are bit-identical to the two calls.
+ *   When M, N and K all exceed 128 the two products run as ONE kernel launch: their tiles
+ *   form one list, longest first, dealt to the CTA pairs so that each pair gets about the
+ *   same work (the weight gradient has few, long tiles; the data gradient many short ones),
+ *   which removes most of the idle SM time the two products have on their own at
+ *   transformer-block sizes.  Otherwise it makes the two calls one after the other.
+ *   Arguments as in the two calls; ws is only used on the two-call path (may be NULL).
+ */
+TWEO_API tweo_status_t tweo_fp8_linear_bwd(const uint8_t* dyq, int64_t lddy, int32_t fmt_dy,
+                                  const uint8_t* xq, int64_t ldx, int32_t fmt_x, const uint8_t* wq,
+                                  int64_t ldw, int32_t fmt_w, const float* sdy_inv, const float* sx_inv,
+                                  const float* sw_inv, uint16_t* dx, int64_t lddx, uint16_t* dw,
+                                  int64_t lddw, int64_t M, int64_t N, int64_t K, void* ws,
+                                  size_t ws_bytes, void* stream);
+
+/*
  * tweo_loss_fwd_bwd -- TWEO penalty and its gradient in one pass (Eq. 3, and
  * the derivative of Eq. 2's lambda(t) * L_TWEO term):
  *   loss_l = (1/n) sum_i (|a_i| / (tau+eps))^p,          l = 0..L-1

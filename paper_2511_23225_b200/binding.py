@@ -24,7 +24,7 @@ LIB_PATH = os.path.join(_HERE, "libtweo_b200.so")
 
 EXPORTS = [
     "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_bwd_dgrad",
-    "tweo_fp8_linear_bwd_wgrad", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
+    "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
 ]
@@ -75,6 +75,8 @@ def lib() -> C.CDLL:
                                                 C.POINTER(_Epilogue), vp, sz, vp]
         L.tweo_fp8_linear_bwd_wgrad.argtypes = [vp, i64, i32, vp, i64, i32, vp, vp, vp, i64, i32, i32,
                                                 i64, i64, i64, vp, sz, vp]
+        L.tweo_fp8_linear_bwd.argtypes = [vp, i64, i32, vp, i64, i32, vp, i64, i32, vp, vp, vp, vp, i64, vp, i64,
+                                          i64, i64, i64, vp, sz, vp]
         L.tweo_loss_fwd_bwd.argtypes = [C.POINTER(vp), i32, i64, f32, f32, f32, f32, vp, vp, C.POINTER(vp), i32,
                                         vp, sz, vp]
         L.tweo_loss_fwd_bwd_static.argtypes = [C.POINTER(vp), i32, i64, f32, f32, f32, f32, vp, vp, C.POINTER(vp),
@@ -280,6 +282,26 @@ def fp8_linear_bwd_wgrad(xq, dyq, sx_inv, sdy_inv, fmt_x=E4M3, fmt_dy=E5M2, dw=N
                                            dw_dtype, 1 if accumulate else 0, M, N, K, *_ws(ws), _stream()),
            "tweo_fp8_linear_bwd_wgrad")
     return dw
+
+
+def fp8_linear_bwd(dyq, xq, wq, sdy_inv, sx_inv, sw_inv, fmt_dy=E5M2, fmt_x=E4M3, fmt_w=E4M3, dx=None, dw=None, ws=None):
+    """tweo_fp8_linear_bwd: dX[M,K] and dW[N,K] (both bf16) of one linear layer in one call."""
+    M, N = dyq.shape
+    M2, K = xq.shape
+    N2, K2 = wq.shape
+    if M != M2 or N != N2 or K != K2:
+        raise ValueError("shapes of dyq [M,N], xq [M,K] and wq [N,K] do not agree")
+    if dx is None:
+        dx = torch.empty((M, K), dtype=torch.bfloat16, device=dyq.device)
+    if dw is None:
+        dw = torch.empty((N, K), dtype=torch.bfloat16, device=dyq.device)
+    _check(lib().tweo_fp8_linear_bwd(_dev(dyq, U8, "dyq"), _rows(dyq, "dyq"), fmt_dy, _dev(xq, U8, "xq"),
+                                     _rows(xq, "xq"), fmt_x, _dev(wq, U8, "wq"), _rows(wq, "wq"), fmt_w,
+                                     _dev(sdy_inv, torch.float32), _dev(sx_inv, torch.float32),
+                                     _dev(sw_inv, torch.float32), _dev(dx, torch.bfloat16, "dx"), _rows(dx, "dx"),
+                                     _dev(dw, torch.bfloat16, "dw"), _rows(dw, "dw"), M, N, K, *_ws(ws), _stream()),
+           "tweo_fp8_linear_bwd")
+    return dx, dw
 
 
 def loss_fwd_bwd(blocks, tau=3.0, eps=1e-6, p=4.0, grad_coeff=1.0, want_grad=True, grad_dtype=BF16,

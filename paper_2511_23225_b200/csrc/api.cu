@@ -60,7 +60,7 @@ const char* tweo_status_string(tweo_status_t s) {
 
 const char* tweo_last_cuda_error(void) { return g_err; }
 
-int32_t tweo_version(void) { return 200; }
+int32_t tweo_version(void) { return 210; }
 
 uint64_t tweo_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

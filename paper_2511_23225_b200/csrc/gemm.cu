@@ -37,11 +37,15 @@
 #include <atomic>
 #include <cstdlib>
 #include <mutex>
+#include <queue>
+#include <utility>
+#include <vector>
 
 #include "common.cuh"
 
 #include "gemm_common.cuh"
 #include "gemm_pair.cuh"
+#include "gemm_pair_group.cuh"
 #include "gemm_skinny.cuh"
 #include "tc_ptx.cuh"
 
@@ -422,6 +426,8 @@ std::atomic<uint32_t> g_sk_epoch{0};
 // TWEO_GEMM_NO_PAIR=1 in the environment keeps every GEMM on the single-CTA kernel (A/B timing).
 // TWEO_GEMM_NO_SKINNY=1 sends small-M forward products through the general kernels (A/B timing).
 const bool g_disable_skinny = [] { const char* e = getenv("TWEO_GEMM_NO_SKINNY"); return e && e[0] == '1'; }();
+// TWEO_GEMM_NO_GROUP=1 makes tweo_fp8_linear_bwd run its two products as two launches (A/B timing).
+const bool g_disable_group = [] { const char* e = getenv("TWEO_GEMM_NO_GROUP"); return e && e[0] == '1'; }();
 const bool g_disable_pair = [] { const char* e = getenv("TWEO_GEMM_NO_PAIR"); return e && e[0] == '1'; }();
 
 // Band height of the tile numbering: the `workers` tiles in flight cover about g x workers/g
@@ -651,6 +657,104 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   return check_launch("gemm_fp8_skinny_kernel");
 }
 
+// dX and dW of one linear layer in ONE launch of the CTA-pair kernel (see gemm_pair_group.cuh).
+tweo_status_t run_bwd_group(const uint8_t* dyq, int64_t lddy, int fmt_dy, const uint8_t* xq, int64_t ldx, int fmt_x,
+                            const uint8_t* wq, int64_t ldw, int fmt_w, const float* sdy_inv, const float* sx_inv,
+                            const float* sw_inv, uint16_t* dx, int64_t lddx, uint16_t* dw, int64_t lddw, int64_t M,
+                            int64_t N, int64_t K, cudaStream_t st) {
+  constexpr int STAGES = 6;
+  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
+  auto kern = gemm_fp8_pair_group_kernel<STAGES>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_done = true;
+  }
+  const int pairs_all = sm_count() / 2;
+  PairGroupParams g;
+  // product D: dX[M,K] = dYq[M,N] . Wq[N,K] (contraction N); product W: dW[N,K] = dYq^T . Xq (contraction M)
+  struct Desc {
+    const uint8_t *a, *b;
+    int64_t lda, ldb, Md, Nd, Kc;
+    int fa, fb;
+    bool a_mn;
+    uint16_t* d;
+    int64_t ldd;
+    const float *sa, *sb;
+  } d[2] = {{dyq, wq, lddy, ldw, M, K, N, fmt_dy, fmt_w, false, dx, lddx, sdy_inv, sw_inv},
+            {dyq, xq, lddy, ldx, N, K, M, fmt_dy, fmt_x, true, dw, lddw, sdy_inv, sx_inv}};
+  // the product with the longer tiles goes first in the tile list
+  if ((d[1].Kc + BK - 1) / BK > (d[0].Kc + BK - 1) / BK) std::swap(d[0], d[1]);
+  int tiles[2], cost[2];
+  for (int i = 0; i < 2; ++i) {
+    GroupProblem& q = g.pr[i];
+    q.Md = (int32_t)d[i].Md;
+    q.Nd = (int32_t)d[i].Nd;
+    q.tiles_m = (int32_t)((d[i].Md + 2 * BM - 1) / (2 * BM));
+    q.tiles_n = (int32_t)((d[i].Nd + 255) / 256);
+    q.k_blocks = (int32_t)((d[i].Kc + BK - 1) / BK);
+    q.raster_g = raster_band(q.tiles_m, pairs_all);
+    q.a_mn = d[i].a_mn ? 1 : 0;
+    q.b_mn = 1;
+    q.idesc = make_idesc(d[i].fa, d[i].fb, d[i].a_mn, true, 256, 256);
+    q.sa_inv = d[i].sa;
+    q.sb_inv = d[i].sb;
+    tiles[i] = q.tiles_m * q.tiles_n;
+    cost[i] = (q.k_blocks < 8 ? 8 : q.k_blocks) + 2;  // k-blocks, with a floor for the epilogue of short tiles
+    bool ok = make_out_map(&g.md[i], d[i].d, d[i].Nd, d[i].Md, d[i].ldd, false);
+    if (d[i].a_mn) ok = ok && make_map(&g.ma[i], d[i].a, d[i].Md, d[i].Kc, d[i].lda, BK);
+    else ok = ok && make_map(&g.ma[i], d[i].a, d[i].Kc, d[i].Md, d[i].lda, BM);
+    ok = ok && make_map(&g.mb[i], d[i].b, d[i].Nd, d[i].Kc, d[i].ldb, BK);
+    if (!ok) {
+      cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+      return TWEO_ERR_CUDA;
+    }
+  }
+  g.tiles0 = tiles[0];
+  g.total_tiles = tiles[0] + tiles[1];
+  g.pad = 0;
+  int pairs = pairs_all < g.total_tiles ? pairs_all : g.total_tiles;
+  g.use_lists = (g.total_tiles <= kGroupMaxTiles && pairs <= kGroupMaxPairs) ? 1 : 0;
+  if (g.use_lists) {
+    // longest processing time first: every tile goes to the pair with the least work so far
+    typedef std::pair<int64_t, int> Load;  // (work, pair); smallest on top, ties to the lower pair index
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int p = 0; p < pairs; ++p) heap.push(Load(0, p));
+    uint8_t owner[kGroupMaxTiles];
+    int count[kGroupMaxPairs + 1] = {0};
+    for (int t = 0; t < g.total_tiles; ++t) {
+      Load l = heap.top();
+      heap.pop();
+      owner[t] = (uint8_t)l.second;
+      ++count[l.second];
+      l.first += cost[t < tiles[0] ? 0 : 1];
+      heap.push(l);
+    }
+    int fill[kGroupMaxPairs + 1];
+    g.first[0] = 0;
+    for (int p = 0; p < pairs; ++p) {
+      g.first[p + 1] = (uint16_t)(g.first[p] + count[p]);
+      fill[p] = g.first[p];
+    }
+    for (int t = 0; t < g.total_tiles; ++t) g.list[fill[owner[t]]++] = (uint16_t)t;  // ascending t within a pair
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, g));
+  count_launch();
+  return check_launch("gemm_fp8_pair_group_kernel");
+}
+
 bool fmt_ok(int f) { return f == TWEO_E4M3 || f == TWEO_E5M2; }
 
 tweo_status_t fill_epilogue(GemmParams& p, const tweo_epilogue_t* epi) {
@@ -774,5 +878,29 @@ tweo_status_t tweo_fp8_linear_bwd_wgrad(const uint8_t* xq, int64_t ldx, int32_t 
                   (cudaStream_t)stream);
 }
 
-}  // extern "C"
+tweo_status_t tweo_fp8_linear_bwd(const uint8_t* dyq, int64_t lddy, int32_t fmt_dy, const uint8_t* xq, int64_t ldx,
+                                  int32_t fmt_x, const uint8_t* wq, int64_t ldw, int32_t fmt_w, const float* sdy_inv,
+                                  const float* sx_inv, const float* sw_inv, uint16_t* dx, int64_t lddx, uint16_t* dw,
+                                  int64_t lddw, int64_t M, int64_t N, int64_t K, void* ws, size_t ws_bytes,
+                                  void* stream) {
+  if (!dyq || !xq || !wq || !sdy_inv || !sx_inv || !sw_inv || !dx || !dw) return TWEO_ERR_INVALID_ARG;
+  if (!fmt_ok(fmt_dy) || !fmt_ok(fmt_x) || !fmt_ok(fmt_w)) return TWEO_ERR_INVALID_ARG;
+  if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
+  if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  if (!tweo_detail::aligned16(dyq) || !tweo_detail::aligned16(xq) || !tweo_detail::aligned16(wq) ||
+      !tweo_detail::aligned16(dx) || !tweo_detail::aligned16(dw) || (lddy & 15) || (ldx & 15) || (ldw & 15) ||
+      (lddx & 7) || (lddw & 7))
+    return TWEO_ERR_ALIGNMENT;
+  // both outputs large enough for 256 x 256 tiles: one launch; else the two products one after the other
+  if (M > 128 && N > 128 && K > 128 && !g_disable_pair && !g_disable_group)
+    return run_bwd_group(dyq, lddy, fmt_dy, xq, ldx, fmt_x, wq, ldw, fmt_w, sdy_inv, sx_inv, sw_inv, dx, lddx, dw, lddw,
+                         M, N, K, (cudaStream_t)stream);
+  tweo_status_t s = tweo_fp8_linear_bwd_dgrad(dyq, lddy, fmt_dy, wq, ldw, fmt_w, sdy_inv, sw_inv, dx, lddx, M, N, K,
+                                              nullptr, ws, ws_bytes, stream);
+  if (s != TWEO_OK) return s;
+  return tweo_fp8_linear_bwd_wgrad(xq, ldx, fmt_x, dyq, lddy, fmt_dy, sx_inv, sdy_inv, dw, lddw, TWEO_BF16, 0, M, N, K,
+                                   ws, ws_bytes, stream);
+}
 
+}  // extern "C"

@@ -1,0 +1,276 @@
+// Two FP8 GEMMs in one launch of the CTA-pair kernel: the data gradient and the weight gradient
+// of a linear layer, which the backward pass needs together and which share dY.  Launched
+// separately, each leaves SMs idle -- the weight gradient of a transformer linear has only a few
+// dozen (long) tiles, the data gradient often 1.3 waves of short ones.  Here the tiles of both
+// products form one list, longest first, and the host assigns them to the CTA pairs by the
+// longest-processing-time rule (each tile goes to the pair with the least work so far), so the
+// long tiles start at once and the short ones fill in around them; one ramp-up and one tail
+// instead of two.
+//
+// The kernel is the CTA-pair kernel of gemm_pair.cuh (256 x 256 tiles, tcgen05 cta_group::2,
+// TMA-fed ring, two accumulators in tensor memory, staged TMA-store epilogue) with the operand
+// layouts taken at run time per product, bf16 outputs only, no fused epilogue and no splitting
+// along the contraction.  Every wait is bounded.
+#pragma once
+
+#include <cuda.h>
+
+#include "gemm_common.cuh"
+#include "tc_ptx.cuh"
+
+namespace tweo_detail {
+
+constexpr int kGroupMaxTiles = 1024;  // beyond that the tiles are dealt round-robin (balance is no issue then)
+constexpr int kGroupMaxPairs = 127;
+
+struct GroupProblem {
+  int32_t Md, Nd;
+  int32_t tiles_m, tiles_n, k_blocks, raster_g;
+  int32_t a_mn, b_mn;  // operand stored [Kc, rows] (1) or [rows, Kc] (0)
+  uint32_t idesc;
+  const float* sa_inv;
+  const float* sb_inv;
+};
+
+struct alignas(64) PairGroupParams {
+  CUtensorMap ma[2], mb[2], md[2];
+  GroupProblem pr[2];
+  int32_t tiles0;        // tiles of product 0; they are numbered first
+  int32_t total_tiles;
+  int32_t use_lists;     // the per-pair lists are valid (total_tiles <= kGroupMaxTiles)
+  int32_t pad;
+  uint16_t first[kGroupMaxPairs + 1];  // pair p computes list[first[p]] .. list[first[p + 1] - 1], in that order
+  uint16_t list[kGroupMaxTiles];       // tile numbers
+};
+
+// The tile list of one CTA pair, identical in every warp role.
+struct GroupSched {
+  int pos, end, t, worker, workers;
+  __device__ GroupSched(const PairGroupParams& g, int worker_, int workers_)
+      : pos(g.use_lists ? g.first[worker_] : 0), end(g.use_lists ? g.first[worker_ + 1] : 0), t(-1), worker(worker_),
+        workers(workers_) {}
+  __device__ bool next(const PairGroupParams& g, int& prob, int& tile) {
+    if (g.use_lists) {
+      if (pos >= end) return false;
+      t = g.list[pos++];
+    } else {
+      t = t < 0 ? worker : t + workers;
+      if (t >= g.total_tiles) return false;
+    }
+    prob = t >= g.tiles0 ? 1 : 0;
+    tile = prob ? t - g.tiles0 : t;
+    return true;
+  }
+};
+
+__device__ __forceinline__ void group_tile_coords(const GroupProblem& q, int tile, int& tm, int& tn) {
+  const int per_band = q.raster_g * q.tiles_n;
+  const int band = tile / per_band;
+  const int first = band * q.raster_g;
+  const int rows = min(q.raster_g, q.tiles_m - first);
+  const int in = tile - band * per_band;
+  tn = in / rows;
+  tm = first + in - tn * rows;
+}
+
+template <int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams g) {
+  constexpr int BN = 256;                 // tile columns of the pair
+  constexpr uint32_t A_BYTES = BM * BK;   // this CTA's 128 rows of A
+  constexpr uint32_t B_BYTES = 128 * BK;  // this CTA's 128 of the 256 columns of B
+  constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr uint32_t TMEM_COLS = 512;
+  constexpr int CH = 64;                  // bf16 columns per 128-byte staging row
+
+  extern __shared__ uint8_t smem_dyn[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  constexpr uint32_t EPI_BUF = 32 * 128;
+  constexpr uint32_t EPI_BYTES = 4 * 2 * EPI_BUF;
+  uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES);
+  // bars: [0,STAGES) full, [STAGES,2*STAGES) empty, then tfull[2], tempty[2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 8);  // four epilogue warps of each CTA of the pair
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // both CTAs' barriers are initialised before anyone signals across
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int pair = blockIdx.x >> 1;
+  const int num_pairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      GroupSched sched(g, pair, num_pairs);
+      int prob, tile;
+      while (ok && sched.next(g, prob, tile)) {
+        const GroupProblem& q = g.pr[prob];
+        int tm, tn;
+        group_tile_coords(q, tile, tm, tn);
+        const int m0 = tm * (2 * BM) + (int)rank * BM;  // this CTA's rows
+        const int n0 = tn * BN + (int)rank * 128;       // this CTA's half of B
+        const bool a_mn = q.a_mn != 0, b_mn = q.b_mn != 0;
+        const CUtensorMap* ma = &g.ma[prob];
+        const CUtensorMap* mb = &g.mb[prob];
+        for (int kb = 0; kb < q.k_blocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
+          const uint32_t fb = map_to_cta(full_bar(stage), 0);
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+          const int k0 = kb * BK;
+          if (a_mn) tma_load_2d_pair(sa, ma, m0, k0, fb);
+          else tma_load_2d_pair(sa, ma, k0, m0, fb);
+          if (b_mn) tma_load_2d_pair(sb, mb, n0, k0, fb);
+          else tma_load_2d_pair(sb, mb, k0, n0, fb);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && leader) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      GroupSched sched(g, pair, num_pairs);
+      int prob, tile;
+      while (ok && sched.next(g, prob, tile)) {
+        const GroupProblem& q = g.pr[prob];
+        // K-major: step 32 bytes inside the swizzle span; MN-major: step 32 rows of 128 B
+        const uint32_t a_step = q.a_mn ? UMMA_K * 128 : UMMA_K;
+        const uint32_t b_step = q.b_mn ? UMMA_K * 128 : UMMA_K;
+        const uint32_t idesc = q.idesc;
+        const int k_blocks = q.k_blocks;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_f8_pair(d_tmem, make_smem_desc(sa + k * a_step, BK * 128), make_smem_desc(sb + k * b_step, BK * 128),
+                         idesc, (uint32_t)((kb | k) != 0));
+          umma_commit_pair(map_to_cta(empty_bar(stage), 0));  // frees the stage in both CTAs
+          umma_commit_pair(map_to_cta(empty_bar(stage), 1));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit_pair(map_to_cta(tfull_bar(acc), 0));      // accumulator complete, both CTAs
+        umma_commit_pair(map_to_cta(tfull_bar(acc), 1));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    const int quarter = warp & 3;
+    const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
+    const uint32_t row_off = (uint32_t)lane * 128u;
+    const uint32_t swz = (uint32_t)(lane & 7);
+    const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
+    uint32_t it = 0;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    GroupSched sched(g, pair, num_pairs);
+    int prob, tile;
+    while (ok && sched.next(g, prob, tile)) {
+      const GroupProblem& q = g.pr[prob];
+      const CUtensorMap* md = &g.md[prob];
+      const float alpha = __fmul_rn(__ldg(q.sa_inv), __ldg(q.sb_inv));
+      const int Md = q.Md, Nd = q.Nd;
+      int tm, tn;
+      group_tile_coords(q, tile, tm, tn);
+      const int m0 = tm * (2 * BM) + (int)rank * BM;
+      const int n0 = tn * BN;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row0 = m0 + quarter * 32;
+#pragma unroll 1
+      for (int c = 0; c < BN / CH; ++c) {
+        const int col0 = n0 + c * CH;
+        if (col0 >= Nd) break;
+        uint32_t r[CH];
+        const uint32_t taddr = tmem_base + tlane + (uint32_t)(acc * BN + c * CH);
+        tmem_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+        tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+        tmem_ld_wait();
+        if (row0 >= Md) continue;
+        const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
+        if (lane == 0) bulk_wait_read<1>();
+        __syncwarp();
+        uint32_t packed[CH / 2];
+#pragma unroll
+        for (int j = 0; j < CH / 2; ++j)
+          packed[j] = f32x2_to_bf16x2(__fmul_rn(__uint_as_float(r[2 * j]), alpha),
+                                      __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha));
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1], packed[4 * j + 2],
+                       packed[4 * j + 3]);
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(md, col0, row0, buf);
+          bulk_commit();
+        }
+        ++it;
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's barrier
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+    if (lane == 0) bulk_wait_all();
+  }
+
+  // Neither CTA may leave (or free tensor memory) while the other can still signal its
+  // barriers or have MMAs reading its shared memory.
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace tweo_detail

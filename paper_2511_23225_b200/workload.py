@@ -2,7 +2,7 @@
 
 A step is one pass of every stage over one batch of synthetic input: for each
 linear of the block, the per-tensor FP8 casts of X, W (E4M3) and dY (E5M2) with
-current scaling, the forward, data-gradient and weight-gradient GEMMs, and then
+current scaling, the forward GEMM and the backward call (data and weight gradient), and then
 the TWEO loss and gradient on the block output(s).  This module only sequences
 library calls and owns the device buffers; all arithmetic happens in the CUDA
 kernels behind ``binding``.
@@ -103,10 +103,9 @@ class BlockStep:
 
     def gemms(self, lb: LinearBuffers):
         tw.fp8_linear_fwd(lb.qx.q, lb.qw.q, lb.qx.scale_inv, lb.qw.scale_inv, y=lb.y, ws=self.gemm_ws)
-        tw.fp8_linear_bwd_dgrad(lb.qdy.q, lb.qw.q, lb.qdy.scale_inv, lb.qw.scale_inv, fmt_dy=self.grad_fmt, dx=lb.dx,
-                                ws=self.gemm_ws)
-        tw.fp8_linear_bwd_wgrad(lb.qx.q, lb.qdy.q, lb.qx.scale_inv, lb.qdy.scale_inv, fmt_dy=self.grad_fmt, dw=lb.dw,
-                                ws=self.gemm_ws)
+        # both gradients in one call (one kernel launch when the shapes allow)
+        tw.fp8_linear_bwd(lb.qdy.q, lb.qx.q, lb.qw.q, lb.qdy.scale_inv, lb.qx.scale_inv, lb.qw.scale_inv,
+                          fmt_dy=self.grad_fmt, dx=lb.dx, dw=lb.dw, ws=self.gemm_ws)
 
     def tweo(self):
         c = self.lam / self.n_blocks

@@ -329,6 +329,38 @@ def test_gemms_split_along_contraction(tw, name, M, K, N, dw_f32):
         assert rel_fro(got.float().cpu().numpy(), plain.float().cpu().numpy().astype(np.float64)) <= 1e-3, what
 
 
+@pytest.mark.parametrize("name,M,K,N", [("cfg1", 512, 256, 1024), ("ragged_all", 300, 400, 272),
+                                        ("block_rows", 2048, 768, 2304), ("small_falls_back", 64, 256, 256)],
+                         ids=["cfg1", "ragged_all", "block_rows", "small_falls_back"])
+@pytest.mark.parametrize("fmt_g", [E5M2, E4M3], ids=["e5m2grad", "e4m3grad"])
+def test_backward_in_one_call_equals_the_two_calls(tw, name, M, K, N, fmt_g):
+    """tweo_fp8_linear_bwd (both gradients, one launch when the shapes allow) against dgrad + wgrad:
+    the same bits, and the oracle's values."""
+    if name == "cfg1":
+        x, w, dy = synth.linear_inputs(1, 0)
+    else:
+        x = synth.normal_with_outlier_channels_bf16(110, (M, K))
+        w = synth.normal_bf16(111, (N, K), 0.02)
+        dy = synth.normal_bf16(112, (M, N), 1e-3)
+    qx, qw, qd = quantized_operands(x, w, dy, fmt_g)
+    xq, wq, dyq = (torch.from_numpy(q["q"]).cuda() for q in (qx, qw, qd))
+    sx, sw, sd = (dev_scalar(q["scale_inv"]) for q in (qx, qw, qd))
+    dx1, dw1 = tw.fp8_linear_bwd(dyq, xq, wq, sd, sx, sw, fmt_dy=fmt_g)
+    dx0 = tw.fp8_linear_bwd_dgrad(dyq, wq, sd, sw, fmt_dy=fmt_g)
+    dw0 = tw.fp8_linear_bwd_wgrad(xq, dyq, sx, sd, fmt_dy=fmt_g)
+    torch.cuda.synchronize()
+    assert tw.read_device_status() == 0
+    assert torch.equal(dx1.view(torch.int16), dx0.view(torch.int16))
+    assert torch.equal(dw1.view(torch.int16), dw0.view(torch.int16))
+    g = np.random.Generator(np.random.PCG64(13))
+    r, c = sample_points(g, M, K, n_rows=2, n_pts=1500)
+    ref = orc.gemm_dgrad_at(qd["q"], fmt_g, qw["q"], E4M3, qd["scale_inv"], qw["scale_inv"], r, c)
+    assert rel_fro(dx1.float().cpu().numpy()[r, c], ref) <= GEMM_TOL
+    r, c = sample_points(g, N, K, n_rows=2, n_pts=1500)
+    ref = orc.gemm_wgrad_at(qx["q"], E4M3, qd["q"], fmt_g, qx["scale_inv"], qd["scale_inv"], r, c)
+    assert rel_fro(dw1.float().cpu().numpy()[r, c], ref) <= GEMM_TOL
+
+
 def test_wgrad_fp32_output_and_accumulate(tw):
     x = synth.normal_bf16(80, (640, 256))
     w = synth.normal_bf16(81, (384, 256), 0.02)
