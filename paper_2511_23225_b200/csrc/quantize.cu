@@ -25,16 +25,22 @@ using namespace tweo_detail;
 
 constexpr int kThreads = 256;
 
-// Largest |x| of a packed pair of bf16, as raw 15-bit-exponent+mantissa patterns, NaN -> 0.
-__device__ __forceinline__ uint32_t absmax_bits(uint32_t m, uint32_t w) {
-  uint32_t lo = w & 0x7FFFu, hi = (w >> 16) & 0x7FFFu;
-  lo = lo > 0x7F80u ? 0u : lo;
-  hi = hi > 0x7F80u ? 0u : hi;
-  return max(m, max(lo, hi));
+// Running maximum of |x| over packed pairs of bf16, kept as two 16-bit lanes of sign-stripped bit
+// patterns (which order like the magnitudes); NaN patterns (> 0x7F80) count as 0.  Four integer
+// SIMD instructions per pair of elements.
+__device__ __forceinline__ uint32_t absmax_bits(uint32_t m2, uint32_t w) {
+  uint32_t a = w & 0x7FFF7FFFu;
+  a &= __vcmpleu2(a, 0x7F807F80u);
+  return __vmaxu2(m2, a);
 }
+// the larger of the two lanes: the bit pattern of max |x| as a bf16 value
+__device__ __forceinline__ uint32_t absmax_fold(uint32_t m2) { return max(m2 & 0xFFFFu, m2 >> 16); }
+// true if either bf16 of the pair is a NaN
+__device__ __forceinline__ bool pair_has_nan(uint32_t w) { return __vcmpgtu2(w & 0x7FFF7FFFu, 0x7F807F80u) != 0u; }
 
-__device__ __forceinline__ void cta_amax_to_global(uint32_t m, float* amax) {
+__device__ __forceinline__ void cta_amax_to_global(uint32_t m2, float* amax) {
   __shared__ uint32_t part[kThreads / 32];
+  uint32_t m = absmax_fold(m2);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
   if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = m;
@@ -80,27 +86,41 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint16_t* x, int64
   cta_amax_to_global(m, amax);
 }
 
-// 16 elements: two 16-byte loads -> one 16-byte store.
+// Two binary32 values -> two FP8 codes, no NaN handling (callers route NaN inputs elsewhere).
 template <int FMT>
-__device__ __forceinline__ uint4 cast16(const uint4 a, const uint4 b, float scale, uint32_t& sat, uint32_t& m,
-                                        bool want_amax) {
+__device__ __forceinline__ uint32_t cvt_fp8x2_finite(float lo, float hi) {
+  uint16_t r;
+  if (FMT == TWEO_E4M3) asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  else asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// 16 elements: two 16-byte loads -> one 16-byte store.  SAT counts elements whose scaled value
+// exceeds the format's range, AMAX folds |x| into the running maximum m2.  The scaled value of a
+// finite or infinite input is never NaN (the scale is positive and finite), so only inputs that
+// are NaN themselves need the converter's NaN fix-up; they are rare and take the slow branch.
+template <int FMT, bool SAT, bool AMAX>
+__device__ __forceinline__ uint4 cast16(const uint4 a, const uint4 b, float scale, uint32_t& sat, uint32_t& m2) {
   const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
   uint32_t c[8];
   const float fmax = FMT == TWEO_E4M3 ? kE4M3Max : kE5M2Max;
+  bool any_nan = false;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) any_nan |= pair_has_nan(w[j]);
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     float lo = __fmul_rn(bf16lo_to_f32(w[j]), scale);
     float hi = __fmul_rn(bf16hi_to_f32(w[j]), scale);
-    sat += (fabsf(lo) > fmax) + (fabsf(hi) > fmax);
-    c[j] = cvt_fp8x2<FMT>(lo, hi);
-    if (want_amax) m = absmax_bits(m, w[j]);
+    if (SAT) sat += (fabsf(lo) > fmax) + (fabsf(hi) > fmax);
+    c[j] = any_nan ? cvt_fp8x2<FMT>(lo, hi) : cvt_fp8x2_finite<FMT>(lo, hi);
+    if (AMAX) m2 = absmax_bits(m2, w[j]);
   }
   return make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16));
 }
 
 // CURRENT mode reads *amax (finished by the previous kernel) and derives the scale;
 // GIVEN mode reads *scale and accumulates amax while casting.
-template <int FMT, bool GIVEN>
+template <int FMT, bool GIVEN, bool SAT>
 __global__ void __launch_bounds__(kThreads)
 cast_kernel(const uint16_t* x, int64_t n, float* scale, float* scale_inv, float* amax, uint8_t* q,
             uint32_t* sat_count) {
@@ -132,7 +152,7 @@ cast_kernel(const uint16_t* x, int64_t n, float* scale, float* scale_inv, float*
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       int64_t i = base + (int64_t)u * kThreads;
-      if (i < n16) __stcs(qv + i, cast16<FMT>(v[u][0], v[u][1], s, sat, m, GIVEN));
+      if (i < n16) __stcs(qv + i, cast16<FMT, SAT, GIVEN>(v[u][0], v[u][1], s, sat, m));
     }
   }
   if (blockIdx.x == 0 && threadIdx.x < 16) {  // ragged tail: n % 16 elements
@@ -145,7 +165,7 @@ cast_kernel(const uint16_t* x, int64_t n, float* scale, float* scale_inv, float*
       if (GIVEN) m = absmax_bits(m, w);
     }
   }
-  if (sat_count) {
+  if (SAT) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sat += __shfl_xor_sync(0xFFFFFFFFu, sat, o);
     if ((threadIdx.x & 31) == 0 && sat) atomicAdd(sat_count, sat);
@@ -217,7 +237,7 @@ __global__ void __launch_bounds__(kThreads) amax_batch_kernel(const __grid_const
       int64_t i = (nvec << 3) + threadIdx.x;
       if (i < n) m = absmax_bits(m, (uint32_t)x[i]);
     }
-    m = cta_max(m, part);
+    m = cta_max(absmax_fold(m), part);
     if (threadIdx.x == 0) slots[ti * kMaxAmaxGrid + blockIdx.x] = m;
   }
 }
@@ -259,7 +279,7 @@ __global__ void __launch_bounds__(kThreads) cast_batch_kernel(const __grid_const
 #pragma unroll
       for (int u = 0; u < 2; ++u) {
         int64_t i = base + (int64_t)u * kThreads;
-        if (i < n16) __stcs(qv + i, cast16<FMT>(v[u][0], v[u][1], s, sat, mm, false));
+        if (i < n16) __stcs(qv + i, cast16<FMT, false, false>(v[u][0], v[u][1], s, sat, mm));
       }
     }
     if (blockIdx.x == 0 && threadIdx.x < 16) {  // ragged tail: n % 16 elements
@@ -332,13 +352,17 @@ tweo_status_t launch_single(const tweo_quant_desc_t& d, cudaStream_t st) {
     count_launch();
   }
   const int grid = grid_for(d.n >> 4, kThreads * 2, 8);
+#define TWEO_CAST(FMT, GIVEN, SAT) \
+  cast_kernel<FMT, GIVEN, SAT><<<grid, kThreads, 0, st>>>(d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count)
+  const bool sat = d.sat_count != nullptr;
   if (d.fmt == TWEO_E4M3) {
-    if (given) cast_kernel<TWEO_E4M3, true><<<grid, kThreads, 0, st>>>(d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count);
-    else cast_kernel<TWEO_E4M3, false><<<grid, kThreads, 0, st>>>(d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count);
+    if (given) { if (sat) TWEO_CAST(TWEO_E4M3, true, true); else TWEO_CAST(TWEO_E4M3, true, false); }
+    else { if (sat) TWEO_CAST(TWEO_E4M3, false, true); else TWEO_CAST(TWEO_E4M3, false, false); }
   } else {
-    if (given) cast_kernel<TWEO_E5M2, true><<<grid, kThreads, 0, st>>>(d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count);
-    else cast_kernel<TWEO_E5M2, false><<<grid, kThreads, 0, st>>>(d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count);
+    if (given) { if (sat) TWEO_CAST(TWEO_E5M2, true, true); else TWEO_CAST(TWEO_E5M2, true, false); }
+    else { if (sat) TWEO_CAST(TWEO_E5M2, false, true); else TWEO_CAST(TWEO_E5M2, false, false); }
   }
+#undef TWEO_CAST
   count_launch();
   return check_launch("tweo_quantize_per_tensor");
 }
