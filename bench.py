@@ -39,9 +39,9 @@ sys.path.insert(0, ROOT)
 METRIC = "fp8_linear_fwd_bwd_tflops_with_tweo_loss"
 UNIT = "TFLOP/s"
 FP8_DATASHEET_TFLOPS = 4500.0
-# DRAM traffic of the dominant kernel family (the 12 GEMM launches of a config-2 step), per launch, from
-# the ncu capture summarised in profiles/gemm_dram_traffic_bench_cfg2.md; valid for that library version only.
-GEMM_TRAFFIC = {"library_version": 200, "workload": "cfg2", "bytes_per_launch": 18.03e6}
+# DRAM traffic of the dominant kernel family (the 8 GEMM launches of a config-2 step), per launch, from
+# the ncu capture summarised in profiles/launch_list_bench_cfg2.md; valid for that library version only.
+GEMM_TRAFFIC = {"library_version": 210, "workload": "cfg2", "bytes_per_launch": 20.45e6}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, FALLBACK_BF16_SUSTAINED = 6650.0, 1590.0, 1400.0
 
 
@@ -390,12 +390,10 @@ def run_cuda(args):
     if dom == "gemm" and tw.version() == GEMM_TRAFFIC["library_version"] and args.workload == GEMM_TRAFFIC["workload"]:
         roof["traffic"] = GEMM_TRAFFIC["bytes_per_launch"]
         roof["algorithmic_bytes_per_launch"] = sum(
-            lb.M * lb.lin.K + lb.lin.K * lb.lin.N + 2 * lb.M * lb.lin.N           # fwd:  X, W in; Y out
-            + lb.M * lb.lin.N + lb.lin.K * lb.lin.N + 2 * lb.M * lb.lin.K         # dgrad: dY, W in; dX out
-            + lb.M * lb.lin.K + lb.M * lb.lin.N + 2 * lb.lin.K * lb.lin.N         # wgrad: X, dY in; dW out
-            for lb in bs.linears) / (3.0 * len(bs.linears))
-    roof["kernel"] = dom
-    roof["avg_launch_us"] = kernels[dom]["avg_launch_us"]
+            lb.M * lb.lin.K + lb.lin.K * lb.lin.N + 2 * lb.M * lb.lin.N             # forward: X, W in; Y out
+            + lb.M * lb.lin.N + lb.lin.K * lb.lin.N + lb.M * lb.lin.K               # backward: dY, W, X in;
+            + 2 * lb.M * lb.lin.K + 2 * lb.lin.K * lb.lin.N                         #           dX, dW out
+            for lb in bs.linears) / (2.0 * len(bs.linears))
 
     workload_cfg = {"workload": workload_name(cfg_idx), "tokens_per_gpu": bs.M,
                     "linears": [f"{l.name}:{l.K}x{l.N}" for l in bs.cfg.linears], "tweo_blocks": bs.n_blocks,
