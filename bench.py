@@ -476,7 +476,7 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=4096)
     ap.add_argument("--ref-rows", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--also", default="cfg4", help="comma-separated other configs to run briefly (N=1 only); '' for none")
+    ap.add_argument("--also", default="cfg4,cfg3", help="comma-separated other configs to run briefly (N=1 only); '' for none")
     ap.add_argument("--also-steps", type=int, default=20)
     ap.add_argument("--no-w8a8", action="store_true", help="skip the config 5 inference GEMM sweep")
     args = ap.parse_args()
