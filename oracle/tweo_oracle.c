@@ -11,7 +11,9 @@
  *     whole tensor, E4M3 forward / E5M2 gradients; E4M3 range +-448 from the
  *     paper's introduction) with the OCP FP8 code tables,
  *   - the three linear-layer contractions on the quantised operands,
- *   - symmetric AbsMax b-bit quantisation (paper Eq. 4).
+ *   - symmetric AbsMax b-bit quantisation (paper Eq. 4),
+ *   - the block output A = x + f(x) the regulariser acts on (paper Sec. 3.3) and the
+ *     delayed-scaling state (paper Sec. 4.2: amax history of length 16).
  *
  * Floating point is FP64 unless the step is *defined* in FP32 (the scale, the
  * scaled value that gets rounded to FP8).  There is no blocking, no SIMD, no
@@ -370,4 +372,37 @@ double oracle_absmax_scale(const double* x, int64_t n, double eps) {
   double m = 0.0;
   for (int64_t i = 0; i < n; ++i) if (fabs(x[i]) > m) m = fabs(x[i]);
   return m + eps;
+}
+
+/* ------------------------------------------------------------------ block output */
+/* The regulariser acts on the block output A^(l) = x + f(x) (Sec. 3.3: the residual
+ * stream plus the block's branch).  With bf16 activations the sum is formed in binary32
+ * and rounded once more to bf16 (round to nearest even): a_i = bf16(fl32(x_i + f_i)).
+ * Everything downstream (Eq. 3, its gradient, amax, the FP8 cast for the next block) is
+ * the functions above applied to these bf16 values. */
+void oracle_residual_add_bf16(const uint16_t* x, const uint16_t* f, int64_t n, uint16_t* a) {
+  for (int64_t i = 0; i < n; ++i) {
+    volatile float s = bf16_bits_to_f32(x[i]) + bf16_bits_to_f32(f[i]); /* one binary32 add */
+    a[i] = oracle_f64_to_bf16((double)s);
+  }
+}
+
+/* ------------------------------------------------------------------ delayed scaling */
+/* Sec. 4.2: per-tensor delayed scaling with an amax history of length H (16 in the paper).
+ * One update per training step and tensor: the history moves one place (the oldest value
+ * drops out), the step's amax enters at index 0, and the scale for the NEXT step is
+ * FP8MAX / max(history) -- as oracle_scale_from_amax computes it.  If that maximum is zero
+ * or not finite the previous scale is kept. */
+void oracle_delayed_scaling_update(float* history, int H, float amax_new, int fmt, float* scale, float* scale_inv) {
+  for (int j = H - 1; j > 0; --j) history[j] = history[j - 1];
+  history[0] = amax_new;
+  float m = 0.0f;
+  for (int j = 0; j < H; ++j)
+    if (history[j] > m) m = history[j]; /* false for NaN */
+  if (m > 0.0f && isfinite(m)) {
+    oracle_scale_from_amax(m, fmt, scale, scale_inv);
+  } else {
+    volatile float inv = 1.0f / *scale;
+    *scale_inv = inv;
+  }
 }

@@ -84,6 +84,8 @@ def lib():
             L.oracle_tweo_grad_block.argtypes = [C.c_void_p, C.c_int64, C.c_double, C.c_double, C.c_double,
                                                  C.c_double, C.c_void_p]
             L.oracle_absmax_qmax.restype = C.c_int
+            L.oracle_residual_add_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
+            L.oracle_delayed_scaling_update.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_int, C.c_void_p, C.c_void_p]
             L.oracle_absmax_qmax.argtypes = [C.c_int]
             L.oracle_absmax_quantize.restype = None
             L.oracle_absmax_quantize.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_double, C.c_void_p]
@@ -293,3 +295,23 @@ def absmax_dequantize(xq, bits: int, s: float) -> np.ndarray:
     x = np.empty(xq.shape, dtype=np.float64)
     lib().oracle_absmax_dequantize(xq.ctypes.data, xq.size, bits, float(s), x.ctypes.data)
     return x
+
+
+def residual_add_bf16(x_bits, f_bits) -> np.ndarray:
+    """Block output a = bf16(fl32(x + f)) of two bf16 tensors (Sec. 3.3)."""
+    x, f = _u16(x_bits), _u16(f_bits)
+    assert x.shape == f.shape
+    a = np.empty(x.shape, dtype=np.uint16)
+    lib().oracle_residual_add_bf16(x.ctypes.data, f.ctypes.data, x.size, a.ctypes.data)
+    return a
+
+
+def delayed_scaling_update(history, amax_new, fmt: int, scale):
+    """One delayed-scaling step for one tensor (Sec. 4.2).  `history` (float32 [H]) is updated in
+    place; returns (scale, scale_inv) for the next step."""
+    h = np.ascontiguousarray(history, dtype=np.float32)
+    assert h is history or np.shares_memory(h, history), "history must be a contiguous float32 array"
+    s = np.array([scale], dtype=np.float32)
+    si = np.zeros(1, dtype=np.float32)
+    lib().oracle_delayed_scaling_update(h.ctypes.data, h.size, float(amax_new), fmt, s.ctypes.data, si.ctypes.data)
+    return np.float32(s[0]), np.float32(si[0])
