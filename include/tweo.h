@@ -72,7 +72,8 @@ typedef enum {
   TWEO_OP_LINEAR_DGRAD = 2,
   TWEO_OP_LINEAR_WGRAD = 3,
   TWEO_OP_LOSS = 4,
-  TWEO_OP_W8A8 = 5
+  TWEO_OP_W8A8 = 5,
+  TWEO_OP_BLOCK_OUTPUT = 6
 } tweo_op_t;
 
 /* Upper bound on the number of block outputs one tweo_loss_fwd_bwd call takes. */
@@ -236,6 +237,40 @@ TWEO_API tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, in
                                 float eps, float p, float grad_coeff, float* loss,
                                 float* loss_per_block, void* const* grad, int32_t grad_dtype, void* ws,
                                 size_t ws_bytes, void* stream);
+
+/*
+ * tweo_block_output_fused -- the block output and everything that touches it once, in one pass
+ * (Sec. 3.3: the penalty acts on A = x + f(x), the residual stream plus the block's branch;
+ * Sec. 4.2: with delayed scaling the FP8 scale of A for the next block is known beforehand):
+ *   a_i   = bf16( fl32(x_i + f_i) )                  written to a [n] (may alias x or f)
+ *   *loss = (1/n) sum_i (|a_i| / (tau+eps))^p        this block's term of Eq. 3
+ *   g_i   = grad_coeff * p * sign(a_i) |a_i|^(p-1) / (n (tau+eps)^p)   -> grad [n] bf16, or NULL
+ *   *amax = max_i |a_i|                              (feeds tweo_delayed_scaling_update)
+ *   aq_i  = sat_rne_fp8( fl32(a_i * *q_scale) )      -> aq [n] in format q_fmt, or NULL
+ * Every output equals, bit for bit, what tweo_loss_fwd_bwd (L = 1, bf16 gradient) and
+ * tweo_quantize_per_tensor (GIVEN) produce from the stored a.  x, f: bf16 [n], device.
+ * loss, amax: device float*.  q_scale: device const float*, required with aq.  grad must
+ * not alias x, f or a.  Needs a zero-initialised workspace of
+ * tweo_workspace_bytes(TWEO_OP_BLOCK_OUTPUT) bytes; the reduction order is fixed, so results
+ * are reproducible run to run.
+ */
+TWEO_API tweo_status_t tweo_block_output_fused(const uint16_t* x, const uint16_t* f, int64_t n, float tau,
+                                      float eps, float p, float grad_coeff, uint16_t* a, uint16_t* grad,
+                                      float* loss, float* amax, uint8_t* aq, int32_t q_fmt,
+                                      const float* q_scale, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * tweo_delayed_scaling_update -- one step of delayed per-tensor scaling for n_tensors tensors of
+ * one FP8 format (Sec. 4.2: amax history of length 16 in the paper's runs).  For every tensor t:
+ * the history amax_history[t][0..history_len) moves one place (the oldest value drops out),
+ * amax_new[t] enters at index 0, and scale[t] = fl32(FP8MAX / max(history)) (clamped to FLT_MAX)
+ * becomes the scale for the NEXT step; if that maximum is zero or not finite scale[t] is kept.
+ * scale_inv[t] = fl32(1 / scale[t]).  All pointers are device pointers; start from a zeroed
+ * history and scale 1.  Under data parallelism amax_new must already be the maximum over ranks.
+ */
+TWEO_API tweo_status_t tweo_delayed_scaling_update(float* amax_history, int32_t history_len,
+                                          const float* amax_new, float* scale, float* scale_inv,
+                                          int32_t n_tensors, int32_t fmt, void* stream);
 
 /*
  * tweo_loss_fwd_bwd_static -- tweo_loss_fwd_bwd without a workspace argument.

@@ -16,7 +16,7 @@ import torch
 E4M3, E5M2 = 0, 1
 SCALE_CURRENT, SCALE_GIVEN = 0, 1
 BF16, F32, FP8_E4M3 = 0, 1, 2
-OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_DGRAD, OP_LINEAR_WGRAD, OP_LOSS, OP_W8A8 = range(6)
+OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_DGRAD, OP_LINEAR_WGRAD, OP_LOSS, OP_W8A8, OP_BLOCK_OUTPUT = range(7)
 MAX_BLOCKS = 128
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -25,6 +25,7 @@ LIB_PATH = os.path.join(_HERE, "libtweo_b200.so")
 EXPORTS = [
     "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_bwd_dgrad",
     "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
+    "tweo_block_output_fused", "tweo_delayed_scaling_update",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
 ]
@@ -81,6 +82,8 @@ def lib() -> C.CDLL:
                                         vp, sz, vp]
         L.tweo_loss_fwd_bwd_static.argtypes = [C.POINTER(vp), i32, i64, f32, f32, f32, f32, vp, vp, C.POINTER(vp),
                                                i32, vp]
+        L.tweo_block_output_fused.argtypes = [vp, vp, i64, f32, f32, f32, f32, vp, vp, vp, vp, vp, i32, vp, vp, sz, vp]
+        L.tweo_delayed_scaling_update.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp]
         L.tweo_w8a8_static_gemm.argtypes = [vp, i32, i64, vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, sz, vp]
         L.tweo_workspace_bytes.argtypes = [i32, i64, i64, i64]
         L.tweo_workspace_bytes.restype = sz
@@ -392,3 +395,52 @@ def w8a8_static_gemm(x, sx, wq, sw_inv, y=None, ws=None) -> torch.Tensor:
                                        _dev(y, torch.bfloat16, "y"), _rows(y, "y"), M, N, K, ws.data_ptr(),
                                        ws.numel(), _stream()), "tweo_w8a8_static_gemm")
     return y
+
+
+def block_output_fused(x, f, tau=3.0, eps=1e-6, p=4.0, grad_coeff=1.0, want_grad=True, q_fmt=None, q_scale=None,
+                       a=None, grad=None, aq=None, ws=None):
+    """tweo_block_output_fused: a = x + f with the TWEO loss term, its gradient, amax(a) and (with
+    q_fmt / q_scale) the FP8 codes of a, in one pass.  Returns (a, loss [1], amax [1], grad or None, aq or None)."""
+    if x.shape != f.shape or not x.is_contiguous() or not f.is_contiguous():
+        raise ValueError("x and f must be contiguous and of equal shape")
+    dev = x.device
+    if a is None:
+        a = torch.empty_like(x)
+    if want_grad and grad is None:
+        grad = torch.empty_like(x)
+    if not want_grad:
+        grad = None
+    if q_fmt is not None:
+        if q_scale is None:
+            raise ValueError("the FP8 copy needs q_scale")
+        if aq is None:
+            aq = torch.empty(x.shape, dtype=torch.uint8, device=dev)
+    else:
+        aq = None
+    if ws is None:
+        ws = new_workspace(OP_BLOCK_OUTPUT)
+    out = torch.empty(2, dtype=torch.float32, device=dev)
+    _check(lib().tweo_block_output_fused(_dev(x, torch.bfloat16, "x"), _dev(f, torch.bfloat16, "f"), x.numel(), tau, eps,
+                                         p, grad_coeff, _dev(a, torch.bfloat16, "a"),
+                                         _dev(grad, torch.bfloat16, "grad") if grad is not None else None,
+                                         out[0:1].data_ptr(), out[1:2].data_ptr(),
+                                         _dev(aq, U8, "aq") if aq is not None else None,
+                                         q_fmt if q_fmt is not None else 0,
+                                         _dev(q_scale, torch.float32, "q_scale") if q_scale is not None else None,
+                                         ws.data_ptr(), ws.numel(), _stream()), "tweo_block_output_fused")
+    return a, out[0:1], out[1:2], grad, aq
+
+
+def delayed_scaling_update(amax_history, amax_new, scale, scale_inv, fmt):
+    """tweo_delayed_scaling_update: rolls the [T, H] amax history, inserts amax_new [T] and refreshes
+    scale / scale_inv [T] for the next step (all float32 CUDA tensors, updated in place)."""
+    T, H = amax_history.shape
+    if not amax_history.is_contiguous():
+        raise ValueError("amax_history must be contiguous [T, H]")
+    for t, name in ((amax_new, "amax_new"), (scale, "scale"), (scale_inv, "scale_inv")):
+        if t.numel() != T or not t.is_contiguous():
+            raise ValueError(f"{name} must hold one value per tensor")
+    _check(lib().tweo_delayed_scaling_update(_dev(amax_history, torch.float32, "amax_history"), H,
+                                             _dev(amax_new, torch.float32), _dev(scale, torch.float32),
+                                             _dev(scale_inv, torch.float32), T, fmt, _stream()),
+           "tweo_delayed_scaling_update")

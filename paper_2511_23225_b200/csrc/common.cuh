@@ -81,6 +81,28 @@ __device__ __forceinline__ float scale_from_amax(float amax, int fmt) {
   return s;
 }
 
+// Running maximum of |x| over packed pairs of bf16, kept as two 16-bit lanes of sign-stripped bit
+// patterns (which order like the magnitudes); NaN patterns (> 0x7F80) count as 0.  Four integer
+// SIMD instructions per pair of elements.
+__device__ __forceinline__ uint32_t absmax_bits(uint32_t m2, uint32_t w) {
+  uint32_t a = w & 0x7FFF7FFFu;
+  a &= __vcmpleu2(a, 0x7F807F80u);
+  return __vmaxu2(m2, a);
+}
+// the larger of the two lanes: the bit pattern of max |x| as a bf16 value
+__device__ __forceinline__ uint32_t absmax_fold(uint32_t m2) { return max(m2 & 0xFFFFu, m2 >> 16); }
+// true if either bf16 of the pair is a NaN
+__device__ __forceinline__ bool pair_has_nan(uint32_t w) { return __vcmpgtu2(w & 0x7FFF7FFFu, 0x7F807F80u) != 0u; }
+
+// Two binary32 values -> two FP8 codes, no NaN handling (callers route NaN inputs elsewhere).
+template <int FMT>
+__device__ __forceinline__ uint32_t cvt_fp8x2_finite(float lo, float hi) {
+  uint16_t r;
+  if (FMT == TWEO_E4M3) asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  else asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
