@@ -343,6 +343,30 @@ def whole_job_value(flops_per_rank_step: float, ms_per_step: float, world: int) 
     return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
 
 
+def block_output_bench(torch, tw, peaks, reps=10):
+    """The fused block-output pass (x + f -> a, TWEO loss and gradient, amax, E4M3 copy with a given
+    scale) at the block-output sizes of configs 2 and 4: 4 B read + 5 B written per element."""
+    side = torch.cuda.Stream()
+    rows = []
+    for name, n in (("cfg2 [8192x768]", 8192 * 768), ("cfg4 [16384x2048]", 16384 * 2048)):
+        x = torch.randn(n, device="cuda").to(torch.bfloat16)
+        f = (0.3 * torch.randn(n, device="cuda")).to(torch.bfloat16)
+        a, g = torch.empty_like(x), torch.empty_like(x)
+        aq = torch.empty(n, dtype=torch.uint8, device="cuda")
+        qs = torch.full((1,), 448.0 / 8.0, dtype=torch.float32, device="cuda")
+        ws = tw.new_workspace(tw.OP_BLOCK_OUTPUT)
+        fn = lambda: [tw.block_output_fused(x, f, 3.0, 1e-6, 4.0, 0.01, True, tw.E4M3, qs, a=a, grad=g, aq=aq, ws=ws)
+                      for _ in range(reps)]
+        fn()
+        torch.cuda.synchronize()
+        us = 1e3 * _time_replays(torch, _graph_of(torch, side, fn), 5) / reps
+        rows.append({"tensor": name, "elements": n, "us": us, "gbs": 9.0 * n / us / 1e3,
+                     "frac_of_hbm_peak": 9.0 * n / us / 1e3 / peaks["hbm"]})
+        del x, f, a, g, aq
+    torch.cuda.empty_cache()
+    return rows
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -427,9 +451,10 @@ def run_cuda(args):
             del obs, o
             torch.cuda.empty_cache()
 
-    w8a8 = None
+    w8a8, block_rows = None, None
     if world == 1 and not args.no_w8a8:
         w8a8 = w8a8_sweep(torch, tw, peaks)
+        block_rows = block_output_bench(torch, tw, peaks)
         if tw.read_device_status() != 0:
             raise SystemExit("device status reports an expired wait")
 
@@ -454,6 +479,8 @@ def run_cuda(args):
             line["other_workloads"] = others
         if w8a8:
             line["cfg5_w8a8_static_gemm"] = w8a8
+        if block_rows:
+            line["block_output_fused"] = block_rows
         if world == 1 and not args.no_cpu_baseline:
             f, t = oracle_sample_step(cfg_idx, args.cpu_rows)
             line["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",

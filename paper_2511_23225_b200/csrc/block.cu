@@ -6,7 +6,7 @@
 // residual addition itself: read x and f, form a = bf16(fl32(x + f)), and in the same pass
 // emit a, the penalty's partial sums, its gradient, amax(a) and the FP8 codes of a.  That is
 // 4 B read + up to 5 B written per element instead of the 13 B of add, penalty and cast as
-// three passes.  HBM-bound streaming kernel: 4 x 16-byte loads per thread per 16 elements,
+// three passes.  HBM-bound streaming kernel: 8 x 16-byte loads in flight per thread (two groups of 16 elements),
 // fp32 per group / fp64 per thread accumulation, per-CTA partial sum and partial maximum to
 // the workspace, the last CTA (ticket) reduces them in a fixed order.
 //
@@ -86,34 +86,49 @@ __global__ void __launch_bounds__(kThreads) block_output_kernel(const BlockArgs 
   const int64_t stride = (int64_t)gridDim.x * kThreads;
   double acc = 0.0;
   uint32_t m2 = 0;
-  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n16; i += stride) {
-    const uint4 x0 = __ldcs(xv + 2 * i), x1 = __ldcs(xv + 2 * i + 1);
-    const uint4 f0 = __ldcs(fv + 2 * i), f1 = __ldcs(fv + 2 * i + 1);
-    const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-    const uint32_t fw[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
-    uint32_t aw[8], gw[8], c[8];
-    float t = 0.0f;
-    bool any_nan = false;
+  // two groups of 16 elements per thread and iteration: eight 16-byte loads in flight
+  for (int64_t base = (int64_t)blockIdx.x * kThreads + threadIdx.x; base < n16; base += 2 * stride) {
+    uint4 xr[2][2], fr[2][2];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      aw[j] = add_pair<FAST, GRAD>(xw[j], fw[j], args.k_grad, args.p, t, gw[j]);
-      m2 = absmax_bits(m2, aw[j]);
-      if (QFMT >= 0) any_nan |= pair_has_nan(aw[j]);
+    for (int u = 0; u < 2; ++u) {
+      const int64_t i = base + u * stride;
+      if (i < n16) {
+        xr[u][0] = __ldcs(xv + 2 * i);
+        xr[u][1] = __ldcs(xv + 2 * i + 1);
+        fr[u][0] = __ldcs(fv + 2 * i);
+        fr[u][1] = __ldcs(fv + 2 * i + 1);
+      }
     }
-    acc += (double)t;
-    __stcs(av + 2 * i, make_uint4(aw[0], aw[1], aw[2], aw[3]));
-    __stcs(av + 2 * i + 1, make_uint4(aw[4], aw[5], aw[6], aw[7]));
-    if (GRAD) {
-      __stcs(gv + 2 * i, make_uint4(gw[0], gw[1], gw[2], gw[3]));
-      __stcs(gv + 2 * i + 1, make_uint4(gw[4], gw[5], gw[6], gw[7]));
-    }
-    if (QFMT >= 0) {
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int64_t i = base + u * stride;
+      if (i >= n16) continue;
+      const uint32_t xw[8] = {xr[u][0].x, xr[u][0].y, xr[u][0].z, xr[u][0].w, xr[u][1].x, xr[u][1].y, xr[u][1].z, xr[u][1].w};
+      const uint32_t fw[8] = {fr[u][0].x, fr[u][0].y, fr[u][0].z, fr[u][0].w, fr[u][1].x, fr[u][1].y, fr[u][1].z, fr[u][1].w};
+      uint32_t aw[8], gw[8], c[8];
+      float t = 0.0f;
+      bool any_nan = false;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        const float lo = __fmul_rn(bf16lo_to_f32(aw[j]), qs), hi = __fmul_rn(bf16hi_to_f32(aw[j]), qs);
-        c[j] = any_nan ? cvt_fp8x2<QFMT < 0 ? 0 : QFMT>(lo, hi) : cvt_fp8x2_finite<QFMT < 0 ? 0 : QFMT>(lo, hi);
+        aw[j] = add_pair<FAST, GRAD>(xw[j], fw[j], args.k_grad, args.p, t, gw[j]);
+        m2 = absmax_bits(m2, aw[j]);
+        if (QFMT >= 0) any_nan |= pair_has_nan(aw[j]);
       }
-      __stcs(qv + i, make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16)));
+      acc += (double)t;
+      __stcs(av + 2 * i, make_uint4(aw[0], aw[1], aw[2], aw[3]));
+      __stcs(av + 2 * i + 1, make_uint4(aw[4], aw[5], aw[6], aw[7]));
+      if (GRAD) {
+        __stcs(gv + 2 * i, make_uint4(gw[0], gw[1], gw[2], gw[3]));
+        __stcs(gv + 2 * i + 1, make_uint4(gw[4], gw[5], gw[6], gw[7]));
+      }
+      if (QFMT >= 0) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float lo = __fmul_rn(bf16lo_to_f32(aw[j]), qs), hi = __fmul_rn(bf16hi_to_f32(aw[j]), qs);
+          c[j] = any_nan ? cvt_fp8x2<QFMT < 0 ? 0 : QFMT>(lo, hi) : cvt_fp8x2_finite<QFMT < 0 ? 0 : QFMT>(lo, hi);
+        }
+        __stcs(qv + i, make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16)));
+      }
     }
   }
   // ragged tail (n % 16 elements), first threads of CTA 0
@@ -201,7 +216,7 @@ void launch_q(int qfmt, int grid, cudaStream_t st, const BlockArgs& a) {
 }
 
 int block_grid(int64_t n) {
-  int64_t want = ((n >> 4) + kThreads - 1) / kThreads;
+  int64_t want = ((n >> 4) + 2 * kThreads - 1) / (2 * kThreads);
   const int64_t cap = (int64_t)sm_count() * 8;
   if (want > cap) want = cap;
   return (int)(want < 1 ? 1 : want);
