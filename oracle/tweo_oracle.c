@@ -374,6 +374,46 @@ double oracle_absmax_scale(const double* x, int64_t n, double eps) {
   return m + eps;
 }
 
+/* The same quantiser on bf16 tensors in the arithmetic an 8-bit kernel uses, so that the
+ * integer codes can be compared bit for bit: everything in binary32, each operation
+ * rounded once, in the order Eq. 4 writes them --
+ *   s   = fl32(max|X| + eps)                 (per tensor, or per row: one s per channel / token)
+ *   X_q = clamp(rne_int(fl32(fl32(X / s) * Q_b)), -Q_b, Q_b)
+ * NaN elements are skipped by the maximum and quantise to 0. */
+float oracle_absmax_scale_bf16(const uint16_t* x, int64_t n, float eps) {
+  volatile float s = oracle_amax_bf16(x, n) + eps;
+  return s;
+}
+
+void oracle_absmax_quantize_bf16(const uint16_t* x, int64_t n, int bits, float s, int8_t* xq) {
+  const float Q = (float)oracle_absmax_qmax(bits);
+  for (int64_t i = 0; i < n; ++i) {
+    volatile float d = bf16_bits_to_f32(x[i]) / s;
+    volatile float t = d * Q;
+    float r = nearbyintf(t);
+    if (r > Q) r = Q;
+    if (r < -Q) r = -Q;
+    xq[i] = (t != t) ? 0 : (int8_t)r;
+  }
+}
+
+/* 8-bit linear on the integer codes (Sec. 4.3): Y_mn = (sum_k Xq_mk * Wq_nk) * (sx_m / Q_b) * (sw_n / Q_b),
+ * i.e. the product of the dequantised operands of Eq. 4, with one scale per tensor or per
+ * row (token for X, output channel for W).  The integer sum is exact; the scales are applied
+ * in FP64.  Evaluated at the listed (row, col) points. */
+void oracle_int8_gemm_at(const int8_t* xq, int64_t ldx, const int8_t* wq, int64_t ldw, const float* sx,
+                         int sx_per_row, const float* sw, int sw_per_row, int bits, int64_t K,
+                         const int64_t* rows, const int64_t* cols, int64_t npts, double* y) {
+  const double Q = (double)oracle_absmax_qmax(bits);
+  for (int64_t t = 0; t < npts; ++t) {
+    const int64_t m = rows[t], n = cols[t];
+    int64_t acc = 0;
+    for (int64_t k = 0; k < K; ++k) acc += (int64_t)xq[m * ldx + k] * (int64_t)wq[n * ldw + k];
+    const double a = (double)sx[sx_per_row ? m : 0] / Q, b = (double)sw[sw_per_row ? n : 0] / Q;
+    y[t] = (double)acc * a * b;
+  }
+}
+
 /* ------------------------------------------------------------------ block output */
 /* The regulariser acts on the block output A^(l) = x + f(x) (Sec. 3.3: the residual
  * stream plus the block's branch).  With bf16 activations the sum is formed in binary32

@@ -84,6 +84,11 @@ def lib():
             L.oracle_tweo_grad_block.argtypes = [C.c_void_p, C.c_int64, C.c_double, C.c_double, C.c_double,
                                                  C.c_double, C.c_void_p]
             L.oracle_absmax_qmax.restype = C.c_int
+            L.oracle_absmax_scale_bf16.argtypes = [C.c_void_p, C.c_int64, C.c_float]
+            L.oracle_absmax_scale_bf16.restype = C.c_float
+            L.oracle_absmax_quantize_bf16.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_float, C.c_void_p]
+            L.oracle_int8_gemm_at.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int, C.c_void_p,
+                                              C.c_int, C.c_int, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
             L.oracle_residual_add_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
             L.oracle_delayed_scaling_update.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_int, C.c_void_p, C.c_void_p]
             L.oracle_absmax_qmax.argtypes = [C.c_int]
@@ -315,3 +320,40 @@ def delayed_scaling_update(history, amax_new, fmt: int, scale):
     si = np.zeros(1, dtype=np.float32)
     lib().oracle_delayed_scaling_update(h.ctypes.data, h.size, float(amax_new), fmt, s.ctypes.data, si.ctypes.data)
     return np.float32(s[0]), np.float32(si[0])
+
+
+def absmax_quantize_bf16(x_bits, bits: int, eps, per_row: bool = False, s=None):
+    """Eq. 4 on a bf16 tensor in binary32 arithmetic: returns (codes int8, s float32 [1] or [rows]).
+    `s` given: static scale(s); else s = max|x| + eps per tensor or per row of the 2-D tensor."""
+    x = _u16(x_bits)
+    q = np.empty(x.shape, dtype=np.int8)
+    L = lib()
+    if per_row:
+        assert x.ndim == 2
+        sv = np.empty(x.shape[0], dtype=np.float32) if s is None else np.ascontiguousarray(s, dtype=np.float32)
+        for r in range(x.shape[0]):
+            row = np.ascontiguousarray(x[r])
+            if s is None:
+                sv[r] = L.oracle_absmax_scale_bf16(row.ctypes.data, row.size, float(np.float32(eps)))
+            qr = np.empty(row.shape, dtype=np.int8)
+            L.oracle_absmax_quantize_bf16(row.ctypes.data, row.size, bits, float(sv[r]), qr.ctypes.data)
+            q[r] = qr
+        return q, sv
+    sv = np.float32(L.oracle_absmax_scale_bf16(x.ctypes.data, x.size, float(np.float32(eps)))) if s is None else np.float32(s)
+    L.oracle_absmax_quantize_bf16(x.ctypes.data, x.size, bits, float(sv), q.ctypes.data)
+    return q, np.array([sv], dtype=np.float32)
+
+
+def int8_gemm_at(xq, wq, sx, sw, bits: int, rows, cols) -> np.ndarray:
+    """Y[m,n] = (sum_k xq[m,k] wq[n,k]) (sx/Q)(sw/Q) at the given points; sx, sw hold 1 value or one per row."""
+    xq = np.ascontiguousarray(xq, dtype=np.int8)
+    wq = np.ascontiguousarray(wq, dtype=np.int8)
+    sx = np.ascontiguousarray(sx, dtype=np.float32).reshape(-1)
+    sw = np.ascontiguousarray(sw, dtype=np.float32).reshape(-1)
+    assert sx.size in (1, xq.shape[0]) and sw.size in (1, wq.shape[0]) and xq.shape[1] == wq.shape[1]
+    rows, cols = _pts(rows, cols)
+    out = np.empty(rows.size, dtype=np.float64)
+    lib().oracle_int8_gemm_at(xq.ctypes.data, xq.shape[1], wq.ctypes.data, wq.shape[1], sx.ctypes.data,
+                              1 if sx.size > 1 else 0, sw.ctypes.data, 1 if sw.size > 1 else 0, bits, xq.shape[1],
+                              rows.ctypes.data, cols.ctypes.data, rows.size, out.ctypes.data)
+    return out
