@@ -73,8 +73,10 @@ typedef enum {
   TWEO_OP_LINEAR_WGRAD = 3,
   TWEO_OP_LOSS = 4,
   TWEO_OP_W8A8 = 5,
-  TWEO_OP_BLOCK_OUTPUT = 6
+  TWEO_OP_BLOCK_OUTPUT = 6,
+  TWEO_OP_ABSMAX = 7
 } tweo_op_t;
+typedef enum { TWEO_GRAN_TENSOR = 0, TWEO_GRAN_ROW = 1 } tweo_granularity_t;
 
 /* Upper bound on the number of block outputs one tweo_loss_fwd_bwd call takes. */
 #define TWEO_MAX_BLOCKS 128
@@ -318,6 +320,37 @@ TWEO_API tweo_status_t tweo_w8a8_static_gemm(const void* x, int32_t x_dtype, int
                                     const uint8_t* wq, int64_t ldw, const float* sw_inv, uint16_t* y,
                                     int64_t ldy, int64_t M, int64_t N, int64_t K, void* ws,
                                     size_t ws_bytes, void* stream);
+
+/*
+ * tweo_absmax_quantize -- symmetric AbsMax b-bit quantisation (Sec. 4.3, Eq. 4):
+ *   s = max|X| + eps,  X_q = round(X / s * Q_b),  Q_b = 2^(b-1) - 1   (Q_8 = 127, Q_6 = 31),
+ * with one s for the whole tensor (TWEO_GRAN_TENSOR: the paper's "T") or one per row
+ * (TWEO_GRAN_ROW: per output channel "C" for a weight [N,K], per token "K" for an activation
+ * [M,K]).  x [rows, cols] bf16, row pitch ldx elements; q [rows, cols] int8 codes in
+ * [-Q_b, Q_b], row pitch ldq; s: device float [1] or [rows].
+ *   mode CURRENT: s is computed and written; mode GIVEN: s is read (static quantisation) and
+ *   values beyond it clamp to +-Q_b.  Arithmetic: binary32, each operation rounded once, in
+ *   the order of Eq. 4 -- s = fl32(amax + eps), q = clamp(rne(fl32(fl32(x / s) * Q_b))); ties
+ *   to even; NaN -> 0 and skipped by the maximum.  2 <= bits <= 8.
+ *   TWEO_GRAN_TENSOR needs a dense tensor (ldx == cols == ldq) and, in CURRENT mode, a
+ *   workspace of tweo_workspace_bytes(TWEO_OP_ABSMAX) bytes (any contents).
+ */
+TWEO_API tweo_status_t tweo_absmax_quantize(const uint16_t* x, int64_t rows, int64_t cols, int64_t ldx,
+                                   int32_t bits, int32_t granularity, int32_t mode, float eps, float* s,
+                                   int8_t* q, int64_t ldq, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * tweo_int8_linear -- the 8-bit (or b-bit) integer linear of Sec. 4.3 on Eq. 4's codes:
+ *   Y[M,N] = (sum_k Xq[m,k] Wq[n,k]) * (sx[m or 0] / Q_b) * (sw[n or 0] / Q_b)  -> bf16,
+ * the product of the dequantised operands.  Integer tensor cores, int32 accumulation (exact).
+ * xq [M,K], wq [N,K] int8 codes (row pitches multiples of 16); sx: device float [1] (per tensor,
+ * static or not) or [M] (per token) with sx_per_row != 0; sw: [1] or [N] (per channel) with
+ * sw_per_row != 0.  Shapes: N % 16 == 0, K % 16 == 0, any M >= 1.
+ */
+TWEO_API tweo_status_t tweo_int8_linear(const int8_t* xq, int64_t ldx, const float* sx, int32_t sx_per_row,
+                               const int8_t* wq, int64_t ldw, const float* sw, int32_t sw_per_row,
+                               int32_t bits, uint16_t* y, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                               void* stream);
 
 /* ---------------------------------------------------------------- helpers */
 

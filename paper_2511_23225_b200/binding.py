@@ -16,7 +16,8 @@ import torch
 E4M3, E5M2 = 0, 1
 SCALE_CURRENT, SCALE_GIVEN = 0, 1
 BF16, F32, FP8_E4M3 = 0, 1, 2
-OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_DGRAD, OP_LINEAR_WGRAD, OP_LOSS, OP_W8A8, OP_BLOCK_OUTPUT = range(7)
+OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_DGRAD, OP_LINEAR_WGRAD, OP_LOSS, OP_W8A8, OP_BLOCK_OUTPUT, OP_ABSMAX = range(8)
+GRAN_TENSOR, GRAN_ROW = 0, 1
 MAX_BLOCKS = 128
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -25,7 +26,7 @@ LIB_PATH = os.path.join(_HERE, "libtweo_b200.so")
 EXPORTS = [
     "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_bwd_dgrad",
     "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
-    "tweo_block_output_fused", "tweo_delayed_scaling_update",
+    "tweo_block_output_fused", "tweo_delayed_scaling_update", "tweo_absmax_quantize", "tweo_int8_linear",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
 ]
@@ -84,6 +85,8 @@ def lib() -> C.CDLL:
                                                i32, vp]
         L.tweo_block_output_fused.argtypes = [vp, vp, i64, f32, f32, f32, f32, vp, vp, vp, vp, vp, i32, vp, vp, sz, vp]
         L.tweo_delayed_scaling_update.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp]
+        L.tweo_absmax_quantize.argtypes = [vp, i64, i64, i64, i32, i32, i32, f32, vp, vp, i64, vp, sz, vp]
+        L.tweo_int8_linear.argtypes = [vp, i64, vp, i32, vp, i64, vp, i32, i32, vp, i64, i64, i64, i64, vp]
         L.tweo_w8a8_static_gemm.argtypes = [vp, i32, i64, vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, sz, vp]
         L.tweo_workspace_bytes.argtypes = [i32, i64, i64, i64]
         L.tweo_workspace_bytes.restype = sz
@@ -444,3 +447,36 @@ def delayed_scaling_update(amax_history, amax_new, scale, scale_inv, fmt):
                                              _dev(amax_new, torch.float32), _dev(scale, torch.float32),
                                              _dev(scale_inv, torch.float32), T, fmt, _stream()),
            "tweo_delayed_scaling_update")
+
+
+def absmax_quantize(x, bits=8, granularity=GRAN_TENSOR, eps=1e-6, s=None, ws=None):
+    """tweo_absmax_quantize (Eq. 4): int8 codes of a 2-D bf16 tensor and its scale(s) s ([1] or [rows]).
+    With `s` given the quantisation is static."""
+    if x.dim() != 2 or x.stride(1) != 1:
+        raise ValueError("x must be 2-D with contiguous rows")
+    rows, cols = x.shape
+    mode = SCALE_GIVEN if s is not None else SCALE_CURRENT
+    if s is None:
+        s = torch.empty(rows if granularity == GRAN_ROW else 1, dtype=torch.float32, device=x.device)
+    q = torch.empty((rows, cols), dtype=torch.int8, device=x.device)
+    if ws is None and granularity == GRAN_TENSOR and mode == SCALE_CURRENT:
+        ws = new_workspace(OP_ABSMAX)
+    _check(lib().tweo_absmax_quantize(_dev(x, torch.bfloat16, "x"), rows, cols, x.stride(0), bits, granularity, mode,
+                                      eps, _dev(s, torch.float32, "s"), q.data_ptr(), q.stride(0), *_ws(ws), _stream()),
+           "tweo_absmax_quantize")
+    return q, s
+
+
+def int8_linear(xq, sx, wq, sw, bits=8, y=None):
+    """tweo_int8_linear: Y = (Xq . Wq^T) (sx/Q)(sw/Q) -> bf16; sx holds 1 value or one per row of xq, sw 1 or one per row of wq."""
+    M, K = xq.shape
+    N, K2 = wq.shape
+    if K != K2:
+        raise ValueError("inner dimensions differ")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=xq.device)
+    _check(lib().tweo_int8_linear(_dev(xq, torch.int8, "xq"), _rows(xq, "xq"), _dev(sx, torch.float32, "sx"),
+                                  1 if sx.numel() > 1 else 0, _dev(wq, torch.int8, "wq"), _rows(wq, "wq"),
+                                  _dev(sw, torch.float32, "sw"), 1 if sw.numel() > 1 else 0, bits,
+                                  _dev(y, torch.bfloat16, "y"), _rows(y, "y"), M, N, K, _stream()), "tweo_int8_linear")
+    return y

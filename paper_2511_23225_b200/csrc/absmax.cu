@@ -1,0 +1,178 @@
+// Symmetric AbsMax b-bit quantisation (Eq. 4): s = max|X| + eps, X_q = round(X / s * Q_b),
+// Q_b = 2^(b-1) - 1, with one s per tensor or per row (per output channel of a weight, per
+// token of an activation), computed now or given (static).  Codes are int8 (b = 6 uses the
+// same container).  Everything is binary32, each operation rounded once, in Eq. 4's order:
+//   s = fl32(amax + eps);  t = fl32(fl32(x / s) * Q_b);  q = clamp(rne_int(t), -Q_b, Q_b);  NaN -> 0.
+// HBM-bound streaming kernels: 16-byte loads of 8 bf16, 16-byte stores of 16 codes.
+//   per row   : one CTA per row (grid-stride over rows): maximum of the row, then the cast;
+//               the second read of the row comes from L1/L2.
+//   per tensor: kernel 1 writes per-CTA maxima to workspace slots, kernel 2 reduces them in
+//               every CTA and casts (no atomics, no reset kernel); static s skips kernel 1.
+#include <cuda_runtime.h>
+
+#include "common.cuh"
+
+namespace {
+
+using namespace tweo_detail;
+
+constexpr int kThreads = 256;
+constexpr int kMaxSlots = 2048;
+
+__device__ __forceinline__ uint32_t cta_max_bits(uint32_t m, uint32_t* part) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = m;
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) m = max(m, part[w]);
+  return m;
+}
+
+__device__ __forceinline__ int quant1(float x, float s, float Q) {
+  const float t = __fmul_rn(__fdiv_rn(x, s), Q);
+  int r = __float2int_rn(t);  // ties to even; NaN -> 0; saturates
+  const int q = (int)Q;
+  return max(-q, min(q, r));
+}
+
+// 16 bf16 (two 16-byte vectors) -> 16 int8 codes
+__device__ __forceinline__ uint4 quant16(const uint4 a, const uint4 b, float s, float Q) {
+  const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+  uint32_t c[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int q0 = quant1(bf16lo_to_f32(w[2 * j]), s, Q), q1 = quant1(bf16hi_to_f32(w[2 * j]), s, Q);
+    const int q2 = quant1(bf16lo_to_f32(w[2 * j + 1]), s, Q), q3 = quant1(bf16hi_to_f32(w[2 * j + 1]), s, Q);
+    c[j] = (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) |
+           ((uint32_t)(q3 & 0xFF) << 24);
+  }
+  return make_uint4(c[0], c[1], c[2], c[3]);
+}
+
+// maximum of |x| over [x, x+n) by this CTA's threads (packed lanes, see absmax_bits)
+__device__ __forceinline__ uint32_t span_absmax(const uint16_t* x, int64_t n, int64_t first_vec, int64_t vec_stride) {
+  uint32_t m2 = 0;
+  const bool vec_ok = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
+  const int64_t nvec = vec_ok ? (n >> 3) : 0;
+  const uint4* xv = reinterpret_cast<const uint4*>(x);
+  for (int64_t i = first_vec; i < nvec; i += vec_stride) {
+    const uint4 v = __ldg(xv + i);
+    m2 = absmax_bits(m2, v.x);
+    m2 = absmax_bits(m2, v.y);
+    m2 = absmax_bits(m2, v.z);
+    m2 = absmax_bits(m2, v.w);
+  }
+  for (int64_t i = (nvec << 3) + first_vec; i < n; i += vec_stride) m2 = absmax_bits(m2, (uint32_t)x[i]);
+  return m2;
+}
+
+__device__ __forceinline__ void span_quantize(const uint16_t* x, int8_t* q, int64_t n, float s, float Q,
+                                              int64_t first, int64_t stride) {
+  const bool vec_ok = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(q)) & 15u) == 0;
+  const int64_t n16 = vec_ok ? (n >> 4) : 0;
+  const uint4* xv = reinterpret_cast<const uint4*>(x);
+  uint4* qv = reinterpret_cast<uint4*>(q);
+  for (int64_t i = first; i < n16; i += stride) __stcs(qv + i, quant16(__ldcs(xv + 2 * i), __ldcs(xv + 2 * i + 1), s, Q));
+  for (int64_t i = (n16 << 4) + first; i < n; i += stride)
+    q[i] = (int8_t)quant1(bf16lo_to_f32((uint32_t)x[i]), s, Q);
+}
+
+// one scale per row
+template <bool GIVEN>
+__global__ void __launch_bounds__(kThreads)
+absmax_rows_kernel(const uint16_t* x, int64_t rows, int64_t cols, int64_t ldx, float eps, float Q, float* s_out,
+                   int8_t* q, int64_t ldq) {
+  __shared__ uint32_t part[kThreads / 32];
+  for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+    const uint16_t* xr = x + r * ldx;
+    float s;
+    if (GIVEN) {
+      s = __ldg(s_out + r);
+    } else {
+      const uint32_t m = cta_max_bits(absmax_fold(span_absmax(xr, cols, threadIdx.x, kThreads)), part);
+      s = __fadd_rn(__uint_as_float(m << 16), eps);
+      if (threadIdx.x == 0) s_out[r] = s;
+    }
+    span_quantize(xr, q + r * ldq, cols, s, Q, threadIdx.x, kThreads);
+  }
+}
+
+// one scale for the whole (contiguous) tensor: per-CTA maxima ...
+__global__ void __launch_bounds__(kThreads) absmax_slots_kernel(const uint16_t* x, int64_t n, uint32_t* slots) {
+  __shared__ uint32_t part[kThreads / 32];
+  const uint32_t m = cta_max_bits(
+      absmax_fold(span_absmax(x, n, (int64_t)blockIdx.x * kThreads + threadIdx.x, (int64_t)gridDim.x * kThreads)), part);
+  if (threadIdx.x == 0) slots[blockIdx.x] = m;
+}
+
+// ... then every CTA reduces them itself and casts its share
+template <bool GIVEN>
+__global__ void __launch_bounds__(kThreads)
+absmax_tensor_kernel(const uint16_t* x, int64_t n, float eps, float Q, float* s_io, const uint32_t* slots, int n_slots,
+                     int8_t* q) {
+  __shared__ uint32_t part[kThreads / 32];
+  float s;
+  if (GIVEN) {
+    s = __ldg(s_io);
+  } else {
+    uint32_t m = 0;
+    for (int k = threadIdx.x; k < n_slots; k += kThreads) m = max(m, __ldcg(slots + k));
+    m = cta_max_bits(m, part);
+    s = __fadd_rn(__uint_as_float(m << 16), eps);
+    if (blockIdx.x == 0 && threadIdx.x == 0) *s_io = s;
+  }
+  span_quantize(x, q, n, s, Q, (int64_t)blockIdx.x * kThreads + threadIdx.x, (int64_t)gridDim.x * kThreads);
+}
+
+int grid_cap(int64_t want, int per_sm) {
+  const int64_t cap = (int64_t)sm_count() * per_sm;
+  if (want > cap) want = cap;
+  return (int)(want < 1 ? 1 : want);
+}
+
+}  // namespace
+
+namespace tweo_detail {
+size_t absmax_workspace_bytes() { return (size_t)kMaxSlots * sizeof(uint32_t); }
+}
+
+extern "C" tweo_status_t tweo_absmax_quantize(const uint16_t* x, int64_t rows, int64_t cols, int64_t ldx, int32_t bits,
+                                              int32_t granularity, int32_t mode, float eps, float* s, int8_t* q,
+                                              int64_t ldq, void* ws, size_t ws_bytes, void* stream) {
+  if (rows < 0 || cols < 0 || !s) return TWEO_ERR_INVALID_ARG;
+  if (bits < 2 || bits > 8) return TWEO_ERR_INVALID_ARG;
+  if (granularity != TWEO_GRAN_TENSOR && granularity != TWEO_GRAN_ROW) return TWEO_ERR_INVALID_ARG;
+  if (mode != TWEO_SCALE_CURRENT && mode != TWEO_SCALE_GIVEN) return TWEO_ERR_INVALID_ARG;
+  if (!(eps >= 0.0f)) return TWEO_ERR_INVALID_ARG;
+  if (rows * cols > 0 && (!x || !q || ldx < cols || ldq < cols)) return TWEO_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const float Q = (float)((1 << (bits - 1)) - 1);
+  const bool given = mode == TWEO_SCALE_GIVEN;
+  if (granularity == TWEO_GRAN_ROW) {
+    if (rows == 0) return TWEO_OK;
+    const int grid = grid_cap(rows, 8);
+    if (given) absmax_rows_kernel<true><<<grid, kThreads, 0, st>>>(x, rows, cols, ldx, eps, Q, s, q, ldq);
+    else absmax_rows_kernel<false><<<grid, kThreads, 0, st>>>(x, rows, cols, ldx, eps, Q, s, q, ldq);
+    count_launch();
+    return check_launch("absmax_rows_kernel");
+  }
+  if (rows > 1 && (ldx != cols || ldq != cols)) return TWEO_ERR_UNSUPPORTED_SHAPE;  // one scale: dense tensor
+  const int64_t n = rows * cols;
+  uint32_t* slots = reinterpret_cast<uint32_t*>(ws);
+  int n_slots = 0;
+  if (!given) {
+    if (!ws || ws_bytes < absmax_workspace_bytes()) return TWEO_ERR_WORKSPACE_TOO_SMALL;
+    if (!aligned16(ws)) return TWEO_ERR_ALIGNMENT;
+    n_slots = grid_cap(((n >> 3) + kThreads * 4 - 1) / (kThreads * 4), 8);
+    if (n_slots > kMaxSlots) n_slots = kMaxSlots;
+    absmax_slots_kernel<<<n_slots, kThreads, 0, st>>>(x, n, slots);
+    count_launch();
+  }
+  const int grid = grid_cap(((n >> 4) + kThreads * 2 - 1) / (kThreads * 2), 8);
+  if (given) absmax_tensor_kernel<true><<<grid, kThreads, 0, st>>>(x, n, eps, Q, s, slots, n_slots, q);
+  else absmax_tensor_kernel<false><<<grid, kThreads, 0, st>>>(x, n, eps, Q, s, slots, n_slots, q);
+  count_launch();
+  return check_launch("absmax_tensor_kernel");
+}

@@ -39,6 +39,7 @@ tweo_status_t check_launch(const char* what) {
 
 size_t quantize_workspace_bytes();
 size_t block_output_workspace_bytes();
+size_t absmax_workspace_bytes();
 // Blocks per tensor of the loss kernel; also fixes the workspace size.
 int loss_blocks_per_tensor(int64_t n, int L);
 
@@ -80,6 +81,8 @@ size_t tweo_workspace_bytes(int32_t op, int64_t M, int64_t N, int64_t K) {
     case TWEO_OP_LINEAR_WGRAD:
       // optional: lets the GEMM split tiles along the contraction (parked fp32 accumulators + flags)
       return stream_k_bytes;
+    case TWEO_OP_ABSMAX:
+      return tweo_detail::absmax_workspace_bytes();
     case TWEO_OP_BLOCK_OUTPUT:
       return tweo_detail::block_output_workspace_bytes();
     case TWEO_OP_W8A8: {

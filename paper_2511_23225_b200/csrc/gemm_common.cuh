@@ -30,6 +30,11 @@ struct GemmParams {
   int32_t q_fmt;
   const float* q_scale;
   uint32_t idesc;
+  // integer (Eq. 4) linear only: y = float(acc) * (row_scale[m or 0] * post_scale) * col_scale[n or 0]
+  const float* row_scale;
+  const float* col_scale;
+  int32_t row_scale_per_row, col_scale_per_col;
+  float post_scale;
   // stream-K: tiles [0, sk_tiles) are split along the contraction, the rest dealt whole
   int32_t sk_tiles;
   float* sk_partials;   // [grid][BM*BN] raw accumulators of shares that do not own their tile

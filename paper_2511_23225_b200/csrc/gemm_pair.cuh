@@ -143,7 +143,9 @@ __device__ __noinline__ float pair_partial_share(const GemmParams& p, const CUte
   return run_amax;
 }
 
-template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32>
+// I8: the operands are 8-bit integers (tcgen05 kind::i8, int32 accumulators) and the epilogue
+// applies the Eq. 4 dequantisation with one scale per tensor or per row / column.
+template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32, bool I8 = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ GemmParams p) {
@@ -246,7 +248,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint64_t adesc = make_smem_desc(sa + (A_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
             const uint64_t bdesc = make_smem_desc(sb + (B_MN ? k * UMMA_K * 128 : k * UMMA_K), BK * 128);
-            umma_f8_pair(d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != kb0 || k != 0));
+            if (I8) umma_i8_pair(d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != kb0 || k != 0));
+            else umma_f8_pair(d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != kb0 || k != 0));
           }
           umma_commit_pair(map_to_cta(empty_bar(stage), 0));  // frees the stage in both CTAs
           umma_commit_pair(map_to_cta(empty_bar(stage), 1));
@@ -262,7 +265,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
     const int quarter = warp & 3;
-    const float alpha = __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
+    const float alpha = I8 ? 1.0f : __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
     const float qs = p.out_q ? __ldg(p.q_scale) : 0.0f;
     constexpr int CH = OUT_F32 ? 32 : 64;
     const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
@@ -308,6 +311,16 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         if (!OUT_F32) tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[CH - 32]));
         tmem_ld_wait();
         if (row0 >= p.Md) continue;
+        if (I8) {
+          // int32 accumulators -> binary32, then the two Eq. 4 scales (row first, then column)
+          const float ar = __fmul_rn(__ldg(p.row_scale + (p.row_scale_per_row ? min(row, p.Md - 1) : 0)), p.post_scale);
+          const float ac0 = __ldg(p.col_scale);
+#pragma unroll
+          for (int j = 0; j < CH; ++j) {
+            const float ac = p.col_scale_per_col ? __ldg(p.col_scale + min(col0 + j, p.Nd - 1)) : ac0;
+            r[j] = __float_as_uint(__fmul_rn(__fmul_rn(__int2float_rn((int)r[j]), ar), ac));
+          }
+        }
         const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
         if (lane == 0) bulk_wait_read<1>();
         __syncwarp();
