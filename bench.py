@@ -367,6 +367,40 @@ def block_output_bench(torch, tw, peaks, reps=10):
     return rows
 
 
+def int8_bench(torch, tw, peaks, reps=10):
+    """The paper's literal 8-bit path (Eq. 4 AbsMax codes, integer tensor cores) at a config-5 shape:
+    quantiser rates (2 B read + 1 B written per element, twice that read when the scale is computed) and
+    the int8 linear W(C)A(K) / W(T)A(T) for M = 1024 and 8192."""
+    side = torch.cuda.Stream()
+    out = {"quantize": [], "linear": []}
+    K, N = 4096, 11008
+    w = (0.02 * torch.randn((N, K), device="cuda")).to(torch.bfloat16)
+    for M in (1024, 8192):
+        x = torch.randn((M, K), device="cuda").to(torch.bfloat16)
+        for gname, gran in (("T", tw.GRAN_TENSOR), ("row", tw.GRAN_ROW)):
+            ws = tw.new_workspace(tw.OP_ABSMAX)
+            fn = lambda: [tw.absmax_quantize(x, 8, gran, 1e-6, ws=ws) for _ in range(reps)]
+            fn()
+            torch.cuda.synchronize()
+            us = 1e3 * _time_replays(torch, _graph_of(torch, side, fn), 5) / reps
+            out["quantize"].append({"tensor": f"[{M}x{K}]", "granularity": gname, "us": us,
+                                    "gbs": 5.0 * M * K / us / 1e3, "frac_of_hbm_peak": 5.0 * M * K / us / 1e3 / peaks["hbm"]})
+            xq, sx = tw.absmax_quantize(x, 8, gran, 1e-6, ws=ws)
+            wq, sw = tw.absmax_quantize(w, 8, gran, 1e-6, ws=ws)
+            y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            fn = lambda: [tw.int8_linear(xq, sx, wq, sw, 8, y=y) for _ in range(reps)]
+            fn()
+            torch.cuda.synchronize()
+            us = 1e3 * _time_replays(torch, _graph_of(torch, side, fn), 5) / reps
+            tops = 2.0 * M * K * N / us / 1e6
+            out["linear"].append({"M": M, "K": K, "N": N, "scales": "W(T)A(T)" if gname == "T" else "W(C)A(K)", "us": us,
+                                  "tops": tops, "frac_of_2x_bf16_burst": tops / (2.0 * peaks["bf16"])})
+            del xq, wq, y
+        del x
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -451,10 +485,11 @@ def run_cuda(args):
             del obs, o
             torch.cuda.empty_cache()
 
-    w8a8, block_rows = None, None
+    w8a8, block_rows, int8_rows = None, None, None
     if world == 1 and not args.no_w8a8:
         w8a8 = w8a8_sweep(torch, tw, peaks)
         block_rows = block_output_bench(torch, tw, peaks)
+        int8_rows = int8_bench(torch, tw, peaks)
         if tw.read_device_status() != 0:
             raise SystemExit("device status reports an expired wait")
 
@@ -481,6 +516,8 @@ def run_cuda(args):
             line["cfg5_w8a8_static_gemm"] = w8a8
         if block_rows:
             line["block_output_fused"] = block_rows
+        if int8_rows:
+            line["int8_absmax_path"] = int8_rows
         if world == 1 and not args.no_cpu_baseline:
             f, t = oracle_sample_step(cfg_idx, args.cpu_rows)
             line["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",

@@ -329,9 +329,9 @@ TWEO_API tweo_status_t tweo_w8a8_static_gemm(const void* x, int32_t x_dtype, int
  * [M,K]).  x [rows, cols] bf16, row pitch ldx elements; q [rows, cols] int8 codes in
  * [-Q_b, Q_b], row pitch ldq; s: device float [1] or [rows].
  *   mode CURRENT: s is computed and written; mode GIVEN: s is read (static quantisation) and
- *   values beyond it clamp to +-Q_b.  Arithmetic: binary32, each operation rounded once, in
- *   the order of Eq. 4 -- s = fl32(amax + eps), q = clamp(rne(fl32(fl32(x / s) * Q_b))); ties
- *   to even; NaN -> 0 and skipped by the maximum.  2 <= bits <= 8.
+ *   values beyond it clamp to +-Q_b.  Arithmetic: binary32, each operation rounded once,
+ *   X / s * Q_b evaluated as X * (Q_b / s) -- s = fl32(amax + eps), c = fl32(Q_b / s),
+ *   q = clamp(rne(fl32(x * c))); ties to even; NaN -> 0 and skipped by the maximum.  2 <= bits <= 8.
  *   TWEO_GRAN_TENSOR needs a dense tensor (ldx == cols == ldq) and, in CURRENT mode, a
  *   workspace of tweo_workspace_bytes(TWEO_OP_ABSMAX) bytes (any contents).
  */

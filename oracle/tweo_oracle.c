@@ -378,7 +378,10 @@ double oracle_absmax_scale(const double* x, int64_t n, double eps) {
  * integer codes can be compared bit for bit: everything in binary32, each operation
  * rounded once, in the order Eq. 4 writes them --
  *   s   = fl32(max|X| + eps)                 (per tensor, or per row: one s per channel / token)
- *   X_q = clamp(rne_int(fl32(fl32(X / s) * Q_b)), -Q_b, Q_b)
+ *   c   = fl32(Q_b / s)                      (once per scale)
+ *   X_q = clamp(rne_int(fl32(X * c)), -Q_b, Q_b)
+ * i.e. Eq. 4's X / s * Q_b evaluated as X * (Q_b / s): one division per scale and one
+ * multiplication per element, the form an 8-bit kernel runs at memory speed.
  * NaN elements are skipped by the maximum and quantise to 0. */
 float oracle_absmax_scale_bf16(const uint16_t* x, int64_t n, float eps) {
   volatile float s = oracle_amax_bf16(x, n) + eps;
@@ -387,9 +390,9 @@ float oracle_absmax_scale_bf16(const uint16_t* x, int64_t n, float eps) {
 
 void oracle_absmax_quantize_bf16(const uint16_t* x, int64_t n, int bits, float s, int8_t* xq) {
   const float Q = (float)oracle_absmax_qmax(bits);
+  volatile float c = Q / s;
   for (int64_t i = 0; i < n; ++i) {
-    volatile float d = bf16_bits_to_f32(x[i]) / s;
-    volatile float t = d * Q;
+    volatile float t = bf16_bits_to_f32(x[i]) * c;
     float r = nearbyintf(t);
     if (r > Q) r = Q;
     if (r < -Q) r = -Q;

@@ -1,8 +1,9 @@
 // Symmetric AbsMax b-bit quantisation (Eq. 4): s = max|X| + eps, X_q = round(X / s * Q_b),
 // Q_b = 2^(b-1) - 1, with one s per tensor or per row (per output channel of a weight, per
 // token of an activation), computed now or given (static).  Codes are int8 (b = 6 uses the
-// same container).  Everything is binary32, each operation rounded once, in Eq. 4's order:
-//   s = fl32(amax + eps);  t = fl32(fl32(x / s) * Q_b);  q = clamp(rne_int(t), -Q_b, Q_b);  NaN -> 0.
+// same container).  Everything is binary32, each operation rounded once; Eq. 4's X / s * Q_b is
+// evaluated as X * (Q_b / s), one division per scale and one multiplication per element:
+//   s = fl32(amax + eps);  c = fl32(Q_b / s);  q = clamp(rne_int(fl32(x * c)), -Q_b, Q_b);  NaN -> 0.
 // HBM-bound streaming kernels: 16-byte loads of 8 bf16, 16-byte stores of 16 codes.
 //   per row   : one CTA per row (grid-stride over rows): maximum of the row, then the cast;
 //               the second read of the row comes from L1/L2.
@@ -30,25 +31,25 @@ __device__ __forceinline__ uint32_t cta_max_bits(uint32_t m, uint32_t* part) {
   return m;
 }
 
-__device__ __forceinline__ int quant1(float x, float s, float Q) {
-  const float t = __fmul_rn(__fdiv_rn(x, s), Q);
-  int r = __float2int_rn(t);  // ties to even; NaN -> 0; saturates
+// c = fl32(Q / s)
+__device__ __forceinline__ int quant1(float x, float c, float Q) {
+  const int r = __float2int_rn(__fmul_rn(x, c));  // ties to even; NaN -> 0; saturates
   const int q = (int)Q;
   return max(-q, min(q, r));
 }
 
 // 16 bf16 (two 16-byte vectors) -> 16 int8 codes
-__device__ __forceinline__ uint4 quant16(const uint4 a, const uint4 b, float s, float Q) {
+__device__ __forceinline__ uint4 quant16(const uint4 a, const uint4 b, float c, float Q) {
   const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-  uint32_t c[4];
+  uint32_t pk[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    const int q0 = quant1(bf16lo_to_f32(w[2 * j]), s, Q), q1 = quant1(bf16hi_to_f32(w[2 * j]), s, Q);
-    const int q2 = quant1(bf16lo_to_f32(w[2 * j + 1]), s, Q), q3 = quant1(bf16hi_to_f32(w[2 * j + 1]), s, Q);
-    c[j] = (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) |
+    const int q0 = quant1(bf16lo_to_f32(w[2 * j]), c, Q), q1 = quant1(bf16hi_to_f32(w[2 * j]), c, Q);
+    const int q2 = quant1(bf16lo_to_f32(w[2 * j + 1]), c, Q), q3 = quant1(bf16hi_to_f32(w[2 * j + 1]), c, Q);
+    pk[j] = (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) |
            ((uint32_t)(q3 & 0xFF) << 24);
   }
-  return make_uint4(c[0], c[1], c[2], c[3]);
+  return make_uint4(pk[0], pk[1], pk[2], pk[3]);
 }
 
 // maximum of |x| over [x, x+n) by this CTA's threads (packed lanes, see absmax_bits)
@@ -70,13 +71,24 @@ __device__ __forceinline__ uint32_t span_absmax(const uint16_t* x, int64_t n, in
 
 __device__ __forceinline__ void span_quantize(const uint16_t* x, int8_t* q, int64_t n, float s, float Q,
                                               int64_t first, int64_t stride) {
+  const float c = __fdiv_rn(Q, s);
   const bool vec_ok = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(q)) & 15u) == 0;
   const int64_t n16 = vec_ok ? (n >> 4) : 0;
   const uint4* xv = reinterpret_cast<const uint4*>(x);
   uint4* qv = reinterpret_cast<uint4*>(q);
-  for (int64_t i = first; i < n16; i += stride) __stcs(qv + i, quant16(__ldcs(xv + 2 * i), __ldcs(xv + 2 * i + 1), s, Q));
+  for (int64_t i = first; i < n16; i += 2 * stride) {  // two groups of 16 per iteration: four loads in flight
+    const int64_t i1 = i + stride;
+    const uint4 a0 = __ldcs(xv + 2 * i), b0 = __ldcs(xv + 2 * i + 1);
+    uint4 a1 = a0, b1 = b0;
+    if (i1 < n16) {
+      a1 = __ldcs(xv + 2 * i1);
+      b1 = __ldcs(xv + 2 * i1 + 1);
+    }
+    __stcs(qv + i, quant16(a0, b0, c, Q));
+    if (i1 < n16) __stcs(qv + i1, quant16(a1, b1, c, Q));
+  }
   for (int64_t i = (n16 << 4) + first; i < n; i += stride)
-    q[i] = (int8_t)quant1(bf16lo_to_f32((uint32_t)x[i]), s, Q);
+    q[i] = (int8_t)quant1(bf16lo_to_f32((uint32_t)x[i]), c, Q);
 }
 
 // one scale per row
