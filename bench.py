@@ -236,9 +236,10 @@ def family_breakdown(torch, tw, bs, side, reps):
     return out
 
 
-def measure_workload(torch, tw, cfg_idx, steps, warmup, world, barrier, want_e2e, e2e_steps, local):
+def measure_workload(torch, tw, cfg_idx, steps, warmup, world, barrier, want_e2e, e2e_steps, local, overlap=True):
     from paper_2511_23225_b200.workload import BlockStep
     bs = BlockStep(cfg_idx)
+    bs.overlap = overlap
     bs.make_host_inputs()
     bs.upload()
     torch.cuda.synchronize()
@@ -424,7 +425,8 @@ def run_cuda(args):
         torch.cuda.synchronize()
 
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    r = measure_workload(torch, tw, cfg_idx, args.steps, args.warmup, world, barrier, True, e2e_steps, local)
+    r = measure_workload(torch, tw, cfg_idx, args.steps, args.warmup, world, barrier, True, e2e_steps, local,
+                         overlap=not args.no_overlap)
     bs = r["bs"]
     ms_per_step = max_over_ranks(r["ms_per_step"], "cuda")
     e2e_ms = max_over_ranks(r["e2e_ms_per_step"], "cuda")
@@ -457,7 +459,9 @@ def run_cuda(args):
                     "linears": [f"{l.name}:{l.K}x{l.N}" for l in bs.cfg.linears], "tweo_blocks": bs.n_blocks,
                     "parallelism": f"replicas x{world} (token shards, no data-path collective)",
                     "l2": f"working set {bs.working_set_bytes() / 1e6:.0f} MB per step > 126 MB L2, no flush",
-                    "launch": "cuda graph replay of one captured step"}
+                    "launch": "cuda graph replay of one captured step; two streams inside it: the casts of linear "
+                              "i+1 and the TWEO pass overlap the GEMMs of linear i" if not args.no_overlap
+                    else "cuda graph replay of one captured step, one stream"}
     h2d = bs.h2d_bytes()
     loss_value = r["loss"]
     main_clocks = r["clocks"]
@@ -472,7 +476,8 @@ def run_cuda(args):
             name = name.strip()
             if not name or name == args.workload:
                 continue
-            o = measure_workload(torch, tw, int(name[3:]), args.also_steps, 3, 1, barrier, False, 0, local)
+            o = measure_workload(torch, tw, int(name[3:]), args.also_steps, 3, 1, barrier, False, 0, local,
+                                 overlap=not args.no_overlap)
             obs = o["bs"]
             k = o["kernels"]
             others[name] = {
@@ -542,6 +547,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--also", default="cfg4,cfg3", help="comma-separated other configs to run briefly (N=1 only); '' for none")
     ap.add_argument("--also-steps", type=int, default=20)
+    ap.add_argument("--no-overlap", action="store_true", help="run the step on one stream (casts and GEMMs serialised)")
     ap.add_argument("--no-w8a8", action="store_true", help="skip the config 5 inference GEMM sweep")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -63,6 +63,8 @@ class BlockStep:
             lb.qdy.fmt = grad_fmt
         self.loss = None
         self.host = None
+        self.overlap = True   # casts and TWEO pass on a second stream, overlapping the GEMMs
+        self.side = None
         self.tau, self.eps, self.p, self.lam = 3.0, 1e-6, 4.0, 0.01
 
     # ---- inputs
@@ -113,10 +115,33 @@ class BlockStep:
                                                             grads=self.ga, ws=self.loss_ws)
 
     def step(self):
-        for lb in self.linears:
-            self.quantize_all(lb)
+        """One pass of the hot path.  The linears of a configuration are independent problems (each has
+        its own X, W, dY), so the casts run on a second stream and the GEMMs of linear i overlap the casts of
+        linear i+1 and the TWEO pass: the casts are HBM-bound, the GEMMs tensor-bound, and they share the SMs.
+        Fork / join on the calling stream, so the step can be captured into one CUDA graph."""
+        if not self.overlap:
+            for lb in self.linears:
+                self.quantize_all(lb)
+                self.gemms(lb)
+            self.tweo()
+            return
+        main = torch.cuda.current_stream()
+        if self.side is None:
+            self.side = torch.cuda.Stream()
+        side = self.side
+        side.wait_stream(main)
+        ready = []
+        with torch.cuda.stream(side):
+            for lb in self.linears:
+                self.quantize_all(lb)
+                ev = torch.cuda.Event()
+                ev.record(side)
+                ready.append(ev)
+            self.tweo()
+        for lb, ev in zip(self.linears, ready):
+            main.wait_event(ev)
             self.gemms(lb)
-        self.tweo()
+        main.wait_stream(side)
 
     @property
     def flops_per_step(self) -> int:

@@ -477,3 +477,52 @@ def test_w8a8_static_gemm(tw, M):
     torch.cuda.synchronize()
     assert rel_fro(y.float().cpu().numpy()[r, c], ref) <= GEMM_TOL
     assert torch.equal(y.view(torch.int16), y2.view(torch.int16))   # cast inside == pre-cast codes
+
+
+# ------------------------------------------------------------------ the whole step, one stream vs two
+def test_step_on_two_streams_equals_step_on_one(tw):
+    """The step runner overlaps the casts with the GEMMs on a second stream (directly, and replayed from
+    a CUDA graph): every output must equal the one-stream step bit for bit."""
+    from paper_2511_23225_b200.workload import BlockStep
+    bs = BlockStep(1)
+    bs.make_host_inputs()
+    bs.upload()
+
+    def outputs():
+        torch.cuda.synchronize()
+        out = [bs.loss.clone()] + [g.clone() for g in bs.ga]
+        for lb in bs.linears:
+            out += [t.clone() for t in (lb.qx.q, lb.qw.q, lb.qdy.q, lb.qx.scale, lb.qdy.amax, lb.y, lb.dx, lb.dw)]
+        return out
+
+    def wipe():
+        for lb in bs.linears:
+            for t in (lb.qx.q, lb.qw.q, lb.qdy.q, lb.y, lb.dx, lb.dw):
+                t.zero_()
+        for g in bs.ga:
+            g.zero_()
+
+    bs.overlap = False
+    bs.step()
+    ref = outputs()
+    wipe()
+    bs.overlap = True
+    bs.step()
+    two = outputs()
+    wipe()
+    st = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        bs.step()                      # warm the side stream before capture
+        torch.cuda.synchronize()
+        wipe()
+        with torch.cuda.graph(graph, stream=st):
+            bs.step()
+    torch.cuda.synchronize()
+    wipe()
+    graph.replay()
+    rep = outputs()
+    assert tw.read_device_status() == 0
+    for a, b, c in zip(ref, two, rep):
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+        assert torch.equal(a.view(torch.uint8), c.view(torch.uint8))
