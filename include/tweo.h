@@ -5,10 +5,10 @@
  * What the calls compute follows the TWEO paper (arXiv 2511.23225):
  *   - Sec. 3.3, Eq. 2-3: the penalty  L_TWEO = (1/L) sum_l mean((|A^(l)|/(tau+eps))^p)
  *     on every transformer block output A^(l), weighted by lambda(t);
- *   - Sec. 4.2: every linear layer runs in FP8 with ONE scale per tensor,
+ *   - Sec. 4.3 (the subsection on full FP8 pre-training of LLMs): every linear layer runs in FP8 with ONE scale per tensor,
  *     E4M3 for activations and weights, E5M2 for gradients (the HYBRID recipe),
  *     scales derived from the tensor's absolute maximum;
- *   - Sec. 4.3, Eq. 4 and the "W8(T)A8(T)" discussion: inference with static
+ *   - Sec. 4.4 (the subsection on post-training quantisation), Eq. 4 and the "W8(T)A8(T)" discussion: inference with static
  *     per-tensor scales for weights and activations.
  *
  * Conventions (all calls)
@@ -82,7 +82,7 @@ typedef enum { TWEO_GRAN_TENSOR = 0, TWEO_GRAN_ROW = 1 } tweo_granularity_t;
 #define TWEO_MAX_BLOCKS 128
 
 /*
- * Optional fused outputs of a GEMM epilogue (Sec. 4.2: with delayed scaling the
+ * Optional fused outputs of a GEMM epilogue (Sec. 4.3: with delayed scaling the
  * next layer's scale is known before the GEMM runs, so the cast of the output
  * can ride on the epilogue instead of costing two more passes over it).
  * All three act on the bf16-ROUNDED output values, so that the fused result is
@@ -102,7 +102,7 @@ typedef struct tweo_epilogue_t {
 
 /*
  * tweo_quantize_per_tensor -- amax, scale and FP8 cast of one bf16 tensor
- * (Sec. 4.2: one scaling factor for the entire tensor; E4M3 range +-448).
+ * (Sec. 4.3: one scaling factor for the entire tensor; E4M3 range +-448).
  *   x [n] bf16 in.  q [n] uint8 out (same element order).  n >= 0; n == 0 yields
  *   amax 0, scale 1 (CURRENT) and writes nothing to q.
  *   mode CURRENT: amax = max|x_i|; scale = fl32(FP8MAX/amax) (1 if amax is 0 or
@@ -126,7 +126,7 @@ TWEO_API tweo_status_t tweo_quantize_per_tensor(const uint16_t* x, int64_t n, in
 
 /*
  * tweo_quantize_per_tensor_batch -- tweo_quantize_per_tensor for up to
- * TWEO_MAX_QUANT_BATCH tensors in one pair of kernels (Sec. 4.2: a linear layer casts its
+ * TWEO_MAX_QUANT_BATCH tensors in one pair of kernels (Sec. 4.3: a linear layer casts its
  * activation, its weight and, in the backward pass, its output gradient, each with its
  * own per-tensor scale; casting them together saves launches, which dominate for small
  * tensors).  Every tensor is treated exactly as tweo_quantize_per_tensor would treat it
@@ -155,7 +155,7 @@ TWEO_API tweo_status_t tweo_quantize_per_tensor_batch(const tweo_quant_desc_t* d
                                              size_t ws_bytes, void* stream);
 
 /*
- * tweo_fp8_linear_fwd -- forward GEMM of an FP8 linear layer (Sec. 4.2):
+ * tweo_fp8_linear_fwd -- forward GEMM of an FP8 linear layer (Sec. 4.3):
  *   Y[M,N] = (Xq[M,K] . Wq[N,K]^T) * (*sx_inv) * (*sw_inv), fp32 accumulation on
  *   the tensor cores, result rounded once to bf16.
  *   xq [M,K] codes (fmt_x), wq [N,K] codes (fmt_w), y [M,N] bf16.
@@ -173,7 +173,7 @@ TWEO_API tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const
                                   const tweo_epilogue_t* epi, void* ws, size_t ws_bytes, void* stream);
 
 /*
- * tweo_fp8_linear_bwd_dgrad -- data gradient (Sec. 4.2, gradients in E5M2):
+ * tweo_fp8_linear_bwd_dgrad -- data gradient (Sec. 4.3, gradients in E5M2):
  *   dX[M,K] = (dYq[M,N] . Wq[N,K]) * (*sdy_inv) * (*sw_inv) -> bf16; the
  *   contraction runs over N.  wq is the same buffer the forward call used.
  *   Shapes: N % 16 == 0, K % 16 == 0.  epi may be NULL.
@@ -186,7 +186,7 @@ TWEO_API tweo_status_t tweo_fp8_linear_bwd_dgrad(const uint8_t* dyq, int64_t ldd
                                         void* stream);
 
 /*
- * tweo_fp8_linear_bwd_wgrad -- weight gradient (Sec. 4.2):
+ * tweo_fp8_linear_bwd_wgrad -- weight gradient (Sec. 4.3):
  *   dW[N,K] = (dYq[M,N]^T . Xq[M,K]) * (*sx_inv) * (*sdy_inv); the contraction
  *   runs over the tokens M.  dw has the layout of W.  dw_dtype TWEO_BF16
  *   (uint16_t*) or TWEO_F32 (float*); accumulate != 0 adds into dw instead of
@@ -200,7 +200,7 @@ TWEO_API tweo_status_t tweo_fp8_linear_bwd_wgrad(const uint8_t* xq, int64_t ldx,
                                         void* stream);
 
 /*
- * tweo_fp8_linear_bwd -- both gradients of a linear layer in one call (Sec. 4.2): exactly
+ * tweo_fp8_linear_bwd -- both gradients of a linear layer in one call (Sec. 4.3): exactly
  *   tweo_fp8_linear_bwd_dgrad (dX, bf16) followed by tweo_fp8_linear_bwd_wgrad (dW, bf16,
  *   overwrite), without fused epilogue outputs; results are bit-identical to the two calls.
  *   When M, N and K all exceed 128 the two products run as ONE kernel launch: their tiles
@@ -243,7 +243,7 @@ TWEO_API tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, in
 /*
  * tweo_block_output_fused -- the block output and everything that touches it once, in one pass
  * (Sec. 3.3: the penalty acts on A = x + f(x), the residual stream plus the block's branch;
- * Sec. 4.2: with delayed scaling the FP8 scale of A for the next block is known beforehand):
+ * Sec. 4.3: with delayed scaling the FP8 scale of A for the next block is known beforehand):
  *   a_i   = bf16( fl32(x_i + f_i) )                  written to a [n] (may alias x or f)
  *   *loss = (1/n) sum_i (|a_i| / (tau+eps))^p        this block's term of Eq. 3
  *   g_i   = grad_coeff * p * sign(a_i) |a_i|^(p-1) / (n (tau+eps)^p)   -> grad [n] bf16, or NULL
@@ -263,7 +263,7 @@ TWEO_API tweo_status_t tweo_block_output_fused(const uint16_t* x, const uint16_t
 
 /*
  * tweo_delayed_scaling_update -- one step of delayed per-tensor scaling for n_tensors tensors of
- * one FP8 format (Sec. 4.2: amax history of length 16 in the paper's runs).  For every tensor t:
+ * one FP8 format (Sec. 4.3: amax history of length 16 in the paper's runs).  For every tensor t:
  * the history amax_history[t][0..history_len) moves one place (the oldest value drops out),
  * amax_new[t] enters at index 0, and scale[t] = fl32(FP8MAX / max(history)) (clamped to FLT_MAX)
  * becomes the scale for the NEXT step; if that maximum is zero or not finite scale[t] is kept.
@@ -306,7 +306,7 @@ TWEO_API tweo_status_t tweo_loss_fwd_bwd_static(const uint16_t* const* a, int32_
 
 /*
  * tweo_w8a8_static_gemm -- inference linear with static per-tensor scales for
- * both operands (Sec. 4.3: AbsMax static quantisation, W8(T)A8(T)), in the E4M3
+ * both operands (Sec. 4.4: AbsMax static quantisation, W8(T)A8(T)), in the E4M3
  * flavour: Y[M,N] = (Xq . Wq^T) * (1 / *sx) * (*sw_inv) -> bf16.
  *   x: activations [M,K]; x_dtype TWEO_BF16 (cast inside with the static scale
  *      *sx, saturating; needs a workspace for the codes) or TWEO_FP8_E4M3
@@ -322,7 +322,7 @@ TWEO_API tweo_status_t tweo_w8a8_static_gemm(const void* x, int32_t x_dtype, int
                                     size_t ws_bytes, void* stream);
 
 /*
- * tweo_absmax_quantize -- symmetric AbsMax b-bit quantisation (Sec. 4.3, Eq. 4):
+ * tweo_absmax_quantize -- symmetric AbsMax b-bit quantisation (Sec. 4.4, Eq. 4):
  *   s = max|X| + eps,  X_q = round(X / s * Q_b),  Q_b = 2^(b-1) - 1   (Q_8 = 127, Q_6 = 31),
  * with one s for the whole tensor (TWEO_GRAN_TENSOR: the paper's "T") or one per row
  * (TWEO_GRAN_ROW: per output channel "C" for a weight [N,K], per token "K" for an activation
@@ -340,7 +340,7 @@ TWEO_API tweo_status_t tweo_absmax_quantize(const uint16_t* x, int64_t rows, int
                                    int8_t* q, int64_t ldq, void* ws, size_t ws_bytes, void* stream);
 
 /*
- * tweo_int8_linear -- the 8-bit (or b-bit) integer linear of Sec. 4.3 on Eq. 4's codes:
+ * tweo_int8_linear -- the 8-bit (or b-bit) integer linear of Sec. 4.4 on Eq. 4's codes:
  *   Y[M,N] = (sum_k Xq[m,k] Wq[n,k]) * (sx[m or 0] / Q_b) * (sw[n or 0] / Q_b)  -> bf16,
  * the product of the dequantised operands.  Integer tensor cores, int32 accumulation (exact).
  * xq [M,K], wq [N,K] int8 codes (row pitches multiples of 16); sx: device float [1] (per tensor,

@@ -7,13 +7,13 @@
  *
  *   - the TWEO regulariser (paper Eq. 3) and its derivative (paper Eq. 2 times
  *     Eq. 3, differentiated with respect to each activation),
- *   - per-tensor FP8 scaling and casting (paper Sec. 4.2: one scale for the
+ *   - per-tensor FP8 scaling and casting (paper Sec. 4.3: one scale for the
  *     whole tensor, E4M3 forward / E5M2 gradients; E4M3 range +-448 from the
  *     paper's introduction) with the OCP FP8 code tables,
  *   - the three linear-layer contractions on the quantised operands,
  *   - symmetric AbsMax b-bit quantisation (paper Eq. 4),
  *   - the block output A = x + f(x) the regulariser acts on (paper Sec. 3.3) and the
- *     delayed-scaling state (paper Sec. 4.2: amax history of length 16).
+ *     delayed-scaling state (paper Sec. 4.3: amax history of length 16).
  *
  * Floating point is FP64 unless the step is *defined* in FP32 (the scale, the
  * scaled value that gets rounded to FP8).  There is no blocking, no SIMD, no
@@ -159,7 +159,7 @@ void oracle_fp8_encode_array(const float* v, int64_t n, int fmt, int which, uint
 
 /* ------------------------------------------------- amax / scale / quantize */
 
-/* amax = max_i |x_i| over the whole tensor (one scale per tensor, Sec. 4.2).
+/* amax = max_i |x_i| over the whole tensor (one scale per tensor, Sec. 4.3).
  * NaN elements are skipped (fmax semantics); infinities count. */
 float oracle_amax_bf16(const uint16_t* x, int64_t n) {
   float amax = 0.0f;
@@ -400,7 +400,7 @@ void oracle_absmax_quantize_bf16(const uint16_t* x, int64_t n, int bits, float s
   }
 }
 
-/* 8-bit linear on the integer codes (Sec. 4.3): Y_mn = (sum_k Xq_mk * Wq_nk) * (sx_m / Q_b) * (sw_n / Q_b),
+/* 8-bit linear on the integer codes (Sec. 4.4): Y_mn = (sum_k Xq_mk * Wq_nk) * (sx_m / Q_b) * (sw_n / Q_b),
  * i.e. the product of the dequantised operands of Eq. 4, with one scale per tensor or per
  * row (token for X, output channel for W).  The integer sum is exact; the scales are applied
  * in FP64.  Evaluated at the listed (row, col) points. */
@@ -431,7 +431,7 @@ void oracle_residual_add_bf16(const uint16_t* x, const uint16_t* f, int64_t n, u
 }
 
 /* ------------------------------------------------------------------ delayed scaling */
-/* Sec. 4.2: per-tensor delayed scaling with an amax history of length H (16 in the paper).
+/* Sec. 4.3: per-tensor delayed scaling with an amax history of length H (16 in the paper).
  * One update per training step and tensor: the history moves one place (the oldest value
  * drops out), the step's amax enters at index 0, and the scale for the NEXT step is
  * FP8MAX / max(history) -- as oracle_scale_from_amax computes it.  If that maximum is zero

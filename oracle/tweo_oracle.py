@@ -3,7 +3,7 @@
 TEST INFRASTRUCTURE.  Only tests, the smoke check and the benchmark's CPU
 baseline leg may import this module.  It performs no arithmetic of the method
 itself: every function marshals numpy arrays into the C routines, which are
-the plain restatement of the paper's definitions (Eq. 2-4, Sec. 4.2).  It does
+the plain restatement of the paper's definitions (Eq. 2-4, Sec. 4.3).  It does
 not import, and is not imported by, the CUDA package.
 """
 from __future__ import annotations
@@ -312,7 +312,7 @@ def residual_add_bf16(x_bits, f_bits) -> np.ndarray:
 
 
 def delayed_scaling_update(history, amax_new, fmt: int, scale):
-    """One delayed-scaling step for one tensor (Sec. 4.2).  `history` (float32 [H]) is updated in
+    """One delayed-scaling step for one tensor (Sec. 4.3).  `history` (float32 [H]) is updated in
     place; returns (scale, scale_inv) for the next step."""
     h = np.ascontiguousarray(history, dtype=np.float32)
     assert h is history or np.shares_memory(h, history), "history must be a contiguous float32 array"

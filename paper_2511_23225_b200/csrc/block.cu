@@ -1,7 +1,7 @@
 // Block output in one pass, and the delayed-scaling state update.
 //
 // (1) The TWEO penalty acts on the output of every transformer block, A = x + f(x) (Sec. 3.3),
-// and with delayed per-tensor scaling (Sec. 4.2) the scale of A for the next block's FP8
+// and with delayed per-tensor scaling (Sec. 4.3) the scale of A for the next block's FP8
 // linears is known before A exists.  So everything that touches A once can ride on the
 // residual addition itself: read x and f, form a = bf16(fl32(x + f)), and in the same pass
 // emit a, the penalty's partial sums, its gradient, amax(a) and the FP8 codes of a.  That is

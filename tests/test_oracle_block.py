@@ -1,4 +1,4 @@
-"""Pins for the oracle's block-output sum (Sec. 3.3) and delayed-scaling update (Sec. 4.2)."""
+"""Pins for the oracle's block-output sum (Sec. 3.3) and delayed-scaling update (Sec. 4.3)."""
 import numpy as np
 import torch
 
