@@ -13,7 +13,9 @@
  *   - the three linear-layer contractions on the quantised operands,
  *   - symmetric AbsMax b-bit quantisation (paper Eq. 4),
  *   - the block output A = x + f(x) the regulariser acts on (paper Sec. 3.3) and the
- *     delayed-scaling state (paper Sec. 4.3: amax history of length 16).
+ *     delayed-scaling state (paper Sec. 4.3: amax history of length 16),
+ *   - LayerNorm / RMSNorm (paper Sec. 4.3 runs the LayerNorm components under FP8 too) and
+ *     the MLP activations of the paper's models (Sec. 3.2: GELU, GLU variants).
  *
  * Floating point is FP64 unless the step is *defined* in FP32 (the scale, the
  * scaled value that gets rounded to FP8).  There is no blocking, no SIMD, no
@@ -448,4 +450,57 @@ void oracle_delayed_scaling_update(float* history, int H, float amax_new, int fm
     volatile float inv = 1.0f / *scale;
     *scale_inv = inv;
   }
+}
+
+/* ------------------------------------------------------------------ normalisation and MLP activations */
+/* Sec. 4.3 puts the LayerNorm components under FP8 as well as the linears: the normalised
+ * row is what the next linear consumes, so it is cast with that linear's per-tensor scale.
+ * LayerNorm over the last dimension, written out (FP64):
+ *     mu = (1/d) sum_j x_j,  var = (1/d) sum_j (x_j - mu)^2   (biased),
+ *     y_j = (x_j - mu) / sqrt(var + eps) * gamma_j + beta_j.
+ * rms != 0 gives the RMSNorm of the Llama-style blocks instead: mu := 0 and
+ *     var := (1/d) sum_j x_j^2, no centring; beta may be NULL (zero).
+ * x: bf16 [rows, d]; gamma, beta: binary32 [d]; y: FP64 [rows, d]; mean / rstd (optional): FP64 [rows]. */
+void oracle_layernorm(const uint16_t* x, int64_t rows, int64_t d, const float* gamma, const float* beta,
+                      double eps, int rms, double* y, double* mean, double* rstd) {
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r) {
+    const uint16_t* xr = x + r * d;
+    double mu = 0.0;
+    if (!rms) {
+      for (int64_t j = 0; j < d; ++j) mu += (double)bf16_bits_to_f32(xr[j]);
+      mu /= (double)d;
+    }
+    double var = 0.0;
+    for (int64_t j = 0; j < d; ++j) {
+      const double c = (double)bf16_bits_to_f32(xr[j]) - mu;
+      var += c * c;
+    }
+    var /= (double)d;
+    const double rs = 1.0 / sqrt(var + eps);
+    for (int64_t j = 0; j < d; ++j) {
+      const double c = (double)bf16_bits_to_f32(xr[j]) - mu;
+      y[r * d + j] = c * rs * (double)gamma[j] + (beta ? (double)beta[j] : 0.0);
+    }
+    if (mean) mean[r] = mu;
+    if (rstd) rstd[r] = rs;
+  }
+}
+
+/* The MLP activations the paper's models use (Sec. 3.2: classic MLPs with GELU, modern
+ * MLPs with GLU variants), as their definitions, FP64:
+ *   kind 1  GELU(v) = v * Phi(v) = v/2 * (1 + erf(v / sqrt 2))
+ *   kind 2  GELU, tanh form: v/2 * (1 + tanh( sqrt(2/pi) * (v + 0.044715 v^3) ))
+ *   kind 3  SiLU(v) = v / (1 + exp(-v))   (the gate of SwiGLU: out = SiLU(gate) * up) */
+double oracle_activation(double v, int kind) {
+  switch (kind) {
+    case 1: return 0.5 * v * (1.0 + erf(v / sqrt(2.0)));
+    case 2: return 0.5 * v * (1.0 + tanh(sqrt(2.0 / (4.0 * atan(1.0))) * (v + 0.044715 * v * v * v)));
+    case 3: return v / (1.0 + exp(-v));
+    default: return v;
+  }
+}
+
+void oracle_activation_array(const double* v, int64_t n, int kind, double* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = oracle_activation(v[i], kind);
 }

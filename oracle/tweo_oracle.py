@@ -98,6 +98,13 @@ def lib():
             L.oracle_absmax_dequantize.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_double, C.c_void_p]
             L.oracle_absmax_scale.restype = C.c_double
             L.oracle_absmax_scale.argtypes = [C.c_void_p, C.c_int64, C.c_double]
+            L.oracle_layernorm.restype = None
+            L.oracle_layernorm.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_double, C.c_int,
+                                           C.c_void_p, C.c_void_p, C.c_void_p]
+            L.oracle_activation.restype = C.c_double
+            L.oracle_activation.argtypes = [C.c_double, C.c_int]
+            L.oracle_activation_array.restype = None
+            L.oracle_activation_array.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p]
             _lib = L
     return _lib
 
@@ -357,3 +364,45 @@ def int8_gemm_at(xq, wq, sx, sw, bits: int, rows, cols) -> np.ndarray:
                               1 if sx.size > 1 else 0, sw.ctypes.data, 1 if sw.size > 1 else 0, bits, xq.shape[1],
                               rows.ctypes.data, cols.ctypes.data, rows.size, out.ctypes.data)
     return out
+
+
+ACT_NONE, ACT_GELU_ERF, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3
+
+
+def layernorm(x_bits, gamma, beta, eps, rms: bool = False):
+    """LayerNorm (or RMSNorm) over the last dimension of a bf16 [rows, d] tensor, FP64 (Sec. 4.3 runs the
+    LayerNorm components under FP8 too).  Returns (y [rows, d], mean [rows], rstd [rows])."""
+    x = _u16(x_bits)
+    assert x.ndim == 2
+    rows, d = x.shape
+    g = np.ascontiguousarray(gamma, dtype=np.float32)
+    b = None if beta is None else np.ascontiguousarray(beta, dtype=np.float32)
+    assert g.shape == (d,) and (b is None or b.shape == (d,))
+    y = np.empty((rows, d), dtype=np.float64)
+    mean = np.empty(rows, dtype=np.float64)
+    rstd = np.empty(rows, dtype=np.float64)
+    lib().oracle_layernorm(x.ctypes.data, rows, d, g.ctypes.data, None if b is None else b.ctypes.data, float(eps),
+                           1 if rms else 0, y.ctypes.data, mean.ctypes.data, rstd.ctypes.data)
+    return y, mean, rstd
+
+
+def activation(v, kind: int) -> np.ndarray:
+    """GELU (erf or tanh form) or SiLU of FP64 values (Sec. 3.2: the MLPs of the paper's models)."""
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    out = np.empty(v.shape, dtype=np.float64)
+    lib().oracle_activation_array(v.ctypes.data, v.size, kind, out.ctypes.data)
+    return out
+
+
+def gemm_fwd_act_at(xq, fmt_x, wq, fmt_w, sx_inv, sw_inv, kind: int, rows, cols) -> np.ndarray:
+    """Forward product followed by the MLP activation at the given points.  kind 1/2: GELU(Y[m,n]).
+    kind 3 (SwiGLU): wq holds the gate rows [0, F) then the up rows [F, 2F); returns
+    SiLU(Y[m, n]) * Y[m, F + n] for n < F."""
+    rows, cols = _pts(rows, cols)
+    if kind == ACT_SILU:
+        F = wq.shape[0] // 2
+        assert wq.shape[0] == 2 * F and np.all(cols < F)
+        gate = gemm_fwd_at(xq, fmt_x, wq, fmt_w, sx_inv, sw_inv, rows, cols)
+        up = gemm_fwd_at(xq, fmt_x, wq, fmt_w, sx_inv, sw_inv, rows, cols + F)
+        return activation(gate, ACT_SILU) * up
+    return activation(gemm_fwd_at(xq, fmt_x, wq, fmt_w, sx_inv, sw_inv, rows, cols), kind)
