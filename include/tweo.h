@@ -77,6 +77,8 @@ typedef enum {
   TWEO_OP_ABSMAX = 7
 } tweo_op_t;
 typedef enum { TWEO_GRAN_TENSOR = 0, TWEO_GRAN_ROW = 1 } tweo_granularity_t;
+typedef enum { TWEO_ACT_NONE = 0, TWEO_ACT_GELU = 1, TWEO_ACT_GELU_TANH = 2, TWEO_ACT_SWIGLU = 3 } tweo_act_t;
+typedef enum { TWEO_NORM_LAYER = 0, TWEO_NORM_RMS = 1 } tweo_norm_t;
 
 /* Upper bound on the number of block outputs one tweo_loss_fwd_bwd call takes. */
 #define TWEO_MAX_BLOCKS 128
@@ -171,6 +173,51 @@ TWEO_API tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const
                                   const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy,
                                   int64_t M, int64_t N, int64_t K, int32_t fmt_x, int32_t fmt_w,
                                   const tweo_epilogue_t* epi, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * tweo_fp8_linear_fwd_act -- forward GEMM of an FP8 linear layer with the MLP's activation
+ * applied in the epilogue (Sec. 3.2: the classic MLP with GELU and the gated MLP of the
+ * Llama-style blocks; Sec. 4.3: the next linear consumes FP8, so its input can be cast here
+ * instead of in two more passes over the activation):
+ *   Z[m,n] = (Xq . Wq^T)[m,n] * (*sx_inv) * (*sw_inv)                (binary32)
+ *   TWEO_ACT_GELU       Y = Z * Phi(Z)  (erf form)
+ *   TWEO_ACT_GELU_TANH  Y = Z/2 * (1 + tanh( sqrt(2/pi) (Z + 0.044715 Z^3) ))
+ *   TWEO_ACT_SWIGLU     Y[m,n] = SiLU(Z[m,n]) * Z[m,N+n], n < N: wq holds 2N rows, the N
+ *                       gate rows first, then the N up rows
+ *   TWEO_ACT_NONE       Y = Z (the call forwards to tweo_fp8_linear_fwd; y required)
+ * Y is evaluated in binary32 (the tanh form with the hardware tanh, relative error 2^-11)
+ * and rounded once to bf16; the optional outputs of epi act on the rounded values exactly as
+ * in tweo_fp8_linear_fwd.  xq [M,K], wq [N,K] (SwiGLU: [2N,K]) codes; y [M,N] bf16, or NULL
+ * when only the FP8 copy (epi->out_q) is wanted.  Shapes: M >= 1, N % 16 == 0, K % 16 == 0.
+ * Errors: TWEO_ERR_INVALID_ARG (NULL pointers, bad enums, neither y nor epi->out_q),
+ * TWEO_ERR_UNSUPPORTED_SHAPE, TWEO_ERR_ALIGNMENT.
+ */
+TWEO_API tweo_status_t tweo_fp8_linear_fwd_act(const uint8_t* xq, int64_t ldx, const uint8_t* wq, int64_t ldw,
+                                      const float* sx_inv, const float* sw_inv, int32_t act, uint16_t* y,
+                                      int64_t ldy, int64_t M, int64_t N, int64_t K, int32_t fmt_x,
+                                      int32_t fmt_w, const tweo_epilogue_t* epi, void* stream);
+
+/*
+ * tweo_layernorm_fp8 -- LayerNorm (or RMSNorm) over the last dimension with the FP8 cast of
+ * its output for the following linear in the same pass (Sec. 4.3: the LayerNorm components run
+ * under FP8 together with the linears; with delayed scaling the scale is known beforehand):
+ *   TWEO_NORM_LAYER  mu = mean_j x_j, var = mean_j (x_j - mu)^2,
+ *                    y_j = (x_j - mu) / sqrt(var + eps) * gamma_j + beta_j
+ *   TWEO_NORM_RMS    y_j = x_j / sqrt(mean_j x_j^2 + eps) * gamma_j (+ beta_j if given)
+ * evaluated in binary32 and rounded once to bf16; then, on the rounded values,
+ *   yq_j = sat_rne_fp8( fl32(y_j * *q_scale) ) and *amax = max |y_j| over the whole output
+ * (bit-identical to tweo_quantize_per_tensor(GIVEN) on the stored y).
+ *   x [rows, d] bf16 (row pitch ldx); gamma, beta: device float [d] (beta may be NULL);
+ *   y [rows, d] bf16 or NULL; yq [rows, d] codes (q_fmt) or NULL, q_scale required with yq;
+ *   amax: device float* or NULL; mean, rstd: device float [rows] or NULL (mu and
+ *   1/sqrt(var + eps) per row, for a backward pass).  At least one of y, yq must be given.
+ * Shapes: d % 8 == 0, 8 <= d <= 8192; ldx, ldy, ldq multiples of 8; rows >= 0 (0: only *amax = 0).
+ * Errors: TWEO_ERR_INVALID_ARG, TWEO_ERR_UNSUPPORTED_SHAPE, TWEO_ERR_ALIGNMENT.
+ */
+TWEO_API tweo_status_t tweo_layernorm_fp8(const uint16_t* x, int64_t ldx, int64_t rows, int64_t d, int32_t kind,
+                                 const float* gamma, const float* beta, float eps, uint16_t* y, int64_t ldy,
+                                 uint8_t* yq, int64_t ldq, int32_t q_fmt, const float* q_scale, float* amax,
+                                 float* mean, float* rstd, void* stream);
 
 /*
  * tweo_fp8_linear_bwd_dgrad -- data gradient (Sec. 4.3, gradients in E5M2):

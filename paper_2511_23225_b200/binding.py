@@ -18,13 +18,16 @@ SCALE_CURRENT, SCALE_GIVEN = 0, 1
 BF16, F32, FP8_E4M3 = 0, 1, 2
 OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_DGRAD, OP_LINEAR_WGRAD, OP_LOSS, OP_W8A8, OP_BLOCK_OUTPUT, OP_ABSMAX = range(8)
 GRAN_TENSOR, GRAN_ROW = 0, 1
+ACT_NONE, ACT_GELU, ACT_GELU_TANH, ACT_SWIGLU = 0, 1, 2, 3
+NORM_LAYER, NORM_RMS = 0, 1
 MAX_BLOCKS = 128
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtweo_b200.so")
 
 EXPORTS = [
-    "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_bwd_dgrad",
+    "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_fwd_act",
+    "tweo_layernorm_fp8", "tweo_fp8_linear_bwd_dgrad",
     "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
     "tweo_block_output_fused", "tweo_delayed_scaling_update", "tweo_absmax_quantize", "tweo_int8_linear",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
@@ -73,6 +76,9 @@ def lib() -> C.CDLL:
         L.tweo_quantize_per_tensor_batch.argtypes = [C.POINTER(_QuantDesc), i32, vp, sz, vp]
         L.tweo_fp8_linear_fwd.argtypes = [vp, i64, vp, i64, vp, vp, vp, i64, i64, i64, i64, i32, i32,
                                           C.POINTER(_Epilogue), vp, sz, vp]
+        L.tweo_fp8_linear_fwd_act.argtypes = [vp, i64, vp, i64, vp, vp, i32, vp, i64, i64, i64, i64, i32, i32,
+                                              C.POINTER(_Epilogue), vp]
+        L.tweo_layernorm_fp8.argtypes = [vp, i64, i64, i64, i32, vp, vp, f32, vp, i64, vp, i64, i32, vp, vp, vp, vp, vp]
         L.tweo_fp8_linear_bwd_dgrad.argtypes = [vp, i64, i32, vp, i64, i32, vp, vp, vp, i64, i64, i64, i64,
                                                 C.POINTER(_Epilogue), vp, sz, vp]
         L.tweo_fp8_linear_bwd_wgrad.argtypes = [vp, i64, i32, vp, i64, i32, vp, vp, vp, i64, i32, i32,
@@ -251,6 +257,68 @@ def fp8_linear_fwd(xq, wq, sx_inv, sw_inv, fmt_x=E4M3, fmt_w=E4M3, y=None, out_a
                                      _epilogue(out_amax, out_q, q_fmt, q_scale), *_ws(ws), _stream()),
            "tweo_fp8_linear_fwd")
     return y
+
+
+def fp8_linear_fwd_act(xq, wq, sx_inv, sw_inv, act, fmt_x=E4M3, fmt_w=E4M3, y=None, want_y=True, out_amax=None,
+                       out_q=None, q_fmt=E4M3, q_scale=None):
+    """tweo_fp8_linear_fwd_act: act(Xq . Wq^T * sx_inv * sw_inv) -> bf16 and / or FP8.  For ACT_SWIGLU wq holds
+    the gate rows followed by the up rows and the output has half as many columns as wq has rows.
+    want_y=False with out_q given writes only the FP8 copy.  Returns y (or None)."""
+    M, K = xq.shape
+    N, K2 = wq.shape
+    if K != K2:
+        raise ValueError("inner dimensions differ")
+    if act == ACT_SWIGLU:
+        if N % 2:
+            raise ValueError("SwiGLU needs an even number of weight rows (gate rows, then up rows)")
+        N //= 2
+    if want_y and y is None:
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=xq.device)
+    if not want_y:
+        y = None
+    _check(lib().tweo_fp8_linear_fwd_act(_dev(xq, U8, "xq"), _rows(xq, "xq"), _dev(wq, U8, "wq"), _rows(wq, "wq"),
+                                         _dev(sx_inv, torch.float32), _dev(sw_inv, torch.float32), act,
+                                         _dev(y, torch.bfloat16, "y") if y is not None else None,
+                                         _rows(y, "y") if y is not None else 0, M, N, K, fmt_x, fmt_w,
+                                         _epilogue(out_amax, out_q, q_fmt, q_scale), _stream()),
+           "tweo_fp8_linear_fwd_act")
+    return y
+
+
+def layernorm_fp8(x, gamma, beta=None, eps=1e-5, kind=NORM_LAYER, want_y=True, q_fmt=None, q_scale=None,
+                  want_amax=True, want_stats=False, y=None, yq=None):
+    """tweo_layernorm_fp8: LayerNorm / RMSNorm over the last dimension of a bf16 [rows, d] tensor with the FP8
+    cast of the output (q_fmt, q_scale) and its amax in the same pass.
+    Returns (y or None, yq or None, amax [1] or None, mean [rows] or None, rstd [rows] or None)."""
+    rows, d = x.shape
+    dev = x.device
+    if want_y and y is None:
+        y = torch.empty((rows, d), dtype=torch.bfloat16, device=dev)
+    if not want_y:
+        y = None
+    if q_fmt is not None:
+        if q_scale is None:
+            raise ValueError("the FP8 copy needs q_scale")
+        if yq is None:
+            yq = torch.empty((rows, d), dtype=torch.uint8, device=dev)
+    else:
+        yq = None
+    amax = torch.empty(1, dtype=torch.float32, device=dev) if want_amax else None
+    mean = torch.empty(rows, dtype=torch.float32, device=dev) if want_stats else None
+    rstd = torch.empty(rows, dtype=torch.float32, device=dev) if want_stats else None
+    _check(lib().tweo_layernorm_fp8(_dev(x, torch.bfloat16, "x"), _rows(x, "x"), rows, d, kind,
+                                    _dev(gamma, torch.float32, "gamma"),
+                                    _dev(beta, torch.float32, "beta") if beta is not None else None, eps,
+                                    _dev(y, torch.bfloat16, "y") if y is not None else None,
+                                    _rows(y, "y") if y is not None else 0,
+                                    _dev(yq, U8, "yq") if yq is not None else None,
+                                    _rows(yq, "yq") if yq is not None else 0, q_fmt if q_fmt is not None else 0,
+                                    _dev(q_scale, torch.float32, "q_scale") if q_scale is not None else None,
+                                    amax.data_ptr() if amax is not None else None,
+                                    mean.data_ptr() if mean is not None else None,
+                                    rstd.data_ptr() if rstd is not None else None, _stream()),
+           "tweo_layernorm_fp8")
+    return y, yq, amax, mean, rstd
 
 
 def fp8_linear_bwd_dgrad(dyq, wq, sdy_inv, sw_inv, fmt_dy=E5M2, fmt_w=E4M3, dx=None, out_amax=None, out_q=None,

@@ -605,6 +605,78 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
 #undef TWEO_DISPATCH
 }
 
+// Forward product with the MLP activation in the epilogue (pair kernel only; every tile whole).
+template <int ACT>
+tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, GemmParams& p,
+                              cudaStream_t st) {
+  constexpr int STAGES = 6;
+  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
+  auto kern = gemm_fp8_pair_kernel<false, false, STAGES, false, false, ACT>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_done = true;
+  }
+  p.tiles_m = (p.Md + 2 * BM - 1) / (2 * BM);
+  p.tiles_n = ACT == 3 ? (p.Nd + 127) / 128 : (p.Nd + 255) / 256;
+  p.k_blocks = (p.Kc + BK - 1) / BK;
+  p.sk_tiles = 0;
+  p.sk_partials = nullptr;
+  p.sk_flags = nullptr;
+  p.sk_counters = nullptr;
+  p.epoch = 0;
+  const int tiles = p.tiles_m * p.tiles_n;
+  int pairs = sm_count() / 2;
+  p.raster_g = raster_band(p.tiles_m, pairs);
+  if (pairs > tiles) pairs = tiles;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, p));
+  count_launch();
+  return check_launch("gemm_fp8_pair_kernel (activation epilogue)");
+}
+
+// N: output columns.  SwiGLU: wq has 2 N rows (gate rows, then up rows).
+tweo_status_t run_fwd_act(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
+                          int act, int64_t M, int64_t N, int64_t K, GemmParams p, cudaStream_t st) {
+  if (M > INT32_MAX || 2 * N > INT32_MAX || K > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(xq) || !aligned16(wq) || !aligned16(p.d) || (ldx & 15) || (ldw & 15) || ((p.ldd * 2) & 15))
+    return TWEO_ERR_ALIGNMENT;
+  p.Md = (int32_t)M;
+  p.Nd = (int32_t)N;
+  p.Kc = (int32_t)K;
+  p.idesc = make_idesc(fmt_x, fmt_w, false, false, 256, 256);
+  CUtensorMap ma, mb, md;
+  // without a bf16 output the store is skipped; the map then describes the FP8 output's memory and is never used
+  bool ok = p.d ? make_out_map(&md, p.d, N, M, p.ldd, false) : make_out_map(&md, p.out_q, N / 2, M, p.ldq / 2, false);
+  ok = ok && make_map(&ma, xq, K, M, ldx, BM);
+  ok = ok && make_map(&mb, wq, K, act == TWEO_ACT_SWIGLU ? 2 * N : N, ldw, 128);
+  if (!ok) {
+    cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return TWEO_ERR_CUDA;
+  }
+  if (p.out_amax) {
+    zero_float_kernel<<<1, 1, 0, st>>>(p.out_amax);
+    count_launch();
+  }
+  switch (act) {
+    case TWEO_ACT_GELU: return launch_pair_act<1>(ma, mb, md, p, st);
+    case TWEO_ACT_GELU_TANH: return launch_pair_act<2>(ma, mb, md, p, st);
+    case TWEO_ACT_SWIGLU: return launch_pair_act<3>(ma, mb, md, p, st);
+    default: return TWEO_ERR_INVALID_ARG;
+  }
+}
+
 // Forward product for M <= 128 (see gemm_skinny.cuh): W is streamed once, K is sliced over CTAs.
 tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
                          const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M, int64_t N,
@@ -835,6 +907,27 @@ tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const uint8_t*
   if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
   return tweo_detail::gemm_fwd_codes(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, y, ldy, M, N, K, epi, ws,
                                      ws_bytes, (cudaStream_t)stream);
+}
+
+tweo_status_t tweo_fp8_linear_fwd_act(const uint8_t* xq, int64_t ldx, const uint8_t* wq, int64_t ldw,
+                                      const float* sx_inv, const float* sw_inv, int32_t act, uint16_t* y, int64_t ldy,
+                                      int64_t M, int64_t N, int64_t K, int32_t fmt_x, int32_t fmt_w,
+                                      const tweo_epilogue_t* epi, void* stream) {
+  if (act == TWEO_ACT_NONE)
+    return tweo_fp8_linear_fwd(xq, ldx, wq, ldw, sx_inv, sw_inv, y, ldy, M, N, K, fmt_x, fmt_w, epi, nullptr, 0, stream);
+  if (act != TWEO_ACT_GELU && act != TWEO_ACT_GELU_TANH && act != TWEO_ACT_SWIGLU) return TWEO_ERR_INVALID_ARG;
+  if (!xq || !wq || !sx_inv || !sw_inv || !fmt_ok(fmt_x) || !fmt_ok(fmt_w)) return TWEO_ERR_INVALID_ARG;
+  if (!y && !(epi && epi->out_q)) return TWEO_ERR_INVALID_ARG;  // nothing to write
+  if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
+  if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  GemmParams p{};
+  p.d = y;
+  p.ldd = y ? ldy : 0;
+  p.sa_inv = sx_inv;
+  p.sb_inv = sw_inv;
+  tweo_status_t s = fill_epilogue(p, epi);
+  if (s != TWEO_OK) return s;
+  return run_fwd_act(xq, ldx, fmt_x, wq, ldw, fmt_w, act, M, N, K, p, (cudaStream_t)stream);
 }
 
 tweo_status_t tweo_fp8_linear_bwd_dgrad(const uint8_t* dyq, int64_t lddy, int32_t fmt_dy, const uint8_t* wq,

@@ -106,5 +106,27 @@ __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d) {
   return cvt_fp8x2<FMT>(a, b) | (cvt_fp8x2<FMT>(c, d) << 16);
 }
 
+// MLP activations of the forward epilogue (Sec. 3.2: GELU in the classic MLP, a gated unit in the
+// Llama-style one), on binary32 values.  1: v * Phi(v) with erff; 2: the tanh form with the
+// hardware tanh (relative error 2^-11, an order below the bf16 rounding that follows).
+template <int ACT>
+__device__ __forceinline__ float act_apply(float v) {
+  if (ACT == 1) {
+    const float h = 0.5f * v;
+    return fmaf(h, erff(v * 0.70710678118654752f), h);
+  }
+  if (ACT == 2) {
+    const float u = 0.79788456080286536f * fmaf(0.044715f * v * v, v, v);
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+    const float h = 0.5f * v;
+    return fmaf(h, t, h);
+  }
+  return v;
+}
+// SiLU(gate) * up = gate * up / (1 + exp(-gate))
+__device__ __forceinline__ float swiglu(float gate, float up) {
+  return __fdividef(gate, 1.0f + __expf(-gate)) * up;
+}
 
 }  // namespace tweo_detail

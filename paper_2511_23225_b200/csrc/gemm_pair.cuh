@@ -145,7 +145,14 @@ __device__ __noinline__ float pair_partial_share(const GemmParams& p, const CUte
 
 // I8: the operands are 8-bit integers (tcgen05 kind::i8, int32 accumulators) and the epilogue
 // applies the Eq. 4 dequantisation with one scale per tensor or per row / column.
-template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32, bool I8 = false>
+//
+// ACT (forward product, bf16 / FP8 output): the MLP activation applied to the scaled accumulator
+// before the one rounding to bf16 -- 1: GELU (erf), 2: GELU (tanh form), 3: SwiGLU.  For SwiGLU
+// B holds the gate rows [0, Nd) followed by the up rows [Nd, 2 Nd): the leader CTA loads 128
+// gate rows and its peer the matching 128 up rows, so accumulator columns [0,128) are the gate
+// and [128,256) the up projection of the same 128 output columns, and the tile that is stored
+// is 256 x 128: SiLU(gate) * up.  With p.d == nullptr only the FP8 copy / amax are produced.
+template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32, bool I8 = false, int ACT = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ GemmParams p) {
@@ -209,7 +216,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         int tm, tn;
         tile_coords(p, tile, tm, tn);
         const int m0 = tm * (2 * BM) + (int)rank * BM;  // this CTA's rows
-        const int n0 = tn * BN + (int)rank * 128;       // this CTA's half of B
+        const int n0 = ACT == 3 ? tn * 128 + (int)rank * p.Nd  // gate rows (leader) / up rows (peer)
+                                : tn * BN + (int)rank * 128;   // this CTA's half of B
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
@@ -283,13 +291,13 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       int tm, tn;
       tile_coords(p, tile, tm, tn);
       const int m0 = tm * (2 * BM) + (int)rank * BM;
-      const int n0 = tn * BN;
+      const int n0 = ACT == 3 ? tn * 128 : tn * BN;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int row0 = m0 + quarter * 32;
       const int row = row0 + lane;
       const bool row_ok = row < p.Md;
-      if (kb0 != 0 || kb1 != p.k_blocks) {
+      if (ACT == 0 && (kb0 != 0 || kb1 != p.k_blocks)) {
         // part of a split tile: park the accumulator; the last share to arrive stores the tile
         const float part_amax = pair_partial_share<OUT_F32>(
             p, &tmap_d, tile, kb0, pair, num_pairs, (int)rank, warp - 2,
@@ -302,7 +310,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         continue;
       }
 #pragma unroll 1
-      for (int c = 0; c < BN / CH; ++c) {
+      for (int c = 0; c < (ACT == 3 ? 128 : BN) / CH; ++c) {
         const int col0 = n0 + c * CH;
         if (col0 >= p.Nd) break;
         uint32_t r[CH];
@@ -311,6 +319,19 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         if (!OUT_F32) tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[CH - 32]));
         tmem_ld_wait();
         if (row0 >= p.Md) continue;
+        if (ACT == 3) {
+          // r holds 64 gate columns; fetch the matching up columns 32 at a time and combine in place
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t u[32];
+            tmem_ld32(taddr + 128 + 32 * h, u);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              r[32 * h + j] = __float_as_uint(swiglu(__fmul_rn(__uint_as_float(r[32 * h + j]), alpha),
+                                                     __fmul_rn(__uint_as_float(u[j]), alpha)));
+          }
+        }
         if (I8) {
           // int32 accumulators -> binary32, then the two Eq. 4 scales (row first, then column)
           const float ar = __fmul_rn(__ldg(p.row_scale + (p.row_scale_per_row ? min(row, p.Md - 1) : 0)), p.post_scale);
@@ -335,13 +356,19 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         } else {
           uint32_t packed[CH / 2];
 #pragma unroll
-          for (int j = 0; j < CH / 2; ++j)
-            packed[j] = f32x2_to_bf16x2(__fmul_rn(__uint_as_float(r[2 * j]), alpha),
-                                        __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha));
+          for (int j = 0; j < CH / 2; ++j) {
+            if (ACT == 3)
+              packed[j] = f32x2_to_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+            else
+              packed[j] = f32x2_to_bf16x2(act_apply<ACT>(__fmul_rn(__uint_as_float(r[2 * j]), alpha)),
+                                          act_apply<ACT>(__fmul_rn(__uint_as_float(r[2 * j + 1]), alpha)));
+          }
+          if (ACT == 0 || p.d != nullptr) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1],
-                         packed[4 * j + 2], packed[4 * j + 3]);
+            for (int j = 0; j < 8; ++j)
+              st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1],
+                           packed[4 * j + 2], packed[4 * j + 3]);
+          }
           if ((p.out_amax || p.out_q) && row_ok) {
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -371,7 +398,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) {
+        if (lane == 0 && (ACT == 0 || p.d != nullptr)) {
           if (OUT_F32 && p.accumulate) tma_reduce_add_2d(&tmap_d, col0, row0, buf);
           else tma_store_2d(&tmap_d, col0, row0, buf);
           bulk_commit();
