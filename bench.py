@@ -402,6 +402,59 @@ def int8_bench(torch, tw, peaks, reps=10):
     return out
 
 
+def act_norm_bench(torch, tw, peaks, reps=10):
+    """Activation-fused forward epilogue and FP8 LayerNorm at the benchmark's MLP shapes.  For each linear:
+    the plain forward product, the product with the activation in its epilogue (bf16 + FP8 out, FP8 only),
+    and the streaming passes the fusion removes (read bf16, write FP8) for scale.  LayerNorm: bytes moved
+    per element 2 read + 2 (bf16) and / or 1 (FP8) written."""
+    side = torch.cuda.Stream()
+    out = {"fwd_act": [], "layernorm": []}
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        return 1e3 * _time_replays(torch, _graph_of(torch, side, lambda: [fn() for _ in range(reps)]), 5) / reps
+
+    for name, act, M, K, N in (("cfg2_fc1_gelu", tw.ACT_GELU, 16384, 768, 3072),
+                               ("cfg2_fc1_gelu_tanh", tw.ACT_GELU_TANH, 16384, 768, 3072),
+                               ("cfg4_gate_up_swiglu", tw.ACT_SWIGLU, 8192, 2048, 5632)):
+        Nw = 2 * N if act == tw.ACT_SWIGLU else N
+        xq = torch.randint(0, 120, (M, K), device="cuda", dtype=torch.uint8)
+        wq = torch.randint(0, 120, (Nw, K), device="cuda", dtype=torch.uint8)
+        one = torch.full((1,), 1e-3, dtype=torch.float32, device="cuda")
+        qs = torch.full((1,), 4.0, dtype=torch.float32, device="cuda")
+        y_plain = torch.empty((M, Nw), dtype=torch.bfloat16, device="cuda")
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        yq = torch.empty((M, N), dtype=torch.uint8, device="cuda")
+        flops = 2.0 * M * K * Nw
+        us_plain = timed(lambda: tw.fp8_linear_fwd(xq, wq, one, one, y=y_plain))
+        us_both = timed(lambda: tw.fp8_linear_fwd_act(xq, wq, one, one, act, y=y, out_q=yq, q_scale=qs))
+        us_q = timed(lambda: tw.fp8_linear_fwd_act(xq, wq, one, one, act, want_y=False, out_q=yq, q_scale=qs))
+        out["fwd_act"].append({"case": name, "M": M, "K": K, "N_weight_rows": Nw, "us_plain_product": us_plain,
+                               "us_act_bf16_and_fp8": us_both, "us_act_fp8_only": us_q,
+                               "tflops_plain": flops / us_plain / 1e6, "tflops_act_fp8_only": flops / us_q / 1e6,
+                               "unfused_extra_pass_us_at_hbm_peak": (2.0 * M * Nw + 1.0 * M * N) / peaks["hbm"] / 1e3})
+        del xq, wq, y_plain, y, yq
+    for name, kind, rows, d in (("cfg2_ln_768", tw.NORM_LAYER, 16384 * 8, 768), ("cfg4_rms_2048", tw.NORM_RMS, 8192 * 8, 2048)):
+        x = torch.randn((rows, d), device="cuda").to(torch.bfloat16)
+        gamma = torch.ones(d, device="cuda")
+        beta = torch.zeros(d, device="cuda") if kind == tw.NORM_LAYER else None
+        qs = torch.full((1,), 64.0, dtype=torch.float32, device="cuda")
+        y = torch.empty_like(x)
+        yq = torch.empty((rows, d), dtype=torch.uint8, device="cuda")
+        n = rows * d
+        for label, kw, bytes_per in (("bf16+fp8", dict(y=y, yq=yq, q_fmt=tw.E4M3, q_scale=qs), 5.0),
+                                     ("fp8_only", dict(want_y=False, yq=yq, q_fmt=tw.E4M3, q_scale=qs), 3.0),
+                                     ("bf16_only", dict(y=y), 4.0)):
+            us = timed(lambda: tw.layernorm_fp8(x, gamma, beta, 1e-5, kind, **kw))
+            out["layernorm"].append({"case": name, "rows": rows, "d": d, "outputs": label, "us": us,
+                                     "gbs": bytes_per * n / us / 1e3,
+                                     "frac_of_hbm_peak": bytes_per * n / us / 1e3 / peaks["hbm"]})
+        del x, y, yq
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -490,11 +543,12 @@ def run_cuda(args):
             del obs, o
             torch.cuda.empty_cache()
 
-    w8a8, block_rows, int8_rows = None, None, None
+    w8a8, block_rows, int8_rows, act_rows = None, None, None, None
     if world == 1 and not args.no_w8a8:
         w8a8 = w8a8_sweep(torch, tw, peaks)
         block_rows = block_output_bench(torch, tw, peaks)
         int8_rows = int8_bench(torch, tw, peaks)
+        act_rows = act_norm_bench(torch, tw, peaks)
         if tw.read_device_status() != 0:
             raise SystemExit("device status reports an expired wait")
 
@@ -523,6 +577,8 @@ def run_cuda(args):
             line["block_output_fused"] = block_rows
         if int8_rows:
             line["int8_absmax_path"] = int8_rows
+        if act_rows:
+            line["act_norm_path"] = act_rows
         if world == 1 and not args.no_cpu_baseline:
             f, t = oracle_sample_step(cfg_idx, args.cpu_rows)
             line["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",

@@ -185,8 +185,9 @@ TWEO_API tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const
  *   TWEO_ACT_SWIGLU     Y[m,n] = SiLU(Z[m,n]) * Z[m,N+n], n < N: wq holds 2N rows, the N
  *                       gate rows first, then the N up rows
  *   TWEO_ACT_NONE       Y = Z (the call forwards to tweo_fp8_linear_fwd; y required)
- * Y is evaluated in binary32 (the tanh form with the hardware tanh, relative error 2^-11)
- * and rounded once to bf16; the optional outputs of epi act on the rounded values exactly as
+ * Y is evaluated in binary32 (Phi through the Abramowitz-Stegun 7.1.26 approximation of erfc,
+ * absolute error 1.5e-7; the tanh form with the hardware tanh, relative error 2^-11) and
+ * rounded once to bf16; the optional outputs of epi act on the rounded values exactly as
  * in tweo_fp8_linear_fwd.  xq [M,K], wq [N,K] (SwiGLU: [2N,K]) codes; y [M,N] bf16, or NULL
  * when only the FP8 copy (epi->out_q) is wanted.  Shapes: M >= 1, N % 16 == 0, K % 16 == 0.
  * Errors: TWEO_ERR_INVALID_ARG (NULL pointers, bad enums, neither y nor epi->out_q),

@@ -408,6 +408,19 @@ bool make_out_map(CUtensorMap* map, void* base, int64_t cols, int64_t rows, int6
   return r == CUDA_SUCCESS;
 }
 
+// 2-D FP8 output [rows, cols] (one byte per element): boxes of {64 bytes, 32 rows}, 64-byte swizzle.
+bool make_q_map(CUtensorMap* map, void* base, int64_t cols, int64_t rows, int64_t ld) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld};
+  cuuint32_t box[2] = {64u, 32u};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 uint32_t make_idesc(int fmt_a, int fmt_b, bool a_mn, bool b_mn, int n, int m = BM) {
   // [4,6) accumulator format (1 = fp32)   [7,10) A format   [10,13) B format (0 = E4M3, 1 = E5M2)
   // [15] A major (1 = MN)   [16] B major   [17,23) N >> 3   [24,29) M >> 4
@@ -538,7 +551,7 @@ tweo_status_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CU
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, p));
+  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, md, p));
   count_launch();
   return check_launch("gemm_fp8_pair_kernel");
 }
@@ -605,13 +618,14 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
 #undef TWEO_DISPATCH
 }
 
-// Forward product with the MLP activation in the epilogue (pair kernel only; every tile whole).
+// Forward product with the MLP activation and / or the FP8 copy of the output in the epilogue (pair
+// kernel only; every tile whole; the FP8 copy staged through shared memory, hence 5 stages).
 template <int ACT>
-tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, GemmParams& p,
-                              cudaStream_t st) {
-  constexpr int STAGES = 6;
-  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
-  auto kern = gemm_fp8_pair_kernel<false, false, STAGES, false, false, ACT>;
+tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
+                              const CUtensorMap& mq, GemmParams& p, cudaStream_t st) {
+  constexpr int STAGES = 5;
+  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 4 * 2 * 32 * 64 + 1024 + 256;
+  auto kern = gemm_fp8_pair_kernel<false, false, STAGES, false, false, ACT, true>;
   static bool attr_done = false;
   if (!attr_done) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -641,7 +655,7 @@ tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, cons
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, p));
+  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, mq, p));
   count_launch();
   return check_launch("gemm_fp8_pair_kernel (activation epilogue)");
 }
@@ -656,9 +670,11 @@ tweo_status_t run_fwd_act(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8
   p.Nd = (int32_t)N;
   p.Kc = (int32_t)K;
   p.idesc = make_idesc(fmt_x, fmt_w, false, false, 256, 256);
-  CUtensorMap ma, mb, md;
+  CUtensorMap ma, mb, md, mq;
   // without a bf16 output the store is skipped; the map then describes the FP8 output's memory and is never used
   bool ok = p.d ? make_out_map(&md, p.d, N, M, p.ldd, false) : make_out_map(&md, p.out_q, N / 2, M, p.ldq / 2, false);
+  if (p.out_q) ok = ok && make_q_map(&mq, p.out_q, N, M, p.ldq);
+  else mq = md;
   ok = ok && make_map(&ma, xq, K, M, ldx, BM);
   ok = ok && make_map(&mb, wq, K, act == TWEO_ACT_SWIGLU ? 2 * N : N, ldw, 128);
   if (!ok) {
@@ -670,9 +686,10 @@ tweo_status_t run_fwd_act(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8
     count_launch();
   }
   switch (act) {
-    case TWEO_ACT_GELU: return launch_pair_act<1>(ma, mb, md, p, st);
-    case TWEO_ACT_GELU_TANH: return launch_pair_act<2>(ma, mb, md, p, st);
-    case TWEO_ACT_SWIGLU: return launch_pair_act<3>(ma, mb, md, p, st);
+    case TWEO_ACT_NONE: return launch_pair_act<0>(ma, mb, md, mq, p, st);
+    case TWEO_ACT_GELU: return launch_pair_act<1>(ma, mb, md, mq, p, st);
+    case TWEO_ACT_GELU_TANH: return launch_pair_act<2>(ma, mb, md, mq, p, st);
+    case TWEO_ACT_SWIGLU: return launch_pair_act<3>(ma, mb, md, mq, p, st);
     default: return TWEO_ERR_INVALID_ARG;
   }
 }
@@ -891,6 +908,8 @@ tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const ui
   p.sb_inv = sw_inv;
   tweo_status_t s = fill_epilogue(p, epi);
   if (s != TWEO_OK) return s;
+  if (fused && M > 128 && N > 128 && !g_disable_pair)  // extra outputs leave through shared memory and TMA
+    return run_fwd_act(xq, ldx, fmt_x, wq, ldw, fmt_w, TWEO_ACT_NONE, M, N, K, p, st);
   return run_gemm(Operand{xq, ldx, fmt_x, false}, Operand{wq, ldw, fmt_w, false}, M, N, K, p, ws, ws_bytes, st);
 }
 
@@ -1051,7 +1070,7 @@ tweo_status_t tweo_int8_linear(const int8_t* xq, int64_t ldx, const float* sx, i
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, p));
+  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, md, p));
   count_launch();
   return check_launch("gemm_fp8_pair_kernel (int8)");
 }

@@ -152,10 +152,16 @@ __device__ __noinline__ float pair_partial_share(const GemmParams& p, const CUte
 // gate rows and its peer the matching 128 up rows, so accumulator columns [0,128) are the gate
 // and [128,256) the up projection of the same 128 output columns, and the tile that is stored
 // is 256 x 128: SiLU(gate) * up.  With p.d == nullptr only the FP8 copy / amax are produced.
-template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32, bool I8 = false, int ACT = 0>
+//
+// QST: the FP8 copy of the output leaves through shared memory and a TMA store (tmap_q: 64-byte
+// rows, 64-byte swizzle) like the bf16 tile, instead of 16-byte stores from registers that touch
+// 32 different rows per instruction.  Takes 16 KB of shared memory, so such kernels run with one
+// stage less in the operand ring.
+template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32, bool I8 = false, int ACT = 0, bool QST = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                     const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ GemmParams p) {
+                     const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ CUtensorMap tmap_q,
+                     const __grid_constant__ GemmParams p) {
   constexpr int BN = 256;                 // tile columns of the pair
   constexpr uint32_t A_BYTES = BM * BK;   // this CTA's 128 rows of A
   constexpr uint32_t B_BYTES = 128 * BK;  // this CTA's 128 of the 256 columns of B
@@ -166,8 +172,10 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   constexpr uint32_t EPI_BUF = 32 * 128;
   constexpr uint32_t EPI_BYTES = 4 * 2 * EPI_BUF;
+  constexpr uint32_t Q_BUF = 32 * 64;                       // 32 rows x 64 FP8 codes
+  constexpr uint32_t Q_BYTES = QST ? 4 * 2 * Q_BUF : 0;
   uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES + Q_BYTES);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -277,6 +285,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     const float qs = p.out_q ? __ldg(p.q_scale) : 0.0f;
     constexpr int CH = OUT_F32 ? 32 : 64;
     const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
+    const uint32_t q_base = smem_u32(epi_smem) + EPI_BYTES + (uint32_t)(warp - 2) * 2u * Q_BUF;
+    uint32_t amax2 = 0u;  // packed running maximum of |bf16| bit patterns (whole chunks)
     const uint32_t row_off = (uint32_t)lane * 128u;
     const uint32_t swz = (uint32_t)(lane & 7);
     const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
@@ -369,6 +379,37 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
               st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1],
                            packed[4 * j + 2], packed[4 * j + 3]);
           }
+          if (QST) {
+            // whole chunks inside the output take the packed integer maximum; ragged ones go element by element
+            if (p.out_amax && row_ok) {
+              if (col0 + CH <= p.Nd) {
+#pragma unroll
+                for (int j = 0; j < CH / 2; ++j) amax2 = absmax_bits(amax2, packed[j]);
+              } else {
+#pragma unroll
+                for (int j = 0; j < CH / 2; ++j) {
+                  if (col0 + 2 * j < p.Nd) run_amax = fmaxf(run_amax, fabsf(bf16lo_to_f32(packed[j])));
+                  if (col0 + 2 * j + 1 < p.Nd) run_amax = fmaxf(run_amax, fabsf(bf16hi_to_f32(packed[j])));
+                }
+              }
+            }
+            if (p.out_q) {
+              // 64 codes per row -> 32 rows x 64 B, 16-byte pieces XOR-swizzled with row bits 1-2
+              const uint32_t qbuf = q_base + (it & 1u) * Q_BUF;
+              const uint32_t qrow = qbuf + (uint32_t)lane * 64u;
+              const uint32_t qswz = ((uint32_t)lane >> 1) & 3u;
+#pragma unroll
+              for (int g4 = 0; g4 < 4; ++g4) {
+                uint32_t q[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const uint32_t w0 = packed[8 * g4 + 2 * j], w1 = packed[8 * g4 + 2 * j + 1];
+                  q[j] = p.q_fmt == TWEO_E4M3 ? quant_words<TWEO_E4M3>(w0, w1, qs) : quant_words<TWEO_E5M2>(w0, w1, qs);
+                }
+                st_shared_v4(qrow + (((uint32_t)g4 ^ qswz) << 4), q[0], q[1], q[2], q[3]);
+              }
+            }
+          } else
           if ((p.out_amax || p.out_q) && row_ok) {
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -398,9 +439,12 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0 && (ACT == 0 || p.d != nullptr)) {
-          if (OUT_F32 && p.accumulate) tma_reduce_add_2d(&tmap_d, col0, row0, buf);
-          else tma_store_2d(&tmap_d, col0, row0, buf);
+        if (lane == 0) {
+          if (ACT == 0 || p.d != nullptr) {
+            if (OUT_F32 && p.accumulate) tma_reduce_add_2d(&tmap_d, col0, row0, buf);
+            else tma_store_2d(&tmap_d, col0, row0, buf);
+          }
+          if (QST && p.out_q) tma_store_2d(&tmap_q, col0, row0, q_base + (it & 1u) * Q_BUF);
           bulk_commit();
         }
         ++it;
@@ -413,7 +457,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
     if (lane == 0) bulk_wait_all();
     if (p.out_amax) {
-      run_amax = warp_max(run_amax);
+      run_amax = warp_max(fmaxf(run_amax, __uint_as_float(absmax_fold(amax2) << 16)));
       if (lane == 0 && run_amax > 0.0f)
         atomicMax(reinterpret_cast<unsigned int*>(p.out_amax), __float_as_uint(run_amax));
     }

@@ -37,7 +37,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 constexpr int kNormThreads = 256;
 
-template <int VPL>
+// QFMT: -1 no FP8 output, else the tweo_fp8_t of the codes
+template <int VPL, int QFMT>
 __global__ void __launch_bounds__(kNormThreads) norm_rows_kernel(const NormArgs a) {
   extern __shared__ __align__(16) float gb[];  // gamma [d], beta [d]
   float* s_gamma = gb;
@@ -54,16 +55,41 @@ __global__ void __launch_bounds__(kNormThreads) norm_rows_kernel(const NormArgs 
   const int64_t warp_stride = (int64_t)gridDim.x * warps_per_cta;
   const int nvec = a.d >> 3;
   const float inv_d = 1.0f / (float)a.d;
-  const float qs = a.q ? __ldg(a.q_scale) : 0.0f;
+  const float qs = QFMT >= 0 ? __ldg(a.q_scale) : 0.0f;
   float run_amax = 0.0f;
 
-  for (int64_t row = warp_global; row < a.rows; row += warp_stride) {
-    const uint4* xr = reinterpret_cast<const uint4*>(a.x + row * a.ldx);
-    uint4 v[VPL];
+  // the next row's loads are issued before this row's reductions, so a warp always has a row in flight
+  constexpr bool PREFETCH = VPL <= 8;
+  uint4 nxt[PREFETCH ? VPL : 1];
+  if (PREFETCH && warp_global < a.rows) {
+    const uint4* xr = reinterpret_cast<const uint4*>(a.x + warp_global * a.ldx);
 #pragma unroll
     for (int i = 0; i < VPL; ++i) {
       const int idx = lane + 32 * i;
-      v[i] = idx < nvec ? __ldcs(xr + idx) : make_uint4(0u, 0u, 0u, 0u);
+      nxt[i] = idx < nvec ? __ldcs(xr + idx) : make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+  for (int64_t row = warp_global; row < a.rows; row += warp_stride) {
+    uint4 v[VPL];
+    if (PREFETCH) {
+#pragma unroll
+      for (int i = 0; i < VPL; ++i) v[i] = nxt[i];
+      const int64_t nrow = row + warp_stride;
+      if (nrow < a.rows) {
+        const uint4* xn = reinterpret_cast<const uint4*>(a.x + nrow * a.ldx);
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) {
+          const int idx = lane + 32 * i;
+          nxt[i] = idx < nvec ? __ldcs(xn + idx) : make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+    } else {
+      const uint4* xr = reinterpret_cast<const uint4*>(a.x + row * a.ldx);
+#pragma unroll
+      for (int i = 0; i < VPL; ++i) {
+        const int idx = lane + 32 * i;
+        v[i] = idx < nvec ? __ldcs(xr + idx) : make_uint4(0u, 0u, 0u, 0u);
+      }
     }
     float mu = 0.0f;
     if (!a.rms) {
@@ -114,25 +140,23 @@ __global__ void __launch_bounds__(kNormThreads) norm_rows_kernel(const NormArgs 
           o[k] = f32x2_to_bf16x2(y0, y1);
         }
         if (a.y) __stcs(reinterpret_cast<uint4*>(a.y + row * a.ldy) + idx, make_uint4(o[0], o[1], o[2], o[3]));
-        if (a.q || a.amax) {
+        if (QFMT >= 0 || a.amax) {
           float f[8];
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             f[2 * k] = bf16lo_to_f32(o[k]);
             f[2 * k + 1] = bf16hi_to_f32(o[k]);
           }
+          if (a.amax) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) run_amax = fmaxf(run_amax, fabsf(f[k]));
-          if (a.q) {
-            uint2 c;
-            if (a.q_fmt == TWEO_E4M3) {
-              c.x = cvt_fp8x2<TWEO_E4M3>(__fmul_rn(f[0], qs), __fmul_rn(f[1], qs)) | (cvt_fp8x2<TWEO_E4M3>(__fmul_rn(f[2], qs), __fmul_rn(f[3], qs)) << 16);
-              c.y = cvt_fp8x2<TWEO_E4M3>(__fmul_rn(f[4], qs), __fmul_rn(f[5], qs)) | (cvt_fp8x2<TWEO_E4M3>(__fmul_rn(f[6], qs), __fmul_rn(f[7], qs)) << 16);
-            } else {
-              c.x = cvt_fp8x2<TWEO_E5M2>(__fmul_rn(f[0], qs), __fmul_rn(f[1], qs)) | (cvt_fp8x2<TWEO_E5M2>(__fmul_rn(f[2], qs), __fmul_rn(f[3], qs)) << 16);
-              c.y = cvt_fp8x2<TWEO_E5M2>(__fmul_rn(f[4], qs), __fmul_rn(f[5], qs)) | (cvt_fp8x2<TWEO_E5M2>(__fmul_rn(f[6], qs), __fmul_rn(f[7], qs)) << 16);
-            }
-            __stcs(reinterpret_cast<uint2*>(a.q + row * a.ldq) + idx, c);
+            for (int k = 0; k < 8; ++k) run_amax = fmaxf(run_amax, fabsf(f[k]));
+          }
+          if (QFMT >= 0) {
+            uint32_t c[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)  // NaN -> 0x7F inside cvt_fp8x2
+              c[k] = cvt_fp8x2<QFMT >= 0 ? QFMT : 0>(__fmul_rn(f[2 * k], qs), __fmul_rn(f[2 * k + 1], qs));
+            __stcs(reinterpret_cast<uint2*>(a.q + row * a.ldq) + idx, make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16)));
           }
         }
       }
@@ -144,16 +168,29 @@ __global__ void __launch_bounds__(kNormThreads) norm_rows_kernel(const NormArgs 
   }
 }
 
-template <int VPL>
-cudaError_t launch_norm(const NormArgs& a, int grid, size_t smem, cudaStream_t st) {
+template <int VPL, int QFMT>
+cudaError_t launch_norm_q(const NormArgs& a, int64_t want_ctas, size_t smem, cudaStream_t st) {
   static bool attr_done = false;
   if (!attr_done) {  // gamma and beta of the widest row take 64 KB
-    cudaError_t e = cudaFuncSetAttribute(norm_rows_kernel<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
+    cudaError_t e = cudaFuncSetAttribute(norm_rows_kernel<VPL, QFMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  norm_rows_kernel<VPL><<<grid, kNormThreads, smem, st>>>(a);
+  // persistent grid: as many CTAs as are resident at once
+  int per_sm = 0;
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, norm_rows_kernel<VPL, QFMT>, kNormThreads, smem);
+  if (e != cudaSuccess) return e;
+  const int64_t cap = (int64_t)tweo_detail::sm_count() * (per_sm > 0 ? per_sm : 1);
+  const int grid = (int)(want_ctas < cap ? want_ctas : cap);
+  norm_rows_kernel<VPL, QFMT><<<grid, kNormThreads, smem, st>>>(a);
   return cudaGetLastError();
+}
+
+template <int VPL>
+cudaError_t launch_norm(const NormArgs& a, int64_t want_ctas, size_t smem, cudaStream_t st) {
+  if (!a.q) return launch_norm_q<VPL, -1>(a, want_ctas, smem, st);
+  if (a.q_fmt == TWEO_E4M3) return launch_norm_q<VPL, TWEO_E4M3>(a, want_ctas, smem, st);
+  return launch_norm_q<VPL, TWEO_E5M2>(a, want_ctas, smem, st);
 }
 
 }  // namespace
@@ -198,8 +235,7 @@ extern "C" tweo_status_t tweo_layernorm_fp8(const uint16_t* x, int64_t ldx, int6
   a.eps = eps;
   const int warps_per_cta = kNormThreads / 32;
   const int64_t want = (rows + warps_per_cta - 1) / warps_per_cta;
-  const int64_t cap = (int64_t)tweo_detail::sm_count() * 8;
-  const int grid = (int)(want < cap ? want : cap);
+  const int64_t grid = want;
   const size_t smem = (size_t)d * 2 * sizeof(float);
   const int vpl = (int)((d / 8 + 31) / 32);
   cudaError_t e;
