@@ -504,3 +504,58 @@ double oracle_activation(double v, int kind) {
 void oracle_activation_array(const double* v, int64_t n, int kind, double* out) {
   for (int64_t i = 0; i < n; ++i) out[i] = oracle_activation(v[i], kind);
 }
+
+/* ------------------------------------------------------------------ 8-bit residual stream */
+/* Sec. 4.4 quantises the residual stream too: in y = x + f(x) both the stream x and the
+ * block's branch f(x) are Eq. 4 codes with static per-tensor scales, and so is y -- no
+ * bf16 tensor in between.  As in oracle_absmax_quantize_bf16 everything is binary32, each
+ * operation rounded once, so the integer codes can be compared bit for bit:
+ *   x_i = fl32(xq_i * fl32(sx / Q_b)),  f_i = fl32(fq_i * fl32(sf / Q_b))     Eq. 4, dequantised
+ *   y_i = fl32(x_i + f_i)
+ *   yq_i = clamp(rne_int(fl32(y_i * fl32(Q_b / sy))), -Q_b, Q_b)              Eq. 4 with the static sy */
+void oracle_residual_add_q8(const int8_t* xq, const int8_t* fq, int64_t n, int bits, float sx, float sf, float sy,
+                            int8_t* yq) {
+  const float Q = (float)oracle_absmax_qmax(bits);
+  volatile float cx = sx / Q, cf = sf / Q, cy = Q / sy;
+  for (int64_t i = 0; i < n; ++i) {
+    volatile float x = (float)xq[i] * cx;
+    volatile float f = (float)fq[i] * cf;
+    volatile float y = x + f;
+    volatile float t = y * cy;
+    float r = nearbyintf(t);
+    if (r > Q) r = Q;
+    if (r < -Q) r = -Q;
+    yq[i] = (t != t) ? 0 : (int8_t)r;
+  }
+}
+
+/* The 8-bit linear whose output is requantised with a static per-tensor scale (Sec. 4.4:
+ * W8A8 with the activation scales fixed beforehand), at sampled points, in the binary32
+ * order an integer-tensor-core epilogue uses so the codes compare bit for bit:
+ *   acc  = sum_k Xq_mk Wq_nk                       (exact integer)
+ *   y    = fl32( fl32( fl32(acc) * fl32(sx_m * fl32(1 / Q_b^2)) ) * sw_n )
+ *   yq   = clamp(rne_int(fl32(y * fl32(Q_b / sy))), -Q_b, Q_b)
+ * y equals oracle_int8_gemm_at's FP64 value to binary32 rounding (checked in the tests). */
+void oracle_int8_gemm_q8_at(const int8_t* xq, int64_t ldx, const int8_t* wq, int64_t ldw, const float* sx,
+                            int sx_per_row, const float* sw, int sw_per_row, int bits, float sy, int64_t K,
+                            const int64_t* rows, const int64_t* cols, int64_t npts, int8_t* yq, float* y32) {
+  const float Q = (float)oracle_absmax_qmax(bits);
+  volatile float post = 1.0f / (Q * Q);
+  volatile float cy = Q / sy;
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < npts; ++t) {
+    const int64_t m = rows[t], n = cols[t];
+    int64_t acc = 0;
+    for (int64_t k = 0; k < K; ++k) acc += (int64_t)xq[m * ldx + k] * (int64_t)wq[n * ldw + k];
+    volatile float ar = sx[sx_per_row ? m : 0] * post;
+    volatile float a = (float)(int32_t)acc; /* the tensor core's int32 accumulator, converted round-to-nearest */
+    volatile float b = a * ar;
+    volatile float y = b * sw[sw_per_row ? n : 0];
+    volatile float u = y * cy;
+    float r = nearbyintf(u);
+    if (r > Q) r = Q;
+    if (r < -Q) r = -Q;
+    yq[t] = (u != u) ? 0 : (int8_t)r;
+    if (y32) y32[t] = y;
+  }
+}

@@ -105,6 +105,13 @@ def lib():
             L.oracle_activation.argtypes = [C.c_double, C.c_int]
             L.oracle_activation_array.restype = None
             L.oracle_activation_array.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p]
+            L.oracle_residual_add_q8.restype = None
+            L.oracle_residual_add_q8.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_float, C.c_float,
+                                                 C.c_float, C.c_void_p]
+            L.oracle_int8_gemm_q8_at.restype = None
+            L.oracle_int8_gemm_q8_at.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int,
+                                                 C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_int64, C.c_void_p,
+                                                 C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
             _lib = L
     return _lib
 
@@ -406,3 +413,33 @@ def gemm_fwd_act_at(xq, fmt_x, wq, fmt_w, sx_inv, sw_inv, kind: int, rows, cols)
         up = gemm_fwd_at(xq, fmt_x, wq, fmt_w, sx_inv, sw_inv, rows, cols + F)
         return activation(gate, ACT_SILU) * up
     return activation(gemm_fwd_at(xq, fmt_x, wq, fmt_w, sx_inv, sw_inv, rows, cols), kind)
+
+
+def residual_add_q8(xq, fq, bits: int, sx, sf, sy) -> np.ndarray:
+    """8-bit residual stream (Sec. 4.4): Eq. 4 codes of x + f(x) from the codes of x and f(x), static
+    per-tensor scales, binary32 arithmetic.  Returns int8 codes."""
+    xq = np.ascontiguousarray(xq, dtype=np.int8)
+    fq = np.ascontiguousarray(fq, dtype=np.int8)
+    assert xq.shape == fq.shape
+    yq = np.empty(xq.shape, dtype=np.int8)
+    lib().oracle_residual_add_q8(xq.ctypes.data, fq.ctypes.data, xq.size, bits, float(np.float32(sx)),
+                                 float(np.float32(sf)), float(np.float32(sy)), yq.ctypes.data)
+    return yq
+
+
+def int8_gemm_q8_at(xq, wq, sx, sw, bits: int, sy, rows, cols):
+    """The 8-bit linear with its output requantised by the static per-tensor scale sy, at the given points.
+    Returns (codes int8, y float32): y is the binary32 value the code was taken from."""
+    xq = np.ascontiguousarray(xq, dtype=np.int8)
+    wq = np.ascontiguousarray(wq, dtype=np.int8)
+    sx = np.ascontiguousarray(sx, dtype=np.float32).reshape(-1)
+    sw = np.ascontiguousarray(sw, dtype=np.float32).reshape(-1)
+    assert sx.size in (1, xq.shape[0]) and sw.size in (1, wq.shape[0]) and xq.shape[1] == wq.shape[1]
+    rows, cols = _pts(rows, cols)
+    yq = np.empty(rows.size, dtype=np.int8)
+    y = np.empty(rows.size, dtype=np.float32)
+    lib().oracle_int8_gemm_q8_at(xq.ctypes.data, xq.shape[1], wq.ctypes.data, wq.shape[1], sx.ctypes.data,
+                                 1 if sx.size > 1 else 0, sw.ctypes.data, 1 if sw.size > 1 else 0, bits,
+                                 float(np.float32(sy)), xq.shape[1], rows.ctypes.data, cols.ctypes.data, rows.size,
+                                 yq.ctypes.data, y.ctypes.data)
+    return yq, y
