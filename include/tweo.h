@@ -400,6 +400,30 @@ TWEO_API tweo_status_t tweo_int8_linear(const int8_t* xq, int64_t ldx, const flo
                                int32_t bits, uint16_t* y, int64_t ldy, int64_t M, int64_t N, int64_t K,
                                void* stream);
 
+/*
+ * tweo_int8_linear_q8 -- tweo_int8_linear with the output requantised in the epilogue (Sec. 4.4: with the
+ * residual stream quantised too, a block's linear hands 8-bit codes to the next operation and no bf16
+ * tensor exists in between).  With y the binary32 value tweo_int8_linear would round to bf16,
+ *   yq[m,n] = clamp( rne_int( fl32(y * fl32(Q_b / *sy)) ), -Q_b, Q_b ),  NaN -> 0       (Eq. 4, static scale)
+ * sy: device float [1], the static per-tensor AbsMax scale of the output.  yq [M,N] int8, row pitch ldq a
+ * multiple of 16.  Other arguments, shapes and errors as tweo_int8_linear.
+ */
+TWEO_API tweo_status_t tweo_int8_linear_q8(const int8_t* xq, int64_t ldx, const float* sx, int32_t sx_per_row,
+                                  const int8_t* wq, int64_t ldw, const float* sw, int32_t sw_per_row,
+                                  int32_t bits, const float* sy, int8_t* yq, int64_t ldq, int64_t M, int64_t N,
+                                  int64_t K, void* stream);
+
+/*
+ * tweo_residual_add_q8 -- the residual addition y = x + f(x) on a quantised residual stream (Sec. 4.4):
+ * x, f(x) and y are Eq. 4 codes with static per-tensor scales, binary32 arithmetic, each step rounded once:
+ *   y_i  = fl32( fl32(xq_i * fl32(*sx / Q_b)) + fl32(fq_i * fl32(*sf / Q_b)) )
+ *   yq_i = clamp( rne_int( fl32(y_i * fl32(Q_b / *sy)) ), -Q_b, Q_b )
+ * xq, fq, yq: int8 [n], device, 16-byte aligned (yq may alias xq or fq); sx, sf, sy: device float [1].
+ * 2 <= bits <= 8.  Errors: TWEO_ERR_INVALID_ARG, TWEO_ERR_ALIGNMENT.
+ */
+TWEO_API tweo_status_t tweo_residual_add_q8(const int8_t* xq, const float* sx, const int8_t* fq, const float* sf,
+                                   int64_t n, int32_t bits, const float* sy, int8_t* yq, void* stream);
+
 /* ---------------------------------------------------------------- helpers */
 
 /* Bytes of workspace `op` needs for the given problem (n for QUANTIZE / LOSS is

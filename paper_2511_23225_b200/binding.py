@@ -29,7 +29,7 @@ EXPORTS = [
     "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_fwd_act",
     "tweo_layernorm_fp8", "tweo_fp8_linear_bwd_dgrad",
     "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
-    "tweo_block_output_fused", "tweo_delayed_scaling_update", "tweo_absmax_quantize", "tweo_int8_linear",
+    "tweo_block_output_fused", "tweo_delayed_scaling_update", "tweo_absmax_quantize", "tweo_int8_linear", "tweo_int8_linear_q8", "tweo_residual_add_q8",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
 ]
@@ -93,6 +93,8 @@ def lib() -> C.CDLL:
         L.tweo_delayed_scaling_update.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp]
         L.tweo_absmax_quantize.argtypes = [vp, i64, i64, i64, i32, i32, i32, f32, vp, vp, i64, vp, sz, vp]
         L.tweo_int8_linear.argtypes = [vp, i64, vp, i32, vp, i64, vp, i32, i32, vp, i64, i64, i64, i64, vp]
+        L.tweo_int8_linear_q8.argtypes = [vp, i64, vp, i32, vp, i64, vp, i32, i32, vp, vp, i64, i64, i64, i64, vp]
+        L.tweo_residual_add_q8.argtypes = [vp, vp, vp, vp, i64, i32, vp, vp, vp]
         L.tweo_w8a8_static_gemm.argtypes = [vp, i32, i64, vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, sz, vp]
         L.tweo_workspace_bytes.argtypes = [i32, i64, i64, i64]
         L.tweo_workspace_bytes.restype = sz
@@ -548,3 +550,33 @@ def int8_linear(xq, sx, wq, sw, bits=8, y=None):
                                   _dev(sw, torch.float32, "sw"), 1 if sw.numel() > 1 else 0, bits,
                                   _dev(y, torch.bfloat16, "y"), _rows(y, "y"), M, N, K, _stream()), "tweo_int8_linear")
     return y
+
+
+def int8_linear_q8(xq, sx, wq, sw, sy, bits=8, yq=None):
+    """tweo_int8_linear_q8: the integer linear with its output requantised by the static per-tensor scale sy
+    (Eq. 4) in the epilogue -> int8 codes [M, N]."""
+    M, K = xq.shape
+    N, K2 = wq.shape
+    if K != K2:
+        raise ValueError("inner dimensions differ")
+    if yq is None:
+        yq = torch.empty((M, N), dtype=torch.int8, device=xq.device)
+    _check(lib().tweo_int8_linear_q8(_dev(xq, torch.int8, "xq"), _rows(xq, "xq"), _dev(sx, torch.float32, "sx"),
+                                     1 if sx.numel() > 1 else 0, _dev(wq, torch.int8, "wq"), _rows(wq, "wq"),
+                                     _dev(sw, torch.float32, "sw"), 1 if sw.numel() > 1 else 0, bits,
+                                     _dev(sy, torch.float32, "sy"), _dev(yq, torch.int8, "yq"), _rows(yq, "yq"),
+                                     M, N, K, _stream()), "tweo_int8_linear_q8")
+    return yq
+
+
+def residual_add_q8(xq, sx, fq, sf, sy, bits=8, yq=None):
+    """tweo_residual_add_q8: Eq. 4 codes (static scale sy) of x + f(x) from the codes of x (scale sx) and f(x) (sf)."""
+    if xq.shape != fq.shape or not xq.is_contiguous() or not fq.is_contiguous():
+        raise ValueError("xq and fq must be contiguous and of equal shape")
+    if yq is None:
+        yq = torch.empty_like(xq)
+    _check(lib().tweo_residual_add_q8(_dev(xq, torch.int8, "xq"), _dev(sx, torch.float32, "sx"),
+                                      _dev(fq, torch.int8, "fq"), _dev(sf, torch.float32, "sf"), xq.numel(), bits,
+                                      _dev(sy, torch.float32, "sy"), _dev(yq, torch.int8, "yq"), _stream()),
+           "tweo_residual_add_q8")
+    return yq

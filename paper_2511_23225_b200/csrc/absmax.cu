@@ -188,3 +188,75 @@ extern "C" tweo_status_t tweo_absmax_quantize(const uint16_t* x, int64_t rows, i
   count_launch();
   return check_launch("absmax_tensor_kernel");
 }
+
+// ------------------------------------------------------------------ 8-bit residual stream (Sec. 4.4)
+// yq = Eq. 4 codes (static scale sy) of  xq * (sx / Q) + fq * (sf / Q): 2 bytes read and 1 written per
+// element, 16 codes per 16-byte vector, four vectors of each input in flight per thread.
+namespace {
+
+__device__ __forceinline__ float code_to_f32(uint32_t w, int e) { return (float)(int)(int8_t)(w >> (8 * e)); }
+
+__device__ __forceinline__ uint32_t add4_q8(uint32_t xw, uint32_t fw, float cx, float cf, float cy, float Q) {
+  uint32_t out = 0u;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float y = __fadd_rn(__fmul_rn(code_to_f32(xw, e), cx), __fmul_rn(code_to_f32(fw, e), cf));
+    out |= ((uint32_t)quant1(y, cy, Q) & 0xFFu) << (8 * e);
+  }
+  return out;
+}
+
+__global__ void __launch_bounds__(256) residual_add_q8_kernel(const int8_t* __restrict__ xq, const int8_t* __restrict__ fq,
+                                                              int8_t* __restrict__ yq, int64_t n, float Q,
+                                                              const float* __restrict__ sx, const float* __restrict__ sf,
+                                                              const float* __restrict__ sy) {
+  const float cx = __fdiv_rn(__ldg(sx), Q), cf = __fdiv_rn(__ldg(sf), Q), cy = __fdiv_rn(Q, __ldg(sy));
+  const int64_t nvec = n >> 4;
+  const uint4* xv = reinterpret_cast<const uint4*>(xq);
+  const uint4* fv = reinterpret_cast<const uint4*>(fq);
+  uint4* yv = reinterpret_cast<uint4*>(yq);
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (; i + 3 * stride < nvec; i += 4 * stride) {
+    uint4 a[4], b[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      a[u] = __ldcs(xv + i + u * stride);
+      b[u] = __ldcs(fv + i + u * stride);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      __stcs(yv + i + u * stride, make_uint4(add4_q8(a[u].x, b[u].x, cx, cf, cy, Q), add4_q8(a[u].y, b[u].y, cx, cf, cy, Q),
+                                             add4_q8(a[u].z, b[u].z, cx, cf, cy, Q), add4_q8(a[u].w, b[u].w, cx, cf, cy, Q)));
+  }
+  for (; i < nvec; i += stride) {
+    const uint4 a = __ldcs(xv + i), b = __ldcs(fv + i);
+    __stcs(yv + i, make_uint4(add4_q8(a.x, b.x, cx, cf, cy, Q), add4_q8(a.y, b.y, cx, cf, cy, Q),
+                              add4_q8(a.z, b.z, cx, cf, cy, Q), add4_q8(a.w, b.w, cx, cf, cy, Q)));
+  }
+  // ragged tail (n % 16 codes) by the first threads of the grid
+  const int64_t t = (nvec << 4) + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n) {
+    const float y = __fadd_rn(__fmul_rn((float)xq[t], cx), __fmul_rn((float)fq[t], cf));
+    yq[t] = (int8_t)quant1(y, cy, Q);
+  }
+}
+
+}  // namespace
+
+extern "C" tweo_status_t tweo_residual_add_q8(const int8_t* xq, const float* sx, const int8_t* fq, const float* sf,
+                                              int64_t n, int32_t bits, const float* sy, int8_t* yq, void* stream) {
+  if (n < 0 || bits < 2 || bits > 8 || !sx || !sf || !sy) return TWEO_ERR_INVALID_ARG;
+  if (n == 0) return TWEO_OK;
+  if (!xq || !fq || !yq) return TWEO_ERR_INVALID_ARG;
+  if (!tweo_detail::aligned16(xq) || !tweo_detail::aligned16(fq) || !tweo_detail::aligned16(yq)) return TWEO_ERR_ALIGNMENT;
+  const float Q = (float)((1 << (bits - 1)) - 1);
+  const int64_t nvec = n >> 4;
+  const int64_t want = (nvec + 4 * 256 - 1) / (4 * 256);
+  const int64_t cap = (int64_t)tweo_detail::sm_count() * 8;
+  int grid = (int)(want < cap ? want : cap);
+  if (grid < 1) grid = 1;
+  residual_add_q8_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(xq, fq, yq, n, Q, sx, sf, sy);
+  tweo_detail::count_launch();
+  return tweo_detail::check_launch("residual_add_q8_kernel");
+}

@@ -913,6 +913,82 @@ tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const ui
   return run_gemm(Operand{xq, ldx, fmt_x, false}, Operand{wq, ldw, fmt_w, false}, M, N, K, p, ws, ws_bytes, st);
 }
 
+// The integer (Eq. 4) linear on the pair kernel: bf16 output (y), or 8-bit output requantised with the
+// static scale *sy (yq) -- exactly one of the two.
+tweo_status_t run_int8_linear(const int8_t* xq, int64_t ldx, const float* sx, int32_t sx_per_row, const int8_t* wq,
+                              int64_t ldw, const float* sw, int32_t sw_per_row, int32_t bits, uint16_t* y, int64_t ldy,
+                              int8_t* yq, int64_t ldq, const float* sy, int64_t M, int64_t N, int64_t K,
+                              cudaStream_t stream) {
+  if (!xq || !wq || !sx || !sw || bits < 2 || bits > 8) return TWEO_ERR_INVALID_ARG;
+  if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
+  if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(xq) || !aligned16(wq) || (ldx & 15) || (ldw & 15)) return TWEO_ERR_ALIGNMENT;
+  if (y && (!aligned16(y) || (ldy & 7))) return TWEO_ERR_ALIGNMENT;
+  if (yq && (!aligned16(yq) || (ldq & 15))) return TWEO_ERR_ALIGNMENT;
+  const bool q8 = yq != nullptr;
+  constexpr size_t smem6 = (size_t)6 * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
+  constexpr size_t smem5q = (size_t)5 * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 4 * 2 * 32 * 64 + 1024 + 256;
+  auto kern_bf16 = gemm_fp8_pair_kernel<false, false, 6, false, true>;
+  auto kern_q8 = gemm_fp8_pair_kernel<false, false, 5, false, true, 0, true>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    TWEO_CUDA_TRY(cudaFuncSetAttribute(kern_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem6));
+    TWEO_CUDA_TRY(cudaFuncSetAttribute(kern_q8, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem5q));
+    attr_done = true;
+  }
+  GemmParams p{};
+  p.d = y;
+  p.ldd = ldy;
+  p.Md = (int32_t)M;
+  p.Nd = (int32_t)N;
+  p.Kc = (int32_t)K;
+  p.tiles_m = (int32_t)((M + 2 * BM - 1) / (2 * BM));
+  p.tiles_n = (int32_t)((N + 255) / 256);
+  p.k_blocks = (int32_t)((K + BK - 1) / BK);
+  const int tiles = p.tiles_m * p.tiles_n;
+  int pairs = sm_count() / 2;
+  p.raster_g = raster_band(p.tiles_m, pairs);
+  if (pairs > tiles) pairs = tiles;
+  const float Q = (float)((1 << (bits - 1)) - 1);
+  p.row_scale = sx;
+  p.col_scale = sw;
+  p.row_scale_per_row = sx_per_row ? 1 : 0;
+  p.col_scale_per_col = sw_per_row ? 1 : 0;
+  p.post_scale = 1.0f / (Q * Q);
+  p.q8_qmax = Q;
+  if (q8) {
+    p.out_q = reinterpret_cast<uint8_t*>(yq);
+    p.ldq = ldq;
+    p.q_scale = sy;
+  }
+  // instruction descriptor of kind::i8: int32 accumulators, signed 8-bit A and B, K-major, N = 256, M = 256
+  p.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+  CUtensorMap ma, mb, md;
+  bool ok = q8 ? make_q_map(&md, yq, N, M, ldq) : make_out_map(&md, y, N, M, ldy, false);
+  ok = ok && make_map(&ma, xq, K, M, ldx, BM) && make_map(&mb, wq, K, N, ldw, 128);
+  if (!ok) {
+    cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return TWEO_ERR_CUDA;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = q8 ? smem5q : smem6;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (q8) TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern_q8, ma, mb, md, md, p));   // md doubles as the 8-bit output map
+  else TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern_bf16, ma, mb, md, md, p));
+  count_launch();
+  return check_launch("gemm_fp8_pair_kernel (int8)");
+}
+
 }  // namespace tweo_detail
 
 extern "C" {
@@ -1018,61 +1094,17 @@ tweo_status_t tweo_fp8_linear_bwd(const uint8_t* dyq, int64_t lddy, int32_t fmt_
 tweo_status_t tweo_int8_linear(const int8_t* xq, int64_t ldx, const float* sx, int32_t sx_per_row, const int8_t* wq,
                                int64_t ldw, const float* sw, int32_t sw_per_row, int32_t bits, uint16_t* y, int64_t ldy,
                                int64_t M, int64_t N, int64_t K, void* stream) {
-  using namespace tweo_detail;
-  if (!xq || !wq || !sx || !sw || !y || bits < 2 || bits > 8) return TWEO_ERR_INVALID_ARG;
-  if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
-  if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
-  if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
-  if (!aligned16(xq) || !aligned16(wq) || !aligned16(y) || (ldx & 15) || (ldw & 15) || (ldy & 7)) return TWEO_ERR_ALIGNMENT;
-  constexpr int STAGES = 6;
-  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
-  auto kern = gemm_fp8_pair_kernel<false, false, STAGES, false, true>;
-  static bool attr_done = false;
-  if (!attr_done) {
-    TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_done = true;
-  }
-  GemmParams p{};
-  p.d = y;
-  p.ldd = ldy;
-  p.Md = (int32_t)M;
-  p.Nd = (int32_t)N;
-  p.Kc = (int32_t)K;
-  p.tiles_m = (int32_t)((M + 2 * BM - 1) / (2 * BM));
-  p.tiles_n = (int32_t)((N + 255) / 256);
-  p.k_blocks = (int32_t)((K + BK - 1) / BK);
-  const int tiles = p.tiles_m * p.tiles_n;
-  int pairs = sm_count() / 2;
-  p.raster_g = raster_band(p.tiles_m, pairs);
-  if (pairs > tiles) pairs = tiles;
-  const float Q = (float)((1 << (bits - 1)) - 1);
-  p.row_scale = sx;
-  p.col_scale = sw;
-  p.row_scale_per_row = sx_per_row ? 1 : 0;
-  p.col_scale_per_col = sw_per_row ? 1 : 0;
-  p.post_scale = 1.0f / (Q * Q);
-  // instruction descriptor of kind::i8: int32 accumulators, signed 8-bit A and B, K-major, N = 256, M = 256
-  p.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-  CUtensorMap ma, mb, md;
-  if (!make_out_map(&md, y, N, M, ldy, false) || !make_map(&ma, xq, K, M, ldx, BM) || !make_map(&mb, wq, K, N, ldw, 128)) {
-    cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-    return TWEO_ERR_CUDA;
-  }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(2 * pairs));
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = (cudaStream_t)stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, md, p));
-  count_launch();
-  return check_launch("gemm_fp8_pair_kernel (int8)");
+  if (!y) return TWEO_ERR_INVALID_ARG;
+  return tweo_detail::run_int8_linear(xq, ldx, sx, sx_per_row, wq, ldw, sw, sw_per_row, bits, y, ldy, nullptr, 0,
+                                      nullptr, M, N, K, (cudaStream_t)stream);
+}
+
+tweo_status_t tweo_int8_linear_q8(const int8_t* xq, int64_t ldx, const float* sx, int32_t sx_per_row, const int8_t* wq,
+                                  int64_t ldw, const float* sw, int32_t sw_per_row, int32_t bits, const float* sy,
+                                  int8_t* yq, int64_t ldq, int64_t M, int64_t N, int64_t K, void* stream) {
+  if (!yq || !sy) return TWEO_ERR_INVALID_ARG;
+  return tweo_detail::run_int8_linear(xq, ldx, sx, sx_per_row, wq, ldw, sw, sw_per_row, bits, nullptr, 0, yq, ldq, sy,
+                                      M, N, K, (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -35,6 +35,7 @@ struct GemmParams {
   const float* col_scale;
   int32_t row_scale_per_row, col_scale_per_col;
   float post_scale;
+  float q8_qmax;           // Q_b of an 8-bit (Eq. 4) output; its static scale is read from q_scale
   // stream-K: tiles [0, sk_tiles) are split along the contraction, the rest dealt whole
   int32_t sk_tiles;
   float* sk_partials;   // [grid][BM*BN] raw accumulators of shares that do not own their tile

@@ -172,7 +172,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   constexpr uint32_t EPI_BUF = 32 * 128;
   constexpr uint32_t EPI_BYTES = 4 * 2 * EPI_BUF;
-  constexpr uint32_t Q_BUF = 32 * 64;                       // 32 rows x 64 FP8 codes
+  constexpr bool Q8 = I8 && QST;                            // integer linear with an 8-bit (Eq. 4) output only
+  constexpr uint32_t Q_BUF = 32 * 64;                       // 32 rows x 64 one-byte codes
   constexpr uint32_t Q_BYTES = QST ? 4 * 2 * Q_BUF : 0;
   uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES + Q_BYTES);
@@ -282,7 +283,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
     const int quarter = warp & 3;
     const float alpha = I8 ? 1.0f : __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
-    const float qs = p.out_q ? __ldg(p.q_scale) : 0.0f;
+    const float qs = p.out_q ? (Q8 ? __fdiv_rn(p.q8_qmax, __ldg(p.q_scale)) : __ldg(p.q_scale)) : 0.0f;
     constexpr int CH = OUT_F32 ? 32 : 64;
     const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
     const uint32_t q_base = smem_u32(epi_smem) + EPI_BYTES + (uint32_t)(warp - 2) * 2u * Q_BUF;
@@ -355,7 +356,27 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
         if (lane == 0) bulk_wait_read<1>();
         __syncwarp();
-        if (OUT_F32) {
+        if (Q8) {
+          // Eq. 4 with the static output scale on the binary32 results: clamp(rne_int(y * (Q_b / s))), NaN -> 0
+          const uint32_t qrow = q_base + (it & 1u) * Q_BUF + (uint32_t)lane * 64u;
+          const uint32_t qswz = ((uint32_t)lane >> 1) & 3u;
+          const int qmax = (int)p.q8_qmax;
+#pragma unroll
+          for (int g4 = 0; g4 < 4; ++g4) {
+            uint32_t q[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t w = 0u;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int c = max(-qmax, min(qmax, __float2int_rn(__fmul_rn(__uint_as_float(r[16 * g4 + 4 * j + e]), qs))));
+                w |= ((uint32_t)c & 0xFFu) << (8 * e);
+              }
+              q[j] = w;
+            }
+            st_shared_v4(qrow + (((uint32_t)g4 ^ qswz) << 4), q[0], q[1], q[2], q[3]);
+          }
+        } else if (OUT_F32) {
 #pragma unroll
           for (int j = 0; j < 8; ++j)
             st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4),
@@ -440,7 +461,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
-          if (ACT == 0 || p.d != nullptr) {
+          if (!Q8 && (ACT == 0 || p.d != nullptr)) {
             if (OUT_F32 && p.accumulate) tma_reduce_add_2d(&tmap_d, col0, row0, buf);
             else tma_store_2d(&tmap_d, col0, row0, buf);
           }
