@@ -455,6 +455,44 @@ def act_norm_bench(torch, tw, peaks, reps=10):
     return out
 
 
+def residual8_bench(torch, tw, peaks, reps=10):
+    """The 8-bit residual stream: the integer linear with 8-bit output against the one with bf16 output, and
+    the residual addition on codes (2 B read + 1 B written per element)."""
+    side = torch.cuda.Stream()
+    out = {"linear_q8": [], "residual_add_q8": []}
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        return 1e3 * _time_replays(torch, _graph_of(torch, side, lambda: [fn() for _ in range(reps)]), 5) / reps
+
+    one = torch.ones(1, dtype=torch.float32, device="cuda")
+    for M, K, N in ((8192, 4096, 4096), (8192, 4096, 11008)):
+        xq = torch.randint(-127, 128, (M, K), device="cuda", dtype=torch.int8)
+        wq = torch.randint(-127, 128, (N, K), device="cuda", dtype=torch.int8)
+        sy = torch.full((1,), 3e4, dtype=torch.float32, device="cuda")
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        yq = torch.empty((M, N), dtype=torch.int8, device="cuda")
+        us_bf16 = timed(lambda: tw.int8_linear(xq, one, wq, one, 8, y=y))
+        us_q8 = timed(lambda: tw.int8_linear_q8(xq, one, wq, one, sy, 8, yq=yq))
+        ops = 2.0 * M * K * N
+        out["linear_q8"].append({"M": M, "K": K, "N": N, "us_bf16_out": us_bf16, "us_int8_out": us_q8,
+                                 "tops_bf16_out": ops / us_bf16 / 1e6, "tops_int8_out": ops / us_q8 / 1e6,
+                                 "frac_of_2x_bf16_burst": ops / us_q8 / 1e6 / (2.0 * peaks["bf16"])})
+        del xq, wq, y, yq
+    for n in (8192 * 4096, 16 * 8192 * 4096):
+        xq = torch.randint(-127, 128, (n,), device="cuda", dtype=torch.int8)
+        fq = torch.randint(-127, 128, (n,), device="cuda", dtype=torch.int8)
+        yq = torch.empty_like(xq)
+        s = torch.full((1,), 2.0, dtype=torch.float32, device="cuda")
+        us = timed(lambda: tw.residual_add_q8(xq, s, fq, s, s, 8, yq=yq))
+        out["residual_add_q8"].append({"n": n, "us": us, "gbs": 3.0 * n / us / 1e3,
+                                       "frac_of_hbm_peak": 3.0 * n / us / 1e3 / peaks["hbm"]})
+        del xq, fq, yq
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -543,12 +581,13 @@ def run_cuda(args):
             del obs, o
             torch.cuda.empty_cache()
 
-    w8a8, block_rows, int8_rows, act_rows = None, None, None, None
+    w8a8, block_rows, int8_rows, act_rows, res8_rows = None, None, None, None, None
     if world == 1 and not args.no_w8a8:
         w8a8 = w8a8_sweep(torch, tw, peaks)
         block_rows = block_output_bench(torch, tw, peaks)
         int8_rows = int8_bench(torch, tw, peaks)
         act_rows = act_norm_bench(torch, tw, peaks)
+        res8_rows = residual8_bench(torch, tw, peaks)
         if tw.read_device_status() != 0:
             raise SystemExit("device status reports an expired wait")
 
@@ -579,6 +618,8 @@ def run_cuda(args):
             line["int8_absmax_path"] = int8_rows
         if act_rows:
             line["act_norm_path"] = act_rows
+        if res8_rows:
+            line["residual_stream_8bit"] = res8_rows
         if world == 1 and not args.no_cpu_baseline:
             f, t = oracle_sample_step(cfg_idx, args.cpu_rows)
             line["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",

@@ -415,9 +415,10 @@ TWEO_API tweo_status_t tweo_int8_linear_q8(const int8_t* xq, int64_t ldx, const 
 
 /*
  * tweo_residual_add_q8 -- the residual addition y = x + f(x) on a quantised residual stream (Sec. 4.4):
- * x, f(x) and y are Eq. 4 codes with static per-tensor scales, binary32 arithmetic, each step rounded once:
- *   y_i  = fl32( fl32(xq_i * fl32(*sx / Q_b)) + fl32(fq_i * fl32(*sf / Q_b)) )
- *   yq_i = clamp( rne_int( fl32(y_i * fl32(Q_b / *sy)) ), -Q_b, Q_b )
+ * x, f(x) and y are Eq. 4 codes with static per-tensor scales.  Dequantise, add, quantise; Q_b cancels:
+ *   a = fl32(*sx / *sy),  b = fl32(*sf / *sy)
+ *   yq_i = clamp( rne_int( fl32( fq_i * b + fl32(xq_i * a) ) ), -Q_b, Q_b ),  NaN -> 0
+ * (binary32: one product, one fused multiply-add).
  * xq, fq, yq: int8 [n], device, 16-byte aligned (yq may alias xq or fq); sx, sf, sy: device float [1].
  * 2 <= bits <= 8.  Errors: TWEO_ERR_INVALID_ARG, TWEO_ERR_ALIGNMENT.
  */

@@ -508,20 +508,21 @@ void oracle_activation_array(const double* v, int64_t n, int kind, double* out) 
 /* ------------------------------------------------------------------ 8-bit residual stream */
 /* Sec. 4.4 quantises the residual stream too: in y = x + f(x) both the stream x and the
  * block's branch f(x) are Eq. 4 codes with static per-tensor scales, and so is y -- no
- * bf16 tensor in between.  As in oracle_absmax_quantize_bf16 everything is binary32, each
- * operation rounded once, so the integer codes can be compared bit for bit:
- *   x_i = fl32(xq_i * fl32(sx / Q_b)),  f_i = fl32(fq_i * fl32(sf / Q_b))     Eq. 4, dequantised
- *   y_i = fl32(x_i + f_i)
- *   yq_i = clamp(rne_int(fl32(y_i * fl32(Q_b / sy))), -Q_b, Q_b)              Eq. 4 with the static sy */
+ * bf16 tensor in between.  Dequantising both inputs with Eq. 4, adding, and quantising the sum
+ * with Eq. 4 again, Q_b cancels:
+ *   y_q = clamp( round( (x_q s_x / Q_b + f_q s_f / Q_b) / s_y * Q_b ) ) = clamp( round( x_q (s_x / s_y) + f_q (s_f / s_y) ) ),
+ * one requantisation multiplier per input.  As in oracle_absmax_quantize_bf16 everything is
+ * binary32 so the integer codes can be compared bit for bit:
+ *   a = fl32(sx / sy),  b = fl32(sf / sy)                 (once per tensor)
+ *   t_i = fl32( fq_i * b + fl32(xq_i * a) )               (one product, one fused multiply-add)
+ *   yq_i = clamp(rne_int(t_i), -Q_b, Q_b),  NaN -> 0 */
 void oracle_residual_add_q8(const int8_t* xq, const int8_t* fq, int64_t n, int bits, float sx, float sf, float sy,
                             int8_t* yq) {
   const float Q = (float)oracle_absmax_qmax(bits);
-  volatile float cx = sx / Q, cf = sf / Q, cy = Q / sy;
+  volatile float a = sx / sy, b = sf / sy;
   for (int64_t i = 0; i < n; ++i) {
-    volatile float x = (float)xq[i] * cx;
-    volatile float f = (float)fq[i] * cf;
-    volatile float y = x + f;
-    volatile float t = y * cy;
+    volatile float p = (float)xq[i] * a;
+    volatile float t = fmaf((float)fq[i], b, p);
     float r = nearbyintf(t);
     if (r > Q) r = Q;
     if (r < -Q) r = -Q;

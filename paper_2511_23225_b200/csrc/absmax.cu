@@ -190,27 +190,31 @@ extern "C" tweo_status_t tweo_absmax_quantize(const uint16_t* x, int64_t rows, i
 }
 
 // ------------------------------------------------------------------ 8-bit residual stream (Sec. 4.4)
-// yq = Eq. 4 codes (static scale sy) of  xq * (sx / Q) + fq * (sf / Q): 2 bytes read and 1 written per
-// element, 16 codes per 16-byte vector, four vectors of each input in flight per thread.
+// yq = clamp(rne_int(xq * (sx / sy) + fq * (sf / sy))): Eq. 4 dequantise, add, Eq. 4 quantise with Q_b
+// cancelled.  2 bytes read and 1 written per element, 16 codes per 16-byte vector, four vectors of each
+// input in flight per thread; one product, one fused multiply-add and three conversions per element.
 namespace {
 
 __device__ __forceinline__ float code_to_f32(uint32_t w, int e) { return (float)(int)(int8_t)(w >> (8 * e)); }
 
-__device__ __forceinline__ uint32_t add4_q8(uint32_t xw, uint32_t fw, float cx, float cf, float cy, float Q) {
+__device__ __forceinline__ int add1_q8(float x, float f, float a, float b, int q) {
+  const int r = __float2int_rn(__fmaf_rn(f, b, __fmul_rn(x, a)));  // ties to even; NaN -> 0; saturates
+  return max(-q, min(q, r));
+}
+
+__device__ __forceinline__ uint32_t add4_q8(uint32_t xw, uint32_t fw, float a, float b, int q) {
   uint32_t out = 0u;
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const float y = __fadd_rn(__fmul_rn(code_to_f32(xw, e), cx), __fmul_rn(code_to_f32(fw, e), cf));
-    out |= ((uint32_t)quant1(y, cy, Q) & 0xFFu) << (8 * e);
-  }
+  for (int e = 0; e < 4; ++e) out |= ((uint32_t)add1_q8(code_to_f32(xw, e), code_to_f32(fw, e), a, b, q) & 0xFFu) << (8 * e);
   return out;
 }
 
-__global__ void __launch_bounds__(256) residual_add_q8_kernel(const int8_t* __restrict__ xq, const int8_t* __restrict__ fq,
-                                                              int8_t* __restrict__ yq, int64_t n, float Q,
+__global__ void __launch_bounds__(256) residual_add_q8_kernel(const int8_t* xq, const int8_t* fq,  // yq may alias either
+                                                              int8_t* yq, int64_t n, float Q,
                                                               const float* __restrict__ sx, const float* __restrict__ sf,
                                                               const float* __restrict__ sy) {
-  const float cx = __fdiv_rn(__ldg(sx), Q), cf = __fdiv_rn(__ldg(sf), Q), cy = __fdiv_rn(Q, __ldg(sy));
+  const float a = __fdiv_rn(__ldg(sx), __ldg(sy)), b = __fdiv_rn(__ldg(sf), __ldg(sy));
+  const int q = (int)Q;
   const int64_t nvec = n >> 4;
   const uint4* xv = reinterpret_cast<const uint4*>(xq);
   const uint4* fv = reinterpret_cast<const uint4*>(fq);
@@ -218,27 +222,26 @@ __global__ void __launch_bounds__(256) residual_add_q8_kernel(const int8_t* __re
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   for (; i + 3 * stride < nvec; i += 4 * stride) {
-    uint4 a[4], b[4];
+    uint4 va[4], vb[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      a[u] = __ldcs(xv + i + u * stride);
-      b[u] = __ldcs(fv + i + u * stride);
+      va[u] = __ldcs(xv + i + u * stride);
+      vb[u] = __ldcs(fv + i + u * stride);
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u)
-      __stcs(yv + i + u * stride, make_uint4(add4_q8(a[u].x, b[u].x, cx, cf, cy, Q), add4_q8(a[u].y, b[u].y, cx, cf, cy, Q),
-                                             add4_q8(a[u].z, b[u].z, cx, cf, cy, Q), add4_q8(a[u].w, b[u].w, cx, cf, cy, Q)));
+      __stcs(yv + i + u * stride, make_uint4(add4_q8(va[u].x, vb[u].x, a, b, q), add4_q8(va[u].y, vb[u].y, a, b, q),
+                                             add4_q8(va[u].z, vb[u].z, a, b, q), add4_q8(va[u].w, vb[u].w, a, b, q)));
   }
   for (; i < nvec; i += stride) {
-    const uint4 a = __ldcs(xv + i), b = __ldcs(fv + i);
-    __stcs(yv + i, make_uint4(add4_q8(a.x, b.x, cx, cf, cy, Q), add4_q8(a.y, b.y, cx, cf, cy, Q),
-                              add4_q8(a.z, b.z, cx, cf, cy, Q), add4_q8(a.w, b.w, cx, cf, cy, Q)));
+    const uint4 va = __ldcs(xv + i), vb = __ldcs(fv + i);
+    __stcs(yv + i, make_uint4(add4_q8(va.x, vb.x, a, b, q), add4_q8(va.y, vb.y, a, b, q),
+                              add4_q8(va.z, vb.z, a, b, q), add4_q8(va.w, vb.w, a, b, q)));
   }
   // ragged tail (n % 16 codes) by the first threads of the grid
   const int64_t t = (nvec << 4) + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (t < n) {
-    const float y = __fadd_rn(__fmul_rn((float)xq[t], cx), __fmul_rn((float)fq[t], cf));
-    yq[t] = (int8_t)quant1(y, cy, Q);
+    yq[t] = (int8_t)add1_q8((float)xq[t], (float)fq[t], a, b, q);
   }
 }
 
