@@ -255,7 +255,7 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams g) {
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's barrier
+      if (lane == 0) mbar_arrive_cluster_relaxed(map_to_cta(tempty_bar(acc), 0));  // the leader's barrier
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }

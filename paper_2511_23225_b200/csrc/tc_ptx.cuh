@@ -182,6 +182,14 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// The same arrival without release semantics, for handing an accumulator back to the MMA warp: the
+// epilogue's tcgen05.ld have completed (tcgen05.wait::ld) before it is issued, and nothing else the
+// epilogue wrote is read by the MMA warp, so there is nothing to publish.  The releasing form makes
+// the thread wait until its outstanding TMA stores have drained (measured: 1200-2800 cycles per tile,
+// half of the epilogue's time at contraction 768; this form: 34 cycles).
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1,
                                                  uint32_t leader_bar) {
   asm volatile(
