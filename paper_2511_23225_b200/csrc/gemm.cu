@@ -716,19 +716,12 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   p.sw_inv = sw_inv;
   const int sms = sm_count();
   const int slabs = (int)((N + 127) / 128);
+  // slices of K per slab = CTAs per cluster: as many as give every SM a CTA, a power of two up to the portable
+  // cluster size, at least four k-blocks each
   p.slices = 1;
-  if (ws && aligned16(ws) && ws_bytes >= kWsPartialsOffset + (size_t)sms * kWsPartialBytesPerSm && slabs <= 512) {
-    int s = sms / slabs;                             // one CTA per SM
-    if (s > p.k_blocks / 4) s = p.k_blocks / 4;      // at least four k-blocks per slice
-    // parking partial sums pays for a few tokens, or for a very long K
-    if (p.Mpad > 32) s = (p.k_blocks >= 64 && s >= 2) ? 2 : 1;
-    while (s > 1 && (size_t)slabs * s * p.Mpad * 128 * sizeof(float) > (size_t)sms * kWsPartialBytesPerSm) --s;
-    if (s > 1) {
-      p.slices = s;
-      p.counters = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + kWsCountersOffset);
-      p.partials = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + kWsPartialsOffset);
-    }
-  }
+  while (p.slices < 8 && slabs * p.slices * 2 <= sms && p.k_blocks / (p.slices * 2) >= 4) p.slices *= 2;
+  (void)ws;
+  (void)ws_bytes;
   CUtensorMap mw, mx;
   if (!make_map(&mw, wq, K, N, ldw, BM) || !make_map(&mx, xq, K, M, ldx, p.Mpad)) {
     cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
@@ -741,7 +734,19 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
                                        (int)(200 * 1024 + 1024 + 256)));
     attr_done = true;
   }
-  gemm_fp8_skinny_kernel<<<slabs * p.slices, kThreads, smem, st>>>(mw, mx, p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(slabs * p.slices));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)p.slices;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_fp8_skinny_kernel, mw, mx, p));
   count_launch();
   return check_launch("gemm_fp8_skinny_kernel");
 }

@@ -9,10 +9,12 @@
 // CTA = 192 threads: warp 0 issues TMA loads (W slab 128 x 128 B and X 'Mpad' x 128 B per
 // k-block, 128-byte swizzle, rows beyond M zero-filled), warp 1 owns tensor memory and issues
 // tcgen05.mma kind::f8f6f4 128 x Mpad x 32, warps 2-5 read the accumulator (lane = row of W =
-// output column) and write Y.  With K sliced, every CTA parks its fp32 partial sums in the
-// workspace ([column][token], a few KB), takes a ticket per (slab, warp), and the warp
-// that draws the last ticket adds the slices in slice order and stores -- nobody waits, and
-// the sum does not depend on timing.  All mbarrier waits are bounded.
+// output column) and write Y.  With K sliced, the slices of one slab form a thread-block cluster:
+// every CTA parks its fp32 partial sums in its own shared memory ([token][128 columns], in the
+// ring the loads no longer need), the cluster synchronises, and CTA r sums tokens r, r + S, ...
+// over all S slices in slice order through distributed shared memory and writes those rows of Y
+// (64 contiguous bytes per warp).  No workspace, no atomics, and the sum does not depend on
+// timing.  All mbarrier waits are bounded; the cluster barrier is reached by every thread.
 #pragma once
 
 #include <cuda.h>
@@ -29,16 +31,20 @@ struct SkinnyParams {
   int64_t ldy;
   int32_t M, N, Mpad;      // Mpad: M rounded up to a multiple of 16 (<= 128)
   int32_t k_blocks;        // ceil(K / 128)
-  int32_t slices;          // slices of K
+  int32_t slices;          // slices of K = CTAs per cluster (1, 2, 4 or 8)
   int32_t stages;          // TMA ring depth (<= kSkinnyMaxStages)
   uint32_t stage_bytes;    // 16 KB of W + Mpad * 128 B of X, rounded up to 1 KB
   uint32_t tmem_cols;      // power of two >= max(32, Mpad)
   uint32_t idesc;
   const float* sx_inv;
   const float* sw_inv;
-  float* partials;         // [slab][slice][128 columns][Mpad] fp32, used when slices > 1
-  uint32_t* counters;      // [slab][4] tickets, zero between launches
 };
+
+__device__ __forceinline__ float ld_shared_cluster_f32(uint32_t cluster_addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
+  return v;
+}
 
 // 32 lanes x 16 consecutive 32-bit columns of tensor memory
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -147,68 +153,55 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
           }
         }
       } else {
-        // park the partial sums: [column][token], a lane writes its column's tokens contiguously
-        const size_t unit_floats = (size_t)128 * p.Mpad;
-        float* mine = p.partials + (size_t)(slab * p.slices + slice) * unit_floats + (size_t)(quarter * 32 + lane) * p.Mpad;
+        // park the partial sums in this CTA's shared memory: [token][128 columns] fp32 (the operand ring is
+        // free: the accumulator-complete signal comes after the last MMA has read it)
+        const uint32_t park = smem_base + (uint32_t)(quarter * 32 + lane) * 4u;
         for (int c = 0; c < p.Mpad; c += 16) {
           uint32_t r[16];
           tmem_ld16(tacc + (uint32_t)c, r);
           tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 16; j += 4)
-            __stcg(reinterpret_cast<float4*>(mine + c + j),
-                   make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                               __uint_as_float(r[j + 3])));
-        }
-        __threadfence();
-        __syncwarp();
-        uint32_t ticket = 0;
-        uint32_t* counter = p.counters + slab * 4 + quarter;
-        if (lane == 0) ticket = atomicAdd(counter, 1u);
-        ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
-        if (ticket + 1 == (uint32_t)p.slices) {  // the last slice of this slab: add all slices in order
-          __threadfence();
-          if (lane == 0) *counter = 0u;  // ready for the next launch
-          const float* base = p.partials + (size_t)slab * p.slices * unit_floats + (size_t)(quarter * 32 + lane) * p.Mpad;
-          // 16 tokens of this column at a time, the loads of eight slices in flight together
-          // (32 independent 16-byte loads); the additions still run in slice order
-          for (int m = 0; m < p.M; m += 16) {
-            float4 acc[4];
-#pragma unroll 1
-            for (int s0 = 0; s0 < p.slices; s0 += 8) {
-              float4 v[8][4];
-#pragma unroll
-              for (int t = 0; t < 8; ++t) {
-                const float4* src = reinterpret_cast<const float4*>(base + (size_t)(s0 + t) * unit_floats + m);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) v[t][j] = (s0 + t < p.slices) ? __ldcg(src + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-              }
-#pragma unroll
-              for (int t = 0; t < 8; ++t) {
-                if (s0 + t < p.slices) {
-#pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    if (s0 + t == 0) acc[j] = v[t][j];
-                    else acc[j] = make_float4(acc[j].x + v[t][j].x, acc[j].y + v[t][j].y, acc[j].z + v[t][j].z,
-                                              acc[j].w + v[t][j].w);
-                  }
-                }
-              }
-            }
-            if (col < p.N) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const float a4[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if (m + 4 * j + e < p.M)
-                    p.y[(int64_t)(m + 4 * j + e) * p.ldy + col] = (uint16_t)f32_to_bf16_bits(__fmul_rn(a4[e], alpha));
-              }
-            }
-          }
+          for (int j = 0; j < 16; ++j)
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(park + (uint32_t)(c + j) * 512u), "r"(r[j]) : "memory");
         }
       }
     }
+  }
+
+  if (p.slices > 1) {
+    // every thread of every CTA of the cluster gets here, whatever happened above
+    cluster_sync_all();  // all partial sums are parked and visible
+    if (warp >= 2) {
+      const int quarter = warp & 3;
+      const int col = quarter * 32 + lane;
+      const int n = n0 + col;
+      const float alpha = __fmul_rn(__ldg(p.sx_inv), __ldg(p.sw_inv));
+      const uint32_t mine = smem_base + (uint32_t)col * 4u;
+      uint32_t peer[8];
+#pragma unroll
+      for (int sl = 0; sl < 8; ++sl) peer[sl] = map_to_cta(mine, (uint32_t)(sl < p.slices ? sl : 0));
+      // eight tokens at a time, so up to 64 remote loads are in flight per thread
+      for (int t0 = slice; t0 < p.M; t0 += 8 * p.slices) {
+        float v[8][8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int t = t0 + u * p.slices;
+#pragma unroll
+          for (int sl = 0; sl < 8; ++sl)
+            v[u][sl] = (sl < p.slices && t < p.M) ? ld_shared_cluster_f32(peer[sl] + (uint32_t)t * 512u) : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int t = t0 + u * p.slices;
+          float acc = v[u][0];
+#pragma unroll
+          for (int sl = 1; sl < 8; ++sl)
+            if (sl < p.slices) acc += v[u][sl];  // slice order
+          if (t < p.M && n < p.N) p.y[(int64_t)t * p.ldy + n] = (uint16_t)f32_to_bf16_bits(__fmul_rn(acc, alpha));
+        }
+      }
+    }
+    cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
   }
 
   tc_fence_before();
