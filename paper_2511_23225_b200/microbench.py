@@ -85,6 +85,14 @@ def make(op, M, K, N):
         one, sy = _scalar(1.0), _scalar(3e4)
         yq = torch.empty((M, N), dtype=torch.int8, device="cuda")
         return (lambda: tw.int8_linear_q8(xq, one, wq, one, sy, 8, yq=yq)), 2.0 * M * K * N, "TFLOP/s"
+    if op == "w8a8":          # static W8A8 forward product on already-cast activations (few tokens: the W-streaming kernel)
+        xq, wq = _codes((M, K), 1), _codes((N, K), 2)
+        one = _scalar(1.0)
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        ws = tw.new_workspace(tw.OP_W8A8, M, N, K)
+        if M <= 128:
+            return (lambda: tw.w8a8_static_gemm(xq, one, wq, one, y=y, ws=ws)), 1.0 * (M * K + N * K) + 2.0 * M * N, "GB/s"
+        return (lambda: tw.w8a8_static_gemm(xq, one, wq, one, y=y, ws=ws)), 2.0 * M * K * N, "TFLOP/s"
     if op == "residual_add_q8":
         xq, fq = _codes((M * K,), 1, True), _codes((M * K,), 2, True)
         yq = torch.empty_like(xq)
@@ -94,7 +102,7 @@ def make(op, M, K, N):
 
 
 OPS = ("quantize", "linear", "loss", "block_output", "layernorm", "fwd_gelu", "fwd_swiglu", "absmax", "int8_linear_q8",
-       "residual_add_q8")
+       "residual_add_q8", "w8a8")
 
 
 def main():
