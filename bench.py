@@ -493,6 +493,38 @@ def residual8_bench(torch, tw, peaks, reps=10):
     return out
 
 
+def vendor_fp8_context(torch, tw, reps=10):
+    """Context only, not a product path: the vendor library's FP8 GEMM (torch._scaled_mm) beside this
+    library's forward product on the same shapes, both replayed from a CUDA graph.  Omitted if the call is
+    not available in this torch build."""
+    side = torch.cuda.Stream()
+    out = []
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        return 1e3 * _time_replays(torch, _graph_of(torch, side, lambda: [fn() for _ in range(reps)]), 5) / reps
+
+    for name, M, K, N in (("cfg2_fc1", 8192, 768, 3072), ("cfg4_qkv", 16384, 2048, 6144), ("cfg5_M8192", 8192, 4096, 11008)):
+        try:
+            xq = torch.randint(0, 120, (M, K), device="cuda", dtype=torch.uint8)
+            wq = torch.randint(0, 120, (N, K), device="cuda", dtype=torch.uint8)
+            one = torch.ones(1, dtype=torch.float32, device="cuda")
+            y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            a8, b8 = xq.view(torch.float8_e4m3fn), wq.view(torch.float8_e4m3fn).t()
+            s1 = torch.ones((), dtype=torch.float32, device="cuda")
+            us_vendor = timed(lambda: torch._scaled_mm(a8, b8, scale_a=s1, scale_b=s1, out_dtype=torch.bfloat16))
+            us_ours = timed(lambda: tw.fp8_linear_fwd(xq, wq, one, one, y=y))
+            flops = 2.0 * M * K * N
+            out.append({"case": name, "M": M, "K": K, "N": N, "vendor_scaled_mm_tflops": flops / us_vendor / 1e6,
+                        "this_library_tflops": flops / us_ours / 1e6})
+            del xq, wq, y
+        except Exception as e:  # noqa: BLE001 -- context line only
+            out.append({"case": name, "unavailable": str(e)[:120]})
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -581,13 +613,14 @@ def run_cuda(args):
             del obs, o
             torch.cuda.empty_cache()
 
-    w8a8, block_rows, int8_rows, act_rows, res8_rows = None, None, None, None, None
+    w8a8, block_rows, int8_rows, act_rows, res8_rows, vendor_rows = None, None, None, None, None, None
     if world == 1 and not args.no_w8a8:
         w8a8 = w8a8_sweep(torch, tw, peaks)
         block_rows = block_output_bench(torch, tw, peaks)
         int8_rows = int8_bench(torch, tw, peaks)
         act_rows = act_norm_bench(torch, tw, peaks)
         res8_rows = residual8_bench(torch, tw, peaks)
+        vendor_rows = vendor_fp8_context(torch, tw)
         if tw.read_device_status() != 0:
             raise SystemExit("device status reports an expired wait")
 
@@ -620,6 +653,8 @@ def run_cuda(args):
             line["act_norm_path"] = act_rows
         if res8_rows:
             line["residual_stream_8bit"] = res8_rows
+        if vendor_rows:
+            line["context_vendor_fp8_gemm"] = vendor_rows
         if world == 1 and not args.no_cpu_baseline:
             f, t = oracle_sample_step(cfg_idx, args.cpu_rows)
             line["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
