@@ -560,3 +560,38 @@ void oracle_int8_gemm_q8_at(const int8_t* xq, int64_t ldx, const int8_t* wq, int
     if (y32) y32[t] = y;
   }
 }
+
+/* Per-token variant of the quantised residual stream (Sec. 4.4 reports both per-tensor "A8(T)" and
+ * per-token "A8(K)" activations with the residual quantised): every row (token) m of x and f(x) carries
+ * its own Eq. 4 scale sx[m], sf[m], and the sum gets the AbsMax scale of its own row,
+ *   y_mj  = fl32( fq_mj * fl32(sf[m] / Q_b) + fl32(xq_mj * fl32(sx[m] / Q_b)) )     dequantise and add
+ *   sy[m] = fl32( max_j |y_mj| + eps )                                              Eq. 4, per row
+ *   yq_mj = clamp( rne_int( fl32(y_mj * fl32(Q_b / sy[m])) ), -Q_b, Q_b )
+ * everything in binary32 as in oracle_absmax_quantize_bf16, so the codes compare bit for bit. */
+void oracle_residual_add_q8_rows(const int8_t* xq, const float* sx, const int8_t* fq, const float* sf, int64_t rows,
+                                 int64_t cols, int bits, float eps, int8_t* yq, float* sy) {
+  const float Q = (float)oracle_absmax_qmax(bits);
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < rows; ++m) {
+    volatile float cx = sx[m] / Q, cf = sf[m] / Q;
+    float amax = 0.0f;
+    for (int64_t j = 0; j < cols; ++j) {
+      volatile float p = (float)xq[m * cols + j] * cx;
+      volatile float y = fmaf((float)fq[m * cols + j], cf, p);
+      const float a = fabsf(y);
+      if (a > amax) amax = a; /* false for NaN */
+    }
+    volatile float s = amax + eps;
+    volatile float c = Q / s;
+    sy[m] = s;
+    for (int64_t j = 0; j < cols; ++j) {
+      volatile float p = (float)xq[m * cols + j] * cx;
+      volatile float y = fmaf((float)fq[m * cols + j], cf, p);
+      volatile float t = y * c;
+      float r = nearbyintf(t);
+      if (r > Q) r = Q;
+      if (r < -Q) r = -Q;
+      yq[m * cols + j] = (t != t) ? 0 : (int8_t)r;
+    }
+  }
+}

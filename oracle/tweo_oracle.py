@@ -112,6 +112,9 @@ def lib():
             L.oracle_int8_gemm_q8_at.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int,
                                                  C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_int64, C.c_void_p,
                                                  C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
+            L.oracle_residual_add_q8_rows.restype = None
+            L.oracle_residual_add_q8_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
+                                                      C.c_int, C.c_float, C.c_void_p, C.c_void_p]
             _lib = L
     return _lib
 
@@ -443,3 +446,19 @@ def int8_gemm_q8_at(xq, wq, sx, sw, bits: int, sy, rows, cols):
                                  float(np.float32(sy)), xq.shape[1], rows.ctypes.data, cols.ctypes.data, rows.size,
                                  yq.ctypes.data, y.ctypes.data)
     return yq, y
+
+
+def residual_add_q8_rows(xq, sx, fq, sf, bits: int, eps):
+    """Per-token 8-bit residual stream (Sec. 4.4, A8(K)): codes of x + f(x) with one AbsMax scale per row, from
+    the per-row codes of x and f(x).  Returns (codes int8 [rows, cols], sy float32 [rows])."""
+    xq = np.ascontiguousarray(xq, dtype=np.int8)
+    fq = np.ascontiguousarray(fq, dtype=np.int8)
+    assert xq.ndim == 2 and xq.shape == fq.shape
+    sx = np.ascontiguousarray(sx, dtype=np.float32).reshape(-1)
+    sf = np.ascontiguousarray(sf, dtype=np.float32).reshape(-1)
+    assert sx.size == xq.shape[0] and sf.size == xq.shape[0]
+    yq = np.empty(xq.shape, dtype=np.int8)
+    sy = np.empty(xq.shape[0], dtype=np.float32)
+    lib().oracle_residual_add_q8_rows(xq.ctypes.data, sx.ctypes.data, fq.ctypes.data, sf.ctypes.data, xq.shape[0],
+                                      xq.shape[1], bits, float(np.float32(eps)), yq.ctypes.data, sy.ctypes.data)
+    return yq, sy

@@ -97,3 +97,38 @@ def test_int8_linear_requantised_matches_fp64_chain(per_row):
     assert away.mean() > 0.99 and np.array_equal(codes[away].astype(np.int64), want[away].astype(np.int64))
     assert np.max(np.abs(codes.astype(np.int64) - want.astype(np.int64))) <= 1
     assert np.any(np.abs(codes) == Q) and np.any(np.abs(t) > Q)
+
+
+def test_per_token_residual_add_against_fp64_and_its_own_row_maximum():
+    """Per row: the FP64 statement of Eq. 4 on the dequantised sum (equal away from ties, <= 1 code at them); the
+    largest element of every row maps to +-Q_b; a row is independent of the other rows; with equal scales and
+    eps = 0 the codes are the integer sums rescaled by the row's largest sum."""
+    Q = 127
+    g = np.random.Generator(np.random.PCG64(23))
+    rows, cols = 37, 200
+    xq = g.integers(-Q, Q + 1, (rows, cols), dtype=np.int8)
+    fq = g.integers(-Q, Q + 1, (rows, cols), dtype=np.int8)
+    sx = (0.5 + 3.0 * g.random(rows)).astype(np.float32)
+    sf = (0.05 + 0.5 * g.random(rows)).astype(np.float32)
+    eps = 1e-6
+    yq, sy = orc.residual_add_q8_rows(xq, sx, fq, sf, 8, eps)
+    y64 = xq.astype(np.float64) * (sx.astype(np.float64)[:, None] / Q) + fq.astype(np.float64) * (sf.astype(np.float64)[:, None] / Q)
+    s64 = np.max(np.abs(y64), axis=1) + eps
+    assert np.allclose(sy, s64, rtol=3e-7)
+    t = y64 / s64[:, None] * Q
+    want = np.clip(np.rint(t), -Q, Q)
+    away = np.abs(np.abs(t - np.floor(t)) - 0.5) > 1e-3
+    assert away.mean() > 0.99 and np.array_equal(yq[away].astype(np.float64), want[away])
+    assert np.max(np.abs(yq.astype(np.float64) - want)) <= 1
+    assert np.all(np.max(np.abs(yq.astype(np.int64)), axis=1) == Q)                  # the row maximum takes the last code
+    one, s1 = orc.residual_add_q8_rows(xq[5:6], sx[5:6], fq[5:6], sf[5:6], 8, eps)   # rows do not see each other
+    assert np.array_equal(one[0], yq[5]) and s1[0] == sy[5]
+    same = np.full(rows, 2.0, dtype=np.float32)
+    zq, _ = orc.residual_add_q8_rows(xq, same, fq, same, 8, 0.0)
+    isum = xq.astype(np.int64) + fq.astype(np.int64)
+    want2 = np.rint(isum / np.max(np.abs(isum), axis=1, keepdims=True) * Q)
+    ties = np.abs(np.abs(isum / np.max(np.abs(isum), axis=1, keepdims=True) * Q % 1.0) - 0.5) < 1e-3
+    assert np.array_equal(zq[~ties].astype(np.float64), want2[~ties])
+    # a planted mistake: swapping the two scale vectors changes the codes
+    wq, _ = orc.residual_add_q8_rows(xq, sf, fq, sx, 8, eps)
+    assert not np.array_equal(wq, yq)
