@@ -425,6 +425,20 @@ TWEO_API tweo_status_t tweo_int8_linear_q8(const int8_t* xq, int64_t ldx, const 
 TWEO_API tweo_status_t tweo_residual_add_q8(const int8_t* xq, const float* sx, const int8_t* fq, const float* sf,
                                    int64_t n, int32_t bits, const float* sy, int8_t* yq, void* stream);
 
+/*
+ * tweo_residual_add_q8_rows -- the residual addition on a residual stream quantised per token (Sec. 4.4: the
+ * "A8(K)" granularity, one Eq. 4 scale per row): for every row m of the [rows, cols] codes
+ *   y_mj  = fl32( fq_mj * fl32(sf[m] / Q_b) + fl32(xq_mj * fl32(sx[m] / Q_b)) )
+ *   sy[m] = fl32( max_j |y_mj| + eps )                     the row's own AbsMax scale, written to sy
+ *   yq_mj = clamp( rne_int( fl32(y_mj * fl32(Q_b / sy[m])) ), -Q_b, Q_b ),  NaN -> 0
+ * xq, fq, yq: int8 [rows, cols], dense, device, 16-byte aligned (yq may alias xq or fq); sx, sf, sy: device
+ * float [rows].  cols % 16 == 0, cols <= 8192; 2 <= bits <= 8; eps >= 0.
+ * Errors: TWEO_ERR_INVALID_ARG, TWEO_ERR_UNSUPPORTED_SHAPE, TWEO_ERR_ALIGNMENT.
+ */
+TWEO_API tweo_status_t tweo_residual_add_q8_rows(const int8_t* xq, const float* sx, const int8_t* fq,
+                                        const float* sf, int64_t rows, int64_t cols, int32_t bits, float eps,
+                                        int8_t* yq, float* sy, void* stream);
+
 /* ---------------------------------------------------------------- helpers */
 
 /* Bytes of workspace `op` needs for the given problem (n for QUANTIZE / LOSS is

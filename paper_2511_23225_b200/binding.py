@@ -29,7 +29,7 @@ EXPORTS = [
     "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_fwd_act",
     "tweo_layernorm_fp8", "tweo_fp8_linear_bwd_dgrad",
     "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
-    "tweo_block_output_fused", "tweo_delayed_scaling_update", "tweo_absmax_quantize", "tweo_int8_linear", "tweo_int8_linear_q8", "tweo_residual_add_q8",
+    "tweo_block_output_fused", "tweo_delayed_scaling_update", "tweo_absmax_quantize", "tweo_int8_linear", "tweo_int8_linear_q8", "tweo_residual_add_q8", "tweo_residual_add_q8_rows",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
 ]
@@ -95,6 +95,7 @@ def lib() -> C.CDLL:
         L.tweo_int8_linear.argtypes = [vp, i64, vp, i32, vp, i64, vp, i32, i32, vp, i64, i64, i64, i64, vp]
         L.tweo_int8_linear_q8.argtypes = [vp, i64, vp, i32, vp, i64, vp, i32, i32, vp, vp, i64, i64, i64, i64, vp]
         L.tweo_residual_add_q8.argtypes = [vp, vp, vp, vp, i64, i32, vp, vp, vp]
+        L.tweo_residual_add_q8_rows.argtypes = [vp, vp, vp, vp, i64, i64, i32, f32, vp, vp, vp]
         L.tweo_w8a8_static_gemm.argtypes = [vp, i32, i64, vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, sz, vp]
         L.tweo_workspace_bytes.argtypes = [i32, i64, i64, i64]
         L.tweo_workspace_bytes.restype = sz
@@ -580,3 +581,21 @@ def residual_add_q8(xq, sx, fq, sf, sy, bits=8, yq=None):
                                       _dev(sy, torch.float32, "sy"), _dev(yq, torch.int8, "yq"), _stream()),
            "tweo_residual_add_q8")
     return yq
+
+
+def residual_add_q8_rows(xq, sx, fq, sf, bits=8, eps=1e-6, yq=None):
+    """tweo_residual_add_q8_rows: per-token quantised residual addition.  xq, fq: int8 [rows, cols] with one scale
+    per row (sx, sf: float32 [rows]); returns (codes of x + f(x), their per-row AbsMax scales)."""
+    if xq.dim() != 2 or xq.shape != fq.shape or not xq.is_contiguous() or not fq.is_contiguous():
+        raise ValueError("xq and fq must be contiguous 2-D tensors of equal shape")
+    rows, cols = xq.shape
+    if sx.numel() != rows or sf.numel() != rows:
+        raise ValueError("one scale per row")
+    if yq is None:
+        yq = torch.empty_like(xq)
+    sy = torch.empty(rows, dtype=torch.float32, device=xq.device)
+    _check(lib().tweo_residual_add_q8_rows(_dev(xq, torch.int8, "xq"), _dev(sx, torch.float32, "sx"),
+                                           _dev(fq, torch.int8, "fq"), _dev(sf, torch.float32, "sf"), rows, cols, bits,
+                                           eps, _dev(yq, torch.int8, "yq"), sy.data_ptr() if rows else None, _stream()),
+           "tweo_residual_add_q8_rows")
+    return yq, sy

@@ -263,3 +263,125 @@ extern "C" tweo_status_t tweo_residual_add_q8(const int8_t* xq, const float* sx,
   tweo_detail::count_launch();
   return tweo_detail::check_launch("residual_add_q8_kernel");
 }
+
+// ------------------------------------------------------------------ per-token 8-bit residual stream (Sec. 4.4)
+// One warp per row: the row's codes of x and f(x) stay in registers (VPL 16-byte vectors of each per lane,
+// lane-interleaved), so the dequantised sum is formed once, its maximum found by shuffles, and the codes of the
+// sum written in the same pass: 2 bytes read and 1 written per element plus three scales per row.
+namespace {
+
+struct RowAddArgs {
+  const int8_t* xq;
+  const int8_t* fq;
+  int8_t* yq;
+  const float* sx;
+  const float* sf;
+  float* sy;
+  int64_t rows;
+  int32_t cols;
+  float Q, eps;
+};
+
+template <int VPL>
+__global__ void __launch_bounds__(256) residual_add_q8_rows_kernel(const RowAddArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp_global = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int64_t warp_stride = (int64_t)gridDim.x * 8;
+  const int nvec = a.cols >> 4;
+  const int q = (int)a.Q;
+  for (int64_t row = warp_global; row < a.rows; row += warp_stride) {
+    const uint4* xv = reinterpret_cast<const uint4*>(a.xq + row * a.cols);
+    const uint4* fv = reinterpret_cast<const uint4*>(a.fq + row * a.cols);
+    uint4 vx[VPL], vf[VPL];
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+      const int idx = lane + 32 * i;
+      vx[i] = idx < nvec ? __ldcs(xv + idx) : make_uint4(0u, 0u, 0u, 0u);
+      vf[i] = idx < nvec ? __ldcs(fv + idx) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    const float cx = __fdiv_rn(__ldg(a.sx + row), a.Q), cf = __fdiv_rn(__ldg(a.sf + row), a.Q);
+    float amax = 0.0f;  // padding lanes hold zero codes: their sum is 0
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+      const uint32_t wx[4] = {vx[i].x, vx[i].y, vx[i].z, vx[i].w};
+      const uint32_t wf[4] = {vf[i].x, vf[i].y, vf[i].z, vf[i].w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          amax = fmaxf(amax, fabsf(__fmaf_rn(code_to_f32(wf[k], e), cf, __fmul_rn(code_to_f32(wx[k], e), cx))));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+    const float s = __fadd_rn(amax, a.eps);
+    const float c = __fdiv_rn(a.Q, s);
+    if (lane == 0) a.sy[row] = s;
+    uint4* yv = reinterpret_cast<uint4*>(a.yq + row * a.cols);
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+      const int idx = lane + 32 * i;
+      if (idx < nvec) {
+        const uint32_t wx[4] = {vx[i].x, vx[i].y, vx[i].z, vx[i].w};
+        const uint32_t wf[4] = {vf[i].x, vf[i].y, vf[i].z, vf[i].w};
+        uint32_t o4[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          uint32_t w = 0u;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float y = __fmaf_rn(code_to_f32(wf[k], e), cf, __fmul_rn(code_to_f32(wx[k], e), cx));
+            w |= ((uint32_t)quant1(y, c, a.Q) & 0xFFu) << (8 * e);
+          }
+          o4[k] = w;
+        }
+        __stcs(yv + idx, make_uint4(o4[0], o4[1], o4[2], o4[3]));
+      }
+    }
+    (void)q;
+  }
+}
+
+template <int VPL>
+cudaError_t launch_row_add(const RowAddArgs& a, cudaStream_t st) {
+  int per_sm = 0;
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, residual_add_q8_rows_kernel<VPL>, 256, 0);
+  if (e != cudaSuccess) return e;
+  const int64_t want = (a.rows + 7) / 8;
+  const int64_t cap = (int64_t)tweo_detail::sm_count() * (per_sm > 0 ? per_sm : 1);
+  residual_add_q8_rows_kernel<VPL><<<(int)(want < cap ? want : cap), 256, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" tweo_status_t tweo_residual_add_q8_rows(const int8_t* xq, const float* sx, const int8_t* fq, const float* sf,
+                                                   int64_t rows, int64_t cols, int32_t bits, float eps, int8_t* yq,
+                                                   float* sy, void* stream) {
+  if (rows < 0 || cols < 1 || bits < 2 || bits > 8 || !(eps >= 0.0f)) return TWEO_ERR_INVALID_ARG;
+  if ((cols & 15) || cols > 8192) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  if (rows == 0) return TWEO_OK;
+  if (!xq || !fq || !yq || !sx || !sf || !sy) return TWEO_ERR_INVALID_ARG;
+  if (!tweo_detail::aligned16(xq) || !tweo_detail::aligned16(fq) || !tweo_detail::aligned16(yq)) return TWEO_ERR_ALIGNMENT;
+  RowAddArgs a;
+  a.xq = xq;
+  a.fq = fq;
+  a.yq = yq;
+  a.sx = sx;
+  a.sf = sf;
+  a.sy = sy;
+  a.rows = rows;
+  a.cols = (int32_t)cols;
+  a.Q = (float)((1 << (bits - 1)) - 1);
+  a.eps = eps;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int vpl = (int)((cols / 16 + 31) / 32);
+  cudaError_t e;
+  if (vpl <= 1) e = launch_row_add<1>(a, st);
+  else if (vpl <= 2) e = launch_row_add<2>(a, st);
+  else if (vpl <= 4) e = launch_row_add<4>(a, st);
+  else if (vpl <= 8) e = launch_row_add<8>(a, st);
+  else e = launch_row_add<16>(a, st);
+  if (e != cudaSuccess) return tweo_detail::cuda_fail(e, "residual_add_q8_rows_kernel");
+  tweo_detail::count_launch();
+  return TWEO_OK;
+}

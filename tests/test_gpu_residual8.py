@@ -111,9 +111,59 @@ def test_block_chain_stays_in_8_bits(tw):
     assert np.linalg.norm(deq - true) / np.linalg.norm(true) < 0.03
 
 
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("rows,cols", [(1, 16), (37, 768), (1000, 2048), (9, 4096), (5, 8192), (0, 256)])
+def test_residual_add_q8_rows_bit_exact(tw, rows, cols, bits):
+    Q = orc.absmax_qmax(bits)
+    g = np.random.Generator(np.random.PCG64(rows * 131 + cols + bits))
+    xq = g.integers(-Q, Q + 1, (rows, cols), dtype=np.int8)
+    fq = g.integers(-Q, Q + 1, (rows, cols), dtype=np.int8)
+    sx = (0.5 + 3.0 * g.random(rows)).astype(np.float32)
+    sf = (0.05 + 0.5 * g.random(rows)).astype(np.float32)
+    ref_q, ref_s = orc.residual_add_q8_rows(xq, sx, fq, sf, bits, 1e-6)
+    gx, gf = torch.from_numpy(xq).cuda(), torch.from_numpy(fq).cuda()
+    yq, sy = tw.residual_add_q8_rows(gx, dev(sx) if rows else torch.empty(0, device="cuda"),
+                                     gf, dev(sf) if rows else torch.empty(0, device="cuda"), bits, 1e-6)
+    torch.cuda.synchronize()
+    assert np.array_equal(sy.cpu().numpy().view(np.uint32), ref_s.view(np.uint32))
+    assert np.array_equal(yq.cpu().numpy(), ref_q)
+    if rows:
+        assert np.all(np.max(np.abs(ref_q.astype(np.int64)), axis=1) == Q)
+        out, _ = tw.residual_add_q8_rows(gx, dev(sx), gf, dev(sf), bits, 1e-6, yq=gx)     # y overwrites x
+        torch.cuda.synchronize()
+        assert out is gx and np.array_equal(gx.cpu().numpy(), ref_q)
+
+
+def test_per_token_chain_linear_quantise_add(tw):
+    """A8(K): x codes per token -> integer linear (per-token x per-channel scales) -> per-token codes of f(x) ->
+    per-token codes of x + f(x); every stage against the oracle's stage on the oracle's own inputs."""
+    M, K = 320, 512
+    x = synth.normal_bf16(960, (M, K), 1.0)
+    w = synth.normal_bf16(961, (K, K), 0.04)
+    xq, sx = orc.absmax_quantize_bf16(x, 8, 1e-6, per_row=True)
+    wq, sw = orc.absmax_quantize_bf16(w, 8, 1e-6, per_row=True)
+    f = tw.int8_linear(torch.from_numpy(xq).cuda(), dev(sx), torch.from_numpy(wq).cuda(), dev(sw), 8)
+    r, c = np.divmod(np.arange(M * K), K)
+    f_ref = orc.int8_gemm_at(xq, wq, sx, sw, 8, r, c).reshape(M, K)
+    torch.cuda.synchronize()
+    assert np.linalg.norm(f.float().cpu().numpy() - f_ref) / np.linalg.norm(f_ref) <= 1e-2
+    f_bits = orc.f64_array_to_bf16(f_ref)                     # the oracle's own bf16 f(x) feeds the oracle's next stages
+    fq_ref, sf_ref = orc.absmax_quantize_bf16(f_bits, 8, 1e-6, per_row=True)
+    yq_ref, sy_ref = orc.residual_add_q8_rows(xq, sx, fq_ref, sf_ref, 8, 1e-6)
+    yq, sy = tw.residual_add_q8_rows(torch.from_numpy(xq).cuda(), dev(sx), torch.from_numpy(fq_ref).cuda(), dev(sf_ref), 8, 1e-6)
+    torch.cuda.synchronize()
+    assert np.array_equal(yq.cpu().numpy(), yq_ref) and np.array_equal(sy.cpu().numpy(), sy_ref)
+    true = synth.bf16_bits_to_f32(x).astype(np.float64) + f_ref
+    deq = yq_ref.astype(np.float64) * sy_ref.astype(np.float64)[:, None] / 127.0
+    assert np.linalg.norm(deq - true) / np.linalg.norm(true) < 0.02
+
+
 def test_q8_argument_checks(tw):
     a = torch.zeros(64, dtype=torch.int8, device="cuda")
     with pytest.raises(tw.TweoError):
         tw.residual_add_q8(a, dev(1.0), a, dev(1.0), dev(1.0), bits=9)
     with pytest.raises(tw.TweoError):
         tw.residual_add_q8(a[1:33], dev(1.0), a[1:33], dev(1.0), dev(1.0))          # not 16-byte aligned
+    b = torch.zeros((4, 24), dtype=torch.int8, device="cuda")
+    with pytest.raises(tw.TweoError):
+        tw.residual_add_q8_rows(b, dev([1.0] * 4), b, dev([1.0] * 4))                # cols % 16 != 0
