@@ -517,6 +517,17 @@ def residual8_bench(torch, tw, peaks, reps=10):
         out["residual_add_q8"].append({"n": n, "us": us, "gbs": 3.0 * n / us / 1e3,
                                        "frac_of_hbm_peak": 3.0 * n / us / 1e3 / peaks["hbm"]})
         del xq, fq, yq
+    out["residual_add_q8_rows"] = []
+    for rows, cols in ((16384, 768), (65536, 2048)):        # per token (A8(K)): one scale per row in, one out
+        xq = torch.randint(-127, 128, (rows, cols), device="cuda", dtype=torch.int8)
+        fq = torch.randint(-127, 128, (rows, cols), device="cuda", dtype=torch.int8)
+        yq = torch.empty_like(xq)
+        s = torch.full((rows,), 2.0, dtype=torch.float32, device="cuda")
+        us = timed(lambda: tw.residual_add_q8_rows(xq, s, fq, s, 8, 1e-6, yq=yq))
+        n = rows * cols
+        out["residual_add_q8_rows"].append({"rows": rows, "cols": cols, "us": us, "gbs": 3.0 * n / us / 1e3,
+                                            "frac_of_hbm_peak": 3.0 * n / us / 1e3 / peaks["hbm"]})
+        del xq, fq, yq
     torch.cuda.empty_cache()
     return out
 
