@@ -186,6 +186,9 @@ __device__ __forceinline__ uint32_t cta_max(uint32_t m, uint32_t* part) {
   return m;
 }
 
+// U: 16-byte loads in flight per thread.  Large batches take the deeper variant (more bytes in flight per SM);
+// small ones the shallow one, whose smaller per-CTA share keeps all SMs busy to the end.
+template <int U>
 __global__ void __launch_bounds__(kThreads) amax_batch_kernel(const __grid_constant__ QBatch b, uint32_t* slots) {
   __shared__ uint32_t part[kThreads / 32];
 #pragma unroll 1
@@ -194,17 +197,17 @@ __global__ void __launch_bounds__(kThreads) amax_batch_kernel(const __grid_const
     const int64_t nvec = n >> 3;
     const uint16_t* x = b.t[ti].x;
     const uint4* xv = reinterpret_cast<const uint4*>(x);
-    const int64_t stride = (int64_t)gridDim.x * kThreads * 4;
+    const int64_t stride = (int64_t)gridDim.x * kThreads * U;
     uint32_t m = 0;
-    for (int64_t base = (int64_t)blockIdx.x * kThreads * 4 + threadIdx.x; base < nvec; base += stride) {
-      uint4 v[4];
+    for (int64_t base = (int64_t)blockIdx.x * kThreads * U + threadIdx.x; base < nvec; base += stride) {
+      uint4 v[U];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < U; ++u) {
         int64_t i = base + (int64_t)u * kThreads;
         v[u] = i < nvec ? __ldg(xv + i) : make_uint4(0, 0, 0, 0);
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < U; ++u) {
         m = absmax_bits(m, v[u].x);
         m = absmax_bits(m, v[u].y);
         m = absmax_bits(m, v[u].z);
@@ -220,7 +223,8 @@ __global__ void __launch_bounds__(kThreads) amax_batch_kernel(const __grid_const
   }
 }
 
-template <int FMT>
+// U: pairs of 16-byte loads in flight per thread (see amax_batch_kernel)
+template <int FMT, int U>
 __global__ void __launch_bounds__(kThreads) cast_batch_kernel(const __grid_constant__ QBatch b, const uint32_t* slots) {
   __shared__ uint32_t part[kThreads / 32];
 #pragma unroll 1
@@ -242,12 +246,12 @@ __global__ void __launch_bounds__(kThreads) cast_batch_kernel(const __grid_const
     uint8_t* q = b.t[ti].q;
     const uint4* xv = reinterpret_cast<const uint4*>(x);
     uint4* qv = reinterpret_cast<uint4*>(q);
-    const int64_t stride = (int64_t)gridDim.x * kThreads * 2;
+    const int64_t stride = (int64_t)gridDim.x * kThreads * U;
     uint32_t sat = 0, mm = 0;
-    for (int64_t base = (int64_t)blockIdx.x * kThreads * 2 + threadIdx.x; base < n16; base += stride) {
-      uint4 v[2][2];
+    for (int64_t base = (int64_t)blockIdx.x * kThreads * U + threadIdx.x; base < n16; base += stride) {
+      uint4 v[U][2];
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
+      for (int u = 0; u < U; ++u) {
         int64_t i = base + (int64_t)u * kThreads;
         if (i < n16) {
           v[u][0] = __ldcs(xv + 2 * i);
@@ -255,7 +259,7 @@ __global__ void __launch_bounds__(kThreads) cast_batch_kernel(const __grid_const
         }
       }
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
+      for (int u = 0; u < U; ++u) {
         int64_t i = base + (int64_t)u * kThreads;
         if (i < n16) __stcs(qv + i, cast16<FMT, false, false>(v[u][0], v[u][1], s, sat, mm));
       }
@@ -283,19 +287,29 @@ tweo_status_t launch_batch(const tweo_quant_desc_t* descs, const int* idx, int c
     vec8 += d.n >> 3;
     vec16[d.fmt] += d.n >> 4;
   }
-  b.amax_grid = grid_for(vec8, kThreads * 4, 8);
+  // the deeper variants once a launch has at least two full sweeps of the capped grid at their depth
+  const int64_t sweep = (int64_t)sm_count() * 8 * kThreads;
+  const bool deep_amax = vec8 >= 2 * sweep * 8;
+  b.amax_grid = grid_for(vec8, kThreads * (deep_amax ? 8 : 4), 8);
   if (b.amax_grid > kMaxAmaxGrid) b.amax_grid = kMaxAmaxGrid;
   uint32_t* slots = reinterpret_cast<uint32_t*>(ws);
-  amax_batch_kernel<<<b.amax_grid, kThreads, 0, st>>>(b, slots);
+  if (deep_amax) amax_batch_kernel<8><<<b.amax_grid, kThreads, 0, st>>>(b, slots);
+  else amax_batch_kernel<4><<<b.amax_grid, kThreads, 0, st>>>(b, slots);
   count_launch();
   bool has[2] = {false, false};
   for (int i = 0; i < count; ++i) has[b.t[i].fmt] = true;
   if (has[TWEO_E4M3]) {
-    cast_batch_kernel<TWEO_E4M3><<<grid_for(vec16[TWEO_E4M3], kThreads * 2, 8), kThreads, 0, st>>>(b, slots);
+    if (vec16[TWEO_E4M3] >= 2 * sweep * 4)
+      cast_batch_kernel<TWEO_E4M3, 4><<<grid_for(vec16[TWEO_E4M3], kThreads * 4, 8), kThreads, 0, st>>>(b, slots);
+    else
+      cast_batch_kernel<TWEO_E4M3, 2><<<grid_for(vec16[TWEO_E4M3], kThreads * 2, 8), kThreads, 0, st>>>(b, slots);
     count_launch();
   }
   if (has[TWEO_E5M2]) {
-    cast_batch_kernel<TWEO_E5M2><<<grid_for(vec16[TWEO_E5M2], kThreads * 2, 8), kThreads, 0, st>>>(b, slots);
+    if (vec16[TWEO_E5M2] >= 2 * sweep * 4)
+      cast_batch_kernel<TWEO_E5M2, 4><<<grid_for(vec16[TWEO_E5M2], kThreads * 4, 8), kThreads, 0, st>>>(b, slots);
+    else
+      cast_batch_kernel<TWEO_E5M2, 2><<<grid_for(vec16[TWEO_E5M2], kThreads * 2, 8), kThreads, 0, st>>>(b, slots);
     count_launch();
   }
   return check_launch("quantize batch kernels");
