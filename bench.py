@@ -251,7 +251,6 @@ def measure_workload(torch, tw, cfg_idx, steps, warmup, world, barrier, want_e2e
 
     # The step is a few dozen short kernels; issued one by one from Python the host is the bottleneck,
     # so the launch sequence is captured once into a CUDA graph and replayed (same kernels, same order).
-    host_loss = torch.empty(1, dtype=torch.float32).pin_memory()
     side = torch.cuda.Stream()
     c0 = tw.launch_count()
     step_graph = _graph_of(torch, side, bs.step)
