@@ -347,10 +347,23 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
           // int32 accumulators -> binary32, then the two Eq. 4 scales (row first, then column)
           const float ar = __fmul_rn(__ldg(p.row_scale + (p.row_scale_per_row ? min(row, p.Md - 1) : 0)), p.post_scale);
           const float ac0 = __ldg(p.col_scale);
+          if (p.col_scale_per_col && col0 + CH <= p.Nd && (reinterpret_cast<uintptr_t>(p.col_scale) & 15u) == 0) {
+            // a whole chunk of per-channel scales: 16-byte loads (the same addresses in every lane)
+            const float4* cs = reinterpret_cast<const float4*>(p.col_scale + col0);
 #pragma unroll
-          for (int j = 0; j < CH; ++j) {
-            const float ac = p.col_scale_per_col ? __ldg(p.col_scale + min(col0 + j, p.Nd - 1)) : ac0;
-            r[j] = __float_as_uint(__fmul_rn(__fmul_rn(__int2float_rn((int)r[j]), ar), ac));
+            for (int j4 = 0; j4 < CH / 4; ++j4) {
+              const float4 a4 = __ldg(cs + j4);
+              r[4 * j4] = __float_as_uint(__fmul_rn(__fmul_rn(__int2float_rn((int)r[4 * j4]), ar), a4.x));
+              r[4 * j4 + 1] = __float_as_uint(__fmul_rn(__fmul_rn(__int2float_rn((int)r[4 * j4 + 1]), ar), a4.y));
+              r[4 * j4 + 2] = __float_as_uint(__fmul_rn(__fmul_rn(__int2float_rn((int)r[4 * j4 + 2]), ar), a4.z));
+              r[4 * j4 + 3] = __float_as_uint(__fmul_rn(__fmul_rn(__int2float_rn((int)r[4 * j4 + 3]), ar), a4.w));
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < CH; ++j) {
+              const float ac = p.col_scale_per_col ? __ldg(p.col_scale + min(col0 + j, p.Nd - 1)) : ac0;
+              r[j] = __float_as_uint(__fmul_rn(__fmul_rn(__int2float_rn((int)r[j]), ar), ac));
+            }
           }
         }
         const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
