@@ -41,7 +41,7 @@ UNIT = "TFLOP/s"
 FP8_DATASHEET_TFLOPS = 4500.0
 # DRAM traffic of the dominant kernel family (the 8 GEMM launches of a config-2 step), per launch, from
 # the ncu capture summarised in profiles/launch_list_bench_cfg2.md; valid for that library version only.
-GEMM_TRAFFIC = {"library_version": 211, "workload": "cfg2", "bytes_per_launch": 20.49e6}
+GEMM_TRAFFIC = {"library_version": 212, "workload": "cfg2", "bytes_per_launch": 20.43e6}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, FALLBACK_BF16_SUSTAINED = 6650.0, 1590.0, 1400.0
 
 

@@ -1,6 +1,7 @@
 // Library-wide helpers: status strings, error text, launch counter, workspace sizing.
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -22,6 +23,11 @@ int sm_count() {
     cached[dev] = n;
   }
   return cached[dev];
+}
+
+bool chain_launch_enabled() {
+  static const bool on = [] { const char* e = getenv("TWEO_NO_LAUNCH_CHAIN"); return !(e && e[0] == '1'); }();
+  return on;
 }
 
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
@@ -62,7 +68,7 @@ const char* tweo_status_string(tweo_status_t s) {
 
 const char* tweo_last_cuda_error(void) { return g_err; }
 
-int32_t tweo_version(void) { return 211; }
+int32_t tweo_version(void) { return 212; }
 
 uint64_t tweo_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -33,6 +33,37 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 #ifdef __CUDACC__
 namespace tweo_detail {
 
+bool chain_launch_enabled();  // TWEO_NO_LAUNCH_CHAIN=1 in the environment turns programmatic dependent launch off
+
+// Launches `kern` with `cluster` CTAs per cluster (0: none) and, when enabled, as a programmatic dependent of
+// the kernel before it on the stream (see chain_wait()).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chain(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, unsigned cluster,
+                         Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  unsigned n = 0;
+  if (cluster > 0) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (chain_launch_enabled()) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 constexpr float kE4M3Max = 448.0f;
 constexpr float kE5M2Max = 57344.0f;
 
@@ -102,6 +133,14 @@ __device__ __forceinline__ uint32_t cvt_fp8x2_finite(float lo, float hi) {
   else asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
   return r;
 }
+
+// Programmatic dependent launch: a kernel launched with launch_chain() may become resident while the kernel
+// before it on the stream is still running (its launch latency and prologue are hidden); it must not touch
+// global memory before chain_wait(), which returns once that kernel has completed and its writes are visible.
+// chain_release() lets the next kernel of the chain start launching.  Both are no-ops in a kernel that was
+// launched the ordinary way.
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll

@@ -539,19 +539,7 @@ tweo_status_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CU
     }
   }
   if (p.sk_tiles == 0 && pairs > tiles) pairs = tiles;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(2 * pairs));
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, md, p));
+  TWEO_CUDA_TRY(launch_chain(kern, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, st, 2, ma, mb, md, md, p));
   count_launch();
   return check_launch("gemm_fp8_pair_kernel");
 }
@@ -832,19 +820,7 @@ tweo_status_t run_bwd_group(const uint8_t* dyq, int64_t lddy, int fmt_dy, const 
     }
     for (int t = 0; t < g.total_tiles; ++t) g.list[fill[owner[t]]++] = (uint16_t)t;  // ascending t within a pair
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(2 * pairs));
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, g));
+  TWEO_CUDA_TRY(launch_chain(kern, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, st, 2, g));
   count_launch();
   return check_launch("gemm_fp8_pair_group_kernel");
 }

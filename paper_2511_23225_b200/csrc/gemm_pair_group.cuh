@@ -122,6 +122,9 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams g) {
   cluster_sync_all();  // both CTAs' barriers are initialised before anyone signals across
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // barriers and tensor memory are set up; from here on global memory of the kernel before this one is touched
+  chain_release();
+  chain_wait();
 
   const int pair = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;

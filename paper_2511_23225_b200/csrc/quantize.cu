@@ -191,6 +191,8 @@ __device__ __forceinline__ uint32_t cta_max(uint32_t m, uint32_t* part) {
 template <int U>
 __global__ void __launch_bounds__(kThreads) amax_batch_kernel(const __grid_constant__ QBatch b, uint32_t* slots) {
   __shared__ uint32_t part[kThreads / 32];
+  chain_release();
+  chain_wait();
 #pragma unroll 1
   for (int ti = 0; ti < b.count; ++ti) {
     const int64_t n = b.t[ti].n;
@@ -227,6 +229,8 @@ __global__ void __launch_bounds__(kThreads) amax_batch_kernel(const __grid_const
 template <int FMT, int U>
 __global__ void __launch_bounds__(kThreads) cast_batch_kernel(const __grid_constant__ QBatch b, const uint32_t* slots) {
   __shared__ uint32_t part[kThreads / 32];
+  chain_release();
+  chain_wait();
 #pragma unroll 1
   for (int ti = 0; ti < b.count; ++ti) {
     if (b.t[ti].fmt != FMT) continue;
@@ -293,23 +297,27 @@ tweo_status_t launch_batch(const tweo_quant_desc_t* descs, const int* idx, int c
   b.amax_grid = grid_for(vec8, kThreads * (deep_amax ? 8 : 4), 8);
   if (b.amax_grid > kMaxAmaxGrid) b.amax_grid = kMaxAmaxGrid;
   uint32_t* slots = reinterpret_cast<uint32_t*>(ws);
-  if (deep_amax) amax_batch_kernel<8><<<b.amax_grid, kThreads, 0, st>>>(b, slots);
-  else amax_batch_kernel<4><<<b.amax_grid, kThreads, 0, st>>>(b, slots);
+  if (deep_amax) TWEO_CUDA_TRY(launch_chain(amax_batch_kernel<8>, dim3(b.amax_grid), dim3(kThreads), 0, st, 0, b, slots));
+  else TWEO_CUDA_TRY(launch_chain(amax_batch_kernel<4>, dim3(b.amax_grid), dim3(kThreads), 0, st, 0, b, slots));
   count_launch();
   bool has[2] = {false, false};
   for (int i = 0; i < count; ++i) has[b.t[i].fmt] = true;
   if (has[TWEO_E4M3]) {
     if (vec16[TWEO_E4M3] >= 2 * sweep * 4)
-      cast_batch_kernel<TWEO_E4M3, 4><<<grid_for(vec16[TWEO_E4M3], kThreads * 4, 8), kThreads, 0, st>>>(b, slots);
+      TWEO_CUDA_TRY(launch_chain(cast_batch_kernel<TWEO_E4M3, 4>, dim3(grid_for(vec16[TWEO_E4M3], kThreads * 4, 8)), dim3(kThreads), 0, st, 0, b,
+                                 (const uint32_t*)slots));
     else
-      cast_batch_kernel<TWEO_E4M3, 2><<<grid_for(vec16[TWEO_E4M3], kThreads * 2, 8), kThreads, 0, st>>>(b, slots);
+      TWEO_CUDA_TRY(launch_chain(cast_batch_kernel<TWEO_E4M3, 2>, dim3(grid_for(vec16[TWEO_E4M3], kThreads * 2, 8)), dim3(kThreads), 0, st, 0, b,
+                                 (const uint32_t*)slots));
     count_launch();
   }
   if (has[TWEO_E5M2]) {
     if (vec16[TWEO_E5M2] >= 2 * sweep * 4)
-      cast_batch_kernel<TWEO_E5M2, 4><<<grid_for(vec16[TWEO_E5M2], kThreads * 4, 8), kThreads, 0, st>>>(b, slots);
+      TWEO_CUDA_TRY(launch_chain(cast_batch_kernel<TWEO_E5M2, 4>, dim3(grid_for(vec16[TWEO_E5M2], kThreads * 4, 8)), dim3(kThreads), 0, st, 0, b,
+                                 (const uint32_t*)slots));
     else
-      cast_batch_kernel<TWEO_E5M2, 2><<<grid_for(vec16[TWEO_E5M2], kThreads * 2, 8), kThreads, 0, st>>>(b, slots);
+      TWEO_CUDA_TRY(launch_chain(cast_batch_kernel<TWEO_E5M2, 2>, dim3(grid_for(vec16[TWEO_E5M2], kThreads * 2, 8)), dim3(kThreads), 0, st, 0, b,
+                                 (const uint32_t*)slots));
     count_launch();
   }
   return check_launch("quantize batch kernels");
