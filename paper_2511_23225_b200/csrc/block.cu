@@ -107,12 +107,10 @@ __global__ void __launch_bounds__(kThreads) block_output_kernel(const BlockArgs 
       const uint32_t fw[8] = {fr[u][0].x, fr[u][0].y, fr[u][0].z, fr[u][0].w, fr[u][1].x, fr[u][1].y, fr[u][1].z, fr[u][1].w};
       uint32_t aw[8], gw[8], c[8];
       float t = 0.0f;
-      bool any_nan = false;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         aw[j] = add_pair<FAST, GRAD>(xw[j], fw[j], args.k_grad, args.p, t, gw[j]);
         m2 = absmax_bits(m2, aw[j]);
-        if (QFMT >= 0) any_nan |= pair_has_nan(aw[j]);
       }
       acc += (double)t;
       __stcs(av + 2 * i, make_uint4(aw[0], aw[1], aw[2], aw[3]));
@@ -125,7 +123,7 @@ __global__ void __launch_bounds__(kThreads) block_output_kernel(const BlockArgs 
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const float lo = __fmul_rn(bf16lo_to_f32(aw[j]), qs), hi = __fmul_rn(bf16hi_to_f32(aw[j]), qs);
-          c[j] = any_nan ? cvt_fp8x2<QFMT < 0 ? 0 : QFMT>(lo, hi) : cvt_fp8x2_finite<QFMT < 0 ? 0 : QFMT>(lo, hi);
+          c[j] = cvt_fp8x2<QFMT < 0 ? 0 : QFMT>(lo, hi);
         }
         __stcs(qv + i, make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16)));
       }

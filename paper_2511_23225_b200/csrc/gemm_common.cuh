@@ -107,9 +107,7 @@ __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d) {
   return cvt_fp8x2<FMT>(a, b) | (cvt_fp8x2<FMT>(c, d) << 16);
 }
 
-// Four bf16 values (two packed words) times the scale -> four FP8 codes.  Branch-free: a test for
-// NaN on the packed words with a rare slow path was measured 2x slower (it splits the unrolled
-// epilogue into basic blocks and the loads and conversions of different columns no longer overlap).
+// Four bf16 values (two packed words) times the scale -> four FP8 codes.
 template <int FMT>
 __device__ __forceinline__ uint32_t quant_words(uint32_t w0, uint32_t w1, float qs) {
   return quant4<FMT>(__fmul_rn(bf16lo_to_f32(w0), qs), __fmul_rn(bf16hi_to_f32(w0), qs),

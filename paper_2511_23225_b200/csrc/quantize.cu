@@ -74,23 +74,19 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint16_t* x, int64
 }
 
 // 16 elements: two 16-byte loads -> one 16-byte store.  SAT counts elements whose scaled value
-// exceeds the format's range, AMAX folds |x| into the running maximum m2.  The scaled value of a
-// finite or infinite input is never NaN (the scale is positive and finite), so only inputs that
-// are NaN themselves need the converter's NaN fix-up; they are rare and take the slow branch.
+// exceeds the format's range, AMAX folds |x| into the running maximum m2.  NaN inputs come out of the
+// converter as the code 0x7F (see cvt_fp8x2).
 template <int FMT, bool SAT, bool AMAX>
 __device__ __forceinline__ uint4 cast16(const uint4 a, const uint4 b, float scale, uint32_t& sat, uint32_t& m2) {
   const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
   uint32_t c[8];
   const float fmax = FMT == TWEO_E4M3 ? kE4M3Max : kE5M2Max;
-  bool any_nan = false;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) any_nan |= pair_has_nan(w[j]);
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     float lo = __fmul_rn(bf16lo_to_f32(w[j]), scale);
     float hi = __fmul_rn(bf16hi_to_f32(w[j]), scale);
     if (SAT) sat += (fabsf(lo) > fmax) + (fabsf(hi) > fmax);
-    c[j] = any_nan ? cvt_fp8x2<FMT>(lo, hi) : cvt_fp8x2_finite<FMT>(lo, hi);
+    c[j] = cvt_fp8x2<FMT>(lo, hi);
     if (AMAX) m2 = absmax_bits(m2, w[j]);
   }
   return make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16));
