@@ -119,6 +119,13 @@ __device__ __forceinline__ uint32_t absmax_bits(uint32_t m2, uint32_t w) {
   a &= __vcmpleu2(a, 0x7F807F80u);
   return __vmaxu2(m2, a);
 }
+// The same running maximum kept as two binary32 values (fmaxf skips NaN by itself): four plain instructions per
+// pair of elements.  absmax_f32_bits() gives the result as a bf16 bit pattern like absmax_fold().
+__device__ __forceinline__ void absmax_f32(float& m0, float& m1, uint32_t w) {
+  m0 = fmaxf(m0, fabsf(bf16lo_to_f32(w)));
+  m1 = fmaxf(m1, fabsf(bf16hi_to_f32(w)));
+}
+__device__ __forceinline__ uint32_t absmax_f32_bits(float m0, float m1) { return __float_as_uint(fmaxf(m0, m1)) >> 16; }
 // the larger of the two lanes: the bit pattern of max |x| as a bf16 value
 __device__ __forceinline__ uint32_t absmax_fold(uint32_t m2) { return max(m2 & 0xFFFFu, m2 >> 16); }
 // Programmatic dependent launch: a kernel launched with launch_chain() may become resident while the kernel

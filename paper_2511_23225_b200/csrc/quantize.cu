@@ -196,7 +196,7 @@ __global__ void __launch_bounds__(kThreads) amax_batch_kernel(const __grid_const
     const uint16_t* x = b.t[ti].x;
     const uint4* xv = reinterpret_cast<const uint4*>(x);
     const int64_t stride = (int64_t)gridDim.x * kThreads * U;
-    uint32_t m = 0;
+    float m0 = 0.0f, m1 = 0.0f;
     for (int64_t base = (int64_t)blockIdx.x * kThreads * U + threadIdx.x; base < nvec; base += stride) {
       uint4 v[U];
 #pragma unroll
@@ -206,17 +206,17 @@ __global__ void __launch_bounds__(kThreads) amax_batch_kernel(const __grid_const
       }
 #pragma unroll
       for (int u = 0; u < U; ++u) {
-        m = absmax_bits(m, v[u].x);
-        m = absmax_bits(m, v[u].y);
-        m = absmax_bits(m, v[u].z);
-        m = absmax_bits(m, v[u].w);
+        absmax_f32(m0, m1, v[u].x);
+        absmax_f32(m0, m1, v[u].y);
+        absmax_f32(m0, m1, v[u].z);
+        absmax_f32(m0, m1, v[u].w);
       }
     }
     if (blockIdx.x == 0 && threadIdx.x < 8) {
       int64_t i = (nvec << 3) + threadIdx.x;
-      if (i < n) m = absmax_bits(m, (uint32_t)x[i]);
+      if (i < n) absmax_f32(m0, m1, (uint32_t)x[i]);
     }
-    m = cta_max(absmax_fold(m), part);
+    const uint32_t m = cta_max(absmax_f32_bits(m0, m1), part);
     if (threadIdx.x == 0) slots[ti * kMaxAmaxGrid + blockIdx.x] = m;
   }
 }
