@@ -611,9 +611,13 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
 template <int ACT>
 tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
                               const CUtensorMap& mq, GemmParams& p, cudaStream_t st) {
-  constexpr int STAGES = 5;
-  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 4 * 2 * 32 * 64 + 1024 + 256;
-  auto kern = gemm_fp8_pair_kernel<false, false, STAGES, false, false, ACT, true>;
+  // the per-element epilogues run with eight epilogue warps and four operand stages; SwiGLU (long
+  // contraction, 238 registers) keeps four warps and five stages
+  constexpr int EPIW = ACT == 3 ? 4 : 8;
+  constexpr int STAGES = ACT == 3 ? 5 : 4;
+  constexpr int THREADS = 64 + 32 * EPIW;
+  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + EPIW * 2 * 32 * 128 + EPIW * 2 * 32 * 64 + 1024 + 256;
+  auto kern = gemm_fp8_pair_kernel<false, false, STAGES, false, false, ACT, true, EPIW>;
   static bool attr_done = false;
   if (!attr_done) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -633,7 +637,7 @@ tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, cons
   if (pairs > tiles) pairs = tiles;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs));
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];

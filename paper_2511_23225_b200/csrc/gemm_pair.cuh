@@ -157,8 +157,14 @@ __device__ __noinline__ float pair_partial_share(const GemmParams& p, const CUte
 // rows, 64-byte swizzle) like the bf16 tile, instead of 16-byte stores from registers that touch
 // 32 different rows per instruction.  Takes 16 KB of shared memory, so such kernels run with one
 // stage less in the operand ring.
-template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32, bool I8 = false, int ACT = 0, bool QST = false>
-__global__ void __launch_bounds__(kThreads, 1)
+//
+// EPIW: epilogue warps per CTA (4 or 8).  A warp reads the 32 tensor-memory lanes (warp index mod 4) allows
+// it; with 8 warps two warps share each lane quarter and take half of the tile's columns each.  The
+// epilogues that compute per element (activation, FP8 copy) are bound by the issue rate of one warp per
+// scheduler at short contractions; a second warp per scheduler doubles it.  Costs 48 KB more staging memory
+// (one operand stage less) and caps the kernel at 200 registers per thread.
+template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32, bool I8 = false, int ACT = 0, bool QST = false, int EPIW = 4>
+__global__ void __launch_bounds__(64 + 32 * EPIW, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ CUtensorMap tmap_q,
                      const __grid_constant__ GemmParams p) {
@@ -171,10 +177,11 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   constexpr uint32_t EPI_BUF = 32 * 128;
-  constexpr uint32_t EPI_BYTES = 4 * 2 * EPI_BUF;
+  constexpr uint32_t EPI_BYTES = EPIW * 2 * EPI_BUF;
+  static_assert(EPIW == 4 || EPIW == 8, "epilogue warps per CTA");
   constexpr bool Q8 = I8 && QST;                            // integer linear with an 8-bit (Eq. 4) output only
   constexpr uint32_t Q_BUF = 32 * 64;                       // 32 rows x 64 one-byte codes
-  constexpr uint32_t Q_BYTES = QST ? 4 * 2 * Q_BUF : 0;
+  constexpr uint32_t Q_BYTES = QST ? EPIW * 2 * Q_BUF : 0;
   uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES + Q_BYTES);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
@@ -198,7 +205,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 8);  // four epilogue warps of each CTA of the pair
+      mbar_init(tempty_bar(a), 2 * EPIW);  // the epilogue warps of both CTAs of the pair
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -324,7 +331,10 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         continue;
       }
 #pragma unroll 1
-      for (int c = 0; c < (ACT == 3 ? 128 : BN) / CH; ++c) {
+      // with 8 epilogue warps, warps 2-5 take the first half of the tile's chunks and warps 6-9 the second
+      constexpr int NC = (ACT == 3 ? 128 : BN) / CH, NC_W = NC / (EPIW / 4);
+      const int c_first = ((warp - 2) >> 2) * NC_W;
+      for (int c = c_first; c < c_first + NC_W; ++c) {
         const int col0 = n0 + c * CH;
         if (col0 >= p.Nd) break;
         uint32_t r[CH];
