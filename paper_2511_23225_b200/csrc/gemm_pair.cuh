@@ -9,7 +9,8 @@
 //   full[s]    leader only : leader's producer arrives (+ expected bytes of BOTH CTAs' loads)
 //   empty[s]   each CTA    : leader's MMA thread commits to its own and to the peer's
 //   tfull[a]   each CTA    : same, once a tile's accumulator is complete
-//   tempty[a]  leader only : 4 epilogue warps of each CTA arrive (the peer's remotely)
+//   tempty[a]  leader only : the epilogue warps (4 or 8) of each CTA arrive (the peer's remotely; a relaxed
+//                            arrival: a releasing one would wait for the warp's TMA stores to drain)
 #pragma once
 
 #include <cuda.h>
@@ -290,7 +291,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    // ------------------------------------------------------------ epilogue (warps 2 .. 1 + EPIW, both CTAs)
     const int quarter = warp & 3;
     const float alpha = I8 ? 1.0f : __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
     const float qs = p.out_q ? (Q8 ? __fdiv_rn(p.q8_qmax, __ldg(p.q_scale)) : __ldg(p.q_scale)) : 0.0f;
