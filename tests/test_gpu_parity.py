@@ -531,3 +531,29 @@ def test_step_on_two_streams_equals_step_on_one(tw):
     for a, b, c in zip(ref, two, rep):
         assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
         assert torch.equal(a.view(torch.uint8), c.view(torch.uint8))
+
+
+def test_gemm_paths_repeat_bit_for_bit(tw):
+    """Forty back-to-back repetitions of the forward product, the one-launch backward and the activation-fused
+    forward (no host synchronisation in between, so consecutive launches overlap as far as the launch chain
+    allows): every output must equal the first repetition's bit for bit."""
+    M, K, N = 4096, 768, 2304
+    g = torch.Generator(device="cuda").manual_seed(7)
+    xq = torch.randint(0, 120, (M, K), dtype=torch.uint8, device="cuda", generator=g)
+    wq = torch.randint(0, 120, (N, K), dtype=torch.uint8, device="cuda", generator=g)
+    dyq = torch.randint(0, 120, (M, N), dtype=torch.uint8, device="cuda", generator=g)
+    s, qs = dev_scalar(1e-3), dev_scalar(8.0)
+    ws = tw.new_workspace(tw.OP_LINEAR_WGRAD)
+    first, mismatches = None, 0
+    for _ in range(40):
+        y = tw.fp8_linear_fwd(xq, wq, s, s, ws=ws)
+        dx, dw = tw.fp8_linear_bwd(dyq, xq, wq, s, s, s, fmt_dy=E5M2, ws=ws)
+        yq = torch.empty((M, N), dtype=torch.uint8, device="cuda")
+        ya = tw.fp8_linear_fwd_act(xq, wq, s, s, tw.ACT_GELU_TANH, out_q=yq, q_scale=qs)
+        cur = [t.clone() for t in (y, dx, dw, ya, yq)]
+        if first is None:
+            first = cur
+        else:
+            mismatches += sum(0 if torch.equal(a.view(torch.uint8), b.view(torch.uint8)) else 1 for a, b in zip(first, cur))
+    torch.cuda.synchronize()
+    assert tw.read_device_status() == 0 and mismatches == 0
