@@ -1,0 +1,41 @@
+"""The call sequences shown in the README run as written (shapes small; values are checked elsewhere)."""
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+def test_readme_call_sequences():
+    from paper_2511_23225_b200 import binding as tw
+    M, K, N = 384, 256, 512
+    x = torch.randn(M, K, device="cuda").to(torch.bfloat16)
+    w = (0.02 * torch.randn(N, K, device="cuda")).to(torch.bfloat16)
+    dy = (1e-3 * torch.randn(M, N, device="cuda")).to(torch.bfloat16)
+    ws_q, ws_g = tw.new_workspace(tw.OP_QUANTIZE), tw.new_workspace(tw.OP_LINEAR_WGRAD)
+    qx, qw, qdy = (tw.quantize_per_tensor(t, f, ws=ws_q) for t, f in ((x, tw.E4M3), (w, tw.E4M3), (dy, tw.E5M2)))
+    y = tw.fp8_linear_fwd(qx.q, qw.q, qx.scale_inv, qw.scale_inv, ws=ws_g)
+    dx, dw = tw.fp8_linear_bwd(qdy.q, qx.q, qw.q, qdy.scale_inv, qx.scale_inv, qw.scale_inv, ws=ws_g)
+    assert y.shape == (M, N) and dx.shape == (M, K) and dw.shape == (N, K)
+
+    block_outputs = [torch.randn(M, K, device="cuda").to(torch.bfloat16) for _ in range(3)]
+    loss, per_block, grads = tw.loss_fwd_bwd(block_outputs, 3.0, 1e-6, 4.0, 0.01 / len(block_outputs))
+    assert loss.numel() == 1 and per_block.numel() == 3 and len(grads) == 3
+
+    scale_next = torch.full((1,), 16.0, device="cuda")
+    a, loss_l, amax, grad, aq = tw.block_output_fused(x, x, q_fmt=tw.E4M3, q_scale=scale_next)
+    hist = torch.zeros(1, 16, device="cuda")
+    scale, scale_inv = torch.ones(1, device="cuda"), torch.ones(1, device="cuda")
+    tw.delayed_scaling_update(hist, amax, scale, scale_inv, tw.E4M3)
+    assert aq.dtype == torch.uint8 and abs(float(scale.item()) * float(amax.item()) - 448.0) < 1e-3
+
+    sx_static = torch.full((1,), 448.0 / 6.0, device="cuda")
+    y8 = tw.w8a8_static_gemm(x, sx_static, qw.q, qw.scale_inv)
+    assert y8.shape == (M, N)
+    s_in = torch.full((1,), 6.0, device="cuda")
+    xq, sx = tw.absmax_quantize(x, 8, tw.GRAN_TENSOR, s=s_in)
+    wq8, sw = tw.absmax_quantize(w[:K], 8, tw.GRAN_TENSOR)          # a square [K, K] weight for the residual block
+    sf, sy = torch.full((1,), 2.0, device="cuda"), torch.full((1,), 8.0, device="cuda")
+    fq = tw.int8_linear_q8(xq, sx, wq8, sw, sf)
+    yq = tw.residual_add_q8(xq, sx, fq, sf, sy)
+    torch.cuda.synchronize()
+    assert yq.dtype == torch.int8 and yq.shape == (M, K) and tw.read_device_status() == 0
