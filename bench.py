@@ -694,6 +694,10 @@ def run_cuda(args):
         if vendor_rows:
             line["context_vendor_fp8_gemm"] = vendor_rows
         if world == 1 and not args.no_cpu_baseline:
+            # a bounded sample: at most --cpu-rows tokens, and no more than about 350 GFLOP of oracle work
+            from paper_2511_23225_b200 import synth as _synth
+            _kn = sum(l.K * l.N for l in _synth.CONFIGS[cfg_idx].linears)
+            args.cpu_rows = max(16, min(args.cpu_rows, _synth.CONFIGS[cfg_idx].M, int(3.5e11 / (6 * _kn))))
             f, t = oracle_sample_step(cfg_idx, args.cpu_rows)
             line["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                                     "sample": f"first {args.cpu_rows} of {workload_cfg['tokens_per_gpu']} tokens of every "
@@ -712,7 +716,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--e2e-steps", type=int, default=20)
-    ap.add_argument("--cpu-rows", type=int, default=4096)
+    ap.add_argument("--cpu-rows", type=int, default=8192)
     ap.add_argument("--ref-rows", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--also", default="cfg4,cfg3", help="comma-separated other configs to run briefly (N=1 only); '' for none")
