@@ -453,6 +453,17 @@ TWEO_API tweo_status_t tweo_workspace_init(void* ws, size_t ws_bytes, void* stre
  * the stream reports an error, else TWEO_OK. */
 TWEO_API tweo_status_t tweo_read_device_status(void* stream);
 
+/*
+ * tweo_selftest_bounded_wait -- exercises the error path of the bounded device-side waits (the
+ * conventions above; no passage of the paper).  Launches one small kernel in which one thread waits,
+ * with the same wait routine the GEMM kernels use, for a barrier that nobody signals; after
+ * limit_ns nanoseconds (1 us .. 100 ms, else TWEO_ERR_INVALID_ARG) the wait gives up, records
+ * TWEO_ERR_TIMEOUT in the device status word and the kernel returns normally -- nothing traps and
+ * the context stays usable.  gave_up: device uint32* (or NULL) that receives 1 if the wait expired.
+ * The next tweo_read_device_status() returns TWEO_ERR_TIMEOUT once, then TWEO_OK again.
+ */
+TWEO_API tweo_status_t tweo_selftest_bounded_wait(uint64_t limit_ns, uint32_t* gave_up, void* stream);
+
 TWEO_API const char* tweo_status_string(tweo_status_t s);
 TWEO_API const char* tweo_last_cuda_error(void); /* text of the last failing CUDA call in this thread */
 TWEO_API int32_t tweo_version(void);             /* major * 10000 + minor * 100 + patch */

@@ -30,7 +30,7 @@ EXPORTS = [
     "tweo_layernorm_fp8", "tweo_fp8_linear_bwd_dgrad",
     "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
     "tweo_block_output_fused", "tweo_delayed_scaling_update", "tweo_absmax_quantize", "tweo_int8_linear", "tweo_int8_linear_q8", "tweo_residual_add_q8", "tweo_residual_add_q8_rows",
-    "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status",
+    "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status", "tweo_selftest_bounded_wait",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
 ]
 
@@ -101,6 +101,7 @@ def lib() -> C.CDLL:
         L.tweo_workspace_bytes.restype = sz
         L.tweo_workspace_init.argtypes = [vp, sz, vp]
         L.tweo_read_device_status.argtypes = [vp]
+        L.tweo_selftest_bounded_wait.argtypes = [C.c_uint64, vp, vp]
         L.tweo_status_string.argtypes = [i32]
         L.tweo_status_string.restype = C.c_char_p
         L.tweo_last_cuda_error.restype = C.c_char_p
@@ -162,6 +163,13 @@ def new_workspace(op: int, M: int = 0, N: int = 0, K: int = 0, device="cuda") ->
 
 def read_device_status() -> int:
     return int(lib().tweo_read_device_status(_stream()))
+
+
+def selftest_bounded_wait(limit_ns: int, gave_up: torch.Tensor | None = None) -> None:
+    """tweo_selftest_bounded_wait: one thread waits `limit_ns` for a barrier nobody signals, gives up and
+    records the expiry; read_device_status() then reports it once."""
+    _check(lib().tweo_selftest_bounded_wait(int(limit_ns), _dev(gave_up, torch.int32, "gave_up") if gave_up is not None
+                                            else None, _stream()), "tweo_selftest_bounded_wait")
 
 
 @dataclass

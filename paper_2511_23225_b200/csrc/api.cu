@@ -25,11 +25,6 @@ int sm_count() {
   return cached[dev];
 }
 
-bool chain_launch_enabled() {
-  static const bool on = [] { const char* e = getenv("TWEO_NO_LAUNCH_CHAIN"); return !(e && e[0] == '1'); }();
-  return on;
-}
-
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
 tweo_status_t cuda_fail(cudaError_t e, const char* what) {

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "tweo.h"
 
 namespace tweo_detail {
@@ -22,6 +24,18 @@ unsigned int* device_status_word();  // its device address on the current device
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// One-time set-up that CUDA keeps per device (function attributes): `mask` has one bit per device.
+// device_once_pending() is true while the current device still needs it; two host threads that race
+// here both run the (idempotent) set-up.  Devices beyond 63 are set up on every call.
+inline bool device_once_pending(std::atomic<uint64_t>& mask, int* dev) {
+  *dev = -1;
+  if (cudaGetDevice(dev) != cudaSuccess || *dev < 0 || *dev >= 64) return true;
+  return (mask.load(std::memory_order_acquire) & (1ull << *dev)) == 0;
+}
+inline void device_once_done(std::atomic<uint64_t>& mask, int dev) {
+  if (dev >= 0 && dev < 64) mask.fetch_or(1ull << dev, std::memory_order_release);
+}
+
 }  // namespace tweo_detail
 
 #define TWEO_CUDA_TRY(expr)                                              \
@@ -33,10 +47,8 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 #ifdef __CUDACC__
 namespace tweo_detail {
 
-bool chain_launch_enabled();  // TWEO_NO_LAUNCH_CHAIN=1 in the environment turns programmatic dependent launch off
-
-// Launches `kern` with `cluster` CTAs per cluster (0: none) and, when enabled, as a programmatic dependent of
-// the kernel before it on the stream (see chain_wait()).
+// Launches `kern` with `cluster` CTAs per cluster (0: none) as a programmatic dependent of the kernel before it
+// on the stream (see chain_wait()).
 template <typename... KArgs, typename... Args>
 cudaError_t launch_chain(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, unsigned cluster,
                          Args&&... args) {
@@ -54,11 +66,9 @@ cudaError_t launch_chain(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t s
     attr[n].val.clusterDim.z = 1;
     ++n;
   }
-  if (chain_launch_enabled()) {
-    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[n].val.programmaticStreamSerializationAllowed = 1;
-    ++n;
-  }
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
   cfg.attrs = attr;
   cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);

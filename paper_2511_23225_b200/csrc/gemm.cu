@@ -23,13 +23,12 @@
 // Scheduling.  Tiles are dealt round-robin to the CTAs.  When that would leave SMs idle
 // (fewer tiles than SMs, or a ragged last wave) and the contraction is long, the last
 // tiles are instead cut along the contraction ("stream-K"): their (tile, k-block) units
-// are split evenly over all CTAs.  A CTA whose share starts in the middle of a tile writes
-// its raw fp32 accumulator to a workspace slot and raises a flag; the CTA that owns the
-// tile's first k-block adds the other shares in CTA order (fixed order => reproducible)
-// and runs the epilogue.  Such a share is always the FIRST thing a CTA does and an owner's
-// wait is the LAST step of its stream-K work, so waits cannot form a cycle.
+// are split evenly over all CTAs.  Every share of such a tile parks its raw fp32 accumulator
+// in a workspace slot and takes a ticket; the share that draws the tile's last ticket adds
+// all of them in share order (fixed order => reproducible) and runs the epilogue
+// (gemm_split.cuh).  No CTA waits for another one.
 //
-// Every wait (mbarrier or flag) is bounded: on expiry the CTA records TWEO_ERR_TIMEOUT in
+// Every mbarrier wait is bounded: on expiry the CTA records TWEO_ERR_TIMEOUT in
 // a device status word, drains and exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -47,6 +46,7 @@
 #include "gemm_pair.cuh"
 #include "gemm_pair_group.cuh"
 #include "gemm_skinny.cuh"
+#include "gemm_split.cuh"
 #include "tc_ptx.cuh"
 
 namespace {
@@ -205,53 +205,17 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
-      if (kb0 > 0) {
-        // A share that does not own its tile: park the raw accumulator, raise the flag.
-        float* slot = p.sk_partials + (size_t)blockIdx.x * (BM * BN);
-#pragma unroll 1
-        for (int g = 0; g < BN / 32; ++g) {
-          uint32_t r[32];
-          tmem_ld32(tmem_base + tlane + (uint32_t)(acc * BN + g * 32), r);
-          tmem_ld_wait();
-          float* dst = slot + ((g * 4 + quarter) * 32) * 32 + lane;
-#pragma unroll
-          for (int k = 0; k < 32; ++k) __stcg(dst + k * 32, __uint_as_float(r[k]));
-        }
-        __threadfence();
-        __syncwarp();
-        if (lane == 0) st_release_u32(p.sk_flags + blockIdx.x * 4 + quarter, p.epoch);
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (kb0 != 0 || kb1 != p.k_blocks) {
+        // part of a split tile: park the accumulator; the last share to arrive stores the tile
+        const float part_amax = partial_share<BN, OUT_F32, false>(
+            p, &tmap_d, tile, kb0, (int)blockIdx.x, (int)gridDim.x, 0, quarter,
+            tmem_base + tlane + (uint32_t)(acc * BN), tempty_bar(acc), alpha, qs, epi_base, it, lane,
+            m0 + quarter * 32, n0);
+        it += BN / CH;  // keeps the staging-buffer rotation in step whether or not this warp stored
+        run_amax = fmaxf(run_amax, part_amax);
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
         continue;
-      }
-      int n_contrib = 0;
-      if (kb1 < p.k_blocks) {
-        // Owner of a tile whose later k-blocks went to the following CTAs: wait for them.
-        const int64_t tile_end = (int64_t)(tile + 1) * p.k_blocks;
-        for (int j = blockIdx.x + 1; j < (int)gridDim.x && Sched::share_begin(p, j, gridDim.x) < tile_end; ++j) {
-          const uint32_t* flag = p.sk_flags + j * 4 + quarter;
-          if (ld_acquire_u32(flag) != p.epoch) {
-            const uint64_t t0 = globaltimer_ns();
-            for (uint32_t spin = 1; ld_acquire_u32(flag) != p.epoch; ++spin) {
-              if ((spin & 0xFFu) == 0) {
-                if (*abort_flag) { ok = false; break; }
-                if (globaltimer_ns() - t0 > kWaitLimitNs) {
-                  *abort_flag = 1;
-                  atomicExch(&g_device_status, (unsigned int)TWEO_ERR_TIMEOUT);
-                  ok = false;
-                  break;
-                }
-              }
-            }
-          }
-          ok = __all_sync(0xFFFFFFFFu, ok);
-          if (!ok) break;
-          ++n_contrib;
-        }
-        if (!ok) break;
       }
       const int row0 = m0 + quarter * 32;
       const int row = row0 + lane;
@@ -265,16 +229,6 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         tmem_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
         if (!OUT_F32) tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[CH - 32]));
         tmem_ld_wait();
-        for (int jc = 0; jc < n_contrib; ++jc) {  // add the other shares, in CTA order
-          const float* part = p.sk_partials + (size_t)(blockIdx.x + 1 + jc) * (BM * BN);
-#pragma unroll
-          for (int h = 0; h < CH / 32; ++h) {
-            const float* src = part + (((c * (CH / 32) + h) * 4 + quarter) * 32) * 32 + lane;
-#pragma unroll
-            for (int k = 0; k < 32; ++k)
-              r[h * 32 + k] = __float_as_uint(__uint_as_float(r[h * 32 + k]) + __ldcg(src + k * 32));
-          }
-        }
         if (row0 >= p.Md) continue;  // whole warp past the ragged edge (uniform)
         const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
         // the store issued two chunks ago must have finished reading this buffer
@@ -360,6 +314,20 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 
 __global__ void zero_float_kernel(float* p) { *p = 0.0f; }
 
+// Self-test of the bounded wait: one thread waits on a barrier phase that nobody completes, with the
+// given limit; the wait gives up, records the expiry in the status word and the kernel returns.
+__global__ void bounded_wait_selftest_kernel(uint64_t limit_ns, unsigned int* gave_up) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait_limit(smem_u32(&bar), 0u, &abort_flag, limit_ns);
+    if (gave_up) *gave_up = ok ? 0u : 1u;
+  }
+}
+
 // ----------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -435,14 +403,6 @@ uint32_t make_idesc(int fmt_a, int fmt_b, bool a_mn, bool b_mn, int n, int m = B
   return d;
 }
 
-std::atomic<uint32_t> g_sk_epoch{0};
-// TWEO_GEMM_NO_PAIR=1 in the environment keeps every GEMM on the single-CTA kernel (A/B timing).
-// TWEO_GEMM_NO_SKINNY=1 sends small-M forward products through the general kernels (A/B timing).
-const bool g_disable_skinny = [] { const char* e = getenv("TWEO_GEMM_NO_SKINNY"); return e && e[0] == '1'; }();
-// TWEO_GEMM_NO_GROUP=1 makes tweo_fp8_linear_bwd run its two products as two launches (A/B timing).
-const bool g_disable_group = [] { const char* e = getenv("TWEO_GEMM_NO_GROUP"); return e && e[0] == '1'; }();
-const bool g_disable_pair = [] { const char* e = getenv("TWEO_GEMM_NO_PAIR"); return e && e[0] == '1'; }();
-
 // Band height of the tile numbering: the `workers` tiles in flight cover about g x workers/g
 // tiles, so g near sqrt(workers) keeps the rows of A and the columns of B they touch smallest.
 int raster_band(int tiles_m, int workers) {
@@ -457,10 +417,11 @@ tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
                          void* ws, size_t ws_bytes, cudaStream_t st) {
   constexpr size_t smem = (size_t)STAGES * (BM * BK + BN * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
   auto kern = gemm_fp8_kernel<BN, A_MN, B_MN, STAGES, OUT_F32>;
-  static bool attr_done = false;  // per instantiation
-  if (!attr_done) {
+  static std::atomic<uint64_t> attr_done{0};  // per device
+  int attr_dev = 0;
+  if (device_once_pending(attr_done, &attr_dev)) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_done = true;
+    device_once_done(attr_done, attr_dev);
   }
   p.tiles_m = (p.Md + BM - 1) / BM;
   p.tiles_n = (p.Nd + BN - 1) / BN;
@@ -471,9 +432,7 @@ tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
   p.raster_g = raster_band(p.tiles_m, sms);
   p.sk_tiles = 0;
   p.sk_partials = nullptr;
-  p.sk_flags = nullptr;
   p.sk_counters = nullptr;
-  p.epoch = 0;
   // Stream-K when whole-tile dealing would idle more than ~15 % of the SM-time and the
   // contraction is long enough to pay for the fix-up (a 128 x BN fp32 round trip through L2).
   const size_t sk_need = kWsPartialsOffset + (size_t)sms * kWsPartialBytesPerSm;
@@ -482,11 +441,13 @@ tweo_status_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
       (double)tiles < 0.85 * (double)waves * sms) {
     const int full = tiles / sms;
     p.sk_tiles = full == 0 ? tiles : tiles - (full - 1) * sms;
+    if ((size_t)p.sk_tiles * 4 * sizeof(uint32_t) > kWsPartialsOffset - kWsCountersOffset) p.sk_tiles = 0;  // counters
+  }
+  if (p.sk_tiles > 0) {
     grid = sms;
     if ((int64_t)p.sk_tiles * p.k_blocks < grid) grid = (int)((int64_t)p.sk_tiles * p.k_blocks);
-    p.sk_flags = reinterpret_cast<uint32_t*>(ws);
+    p.sk_counters = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + kWsCountersOffset);
     p.sk_partials = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + kWsPartialsOffset);
-    p.epoch = g_sk_epoch.fetch_add(1, std::memory_order_relaxed) + 1;
   }
   kern<<<grid, kThreads, smem, st>>>(ma, mb, md, p);
   count_launch();
@@ -512,21 +473,21 @@ tweo_status_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CU
                           void* ws, size_t ws_bytes, cudaStream_t st) {
   constexpr int STAGES = 6;
   constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
+  if (p.out_amax || p.out_q) return TWEO_ERR_INVALID_ARG;  // fused outputs belong to the staged instantiations
   auto kern = gemm_fp8_pair_kernel<A_MN, B_MN, STAGES, OUT_F32>;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static std::atomic<uint64_t> attr_done{0};  // per device
+  int attr_dev = 0;
+  if (device_once_pending(attr_done, &attr_dev)) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 0));
-    attr_done = true;
+    device_once_done(attr_done, attr_dev);
   }
   p.tiles_m = (p.Md + 2 * BM - 1) / (2 * BM);
   p.tiles_n = (p.Nd + 255) / 256;
   p.k_blocks = (p.Kc + BK - 1) / BK;
   p.sk_tiles = 0;
   p.sk_partials = nullptr;
-  p.sk_flags = nullptr;
   p.sk_counters = nullptr;
-  p.epoch = 0;
   const int tiles = p.tiles_m * p.tiles_n;
   const int sms = sm_count();
   int pairs = sms / 2;
@@ -564,7 +525,7 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
   p.Kc = (int32_t)Kc;
   const int BN = Nd > 128 ? 256 : 128;
   // CTA pairs (256 x 256 tiles) whenever the output has more than one 128-row block and is wide enough
-  const bool use_pair = Md > 128 && Nd > 128 && !g_disable_pair;
+  const bool use_pair = Md > 128 && Nd > 128;
   p.idesc = use_pair ? make_idesc(A.fmt, B.fmt, A.mn_major, B.mn_major, 256, 256)
                      : make_idesc(A.fmt, B.fmt, A.mn_major, B.mn_major, BN);
 
@@ -608,7 +569,7 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
 
 // Forward product with the MLP activation and / or the FP8 copy of the output in the epilogue (pair
 // kernel only; every tile whole; the FP8 copy staged through shared memory, hence 5 stages).
-template <int ACT>
+template <int ACT, bool B_MN = false>
 tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
                               const CUtensorMap& mq, GemmParams& p, cudaStream_t st) {
   // the per-element epilogues run with eight epilogue warps and four operand stages; SwiGLU (long
@@ -617,20 +578,19 @@ tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, cons
   constexpr int STAGES = ACT == 3 ? 5 : 4;
   constexpr int THREADS = 64 + 32 * EPIW;
   constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + EPIW * 2 * 32 * 128 + EPIW * 2 * 32 * 64 + 1024 + 256;
-  auto kern = gemm_fp8_pair_kernel<false, false, STAGES, false, false, ACT, true, EPIW>;
-  static bool attr_done = false;
-  if (!attr_done) {
+  auto kern = gemm_fp8_pair_kernel<false, B_MN, STAGES, false, false, ACT, true, EPIW>;
+  static std::atomic<uint64_t> attr_done{0};  // per device
+  int attr_dev = 0;
+  if (device_once_pending(attr_done, &attr_dev)) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_done = true;
+    device_once_done(attr_done, attr_dev);
   }
   p.tiles_m = (p.Md + 2 * BM - 1) / (2 * BM);
   p.tiles_n = ACT == 3 ? (p.Nd + 127) / 128 : (p.Nd + 255) / 256;
   p.k_blocks = (p.Kc + BK - 1) / BK;
   p.sk_tiles = 0;
   p.sk_partials = nullptr;
-  p.sk_flags = nullptr;
   p.sk_counters = nullptr;
-  p.epoch = 0;
   const int tiles = p.tiles_m * p.tiles_n;
   int pairs = sm_count() / 2;
   p.raster_g = raster_band(p.tiles_m, pairs);
@@ -652,23 +612,27 @@ tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, cons
   return check_launch("gemm_fp8_pair_kernel (activation epilogue)");
 }
 
-// N: output columns.  SwiGLU: wq has 2 N rows (gate rows, then up rows).
+// D[M,N] = A[M,K] . B with A stored [M,K]; B stored [N,K] (w_mn false: the forward product) or [K,N] (w_mn
+// true: the data gradient, which reads the weight in its forward layout; plain epilogue only).
+// N: output columns, K: contraction.  SwiGLU: wq has 2 N rows (gate rows, then up rows).
 tweo_status_t run_fwd_act(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
-                          int act, int64_t M, int64_t N, int64_t K, GemmParams p, cudaStream_t st) {
+                          bool w_mn, int act, int64_t M, int64_t N, int64_t K, GemmParams p, cudaStream_t st) {
+  if (w_mn && act != TWEO_ACT_NONE) return TWEO_ERR_INVALID_ARG;
   if (M > INT32_MAX || 2 * N > INT32_MAX || K > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
   if (!aligned16(xq) || !aligned16(wq) || !aligned16(p.d) || (ldx & 15) || (ldw & 15) || ((p.ldd * 2) & 15))
     return TWEO_ERR_ALIGNMENT;
   p.Md = (int32_t)M;
   p.Nd = (int32_t)N;
   p.Kc = (int32_t)K;
-  p.idesc = make_idesc(fmt_x, fmt_w, false, false, 256, 256);
+  p.idesc = make_idesc(fmt_x, fmt_w, false, w_mn, 256, 256);
   CUtensorMap ma, mb, md, mq;
   // without a bf16 output the store is skipped; the map then describes the FP8 output's memory and is never used
   bool ok = p.d ? make_out_map(&md, p.d, N, M, p.ldd, false) : make_out_map(&md, p.out_q, N / 2, M, p.ldq / 2, false);
   if (p.out_q) ok = ok && make_q_map(&mq, p.out_q, N, M, p.ldq);
   else mq = md;
   ok = ok && make_map(&ma, xq, K, M, ldx, BM);
-  ok = ok && make_map(&mb, wq, K, act == TWEO_ACT_SWIGLU ? 2 * N : N, ldw, 128);
+  if (w_mn) ok = ok && make_map(&mb, wq, N, K, ldw, BK);
+  else ok = ok && make_map(&mb, wq, K, act == TWEO_ACT_SWIGLU ? 2 * N : N, ldw, 128);
   if (!ok) {
     cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
     return TWEO_ERR_CUDA;
@@ -678,7 +642,8 @@ tweo_status_t run_fwd_act(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8
     count_launch();
   }
   switch (act) {
-    case TWEO_ACT_NONE: return launch_pair_act<0>(ma, mb, md, mq, p, st);
+    case TWEO_ACT_NONE:
+      return w_mn ? launch_pair_act<0, true>(ma, mb, md, mq, p, st) : launch_pair_act<0>(ma, mb, md, mq, p, st);
     case TWEO_ACT_GELU: return launch_pair_act<1>(ma, mb, md, mq, p, st);
     case TWEO_ACT_GELU_TANH: return launch_pair_act<2>(ma, mb, md, mq, p, st);
     case TWEO_ACT_SWIGLU: return launch_pair_act<3>(ma, mb, md, mq, p, st);
@@ -720,11 +685,12 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
     return TWEO_ERR_CUDA;
   }
   const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static std::atomic<uint64_t> attr_done{0};  // per device
+  int attr_dev = 0;
+  if (device_once_pending(attr_done, &attr_dev)) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(gemm_fp8_skinny_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)(200 * 1024 + 1024 + 256)));
-    attr_done = true;
+    device_once_done(attr_done, attr_dev);
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(slabs * p.slices));
@@ -751,10 +717,11 @@ tweo_status_t run_bwd_group(const uint8_t* dyq, int64_t lddy, int fmt_dy, const 
   constexpr int STAGES = 6;
   constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
   auto kern = gemm_fp8_pair_group_kernel<STAGES>;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static std::atomic<uint64_t> attr_done{0};  // per device
+  int attr_dev = 0;
+  if (device_once_pending(attr_done, &attr_dev)) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_done = true;
+    device_once_done(attr_done, attr_dev);
   }
   const int pairs_all = sm_count() / 2;
   PairGroupParams g;
@@ -884,7 +851,7 @@ tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const ui
                              int64_t N, int64_t K, const tweo_epilogue_t* epi, void* ws, size_t ws_bytes,
                              cudaStream_t st) {
   const bool fused = epi && (epi->out_amax || epi->out_q);
-  if (M <= 128 && !fused && !g_disable_skinny)  // few tokens: stream W once, tokens on the MMA's N side
+  if (M <= 128 && !fused)  // few tokens: stream W once, tokens on the MMA's N side
     return run_skinny(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, y, ldy, M, N, K, ws, ws_bytes, st);
   GemmParams p{};
   p.d = y;
@@ -893,8 +860,8 @@ tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const ui
   p.sb_inv = sw_inv;
   tweo_status_t s = fill_epilogue(p, epi);
   if (s != TWEO_OK) return s;
-  if (fused && M > 128 && N > 128 && !g_disable_pair)  // extra outputs leave through shared memory and TMA
-    return run_fwd_act(xq, ldx, fmt_x, wq, ldw, fmt_w, TWEO_ACT_NONE, M, N, K, p, st);
+  if (fused && M > 128 && N > 128)  // extra outputs leave through shared memory and TMA
+    return run_fwd_act(xq, ldx, fmt_x, wq, ldw, fmt_w, false, TWEO_ACT_NONE, M, N, K, p, st);
   return run_gemm(Operand{xq, ldx, fmt_x, false}, Operand{wq, ldw, fmt_w, false}, M, N, K, p, ws, ws_bytes, st);
 }
 
@@ -916,11 +883,12 @@ tweo_status_t run_int8_linear(const int8_t* xq, int64_t ldx, const float* sx, in
   constexpr size_t smem5q = (size_t)5 * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 4 * 2 * 32 * 64 + 1024 + 256;
   auto kern_bf16 = gemm_fp8_pair_kernel<false, false, 6, false, true>;
   auto kern_q8 = gemm_fp8_pair_kernel<false, false, 5, false, true, 0, true>;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static std::atomic<uint64_t> attr_done{0};  // per device
+  int attr_dev = 0;
+  if (device_once_pending(attr_done, &attr_dev)) {
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem6));
     TWEO_CUDA_TRY(cudaFuncSetAttribute(kern_q8, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem5q));
-    attr_done = true;
+    device_once_done(attr_done, attr_dev);
   }
   GemmParams p{};
   p.d = y;
@@ -1007,7 +975,7 @@ tweo_status_t tweo_fp8_linear_fwd_act(const uint8_t* xq, int64_t ldx, const uint
   p.sb_inv = sw_inv;
   tweo_status_t s = fill_epilogue(p, epi);
   if (s != TWEO_OK) return s;
-  return run_fwd_act(xq, ldx, fmt_x, wq, ldw, fmt_w, act, M, N, K, p, (cudaStream_t)stream);
+  return run_fwd_act(xq, ldx, fmt_x, wq, ldw, fmt_w, false, act, M, N, K, p, (cudaStream_t)stream);
 }
 
 tweo_status_t tweo_fp8_linear_bwd_dgrad(const uint8_t* dyq, int64_t lddy, int32_t fmt_dy, const uint8_t* wq,
@@ -1025,6 +993,8 @@ tweo_status_t tweo_fp8_linear_bwd_dgrad(const uint8_t* dyq, int64_t lddy, int32_
   tweo_status_t s = fill_epilogue(p, epi);
   if (s != TWEO_OK) return s;
   // dX[M,K] = dYq[M,N] . Wq[N,K]: contraction over N; Wq is stored [N(contraction), K(out)] = MN-major
+  if (epi && (epi->out_amax || epi->out_q) && M > 128 && K > 128)  // extra outputs leave through shared memory and TMA
+    return run_fwd_act(dyq, lddy, fmt_dy, wq, ldw, fmt_w, true, TWEO_ACT_NONE, M, K, N, p, (cudaStream_t)stream);
   return run_gemm(Operand{dyq, lddy, fmt_dy, false}, Operand{wq, ldw, fmt_w, true}, M, K, N, p, ws, ws_bytes,
                   (cudaStream_t)stream);
 }
@@ -1066,7 +1036,7 @@ tweo_status_t tweo_fp8_linear_bwd(const uint8_t* dyq, int64_t lddy, int32_t fmt_
       (lddx & 7) || (lddw & 7))
     return TWEO_ERR_ALIGNMENT;
   // both outputs large enough for 256 x 256 tiles: one launch; else the two products one after the other
-  if (M > 128 && N > 128 && K > 128 && !g_disable_pair && !g_disable_group)
+  if (M > 128 && N > 128 && K > 128)
     return run_bwd_group(dyq, lddy, fmt_dy, xq, ldx, fmt_x, wq, ldw, fmt_w, sdy_inv, sx_inv, sw_inv, dx, lddx, dw, lddw,
                          M, N, K, (cudaStream_t)stream);
   tweo_status_t s = tweo_fp8_linear_bwd_dgrad(dyq, lddy, fmt_dy, wq, ldw, fmt_w, sdy_inv, sw_inv, dx, lddx, M, N, K,
@@ -1074,6 +1044,13 @@ tweo_status_t tweo_fp8_linear_bwd(const uint8_t* dyq, int64_t lddy, int32_t fmt_
   if (s != TWEO_OK) return s;
   return tweo_fp8_linear_bwd_wgrad(xq, ldx, fmt_x, dyq, lddy, fmt_dy, sx_inv, sdy_inv, dw, lddw, TWEO_BF16, 0, M, N, K,
                                    ws, ws_bytes, stream);
+}
+
+tweo_status_t tweo_selftest_bounded_wait(uint64_t limit_ns, uint32_t* gave_up, void* stream) {
+  if (limit_ns < 1000ull || limit_ns > 100000000ull) return TWEO_ERR_INVALID_ARG;  // 1 us .. 100 ms
+  bounded_wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(limit_ns, gave_up);
+  tweo_detail::count_launch();
+  return tweo_detail::check_launch("bounded_wait_selftest_kernel");
 }
 
 tweo_status_t tweo_int8_linear(const int8_t* xq, int64_t ldx, const float* sx, int32_t sx_per_row, const int8_t* wq,

@@ -38,15 +38,13 @@ struct GemmParams {
   float q8_qmax;           // Q_b of an 8-bit (Eq. 4) output; its static scale is read from q_scale
   // stream-K: tiles [0, sk_tiles) are split along the contraction, the rest dealt whole
   int32_t sk_tiles;
-  float* sk_partials;   // [grid][BM*BN] raw accumulators of shares that do not own their tile
-  uint32_t* sk_flags;   // [grid][4] per epilogue warp: == epoch once the share is written
-  uint32_t* sk_counters;  // CTA-pair kernel: [sk_tiles][2][4] tickets per (tile, CTA of the pair, epilogue warp)
-  uint32_t epoch;
+  float* sk_partials;   // parked raw accumulators of the shares of split tiles: two slots per worker
+  uint32_t* sk_counters;  // tickets per (tile, CTA of the pair, epilogue warp): [sk_tiles][2][4], single CTA [sk_tiles][4]
 };
 
 // Workspace layout of the linear calls (bytes from the workspace base):
-//   [0, 4096)       flags of the single-CTA kernel's split tiles (4 words per CTA)
-//   [4096, 12288)   ticket counters of the CTA-pair kernel's split tiles (8 words per tile)
+//   [0, 4096)       unused
+//   [4096, 12288)   ticket counters of the split tiles (CTA-pair kernel 8 words per tile, single-CTA kernel 4)
 //   [12288, ...)    parked fp32 accumulators: 256 KB per SM
 constexpr size_t kWsCountersOffset = 4096;
 constexpr size_t kWsPartialsOffset = 12288;

@@ -16,133 +16,10 @@
 #include <cuda.h>
 
 #include "gemm_common.cuh"
+#include "gemm_split.cuh"
 #include "tc_ptx.cuh"
 
 namespace tweo_detail {
-
-// A share of the pair kernel that covers only part of a split tile.  Parks this warp's
-// 32 x 256 block of the raw accumulator in the workspace ([column][row], so every store is
-// one full line), hands the accumulator back to the MMA warp and takes a ticket; the warp
-// that draws the last ticket of the tile adds the parked blocks of ALL shares in share order
-// (= ascending k, whoever arrived last, so the sum does not depend on timing) and stores the
-// result.  Nobody waits for anybody.  Kept out of line: it is rare and register-hungry.
-constexpr size_t kPairCtaFloats = 128 * 256;   // one CTA's half of a parked 256 x 256 accumulator
-constexpr size_t kPairWarpFloats = 32 * 256;   // one epilogue warp's block of it
-
-template <bool OUT_F32>
-__device__ __noinline__ float pair_partial_share(const GemmParams& p, const CUtensorMap* tmap_d, int tile, int kb0,
-                                                int pair, int num_pairs, int rank, int wslot,
-                                                uint32_t tacc, uint32_t tempty_leader, float alpha, float qs,
-                                                uint32_t epi_base, uint32_t it, int lane, int row0, int n0) {
-  constexpr int CH = OUT_F32 ? 32 : 64;
-  constexpr uint32_t EPI_BUF = 32 * 128;
-  float run_amax = 0.0f;
-  float* slot = p.sk_partials + ((size_t)(pair * 2 + (kb0 > 0 ? 0 : 1)) * 2 + rank) * kPairCtaFloats +
-                (size_t)wslot * kPairWarpFloats;
-#pragma unroll 1
-  for (int g = 0; g < 8; ++g) {
-    uint32_t r[32];
-    tmem_ld32(tacc + (uint32_t)(g * 32), r);
-    tmem_ld_wait();
-    float* dst = slot + g * 1024 + lane;
-#pragma unroll
-    for (int k = 0; k < 32; ++k) __stcg(dst + k * 32, __uint_as_float(r[k]));
-  }
-  tc_fence_before();
-  __syncwarp();
-  if (lane == 0) mbar_arrive_cluster(tempty_leader);
-  // which pairs hold a share of this tile (they are consecutive)
-  const int64_t t_begin = (int64_t)tile * p.k_blocks, t_end = t_begin + p.k_blocks;
-  int j_first = pair;
-  while (j_first > 0 && Sched::share_begin(p, j_first, num_pairs) > t_begin) --j_first;
-  int j_last = pair;
-  while (j_last + 1 < num_pairs && Sched::share_begin(p, j_last + 1, num_pairs) < t_end) ++j_last;
-  const int n_shares = j_last - j_first + 1;
-  __threadfence();
-  __syncwarp();
-  uint32_t ticket = 0;
-  uint32_t* counter = p.sk_counters + ((size_t)tile * 2 + rank) * 4 + wslot;
-  if (lane == 0) ticket = atomicAdd(counter, 1u);
-  ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
-  if (ticket + 1 != (uint32_t)n_shares) return 0.0f;  // not the last share of this tile: done
-  __threadfence();
-  if (lane == 0) *counter = 0u;  // ready for the next launch
-  const uint32_t row_off = (uint32_t)lane * 128u;
-  const uint32_t swz = (uint32_t)(lane & 7);
-  const int row = row0 + lane;
-#pragma unroll 1
-  for (int c = 0; c < 256 / CH; ++c) {
-    const int col0 = n0 + c * CH;
-    if (col0 >= p.Nd || row0 >= p.Md) break;  // uniform across the warp
-    uint32_t r[CH];
-#pragma unroll 1
-    for (int sidx = 0; sidx < n_shares; ++sidx) {
-      const int j = j_first + sidx;
-      const int sel = Sched::share_begin(p, j, num_pairs) > t_begin ? 0 : 1;
-      const float* src = p.sk_partials + ((size_t)(j * 2 + sel) * 2 + rank) * kPairCtaFloats +
-                         (size_t)wslot * kPairWarpFloats + (size_t)(c * CH) * 32 + lane;
-      if (sidx == 0) {
-#pragma unroll
-        for (int k = 0; k < CH; ++k) r[k] = __float_as_uint(__ldcg(src + k * 32));
-      } else {
-#pragma unroll
-        for (int k = 0; k < CH; ++k) r[k] = __float_as_uint(__uint_as_float(r[k]) + __ldcg(src + k * 32));
-      }
-    }
-    const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
-    ++it;
-    if (lane == 0) bulk_wait_read<1>();
-    __syncwarp();
-    if (OUT_F32) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4),
-                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j]), alpha)),
-                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 1]), alpha)),
-                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 2]), alpha)),
-                     __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 3]), alpha)));
-    } else {
-      uint32_t packed[CH / 2];
-#pragma unroll
-      for (int j = 0; j < CH / 2; ++j)
-        packed[j] = f32x2_to_bf16x2(__fmul_rn(__uint_as_float(r[2 * j]), alpha),
-                                    __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha));
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1], packed[4 * j + 2],
-                     packed[4 * j + 3]);
-      if ((p.out_amax || p.out_q) && row < p.Md) {
-#pragma unroll 1
-        for (int j = 0; j < CH / 4; ++j) {  // groups of four columns
-          const uint32_t w0 = packed[2 * j], w1 = packed[2 * j + 1];
-          float v[4] = {bf16lo_to_f32(w0), bf16hi_to_f32(w0), bf16lo_to_f32(w1), bf16hi_to_f32(w1)};
-          if (col0 + 4 * j < p.Nd) {
-            run_amax = fmaxf(run_amax, fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))));
-            if (p.out_q) {
-              const uint32_t q = p.q_fmt == TWEO_E4M3
-                                     ? quant4<TWEO_E4M3>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs),
-                                                         __fmul_rn(v[2], qs), __fmul_rn(v[3], qs))
-                                     : quant4<TWEO_E5M2>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs),
-                                                         __fmul_rn(v[2], qs), __fmul_rn(v[3], qs));
-              *reinterpret_cast<uint32_t*>(p.out_q + (int64_t)row * p.ldq + col0 + 4 * j) = q;
-            }
-          }
-        }
-      }
-    }
-    fence_async_smem();
-    __syncwarp();
-    if (lane == 0) {
-      if (OUT_F32 && p.accumulate) tma_reduce_add_2d(tmap_d, col0, row0, buf);
-      else tma_store_2d(tmap_d, col0, row0, buf);
-      bulk_commit();
-    }
-  }
-  // the caller's buffer rotation does not know how many chunks were stored here
-  if (lane == 0) bulk_wait_read<0>();
-  __syncwarp();
-  return run_amax;
-}
 
 // I8: the operands are 8-bit integers (tcgen05 kind::i8, int32 accumulators) and the epilogue
 // applies the Eq. 4 dequantisation with one scale per tensor or per row / column.
@@ -321,7 +198,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       const bool row_ok = row < p.Md;
       if (ACT == 0 && (kb0 != 0 || kb1 != p.k_blocks)) {
         // part of a split tile: park the accumulator; the last share to arrive stores the tile
-        const float part_amax = pair_partial_share<OUT_F32>(
+        const float part_amax = partial_share<BN, OUT_F32, true>(
             p, &tmap_d, tile, kb0, pair, num_pairs, (int)rank, warp - 2,
             tmem_base + tlane + (uint32_t)(acc * BN), map_to_cta(tempty_bar(acc), 0), alpha, qs, epi_base, it, lane,
             row0, n0);
@@ -457,33 +334,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                 st_shared_v4(qrow + (((uint32_t)g4 ^ qswz) << 4), q[0], q[1], q[2], q[3]);
               }
             }
-          } else
-          if ((p.out_amax || p.out_q) && row_ok) {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              uint32_t q[8];
-#pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                const uint32_t w0 = packed[16 * h + 2 * j], w1 = packed[16 * h + 2 * j + 1];
-                float v[4] = {bf16lo_to_f32(w0), bf16hi_to_f32(w0), bf16lo_to_f32(w1), bf16hi_to_f32(w1)};
-                if (col0 + 32 * h + 4 * j < p.Nd)
-                  run_amax = fmaxf(run_amax, fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))));
-                if (p.out_q) {
-                  if (p.q_fmt == TWEO_E4M3)
-                    q[j] = quant4<TWEO_E4M3>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
-                                             __fmul_rn(v[3], qs));
-                  else
-                    q[j] = quant4<TWEO_E5M2>(__fmul_rn(v[0], qs), __fmul_rn(v[1], qs), __fmul_rn(v[2], qs),
-                                             __fmul_rn(v[3], qs));
-                }
-              }
-              if (p.out_q) {
-                uint8_t* qrow = p.out_q + (int64_t)row * p.ldq + col0 + 32 * h;
-                if (col0 + 32 * h < p.Nd) *reinterpret_cast<uint4*>(qrow) = make_uint4(q[0], q[1], q[2], q[3]);
-                if (col0 + 32 * h + 16 < p.Nd) *reinterpret_cast<uint4*>(qrow + 16) = make_uint4(q[4], q[5], q[6], q[7]);
-              }
-            }
           }
+          // (without QST the kernel has no fused outputs: the host sends those products to a QST instantiation)
         }
         fence_async_smem();
         __syncwarp();

@@ -217,33 +217,33 @@ void launch(dim3 grid, cudaStream_t st, const LossPtrs& ptrs, const LossArgs& ar
   tweo_loss_kernel<FAST, GRAD, GRAD_F32><<<grid, kLossThreads, 0, st>>>(ptrs, args);
 }
 
-}  // namespace
-
-extern "C" tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, int64_t n_per_tensor, float tau,
-                                           float eps, float p, float grad_coeff, float* loss,
-                                           float* loss_per_block, void* const* grad, int32_t grad_dtype,
-                                           void* ws, size_t ws_bytes, void* stream) {
+// Argument checks, kernel arguments and launch shared by the two entry points; they differ only in where the
+// scratch memory (ticket counter at byte 0, partial sums from byte 256) lives.
+tweo_status_t check_loss_args(const uint16_t* const* a, int32_t L, int64_t n_per_tensor, float tau, float eps, float p,
+                              const float* loss, void* const* grad, int32_t grad_dtype) {
   if (!a || !loss || L < 1 || L > TWEO_MAX_BLOCKS || n_per_tensor < 0) return TWEO_ERR_INVALID_ARG;
   if (!(p > 1.0f) || !(tau + eps > 0.0f)) return TWEO_ERR_INVALID_ARG;
   if (grad && grad_dtype != TWEO_BF16 && grad_dtype != TWEO_F32) return TWEO_ERR_INVALID_ARG;
-  const size_t need = tweo_workspace_bytes(TWEO_OP_LOSS, n_per_tensor, L, 0);
-  if (!ws || ws_bytes < need) return TWEO_ERR_WORKSPACE_TOO_SMALL;
-  if (!aligned16(ws)) return TWEO_ERR_ALIGNMENT;
-
-  LossPtrs ptrs;
   for (int l = 0; l < L; ++l) {
     if (!a[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
     if (!aligned16(a[l])) return TWEO_ERR_ALIGNMENT;
-    ptrs.a[l] = a[l];
-    ptrs.g[l] = nullptr;
     if (grad) {
       if (!grad[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
       if (!aligned16(grad[l])) return TWEO_ERR_ALIGNMENT;
       if (grad_dtype == TWEO_F32 && grad[l] == (const void*)a[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
-      ptrs.g[l] = grad[l];
     }
   }
+  return TWEO_OK;
+}
 
+tweo_status_t launch_loss(const uint16_t* const* a, int32_t L, int64_t n_per_tensor, float tau, float eps, float p,
+                          float grad_coeff, float* loss, float* loss_per_block, void* const* grad, int32_t grad_dtype,
+                          void* scratch, int blocks_per_tensor, cudaStream_t st, const char* what) {
+  LossPtrs ptrs;
+  for (int l = 0; l < L; ++l) {
+    ptrs.a[l] = a[l];
+    ptrs.g[l] = grad ? grad[l] : nullptr;
+  }
   LossArgs args;
   args.n = n_per_tensor;
   args.L = L;
@@ -254,11 +254,10 @@ extern "C" tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, 
   args.k_grad = n_per_tensor > 0 ? (float)((double)grad_coeff * (double)p / norm) : 0.0f;
   args.loss = loss;
   args.loss_per_block = loss_per_block;
-  args.ticket = reinterpret_cast<unsigned int*>(ws);
-  args.partials = reinterpret_cast<double*>(reinterpret_cast<char*>(ws) + 256);
+  args.ticket = reinterpret_cast<unsigned int*>(scratch);
+  args.partials = reinterpret_cast<double*>(reinterpret_cast<char*>(scratch) + 256);
 
-  dim3 grid((unsigned)tweo_detail::loss_blocks_per_tensor(n_per_tensor, L), (unsigned)L);
-  cudaStream_t st = (cudaStream_t)stream;
+  dim3 grid((unsigned)blocks_per_tensor, (unsigned)L);
   const bool fast = (p == 4.0f);
   const bool has_grad = grad != nullptr;
   const bool f32 = grad_dtype == TWEO_F32;
@@ -272,7 +271,22 @@ extern "C" tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, 
     else launch<false, true, false>(grid, st, ptrs, args);
   }
   tweo_detail::count_launch();
-  return tweo_detail::check_launch("tweo_loss_kernel");
+  return tweo_detail::check_launch(what);
+}
+
+}  // namespace
+
+extern "C" tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, int64_t n_per_tensor, float tau,
+                                           float eps, float p, float grad_coeff, float* loss,
+                                           float* loss_per_block, void* const* grad, int32_t grad_dtype,
+                                           void* ws, size_t ws_bytes, void* stream) {
+  tweo_status_t s = check_loss_args(a, L, n_per_tensor, tau, eps, p, loss, grad, grad_dtype);
+  if (s != TWEO_OK) return s;
+  const size_t need = tweo_workspace_bytes(TWEO_OP_LOSS, n_per_tensor, L, 0);
+  if (!ws || ws_bytes < need) return TWEO_ERR_WORKSPACE_TOO_SMALL;
+  if (!aligned16(ws)) return TWEO_ERR_ALIGNMENT;
+  return launch_loss(a, L, n_per_tensor, tau, eps, p, grad_coeff, loss, loss_per_block, grad, grad_dtype, ws,
+                     tweo_detail::loss_blocks_per_tensor(n_per_tensor, L), (cudaStream_t)stream, "tweo_loss_kernel");
 }
 
 // ---------------------------------------------------------------------------------------
@@ -315,62 +329,19 @@ extern "C" tweo_status_t tweo_loss_fwd_bwd_static(const uint16_t* const* a, int3
                                                   float tau, float eps, float p, float grad_coeff, float* loss,
                                                   float* loss_per_block, void* const* grad, int32_t grad_dtype,
                                                   void* stream) {
-  if (!a || !loss || L < 1 || L > TWEO_MAX_BLOCKS || n_per_tensor < 0) return TWEO_ERR_INVALID_ARG;
-  if (!(p > 1.0f) || !(tau + eps > 0.0f)) return TWEO_ERR_INVALID_ARG;
-  if (grad && grad_dtype != TWEO_BF16 && grad_dtype != TWEO_F32) return TWEO_ERR_INVALID_ARG;
+  tweo_status_t s = check_loss_args(a, L, n_per_tensor, tau, eps, p, loss, grad, grad_dtype);
+  if (s != TWEO_OK) return s;
   const int blocks = tweo_detail::loss_blocks_per_tensor(n_per_tensor, L);
   if ((size_t)blocks * (size_t)L > kStaticPartials) {
     // more partial sums than the built-in scratch holds: use tweo_loss_fwd_bwd with a workspace
     return TWEO_ERR_WORKSPACE_TOO_SMALL;
   }
-
-  LossPtrs ptrs;
-  for (int l = 0; l < L; ++l) {
-    if (!a[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
-    if (!aligned16(a[l])) return TWEO_ERR_ALIGNMENT;
-    ptrs.a[l] = a[l];
-    ptrs.g[l] = nullptr;
-    if (grad) {
-      if (!grad[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
-      if (!aligned16(grad[l])) return TWEO_ERR_ALIGNMENT;
-      if (grad_dtype == TWEO_F32 && grad[l] == (const void*)a[l] && n_per_tensor > 0) return TWEO_ERR_INVALID_ARG;
-      ptrs.g[l] = grad[l];
-    }
-  }
-
   void* scratch = nullptr;
-  tweo_status_t s = static_scratch_for_current_device(&scratch);
+  s = static_scratch_for_current_device(&scratch);
   if (s != TWEO_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
   // The array keeps whatever the previous call left; the ticket counter must start at zero.
   TWEO_CUDA_TRY(cudaMemsetAsync(scratch, 0, 256, st));
-
-  LossArgs args;
-  args.n = n_per_tensor;
-  args.L = L;
-  args.p = p;
-  const double d = (double)tau + (double)eps;
-  const double norm = (double)n_per_tensor * pow(d, (double)p);
-  args.inv_norm = n_per_tensor > 0 ? 1.0 / norm : 0.0;
-  args.k_grad = n_per_tensor > 0 ? (float)((double)grad_coeff * (double)p / norm) : 0.0f;
-  args.loss = loss;
-  args.loss_per_block = loss_per_block;
-  args.ticket = reinterpret_cast<unsigned int*>(scratch);
-  args.partials = reinterpret_cast<double*>(reinterpret_cast<char*>(scratch) + 256);
-
-  dim3 grid((unsigned)blocks, (unsigned)L);
-  const bool fast = (p == 4.0f);
-  const bool has_grad = grad != nullptr;
-  const bool f32 = grad_dtype == TWEO_F32;
-  if (fast) {
-    if (!has_grad) launch<true, false, false>(grid, st, ptrs, args);
-    else if (f32) launch<true, true, true>(grid, st, ptrs, args);
-    else launch<true, true, false>(grid, st, ptrs, args);
-  } else {
-    if (!has_grad) launch<false, false, false>(grid, st, ptrs, args);
-    else if (f32) launch<false, true, true>(grid, st, ptrs, args);
-    else launch<false, true, false>(grid, st, ptrs, args);
-  }
-  tweo_detail::count_launch();
-  return tweo_detail::check_launch("tweo_loss_kernel (static scratch)");
+  return launch_loss(a, L, n_per_tensor, tau, eps, p, grad_coeff, loss, loss_per_block, grad, grad_dtype, scratch,
+                     blocks, st, "tweo_loss_kernel (static scratch)");
 }

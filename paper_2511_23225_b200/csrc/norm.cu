@@ -170,11 +170,12 @@ __global__ void __launch_bounds__(kNormThreads) norm_rows_kernel(const NormArgs 
 
 template <int VPL, int QFMT>
 cudaError_t launch_norm_q(const NormArgs& a, int64_t want_ctas, size_t smem, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {  // gamma and beta of the widest row take 64 KB
+  static std::atomic<uint64_t> attr_done{0};  // per device
+  int attr_dev = 0;
+  if (device_once_pending(attr_done, &attr_dev)) {  // gamma and beta of the widest row take 64 KB
     cudaError_t e = cudaFuncSetAttribute(norm_rows_kernel<VPL, QFMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    device_once_done(attr_done, attr_dev);
   }
   // persistent grid: as many CTAs as are resident at once
   int per_sm = 0;

@@ -463,7 +463,7 @@ def test_forward_few_tokens_streams_w(tw, M, K, N, with_ws):
 
 # ------------------------------------------------------------------ static W8A8
 @pytest.mark.parametrize("K,N", [(4096, 4096), (4096, 11008), (11008, 4096)], ids=["4096x4096", "4096x11008", "11008x4096"])
-@pytest.mark.parametrize("M", [1, 16, 128, 1024])
+@pytest.mark.parametrize("M", [1, 16, 128, 1024, 8192])
 def test_w8a8_static_gemm(tw, M, K, N):
     w = synth.w8a8_weight(K, N)
     qw = orc.quantize_per_tensor_current(w, E4M3)

@@ -38,7 +38,8 @@ def at(t: torch.Tensor, r, c) -> np.ndarray:
     return t[ri, ci].float().cpu().numpy().astype(np.float64)
 
 
-@pytest.mark.parametrize("cfg,linears", [(2, (0, 1, 2, 3)), (4, (0, 4))], ids=["cfg2_all_linears", "cfg4_qkv_and_down"])
+@pytest.mark.parametrize("cfg,linears", [(2, (0, 1, 2, 3)), (4, (0, 4)), (3, (0, 1, 2, 3))],
+                         ids=["cfg2_all_linears", "cfg4_qkv_and_down", "cfg3_all_linears_12_block_outputs"])
 def test_full_size_step_replayed_from_a_graph(tw, cfg, linears):
     from paper_2511_23225_b200.workload import BlockStep
     bs = BlockStep(cfg)
@@ -81,10 +82,22 @@ def test_full_size_step_replayed_from_a_graph(tw, cfg, linears):
         assert rel_fro(at(lb.dw, r, c), orc.gemm_wgrad_at(qx["q"], E4M3, qd["q"], E5M2, qx["scale_inv"], qd["scale_inv"], r, c)) <= GEMM_TOL
     tau, eps, p, c = (float(np.float32(v)) for v in (bs.tau, bs.eps, bs.p, bs.lam / bs.n_blocks))
     blocks = host["bits"]["a"]
-    ref_loss = float(np.mean([orc.tweo_loss_block(a, tau, eps, p) for a in blocks]))
+    per_draw = {}                                   # block outputs that share a draw share the oracle's value
+    for a in blocks:
+        if id(a) not in per_draw:
+            per_draw[id(a)] = orc.tweo_loss_block(a, tau, eps, p)
+    per_block = [per_draw[id(a)] for a in blocks]
+    ref_loss = float(np.mean(per_block))
     assert abs(bs.loss.item() - ref_loss) <= 1e-5 * abs(ref_loss)
+    got_pb = bs.loss_per_block.cpu().numpy().astype(np.float64)
+    assert len(got_pb) == bs.n_blocks and np.all(np.abs(got_pb - per_block) <= 1e-5 * np.abs(per_block))
     a0 = np.ascontiguousarray(blocks[0][:64])       # the gradient of the first 64 rows of the first block output
     n_all = blocks[0].size
     ref_g = orc.tweo_grad_block(a0, tau, eps, p, c) * a0.size / n_all
     got_g = bs.ga[0][:64].float().cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got_g - ref_g) <= np.abs(ref_g) * 2.0 ** -8 + 1e-45)
+    last = bs.n_blocks - 1                          # and the last 64 rows of the last block output
+    a1 = np.ascontiguousarray(blocks[last][-64:])
+    ref_g = orc.tweo_grad_block(a1, tau, eps, p, c) * a1.size / n_all
+    got_g = bs.ga[last][-64:].float().cpu().numpy().astype(np.float64)
     assert np.all(np.abs(got_g - ref_g) <= np.abs(ref_g) * 2.0 ** -8 + 1e-45)

@@ -44,6 +44,33 @@ def test_static_scratch_entry_matches_workspace_entry_twice(grad_dtype):
             assert torch.linalg.norm(g64 - r64) <= TWEO_TOL * torch.linalg.norm(r64)
 
 
+def test_static_scratch_entry_allocates_nothing_and_agrees_with_the_oracle():
+    """With the outputs preallocated, a call changes neither the device memory in use (driver view) nor
+    what torch's pool holds; and the results are the CPU oracle's, not just the other entry point's."""
+    from oracle import tweo_oracle as orc
+    from paper_2511_23225_b200 import binding as tw
+    bits = [synth.normal_with_outlier_channels_bf16(340 + i, (515, 77)) for i in range(2)]
+    blocks = [to_gpu_bf16(b) for b in bits]
+    grads = [torch.empty(b.shape, dtype=torch.float32, device="cuda") for b in blocks]
+    loss = torch.empty(1, dtype=torch.float32, device="cuda")
+    per = torch.empty(2, dtype=torch.float32, device="cuda")
+    c = 0.01 / 2
+    tw.loss_fwd_bwd_static(blocks, 3.0, 1e-6, 4.0, c, True, tw.F32, grads=grads, loss=loss, per_block_out=per)
+    torch.cuda.synchronize()                         # first call on the device done: the address is cached
+    free0, _ = torch.cuda.mem_get_info()
+    held0 = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved())
+    tw.loss_fwd_bwd_static(blocks, 3.0, 1e-6, 4.0, c, True, tw.F32, grads=grads, loss=loss, per_block_out=per)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == held0
+    ref = [orc.tweo_loss_block(b, 3.0, 1e-6, 4.0) for b in bits]
+    assert abs(loss.item() - np.mean(ref)) <= TWEO_TOL * abs(np.mean(ref))
+    assert np.all(np.abs(per.cpu().numpy() - ref) <= TWEO_TOL * np.abs(ref))
+    for g, b in zip(grads, bits):
+        want = orc.tweo_grad_block(b, 3.0, 1e-6, 4.0, c)
+        assert np.linalg.norm(g.cpu().numpy().astype(np.float64) - want) <= TWEO_TOL * np.linalg.norm(want)
+
+
 def test_static_scratch_entry_rejects_bad_arguments():
     from paper_2511_23225_b200 import binding as tw
     a = torch.zeros(64, dtype=torch.bfloat16, device="cuda")
