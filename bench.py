@@ -1,24 +1,35 @@
 #!/usr/bin/env python
 """Benchmark of the FP8 per-tensor linear + TWEO-loss hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg1|cfg3|cfg4] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4|cfg1|cfg2|cfg3] [--variant fused|plain|unfused]
+                    [--impl reference]
 
 One step = per linear of the block: per-tensor FP8 casts of X, W (E4M3) and dY
 (E5M2) with current scaling, forward / dgrad / wgrad GEMMs; then the TWEO loss
-and gradient on the block output.  Prints ONE JSON line (rank 0).
+and gradient on the block output.  In the default variant ("fused") the forward
+and data-gradient GEMMs also emit amax and the FP8 copy of their output from the
+epilogue, with delayed scales.  Prints ONE JSON line (rank 0).
 
   value        FP8 linear fwd+bwd TFLOP/s over the whole step (casts and the TWEO
                pass included in the time, 6*M*K*N flop per linear), inputs resident
                in HBM, CUDA-event timed, max over ranks, summed over ranks (weak
                scaling: every rank runs its own token shard, no data-path collective).
+  variants     the same step without the fused outputs ("plain") and with those outputs
+               produced by separate cast passes ("unfused").
+  sustained    the step graph and the GEMM family replayed for >= 2 s each, with the
+               clocks seen, against 2 x the sustained bf16 figure.
   e2e          same metric with the step's inputs copied from pinned host memory and
                the loss read back inside the timed region.
   roofline     dominant kernel family (largest share of the step): its launches of one
                step replayed alone from a CUDA graph between two events; algorithmic
                flops or bytes / that duration, against the measured peak in
                MEASURED_PEAKS.json (fallback stated if absent).
+  fractions    compact table: every configuration's roofline fractions.
   other_workloads  short runs of the other training configs (N=1), same measurements.
   cpu_baseline the CPU oracle, as it stands, timed on a bounded sample (N=1, rank 0).
+
+HBM-bound rows are timed over rotating buffer sets larger than the 126 MB L2 (every row
+says `l2_resident: false`; rows that deliberately replay one buffer say true).
 
 `--impl reference` times the CPU oracle alone (there is no reference code for this
 paper; the oracle is the reference arm).
@@ -39,9 +50,9 @@ sys.path.insert(0, ROOT)
 METRIC = "fp8_linear_fwd_bwd_tflops_with_tweo_loss"
 UNIT = "TFLOP/s"
 FP8_DATASHEET_TFLOPS = 4500.0
-# DRAM traffic of the dominant kernel family (the 8 GEMM launches of a config-2 step), per launch, from
-# the ncu capture summarised in profiles/launch_list_bench_cfg2.md; valid for that library version only.
-GEMM_TRAFFIC = {"library_version": 212, "workload": "cfg2", "bytes_per_launch": 20.43e6}
+# DRAM traffic of the dominant kernel family (the GEMM launches of a step), per launch, from the ncu captures of
+# single launches summarised under profiles/; reported only while the GEMM sources are the ones profiled.
+GEMM_TRAFFIC = {"sources": "", "workload": "cfg4", "variant": "fused", "bytes_per_launch": None, "from": ""}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, FALLBACK_BF16_SUSTAINED = 6650.0, 1590.0, 1400.0
 
 
@@ -180,6 +191,10 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- CUDA arm
+L2_BYTES = 126e6
+ROTATE_BYTES = 2.5 * L2_BYTES      # distinct bytes a rotating row touches before it returns to a buffer
+
+
 def _graph_of(torch, stream, fn):
     g = torch.cuda.CUDAGraph()
     with torch.cuda.stream(stream):
@@ -202,45 +217,115 @@ def _time_replays(torch, graph, reps):
     return e0.elapsed_time(e1) / reps
 
 
-def family_breakdown(torch, tw, bs, side, reps):
+def rotating_us(torch, side, make_set, call, bytes_per_call, reps=5, max_sets=48):
+    """Microseconds per call of an HBM-bound operation timed over enough distinct buffer sets that a set is
+    only touched again after more than ROTATE_BYTES of other data went through the L2: the sets are visited
+    in turn inside one CUDA graph, which is replayed back to back between two events."""
+    n_sets = int(max(2, min(max_sets, -(-ROTATE_BYTES // max(1.0, bytes_per_call)) + 1)))
+    sets = [make_set(i) for i in range(n_sets)]
+
+    def fn():
+        for st in sets:
+            call(st)
+    fn()
+    torch.cuda.synchronize()
+    us = 1e3 * _time_replays(torch, _graph_of(torch, side, fn), reps) / n_sets
+    del sets
+    return us, n_sets
+
+
+def launch_floor_us(torch, tw, side, n=20):
+    """Duration of the smallest kernel of the library (one thread per tensor of a delayed-scaling update) in the
+    same setting as every other row -- launches chained in a replayed CUDA graph: the floor any launch pays."""
+    h = torch.zeros((1, 16), dtype=torch.float32, device="cuda")
+    v = torch.ones(1, dtype=torch.float32, device="cuda")
+    sc, si = torch.ones(1, dtype=torch.float32, device="cuda"), torch.ones(1, dtype=torch.float32, device="cuda")
+    fn = lambda: [tw.delayed_scaling_update(h, v, sc, si, tw.E4M3) for _ in range(n)]
+    fn()
+    torch.cuda.synchronize()
+    return 1e3 * _time_replays(torch, _graph_of(torch, side, fn), 5) / n
+
+
+def family_breakdown(torch, tw, bs, side, reps, peaks):
     """Times each kernel family of the step on its own: the family's launches of one step are
     captured into a CUDA graph and replayed back to back between two events (so no host gaps
-    and no other family's kernels inside the timed region)."""
+    and no other family's kernels inside the timed region).  A family whose tensors would fit the L2
+    between replays is timed over rotating copies of them."""
     def all_quantize():
         for lb in bs.linears:
             bs.quantize_all(lb)
 
-    def all_gemms():
-        for lb in bs.linears:
-            bs.gemms(lb)
-
     n_el = sum(lb.x.numel() + lb.w.numel() + lb.dy.numel() for lb in bs.linears)
     n_a = sum(t.numel() for t in bs.a)
-    fams = {
-        "quantize": (all_quantize, 5.0 * n_el, "GB/s"),           # 2 + 2 read, 1 written per element
-        "gemm": (all_gemms, float(bs.flops_per_step), "TFLOP/s"),
-        "tweo_loss": (bs.tweo, 4.0 * n_a, "GB/s"),                # 2 read + 2 written per element
-    }
     out = {}
-    for name, (fn, work, unit) in fams.items():
-        c0 = tw.launch_count()
-        g = _graph_of(torch, side, fn)
-        launches = tw.launch_count() - c0
-        ms = _time_replays(torch, g, reps)
+
+    def record(name, ms, launches, work, unit, l2_resident, **extra):
         rate = work / (ms * 1e-3)
         out[name] = {"ms_per_step": ms, "launches_per_step": int(launches), "avg_launch_us": 1e3 * ms / max(1, launches),
-                     "achieved": rate / 1e12 if unit == "TFLOP/s" else rate / 1e9, "unit": unit}
+                     "achieved": rate / 1e12 if unit == "TFLOP/s" else rate / 1e9, "unit": unit,
+                     "l2_resident": bool(l2_resident), **extra}
+
+    # casts: 2 + 2 read, 1 written per element
+    c0 = tw.launch_count()
+    g = _graph_of(torch, side, all_quantize)
+    launches = tw.launch_count() - c0
+    record("quantize", _time_replays(torch, g, reps), launches, 5.0 * n_el, "GB/s", 3.0 * n_el < ROTATE_BYTES)
+    # GEMMs (+ the fused outputs and the two scale-update launches in the fused variant)
+    c0 = tw.launch_count()
+    g = _graph_of(torch, side, bs.all_gemms)
+    launches = tw.launch_count() - c0
+    gemm_bytes = sum(3 * lb.M * lb.lin.K + 3 * lb.lin.K * lb.lin.N + 3 * lb.M * lb.lin.N for lb in bs.linears)
+    record("gemm", _time_replays(torch, g, reps), launches, float(bs.flops_per_step), "TFLOP/s", gemm_bytes < ROTATE_BYTES)
+    # TWEO loss + gradient: 2 read + 2 written per element; rotated when the block outputs would stay in L2
+    if 4.0 * n_a >= ROTATE_BYTES:
+        c0 = tw.launch_count()
+        g = _graph_of(torch, side, bs.tweo)
+        launches = tw.launch_count() - c0
+        record("tweo_loss", _time_replays(torch, g, reps), launches, 4.0 * n_a, "GB/s", False, buffer_sets=1)
+    else:
+        ws = bs.loss_ws
+        c = bs.lam / bs.n_blocks
+
+        def make_set(i):
+            return ([t.clone() for t in bs.a], [torch.empty_like(t) for t in bs.a])
+
+        def call(st):
+            tw.loss_fwd_bwd(st[0], bs.tau, bs.eps, bs.p, c, True, tw.BF16, grads=st[1], ws=ws)
+        us, n_sets = rotating_us(torch, side, make_set, call, 4.0 * n_a, reps=reps)
+        record("tweo_loss", us * 1e-3, 1, 4.0 * n_a, "GB/s", False, buffer_sets=n_sets,
+               us_at_hbm_peak=4.0 * n_a / peaks["hbm"] / 1e3)
     tot = sum(v["ms_per_step"] for v in out.values())
     for v in out.values():
         v["share"] = v["ms_per_step"] / tot
     return out
 
 
-def measure_workload(torch, tw, cfg_idx, steps, warmup, world, barrier, want_e2e, e2e_steps, local, overlap=True):
+def sustained_leg(torch, graph, est_ms, local, seconds=2.0):
+    """Replays `graph` back to back for at least `seconds`; returns ms per replay and the clocks seen."""
+    reps = int(max(10, -(-seconds * 1e3 // max(est_ms, 1e-3))))
+    sampler = ClockSampler(local, period_s=0.05)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    sampler.start()
+    e0.record()
+    for _ in range(reps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    return {"replays": reps, "seconds": ms * 1e-3, "ms_per_replay": ms / reps, "clocks": clocks}
+
+
+def measure_workload(torch, tw, cfg_idx, variant, steps, warmup, barrier, local, host=None, want_e2e=False, e2e_steps=0,
+                     overlap=True, want_sustained=False, peaks=None):
     from paper_2511_23225_b200.workload import BlockStep
-    bs = BlockStep(cfg_idx)
+    bs = BlockStep(cfg_idx, variant=variant)
     bs.overlap = overlap
-    bs.make_host_inputs()
+    if host is None:
+        bs.make_host_inputs()
+    else:
+        bs.host = host
     bs.upload()
     torch.cuda.synchronize()
     for _ in range(max(3, warmup)):
@@ -260,7 +345,7 @@ def measure_workload(torch, tw, cfg_idx, steps, warmup, world, barrier, want_e2e
     barrier()
 
     # ---- timed region: K steps, inputs resident in HBM
-    sampler = ClockSampler(local)
+    sampler = ClockSampler(local, period_s=0.005)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     sampler.start()
@@ -279,7 +364,7 @@ def measure_workload(torch, tw, cfg_idx, steps, warmup, world, barrier, want_e2e
     # two sets of buffers, so the copy of step i + 1 (copy stream) overlaps step i (compute stream); every
     # step's inputs still cross the bus inside the timed region and the host reads every step's loss.
     if want_e2e:
-        bs2 = BlockStep(cfg_idx)
+        bs2 = BlockStep(cfg_idx, variant=variant)
         bs2.overlap = overlap
         bs2.host = bs.host                      # the same pinned host tensors
         bs2.upload()
@@ -321,15 +406,25 @@ def measure_workload(torch, tw, cfg_idx, steps, warmup, world, barrier, want_e2e
         res["e2e_ms_per_step"] = e0.elapsed_time(e1) / e2e_steps
         res["loss"] = float(losses[(e2e_steps - 1) & 1].item())
         del bs2, up_graphs, step_graphs
-    res["kernels"] = family_breakdown(torch, tw, bs, side, max(5, min(steps, 50)))
+        torch.cuda.empty_cache()
+    res["kernels"] = family_breakdown(torch, tw, bs, side, max(5, min(steps, 50)), peaks)
+    if want_sustained:
+        # the box is power-limited: a >= 2 s loop settles at a lower clock than a burst of a few milliseconds
+        st = sustained_leg(torch, step_graph, res["ms_per_step"], local)
+        gg = _graph_of(torch, side, bs.all_gemms)
+        sg = sustained_leg(torch, gg, res["kernels"]["gemm"]["ms_per_step"], local)
+        res["sustained"] = {"step": st, "gemm": sg}
+        del gg
+    del step_graph
     return res
 
 
 def w8a8_sweep(torch, tw, peaks, reps=10):
     """Config 5: the static per-tensor W8A8 linear at LLaMA-7B shapes, E4M3 codes in (the cast of bf16
-    activations is the GIVEN-scale cast timed elsewhere).  Each call is replayed `reps` times from a CUDA
-    graph between two events.  M <= 128 is bound by streaming W (bytes / time against the HBM copy
-    peak; in this back-to-back replay W may partly sit in the 126 MB L2), larger M by the tensor pipe."""
+    activations is the GIVEN-scale cast timed elsewhere).  M <= 128 is bound by streaming W: it is timed COLD,
+    over a rotation of distinct weight buffers larger than the L2 (a decoder layer's weights are not in L2 when
+    its turn comes), and also replayed on one buffer (`us_replayed`, W partly L2-resident).  Larger M is bound
+    by the tensor pipe and replayed from a CUDA graph."""
     side = torch.cuda.Stream()
     one = torch.ones(1, dtype=torch.float32, device="cuda")
     g = torch.Generator(device="cuda").manual_seed(5)
@@ -346,8 +441,17 @@ def w8a8_sweep(torch, tw, peaks, reps=10):
             us = 1e3 * _time_replays(torch, _graph_of(torch, side, fn), 5) / reps
             flops, nbytes = 2.0 * M * K * N, float(M * K + K * N + 2 * M * N)
             hbm_us, tc_us = nbytes / peaks["hbm"] / 1e3, flops / (2.0 * peaks["bf16"]) / 1e6
-            rows.append({"M": M, "K": K, "N": N, "us": us, "tflops": flops / us / 1e6, "gbs": nbytes / us / 1e3,
-                         "bound": "hbm" if hbm_us > tc_us else "tensor", "frac_of_roofline": max(hbm_us, tc_us) / us})
+            row = {"M": M, "K": K, "N": N, "bound": "hbm" if hbm_us > tc_us else "tensor"}
+            if M <= 128:
+                cold_us, n_sets = rotating_us(torch, side, lambda i: wq.clone(),
+                                              lambda w: tw.w8a8_static_gemm(xq, one, w, one, y=y, ws=ws), nbytes)
+                row.update({"us": cold_us, "us_replayed": us, "weight_buffers": n_sets, "l2_resident": False,
+                            "gbs": nbytes / cold_us / 1e3, "frac_of_roofline": hbm_us / cold_us,
+                            "frac_of_roofline_replayed": hbm_us / us})
+            else:
+                row.update({"us": us, "tflops": flops / us / 1e6, "l2_resident": nbytes < L2_BYTES,
+                            "frac_of_roofline": max(hbm_us, tc_us) / us})
+            rows.append(row)
             del xq, y, ws
         del wq
         torch.cuda.empty_cache()
@@ -371,27 +475,67 @@ def whole_job_value(flops_per_rank_step: float, ms_per_step: float, world: int) 
     return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
 
 
-def block_output_bench(torch, tw, peaks, reps=10):
+def _hbm_row(peaks, us, nbytes, **kw):
+    return {**kw, "us": us, "gbs": nbytes / us / 1e3, "frac_of_hbm_peak": nbytes / us / 1e3 / peaks["hbm"],
+            "l2_resident": False}
+
+
+def streaming_bench(torch, tw, peaks):
+    """The per-tensor cast (current and given scale) and the TWEO loss + gradient at the tensor sizes of the
+    configurations, each over rotating buffer sets (inputs never L2-resident): bytes / time against the copy peak."""
+    side = torch.cuda.Stream()
+    rows = {"quantize_current": [], "quantize_given": [], "tweo_loss": []}
+    sizes = (("cfg2 X [8192x768]", 8192 * 768), ("cfg2 dY [8192x3072]", 8192 * 3072), ("cfg4 X [16384x2048]", 16384 * 2048),
+             ("cfg4 dY [16384x6144]", 16384 * 6144))
+    ws = tw.new_workspace(tw.OP_QUANTIZE)
+    for name, n in sizes:
+        def make_set(i):
+            x = torch.randn(n, device="cuda").to(torch.bfloat16)
+            return x, tw.quantize_per_tensor(x, tw.E4M3, ws=ws)
+        us, k = rotating_us(torch, side, make_set, lambda st: tw.quantize_per_tensor(st[0], tw.E4M3, out=st[1], ws=ws), 3.0 * n)
+        rows["quantize_current"].append(_hbm_row(peaks, us, 5.0 * n, tensor=name, buffer_sets=k))
+        sc = torch.full((1,), 64.0, dtype=torch.float32, device="cuda")
+
+        def make_given(i):
+            x = torch.randn(n, device="cuda").to(torch.bfloat16)
+            return x, tw.quantize_per_tensor(x, tw.E4M3, tw.SCALE_GIVEN, scale=sc)
+        us, k = rotating_us(torch, side, make_given,
+                            lambda st: tw.quantize_per_tensor(st[0], tw.E4M3, tw.SCALE_GIVEN, out=st[1]), 3.0 * n)
+        rows["quantize_given"].append(_hbm_row(peaks, us, 3.0 * n, tensor=name, buffer_sets=k))
+        torch.cuda.empty_cache()
+    floor = launch_floor_us(torch, tw, side)
+    for name, n in (("cfg2 A [8192x768]", 8192 * 768), ("cfg4 A [16384x2048]", 16384 * 2048),
+                    ("cfg3 A [50432x768]", 50432 * 768)):
+        lws = tw.new_workspace(tw.OP_LOSS, n, 1)
+
+        def make_a(i):
+            a = torch.randn(n, device="cuda").to(torch.bfloat16)
+            return [a], [torch.empty_like(a)]
+        us, k = rotating_us(torch, side, make_a,
+                            lambda st: tw.loss_fwd_bwd(st[0], 3.0, 1e-6, 4.0, 0.01, True, tw.BF16, grads=st[1], ws=lws), 4.0 * n)
+        rows["tweo_loss"].append(_hbm_row(peaks, us, 4.0 * n, tensor=name, buffer_sets=k, us_at_hbm_peak=4.0 * n / peaks["hbm"] / 1e3,
+                                          launch_floor_us=floor))
+        torch.cuda.empty_cache()
+    return rows
+
+
+def block_output_bench(torch, tw, peaks):
     """The fused block-output pass (x + f -> a, TWEO loss and gradient, amax, E4M3 copy with a given
     scale) at the block-output sizes of configs 2 and 4: 4 B read + 5 B written per element."""
     side = torch.cuda.Stream()
     rows = []
+    qs = torch.full((1,), 448.0 / 8.0, dtype=torch.float32, device="cuda")
+    ws = tw.new_workspace(tw.OP_BLOCK_OUTPUT)
     for name, n in (("cfg2 [8192x768]", 8192 * 768), ("cfg4 [16384x2048]", 16384 * 2048)):
-        x = torch.randn(n, device="cuda").to(torch.bfloat16)
-        f = (0.3 * torch.randn(n, device="cuda")).to(torch.bfloat16)
-        a, g = torch.empty_like(x), torch.empty_like(x)
-        aq = torch.empty(n, dtype=torch.uint8, device="cuda")
-        qs = torch.full((1,), 448.0 / 8.0, dtype=torch.float32, device="cuda")
-        ws = tw.new_workspace(tw.OP_BLOCK_OUTPUT)
-        fn = lambda: [tw.block_output_fused(x, f, 3.0, 1e-6, 4.0, 0.01, True, tw.E4M3, qs, a=a, grad=g, aq=aq, ws=ws)
-                      for _ in range(reps)]
-        fn()
-        torch.cuda.synchronize()
-        us = 1e3 * _time_replays(torch, _graph_of(torch, side, fn), 5) / reps
-        rows.append({"tensor": name, "elements": n, "us": us, "gbs": 9.0 * n / us / 1e3,
-                     "frac_of_hbm_peak": 9.0 * n / us / 1e3 / peaks["hbm"]})
-        del x, f, a, g, aq
-    torch.cuda.empty_cache()
+        def make_set(i):
+            x = torch.randn(n, device="cuda").to(torch.bfloat16)
+            f = (0.3 * torch.randn(n, device="cuda")).to(torch.bfloat16)
+            return x, f, torch.empty_like(x), torch.empty_like(x), torch.empty(n, dtype=torch.uint8, device="cuda")
+        us, k = rotating_us(torch, side, make_set,
+                            lambda s: tw.block_output_fused(s[0], s[1], 3.0, 1e-6, 4.0, 0.01, True, tw.E4M3, qs, a=s[2],
+                                                            grad=s[3], aq=s[4], ws=ws), 9.0 * n)
+        rows.append(_hbm_row(peaks, us, 9.0 * n, tensor=name, elements=n, buffer_sets=k))
+        torch.cuda.empty_cache()
     return rows
 
 
@@ -407,12 +551,9 @@ def int8_bench(torch, tw, peaks, reps=10):
         x = torch.randn((M, K), device="cuda").to(torch.bfloat16)
         for gname, gran in (("T", tw.GRAN_TENSOR), ("row", tw.GRAN_ROW)):
             ws = tw.new_workspace(tw.OP_ABSMAX)
-            fn = lambda: [tw.absmax_quantize(x, 8, gran, 1e-6, ws=ws) for _ in range(reps)]
-            fn()
-            torch.cuda.synchronize()
-            us = 1e3 * _time_replays(torch, _graph_of(torch, side, fn), 5) / reps
-            out["quantize"].append({"tensor": f"[{M}x{K}]", "granularity": gname, "us": us,
-                                    "gbs": 5.0 * M * K / us / 1e3, "frac_of_hbm_peak": 5.0 * M * K / us / 1e3 / peaks["hbm"]})
+            us, k = rotating_us(torch, side, lambda i: torch.randn((M, K), device="cuda").to(torch.bfloat16),
+                                lambda xs: tw.absmax_quantize(xs, 8, gran, 1e-6, ws=ws), 3.0 * M * K)
+            out["quantize"].append(_hbm_row(peaks, us, 5.0 * M * K, tensor=f"[{M}x{K}]", granularity=gname, buffer_sets=k))
             xq, sx = tw.absmax_quantize(x, 8, gran, 1e-6, ws=ws)
             wq, sw = tw.absmax_quantize(w, 8, gran, 1e-6, ws=ws)
             y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
@@ -433,7 +574,7 @@ def act_norm_bench(torch, tw, peaks, reps=10):
     """Activation-fused forward epilogue and FP8 LayerNorm at the benchmark's MLP shapes.  For each linear:
     the plain forward product, the product with the activation in its epilogue (bf16 + FP8 out, FP8 only),
     and the streaming passes the fusion removes (read bf16, write FP8) for scale.  LayerNorm: bytes moved
-    per element 2 read + 2 (bf16) and / or 1 (FP8) written."""
+    per element 2 read + 2 (bf16) and / or 1 (FP8) written, over rotating buffers."""
     side = torch.cuda.Stream()
     out = {"fwd_act": [], "layernorm": []}
 
@@ -463,28 +604,31 @@ def act_norm_bench(torch, tw, peaks, reps=10):
                                "unfused_extra_pass_us_at_hbm_peak": (2.0 * M * Nw + 1.0 * M * N) / peaks["hbm"] / 1e3})
         del xq, wq, y_plain, y, yq
     for name, kind, rows, d in (("cfg2_ln_768", tw.NORM_LAYER, 16384 * 8, 768), ("cfg4_rms_2048", tw.NORM_RMS, 8192 * 8, 2048)):
-        x = torch.randn((rows, d), device="cuda").to(torch.bfloat16)
         gamma = torch.ones(d, device="cuda")
         beta = torch.zeros(d, device="cuda") if kind == tw.NORM_LAYER else None
         qs = torch.full((1,), 64.0, dtype=torch.float32, device="cuda")
-        y = torch.empty_like(x)
-        yq = torch.empty((rows, d), dtype=torch.uint8, device="cuda")
         n = rows * d
-        for label, kw, bytes_per in (("bf16+fp8", dict(y=y, yq=yq, q_fmt=tw.E4M3, q_scale=qs), 5.0),
-                                     ("fp8_only", dict(want_y=False, yq=yq, q_fmt=tw.E4M3, q_scale=qs), 3.0),
-                                     ("bf16_only", dict(y=y), 4.0)):
-            us = timed(lambda: tw.layernorm_fp8(x, gamma, beta, 1e-5, kind, **kw))
-            out["layernorm"].append({"case": name, "rows": rows, "d": d, "outputs": label, "us": us,
-                                     "gbs": bytes_per * n / us / 1e3,
-                                     "frac_of_hbm_peak": bytes_per * n / us / 1e3 / peaks["hbm"]})
-        del x, y, yq
-    torch.cuda.empty_cache()
+        for label, want_y, want_q, bytes_per in (("bf16+fp8", True, True, 5.0), ("fp8_only", False, True, 3.0),
+                                                 ("bf16_only", True, False, 4.0)):
+            def make_set(i):
+                x = torch.randn((rows, d), device="cuda").to(torch.bfloat16)
+                return (x, torch.empty_like(x) if want_y else None,
+                        torch.empty((rows, d), dtype=torch.uint8, device="cuda") if want_q else None)
+
+            def call(st):
+                kw = dict(y=st[1]) if want_y else dict(want_y=False)
+                if want_q:
+                    kw.update(yq=st[2], q_fmt=tw.E4M3, q_scale=qs)
+                tw.layernorm_fp8(st[0], gamma, beta, 1e-5, kind, **kw)
+            us, k = rotating_us(torch, side, make_set, call, bytes_per * n, max_sets=4)
+            out["layernorm"].append(_hbm_row(peaks, us, bytes_per * n, case=name, rows=rows, d=d, outputs=label, buffer_sets=k))
+            torch.cuda.empty_cache()
     return out
 
 
 def residual8_bench(torch, tw, peaks, reps=10):
     """The 8-bit residual stream: the integer linear with 8-bit output against the one with bf16 output, and
-    the residual addition on codes (2 B read + 1 B written per element)."""
+    the residual addition on codes (2 B read + 1 B written per element), over rotating buffers."""
     side = torch.cuda.Stream()
     out = {"linear_q8": [], "residual_add_q8": []}
 
@@ -507,27 +651,25 @@ def residual8_bench(torch, tw, peaks, reps=10):
                                  "tops_bf16_out": ops / us_bf16 / 1e6, "tops_int8_out": ops / us_q8 / 1e6,
                                  "frac_of_2x_bf16_burst": ops / us_q8 / 1e6 / (2.0 * peaks["bf16"])})
         del xq, wq, y, yq
+    s1 = torch.full((1,), 2.0, dtype=torch.float32, device="cuda")
     for n in (8192 * 4096, 16 * 8192 * 4096):
-        xq = torch.randint(-127, 128, (n,), device="cuda", dtype=torch.int8)
-        fq = torch.randint(-127, 128, (n,), device="cuda", dtype=torch.int8)
-        yq = torch.empty_like(xq)
-        s = torch.full((1,), 2.0, dtype=torch.float32, device="cuda")
-        us = timed(lambda: tw.residual_add_q8(xq, s, fq, s, s, 8, yq=yq))
-        out["residual_add_q8"].append({"n": n, "us": us, "gbs": 3.0 * n / us / 1e3,
-                                       "frac_of_hbm_peak": 3.0 * n / us / 1e3 / peaks["hbm"]})
-        del xq, fq, yq
+        mk = lambda i: (torch.randint(-127, 128, (n,), device="cuda", dtype=torch.int8),
+                        torch.randint(-127, 128, (n,), device="cuda", dtype=torch.int8),
+                        torch.empty(n, device="cuda", dtype=torch.int8))
+        us, k = rotating_us(torch, side, mk, lambda s: tw.residual_add_q8(s[0], s1, s[1], s1, s1, 8, yq=s[2]), 3.0 * n,
+                            max_sets=6)
+        out["residual_add_q8"].append(_hbm_row(peaks, us, 3.0 * n, n=n, buffer_sets=k))
+        torch.cuda.empty_cache()
     out["residual_add_q8_rows"] = []
     for rows, cols in ((16384, 768), (65536, 2048)):        # per token (A8(K)): one scale per row in, one out
-        xq = torch.randint(-127, 128, (rows, cols), device="cuda", dtype=torch.int8)
-        fq = torch.randint(-127, 128, (rows, cols), device="cuda", dtype=torch.int8)
-        yq = torch.empty_like(xq)
         s = torch.full((rows,), 2.0, dtype=torch.float32, device="cuda")
-        us = timed(lambda: tw.residual_add_q8_rows(xq, s, fq, s, 8, 1e-6, yq=yq))
         n = rows * cols
-        out["residual_add_q8_rows"].append({"rows": rows, "cols": cols, "us": us, "gbs": 3.0 * n / us / 1e3,
-                                            "frac_of_hbm_peak": 3.0 * n / us / 1e3 / peaks["hbm"]})
-        del xq, fq, yq
-    torch.cuda.empty_cache()
+        mk = lambda i: (torch.randint(-127, 128, (rows, cols), device="cuda", dtype=torch.int8),
+                        torch.randint(-127, 128, (rows, cols), device="cuda", dtype=torch.int8),
+                        torch.empty((rows, cols), device="cuda", dtype=torch.int8))
+        us, k = rotating_us(torch, side, mk, lambda st: tw.residual_add_q8_rows(st[0], s, st[1], s, 8, 1e-6, yq=st[2]), 3.0 * n)
+        out["residual_add_q8_rows"].append(_hbm_row(peaks, us, 3.0 * n, rows=rows, cols=cols, buffer_sets=k))
+        torch.cuda.empty_cache()
     return out
 
 
@@ -563,6 +705,23 @@ def vendor_fp8_context(torch, tw, reps=10):
     return out
 
 
+def gemm_sources_digest() -> str:
+    """SHA-256 over the GEMM kernels' source files: DRAM counters taken under a profiler are reported only for
+    the kernels they were taken from."""
+    import hashlib
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2511_23225_b200", "csrc")
+    for f in ("gemm.cu", "gemm_pair.cuh", "gemm_pair_group.cuh", "gemm_split.cuh", "gemm_common.cuh", "tc_ptx.cuh", "common.cuh"):
+        with open(os.path.join(d, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def gemm_summary(k, fp8_burst):
+    return {"gemm_tflops": k["gemm"]["achieved"], "gemm_frac_of_2x_bf16_burst": k["gemm"]["achieved"] / fp8_burst,
+            "gemm_pct_of_fp8_datasheet": 100.0 * k["gemm"]["achieved"] / FP8_DATASHEET_TFLOPS}
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -585,50 +744,97 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    overlap = not args.no_overlap
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    r = measure_workload(torch, tw, cfg_idx, args.steps, args.warmup, world, barrier, True, e2e_steps, local,
-                         overlap=not args.no_overlap)
+    r = measure_workload(torch, tw, cfg_idx, args.variant, args.steps, args.warmup, barrier, local, want_e2e=True,
+                         e2e_steps=e2e_steps, overlap=overlap, want_sustained=(world == 1 and not args.no_sustained),
+                         peaks=peaks)
     bs = r["bs"]
+    host = bs.host
     ms_per_step = max_over_ranks(r["ms_per_step"], "cuda")
     e2e_ms = max_over_ranks(r["e2e_ms_per_step"], "cuda")
     value = whole_job_value(bs.flops_per_step, ms_per_step, world)
     e2e_value = whole_job_value(bs.flops_per_step, e2e_ms, world)
     kernels = r["kernels"]
+    flops_per_step = bs.flops_per_step
 
     # Roofline of the dominant kernel family.  FP8 dense peak = 2 x the measured bf16 figure (nominal
-    # ratio); the burst figure, because the family is timed alone in short replays.
+    # ratio): the burst figure for the family timed alone in short replays, the sustained one for the >= 2 s loop.
     dom = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
     fp8_burst, fp8_sustained = 2.0 * peaks["bf16"], 2.0 * peaks["bf16_sustained"]
     of = "of measured" if peaks["source"] == "measured" else "of fallback"
     if dom == "gemm":
         roof = {"bound": "tensor", "achieved": kernels["gemm"]["achieved"], "peak": fp8_burst, "unit": "TFLOP/s",
-                "peak_source": of + " (2 x burst bf16)"}
+                "peak_source": of + " (2 x burst bf16)", "kernel_family": f"the {kernels['gemm']['launches_per_step']} "
+                f"GEMM-family launches of one {args.variant} step"}
     else:
         roof = {"bound": "hbm", "achieved": kernels[dom]["achieved"], "peak": peaks["hbm"], "unit": "GB/s",
                 "peak_source": of + " (copy bandwidth)"}
     roof["frac"] = roof["achieved"] / roof["peak"]
+    if dom == "gemm":
+        roof["frac_of_fp8_datasheet_4500"] = roof["achieved"] / FP8_DATASHEET_TFLOPS
     roof["traffic"] = None
-    if dom == "gemm" and tw.version() == GEMM_TRAFFIC["library_version"] and args.workload == GEMM_TRAFFIC["workload"]:
+    if (dom == "gemm" and GEMM_TRAFFIC["sources"] == gemm_sources_digest() and args.workload == GEMM_TRAFFIC["workload"]
+            and args.variant == GEMM_TRAFFIC["variant"]):
         roof["traffic"] = GEMM_TRAFFIC["bytes_per_launch"]
-        roof["algorithmic_bytes_per_launch"] = sum(
-            lb.M * lb.lin.K + lb.lin.K * lb.lin.N + 2 * lb.M * lb.lin.N             # forward: X, W in; Y out
-            + lb.M * lb.lin.N + lb.lin.K * lb.lin.N + lb.M * lb.lin.K               # backward: dY, W, X in;
-            + 2 * lb.M * lb.lin.K + 2 * lb.lin.K * lb.lin.N                         #           dX, dW out
-            for lb in bs.linears) / (2.0 * len(bs.linears))
+        roof["traffic_from"] = GEMM_TRAFFIC["from"]
+    sustained = None
+    if "sustained" in r:
+        st, sg = r["sustained"]["step"], r["sustained"]["gemm"]
+        g_tf = flops_per_step / (sg["ms_per_replay"] * 1e-3) / 1e12
+        sustained = {
+            "step": {"seconds": st["seconds"], "steps": st["replays"], "ms_per_step": st["ms_per_replay"],
+                     "value": flops_per_step / (st["ms_per_replay"] * 1e-3) / 1e12, "unit": UNIT, "clocks": st["clocks"]},
+            "gemm_family": {"seconds": sg["seconds"], "replays": sg["replays"], "ms_per_replay": sg["ms_per_replay"],
+                            "achieved": g_tf, "unit": UNIT, "peak": fp8_sustained,
+                            "peak_source": of + " (2 x sustained bf16)", "frac": g_tf / fp8_sustained,
+                            "frac_of_fp8_datasheet_4500": g_tf / FP8_DATASHEET_TFLOPS, "clocks": sg["clocks"]},
+        }
+        roof["sustained"] = {"achieved": g_tf, "peak": fp8_sustained, "frac": g_tf / fp8_sustained}
 
-    workload_cfg = {"workload": workload_name(cfg_idx), "tokens_per_gpu": bs.M,
+    workload_cfg = {"workload": workload_name(cfg_idx), "variant": args.variant, "tokens_per_gpu": bs.M,
                     "linears": [f"{l.name}:{l.K}x{l.N}" for l in bs.cfg.linears], "tweo_blocks": bs.n_blocks,
                     "parallelism": f"replicas x{world} (token shards, no data-path collective)",
                     "l2": f"working set {bs.working_set_bytes() / 1e6:.0f} MB per step > 126 MB L2, no flush",
                     "launch": "cuda graph replay of one captured step; two streams inside it: the casts of linear "
-                              "i+1 and the TWEO pass overlap the GEMMs of linear i" if not args.no_overlap
+                              "i+1 and the TWEO pass overlap the GEMMs of linear i" if overlap
                     else "cuda graph replay of one captured step, one stream"}
+    if args.variant == "fused":
+        workload_cfg["epilogue"] = ("forward and data-gradient GEMMs emit bf16 + amax + FP8 copy (Y E4M3, dX E5M2) with "
+                                    "delayed scales (history 16); 2 scale-update launches per step")
     h2d = bs.h2d_bytes()
     loss_value = r["loss"]
     main_clocks = r["clocks"]
     launches_per_step = r["launches_per_step"]
     del bs, r
     torch.cuda.empty_cache()
+
+    fractions = {args.workload: {"variant": args.variant, "step_tflops": value / world, **gemm_summary(kernels, fp8_burst),
+                                 "quantize_frac_of_hbm": kernels["quantize"]["achieved"] / peaks["hbm"],
+                                 "tweo_frac_of_hbm": kernels["tweo_loss"]["achieved"] / peaks["hbm"]}}
+    if sustained:
+        fractions[args.workload]["gemm_frac_of_2x_bf16_sustained_2s"] = sustained["gemm_family"]["frac"]
+
+    # ---- the same workload without the fused outputs, and with them produced by separate passes
+    variants = {}
+    if world == 1 and not args.no_variants:
+        for v in VARIANT_ORDER:
+            if v == args.variant:
+                continue
+            o = measure_workload(torch, tw, cfg_idx, v, args.also_steps, 3, barrier, local, host=host, overlap=overlap,
+                                 peaks=peaks)
+            k = o["kernels"]
+            variants[v] = {"ms_per_step": o["ms_per_step"], "value": flops_per_step / (o["ms_per_step"] * 1e-3) / 1e12,
+                           "unit": UNIT, "launches_per_step": o["launches_per_step"], **gemm_summary(k, fp8_burst),
+                           "gemm_ms": k["gemm"]["ms_per_step"], "clocks": o["clocks"]}
+            del o
+            torch.cuda.empty_cache()
+        fractions[args.workload]["step_tflops_by_variant"] = {args.variant: value / world,
+                                                              **{v: d["value"] for v, d in variants.items()}}
+        fractions[args.workload]["gemm_frac_by_variant"] = {
+            args.variant: kernels["gemm"]["achieved"] / fp8_burst,
+            **{v: d["gemm_frac_of_2x_bf16_burst"] for v, d in variants.items()}}
+    del host
 
     # ---- the other training configurations, short runs (context for the large shapes)
     others = {}
@@ -637,23 +843,39 @@ def run_cuda(args):
             name = name.strip()
             if not name or name == args.workload:
                 continue
-            o = measure_workload(torch, tw, int(name[3:]), args.also_steps, 3, 1, barrier, False, 0, local,
-                                 overlap=not args.no_overlap)
-            obs = o["bs"]
-            k = o["kernels"]
-            others[name] = {
-                "workload": workload_name(int(name[3:])), "steps": args.also_steps, "ms_per_step": o["ms_per_step"],
-                "value": obs.flops_per_step / (o["ms_per_step"] * 1e-3) / 1e12, "unit": UNIT,
-                "gemm_tflops": k["gemm"]["achieved"], "gemm_frac_of_fp8_burst_peak": k["gemm"]["achieved"] / fp8_burst,
-                "gemm_pct_of_fp8_datasheet_peak": 100.0 * k["gemm"]["achieved"] / FP8_DATASHEET_TFLOPS,
-                "quantize_gbs": k["quantize"]["achieved"], "tweo_loss_gbs": k["tweo_loss"]["achieved"],
-                "shares": {n: v["share"] for n, v in k.items()}, "clocks": o["clocks"]}
-            del obs, o
-            torch.cuda.empty_cache()
+            ci = int(name[3:])
+            entry = {"workload": workload_name(ci), "steps": args.also_steps}
+            ohost = None
+            for v in (args.variant, "plain") if args.variant != "plain" else ("plain",):
+                o = measure_workload(torch, tw, ci, v, args.also_steps, 3, barrier, local, host=ohost, overlap=overlap,
+                                     peaks=peaks)
+                obs = o["bs"]
+                ohost = obs.host
+                k = o["kernels"]
+                entry[v] = {"ms_per_step": o["ms_per_step"], "value": obs.flops_per_step / (o["ms_per_step"] * 1e-3) / 1e12,
+                            "unit": UNIT, **gemm_summary(k, fp8_burst), "quantize_gbs": k["quantize"]["achieved"],
+                            "tweo_loss_gbs": k["tweo_loss"]["achieved"],
+                            "tweo_l2_resident": k["tweo_loss"]["l2_resident"],
+                            "shares": {n: x["share"] for n, x in k.items()}, "clocks": o["clocks"]}
+                del obs, o
+                torch.cuda.empty_cache()
+            others[name] = entry
+            first = entry[args.variant]
+            fractions[name] = {"variant": args.variant, "step_tflops": first["value"],
+                               "gemm_tflops": first["gemm_tflops"],
+                               "gemm_frac_of_2x_bf16_burst": first["gemm_frac_of_2x_bf16_burst"],
+                               "gemm_pct_of_fp8_datasheet": first["gemm_pct_of_fp8_datasheet"],
+                               "quantize_frac_of_hbm": first["quantize_gbs"] / peaks["hbm"],
+                               "tweo_frac_of_hbm": first["tweo_loss_gbs"] / peaks["hbm"]}
+            if "plain" in entry and args.variant != "plain":
+                fractions[name]["plain_step_tflops"] = entry["plain"]["value"]
+                fractions[name]["plain_gemm_frac_of_2x_bf16_burst"] = entry["plain"]["gemm_frac_of_2x_bf16_burst"]
+            del ohost
 
-    w8a8, block_rows, int8_rows, act_rows, res8_rows, vendor_rows = None, None, None, None, None, None
+    w8a8, stream_rows, block_rows, int8_rows, act_rows, res8_rows, vendor_rows = (None,) * 7
     if world == 1 and not args.no_w8a8:
         w8a8 = w8a8_sweep(torch, tw, peaks)
+        stream_rows = streaming_bench(torch, tw, peaks)
         block_rows = block_output_bench(torch, tw, peaks)
         int8_rows = int8_bench(torch, tw, peaks)
         act_rows = act_norm_bench(torch, tw, peaks)
@@ -661,6 +883,13 @@ def run_cuda(args):
         vendor_rows = vendor_fp8_context(torch, tw)
         if tw.read_device_status() != 0:
             raise SystemExit("device status reports an expired wait")
+        small = [x["frac_of_roofline"] for x in w8a8 if x["M"] <= 128]
+        fractions["cfg5"] = {
+            "M8192_frac_of_roofline": [x["frac_of_roofline"] for x in w8a8 if x["M"] == 8192],
+            "M1024_frac_of_roofline": [x["frac_of_roofline"] for x in w8a8 if x["M"] == 1024],
+            "M_le_128_cold_w_frac_of_hbm_roofline_min_max": [min(small), max(small)]}
+        fractions["streaming_kernels_frac_of_hbm"] = {
+            fam: {x["tensor"]: x["frac_of_hbm_peak"] for x in rows_} for fam, rows_ in stream_rows.items()}
 
     if rank == 0:
         line = {
@@ -669,20 +898,29 @@ def run_cuda(args):
             "vs_baseline": None, "dtype": "fp8_e4m3xe5m2_fp32acc", "data": "synthetic",
             "config": workload_cfg,
             "pct_of_fp8_datasheet_peak": 100.0 * value / world / FP8_DATASHEET_TFLOPS,
-            "pct_of_fp8_measured_peak": 100.0 * value / world / fp8_sustained,
+            "pct_of_fp8_measured_peak": 100.0 * value / world / fp8_burst,
             "gemm_only_tflops": world * kernels["gemm"]["achieved"],
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4,
-                    "steps": e2e_steps, "pipelining": "two sets of device buffers: the copy of step i+1 overlaps step i"},
+                    "steps": e2e_steps, "pipelining": "two sets of device buffers: the copy of step i+1 overlaps step i",
+                    "d2h": "only the 4-byte loss is read back every step; Y, dX, dW, the FP8 copies and the TWEO gradient "
+                           "stay on the device, as a training step leaves them"},
             "gpu_launches": int(launches_per_step * args.steps),
             "clocks": main_clocks,
             "roofline": roof,
+            "fractions": fractions,
             "kernels": kernels,
             "tweo_loss": loss_value,
         }
+        if sustained:
+            line["sustained"] = sustained
+        if variants:
+            line["variants"] = variants
         if others:
             line["other_workloads"] = others
         if w8a8:
             line["cfg5_w8a8_static_gemm"] = w8a8
+        if stream_rows:
+            line["streaming_kernels"] = stream_rows
         if block_rows:
             line["block_output_fused"] = block_rows
         if int8_rows:
@@ -708,21 +946,29 @@ def run_cuda(args):
     return 0
 
 
+VARIANT_ORDER = ("fused", "plain", "unfused")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--variant", default="fused", choices=list(VARIANT_ORDER),
+                    help="fused: GEMM epilogues emit amax + FP8 copies (delayed scales); plain: bf16 outputs only; "
+                         "unfused: the same outputs as fused by separate cast passes")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--cpu-rows", type=int, default=8192)
     ap.add_argument("--ref-rows", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--also", default="cfg4,cfg3", help="comma-separated other configs to run briefly (N=1 only); '' for none")
+    ap.add_argument("--also", default="cfg2,cfg3", help="comma-separated other configs to run briefly (N=1 only); '' for none")
     ap.add_argument("--also-steps", type=int, default=20)
     ap.add_argument("--no-overlap", action="store_true", help="run the step on one stream (casts and GEMMs serialised)")
-    ap.add_argument("--no-w8a8", action="store_true", help="skip the config 5 inference GEMM sweep")
+    ap.add_argument("--no-w8a8", action="store_true", help="skip the config 5 sweep and the single-kernel rows")
+    ap.add_argument("--no-variants", action="store_true", help="skip the plain / unfused variants of the workload")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the >= 2 s replay legs")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps > 50:

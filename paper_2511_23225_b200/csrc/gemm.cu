@@ -692,19 +692,8 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
                                        (int)(200 * 1024 + 1024 + 256)));
     device_once_done(attr_done, attr_dev);
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(slabs * p.slices));
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)p.slices;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_fp8_skinny_kernel, mw, mx, p));
+  TWEO_CUDA_TRY(launch_chain(gemm_fp8_skinny_kernel, dim3((unsigned)(slabs * p.slices)), dim3(kThreads), smem, st,
+                             (unsigned)p.slices, mw, mx, p));
   count_launch();
   return check_launch("gemm_fp8_skinny_kernel");
 }

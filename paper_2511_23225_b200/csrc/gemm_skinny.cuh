@@ -97,12 +97,25 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
   const int kb1 = (int)((int64_t)p.k_blocks * (slice + 1) / p.slices);
   const uint32_t x_bytes = (uint32_t)p.Mpad * 128u;
 
+  // The kernel may have been launched while the kernel before it on the stream is still running (programmatic
+  // dependent launch).  W is a static weight, not something that kernel produced, so the first ring of W loads is
+  // issued at once; everything that can depend on the previous kernel -- the activations, the two scales, the
+  // output buffer -- is touched only after chain_wait().
+  chain_release();
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      for (int kb = kb0; kb < kb1; ++kb) {
+      const int pre = min(p.stages, kb1 - kb0);   // the ring is empty: these stages need no wait
+      for (int i = 0; i < pre; ++i) {
+        mbar_expect_tx(full_bar(i), BM * BK + x_bytes);
+        tma_load_2d(smem_base + i * p.stage_bytes, &tmap_w, (kb0 + i) * BK, n0, full_bar(i));
+      }
+      chain_wait();
+      for (int i = 0; i < pre; ++i)
+        tma_load_2d(smem_base + i * p.stage_bytes + BM * BK, &tmap_x, (kb0 + i) * BK, 0, full_bar(i));
+      int stage = pre == p.stages ? 0 : pre;
+      uint32_t phase = pre == p.stages ? 1u : 0u;
+      for (int kb = kb0 + pre; kb < kb1; ++kb) {
         if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) break;
         const uint32_t fb = full_bar(stage);
         mbar_expect_tx(fb, BM * BK + x_bytes);
@@ -114,6 +127,7 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
+    chain_wait();
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
@@ -134,6 +148,7 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
+    chain_wait();
     const int quarter = warp & 3;  // tensor-memory lanes [32*quarter, 32*quarter+32) belong to this warp
     const int col = n0 + quarter * 32 + lane;  // output column of this lane (= row of W)
     const float alpha = __fmul_rn(__ldg(p.sx_inv), __ldg(p.sw_inv));

@@ -2,10 +2,20 @@
 
 A step is one pass of every stage over one batch of synthetic input: for each
 linear of the block, the per-tensor FP8 casts of X, W (E4M3) and dY (E5M2) with
-current scaling, the forward GEMM and the backward call (data and weight gradient), and then
-the TWEO loss and gradient on the block output(s).  This module only sequences
-library calls and owns the device buffers; all arithmetic happens in the CUDA
-kernels behind ``binding``.
+current scaling, the forward GEMM and the two backward GEMMs, and then the TWEO
+loss and gradient on the block output(s).  Three variants of the GEMM part:
+
+  "fused"    (Sec. 4.3, delayed scaling) the forward and the data-gradient GEMM also
+             emit, from their epilogues, the amax of their bf16 output and its FP8
+             copy (Y in E4M3, dX in the gradient format) with the scale the amax
+             history of the earlier steps gives; one more small launch per format
+             rolls the histories and refreshes the scales for the next step;
+  "plain"    the GEMMs write bf16 only (data and weight gradient in one launch);
+  "unfused"  "plain" plus separate given-scale casts of Y and dX -- the same outputs
+             as "fused", produced by extra passes over the stored outputs.
+
+This module only sequences library calls and owns the device buffers; all
+arithmetic happens in the CUDA kernels behind ``binding``.
 """
 from __future__ import annotations
 
@@ -15,6 +25,9 @@ import torch
 from . import binding as tw
 from . import synth
 
+VARIANTS = ("fused", "plain", "unfused")
+AMAX_HISTORY = 16          # Sec. 4.3: amax history length of the delayed-scaling recipe
+
 
 def _pinned_bf16(bits: np.ndarray) -> torch.Tensor:
     t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
@@ -22,7 +35,7 @@ def _pinned_bf16(bits: np.ndarray) -> torch.Tensor:
 
 
 class LinearBuffers:
-    def __init__(self, lin: synth.Linear, M: int, device):
+    def __init__(self, lin: synth.Linear, M: int, device, fused_outputs: bool):
         self.lin, self.M = lin, M
         bf, u8, f32 = torch.bfloat16, torch.uint8, torch.float32
         K, N = lin.K, lin.N
@@ -36,6 +49,9 @@ class LinearBuffers:
         self.y = torch.empty((M, N), dtype=bf, device=device)
         self.dx = torch.empty((M, K), dtype=bf, device=device)
         self.dw = torch.empty((N, K), dtype=bf, device=device)
+        # FP8 copies of the outputs for the layer that consumes them (fused / unfused variants)
+        self.yq = torch.empty((M, N), dtype=u8, device=device) if fused_outputs else None
+        self.dxq = torch.empty((M, K), dtype=u8, device=device) if fused_outputs else None
 
     @property
     def flops(self) -> int:
@@ -45,13 +61,17 @@ class LinearBuffers:
 class BlockStep:
     """Device buffers + the launch sequence for one configuration (1..4)."""
 
-    def __init__(self, cfg_idx: int, M: int | None = None, device="cuda", grad_fmt=tw.E5M2):
+    def __init__(self, cfg_idx: int, M: int | None = None, device="cuda", grad_fmt=tw.E5M2, variant: str = "plain"):
+        if variant not in VARIANTS:
+            raise ValueError(f"variant must be one of {VARIANTS}")
         self.cfg = synth.CONFIGS[cfg_idx]
         self.cfg_idx = cfg_idx
         self.M = self.cfg.M if M is None else M
         self.device = device
         self.grad_fmt = grad_fmt
-        self.linears = [LinearBuffers(l, self.M, device) for l in self.cfg.linears]
+        self.variant = variant
+        extra = variant != "plain"
+        self.linears = [LinearBuffers(l, self.M, device, extra) for l in self.cfg.linears]
         self.n_blocks = self.cfg.n_blocks
         n = self.M * self.cfg.d
         self.a = [torch.empty((self.M, self.cfg.d), dtype=torch.bfloat16, device=device) for _ in range(self.n_blocks)]
@@ -66,6 +86,15 @@ class BlockStep:
         self.overlap = True   # casts and TWEO pass on a second stream, overlapping the GEMMs
         self.side = None
         self.tau, self.eps, self.p, self.lam = 3.0, 1e-6, 4.0, 0.01
+        if extra:
+            # delayed-scaling state of the outputs: one slot per linear, Y (E4M3) and dX (gradient format)
+            nl, f32 = len(self.linears), torch.float32
+            z = lambda *s: torch.zeros(s, dtype=f32, device=device)
+            self.amax_y, self.amax_dx = z(nl), z(nl)
+            self.hist_y, self.hist_dx = z(nl, AMAX_HISTORY), z(nl, AMAX_HISTORY)
+            self.scale_y, self.scale_dx = torch.ones(nl, dtype=f32, device=device), torch.ones(nl, dtype=f32, device=device)
+            self.scale_inv_y, self.scale_inv_dx = torch.ones(nl, dtype=f32, device=device), torch.ones(nl, dtype=f32, device=device)
+            self._scratch = z(4)
 
     # ---- inputs
     def make_host_inputs(self):
@@ -103,11 +132,41 @@ class BlockStep:
         # X, W (E4M3) and dY (E5M2), each with its own per-tensor scale, in one launch
         tw.quantize_per_tensor_batch([lb.x, lb.w, lb.dy], [lb.qx, lb.qw, lb.qdy], ws=self.quant_ws)
 
-    def gemms(self, lb: LinearBuffers):
+    def gemms(self, lb: LinearBuffers, i: int = 0):
+        if self.variant == "fused":
+            tw.fp8_linear_fwd(lb.qx.q, lb.qw.q, lb.qx.scale_inv, lb.qw.scale_inv, y=lb.y, out_amax=self.amax_y[i:i + 1],
+                              out_q=lb.yq, q_fmt=tw.E4M3, q_scale=self.scale_y[i:i + 1], ws=self.gemm_ws)
+            tw.fp8_linear_bwd_dgrad(lb.qdy.q, lb.qw.q, lb.qdy.scale_inv, lb.qw.scale_inv, fmt_dy=self.grad_fmt, dx=lb.dx,
+                                    out_amax=self.amax_dx[i:i + 1], out_q=lb.dxq, q_fmt=self.grad_fmt,
+                                    q_scale=self.scale_dx[i:i + 1], ws=self.gemm_ws)
+            tw.fp8_linear_bwd_wgrad(lb.qx.q, lb.qdy.q, lb.qx.scale_inv, lb.qdy.scale_inv, fmt_dy=self.grad_fmt, dw=lb.dw,
+                                    ws=self.gemm_ws)
+            return
         tw.fp8_linear_fwd(lb.qx.q, lb.qw.q, lb.qx.scale_inv, lb.qw.scale_inv, y=lb.y, ws=self.gemm_ws)
         # both gradients in one call (one kernel launch when the shapes allow)
         tw.fp8_linear_bwd(lb.qdy.q, lb.qx.q, lb.qw.q, lb.qdy.scale_inv, lb.qx.scale_inv, lb.qw.scale_inv,
                           fmt_dy=self.grad_fmt, dx=lb.dx, dw=lb.dw, ws=self.gemm_ws)
+        if self.variant == "unfused":
+            # the same extra outputs by separate passes: given-scale casts of the stored Y and dX
+            s = self._scratch
+            tw.quantize_per_tensor(lb.y, tw.E4M3, tw.SCALE_GIVEN,
+                                   out=tw.Quantized(lb.yq, self.scale_y[i:i + 1], s[0:1], self.amax_y[i:i + 1], None, tw.E4M3))
+            tw.quantize_per_tensor(lb.dx, self.grad_fmt, tw.SCALE_GIVEN,
+                                   out=tw.Quantized(lb.dxq, self.scale_dx[i:i + 1], s[1:2], self.amax_dx[i:i + 1], None,
+                                                    self.grad_fmt))
+
+    def update_output_scales(self):
+        """Delayed scaling of the outputs (Sec. 4.3): this step's amax values enter the histories and the scales
+        the NEXT step's epilogues use are refreshed; one launch per FP8 format."""
+        if self.variant == "plain":
+            return
+        tw.delayed_scaling_update(self.hist_y, self.amax_y, self.scale_y, self.scale_inv_y, tw.E4M3)
+        tw.delayed_scaling_update(self.hist_dx, self.amax_dx, self.scale_dx, self.scale_inv_dx, self.grad_fmt)
+
+    def all_gemms(self):
+        for i, lb in enumerate(self.linears):
+            self.gemms(lb, i)
+        self.update_output_scales()
 
     def tweo(self):
         c = self.lam / self.n_blocks
@@ -120,9 +179,10 @@ class BlockStep:
         linear i+1 and the TWEO pass: the casts are HBM-bound, the GEMMs tensor-bound, and they share the SMs.
         Fork / join on the calling stream, so the step can be captured into one CUDA graph."""
         if not self.overlap:
-            for lb in self.linears:
+            for i, lb in enumerate(self.linears):
                 self.quantize_all(lb)
-                self.gemms(lb)
+                self.gemms(lb, i)
+            self.update_output_scales()
             self.tweo()
             return
         main = torch.cuda.current_stream()
@@ -138,9 +198,10 @@ class BlockStep:
                 ev.record(side)
                 ready.append(ev)
             self.tweo()
-        for lb, ev in zip(self.linears, ready):
+        for i, (lb, ev) in enumerate(zip(self.linears, ready)):
             main.wait_event(ev)
-            self.gemms(lb)
+            self.gemms(lb, i)
+        self.update_output_scales()
         main.wait_stream(side)
 
     @property
@@ -150,8 +211,9 @@ class BlockStep:
     def working_set_bytes(self) -> int:
         tot = 0
         for lb in self.linears:
-            for t in (lb.x, lb.w, lb.dy, lb.qx.q, lb.qw.q, lb.qdy.q, lb.y, lb.dx, lb.dw):
-                tot += t.numel() * t.element_size()
+            for t in (lb.x, lb.w, lb.dy, lb.qx.q, lb.qw.q, lb.qdy.q, lb.y, lb.dx, lb.dw, lb.yq, lb.dxq):
+                if t is not None:
+                    tot += t.numel() * t.element_size()
         for t in self.a + self.ga:
             tot += t.numel() * t.element_size()
         return tot

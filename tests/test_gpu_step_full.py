@@ -101,3 +101,56 @@ def test_full_size_step_replayed_from_a_graph(tw, cfg, linears):
     ref_g = orc.tweo_grad_block(a1, tau, eps, p, c) * a1.size / n_all
     got_g = bs.ga[last][-64:].float().cpu().numpy().astype(np.float64)
     assert np.all(np.abs(got_g - ref_g) <= np.abs(ref_g) * 2.0 ** -8 + 1e-45)
+
+
+def test_full_size_fused_step_config4(tw):
+    """Config 4 as the benchmark runs it by default: forward and data-gradient GEMMs with the fused epilogue
+    (amax + FP8 copy of the output with a delayed scale, Sec. 4.3), replayed from a CUDA graph.  For the checked
+    linears: the bf16 outputs against the oracle's FP64 products on sampled points; the epilogue's amax and codes
+    bit for bit against the oracle's amax and given-scale cast of the output as stored, with the scale the
+    oracle's delayed-scaling rule derives from that amax (the inputs do not change between steps, so the history's
+    maximum is this step's amax); and the scale state left for the next step."""
+    from paper_2511_23225_b200.workload import BlockStep
+    bs = BlockStep(4, variant="fused")
+    host = bs.make_host_inputs()
+    bs.upload()
+    torch.cuda.synchronize()                        # the first step's amax values enter the scale histories
+    st = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        bs.step()                                   # first step: scales start at 1, the amax values enter the histories
+        bs.step()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=st):
+            bs.step()
+    torch.cuda.synchronize()
+    for lb in bs.linears:
+        for t in (lb.y, lb.dx, lb.dw, lb.yq, lb.dxq):
+            t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert tw.read_device_status() == 0
+    g = np.random.Generator(np.random.PCG64(4321))
+    for li in (1, 4):                               # o-projection and down-projection
+        lb = bs.linears[li]
+        x, w, dy = host["bits"]["lin"][li]
+        qx, qw, qd = (orc.quantize_per_tensor_current(x, E4M3), orc.quantize_per_tensor_current(w, E4M3),
+                      orc.quantize_per_tensor_current(dy, E5M2))
+        M, K = qx["q"].shape
+        N = qw["q"].shape[0]
+        r, c = points(g, M, N)
+        assert rel_fro(at(lb.y, r, c), orc.gemm_fwd_at(qx["q"], E4M3, qw["q"], E4M3, qx["scale_inv"], qw["scale_inv"], r, c)) <= GEMM_TOL
+        r, c = points(g, M, K)
+        assert rel_fro(at(lb.dx, r, c), orc.gemm_dgrad_at(qd["q"], E5M2, qw["q"], E4M3, qd["scale_inv"], qw["scale_inv"], r, c)) <= GEMM_TOL
+        r, c = points(g, N, K, n_rows=1, n_pts=512)
+        assert rel_fro(at(lb.dw, r, c), orc.gemm_wgrad_at(qx["q"], E4M3, qd["q"], E5M2, qx["scale_inv"], qd["scale_inv"], r, c)) <= GEMM_TOL
+        for out, outq, amax, scale, hist, fmt in ((lb.y, lb.yq, bs.amax_y, bs.scale_y, bs.hist_y, E4M3),
+                                                  (lb.dx, lb.dxq, bs.amax_dx, bs.scale_dx, bs.hist_dx, E5M2)):
+            bits = out.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+            want_amax = orc.amax_bf16(bits)
+            assert np.float32(amax[li].item()) == want_amax
+            want_scale = orc.scale_from_amax(want_amax, fmt)[0]
+            assert np.float32(scale[li].item()) == np.float32(want_scale)
+            assert np.float32(hist[li].max().item()) == want_amax
+            q_ref, _ = orc.quantize_bf16(bits, fmt, np.float32(want_scale))
+            assert np.array_equal(outq.cpu().numpy(), q_ref)
