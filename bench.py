@@ -799,6 +799,8 @@ def run_cuda(args):
                     "launch": "cuda graph replay of one captured step; two streams inside it: the casts of linear "
                               "i+1 and the TWEO pass overlap the GEMMs of linear i" if overlap
                     else "cuda graph replay of one captured step, one stream"}
+    if args.variant != "fused":
+        workload_cfg["launch"] += "; the three products of two linears share one grouped launch (the linears are independent problems)"
     if args.variant == "fused":
         workload_cfg["epilogue"] = ("forward and data-gradient GEMMs emit bf16 + amax + FP8 copy (Y E4M3, dX E5M2) with "
                                     "delayed scales (history 16); 2 scale-update launches per step")

@@ -266,6 +266,44 @@ TWEO_API tweo_status_t tweo_fp8_linear_bwd(const uint8_t* dyq, int64_t lddy, int
                                   size_t ws_bytes, void* stream);
 
 /*
+ * tweo_fp8_linear_group -- up to TWEO_MAX_GROUP products of FP8 linear layers that do not depend on each other,
+ * in ONE kernel launch (Sec. 4.3: every linear of the network runs these three products; which of them are
+ * independent is the caller's knowledge -- the forward products of projections that share an input, the weight
+ * gradients of several layers, the data and weight gradient of one layer).  Each problem is exactly
+ *   TWEO_PRODUCT_FWD    out = Y [M,N]  = tweo_fp8_linear_fwd       (xq, wq;  sx_inv, sw_inv)
+ *   TWEO_PRODUCT_DGRAD  out = dX [M,K] = tweo_fp8_linear_bwd_dgrad (dyq, wq; sdy_inv, sw_inv)
+ *   TWEO_PRODUCT_WGRAD  out = dW [N,K] = tweo_fp8_linear_bwd_wgrad (xq, dyq; sx_inv, sdy_inv; bf16, overwrite)
+ * without fused epilogue outputs and without a workspace; results are bit-identical to those calls.  A launch costs
+ * a fixed few microseconds (set-up, first loads, last epilogue) and leaves SMs idle at its ragged end; the tiles of
+ * all problems of a group form one list, longest first, dealt to the CTA pairs so that each gets about the same
+ * work, with one ramp-up and one tail for the whole group.
+ *   problems: HOST array of `count` descriptors (read during the call, not kept); only the operands the product
+ *   uses need to be set.  No output may alias an operand or another output of the group.
+ *   Shapes: as the single calls, and both dimensions of every output must exceed 128
+ *   (else TWEO_ERR_UNSUPPORTED_SHAPE: make the single call).
+ *   Errors: TWEO_ERR_INVALID_ARG (count, NULL pointers, enums), TWEO_ERR_UNSUPPORTED_SHAPE, TWEO_ERR_ALIGNMENT.
+ */
+#define TWEO_MAX_GROUP 8
+typedef enum { TWEO_PRODUCT_FWD = 0, TWEO_PRODUCT_DGRAD = 1, TWEO_PRODUCT_WGRAD = 2 } tweo_product_t;
+typedef struct tweo_linear_problem_t {
+  int32_t product;                      /* tweo_product_t */
+  int32_t fmt_x, fmt_w, fmt_dy;         /* tweo_fp8_t of the operands used */
+  const uint8_t* xq;                    /* [M,K] codes: FWD, WGRAD */
+  int64_t ldx;
+  const uint8_t* wq;                    /* [N,K] codes: FWD, DGRAD */
+  int64_t ldw;
+  const uint8_t* dyq;                   /* [M,N] codes: DGRAD, WGRAD */
+  int64_t lddy;
+  const float* sx_inv;                  /* device scalars */
+  const float* sw_inv;
+  const float* sdy_inv;
+  uint16_t* out;                        /* bf16: Y [M,N], dX [M,K] or dW [N,K] */
+  int64_t ldo;
+  int64_t M, N, K;
+} tweo_linear_problem_t;
+TWEO_API tweo_status_t tweo_fp8_linear_group(const tweo_linear_problem_t* problems, int32_t count, void* stream);
+
+/*
  * tweo_loss_fwd_bwd -- TWEO penalty and its gradient in one pass (Eq. 3, and
  * the derivative of Eq. 2's lambda(t) * L_TWEO term):
  *   loss_l = (1/n) sum_i (|a_i| / (tau+eps))^p,          l = 0..L-1

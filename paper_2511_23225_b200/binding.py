@@ -28,7 +28,7 @@ LIB_PATH = os.path.join(_HERE, "libtweo_b200.so")
 EXPORTS = [
     "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_fwd_act",
     "tweo_layernorm_fp8", "tweo_fp8_linear_bwd_dgrad",
-    "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
+    "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_fp8_linear_group", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
     "tweo_block_output_fused", "tweo_delayed_scaling_update", "tweo_absmax_quantize", "tweo_int8_linear", "tweo_int8_linear_q8", "tweo_residual_add_q8", "tweo_residual_add_q8_rows",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status", "tweo_selftest_bounded_wait",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
@@ -52,6 +52,16 @@ class _QuantDesc(C.Structure):
 
 
 MAX_QUANT_BATCH = 8
+MAX_GROUP = 8
+PRODUCT_FWD, PRODUCT_DGRAD, PRODUCT_WGRAD = 0, 1, 2
+
+
+class _LinearProblem(C.Structure):
+    _fields_ = [("product", C.c_int32), ("fmt_x", C.c_int32), ("fmt_w", C.c_int32), ("fmt_dy", C.c_int32),
+                ("xq", C.c_void_p), ("ldx", C.c_int64), ("wq", C.c_void_p), ("ldw", C.c_int64),
+                ("dyq", C.c_void_p), ("lddy", C.c_int64), ("sx_inv", C.c_void_p), ("sw_inv", C.c_void_p),
+                ("sdy_inv", C.c_void_p), ("out", C.c_void_p), ("ldo", C.c_int64),
+                ("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64)]
 
 
 class _Epilogue(C.Structure):
@@ -85,6 +95,7 @@ def lib() -> C.CDLL:
                                                 i64, i64, i64, vp, sz, vp]
         L.tweo_fp8_linear_bwd.argtypes = [vp, i64, i32, vp, i64, i32, vp, i64, i32, vp, vp, vp, vp, i64, vp, i64,
                                           i64, i64, i64, vp, sz, vp]
+        L.tweo_fp8_linear_group.argtypes = [C.POINTER(_LinearProblem), i32, vp]
         L.tweo_loss_fwd_bwd.argtypes = [C.POINTER(vp), i32, i64, f32, f32, f32, f32, vp, vp, C.POINTER(vp), i32,
                                         vp, sz, vp]
         L.tweo_loss_fwd_bwd_static.argtypes = [C.POINTER(vp), i32, i64, f32, f32, f32, f32, vp, vp, C.POINTER(vp),
@@ -387,6 +398,41 @@ def fp8_linear_bwd(dyq, xq, wq, sdy_inv, sx_inv, sw_inv, fmt_dy=E5M2, fmt_x=E4M3
                                      _dev(dw, torch.bfloat16, "dw"), _rows(dw, "dw"), M, N, K, *_ws(ws), _stream()),
            "tweo_fp8_linear_bwd")
     return dx, dw
+
+
+def fp8_linear_group(problems):
+    """tweo_fp8_linear_group: independent linear-layer products in one launch.  `problems` is a list of dicts:
+    {"product": PRODUCT_FWD, "xq", "wq", "sx_inv", "sw_inv", "out" [M,N]}, {"product": PRODUCT_DGRAD, "dyq", "wq",
+    "sdy_inv", "sw_inv", "out" [M,K]} or {"product": PRODUCT_WGRAD, "xq", "dyq", "sx_inv", "sdy_inv", "out" [N,K]},
+    each optionally with "fmt_x", "fmt_w", "fmt_dy" (defaults E4M3, E4M3, E5M2).  Outputs are bf16 tensors."""
+    n = len(problems)
+    if not 1 <= n <= MAX_GROUP:
+        raise ValueError("need 1..MAX_GROUP problems")
+    arr = (_LinearProblem * n)()
+    for q, d in zip(arr, problems):
+        q.product = d["product"]
+        q.fmt_x, q.fmt_w, q.fmt_dy = d.get("fmt_x", E4M3), d.get("fmt_w", E4M3), d.get("fmt_dy", E5M2)
+        xq, wq, dyq = d.get("xq"), d.get("wq"), d.get("dyq")
+        if q.product == PRODUCT_FWD:
+            (M, K), N = xq.shape, wq.shape[0]
+        elif q.product == PRODUCT_DGRAD:
+            (M, N), K = dyq.shape, wq.shape[1]
+        elif q.product == PRODUCT_WGRAD:
+            (M, K), N = xq.shape, dyq.shape[1]
+        else:
+            raise ValueError("product must be PRODUCT_FWD, PRODUCT_DGRAD or PRODUCT_WGRAD")
+        q.M, q.N, q.K = M, N, K
+        if xq is not None:
+            q.xq, q.ldx = _dev(xq, U8, "xq"), _rows(xq, "xq")
+        if wq is not None:
+            q.wq, q.ldw = _dev(wq, U8, "wq"), _rows(wq, "wq")
+        if dyq is not None:
+            q.dyq, q.lddy = _dev(dyq, U8, "dyq"), _rows(dyq, "dyq")
+        for name in ("sx_inv", "sw_inv", "sdy_inv"):
+            if d.get(name) is not None:
+                setattr(q, name, _dev(d[name], torch.float32, name))
+        q.out, q.ldo = _dev(d["out"], torch.bfloat16, "out"), _rows(d["out"], "out")
+    _check(lib().tweo_fp8_linear_group(arr, n, _stream()), "tweo_fp8_linear_group")
 
 
 def loss_fwd_bwd(blocks, tau=3.0, eps=1e-6, p=4.0, grad_coeff=1.0, want_grad=True, grad_dtype=BF16,

@@ -33,6 +33,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstdlib>
 #include <mutex>
@@ -312,7 +313,12 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 }
 
 
-__global__ void zero_float_kernel(float* p) { *p = 0.0f; }
+// Clears the amax cell of a fused epilogue.  Launched in the chain: the previous kernel may still read the cell.
+__global__ void zero_float_kernel(float* p) {
+  chain_release();
+  chain_wait();
+  *p = 0.0f;
+}
 
 // Self-test of the bounded wait: one thread waits on a barrier phase that nobody completes, with the
 // given limit; the wait gives up, records the expiry in the status word and the kernel returns.
@@ -544,7 +550,7 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
     return TWEO_ERR_CUDA;
   }
   if (p.out_amax) {
-    zero_float_kernel<<<1, 1, 0, st>>>(p.out_amax);
+    TWEO_CUDA_TRY(launch_chain(zero_float_kernel, dim3(1), dim3(1), 0, st, 0, p.out_amax));
     count_launch();
   }
   if (use_pair) {
@@ -567,18 +573,17 @@ tweo_status_t run_gemm(const Operand& A, const Operand& B, int64_t Md, int64_t N
 #undef TWEO_DISPATCH
 }
 
-// Forward product with the MLP activation and / or the FP8 copy of the output in the epilogue (pair
-// kernel only; every tile whole; the FP8 copy staged through shared memory, hence 5 stages).
-template <int ACT, bool B_MN = false>
-tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
-                              const CUtensorMap& mq, GemmParams& p, cudaStream_t st) {
-  // the per-element epilogues run with eight epilogue warps and four operand stages; SwiGLU (long
-  // contraction, 238 registers) keeps four warps and five stages
-  constexpr int EPIW = ACT == 3 ? 4 : 8;
-  constexpr int STAGES = ACT == 3 ? 5 : 4;
+// Forward product (or data gradient) with the MLP activation and / or the FP8 copy of the output in the
+// epilogue (pair kernel only; every tile whole; the FP8 copy staged through shared memory).
+// EPIW epilogue warps, STAGES operand stages, EBUF staging buffers per epilogue warp.
+template <int ACT, bool B_MN, int EPIW, int STAGES, int EBUF>
+tweo_status_t launch_pair_act_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
+                                  const CUtensorMap& mq, GemmParams& p, cudaStream_t st) {
   constexpr int THREADS = 64 + 32 * EPIW;
-  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + EPIW * 2 * 32 * 128 + EPIW * 2 * 32 * 64 + 1024 + 256;
-  auto kern = gemm_fp8_pair_kernel<false, B_MN, STAGES, false, false, ACT, true, EPIW>;
+  constexpr size_t smem =
+      (size_t)STAGES * (BM * BK + 128 * BK) + EPIW * EBUF * 32 * 128 + EPIW * EBUF * 32 * 64 + 1024 + 256;
+  static_assert(smem <= 227 * 1024, "shared memory per CTA");
+  auto kern = gemm_fp8_pair_kernel<false, B_MN, STAGES, false, false, ACT, true, EPIW, EBUF>;
   static std::atomic<uint64_t> attr_done{0};  // per device
   int attr_dev = 0;
   if (device_once_pending(attr_done, &attr_dev)) {
@@ -595,21 +600,23 @@ tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, cons
   int pairs = sm_count() / 2;
   p.raster_g = raster_band(p.tiles_m, pairs);
   if (pairs > tiles) pairs = tiles;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(2 * pairs));
-  cfg.blockDim = dim3(THREADS);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  TWEO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, md, mq, p));
+  TWEO_CUDA_TRY(launch_chain(kern, dim3((unsigned)(2 * pairs)), dim3(THREADS), smem, st, 2, ma, mb, md, mq, p));
   count_launch();
-  return check_launch("gemm_fp8_pair_kernel (activation epilogue)");
+  return check_launch("gemm_fp8_pair_kernel (fused epilogue)");
+}
+
+// Which configuration a product with a per-element epilogue takes (measured on B200, microseconds, forward
+// product with bf16 + amax + FP8 outputs; (epilogue warps, operand stages, staging buffers)):
+//   [8192x768].[2304x768]^T    (8,4,2) 19.3  (4,5,2) 19.1  (8,5,1) 18.3  (4,6,1) 20.7
+//   [16384x2048].[6144x2048]^T (8,4,2) 169.6 (4,5,2) 158.7 (8,5,1) 161.9 (4,6,1) 156.9
+// Short contractions are bound by the epilogue's issue rate (eight warps), long ones by the main loop, which
+// wants the deepest operand ring; one staging buffer per warp pays for the extra stage in both.
+template <int ACT, bool B_MN = false>
+tweo_status_t launch_pair_act(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
+                              const CUtensorMap& mq, GemmParams& p, cudaStream_t st) {
+  if (ACT == 3 || (p.Kc + BK - 1) / BK >= 16)          // SwiGLU (238 registers) always takes four warps
+    return launch_pair_act_cfg<ACT, B_MN, 4, 6, 1>(ma, mb, md, mq, p, st);
+  return launch_pair_act_cfg<(ACT == 3 ? 0 : ACT), B_MN, 8, 5, 1>(ma, mb, md, mq, p, st);
 }
 
 // D[M,N] = A[M,K] . B with A stored [M,K]; B stored [N,K] (w_mn false: the forward product) or [K,N] (w_mn
@@ -638,7 +645,7 @@ tweo_status_t run_fwd_act(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8
     return TWEO_ERR_CUDA;
   }
   if (p.out_amax) {
-    zero_float_kernel<<<1, 1, 0, st>>>(p.out_amax);
+    TWEO_CUDA_TRY(launch_chain(zero_float_kernel, dim3(1), dim3(1), 0, st, 0, p.out_amax));
     count_launch();
   }
   switch (act) {
@@ -665,18 +672,22 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   p.Mpad = (int32_t)((M + 15) / 16 * 16);
   p.k_blocks = (int32_t)((K + BK - 1) / BK);
   p.stage_bytes = (uint32_t)((BM * BK + p.Mpad * 128 + 1023) / 1024 * 1024);
-  p.stages = (int32_t)((200 * 1024) / p.stage_bytes);
+  // A ring of at most 100 KB, so that two CTAs fit an SM: the CTAs of the next kernel of a launch chain become
+  // resident (and fetch their first ring of W) while this kernel's are still reducing and writing.
+  p.stages = (int32_t)((100 * 1024) / p.stage_bytes);
   if (p.stages > kSkinnyMaxStages) p.stages = kSkinnyMaxStages;
+  if (p.stages < 2) p.stages = 2;
   p.tmem_cols = p.Mpad <= 32 ? 32u : (p.Mpad <= 64 ? 64u : 128u);
   p.idesc = make_idesc(fmt_w, fmt_x, false, false, p.Mpad, BM);
   p.sx_inv = sx_inv;
   p.sw_inv = sw_inv;
   const int sms = sm_count();
   const int slabs = (int)((N + 127) / 128);
-  // slices of K per slab = CTAs per cluster: as many as give every SM a CTA, a power of two up to the portable
-  // cluster size, at least four k-blocks each
+  // slices of K per slab = CTAs per cluster: the largest count up to the portable cluster size that keeps the grid
+  // within two CTAs per SM and leaves every slice at least four k-blocks
   p.slices = 1;
-  while (p.slices < 8 && slabs * p.slices * 2 <= sms && p.k_blocks / (p.slices * 2) >= 4) p.slices *= 2;
+  for (int sl = 2; sl <= 8; ++sl)
+    if (slabs * sl <= 2 * sms && p.k_blocks / sl >= 4) p.slices = sl;
   (void)ws;
   (void)ws_bytes;
   CUtensorMap mw, mx;
@@ -698,14 +709,23 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   return check_launch("gemm_fp8_skinny_kernel");
 }
 
-// dX and dW of one linear layer in ONE launch of the CTA-pair kernel (see gemm_pair_group.cuh).
-tweo_status_t run_bwd_group(const uint8_t* dyq, int64_t lddy, int fmt_dy, const uint8_t* xq, int64_t ldx, int fmt_x,
-                            const uint8_t* wq, int64_t ldw, int fmt_w, const float* sdy_inv, const float* sx_inv,
-                            const float* sw_inv, uint16_t* dx, int64_t lddx, uint16_t* dw, int64_t lddw, int64_t M,
-                            int64_t N, int64_t K, cudaStream_t st) {
+// Up to kGroupMaxProblems independent products in ONE launch of the CTA-pair kernel (see gemm_pair_group.cuh).
+// D[Md,Nd] = A . B over Kc; A stored [Md,Kc] (a_mn false) or [Kc,Md]; B stored [Nd,Kc] (b_mn false) or [Kc,Nd].
+struct GroupDesc {
+  const uint8_t *a, *b;
+  int64_t lda, ldb, Md, Nd, Kc;
+  int fa, fb;
+  bool a_mn, b_mn;
+  uint16_t* d;
+  int64_t ldd;
+  const float *sa, *sb;
+};
+
+template <int LIST>
+tweo_status_t run_group_list(GroupDesc* d, int n, cudaStream_t st) {
   constexpr int STAGES = 6;
   constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
-  auto kern = gemm_fp8_pair_group_kernel<STAGES>;
+  auto kern = gemm_fp8_pair_group_kernel<STAGES, LIST>;
   static std::atomic<uint64_t> attr_done{0};  // per device
   int attr_dev = 0;
   if (device_once_pending(attr_done, &attr_dev)) {
@@ -713,22 +733,11 @@ tweo_status_t run_bwd_group(const uint8_t* dyq, int64_t lddy, int fmt_dy, const 
     device_once_done(attr_done, attr_dev);
   }
   const int pairs_all = sm_count() / 2;
-  PairGroupParams g;
-  // product D: dX[M,K] = dYq[M,N] . Wq[N,K] (contraction N); product W: dW[N,K] = dYq^T . Xq (contraction M)
-  struct Desc {
-    const uint8_t *a, *b;
-    int64_t lda, ldb, Md, Nd, Kc;
-    int fa, fb;
-    bool a_mn;
-    uint16_t* d;
-    int64_t ldd;
-    const float *sa, *sb;
-  } d[2] = {{dyq, wq, lddy, ldw, M, K, N, fmt_dy, fmt_w, false, dx, lddx, sdy_inv, sw_inv},
-            {dyq, xq, lddy, ldx, N, K, M, fmt_dy, fmt_x, true, dw, lddw, sdy_inv, sx_inv}};
-  // the product with the longer tiles goes first in the tile list
-  if ((d[1].Kc + BK - 1) / BK > (d[0].Kc + BK - 1) / BK) std::swap(d[0], d[1]);
-  int tiles[2], cost[2];
-  for (int i = 0; i < 2; ++i) {
+  static thread_local PairGroupParams<LIST> g;   // 8 - 20 KB: kept off the stack
+  g.n_problems = n;
+  int cost[kGroupMaxProblems];
+  g.tile_start[0] = 0;
+  for (int i = 0; i < n; ++i) {
     GroupProblem& q = g.pr[i];
     q.Md = (int32_t)d[i].Md;
     q.Nd = (int32_t)d[i].Nd;
@@ -737,39 +746,42 @@ tweo_status_t run_bwd_group(const uint8_t* dyq, int64_t lddy, int fmt_dy, const 
     q.k_blocks = (int32_t)((d[i].Kc + BK - 1) / BK);
     q.raster_g = raster_band(q.tiles_m, pairs_all);
     q.a_mn = d[i].a_mn ? 1 : 0;
-    q.b_mn = 1;
-    q.idesc = make_idesc(d[i].fa, d[i].fb, d[i].a_mn, true, 256, 256);
+    q.b_mn = d[i].b_mn ? 1 : 0;
+    q.idesc = make_idesc(d[i].fa, d[i].fb, d[i].a_mn, d[i].b_mn, 256, 256);
     q.sa_inv = d[i].sa;
     q.sb_inv = d[i].sb;
-    tiles[i] = q.tiles_m * q.tiles_n;
+    g.tile_start[i + 1] = g.tile_start[i] + q.tiles_m * q.tiles_n;
     cost[i] = (q.k_blocks < 8 ? 8 : q.k_blocks) + 2;  // k-blocks, with a floor for the epilogue of short tiles
     bool ok = make_out_map(&g.md[i], d[i].d, d[i].Nd, d[i].Md, d[i].ldd, false);
     if (d[i].a_mn) ok = ok && make_map(&g.ma[i], d[i].a, d[i].Md, d[i].Kc, d[i].lda, BK);
     else ok = ok && make_map(&g.ma[i], d[i].a, d[i].Kc, d[i].Md, d[i].lda, BM);
-    ok = ok && make_map(&g.mb[i], d[i].b, d[i].Nd, d[i].Kc, d[i].ldb, BK);
+    if (d[i].b_mn) ok = ok && make_map(&g.mb[i], d[i].b, d[i].Nd, d[i].Kc, d[i].ldb, BK);
+    else ok = ok && make_map(&g.mb[i], d[i].b, d[i].Kc, d[i].Nd, d[i].ldb, 128);   // a pair CTA loads half of B
     if (!ok) {
       cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
       return TWEO_ERR_CUDA;
     }
   }
-  g.tiles0 = tiles[0];
-  g.total_tiles = tiles[0] + tiles[1];
+  for (int i = n; i <= kGroupMaxProblems; ++i) g.tile_start[i] = g.tile_start[n];
+  g.total_tiles = g.tile_start[n];
   g.pad = 0;
   int pairs = pairs_all < g.total_tiles ? pairs_all : g.total_tiles;
-  g.use_lists = (g.total_tiles <= kGroupMaxTiles && pairs <= kGroupMaxPairs) ? 1 : 0;
+  g.use_lists = (g.total_tiles <= LIST && pairs <= kGroupMaxPairs) ? 1 : 0;
   if (g.use_lists) {
     // longest processing time first: every tile goes to the pair with the least work so far
     typedef std::pair<int64_t, int> Load;  // (work, pair); smallest on top, ties to the lower pair index
     std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
     for (int p = 0; p < pairs; ++p) heap.push(Load(0, p));
-    uint8_t owner[kGroupMaxTiles];
+    static thread_local uint8_t owner[LIST];
     int count[kGroupMaxPairs + 1] = {0};
+    int prob = 0;
     for (int t = 0; t < g.total_tiles; ++t) {
+      while (t >= g.tile_start[prob + 1]) ++prob;
       Load l = heap.top();
       heap.pop();
       owner[t] = (uint8_t)l.second;
       ++count[l.second];
-      l.first += cost[t < tiles[0] ? 0 : 1];
+      l.first += cost[prob];
       heap.push(l);
     }
     int fill[kGroupMaxPairs + 1];
@@ -783,6 +795,28 @@ tweo_status_t run_bwd_group(const uint8_t* dyq, int64_t lddy, int fmt_dy, const 
   TWEO_CUDA_TRY(launch_chain(kern, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, st, 2, g));
   count_launch();
   return check_launch("gemm_fp8_pair_group_kernel");
+}
+
+tweo_status_t run_group(GroupDesc* d, int n, cudaStream_t st) {
+  if (n < 1 || n > kGroupMaxProblems) return TWEO_ERR_INVALID_ARG;
+  // the products with the longer tiles go first in the tile list (stable: equal lengths keep the caller's order)
+  std::stable_sort(d, d + n, [](const GroupDesc& x, const GroupDesc& y) {
+    return (x.Kc + BK - 1) / BK > (y.Kc + BK - 1) / BK;
+  });
+  int64_t tiles = 0;
+  for (int i = 0; i < n; ++i) tiles += ((d[i].Md + 2 * BM - 1) / (2 * BM)) * ((d[i].Nd + 255) / 256);
+  return tiles <= kGroupListSmall ? run_group_list<kGroupListSmall>(d, n, st) : run_group_list<kGroupListLarge>(d, n, st);
+}
+
+// dX and dW of one linear layer as a group of two products.
+tweo_status_t run_bwd_group(const uint8_t* dyq, int64_t lddy, int fmt_dy, const uint8_t* xq, int64_t ldx, int fmt_x,
+                            const uint8_t* wq, int64_t ldw, int fmt_w, const float* sdy_inv, const float* sx_inv,
+                            const float* sw_inv, uint16_t* dx, int64_t lddx, uint16_t* dw, int64_t lddw, int64_t M,
+                            int64_t N, int64_t K, cudaStream_t st) {
+  // product D: dX[M,K] = dYq[M,N] . Wq[N,K] (contraction N); product W: dW[N,K] = dYq^T . Xq (contraction M)
+  GroupDesc d[2] = {{dyq, wq, lddy, ldw, M, K, N, fmt_dy, fmt_w, false, true, dx, lddx, sdy_inv, sw_inv},
+                    {dyq, xq, lddy, ldx, N, K, M, fmt_dy, fmt_x, true, true, dw, lddw, sdy_inv, sx_inv}};
+  return run_group(d, 2, st);
 }
 
 bool fmt_ok(int f) { return f == TWEO_E4M3 || f == TWEO_E5M2; }
@@ -1033,6 +1067,39 @@ tweo_status_t tweo_fp8_linear_bwd(const uint8_t* dyq, int64_t lddy, int32_t fmt_
   if (s != TWEO_OK) return s;
   return tweo_fp8_linear_bwd_wgrad(xq, ldx, fmt_x, dyq, lddy, fmt_dy, sx_inv, sdy_inv, dw, lddw, TWEO_BF16, 0, M, N, K,
                                    ws, ws_bytes, stream);
+}
+
+tweo_status_t tweo_fp8_linear_group(const tweo_linear_problem_t* problems, int32_t count, void* stream) {
+  if (!problems || count < 1 || count > TWEO_MAX_GROUP) return TWEO_ERR_INVALID_ARG;
+  GroupDesc d[TWEO_MAX_GROUP];
+  for (int i = 0; i < count; ++i) {
+    const tweo_linear_problem_t& q = problems[i];
+    const int64_t M = q.M, N = q.N, K = q.K;
+    if (!q.out || M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
+    if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
+    if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
+    if (!tweo_detail::aligned16(q.out) || (q.ldo & 7)) return TWEO_ERR_ALIGNMENT;
+    switch (q.product) {
+      case TWEO_PRODUCT_FWD:    // Y[M,N] = Xq[M,K] . Wq[N,K]^T
+        if (!q.xq || !q.wq || !q.sx_inv || !q.sw_inv || !fmt_ok(q.fmt_x) || !fmt_ok(q.fmt_w)) return TWEO_ERR_INVALID_ARG;
+        d[i] = GroupDesc{q.xq, q.wq, q.ldx, q.ldw, M, N, K, q.fmt_x, q.fmt_w, false, false, q.out, q.ldo, q.sx_inv, q.sw_inv};
+        break;
+      case TWEO_PRODUCT_DGRAD:  // dX[M,K] = dYq[M,N] . Wq[N,K]
+        if (!q.dyq || !q.wq || !q.sdy_inv || !q.sw_inv || !fmt_ok(q.fmt_dy) || !fmt_ok(q.fmt_w)) return TWEO_ERR_INVALID_ARG;
+        d[i] = GroupDesc{q.dyq, q.wq, q.lddy, q.ldw, M, K, N, q.fmt_dy, q.fmt_w, false, true, q.out, q.ldo, q.sdy_inv, q.sw_inv};
+        break;
+      case TWEO_PRODUCT_WGRAD:  // dW[N,K] = dYq[M,N]^T . Xq[M,K]
+        if (!q.dyq || !q.xq || !q.sdy_inv || !q.sx_inv || !fmt_ok(q.fmt_dy) || !fmt_ok(q.fmt_x)) return TWEO_ERR_INVALID_ARG;
+        d[i] = GroupDesc{q.dyq, q.xq, q.lddy, q.ldx, N, K, M, q.fmt_dy, q.fmt_x, true, true, q.out, q.ldo, q.sdy_inv, q.sx_inv};
+        break;
+      default:
+        return TWEO_ERR_INVALID_ARG;
+    }
+    if (d[i].Md <= 128 || d[i].Nd <= 128) return TWEO_ERR_UNSUPPORTED_SHAPE;   // the pair kernel's 256 x 256 tiles
+    if (!tweo_detail::aligned16(d[i].a) || !tweo_detail::aligned16(d[i].b) || (d[i].lda & 15) || (d[i].ldb & 15))
+      return TWEO_ERR_ALIGNMENT;
+  }
+  return run_group(d, count, (cudaStream_t)stream);
 }
 
 tweo_status_t tweo_selftest_bounded_wait(uint64_t limit_ns, uint32_t* gave_up, void* stream) {

@@ -99,6 +99,18 @@ struct Sched {
   }
 };
 
+// The tiles of one worker of the CTA-pair kernel, in the order all three warp roles walk them: the
+// stream-K / round-robin list of Sched with the banded tile numbering.
+struct TileWalk {
+  Sched sched;
+  __device__ TileWalk(const GemmParams& p, int worker, int workers) : sched(p, worker, workers) {}
+  __device__ bool next(const GemmParams& p, int& tile, int& tm, int& tn, int& kb0, int& kb1) {
+    if (!sched.next(tile, kb0, kb1)) return false;
+    tile_coords(p, tile, tm, tn);
+    return true;
+  }
+};
+
 // ----------------------------------------------------------------- epilogue helpers
 template <int FMT>
 __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d) {

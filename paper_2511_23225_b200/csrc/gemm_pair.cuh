@@ -41,7 +41,12 @@ namespace tweo_detail {
 // epilogues that compute per element (activation, FP8 copy) are bound by the issue rate of one warp per
 // scheduler at short contractions; a second warp per scheduler doubles it.  Costs 48 KB more staging memory
 // (one operand stage less) and caps the kernel at 200 registers per thread.
-template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32, bool I8 = false, int ACT = 0, bool QST = false, int EPIW = 4>
+//
+// EBUF: staging buffers per epilogue warp (2: a chunk is staged while the store of the one before it drains;
+// 1: half the staging memory, which buys an operand stage -- with eight warps the second warp of a scheduler
+// covers the wait).
+template <bool A_MN, bool B_MN, int STAGES, bool OUT_F32, bool I8 = false, int ACT = 0, bool QST = false, int EPIW = 4,
+          int EBUF = 2>
 __global__ void __launch_bounds__(64 + 32 * EPIW, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const __grid_constant__ CUtensorMap tmap_d, const __grid_constant__ CUtensorMap tmap_q,
@@ -55,11 +60,12 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   constexpr uint32_t EPI_BUF = 32 * 128;
-  constexpr uint32_t EPI_BYTES = EPIW * 2 * EPI_BUF;
+  constexpr uint32_t EPI_BYTES = EPIW * EBUF * EPI_BUF;
+  static_assert(EBUF == 1 || EBUF == 2, "staging buffers per epilogue warp");
   static_assert(EPIW == 4 || EPIW == 8, "epilogue warps per CTA");
   constexpr bool Q8 = I8 && QST;                            // integer linear with an 8-bit (Eq. 4) output only
   constexpr uint32_t Q_BUF = 32 * 64;                       // 32 rows x 64 one-byte codes
-  constexpr uint32_t Q_BYTES = QST ? EPIW * 2 * Q_BUF : 0;
+  constexpr uint32_t Q_BYTES = QST ? EPIW * EBUF * Q_BUF : 0;
   uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES + Q_BYTES);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
@@ -94,9 +100,10 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   cluster_sync_all();  // both CTAs' barriers are initialised before anyone signals across
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // barriers and tensor memory are set up; from here on global memory of the kernel before this one is touched
+  // Barriers and tensor memory are set up.  The next kernel of the launch chain may start its own set-up now;
+  // every role works out its tile list first and only then waits for the kernel before this one (whose
+  // outputs may be this kernel's operands): nothing before chain_wait() touches global memory.
   chain_release();
-  chain_wait();
 
   const int pair = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;
@@ -107,21 +114,22 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      Sched sched(p, pair, num_pairs);
-      int tile, kb0, kb1;
-      while (ok && sched.next(tile, kb0, kb1)) {
-        int tm, tn;
-        tile_coords(p, tile, tm, tn);
+      TileWalk walk(p, pair, num_pairs);
+      tma_prefetch_desc(&tmap_a);
+      tma_prefetch_desc(&tmap_b);
+      chain_wait();
+      int tile, tm, tn, kb0, kb1;
+      while (ok && walk.next(p, tile, tm, tn, kb0, kb1)) {
         const int m0 = tm * (2 * BM) + (int)rank * BM;  // this CTA's rows
         const int n0 = ACT == 3 ? tn * 128 + (int)rank * p.Nd  // gate rows (leader) / up rows (peer)
                                 : tn * BN + (int)rank * 128;   // this CTA's half of B
         for (int kb = kb0; kb < kb1; ++kb) {
+          const int k0 = kb * BK;
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
           const uint32_t fb = map_to_cta(full_bar(stage), 0);
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
-          const int k0 = kb * BK;
           if (A_MN) tma_load_2d_pair(sa, &tmap_a, m0, k0, fb);
           else tma_load_2d_pair(sa, &tmap_a, k0, m0, fb);
           if (B_MN) tma_load_2d_pair(sb, &tmap_b, n0, k0, fb);
@@ -138,9 +146,10 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      Sched sched(p, pair, num_pairs);
-      int tile, kb0, kb1;
-      while (ok && sched.next(tile, kb0, kb1)) {
+      TileWalk walk(p, pair, num_pairs);
+      chain_wait();
+      int tile, tm, tn, kb0, kb1;
+      while (ok && walk.next(p, tile, tm, tn, kb0, kb1)) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
@@ -169,13 +178,19 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2 .. 1 + EPIW, both CTAs)
+    chain_wait();
     const int quarter = warp & 3;
     const float alpha = I8 ? 1.0f : __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
     const float qs = p.out_q ? (Q8 ? __fdiv_rn(p.q8_qmax, __ldg(p.q_scale)) : __ldg(p.q_scale)) : 0.0f;
     constexpr int CH = OUT_F32 ? 32 : 64;
-    const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
-    const uint32_t q_base = smem_u32(epi_smem) + EPI_BYTES + (uint32_t)(warp - 2) * 2u * Q_BUF;
-    uint32_t amax2 = 0u;  // packed running maximum of |bf16| bit patterns (whole chunks)
+    const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * (uint32_t)EBUF * EPI_BUF;
+    const uint32_t q_base = smem_u32(epi_smem) + EPI_BYTES + (uint32_t)(warp - 2) * (uint32_t)EBUF * Q_BUF;
+    // Running maximum for the fused amax.  Rounding to bf16 and the multiplication by the (positive) dequantisation
+    // scale are monotone in the magnitude, so max |bf16(acc * alpha)| = bf16(max |acc| * alpha): without an activation
+    // the maximum runs over the raw accumulators (one instruction per element), with one over the activation's
+    // binary32 results; the scale and the rounding are applied once at the end.  Accumulator rows and columns beyond
+    // the output are zero (the loader zero-fills), except the columns of a ragged SwiGLU tile, which are masked.
+    float run_max = 0.0f;
     const uint32_t row_off = (uint32_t)lane * 128u;
     const uint32_t swz = (uint32_t)(lane & 7);
     const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
@@ -184,19 +199,16 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    Sched sched(p, pair, num_pairs);
-    int tile, kb0, kb1;
-    while (ok && sched.next(tile, kb0, kb1)) {
-      int tm, tn;
-      tile_coords(p, tile, tm, tn);
+    TileWalk walk(p, pair, num_pairs);
+    int tile, tm, tn, kb0, kb1;
+    while (ok && walk.next(p, tile, tm, tn, kb0, kb1)) {
       const int m0 = tm * (2 * BM) + (int)rank * BM;
       const int n0 = ACT == 3 ? tn * 128 : tn * BN;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int row0 = m0 + quarter * 32;
       const int row = row0 + lane;
-      const bool row_ok = row < p.Md;
-      if (ACT == 0 && (kb0 != 0 || kb1 != p.k_blocks)) {
+      if (ACT == 0 && !QST && EBUF == 2 && (kb0 != 0 || kb1 != p.k_blocks)) {
         // part of a split tile: park the accumulator; the last share to arrive stores the tile
         const float part_amax = partial_share<BN, OUT_F32, true>(
             p, &tmap_d, tile, kb0, pair, num_pairs, (int)rank, warp - 2,
@@ -208,10 +220,10 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         if (acc == 0) acc_phase ^= 1u;
         continue;
       }
-#pragma unroll 1
       // with 8 epilogue warps, warps 2-5 take the first half of the tile's chunks and warps 6-9 the second
       constexpr int NC = (ACT == 3 ? 128 : BN) / CH, NC_W = NC / (EPIW / 4);
       const int c_first = ((warp - 2) >> 2) * NC_W;
+#pragma unroll 1
       for (int c = c_first; c < c_first + NC_W; ++c) {
         const int col0 = n0 + c * CH;
         if (col0 >= p.Nd) break;
@@ -257,12 +269,13 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             }
           }
         }
-        const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
-        if (lane == 0) bulk_wait_read<1>();
+        const uint32_t ebuf = EBUF == 2 ? (it & 1u) : 0u;
+        const uint32_t buf = epi_base + ebuf * EPI_BUF;
+        if (lane == 0) bulk_wait_read<EBUF - 1>();
         __syncwarp();
         if (Q8) {
           // Eq. 4 with the static output scale on the binary32 results: clamp(rne_int(y * (Q_b / s))), NaN -> 0
-          const uint32_t qrow = q_base + (it & 1u) * Q_BUF + (uint32_t)lane * 64u;
+          const uint32_t qrow = q_base + ebuf * Q_BUF + (uint32_t)lane * 64u;
           const uint32_t qswz = ((uint32_t)lane >> 1) & 3u;
           const int qmax = (int)p.q8_qmax;
 #pragma unroll
@@ -290,13 +303,31 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                          __float_as_uint(__fmul_rn(__uint_as_float(r[4 * j + 3]), alpha)));
         } else {
           uint32_t packed[CH / 2];
+          const bool want_max = QST && p.out_amax != nullptr;
+          const bool whole = ACT != 3 || col0 + CH <= p.Nd;   // only a ragged SwiGLU chunk has live columns beyond Nd
+          if (ACT == 0 && want_max) {
+#pragma unroll
+            for (int j = 0; j < CH; ++j) run_max = fmaxf(run_max, fabsf(__uint_as_float(r[j])));
+          }
 #pragma unroll
           for (int j = 0; j < CH / 2; ++j) {
-            if (ACT == 3)
-              packed[j] = f32x2_to_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-            else
-              packed[j] = f32x2_to_bf16x2(act_apply<ACT>(__fmul_rn(__uint_as_float(r[2 * j]), alpha)),
-                                          act_apply<ACT>(__fmul_rn(__uint_as_float(r[2 * j + 1]), alpha)));
+            float v0, v1;
+            if (ACT == 3) {
+              v0 = __uint_as_float(r[2 * j]);
+              v1 = __uint_as_float(r[2 * j + 1]);
+            } else {
+              v0 = act_apply<ACT>(__fmul_rn(__uint_as_float(r[2 * j]), alpha));
+              v1 = act_apply<ACT>(__fmul_rn(__uint_as_float(r[2 * j + 1]), alpha));
+            }
+            if (ACT != 0 && want_max) {
+              if (whole) {
+                run_max = fmaxf(run_max, fmaxf(fabsf(v0), fabsf(v1)));
+              } else {
+                if (col0 + 2 * j < p.Nd) run_max = fmaxf(run_max, fabsf(v0));
+                if (col0 + 2 * j + 1 < p.Nd) run_max = fmaxf(run_max, fabsf(v1));
+              }
+            }
+            packed[j] = f32x2_to_bf16x2(v0, v1);
           }
           if (ACT == 0 || p.d != nullptr) {
 #pragma unroll
@@ -305,22 +336,9 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                            packed[4 * j + 2], packed[4 * j + 3]);
           }
           if (QST) {
-            // whole chunks inside the output take the packed integer maximum; ragged ones go element by element
-            if (p.out_amax && row_ok) {
-              if (col0 + CH <= p.Nd) {
-#pragma unroll
-                for (int j = 0; j < CH / 2; ++j) amax2 = absmax_bits(amax2, packed[j]);
-              } else {
-#pragma unroll
-                for (int j = 0; j < CH / 2; ++j) {
-                  if (col0 + 2 * j < p.Nd) run_amax = fmaxf(run_amax, fabsf(bf16lo_to_f32(packed[j])));
-                  if (col0 + 2 * j + 1 < p.Nd) run_amax = fmaxf(run_amax, fabsf(bf16hi_to_f32(packed[j])));
-                }
-              }
-            }
             if (p.out_q) {
               // 64 codes per row -> 32 rows x 64 B, 16-byte pieces XOR-swizzled with row bits 1-2
-              const uint32_t qbuf = q_base + (it & 1u) * Q_BUF;
+              const uint32_t qbuf = q_base + ebuf * Q_BUF;
               const uint32_t qrow = qbuf + (uint32_t)lane * 64u;
               const uint32_t qswz = ((uint32_t)lane >> 1) & 3u;
 #pragma unroll
@@ -344,7 +362,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             if (OUT_F32 && p.accumulate) tma_reduce_add_2d(&tmap_d, col0, row0, buf);
             else tma_store_2d(&tmap_d, col0, row0, buf);
           }
-          if (QST && p.out_q) tma_store_2d(&tmap_q, col0, row0, q_base + (it & 1u) * Q_BUF);
+          if (QST && p.out_q) tma_store_2d(&tmap_q, col0, row0, q_base + ebuf * Q_BUF);
           bulk_commit();
         }
         ++it;
@@ -357,7 +375,11 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
     if (lane == 0) bulk_wait_all();
     if (p.out_amax) {
-      run_amax = warp_max(fmaxf(run_amax, __uint_as_float(absmax_fold(amax2) << 16)));
+      if (QST) {
+        const float m = ACT == 0 ? __fmul_rn(run_max, fabsf(alpha)) : run_max;
+        run_amax = fmaxf(run_amax, __uint_as_float(f32_to_bf16_bits(m) << 16));   // the same rounding the stored values got
+      }
+      run_amax = warp_max(run_amax);
       if (lane == 0 && run_amax > 0.0f)
         atomicMax(reinterpret_cast<unsigned int*>(p.out_amax), __float_as_uint(run_amax));
     }

@@ -1,11 +1,14 @@
-// Two FP8 GEMMs in one launch of the CTA-pair kernel: the data gradient and the weight gradient
-// of a linear layer, which the backward pass needs together and which share dY.  Launched
-// separately, each leaves SMs idle -- the weight gradient of a transformer linear has only a few
-// dozen (long) tiles, the data gradient often 1.3 waves of short ones.  Here the tiles of both
-// products form one list, longest first, and the host assigns them to the CTA pairs by the
-// longest-processing-time rule (each tile goes to the pair with the least work so far), so the
-// long tiles start at once and the short ones fill in around them; one ramp-up and one tail
-// instead of two.
+// Several independent FP8 GEMMs in one launch of the CTA-pair kernel.  The case it was built for is
+// the data gradient and the weight gradient of a linear layer, which the backward pass needs
+// together and which share dY: launched separately, each leaves SMs idle -- the weight gradient of a
+// transformer linear has only a few dozen (long) tiles, the data gradient often 1.3 waves of short
+// ones.  More generally every launch pays a fixed cost (launch, set-up, the first cold loads, the
+// last tile's epilogue: about 5 us, a third of a product of a GPT-2-small-sized linear), so up to
+// kGroupMaxProblems products that do not depend on each other -- the forward products of several
+// linears, or all their gradients -- share one.  The tiles of all products form one list, longest
+// first, and the host assigns them to the CTA pairs by the longest-processing-time rule (each tile
+// goes to the pair with the least work so far), so the long tiles start at once and the short ones
+// fill in around them; one ramp-up and one tail for the whole group.
 //
 // The kernel is the CTA-pair kernel of gemm_pair.cuh (256 x 256 tiles, tcgen05 cta_group::2,
 // TMA-fed ring, two accumulators in tensor memory, staged TMA-store epilogue) with the operand
@@ -20,7 +23,9 @@
 
 namespace tweo_detail {
 
-constexpr int kGroupMaxTiles = 1024;  // beyond that the tiles are dealt round-robin (balance is no issue then)
+constexpr int kGroupMaxProblems = 8;
+constexpr int kGroupListSmall = 2048;  // tile-list capacities the kernel is built for (the list travels in the
+constexpr int kGroupListLarge = 8192;  // kernel parameters); beyond the large one tiles are dealt round-robin
 constexpr int kGroupMaxPairs = 127;
 
 struct GroupProblem {
@@ -32,24 +37,28 @@ struct GroupProblem {
   const float* sb_inv;
 };
 
+template <int LIST>
 struct alignas(64) PairGroupParams {
-  CUtensorMap ma[2], mb[2], md[2];
-  GroupProblem pr[2];
-  int32_t tiles0;        // tiles of product 0; they are numbered first
+  CUtensorMap ma[kGroupMaxProblems], mb[kGroupMaxProblems], md[kGroupMaxProblems];
+  GroupProblem pr[kGroupMaxProblems];
+  int32_t n_problems;
+  int32_t tile_start[kGroupMaxProblems + 1];  // product i owns the tile numbers [tile_start[i], tile_start[i + 1])
   int32_t total_tiles;
-  int32_t use_lists;     // the per-pair lists are valid (total_tiles <= kGroupMaxTiles)
+  int32_t use_lists;     // the per-pair lists are valid (total_tiles <= LIST)
   int32_t pad;
   uint16_t first[kGroupMaxPairs + 1];  // pair p computes list[first[p]] .. list[first[p + 1] - 1], in that order
-  uint16_t list[kGroupMaxTiles];       // tile numbers
+  uint16_t list[LIST];                 // tile numbers
 };
 
 // The tile list of one CTA pair, identical in every warp role.
 struct GroupSched {
   int pos, end, t, worker, workers;
-  __device__ GroupSched(const PairGroupParams& g, int worker_, int workers_)
+  template <int LIST>
+  __device__ GroupSched(const PairGroupParams<LIST>& g, int worker_, int workers_)
       : pos(g.use_lists ? g.first[worker_] : 0), end(g.use_lists ? g.first[worker_ + 1] : 0), t(-1), worker(worker_),
         workers(workers_) {}
-  __device__ bool next(const PairGroupParams& g, int& prob, int& tile) {
+  template <int LIST>
+  __device__ bool next(const PairGroupParams<LIST>& g, int& prob, int& tile) {
     if (g.use_lists) {
       if (pos >= end) return false;
       t = g.list[pos++];
@@ -57,8 +66,9 @@ struct GroupSched {
       t = t < 0 ? worker : t + workers;
       if (t >= g.total_tiles) return false;
     }
-    prob = t >= g.tiles0 ? 1 : 0;
-    tile = prob ? t - g.tiles0 : t;
+    prob = 0;
+    while (prob + 1 < g.n_problems && t >= g.tile_start[prob + 1]) ++prob;
+    tile = t - g.tile_start[prob];
     return true;
   }
 };
@@ -73,9 +83,9 @@ __device__ __forceinline__ void group_tile_coords(const GroupProblem& q, int til
   tm = first + in - tn * rows;
 }
 
-template <int STAGES>
+template <int STAGES, int LIST>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams g) {
+gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams<LIST> g) {
   constexpr int BN = 256;                 // tile columns of the pair
   constexpr uint32_t A_BYTES = BM * BK;   // this CTA's 128 rows of A
   constexpr uint32_t B_BYTES = 128 * BK;  // this CTA's 128 of the 256 columns of B
@@ -122,9 +132,10 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams g) {
   cluster_sync_all();  // both CTAs' barriers are initialised before anyone signals across
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // barriers and tensor memory are set up; from here on global memory of the kernel before this one is touched
+  // Barriers and tensor memory are set up: the next kernel of the launch chain may start its own set-up.  Every
+  // role prepares its tile list first and only then waits for the kernel before this one; nothing before
+  // chain_wait() touches global memory.
   chain_release();
-  chain_wait();
 
   const int pair = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;
@@ -136,6 +147,11 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams g) {
       uint32_t phase = 0;
       bool ok = true;
       GroupSched sched(g, pair, num_pairs);
+      for (int i = 0; i < g.n_problems; ++i) {
+        tma_prefetch_desc(&g.ma[i]);
+        tma_prefetch_desc(&g.mb[i]);
+      }
+      chain_wait();
       int prob, tile;
       while (ok && sched.next(g, prob, tile)) {
         const GroupProblem& q = g.pr[prob];
@@ -170,6 +186,7 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams g) {
       uint32_t acc_phase = 0;
       bool ok = true;
       GroupSched sched(g, pair, num_pairs);
+      chain_wait();
       int prob, tile;
       while (ok && sched.next(g, prob, tile)) {
         const GroupProblem& q = g.pr[prob];
@@ -203,6 +220,7 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams g) {
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    chain_wait();
     const int quarter = warp & 3;
     const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
     const uint32_t row_off = (uint32_t)lane * 128u;

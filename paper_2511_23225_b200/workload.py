@@ -10,7 +10,9 @@ loss and gradient on the block output(s).  Three variants of the GEMM part:
              copy (Y in E4M3, dX in the gradient format) with the scale the amax
              history of the earlier steps gives; one more small launch per format
              rolls the histories and refreshes the scales for the next step;
-  "plain"    the GEMMs write bf16 only (data and weight gradient in one launch);
+  "plain"    the GEMMs write bf16 only; the linears of a configuration are independent problems here (each has
+             its own X, W and dY), so the three products of TWO linears share one grouped launch
+             (the fused variant's epilogue kernels run one product per launch);
   "unfused"  "plain" plus separate given-scale casts of Y and dX -- the same outputs
              as "fused", produced by extra passes over the stored outputs.
 
@@ -147,13 +149,47 @@ class BlockStep:
         tw.fp8_linear_bwd(lb.qdy.q, lb.qx.q, lb.qw.q, lb.qdy.scale_inv, lb.qx.scale_inv, lb.qw.scale_inv,
                           fmt_dy=self.grad_fmt, dx=lb.dx, dw=lb.dw, ws=self.gemm_ws)
         if self.variant == "unfused":
-            # the same extra outputs by separate passes: given-scale casts of the stored Y and dX
-            s = self._scratch
-            tw.quantize_per_tensor(lb.y, tw.E4M3, tw.SCALE_GIVEN,
-                                   out=tw.Quantized(lb.yq, self.scale_y[i:i + 1], s[0:1], self.amax_y[i:i + 1], None, tw.E4M3))
-            tw.quantize_per_tensor(lb.dx, self.grad_fmt, tw.SCALE_GIVEN,
-                                   out=tw.Quantized(lb.dxq, self.scale_dx[i:i + 1], s[1:2], self.amax_dx[i:i + 1], None,
-                                                    self.grad_fmt))
+            self.cast_outputs(lb, i)
+
+    def cast_outputs(self, lb: LinearBuffers, i: int):
+        """The extra outputs of the fused variant by separate passes: given-scale casts of the stored Y and dX."""
+        s = self._scratch
+        tw.quantize_per_tensor(lb.y, tw.E4M3, tw.SCALE_GIVEN,
+                               out=tw.Quantized(lb.yq, self.scale_y[i:i + 1], s[0:1], self.amax_y[i:i + 1], None, tw.E4M3))
+        tw.quantize_per_tensor(lb.dx, self.grad_fmt, tw.SCALE_GIVEN,
+                               out=tw.Quantized(lb.dxq, self.scale_dx[i:i + 1], s[1:2], self.amax_dx[i:i + 1], None,
+                                                self.grad_fmt))
+
+    def group_ok(self, lb: LinearBuffers) -> bool:
+        """Whether all three products of this linear can go into a grouped launch (outputs wider and taller than 128)."""
+        return self.variant != "fused" and min(self.M, lb.lin.K, lb.lin.N) > 128
+
+    def gemms_grouped(self, lbs):
+        """Forward, data-gradient and weight-gradient product of each of the given linears in ONE launch."""
+        probs = []
+        for lb in lbs:
+            probs += [dict(product=tw.PRODUCT_FWD, xq=lb.qx.q, wq=lb.qw.q, sx_inv=lb.qx.scale_inv, sw_inv=lb.qw.scale_inv, out=lb.y),
+                      dict(product=tw.PRODUCT_DGRAD, dyq=lb.qdy.q, wq=lb.qw.q, sdy_inv=lb.qdy.scale_inv, sw_inv=lb.qw.scale_inv,
+                           fmt_dy=self.grad_fmt, out=lb.dx),
+                      dict(product=tw.PRODUCT_WGRAD, xq=lb.qx.q, dyq=lb.qdy.q, sx_inv=lb.qx.scale_inv, sdy_inv=lb.qdy.scale_inv,
+                           fmt_dy=self.grad_fmt, out=lb.dw)]
+        tw.fp8_linear_group(probs)
+
+    def gemm_batches(self):
+        """The linears in launch order: pairs that share a grouped launch (plain variant), else one by one."""
+        idx = list(range(len(self.linears)))
+        if not all(self.group_ok(lb) for lb in self.linears):
+            return [[i] for i in idx]
+        return [idx[i:i + 2] for i in range(0, len(idx), 2)]
+
+    def run_gemm_batch(self, batch):
+        if len(batch) == 1 and not self.group_ok(self.linears[batch[0]]):
+            self.gemms(self.linears[batch[0]], batch[0])
+        else:
+            self.gemms_grouped([self.linears[i] for i in batch])
+            if self.variant == "unfused":
+                for i in batch:
+                    self.cast_outputs(self.linears[i], i)
 
     def update_output_scales(self):
         """Delayed scaling of the outputs (Sec. 4.3): this step's amax values enter the histories and the scales
@@ -164,8 +200,8 @@ class BlockStep:
         tw.delayed_scaling_update(self.hist_dx, self.amax_dx, self.scale_dx, self.scale_inv_dx, self.grad_fmt)
 
     def all_gemms(self):
-        for i, lb in enumerate(self.linears):
-            self.gemms(lb, i)
+        for batch in self.gemm_batches():
+            self.run_gemm_batch(batch)
         self.update_output_scales()
 
     def tweo(self):
@@ -179,9 +215,10 @@ class BlockStep:
         linear i+1 and the TWEO pass: the casts are HBM-bound, the GEMMs tensor-bound, and they share the SMs.
         Fork / join on the calling stream, so the step can be captured into one CUDA graph."""
         if not self.overlap:
-            for i, lb in enumerate(self.linears):
-                self.quantize_all(lb)
-                self.gemms(lb, i)
+            for batch in self.gemm_batches():
+                for i in batch:
+                    self.quantize_all(self.linears[i])
+                self.run_gemm_batch(batch)
             self.update_output_scales()
             self.tweo()
             return
@@ -198,9 +235,9 @@ class BlockStep:
                 ev.record(side)
                 ready.append(ev)
             self.tweo()
-        for i, (lb, ev) in enumerate(zip(self.linears, ready)):
-            main.wait_event(ev)
-            self.gemms(lb, i)
+        for batch in self.gemm_batches():
+            main.wait_event(ready[batch[-1]])       # the casts of the batch's last linear: the earlier ones are done too
+            self.run_gemm_batch(batch)
         self.update_output_scales()
         main.wait_stream(side)
 

@@ -1,0 +1,82 @@
+"""tweo_fp8_linear_group: several independent linear-layer products in one launch.  Every output must equal the
+single call's bit for bit (same tiles, same order along the contraction) and match the oracle's FP64 product."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tweo_oracle as orc
+from paper_2511_23225_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+E4M3, E5M2 = 0, 1
+GEMM_TOL = 1e-2
+
+
+@pytest.fixture(scope="module")
+def tw():
+    from paper_2511_23225_b200 import binding
+    binding.lib()
+    return binding
+
+
+def dev_scalar(v):
+    return torch.tensor([float(v)], dtype=torch.float32, device="cuda")
+
+
+def make_linear(seed, M, K, N, fmt_g=E5M2):
+    x = synth.normal_with_outlier_channels_bf16(seed, (M, K))
+    w = synth.normal_bf16(seed + 1, (N, K), 0.02)
+    dy = synth.normal_bf16(seed + 2, (M, N), 1e-3)
+    q = [orc.quantize_per_tensor_current(x, E4M3), orc.quantize_per_tensor_current(w, E4M3),
+         orc.quantize_per_tensor_current(dy, fmt_g)]
+    dev = [torch.from_numpy(t["q"]).cuda() for t in q]
+    sc = [dev_scalar(t["scale_inv"]) for t in q]
+    return q, dev, sc
+
+
+def rel(got, ref):
+    return float(np.linalg.norm(got.float().cpu().numpy().astype(np.float64) - ref) / np.linalg.norm(ref))
+
+
+@pytest.mark.parametrize("fmt_g", [E5M2, E4M3], ids=["e5m2grad", "e4m3grad"])
+def test_group_of_seven_products_equals_the_single_calls(tw, fmt_g):
+    lins = [make_linear(600, 300, 400, 272, fmt_g), make_linear(610, 1024, 768, 2304, fmt_g),
+            make_linear(620, 2048, 256, 384, fmt_g)]
+    problems, singles, refs = [], [], []
+    for (q, (xq, wq, dyq), (sx, sw, sd)) in lins:
+        M, K = xq.shape
+        N = wq.shape[0]
+        bf = lambda r, c: torch.zeros((r, c), dtype=torch.bfloat16, device="cuda")
+        problems += [dict(product=tw.PRODUCT_FWD, xq=xq, wq=wq, sx_inv=sx, sw_inv=sw, out=bf(M, N)),
+                     dict(product=tw.PRODUCT_DGRAD, dyq=dyq, wq=wq, sdy_inv=sd, sw_inv=sw, fmt_dy=fmt_g, out=bf(M, K)),
+                     dict(product=tw.PRODUCT_WGRAD, xq=xq, dyq=dyq, sx_inv=sx, sdy_inv=sd, fmt_dy=fmt_g, out=bf(N, K))]
+        singles += [tw.fp8_linear_fwd(xq, wq, sx, sw), tw.fp8_linear_bwd_dgrad(dyq, wq, sd, sw, fmt_dy=fmt_g),
+                    tw.fp8_linear_bwd_wgrad(xq, dyq, sx, sd, fmt_dy=fmt_g)]
+        refs += [orc.gemm_fwd(q[0]["q"], E4M3, q[1]["q"], E4M3, q[0]["scale_inv"], q[1]["scale_inv"]),
+                 orc.gemm_dgrad(q[2]["q"], fmt_g, q[1]["q"], E4M3, q[2]["scale_inv"], q[1]["scale_inv"]),
+                 orc.gemm_wgrad(q[0]["q"], E4M3, q[2]["q"], fmt_g, q[0]["scale_inv"], q[2]["scale_inv"])]
+    problems, singles, refs = problems[:7] + problems[8:], singles[:7] + singles[8:], refs[:7] + refs[8:]   # 8 of the 9
+    tw.fp8_linear_group(problems)
+    tw.fp8_linear_group(problems[3:5])          # a group of two, again into the same outputs
+    torch.cuda.synchronize()
+    assert tw.read_device_status() == 0
+    for prob, one, ref in zip(problems, singles, refs):
+        assert torch.equal(prob["out"].view(torch.int16), one.view(torch.int16)), prob["product"]
+        assert rel(prob["out"], ref) <= GEMM_TOL
+
+
+def test_group_rejects_what_it_cannot_tile(tw):
+    q, (xq, wq, dyq), (sx, sw, sd) = make_linear(630, 64, 256, 256)
+    out = torch.empty((64, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(tw.TweoError) as e:
+        tw.fp8_linear_group([dict(product=tw.PRODUCT_FWD, xq=xq, wq=wq, sx_inv=sx, sw_inv=sw, out=out)])   # 64 rows
+    assert e.value.status == 2
+    with pytest.raises(ValueError):
+        tw.fp8_linear_group([])
+    with pytest.raises(ValueError):
+        tw.fp8_linear_group([dict(product=7, xq=xq, wq=wq, sx_inv=sx, sw_inv=sw, out=out)])
+    big = torch.empty((256, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(tw.TweoError) as e:      # a product whose operands were not given
+        tw.fp8_linear_group([dict(product=tw.PRODUCT_DGRAD, dyq=dyq.new_zeros((256, 256)), wq=wq, sw_inv=sw, out=big)])
+    assert e.value.status == 1
