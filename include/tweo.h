@@ -318,8 +318,9 @@ TWEO_API tweo_status_t tweo_fp8_linear_group(const tweo_linear_problem_t* proble
  *      grad_dtype), or NULL for loss only.  grad[l] may alias a[l] only if
  *      grad_dtype is bf16 (in-place).
  *   p = 4 (the paper's setting) runs a fast path; other p > 1 a generic one.
- *   Needs a workspace (TWEO_OP_LOSS); the sum is reduced in a fixed order, so
- *   results are bit-reproducible run to run.
+ *   Needs a workspace (TWEO_OP_LOSS, any contents); the sum is reduced in a fixed order,
+ *   so results are bit-reproducible run to run.  Two kernels: the streaming pass and a
+ *   one-CTA kernel that adds its partial sums.
  */
 TWEO_API tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, int64_t n_per_tensor, float tau,
                                 float eps, float p, float grad_coeff, float* loss,
@@ -338,8 +339,8 @@ TWEO_API tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, in
  * Every output equals, bit for bit, what tweo_loss_fwd_bwd (L = 1, bf16 gradient) and
  * tweo_quantize_per_tensor (GIVEN) produce from the stored a.  x, f: bf16 [n], device.
  * loss, amax: device float*.  q_scale: device const float*, required with aq.  grad must
- * not alias x, f or a.  Needs a zero-initialised workspace of
- * tweo_workspace_bytes(TWEO_OP_BLOCK_OUTPUT) bytes; the reduction order is fixed, so results
+ * not alias x, f or a.  Needs a workspace of
+ * tweo_workspace_bytes(TWEO_OP_BLOCK_OUTPUT) bytes (any contents); the reduction order is fixed, so results
  * are reproducible run to run.
  */
 TWEO_API tweo_status_t tweo_block_output_fused(const uint16_t* x, const uint16_t* f, int64_t n, float tau,
@@ -369,14 +370,14 @@ TWEO_API tweo_status_t tweo_delayed_scaling_update(float* amax_history, int32_t 
  * pool at start-up and forbids later cudaMalloc calls, a plug-in running inside a host
  * application that owns the allocator, or a control loop that cannot tolerate the latency
  * or the possible failure of an allocation.  For them the scratch memory of the loss
- * kernel (its per-CTA partial sums and its ticket counter) is a fixed 33024-byte array
+ * kernel (its per-CTA partial sums) is a fixed 33024-byte array
  * compiled into the library; every GPU that loads the library holds it until the process
  * exits.  Inputs and outputs are still the caller's.  Arguments, results and numerics are
  * those of tweo_loss_fwd_bwd (same kernel, same reduction order).
  *
  *   Limit: L * (CTAs per tensor) must not exceed 4096 partial sums; beyond that the call
  *     returns TWEO_ERR_WORKSPACE_TOO_SMALL and does nothing (on a 148-SM B200 the kernel
- *     uses at most 1184 + L CTAs, so every L <= TWEO_MAX_BLOCKS fits).
+ *     uses at most 888 + L CTAs, so every L <= TWEO_MAX_BLOCKS fits).
  *   The call performs no cudaMalloc / cudaFree and calls no allocating routine.
  *   First call on a device: looks up the array's device address (once per device, with
  *     that device current).  Make that first call outside any stream capture.

@@ -139,9 +139,7 @@ absmax_tensor_kernel(const uint16_t* x, int64_t n, float eps, float Q, float* s_
 }
 
 int grid_cap(int64_t want, int per_sm) {
-  const int64_t cap = (int64_t)sm_count() * per_sm;
-  if (want > cap) want = cap;
-  return (int)(want < 1 ? 1 : want);
+  return balanced_grid(want, (int64_t)sm_count() * per_sm);
 }
 
 }  // namespace
@@ -256,9 +254,7 @@ extern "C" tweo_status_t tweo_residual_add_q8(const int8_t* xq, const float* sx,
   const float Q = (float)((1 << (bits - 1)) - 1);
   const int64_t nvec = n >> 4;
   const int64_t want = (nvec + 4 * 256 - 1) / (4 * 256);
-  const int64_t cap = (int64_t)tweo_detail::sm_count() * 8;
-  int grid = (int)(want < cap ? want : cap);
-  if (grid < 1) grid = 1;
+  const int grid = tweo_detail::balanced_grid(want, (int64_t)tweo_detail::sm_count() * 8);
   residual_add_q8_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(xq, fq, yq, n, Q, sx, sf, sy);
   tweo_detail::count_launch();
   return tweo_detail::check_launch("residual_add_q8_kernel");
@@ -348,7 +344,7 @@ cudaError_t launch_row_add(const RowAddArgs& a, cudaStream_t st) {
   if (e != cudaSuccess) return e;
   const int64_t want = (a.rows + 7) / 8;
   const int64_t cap = (int64_t)tweo_detail::sm_count() * (per_sm > 0 ? per_sm : 1);
-  residual_add_q8_rows_kernel<VPL><<<(int)(want < cap ? want : cap), 256, 0, st>>>(a);
+  residual_add_q8_rows_kernel<VPL><<<tweo_detail::balanced_grid(want, cap), 256, 0, st>>>(a);
   return cudaGetLastError();
 }
 

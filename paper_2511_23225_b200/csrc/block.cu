@@ -8,7 +8,8 @@
 // 4 B read + up to 5 B written per element instead of the 13 B of add, penalty and cast as
 // three passes.  HBM-bound streaming kernel: 8 x 16-byte loads in flight per thread (two groups of 16 elements),
 // fp32 per group / fp64 per thread accumulation, per-CTA partial sum and partial maximum to
-// the workspace, the last CTA (ticket) reduces them in a fixed order.
+// the workspace; a one-CTA kernel launched in the same chain reduces them in a fixed order (the
+// streaming CTAs end without fence, ticket or wait: see loss.cu).
 //
 // (2) One tiny kernel keeps the amax history of every tensor (length H, 16 in the paper) and
 // derives next step's scales from the maximum over the window.
@@ -37,7 +38,7 @@ struct BlockArgs {
   float* amax;
   double* part_sum;   // [grid]
   uint32_t* part_max; // [grid]
-  unsigned int* ticket;
+  int parts;          // grid of the streaming kernel
 };
 
 __device__ __forceinline__ double warp_sum(double v) {
@@ -76,6 +77,8 @@ __device__ __forceinline__ uint32_t add_pair(uint32_t xw, uint32_t fw, float k, 
 // QFMT: -1 no FP8 copy, else TWEO_E4M3 / TWEO_E5M2
 template <bool FAST, bool GRAD, int QFMT>
 __global__ void __launch_bounds__(kThreads) block_output_kernel(const BlockArgs args) {
+  chain_release();   // launched in a chain: nothing of the kernel before this one is touched before the wait
+  chain_wait();
   const int64_t n16 = args.n >> 4;
   const uint4* xv = reinterpret_cast<const uint4*>(args.x);
   const uint4* fv = reinterpret_cast<const uint4*>(args.f);
@@ -148,10 +151,9 @@ __global__ void __launch_bounds__(kThreads) block_output_kernel(const BlockArgs 
     }
   }
 
-  // CTA reduction in a fixed order, then the last CTA reduces the partial results
+  // CTA reduction in a fixed order; one partial sum and one partial maximum per CTA
   __shared__ double warp_part[kThreads / 32];
   __shared__ uint32_t warp_maxv[kThreads / 32];
-  __shared__ bool is_last;
   acc = warp_sum(acc);
   uint32_t m = absmax_fold(m2);
 #pragma unroll
@@ -171,22 +173,33 @@ __global__ void __launch_bounds__(kThreads) block_output_kernel(const BlockArgs 
     }
     args.part_sum[blockIdx.x] = s;
     args.part_max[blockIdx.x] = mm;
-    __threadfence();
-    is_last = atomicAdd(args.ticket, 1u) == gridDim.x - 1;
   }
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
+}
+
+// One CTA adds the partial sums (thread-strided with independent loads, then a fixed tree) and takes the maximum.
+__global__ void __launch_bounds__(kThreads) block_output_finish_kernel(const BlockArgs args) {
+  chain_release();
+  chain_wait();   // the streaming kernel has completed: its partial results are visible
+  __shared__ double warp_part[kThreads / 32];
+  __shared__ uint32_t warp_maxv[kThreads / 32];
+  const unsigned int parts = (unsigned int)args.parts;
   double s = 0.0;
   uint32_t mm = 0;
-  for (unsigned int b = threadIdx.x; b < gridDim.x; b += kThreads) {
-    s += __ldcg(&args.part_sum[b]);
-    mm = max(mm, __ldcg(&args.part_max[b]));
+  for (unsigned int b0 = threadIdx.x; b0 < parts; b0 += kThreads * 4) {
+    double v[4];
+    uint32_t w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const unsigned int b = b0 + (unsigned int)(kThreads * j);
+      v[j] = b < parts ? __ldcg(&args.part_sum[b]) : 0.0;
+      w[j] = b < parts ? __ldcg(&args.part_max[b]) : 0u;
+    }
+    s += (v[0] + v[1]) + (v[2] + v[3]);
+    mm = max(max(mm, max(w[0], w[1])), max(w[2], w[3]));
   }
   s = warp_sum(s);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) mm = max(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, o));
-  __syncthreads();
   if ((threadIdx.x & 31) == 0) {
     warp_part[threadIdx.x >> 5] = s;
     warp_maxv[threadIdx.x >> 5] = mm;
@@ -202,22 +215,18 @@ __global__ void __launch_bounds__(kThreads) block_output_kernel(const BlockArgs 
     }
     *args.loss = (float)(tot * args.inv_norm);
     *args.amax = __uint_as_float(mx << 16);
-    *args.ticket = 0u;  // ready for the next call
   }
 }
 
 template <bool FAST, bool GRAD>
 void launch_q(int qfmt, int grid, cudaStream_t st, const BlockArgs& a) {
-  if (qfmt < 0) block_output_kernel<FAST, GRAD, -1><<<grid, kThreads, 0, st>>>(a);
-  else if (qfmt == TWEO_E4M3) block_output_kernel<FAST, GRAD, TWEO_E4M3><<<grid, kThreads, 0, st>>>(a);
-  else block_output_kernel<FAST, GRAD, TWEO_E5M2><<<grid, kThreads, 0, st>>>(a);
+  if (qfmt < 0) launch_chain(block_output_kernel<FAST, GRAD, -1>, dim3(grid), dim3(kThreads), 0, st, 0, a);
+  else if (qfmt == TWEO_E4M3) launch_chain(block_output_kernel<FAST, GRAD, TWEO_E4M3>, dim3(grid), dim3(kThreads), 0, st, 0, a);
+  else launch_chain(block_output_kernel<FAST, GRAD, TWEO_E5M2>, dim3(grid), dim3(kThreads), 0, st, 0, a);
 }
 
 int block_grid(int64_t n) {
-  int64_t want = ((n >> 4) + 2 * kThreads - 1) / (2 * kThreads);
-  const int64_t cap = (int64_t)sm_count() * 8;
-  if (want > cap) want = cap;
-  return (int)(want < 1 ? 1 : want);
+  return balanced_grid(((n >> 4) + 2 * kThreads - 1) / (2 * kThreads), (int64_t)sm_count() * 8);
 }
 
 __global__ void delayed_scaling_kernel(float* history, int H, const float* amax_new, float* scale, float* scale_inv,
@@ -276,7 +285,7 @@ extern "C" tweo_status_t tweo_block_output_fused(const uint16_t* x, const uint16
   args.k_grad = n > 0 ? (float)((double)grad_coeff * (double)p / norm) : 0.0f;
   args.loss = loss;
   args.amax = amax;
-  args.ticket = reinterpret_cast<unsigned int*>(ws);
+  args.parts = grid;
   args.part_sum = reinterpret_cast<double*>(reinterpret_cast<char*>(ws) + 256);
   args.part_max = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + 256 + (size_t)sm_count() * 8 * sizeof(double));
   cudaStream_t st = (cudaStream_t)stream;
@@ -289,7 +298,8 @@ extern "C" tweo_status_t tweo_block_output_fused(const uint16_t* x, const uint16
     if (grad) launch_q<false, true>(qf, grid, st, args);
     else launch_q<false, false>(qf, grid, st, args);
   }
-  count_launch();
+  launch_chain(block_output_finish_kernel, dim3(1), dim3(kThreads), 0, st, 0, args);
+  count_launch(2);
   return check_launch("block_output_kernel");
 }
 

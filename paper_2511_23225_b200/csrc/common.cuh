@@ -22,6 +22,16 @@ tweo_status_t check_launch(const char* what);              // cudaGetLastError a
 tweo_status_t read_and_clear_device_status(cudaStream_t stream);
 unsigned int* device_status_word();  // its device address on the current device (nullptr on failure)
 
+// Grid of a streaming kernel whose CTAs walk `iters` equal pieces of work with a grid-stride loop, at most `cap`
+// CTAs: every CTA gets the same number of pieces (or one less), so no SM waits for a straggler that drew one more
+// sweep than the average -- with iters = 3.5 x cap a capped grid would finish at 4 sweeps, 13 % late.
+inline int balanced_grid(int64_t iters, int64_t cap) {
+  if (cap < 1) cap = 1;
+  if (iters <= cap) return (int)(iters < 1 ? 1 : iters);
+  const int64_t per = (iters + cap - 1) / cap;
+  return (int)((iters + per - 1) / per);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // One-time set-up that CUDA keeps per device (function attributes): `mask` has one bit per device.
@@ -108,6 +118,34 @@ __device__ __forceinline__ uint32_t f32x2_to_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
+}
+
+// Packed binary32 pairs (sm_100: one instruction works on two IEEE lanes, each rounded to nearest-even exactly as
+// the scalar instruction would).  A pair lives in a 64-bit register; packing and unpacking are register moves.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+// the two bf16 values of a packed word as a binary32 pair (exact)
+__device__ __forceinline__ uint64_t bf16x2_to_f32x2(uint32_t w) { return pack_f32x2(bf16lo_to_f32(w), bf16hi_to_f32(w)); }
+__device__ __forceinline__ uint32_t f32x2_pair_to_bf16x2(uint64_t v) {
+  float lo, hi;
+  unpack_f32x2(v, lo, hi);
+  return f32x2_to_bf16x2(lo, hi);
 }
 
 // per-tensor scale from amax: fl32(FP8MAX / amax); 1 for amax == 0 or non-finite;

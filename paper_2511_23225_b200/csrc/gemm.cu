@@ -185,7 +185,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int quarter = warp & 3;  // tensor-memory lanes [32*quarter, 32*quarter+32) belong to this warp
-    const float alpha = __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
+    const float alpha = dequant_alpha(p.sa_inv, p.sb_inv, p.sa_is_scale);
     const float qs = p.out_q ? __ldg(p.q_scale) : 0.0f;
     constexpr int CH = OUT_F32 ? 32 : 64;  // output columns per 128-byte staging row
     const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
@@ -660,8 +660,8 @@ tweo_status_t run_fwd_act(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8
 
 // Forward product for M <= 128 (see gemm_skinny.cuh): W is streamed once, K is sliced over CTAs.
 tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
-                         const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M, int64_t N,
-                         int64_t K, void* ws, size_t ws_bytes, cudaStream_t st) {
+                         const float* sx_inv, const float* sw_inv, bool sx_is_scale, uint16_t* y, int64_t ldy, int64_t M,
+                         int64_t N, int64_t K, void* ws, size_t ws_bytes, cudaStream_t st) {
   if (N > INT32_MAX || K > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
   if (!aligned16(xq) || !aligned16(wq) || (ldx & 15) || (ldw & 15)) return TWEO_ERR_ALIGNMENT;
   SkinnyParams p{};
@@ -681,6 +681,7 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   p.idesc = make_idesc(fmt_w, fmt_x, false, false, p.Mpad, BM);
   p.sx_inv = sx_inv;
   p.sw_inv = sw_inv;
+  p.sx_is_scale = sx_is_scale ? 1 : 0;
   const int sms = sm_count();
   const int slabs = (int)((N + 127) / 128);
   // slices of K per slab = CTAs per cluster: the largest count up to the portable cluster size that keeps the grid
@@ -872,15 +873,16 @@ unsigned int* device_status_word() {
 tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
                              const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
                              int64_t N, int64_t K, const tweo_epilogue_t* epi, void* ws, size_t ws_bytes,
-                             cudaStream_t st) {
+                             cudaStream_t st, bool sx_is_scale) {
   const bool fused = epi && (epi->out_amax || epi->out_q);
   if (M <= 128 && !fused)  // few tokens: stream W once, tokens on the MMA's N side
-    return run_skinny(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, y, ldy, M, N, K, ws, ws_bytes, st);
+    return run_skinny(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, sx_is_scale, y, ldy, M, N, K, ws, ws_bytes, st);
   GemmParams p{};
   p.d = y;
   p.ldd = ldy;
   p.sa_inv = sx_inv;
   p.sb_inv = sw_inv;
+  p.sa_is_scale = sx_is_scale ? 1 : 0;
   tweo_status_t s = fill_epilogue(p, epi);
   if (s != TWEO_OK) return s;
   if (fused && M > 128 && N > 128)  // extra outputs leave through shared memory and TMA
@@ -977,7 +979,7 @@ tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const uint8_t*
   if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
   if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
   return tweo_detail::gemm_fwd_codes(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, y, ldy, M, N, K, epi, ws,
-                                     ws_bytes, (cudaStream_t)stream);
+                                     ws_bytes, (cudaStream_t)stream, false);
 }
 
 tweo_status_t tweo_fp8_linear_fwd_act(const uint8_t* xq, int64_t ldx, const uint8_t* wq, int64_t ldw,

@@ -22,6 +22,7 @@ struct GemmParams {
   int32_t raster_g;    // tiles are numbered in bands of raster_g tile rows (see tile_coords)
   const float* sa_inv;
   const float* sb_inv;
+  int32_t sa_is_scale;  // *sa_inv holds the scale itself, not its reciprocal (static W8A8: the calibrated scale)
   int32_t out_f32;     // 0: bf16 out, 1: fp32 out
   int32_t accumulate;  // fp32 out only
   float* out_amax;
@@ -112,6 +113,13 @@ struct TileWalk {
 };
 
 // ----------------------------------------------------------------- epilogue helpers
+// Dequantisation factor of a product: (1 / scale_a) * (1 / scale_b), each reciprocal rounded once.
+__device__ __forceinline__ float dequant_alpha(const float* sa, const float* sb_inv, int sa_is_scale) {
+  float a = __ldg(sa);
+  if (sa_is_scale) a = __fdiv_rn(1.0f, a);
+  return __fmul_rn(a, __ldg(sb_inv));
+}
+
 template <int FMT>
 __device__ __forceinline__ uint32_t quant4(float a, float b, float c, float d) {
   return cvt_fp8x2<FMT>(a, b) | (cvt_fp8x2<FMT>(c, d) << 16);

@@ -180,7 +180,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     // ------------------------------------------------------------ epilogue (warps 2 .. 1 + EPIW, both CTAs)
     chain_wait();
     const int quarter = warp & 3;
-    const float alpha = I8 ? 1.0f : __fmul_rn(__ldg(p.sa_inv), __ldg(p.sb_inv));
+    const float alpha = I8 ? 1.0f : dequant_alpha(p.sa_inv, p.sb_inv, p.sa_is_scale);
     const float qs = p.out_q ? (Q8 ? __fdiv_rn(p.q8_qmax, __ldg(p.q_scale)) : __ldg(p.q_scale)) : 0.0f;
     constexpr int CH = OUT_F32 ? 32 : 64;
     const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * (uint32_t)EBUF * EPI_BUF;

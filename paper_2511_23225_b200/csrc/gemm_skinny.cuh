@@ -38,6 +38,7 @@ struct SkinnyParams {
   uint32_t idesc;
   const float* sx_inv;
   const float* sw_inv;
+  int32_t sx_is_scale;     // *sx_inv holds the activation scale itself, not its reciprocal
 };
 
 __device__ __forceinline__ float ld_shared_cluster_f32(uint32_t cluster_addr) {
@@ -151,7 +152,7 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
     chain_wait();
     const int quarter = warp & 3;  // tensor-memory lanes [32*quarter, 32*quarter+32) belong to this warp
     const int col = n0 + quarter * 32 + lane;  // output column of this lane (= row of W)
-    const float alpha = __fmul_rn(__ldg(p.sx_inv), __ldg(p.sw_inv));
+    const float alpha = dequant_alpha(p.sx_inv, p.sw_inv, p.sx_is_scale);
     if (mbar_wait(done_bar, 0, abort_flag)) {
       tc_fence_after();
       const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16);
@@ -190,7 +191,7 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
       const int quarter = warp & 3;
       const int col = quarter * 32 + lane;
       const int n = n0 + col;
-      const float alpha = __fmul_rn(__ldg(p.sx_inv), __ldg(p.sw_inv));
+      const float alpha = dequant_alpha(p.sx_inv, p.sw_inv, p.sx_is_scale);
       const uint32_t mine = smem_base + (uint32_t)col * 4u;
       uint32_t peer[8];
 #pragma unroll

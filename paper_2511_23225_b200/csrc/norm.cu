@@ -182,7 +182,7 @@ cudaError_t launch_norm_q(const NormArgs& a, int64_t want_ctas, size_t smem, cud
   cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, norm_rows_kernel<VPL, QFMT>, kNormThreads, smem);
   if (e != cudaSuccess) return e;
   const int64_t cap = (int64_t)tweo_detail::sm_count() * (per_sm > 0 ? per_sm : 1);
-  const int grid = (int)(want_ctas < cap ? want_ctas : cap);
+  const int grid = tweo_detail::balanced_grid(want_ctas, cap);
   norm_rows_kernel<VPL, QFMT><<<grid, kNormThreads, smem, st>>>(a);
   return cudaGetLastError();
 }

@@ -25,9 +25,9 @@ using namespace tweo_detail;
 
 constexpr int kThreads = 256;
 
-__device__ __forceinline__ void cta_amax_to_global(uint32_t m2, float* amax) {
+// m: this thread's maximum as a bf16 bit pattern
+__device__ __forceinline__ void cta_amax_to_global(uint32_t m, float* amax) {
   __shared__ uint32_t part[kThreads / 32];
-  uint32_t m = absmax_fold(m2);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
   if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = m;
@@ -40,13 +40,19 @@ __device__ __forceinline__ void cta_amax_to_global(uint32_t m2, float* amax) {
   }
 }
 
+// The single-tensor kernels are launched in a chain too (see chain_wait() in common.cuh): the launch latency and
+// the few instructions before the wait overlap the tail of the kernel before them.
 __global__ void init_kernel(float* amax, uint32_t* sat_count, const float* scale_in, float* scale_inv) {
+  chain_release();
+  chain_wait();
   *amax = 0.0f;
   if (sat_count) *sat_count = 0u;
   if (scale_in) *scale_inv = __fdiv_rn(1.0f, *scale_in);
 }
 
 __global__ void __launch_bounds__(kThreads) amax_kernel(const uint16_t* x, int64_t n, float* amax) {
+  chain_release();
+  chain_wait();
   const int64_t nvec = n >> 3;
   const uint4* xv = reinterpret_cast<const uint4*>(x);
   const int64_t stride = (int64_t)gridDim.x * kThreads * 4;
@@ -70,34 +76,38 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint16_t* x, int64
     int64_t i = (nvec << 3) + threadIdx.x;
     if (i < n) m = absmax_bits(m, (uint32_t)x[i]);
   }
-  cta_amax_to_global(m, amax);
+  cta_amax_to_global(absmax_fold(m), amax);
 }
 
 // 16 elements: two 16-byte loads -> one 16-byte store.  SAT counts elements whose scaled value
 // exceeds the format's range, AMAX folds |x| into the running maximum m2.  NaN inputs come out of the
 // converter as the code 0x7F (see cvt_fp8x2).
 template <int FMT, bool SAT, bool AMAX>
-__device__ __forceinline__ uint4 cast16(const uint4 a, const uint4 b, float scale, uint32_t& sat, uint32_t& m2) {
+__device__ __forceinline__ uint4 cast16(const uint4 a, const uint4 b, float scale, uint32_t& sat, float& m0, float& m1) {
   const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
   uint32_t c[8];
   const float fmax = FMT == TWEO_E4M3 ? kE4M3Max : kE5M2Max;
+  const uint64_t ss = pack_f32x2(scale, scale);
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    float lo = __fmul_rn(bf16lo_to_f32(w[j]), scale);
-    float hi = __fmul_rn(bf16hi_to_f32(w[j]), scale);
+    float lo, hi;
+    unpack_f32x2(mul_f32x2(bf16x2_to_f32x2(w[j]), ss), lo, hi);   // one packed multiply, each lane rounded once
     if (SAT) sat += (fabsf(lo) > fmax) + (fabsf(hi) > fmax);
     c[j] = cvt_fp8x2<FMT>(lo, hi);
-    if (AMAX) m2 = absmax_bits(m2, w[j]);
+    if (AMAX) absmax_f32(m0, m1, w[j]);
   }
   return make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16));
 }
 
 // CURRENT mode reads *amax (finished by the previous kernel) and derives the scale;
 // GIVEN mode reads *scale and accumulates amax while casting.
-template <int FMT, bool GIVEN, bool SAT>
+// U: pairs of 16-byte loads in flight per thread (the deeper variant for large tensors, as in the batched form).
+template <int FMT, bool GIVEN, bool SAT, int U>
 __global__ void __launch_bounds__(kThreads)
 cast_kernel(const uint16_t* x, int64_t n, float* scale, float* scale_inv, float* amax, uint8_t* q,
             uint32_t* sat_count) {
+  chain_release();
+  chain_wait();
   float s;
   if (GIVEN) {
     s = *scale;
@@ -111,12 +121,13 @@ cast_kernel(const uint16_t* x, int64_t n, float* scale, float* scale_inv, float*
   const int64_t n16 = n >> 4;
   const uint4* xv = reinterpret_cast<const uint4*>(x);
   uint4* qv = reinterpret_cast<uint4*>(q);
-  const int64_t stride = (int64_t)gridDim.x * kThreads * 2;
-  uint32_t sat = 0, m = 0;
-  for (int64_t base = (int64_t)blockIdx.x * kThreads * 2 + threadIdx.x; base < n16; base += stride) {
-    uint4 v[2][2];
+  const int64_t stride = (int64_t)gridDim.x * kThreads * U;
+  uint32_t sat = 0;
+  float m0 = 0.0f, m1 = 0.0f;   // running maximum of |x| (GIVEN mode), two lanes; fmaxf skips NaN
+  for (int64_t base = (int64_t)blockIdx.x * kThreads * U + threadIdx.x; base < n16; base += stride) {
+    uint4 v[U][2];
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < U; ++u) {
       int64_t i = base + (int64_t)u * kThreads;
       if (i < n16) {
         v[u][0] = __ldcs(xv + 2 * i);
@@ -124,9 +135,9 @@ cast_kernel(const uint16_t* x, int64_t n, float* scale, float* scale_inv, float*
       }
     }
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < U; ++u) {
       int64_t i = base + (int64_t)u * kThreads;
-      if (i < n16) __stcs(qv + i, cast16<FMT, SAT, GIVEN>(v[u][0], v[u][1], s, sat, m));
+      if (i < n16) __stcs(qv + i, cast16<FMT, SAT, GIVEN>(v[u][0], v[u][1], s, sat, m0, m1));
     }
   }
   if (blockIdx.x == 0 && threadIdx.x < 16) {  // ragged tail: n % 16 elements
@@ -136,7 +147,7 @@ cast_kernel(const uint16_t* x, int64_t n, float* scale, float* scale_inv, float*
       float v = __fmul_rn(bf16lo_to_f32(w), s);
       sat += fabsf(v) > (FMT == TWEO_E4M3 ? kE4M3Max : kE5M2Max);
       q[i] = (uint8_t)(cvt_fp8x2<FMT>(v, 0.0f) & 0xFFu);
-      if (GIVEN) m = absmax_bits(m, w);
+      if (GIVEN) absmax_f32(m0, m1, w);
     }
   }
   if (SAT) {
@@ -144,7 +155,7 @@ cast_kernel(const uint16_t* x, int64_t n, float* scale, float* scale_inv, float*
     for (int o = 16; o > 0; o >>= 1) sat += __shfl_xor_sync(0xFFFFFFFFu, sat, o);
     if ((threadIdx.x & 31) == 0 && sat) atomicAdd(sat_count, sat);
   }
-  if (GIVEN) cta_amax_to_global(m, amax);
+  if (GIVEN) cta_amax_to_global(absmax_f32_bits(m0, m1), amax);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -247,7 +258,8 @@ __global__ void __launch_bounds__(kThreads) cast_batch_kernel(const __grid_const
     const uint4* xv = reinterpret_cast<const uint4*>(x);
     uint4* qv = reinterpret_cast<uint4*>(q);
     const int64_t stride = (int64_t)gridDim.x * kThreads * U;
-    uint32_t sat = 0, mm = 0;
+    uint32_t sat = 0;
+    float mm0 = 0.0f, mm1 = 0.0f;
     for (int64_t base = (int64_t)blockIdx.x * kThreads * U + threadIdx.x; base < n16; base += stride) {
       uint4 v[U][2];
 #pragma unroll
@@ -261,7 +273,7 @@ __global__ void __launch_bounds__(kThreads) cast_batch_kernel(const __grid_const
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         int64_t i = base + (int64_t)u * kThreads;
-        if (i < n16) __stcs(qv + i, cast16<FMT, false, false>(v[u][0], v[u][1], s, sat, mm));
+        if (i < n16) __stcs(qv + i, cast16<FMT, false, false>(v[u][0], v[u][1], s, sat, mm0, mm1));
       }
     }
     if (blockIdx.x == 0 && threadIdx.x < 16) {  // ragged tail: n % 16 elements
@@ -322,11 +334,7 @@ tweo_status_t launch_batch(const tweo_quant_desc_t* descs, const int* idx, int c
 constexpr size_t kBatchWsBytes = (size_t)TWEO_MAX_QUANT_BATCH * kMaxAmaxGrid * sizeof(uint32_t);  // 64 KB
 
 int grid_for(int64_t work_items, int per_cta, int ctas_per_sm) {
-  int64_t want = (work_items + per_cta - 1) / per_cta;
-  int64_t cap = (int64_t)sm_count() * ctas_per_sm;
-  if (want > cap) want = cap;
-  if (want < 1) want = 1;
-  return (int)want;
+  return balanced_grid((work_items + per_cta - 1) / per_cta, (int64_t)sm_count() * ctas_per_sm);
 }
 
 tweo_status_t check_desc(const tweo_quant_desc_t& d) {
@@ -339,26 +347,37 @@ tweo_status_t check_desc(const tweo_quant_desc_t& d) {
 }
 
 // One tensor as separate kernels: reset, amax (CURRENT only), cast.
+template <int FMT, bool GIVEN, bool SAT>
+cudaError_t launch_cast(const tweo_quant_desc_t& d, cudaStream_t st) {
+  const int64_t n16 = d.n >> 4;
+  const int64_t sweep = (int64_t)sm_count() * 8 * kThreads;
+  if (n16 >= 2 * sweep * 4)
+    return launch_chain(cast_kernel<FMT, GIVEN, SAT, 4>, dim3(grid_for(n16, kThreads * 4, 8)), dim3(kThreads), 0, st, 0,
+                        d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count);
+  return launch_chain(cast_kernel<FMT, GIVEN, SAT, 2>, dim3(grid_for(n16, kThreads * 2, 8)), dim3(kThreads), 0, st, 0, d.x,
+                      d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count);
+}
+
 tweo_status_t launch_single(const tweo_quant_desc_t& d, cudaStream_t st) {
   const bool given = d.mode == TWEO_SCALE_GIVEN;
-  init_kernel<<<1, 1, 0, st>>>(d.amax, d.sat_count, given ? d.scale : nullptr, d.scale_inv);
+  TWEO_CUDA_TRY(launch_chain(init_kernel, dim3(1), dim3(1), 0, st, 0, d.amax, d.sat_count,
+                             given ? (const float*)d.scale : (const float*)nullptr, d.scale_inv));
   count_launch();
   if (!given) {
-    amax_kernel<<<grid_for(d.n >> 3, kThreads * 4, 8), kThreads, 0, st>>>(d.x, d.n, d.amax);
+    TWEO_CUDA_TRY(launch_chain(amax_kernel, dim3(grid_for(d.n >> 3, kThreads * 4, 8)), dim3(kThreads), 0, st, 0, d.x, d.n,
+                               d.amax));
     count_launch();
   }
-  const int grid = grid_for(d.n >> 4, kThreads * 2, 8);
-#define TWEO_CAST(FMT, GIVEN, SAT) \
-  cast_kernel<FMT, GIVEN, SAT><<<grid, kThreads, 0, st>>>(d.x, d.n, d.scale, d.scale_inv, d.amax, d.q, d.sat_count)
   const bool sat = d.sat_count != nullptr;
+  cudaError_t e;
   if (d.fmt == TWEO_E4M3) {
-    if (given) { if (sat) TWEO_CAST(TWEO_E4M3, true, true); else TWEO_CAST(TWEO_E4M3, true, false); }
-    else { if (sat) TWEO_CAST(TWEO_E4M3, false, true); else TWEO_CAST(TWEO_E4M3, false, false); }
+    if (given) e = sat ? launch_cast<TWEO_E4M3, true, true>(d, st) : launch_cast<TWEO_E4M3, true, false>(d, st);
+    else e = sat ? launch_cast<TWEO_E4M3, false, true>(d, st) : launch_cast<TWEO_E4M3, false, false>(d, st);
   } else {
-    if (given) { if (sat) TWEO_CAST(TWEO_E5M2, true, true); else TWEO_CAST(TWEO_E5M2, true, false); }
-    else { if (sat) TWEO_CAST(TWEO_E5M2, false, true); else TWEO_CAST(TWEO_E5M2, false, false); }
+    if (given) e = sat ? launch_cast<TWEO_E5M2, true, true>(d, st) : launch_cast<TWEO_E5M2, true, false>(d, st);
+    else e = sat ? launch_cast<TWEO_E5M2, false, true>(d, st) : launch_cast<TWEO_E5M2, false, false>(d, st);
   }
-#undef TWEO_CAST
+  TWEO_CUDA_TRY(e);
   count_launch();
   return check_launch("tweo_quantize_per_tensor");
 }

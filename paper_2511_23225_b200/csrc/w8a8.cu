@@ -7,12 +7,8 @@ namespace tweo_detail {
 tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
                              const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
                              int64_t N, int64_t K, const tweo_epilogue_t* epi, void* ws, size_t ws_bytes,
-                             cudaStream_t st);
+                             cudaStream_t st, bool sx_is_scale);
 }
-
-namespace {
-__global__ void reciprocal_kernel(const float* s, float* inv) { *inv = __fdiv_rn(1.0f, *s); }
-}  // namespace
 
 extern "C" tweo_status_t tweo_w8a8_static_gemm(const void* x, int32_t x_dtype, int64_t ldx, const float* sx,
                                                const uint8_t* wq, int64_t ldw, const float* sw_inv, uint16_t* y,
@@ -42,14 +38,13 @@ extern "C" tweo_status_t tweo_w8a8_static_gemm(const void* x, int32_t x_dtype, i
     xq = codes;
     ldxq = K;
   } else {
-    reciprocal_kernel<<<1, 1, 0, st>>>(sx, scalars);
-    count_launch();
-    xq = reinterpret_cast<const uint8_t*>(x);
+    xq = reinterpret_cast<const uint8_t*>(x);   // the GEMM's epilogue forms 1 / *sx itself: no extra launch
     ldxq = ldx;
   }
   // what follows the scalars and the codes serves the GEMM's stream-K fix-up
   size_t used = 256;
   if (x_dtype == TWEO_BF16) used += ((size_t)M * (size_t)K + 255) & ~(size_t)255;
-  return gemm_fwd_codes(xq, ldxq, TWEO_E4M3, wq, ldw, TWEO_E4M3, scalars, sw_inv, y, ldy, M, N, K, nullptr,
-                        reinterpret_cast<char*>(ws) + used, ws_bytes - used, st);
+  const bool pre_cast = x_dtype != TWEO_BF16;
+  return gemm_fwd_codes(xq, ldxq, TWEO_E4M3, wq, ldw, TWEO_E4M3, pre_cast ? sx : scalars, sw_inv, y, ldy, M, N, K, nullptr,
+                        reinterpret_cast<char*>(ws) + used, ws_bytes - used, st, pre_cast);
 }

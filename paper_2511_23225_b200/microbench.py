@@ -49,6 +49,36 @@ def make(op, M, K, N):
             tw.fp8_linear_fwd(xq, wq, s, s, y=y, ws=ws)
             tw.fp8_linear_bwd(dyq, xq, wq, s, s, s, fmt_dy=tw.E5M2, dx=dx, dw=dw, ws=ws)
         return fn, 6.0 * M * K * N, "TFLOP/s"
+    if op == "linear_fused":  # forward and data gradient with the fused epilogue (bf16 + amax + FP8 copy), weight gradient
+        xq, wq, dyq = _codes((M, K), 1), _codes((N, K), 2), _codes((M, N), 3)
+        s, qs = _scalar(1e-3), _scalar(4.0)
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+        dw = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
+        yq = torch.empty((M, N), dtype=torch.uint8, device="cuda")
+        dxq = torch.empty((M, K), dtype=torch.uint8, device="cuda")
+        am = torch.zeros(2, dtype=torch.float32, device="cuda")
+        ws = tw.new_workspace(tw.OP_LINEAR_WGRAD)
+
+        def fn():
+            tw.fp8_linear_fwd(xq, wq, s, s, y=y, out_amax=am[0:1], out_q=yq, q_fmt=tw.E4M3, q_scale=qs, ws=ws)
+            tw.fp8_linear_bwd_dgrad(dyq, wq, s, s, dx=dx, out_amax=am[1:2], out_q=dxq, q_fmt=tw.E5M2, q_scale=qs, ws=ws)
+            tw.fp8_linear_bwd_wgrad(xq, dyq, s, s, dw=dw, ws=ws)
+        return fn, 6.0 * M * K * N, "TFLOP/s"
+    if op == "linear_group":  # forward, data gradient and weight gradient in one grouped launch
+        xq, wq, dyq = _codes((M, K), 1), _codes((N, K), 2), _codes((M, N), 3)
+        s = _scalar(1e-3)
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+        dw = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
+        probs = [dict(product=tw.PRODUCT_FWD, xq=xq, wq=wq, sx_inv=s, sw_inv=s, out=y),
+                 dict(product=tw.PRODUCT_DGRAD, dyq=dyq, wq=wq, sdy_inv=s, sw_inv=s, out=dx),
+                 dict(product=tw.PRODUCT_WGRAD, xq=xq, dyq=dyq, sx_inv=s, sdy_inv=s, out=dw)]
+        return (lambda: tw.fp8_linear_group(probs)), 6.0 * M * K * N, "TFLOP/s"
+    if op == "quantize_given":  # one tensor [M, K], given (delayed / static) scale: single pass, amax as by-product
+        x = _bf16((M, K), 1.0, 1)
+        out = tw.quantize_per_tensor(x, tw.E4M3, tw.SCALE_GIVEN, scale=_scalar(64.0))
+        return (lambda: tw.quantize_per_tensor(x, tw.E4M3, tw.SCALE_GIVEN, out=out)), 3.0 * M * K, "GB/s"
     if op == "loss":          # TWEO loss and bf16 gradient of one [M, K] block output
         a = [_bf16((M, K), 1.0, 1)]
         g = [torch.empty_like(a[0])]
@@ -101,7 +131,7 @@ def make(op, M, K, N):
     raise SystemExit(f"unknown --op {op}")
 
 
-OPS = ("quantize", "linear", "loss", "block_output", "layernorm", "fwd_gelu", "fwd_swiglu", "absmax", "int8_linear_q8",
+OPS = ("quantize", "quantize_given", "linear", "linear_fused", "linear_group", "loss", "block_output", "layernorm", "fwd_gelu", "fwd_swiglu", "absmax", "int8_linear_q8",
        "residual_add_q8", "w8a8")
 
 

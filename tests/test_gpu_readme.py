@@ -16,6 +16,16 @@ def test_readme_call_sequences():
     y = tw.fp8_linear_fwd(qx.q, qw.q, qx.scale_inv, qw.scale_inv, ws=ws_g)
     dx, dw = tw.fp8_linear_bwd(qdy.q, qx.q, qw.q, qdy.scale_inv, qx.scale_inv, qw.scale_inv, ws=ws_g)
     assert y.shape == (M, N) and dx.shape == (M, K) and dw.shape == (N, K)
+    amax_y, scale_y = torch.zeros(1, device="cuda"), torch.full((1,), 32.0, device="cuda")
+    yq = torch.empty((M, N), dtype=torch.uint8, device="cuda")
+    y2 = tw.fp8_linear_fwd(qx.q, qw.q, qx.scale_inv, qw.scale_inv, out_amax=amax_y, out_q=yq, q_fmt=tw.E4M3, q_scale=scale_y)
+    y3, dx3, dw3 = torch.empty_like(y), torch.empty_like(dx), torch.empty_like(dw)
+    tw.fp8_linear_group([
+        dict(product=tw.PRODUCT_FWD, xq=qx.q, wq=qw.q, sx_inv=qx.scale_inv, sw_inv=qw.scale_inv, out=y3),
+        dict(product=tw.PRODUCT_DGRAD, dyq=qdy.q, wq=qw.q, sdy_inv=qdy.scale_inv, sw_inv=qw.scale_inv, out=dx3),
+        dict(product=tw.PRODUCT_WGRAD, xq=qx.q, dyq=qdy.q, sx_inv=qx.scale_inv, sdy_inv=qdy.scale_inv, out=dw3)])
+    assert torch.equal(y2, y) and torch.equal(y3, y) and torch.equal(dx3, dx) and torch.equal(dw3, dw)
+    assert float(amax_y.item()) == float(y.abs().max().item())
 
     block_outputs = [torch.randn(M, K, device="cuda").to(torch.bfloat16) for _ in range(3)]
     loss, per_block, grads = tw.loss_fwd_bwd(block_outputs, 3.0, 1e-6, 4.0, 0.01 / len(block_outputs))
