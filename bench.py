@@ -265,11 +265,13 @@ def family_breakdown(torch, tw, bs, side, reps, peaks):
                      "achieved": rate / 1e12 if unit == "TFLOP/s" else rate / 1e9, "unit": unit,
                      "l2_resident": bool(l2_resident), **extra}
 
-    # casts: 2 + 2 read, 1 written per element
+    # casts: current scaling 2 + 2 read, 1 written per element; delayed scaling (one pass) 2 read, 1 written
+    bytes_per_el = 5.0 if bs.variant == "plain" else 3.0
     c0 = tw.launch_count()
     g = _graph_of(torch, side, all_quantize)
     launches = tw.launch_count() - c0
-    record("quantize", _time_replays(torch, g, reps), launches, 5.0 * n_el, "GB/s", 3.0 * n_el < ROTATE_BYTES)
+    record("quantize", _time_replays(torch, g, reps), launches, bytes_per_el * n_el, "GB/s", 3.0 * n_el < ROTATE_BYTES,
+           bytes_per_element=bytes_per_el)
     # GEMMs (+ the fused outputs and the two scale-update launches in the fused variant)
     c0 = tw.launch_count()
     g = _graph_of(torch, side, bs.all_gemms)
@@ -566,6 +568,17 @@ def int8_bench(torch, tw, peaks, reps=10):
                                   "tops": tops, "frac_of_2x_bf16_burst": tops / (2.0 * peaks["bf16"])})
             del xq, wq, y
         del x
+    # few tokens (Sec. 4.4: small-batch inference): the weight-streaming kernel with integer operands, cold weights
+    out["linear_few_tokens"] = []
+    wq8 = torch.randint(-127, 128, (N, K), device="cuda", dtype=torch.int8)
+    one = torch.ones(1, dtype=torch.float32, device="cuda")
+    for M in (1, 16, 128):
+        xq8 = torch.randint(-127, 128, (M, K), device="cuda", dtype=torch.int8)
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        nbytes = float(M * K + K * N + 2 * M * N)
+        us, k = rotating_us(torch, side, lambda i: wq8.clone(), lambda w_: tw.int8_linear(xq8, one, w_, one, 8, y=y), nbytes)
+        out["linear_few_tokens"].append({"M": M, "K": K, "N": N, "us": us, "weight_buffers": k, "l2_resident": False,
+                                         "gbs": nbytes / us / 1e3, "frac_of_hbm_roofline": nbytes / us / 1e3 / peaks["hbm"]})
     torch.cuda.empty_cache()
     return out
 
@@ -804,6 +817,9 @@ def run_cuda(args):
     if args.variant == "fused":
         workload_cfg["epilogue"] = ("forward and data-gradient GEMMs emit bf16 + amax + FP8 copy (Y E4M3, dX E5M2) with "
                                     "delayed scales (history 16); 2 scale-update launches per step")
+    if args.variant != "plain":
+        workload_cfg["scaling"] = ("delayed (Sec. 4.3): X, W, dY cast in one pass each with the scale from their amax "
+                                   "history; the plain variant uses current scaling (amax pass + cast)")
     h2d = bs.h2d_bytes()
     loss_value = r["loss"]
     main_clocks = r["clocks"]

@@ -658,15 +658,13 @@ tweo_status_t run_fwd_act(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8
   }
 }
 
-// Forward product for M <= 128 (see gemm_skinny.cuh): W is streamed once, K is sliced over CTAs.
-tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
-                         const float* sx_inv, const float* sw_inv, bool sx_is_scale, uint16_t* y, int64_t ldy, int64_t M,
-                         int64_t N, int64_t K, void* ws, size_t ws_bytes, cudaStream_t st) {
+// Forward product for M <= 128 (see gemm_skinny.cuh): W is streamed once, K is sliced over CTAs.  The caller has
+// filled the scale fields of `p`; this fills the shape, the ring and the slicing, and launches.
+template <bool I8>
+tweo_status_t launch_skinny(SkinnyParams& p, const void* xq, int64_t ldx, const void* wq, int64_t ldw, int64_t M, int64_t N,
+                            int64_t K, cudaStream_t st) {
   if (N > INT32_MAX || K > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
   if (!aligned16(xq) || !aligned16(wq) || (ldx & 15) || (ldw & 15)) return TWEO_ERR_ALIGNMENT;
-  SkinnyParams p{};
-  p.y = y;
-  p.ldy = ldy;
   p.M = (int32_t)M;
   p.N = (int32_t)N;
   p.Mpad = (int32_t)((M + 15) / 16 * 16);
@@ -678,10 +676,6 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   if (p.stages > kSkinnyMaxStages) p.stages = kSkinnyMaxStages;
   if (p.stages < 2) p.stages = 2;
   p.tmem_cols = p.Mpad <= 32 ? 32u : (p.Mpad <= 64 ? 64u : 128u);
-  p.idesc = make_idesc(fmt_w, fmt_x, false, false, p.Mpad, BM);
-  p.sx_inv = sx_inv;
-  p.sw_inv = sw_inv;
-  p.sx_is_scale = sx_is_scale ? 1 : 0;
   const int sms = sm_count();
   const int slabs = (int)((N + 127) / 128);
   // slices of K per slab = CTAs per cluster: the largest count up to the portable cluster size that keeps the grid
@@ -689,25 +683,36 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   p.slices = 1;
   for (int sl = 2; sl <= 8; ++sl)
     if (slabs * sl <= 2 * sms && p.k_blocks / sl >= 4) p.slices = sl;
-  (void)ws;
-  (void)ws_bytes;
   CUtensorMap mw, mx;
   if (!make_map(&mw, wq, K, N, ldw, BM) || !make_map(&mx, xq, K, M, ldx, p.Mpad)) {
     cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
     return TWEO_ERR_CUDA;
   }
   const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
+  auto kern = gemm_fp8_skinny_kernel<I8>;
   static std::atomic<uint64_t> attr_done{0};  // per device
   int attr_dev = 0;
   if (device_once_pending(attr_done, &attr_dev)) {
-    TWEO_CUDA_TRY(cudaFuncSetAttribute(gemm_fp8_skinny_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)(200 * 1024 + 1024 + 256)));
+    TWEO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(100 * 1024 + 1024 + 256)));
     device_once_done(attr_done, attr_dev);
   }
-  TWEO_CUDA_TRY(launch_chain(gemm_fp8_skinny_kernel, dim3((unsigned)(slabs * p.slices)), dim3(kThreads), smem, st,
-                             (unsigned)p.slices, mw, mx, p));
+  TWEO_CUDA_TRY(launch_chain(kern, dim3((unsigned)(slabs * p.slices)), dim3(kThreads), smem, st, (unsigned)p.slices, mw,
+                             mx, p));
   count_launch();
   return check_launch("gemm_fp8_skinny_kernel");
+}
+
+tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* wq, int64_t ldw, int fmt_w,
+                         const float* sx_inv, const float* sw_inv, bool sx_is_scale, uint16_t* y, int64_t ldy, int64_t M,
+                         int64_t N, int64_t K, cudaStream_t st) {
+  SkinnyParams p{};
+  p.y = y;
+  p.ldy = ldy;
+  p.idesc = make_idesc(fmt_w, fmt_x, false, false, (int)((M + 15) / 16 * 16), BM);
+  p.sx_inv = sx_inv;
+  p.sw_inv = sw_inv;
+  p.sx_is_scale = sx_is_scale ? 1 : 0;
+  return launch_skinny<false>(p, xq, ldx, wq, ldw, M, N, K, st);
 }
 
 // Up to kGroupMaxProblems independent products in ONE launch of the CTA-pair kernel (see gemm_pair_group.cuh).
@@ -876,7 +881,7 @@ tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const ui
                              cudaStream_t st, bool sx_is_scale) {
   const bool fused = epi && (epi->out_amax || epi->out_q);
   if (M <= 128 && !fused)  // few tokens: stream W once, tokens on the MMA's N side
-    return run_skinny(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, sx_is_scale, y, ldy, M, N, K, ws, ws_bytes, st);
+    return run_skinny(xq, ldx, fmt_x, wq, ldw, fmt_w, sx_inv, sw_inv, sx_is_scale, y, ldy, M, N, K, st);
   GemmParams p{};
   p.d = y;
   p.ldd = ldy;
@@ -904,6 +909,22 @@ tweo_status_t run_int8_linear(const int8_t* xq, int64_t ldx, const float* sx, in
   if (y && (!aligned16(y) || (ldy & 7))) return TWEO_ERR_ALIGNMENT;
   if (yq && (!aligned16(yq) || (ldq & 15))) return TWEO_ERR_ALIGNMENT;
   const bool q8 = yq != nullptr;
+  if (!q8 && M <= 128) {
+    // few tokens (small-batch inference, Sec. 4.4): the weight-streaming kernel with integer operands
+    const int Q_ = (1 << (bits - 1)) - 1;
+    const int Mpad = (int)((M + 15) / 16 * 16);
+    SkinnyParams sp{};
+    sp.y = y;
+    sp.ldy = ldy;
+    // kind::i8 descriptor: int32 accumulators, signed 8-bit A and B, K-major, M = 128 (rows of W), N = padded tokens
+    sp.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(Mpad >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    sp.row_scale = sx;
+    sp.col_scale = sw;
+    sp.row_scale_per_row = sx_per_row ? 1 : 0;
+    sp.col_scale_per_col = sw_per_row ? 1 : 0;
+    sp.post_scale = 1.0f / ((float)Q_ * (float)Q_);
+    return launch_skinny<true>(sp, xq, ldx, wq, ldw, M, N, K, stream);
+  }
   constexpr size_t smem6 = (size_t)6 * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
   constexpr size_t smem5q = (size_t)5 * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 4 * 2 * 32 * 64 + 1024 + 256;
   auto kern_bf16 = gemm_fp8_pair_kernel<false, false, 6, false, true>;

@@ -3,8 +3,9 @@
 // the kernel is organised around that: the operands are swapped -- 128 rows of W are the
 // MMA's M dimension, the (padded) tokens its N dimension -- so the accumulator is only
 // 128 x Mpad and nothing but W moves in bulk.  Each CTA takes one 128-row slab of W and one
-// slice of K; slabs x slices is chosen to give every SM one CTA with a deep ring of TMA stages
-// (up to 200 KB of loads in flight per SM).
+// slice of K; slabs x slices is chosen to give every SM one or two CTAs, each with a ring of TMA stages of
+// up to 100 KB (two CTAs fit an SM, so in a launch chain the next kernel's CTAs fetch their first ring of W
+// while this kernel's still reduce and write).
 //
 // CTA = 192 threads: warp 0 issues TMA loads (W slab 128 x 128 B and X 'Mpad' x 128 B per
 // k-block, 128-byte swizzle, rows beyond M zero-filled), warp 1 owns tensor memory and issues
@@ -39,11 +40,16 @@ struct SkinnyParams {
   const float* sx_inv;
   const float* sw_inv;
   int32_t sx_is_scale;     // *sx_inv holds the activation scale itself, not its reciprocal
+  // integer (Eq. 4) operands: y = float(acc) * (row_scale[token or 0] * post_scale) * col_scale[column or 0]
+  const float* row_scale;
+  const float* col_scale;
+  int32_t row_scale_per_row, col_scale_per_col;
+  float post_scale;
 };
 
-__device__ __forceinline__ float ld_shared_cluster_f32(uint32_t cluster_addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
+__device__ __forceinline__ uint32_t ld_shared_cluster_b32(uint32_t cluster_addr) {
+  uint32_t v;
+  asm volatile("ld.shared::cluster.b32 %0, [%1];" : "=r"(v) : "r"(cluster_addr) : "memory");
   return v;
 }
 
@@ -58,6 +64,19 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "memory");
 }
 
+// One output value from an accumulator word: FP8 operands -- the binary32 sum times the dequantisation factor
+// `alpha`; integer operands -- the int32 sum as binary32, times the token's scale (with Q_b^-2 folded in), times
+// the column's scale `alpha` (the order the CTA-pair kernel's integer epilogue uses).
+template <bool I8>
+__device__ __forceinline__ float skinny_out(const SkinnyParams& p, uint32_t acc, int token, float alpha) {
+  if (!I8) return __fmul_rn(__uint_as_float(acc), alpha);
+  const float ar = __fmul_rn(__ldg(p.row_scale + (p.row_scale_per_row ? token : 0)), p.post_scale);
+  return __fmul_rn(__fmul_rn(__int2float_rn((int)acc), ar), alpha);
+}
+
+// I8: signed 8-bit operands (tcgen05 kind::i8, int32 accumulators: partial sums of K slices add exactly) with the
+// Eq. 4 dequantisation in the epilogue, per tensor or per token (activation rows) / per channel (weight rows).
+template <bool I8>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                        const __grid_constant__ SkinnyParams p) {
@@ -139,9 +158,11 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
         const uint32_t sw = smem_base + stage * p.stage_bytes;
         const uint32_t sx = sw + BM * BK;
 #pragma unroll
-        for (int k = 0; k < BK / UMMA_K; ++k)
-          umma_f8(tmem_base, make_smem_desc(sw + k * UMMA_K, BK * 128), make_smem_desc(sx + k * UMMA_K, BK * 128),
-                  p.idesc, (uint32_t)(kb != kb0 || k != 0));
+        for (int k = 0; k < BK / UMMA_K; ++k) {
+          const uint64_t adesc = make_smem_desc(sw + k * UMMA_K, BK * 128), bdesc = make_smem_desc(sx + k * UMMA_K, BK * 128);
+          if (I8) umma_i8(tmem_base, adesc, bdesc, p.idesc, (uint32_t)(kb != kb0 || k != 0));
+          else umma_f8(tmem_base, adesc, bdesc, p.idesc, (uint32_t)(kb != kb0 || k != 0));
+        }
         umma_commit(empty_bar(stage));
         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
       }
@@ -152,7 +173,8 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
     chain_wait();
     const int quarter = warp & 3;  // tensor-memory lanes [32*quarter, 32*quarter+32) belong to this warp
     const int col = n0 + quarter * 32 + lane;  // output column of this lane (= row of W)
-    const float alpha = dequant_alpha(p.sx_inv, p.sw_inv, p.sx_is_scale);
+    const float alpha = I8 ? __ldg(p.col_scale + (p.col_scale_per_col ? min(col, p.N - 1) : 0))
+                           : dequant_alpha(p.sx_inv, p.sw_inv, p.sx_is_scale);
     if (mbar_wait(done_bar, 0, abort_flag)) {
       tc_fence_after();
       const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16);
@@ -165,7 +187,7 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
 #pragma unroll
             for (int j = 0; j < 16; ++j)
               if (c + j < p.M)
-                p.y[(int64_t)(c + j) * p.ldy + col] = (uint16_t)f32_to_bf16_bits(__fmul_rn(__uint_as_float(r[j]), alpha));
+                p.y[(int64_t)(c + j) * p.ldy + col] = (uint16_t)f32_to_bf16_bits(skinny_out<I8>(p, r[j], c + j, alpha));
           }
         }
       } else {
@@ -191,29 +213,40 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
       const int quarter = warp & 3;
       const int col = quarter * 32 + lane;
       const int n = n0 + col;
-      const float alpha = dequant_alpha(p.sx_inv, p.sw_inv, p.sx_is_scale);
+      const float alpha = I8 ? __ldg(p.col_scale + (p.col_scale_per_col ? min(n, p.N - 1) : 0))
+                             : dequant_alpha(p.sx_inv, p.sw_inv, p.sx_is_scale);
       const uint32_t mine = smem_base + (uint32_t)col * 4u;
       uint32_t peer[8];
 #pragma unroll
       for (int sl = 0; sl < 8; ++sl) peer[sl] = map_to_cta(mine, (uint32_t)(sl < p.slices ? sl : 0));
       // eight tokens at a time, so up to 64 remote loads are in flight per thread
       for (int t0 = slice; t0 < p.M; t0 += 8 * p.slices) {
-        float v[8][8];
+        uint32_t v[8][8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
           const int t = t0 + u * p.slices;
 #pragma unroll
           for (int sl = 0; sl < 8; ++sl)
-            v[u][sl] = (sl < p.slices && t < p.M) ? ld_shared_cluster_f32(peer[sl] + (uint32_t)t * 512u) : 0.0f;
+            v[u][sl] = (sl < p.slices && t < p.M) ? ld_shared_cluster_b32(peer[sl] + (uint32_t)t * 512u) : 0u;
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
           const int t = t0 + u * p.slices;
-          float acc = v[u][0];
+          uint32_t acc;
+          if (I8) {
+            int a = (int)v[u][0];
 #pragma unroll
-          for (int sl = 1; sl < 8; ++sl)
-            if (sl < p.slices) acc += v[u][sl];  // slice order
-          if (t < p.M && n < p.N) p.y[(int64_t)t * p.ldy + n] = (uint16_t)f32_to_bf16_bits(__fmul_rn(acc, alpha));
+            for (int sl = 1; sl < 8; ++sl)
+              if (sl < p.slices) a += (int)v[u][sl];   // exact
+            acc = (uint32_t)a;
+          } else {
+            float a = __uint_as_float(v[u][0]);
+#pragma unroll
+            for (int sl = 1; sl < 8; ++sl)
+              if (sl < p.slices) a += __uint_as_float(v[u][sl]);  // slice order
+            acc = __float_as_uint(a);
+          }
+          if (t < p.M && n < p.N) p.y[(int64_t)t * p.ldy + n] = (uint16_t)f32_to_bf16_bits(skinny_out<I8>(p, acc, t, alpha));
         }
       }
     }

@@ -5,16 +5,18 @@ linear of the block, the per-tensor FP8 casts of X, W (E4M3) and dY (E5M2) with
 current scaling, the forward GEMM and the two backward GEMMs, and then the TWEO
 loss and gradient on the block output(s).  Three variants of the GEMM part:
 
-  "fused"    (Sec. 4.3, delayed scaling) the forward and the data-gradient GEMM also
-             emit, from their epilogues, the amax of their bf16 output and its FP8
-             copy (Y in E4M3, dX in the gradient format) with the scale the amax
-             history of the earlier steps gives; one more small launch per format
-             rolls the histories and refreshes the scales for the next step;
-  "plain"    the GEMMs write bf16 only; the linears of a configuration are independent problems here (each has
+  "fused"    (Sec. 4.3, the delayed-scaling recipe the paper trains with) every cast takes the
+             scale its tensor's amax history of the earlier steps gives: X, W and dY are
+             cast in ONE pass each (the pass also reports this step's amax), and the forward
+             and the data-gradient GEMM emit, from their epilogues, the amax of their bf16
+             output and its FP8 copy (Y in E4M3, dX in the gradient format); one small launch
+             per format rolls the histories and refreshes the scales for the next step;
+  "plain"    current scaling (amax pass, then cast) of X, W and dY; the GEMMs write bf16 only; the linears of a configuration are independent problems here (each has
              its own X, W and dY), so the three products of TWO linears share one grouped launch
              (the fused variant's epilogue kernels run one product per launch);
-  "unfused"  "plain" plus separate given-scale casts of Y and dX -- the same outputs
-             as "fused", produced by extra passes over the stored outputs.
+  "unfused"  the same delayed scaling and the same outputs as "fused", but the FP8 copies and
+             the amax of Y and dX come from separate given-scale casts of the stored outputs
+             after plain (grouped) GEMMs.
 
 This module only sequences library calls and owns the device buffers; all
 arithmetic happens in the CUDA kernels behind ``binding``.
@@ -89,14 +91,22 @@ class BlockStep:
         self.side = None
         self.tau, self.eps, self.p, self.lam = 3.0, 1e-6, 4.0, 0.01
         if extra:
-            # delayed-scaling state of the outputs: one slot per linear, Y (E4M3) and dX (gradient format)
+            # Delayed-scaling state, one slot per tensor, grouped by FP8 format so that one launch updates a group:
+            #   E4M3:            X[0..n), W[n..2n), Y[2n..3n)        gradient format: dY[0..n), dX[n..2n)
             nl, f32 = len(self.linears), torch.float32
             z = lambda *s: torch.zeros(s, dtype=f32, device=device)
-            self.amax_y, self.amax_dx = z(nl), z(nl)
-            self.hist_y, self.hist_dx = z(nl, AMAX_HISTORY), z(nl, AMAX_HISTORY)
-            self.scale_y, self.scale_dx = torch.ones(nl, dtype=f32, device=device), torch.ones(nl, dtype=f32, device=device)
-            self.scale_inv_y, self.scale_inv_dx = torch.ones(nl, dtype=f32, device=device), torch.ones(nl, dtype=f32, device=device)
+            one = lambda k: torch.ones(k, dtype=f32, device=device)
+            self.amax_e, self.hist_e, self.scale_e, self.scale_inv_e = z(3 * nl), z(3 * nl, AMAX_HISTORY), one(3 * nl), one(3 * nl)
+            self.amax_g, self.hist_g, self.scale_g, self.scale_inv_g = z(2 * nl), z(2 * nl, AMAX_HISTORY), one(2 * nl), one(2 * nl)
+            self.amax_y, self.scale_y = self.amax_e[2 * nl:], self.scale_e[2 * nl:]
+            self.amax_dx, self.scale_dx = self.amax_g[nl:], self.scale_g[nl:]
+            self.hist_y, self.hist_dx = self.hist_e[2 * nl:], self.hist_g[nl:]
             self._scratch = z(4)
+            for i, lb in enumerate(self.linears):   # the input casts read and write their slots of the state
+                sl = lambda t, j: t[j:j + 1]
+                lb.qx = tw.Quantized(lb.qx.q, sl(self.scale_e, i), sl(self.scale_inv_e, i), sl(self.amax_e, i), None, tw.E4M3)
+                lb.qw = tw.Quantized(lb.qw.q, sl(self.scale_e, nl + i), sl(self.scale_inv_e, nl + i), sl(self.amax_e, nl + i), None, tw.E4M3)
+                lb.qdy = tw.Quantized(lb.qdy.q, sl(self.scale_g, i), sl(self.scale_inv_g, i), sl(self.amax_g, i), None, grad_fmt)
 
     # ---- inputs
     def make_host_inputs(self):
@@ -131,8 +141,13 @@ class BlockStep:
 
     # ---- the step
     def quantize_all(self, lb: LinearBuffers):
-        # X, W (E4M3) and dY (E5M2), each with its own per-tensor scale, in one launch
-        tw.quantize_per_tensor_batch([lb.x, lb.w, lb.dy], [lb.qx, lb.qw, lb.qdy], ws=self.quant_ws)
+        if self.variant == "plain":
+            # current scaling: X, W (E4M3) and dY (E5M2), each with its own per-tensor scale, in one batch
+            tw.quantize_per_tensor_batch([lb.x, lb.w, lb.dy], [lb.qx, lb.qw, lb.qdy], ws=self.quant_ws)
+            return
+        # delayed scaling: one pass per tensor with the scale from the history; the pass reports this step's amax
+        for t, q in ((lb.x, lb.qx), (lb.w, lb.qw), (lb.dy, lb.qdy)):
+            tw.quantize_per_tensor(t, q.fmt, tw.SCALE_GIVEN, out=q)
 
     def gemms(self, lb: LinearBuffers, i: int = 0):
         if self.variant == "fused":
@@ -192,12 +207,12 @@ class BlockStep:
                     self.cast_outputs(self.linears[i], i)
 
     def update_output_scales(self):
-        """Delayed scaling of the outputs (Sec. 4.3): this step's amax values enter the histories and the scales
-        the NEXT step's epilogues use are refreshed; one launch per FP8 format."""
+        """Delayed scaling (Sec. 4.3): this step's amax values enter the histories and the scales the NEXT step's
+        casts and epilogues use are refreshed; one launch per FP8 format."""
         if self.variant == "plain":
             return
-        tw.delayed_scaling_update(self.hist_y, self.amax_y, self.scale_y, self.scale_inv_y, tw.E4M3)
-        tw.delayed_scaling_update(self.hist_dx, self.amax_dx, self.scale_dx, self.scale_inv_dx, self.grad_fmt)
+        tw.delayed_scaling_update(self.hist_e, self.amax_e, self.scale_e, self.scale_inv_e, tw.E4M3)
+        tw.delayed_scaling_update(self.hist_g, self.amax_g, self.scale_g, self.scale_inv_g, self.grad_fmt)
 
     def all_gemms(self):
         for batch in self.gemm_batches():

@@ -68,6 +68,9 @@ def test_absmax_quantize_static_scale_clamps_and_row_pitch(tw, per_row):
 LIN = [
     ("ragged", 300, 400, 272),
     ("one_token", 1, 512, 512),
+    ("sixteen_tokens_ragged", 16, 1040, 528),      # few tokens: the weight-streaming kernel, K sliced over a cluster
+    ("m128_long_k", 128, 4096, 1040),
+    ("m37_cfg5_width", 37, 4096, 11008),
     ("llama_rows", 1024, 4096, 4096),
 ]
 

@@ -106,7 +106,9 @@ def test_full_size_step_replayed_from_a_graph(tw, cfg, linears):
 def test_full_size_fused_step_config4(tw):
     """Config 4 as the benchmark runs it by default: forward and data-gradient GEMMs with the fused epilogue
     (amax + FP8 copy of the output with a delayed scale, Sec. 4.3), replayed from a CUDA graph.  For the checked
-    linears: the bf16 outputs against the oracle's FP64 products on sampled points; the epilogue's amax and codes
+    linears: the one-pass casts of X, W and dY with their delayed scales bit for bit against the oracle (the inputs
+    do not change between steps, so the delayed scale equals the current one); the bf16 outputs against the
+    oracle's FP64 products on sampled points; the epilogue's amax and codes
     bit for bit against the oracle's amax and given-scale cast of the output as stored, with the scale the
     oracle's delayed-scaling rule derives from that amax (the inputs do not change between steps, so the history's
     maximum is this step's amax); and the scale state left for the next step."""
@@ -118,8 +120,8 @@ def test_full_size_fused_step_config4(tw):
     st = torch.cuda.Stream()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.stream(st):
-        bs.step()                                   # first step: scales start at 1, the amax values enter the histories
-        bs.step()
+        for _ in range(18):                         # scales start at 1; after 17 steps the first step's amax values
+            bs.step()                               # (taken from outputs of badly scaled operands) have left the histories
         torch.cuda.synchronize()
         with torch.cuda.graph(graph, stream=st):
             bs.step()
@@ -136,6 +138,10 @@ def test_full_size_fused_step_config4(tw):
         x, w, dy = host["bits"]["lin"][li]
         qx, qw, qd = (orc.quantize_per_tensor_current(x, E4M3), orc.quantize_per_tensor_current(w, E4M3),
                       orc.quantize_per_tensor_current(dy, E5M2))
+        for got, want in zip((lb.qx, lb.qw, lb.qdy), (qx, qw, qd)):
+            assert np.float32(got.amax.item()) == want["amax"] and np.float32(got.scale.item()) == want["scale"]
+            assert np.float32(got.scale_inv.item()) == want["scale_inv"]
+            assert np.array_equal(got.q.cpu().numpy().reshape(want["q"].shape), want["q"])
         M, K = qx["q"].shape
         N = qw["q"].shape[0]
         r, c = points(g, M, N)
