@@ -20,7 +20,10 @@ namespace tweo_detail {
 
 constexpr int kLossThreads = 256;
 constexpr int kLossUnroll = 4;  // 16-byte vectors in flight per thread
-constexpr int kLossCtasPerSm = 6;  // resident CTAs per SM the grid is sized for (42 registers per thread)
+// CTAs per SM the grid is sized for.  Not the most that fit: in a launch chain the CTAs of the NEXT kernel should
+// find room on the SMs while this kernel still runs, so that they sit at their dependency wait when it ends
+// (measured on [16384 x 2048]: 6 per SM 28.0 us, 4 per SM 25.6 us per call; 3 and 5 in between).
+constexpr int kLossCtasPerSm = 4;
 
 int loss_blocks_per_tensor(int64_t n, int L) {
   if (L < 1) L = 1;
