@@ -52,7 +52,9 @@ UNIT = "TFLOP/s"
 FP8_DATASHEET_TFLOPS = 4500.0
 # DRAM traffic of the dominant kernel family (the GEMM launches of a step), per launch, from the ncu captures of
 # single launches summarised under profiles/; reported only while the GEMM sources are the ones profiled.
-GEMM_TRAFFIC = {"sources": "", "workload": "cfg4", "variant": "fused", "bytes_per_launch": None, "from": ""}
+GEMM_TRAFFIC = {"sources": "3e4cb96b90da18d5", "workload": "cfg4", "variant": "fused", "dram_over_algorithmic": 1.05,
+                "from": "profiles/gemm_pair_fused_epilogue_kernels_cfg2_qkv_cfg4_qkv.md (one linear's three launches, "
+                        "scaled by the algorithmic bytes of the family)"}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, FALLBACK_BF16_SUSTAINED = 6650.0, 1590.0, 1400.0
 
 
@@ -787,10 +789,17 @@ def run_cuda(args):
     if dom == "gemm":
         roof["frac_of_fp8_datasheet_4500"] = roof["achieved"] / FP8_DATASHEET_TFLOPS
     roof["traffic"] = None
-    if (dom == "gemm" and GEMM_TRAFFIC["sources"] == gemm_sources_digest() and args.workload == GEMM_TRAFFIC["workload"]
-            and args.variant == GEMM_TRAFFIC["variant"]):
-        roof["traffic"] = GEMM_TRAFFIC["bytes_per_launch"]
-        roof["traffic_from"] = GEMM_TRAFFIC["from"]
+    if dom == "gemm":
+        extra = 1 if args.variant == "fused" else 0        # the FP8 copy of Y and of dX
+        alg = sum(lb.M * lb.lin.K + lb.lin.K * lb.lin.N + (2 + extra) * lb.M * lb.lin.N        # forward
+                  + lb.M * lb.lin.N + lb.lin.K * lb.lin.N + (2 + extra) * lb.M * lb.lin.K      # data gradient
+                  + lb.M * lb.lin.K + lb.M * lb.lin.N + 2 * lb.lin.K * lb.lin.N                # weight gradient
+                  for lb in bs.linears)
+        roof["algorithmic_bytes_per_launch"] = alg / kernels["gemm"]["launches_per_step"]
+        if (GEMM_TRAFFIC["sources"] == gemm_sources_digest() and args.workload == GEMM_TRAFFIC["workload"]
+                and args.variant == GEMM_TRAFFIC["variant"]):
+            roof["traffic"] = GEMM_TRAFFIC["dram_over_algorithmic"] * roof["algorithmic_bytes_per_launch"]
+            roof["traffic_from"] = GEMM_TRAFFIC["from"]
     sustained = None
     if "sustained" in r:
         st, sg = r["sustained"]["step"], r["sustained"]["gemm"]

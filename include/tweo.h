@@ -377,7 +377,7 @@ TWEO_API tweo_status_t tweo_delayed_scaling_update(float* amax_history, int32_t 
  *
  *   Limit: L * (CTAs per tensor) must not exceed 4096 partial sums; beyond that the call
  *     returns TWEO_ERR_WORKSPACE_TOO_SMALL and does nothing (on a 148-SM B200 the kernel
- *     uses at most 888 + L CTAs, so every L <= TWEO_MAX_BLOCKS fits).
+ *     uses at most 592 + L CTAs, so every L <= TWEO_MAX_BLOCKS fits).
  *   The call performs no cudaMalloc / cudaFree and calls no allocating routine.
  *   First call on a device: looks up the array's device address (once per device, with
  *     that device current).  Make that first call outside any stream capture.
