@@ -254,8 +254,8 @@ def family_breakdown(torch, tw, bs, side, reps, peaks):
     and no other family's kernels inside the timed region).  A family whose tensors would fit the L2
     between replays is timed over rotating copies of them."""
     def all_quantize():
-        for lb in bs.linears:
-            bs.quantize_all(lb)
+        for batch in bs.cast_batches():
+            bs.quantize_all([bs.linears[i] for i in batch])
 
     n_el = sum(lb.x.numel() + lb.w.numel() + lb.dy.numel() for lb in bs.linears)
     n_a = sum(t.numel() for t in bs.a)

@@ -286,6 +286,65 @@ __global__ void __launch_bounds__(kThreads) cast_batch_kernel(const __grid_const
   }
 }
 
+// Batched form for GIVEN (delayed / static) scales: one reset kernel for all tensors of the batch, then one
+// single-pass cast kernel per FP8 format present; every CTA folds its share of a tensor into that tensor's amax
+// with one atomicMax.  Three launches for a linear's (or two linears') tensors instead of two per tensor.
+__global__ void init_batch_kernel(const __grid_constant__ QBatch b) {
+  chain_release();
+  chain_wait();
+  const int ti = threadIdx.x;
+  if (ti < b.count) {
+    *b.t[ti].amax = 0.0f;
+    *b.t[ti].scale_inv = __fdiv_rn(1.0f, *b.t[ti].scale);
+  }
+}
+
+template <int FMT, int U>
+__global__ void __launch_bounds__(kThreads) cast_given_batch_kernel(const __grid_constant__ QBatch b) {
+  chain_release();
+  chain_wait();
+#pragma unroll 1
+  for (int ti = 0; ti < b.count; ++ti) {
+    if (b.t[ti].fmt != FMT) continue;
+    const float s = *b.t[ti].scale;
+    const int64_t n = b.t[ti].n;
+    const int64_t n16 = n >> 4;
+    const uint16_t* x = b.t[ti].x;
+    uint8_t* q = b.t[ti].q;
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    uint4* qv = reinterpret_cast<uint4*>(q);
+    const int64_t stride = (int64_t)gridDim.x * kThreads * U;
+    uint32_t sat = 0;
+    float m0 = 0.0f, m1 = 0.0f;
+    for (int64_t base = (int64_t)blockIdx.x * kThreads * U + threadIdx.x; base < n16; base += stride) {
+      uint4 v[U][2];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        int64_t i = base + (int64_t)u * kThreads;
+        if (i < n16) {
+          v[u][0] = __ldcs(xv + 2 * i);
+          v[u][1] = __ldcs(xv + 2 * i + 1);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        int64_t i = base + (int64_t)u * kThreads;
+        if (i < n16) __stcs(qv + i, cast16<FMT, false, true>(v[u][0], v[u][1], s, sat, m0, m1));
+      }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 16) {  // ragged tail: n % 16 elements
+      int64_t i = (n16 << 4) + threadIdx.x;
+      if (i < n) {
+        const uint32_t w = x[i];
+        q[i] = (uint8_t)(cvt_fp8x2<FMT>(__fmul_rn(bf16lo_to_f32(w), s), 0.0f) & 0xFFu);
+        absmax_f32(m0, m1, w);
+      }
+    }
+    __syncthreads();  // the reduction's shared array may still be read from the previous tensor
+    cta_amax_to_global(absmax_f32_bits(m0, m1), b.t[ti].amax);
+  }
+}
+
 int grid_for(int64_t work_items, int per_cta, int ctas_per_sm);
 
 // Launches the batched form for descs[idx[0..count)] (all CURRENT scaling, no saturation count).
@@ -329,6 +388,43 @@ tweo_status_t launch_batch(const tweo_quant_desc_t* descs, const int* idx, int c
     count_launch();
   }
   return check_launch("quantize batch kernels");
+}
+
+// Launches the given-scale batched form for descs[idx[0..count)] (no saturation count).
+tweo_status_t launch_given_batch(const tweo_quant_desc_t* descs, const int* idx, int count, cudaStream_t st) {
+  QBatch b;
+  b.count = count;
+  b.amax_grid = 0;
+  int64_t vec16[2] = {0, 0};
+  for (int i = 0; i < count; ++i) {
+    const tweo_quant_desc_t& d = descs[idx[i]];
+    b.t[i] = QTensor{d.x, d.q, d.n, d.scale, d.scale_inv, d.amax, d.fmt, 0};
+    vec16[d.fmt] += d.n >> 4;
+  }
+  TWEO_CUDA_TRY(launch_chain(init_batch_kernel, dim3(1), dim3(32), 0, st, 0, b));
+  count_launch();
+  const int64_t sweep = (int64_t)sm_count() * 8 * kThreads;
+  bool has[2] = {false, false};
+  for (int i = 0; i < count; ++i) has[b.t[i].fmt] = true;
+  if (has[TWEO_E4M3]) {
+    if (vec16[TWEO_E4M3] >= 2 * sweep * 4)
+      TWEO_CUDA_TRY(launch_chain(cast_given_batch_kernel<TWEO_E4M3, 4>, dim3(grid_for(vec16[TWEO_E4M3], kThreads * 4, 8)),
+                                 dim3(kThreads), 0, st, 0, b));
+    else
+      TWEO_CUDA_TRY(launch_chain(cast_given_batch_kernel<TWEO_E4M3, 2>, dim3(grid_for(vec16[TWEO_E4M3], kThreads * 2, 8)),
+                                 dim3(kThreads), 0, st, 0, b));
+    count_launch();
+  }
+  if (has[TWEO_E5M2]) {
+    if (vec16[TWEO_E5M2] >= 2 * sweep * 4)
+      TWEO_CUDA_TRY(launch_chain(cast_given_batch_kernel<TWEO_E5M2, 4>, dim3(grid_for(vec16[TWEO_E5M2], kThreads * 4, 8)),
+                                 dim3(kThreads), 0, st, 0, b));
+    else
+      TWEO_CUDA_TRY(launch_chain(cast_given_batch_kernel<TWEO_E5M2, 2>, dim3(grid_for(vec16[TWEO_E5M2], kThreads * 2, 8)),
+                                 dim3(kThreads), 0, st, 0, b));
+    count_launch();
+  }
+  return check_launch("quantize given-scale batch kernels");
 }
 
 constexpr size_t kBatchWsBytes = (size_t)TWEO_MAX_QUANT_BATCH * kMaxAmaxGrid * sizeof(uint32_t);  // 64 KB
@@ -383,23 +479,30 @@ tweo_status_t launch_single(const tweo_quant_desc_t& d, cudaStream_t st) {
 }
 
 // Tensors with CURRENT scaling and no saturation count go through the batched kernels when a
-// workspace is there; the others (GIVEN scale: one pass anyway; saturation count: needs a zeroed
-// counter) are launched one by one.
+// workspace is there; two or more GIVEN-scale tensors without saturation count share the given-scale
+// batch kernels; the others are launched one by one.
 tweo_status_t quantize_many(const tweo_quant_desc_t* descs, int count, void* ws, size_t ws_bytes, cudaStream_t st) {
   for (int i = 0; i < count; ++i) {
     tweo_status_t s = check_desc(descs[i]);
     if (s != TWEO_OK) return s;
   }
   const bool have_ws = ws && ws_bytes >= kBatchWsBytes && aligned16(ws);
-  int idx[TWEO_MAX_QUANT_BATCH];
-  int nb = 0;
+  int idx[TWEO_MAX_QUANT_BATCH], idxg[TWEO_MAX_QUANT_BATCH];
+  int nb = 0, ng = 0;
   for (int i = 0; i < count; ++i) {
-    if (have_ws && descs[i].mode == TWEO_SCALE_CURRENT && !descs[i].sat_count) {
-      idx[nb++] = i;
-    } else {
+    if (have_ws && descs[i].mode == TWEO_SCALE_CURRENT && !descs[i].sat_count) idx[nb++] = i;
+    else if (count > 1 && descs[i].mode == TWEO_SCALE_GIVEN && !descs[i].sat_count) idxg[ng++] = i;
+    else {
       tweo_status_t s = launch_single(descs[i], st);
       if (s != TWEO_OK) return s;
     }
+  }
+  if (ng == 1) {   // a lone given-scale tensor gains nothing from the batched form
+    tweo_status_t s = launch_single(descs[idxg[0]], st);
+    if (s != TWEO_OK) return s;
+  } else if (ng > 1) {
+    tweo_status_t s = launch_given_batch(descs, idxg, ng, st);
+    if (s != TWEO_OK) return s;
   }
   if (nb > 0) return launch_batch(descs, idx, nb, ws, st);
   return TWEO_OK;

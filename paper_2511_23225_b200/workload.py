@@ -101,7 +101,7 @@ class BlockStep:
             self.amax_y, self.scale_y = self.amax_e[2 * nl:], self.scale_e[2 * nl:]
             self.amax_dx, self.scale_dx = self.amax_g[nl:], self.scale_g[nl:]
             self.hist_y, self.hist_dx = self.hist_e[2 * nl:], self.hist_g[nl:]
-            self._scratch = z(4)
+            self._scratch = z(8)
             for i, lb in enumerate(self.linears):   # the input casts read and write their slots of the state
                 sl = lambda t, j: t[j:j + 1]
                 lb.qx = tw.Quantized(lb.qx.q, sl(self.scale_e, i), sl(self.scale_inv_e, i), sl(self.amax_e, i), None, tw.E4M3)
@@ -140,14 +140,22 @@ class BlockStep:
             dst.copy_(src, non_blocking=non_blocking)
 
     # ---- the step
-    def quantize_all(self, lb: LinearBuffers):
-        if self.variant == "plain":
-            # current scaling: X, W (E4M3) and dY (E5M2), each with its own per-tensor scale, in one batch
-            tw.quantize_per_tensor_batch([lb.x, lb.w, lb.dy], [lb.qx, lb.qw, lb.qdy], ws=self.quant_ws)
-            return
-        # delayed scaling: one pass per tensor with the scale from the history; the pass reports this step's amax
-        for t, q in ((lb.x, lb.qx), (lb.w, lb.qw), (lb.dy, lb.qdy)):
-            tw.quantize_per_tensor(t, q.fmt, tw.SCALE_GIVEN, out=q)
+    def quantize_all(self, lbs):
+        """Casts X, W (E4M3) and dY (E5M2) of the given linears (at most two: the batch call takes eight tensors),
+        each tensor with its own per-tensor scale, in one batch call: current scaling in the plain variant; in the
+        others delayed scaling, one pass per tensor with the scale from the history, the pass reporting this step's
+        amax."""
+        if isinstance(lbs, LinearBuffers):
+            lbs = [lbs]
+        xs = [t for lb in lbs for t in (lb.x, lb.w, lb.dy)]
+        qs = [q for lb in lbs for q in (lb.qx, lb.qw, lb.qdy)]
+        modes = None if self.variant == "plain" else [tw.SCALE_GIVEN] * len(xs)
+        tw.quantize_per_tensor_batch(xs, qs, modes, ws=self.quant_ws)
+
+    def cast_batches(self):
+        """The linears in cast order: the first alone (the first GEMM waits for it), then two per batch call."""
+        idx = list(range(len(self.linears)))
+        return [idx[:1]] + [idx[i:i + 2] for i in range(1, len(idx), 2)]
 
     def gemms(self, lb: LinearBuffers, i: int = 0):
         if self.variant == "fused":
@@ -164,16 +172,20 @@ class BlockStep:
         tw.fp8_linear_bwd(lb.qdy.q, lb.qx.q, lb.qw.q, lb.qdy.scale_inv, lb.qx.scale_inv, lb.qw.scale_inv,
                           fmt_dy=self.grad_fmt, dx=lb.dx, dw=lb.dw, ws=self.gemm_ws)
         if self.variant == "unfused":
-            self.cast_outputs(lb, i)
+            self.cast_outputs([i])
 
-    def cast_outputs(self, lb: LinearBuffers, i: int):
-        """The extra outputs of the fused variant by separate passes: given-scale casts of the stored Y and dX."""
+    def cast_outputs(self, batch):
+        """The extra outputs of the fused variant by separate passes: given-scale casts of the stored Y and dX of the
+        linears in `batch`, one batch call."""
         s = self._scratch
-        tw.quantize_per_tensor(lb.y, tw.E4M3, tw.SCALE_GIVEN,
-                               out=tw.Quantized(lb.yq, self.scale_y[i:i + 1], s[0:1], self.amax_y[i:i + 1], None, tw.E4M3))
-        tw.quantize_per_tensor(lb.dx, self.grad_fmt, tw.SCALE_GIVEN,
-                               out=tw.Quantized(lb.dxq, self.scale_dx[i:i + 1], s[1:2], self.amax_dx[i:i + 1], None,
-                                                self.grad_fmt))
+        xs, qs = [], []
+        for k, i in enumerate(batch):
+            lb = self.linears[i]
+            xs += [lb.y, lb.dx]
+            qs += [tw.Quantized(lb.yq, self.scale_y[i:i + 1], s[2 * k:2 * k + 1], self.amax_y[i:i + 1], None, tw.E4M3),
+                   tw.Quantized(lb.dxq, self.scale_dx[i:i + 1], s[2 * k + 1:2 * k + 2], self.amax_dx[i:i + 1], None,
+                                self.grad_fmt)]
+        tw.quantize_per_tensor_batch(xs, qs, [tw.SCALE_GIVEN] * len(xs), ws=self.quant_ws)
 
     def group_ok(self, lb: LinearBuffers) -> bool:
         """Whether all three products of this linear can go into a grouped launch (outputs wider and taller than 128)."""
@@ -203,8 +215,7 @@ class BlockStep:
         else:
             self.gemms_grouped([self.linears[i] for i in batch])
             if self.variant == "unfused":
-                for i in batch:
-                    self.cast_outputs(self.linears[i], i)
+                self.cast_outputs(batch)
 
     def update_output_scales(self):
         """Delayed scaling (Sec. 4.3): this step's amax values enter the histories and the scales the NEXT step's
@@ -230,11 +241,9 @@ class BlockStep:
         linear i+1 and the TWEO pass: the casts are HBM-bound, the GEMMs tensor-bound, and they share the SMs.
         Fork / join on the calling stream, so the step can be captured into one CUDA graph."""
         if not self.overlap:
-            for batch in self.gemm_batches():
-                for i in batch:
-                    self.quantize_all(self.linears[i])
-                self.run_gemm_batch(batch)
-            self.update_output_scales()
+            for batch in self.cast_batches():
+                self.quantize_all([self.linears[i] for i in batch])
+            self.all_gemms()
             self.tweo()
             return
         main = torch.cuda.current_stream()
@@ -242,16 +251,17 @@ class BlockStep:
             self.side = torch.cuda.Stream()
         side = self.side
         side.wait_stream(main)
-        ready = []
+        ready = {}
         with torch.cuda.stream(side):
-            for lb in self.linears:
-                self.quantize_all(lb)
+            for batch in self.cast_batches():
+                self.quantize_all([self.linears[i] for i in batch])
                 ev = torch.cuda.Event()
                 ev.record(side)
-                ready.append(ev)
+                ready[batch[-1]] = ev
             self.tweo()
         for batch in self.gemm_batches():
-            main.wait_event(ready[batch[-1]])       # the casts of the batch's last linear: the earlier ones are done too
+            # the cast batch that holds this GEMM batch's last linear: the earlier ones are done too
+            main.wait_event(ready[min(k for k in ready if k >= batch[-1])])
             self.run_gemm_batch(batch)
         self.update_output_scales()
         main.wait_stream(side)

@@ -148,6 +148,45 @@ def test_quantize_batch_matches_oracle_per_tensor(tw):
             assert int(o.sat_count.item()) == ref["sat_count"]
 
 
+def test_quantize_batch_given_scales_share_one_pass_per_format(tw):
+    """Delayed / static scaling for a whole batch (no saturation count): the tensors of one FP8 format go through one
+    single-pass kernel; codes, amax and the reciprocal scale of every tensor equal its own per-tensor result, with a
+    current-scaling tensor in the same call, twice in a row (the amax words are reset by the call)."""
+    x, w, dy = synth.linear_inputs(2, 1, M=1536)
+    a = synth.normal_with_extreme_outliers_bf16(16, (333, 77))     # ragged size, saturates under its scale
+    n = synth.normal_bf16(17, (4099,), 1.0)
+    n[5], n[4098] = 0x7FC0, 0xFF80                                  # a NaN and -inf (the latter in the ragged tail)
+    e = np.zeros((0,), dtype=np.uint16)
+    bits = [x, w, dy, a, n, e, w]
+    fmts = [E4M3, E4M3, E5M2, E5M2, E4M3, E4M3, E5M2]
+    G, C = tw.SCALE_GIVEN, tw.SCALE_CURRENT
+    modes = [G, G, G, G, G, G, C]
+    scales = [np.float32(v) for v in (0.37, 211.0, 1900.5, 57344.0 / 6.0, 100.0, 1.0, 0.0)]
+    ws = tw.new_workspace(tw.OP_QUANTIZE)
+    xs = [to_gpu_bf16(b) for b in bits]
+    outs = []
+    for b, f, s in zip(xs, fmts, scales):
+        sc = torch.tensor([float(s), 0.0, 123.0, 0.0], dtype=torch.float32, device="cuda")   # a stale amax of 123
+        outs.append(tw.Quantized(torch.empty(b.shape, dtype=torch.uint8, device="cuda"), sc[0:1], sc[1:2], sc[2:3], None, f))
+    c0 = tw.launch_count()
+    for rep in range(2):
+        tw.quantize_per_tensor_batch(xs, outs, modes, ws=ws)
+        torch.cuda.synchronize()
+        for b, f, m, s, o in zip(bits, fmts, modes, scales, outs):
+            if m == G:
+                q_ref, _ = orc.quantize_bf16(b, f, s)
+                assert np.array_equal(o.q.cpu().numpy(), q_ref)
+                assert f32_bits(o.amax) == np_f32_bits(orc.amax_bf16(b))
+                assert f32_bits(o.scale) == np_f32_bits(s)
+                assert f32_bits(o.scale_inv) == np_f32_bits(np.float32(1.0) / s)
+            else:
+                ref = orc.quantize_per_tensor_current(b, f)
+                assert np.array_equal(o.q.cpu().numpy(), ref["q"])
+                assert f32_bits(o.amax) == np_f32_bits(ref["amax"]) and f32_bits(o.scale) == np_f32_bits(ref["scale"])
+    # per call: reset + one cast per format for the six given-scale tensors, amax + one cast for the current one
+    assert tw.launch_count() - c0 == 2 * (3 + 2)
+
+
 def test_quantize_all_bf16_patterns_both_formats(tw):
     """Every finite bf16 value through the GPU cast equals the oracle's code (scale 1 and an odd scale)."""
     bits = np.arange(1 << 16, dtype=np.uint16)
