@@ -15,7 +15,9 @@
  *   - the block output A = x + f(x) the regulariser acts on (paper Sec. 3.3) and the
  *     delayed-scaling state (paper Sec. 4.3: amax history of length 16),
  *   - LayerNorm / RMSNorm (paper Sec. 4.3 runs the LayerNorm components under FP8 too) and
- *     the MLP activations of the paper's models (Sec. 3.2: GELU, GLU variants).
+ *     the MLP activations of the paper's models (Sec. 3.2: GELU, GLU variants),
+ *   - the FP4 step the paper's conclusion looks ahead to: the 4-bit E2M1 element with the same
+ *     per-tensor scaling as the FP8 path.
  *
  * Floating point is FP64 unless the step is *defined* in FP32 (the scale, the
  * scaled value that gets rounded to FP8).  There is no blocking, no SIMD, no
@@ -39,6 +41,7 @@
 
 #define ORACLE_E4M3 0
 #define ORACLE_E5M2 1
+#define ORACLE_E2M1 2 /* 4-bit codes, one per byte (low nibble), where a GEMM routine takes a format */
 
 /* ------------------------------------------------------------------ bf16 */
 
@@ -213,8 +216,10 @@ void oracle_quantize_bf16(const uint16_t* x, int64_t n, int fmt, float scale,
  * Products of two FP8 values are small dyadic rationals, so for the
  * contraction lengths used here the FP64 sums are exact. */
 
+double oracle_fp4_decode(uint8_t code);
 static void fill_table(double* t, int fmt) {
-  for (int c = 0; c < 256; ++c) t[c] = oracle_fp8_decode((uint8_t)c, fmt);
+  for (int c = 0; c < 256; ++c)
+    t[c] = fmt == ORACLE_E2M1 ? oracle_fp4_decode((uint8_t)(c & 0x0F)) : oracle_fp8_decode((uint8_t)c, fmt);
 }
 
 /* forward: Y[i,j] = (sum_k X[i,k] W[j,k]) * sx_inv * sw_inv */
@@ -594,4 +599,69 @@ void oracle_residual_add_q8_rows(const int8_t* xq, const float* sx, const int8_t
       yq[m * cols + j] = (t != t) ? 0 : (int8_t)r;
     }
   }
+}
+
+/* ------------------------------------------------------------------ FP4 (E2M1) */
+/* The paper's conclusion names FP4 training and inference as the step after FP8 and fixes no
+ * format.  Reading taken here: the 4-bit floating-point element of the OCP Microscaling formats
+ * (E2M1: 1 sign bit, 2 exponent bits with bias 1, 1 mantissa bit; no infinities, no NaN), with ONE
+ * scale per tensor exactly as in the FP8 path of Sec. 4.3 (scale = largest finite value / amax).
+ *   code = s e e m;   e = 0: (-1)^s * m * 2^-1 ;   e > 0: (-1)^s * (1 + m / 2) * 2^(e - 1)
+ * so the magnitudes are 0, 0.5, 1, 1.5, 2, 3, 4, 6. */
+double oracle_fp4_decode(uint8_t code) {
+  const int s = (code >> 3) & 1, e = (code >> 1) & 3, m = code & 1;
+  const double mag = e == 0 ? 0.5 * (double)m : ldexp(1.0 + 0.5 * (double)m, e - 1);
+  return s ? -mag : mag;
+}
+
+double oracle_fp4_max(void) { return 6.0; }
+
+/* Saturating round-to-nearest-even, by search over the eight magnitudes (the definition written
+ * out): the closest value wins, an exact tie goes to the code whose last bit is 0.  |v| >= 6
+ * (infinity included) -> sign | 0x7.  The format has no NaN code: a NaN becomes +6 (code 0x7), the
+ * "NaN saturates to the largest positive value" convention of conversions into NaN-less formats.
+ * Zero and values that round to zero keep their sign. */
+uint8_t oracle_fp4_encode(float v) {
+  if (isnan(v)) return 0x7;
+  const uint8_t sign = signbit(v) ? 0x8 : 0x0;
+  const double a = fabs((double)v);
+  if (a >= 6.0) return (uint8_t)(sign | 0x7);
+  int best = 0;
+  double best_d = INFINITY;
+  for (int c = 0; c <= 7; ++c) {
+    const double d = fabs(oracle_fp4_decode((uint8_t)c) - a); /* exact in FP64 */
+    if (d < best_d || (d == best_d && (c & 1) == 0)) { best_d = d; best = c; }
+  }
+  return (uint8_t)(sign | best);
+}
+
+void oracle_fp4_encode_array(const float* v, int64_t n, uint8_t* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = oracle_fp4_encode(v[i]);
+}
+
+/* scale = fl32(6 / amax), scale_inv = fl32(1 / scale); the degenerate cases as in
+ * oracle_scale_from_amax. */
+void oracle_fp4_scale_from_amax(float amax, float* scale, float* scale_inv) {
+  float s = 1.0f;
+  if (amax > 0.0f && isfinite(amax)) {
+    volatile float q = 6.0f / amax;
+    s = q;
+    if (isinf(s)) s = FLT_MAX;
+  }
+  volatile float inv = 1.0f / s;
+  *scale = s;
+  *scale_inv = inv;
+}
+
+/* code_i = encode( fl32( x_i * scale ) ): one binary32 multiply, one saturating RNE onto the
+ * E2M1 grid.  codes: one code per byte.  packed (optional): two codes per byte, element 2i in the
+ * low nibble and element 2i + 1 in the high nibble; an odd n leaves the last high nibble 0. */
+void oracle_fp4_quantize_bf16(const uint16_t* x, int64_t n, float scale, uint8_t* codes, uint8_t* packed) {
+  for (int64_t i = 0; i < n; ++i) {
+    volatile float v = bf16_bits_to_f32(x[i]) * scale;
+    codes[i] = oracle_fp4_encode(v);
+  }
+  if (packed)
+    for (int64_t i = 0; i < (n + 1) / 2; ++i)
+      packed[i] = (uint8_t)(codes[2 * i] | ((2 * i + 1 < n ? codes[2 * i + 1] : 0) << 4));
 }

@@ -17,6 +17,7 @@ import numpy as np
 
 E4M3 = 0
 E5M2 = 1
+E2M1 = 2   # 4-bit codes, one per byte, where a GEMM routine takes a format
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "tweo_oracle.c")
@@ -115,6 +116,17 @@ def lib():
             L.oracle_residual_add_q8_rows.restype = None
             L.oracle_residual_add_q8_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                                       C.c_int, C.c_float, C.c_void_p, C.c_void_p]
+            L.oracle_fp4_decode.restype = C.c_double
+            L.oracle_fp4_decode.argtypes = [C.c_uint8]
+            L.oracle_fp4_max.restype = C.c_double
+            L.oracle_fp4_encode.restype = C.c_uint8
+            L.oracle_fp4_encode.argtypes = [C.c_float]
+            L.oracle_fp4_encode_array.restype = None
+            L.oracle_fp4_encode_array.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+            L.oracle_fp4_scale_from_amax.restype = None
+            L.oracle_fp4_scale_from_amax.argtypes = [C.c_float, C.POINTER(C.c_float), C.POINTER(C.c_float)]
+            L.oracle_fp4_quantize_bf16.restype = None
+            L.oracle_fp4_quantize_bf16.argtypes = [C.c_void_p, C.c_int64, C.c_float, C.c_void_p, C.c_void_p]
             _lib = L
     return _lib
 
@@ -462,3 +474,45 @@ def residual_add_q8_rows(xq, sx, fq, sf, bits: int, eps):
     lib().oracle_residual_add_q8_rows(xq.ctypes.data, sx.ctypes.data, fq.ctypes.data, sf.ctypes.data, xq.shape[0],
                                       xq.shape[1], bits, float(np.float32(eps)), yq.ctypes.data, sy.ctypes.data)
     return yq, sy
+
+
+# ---------------------------------------------------------------- FP4 (E2M1), per-tensor scale
+def fp4_decode(code: int) -> float:
+    return float(lib().oracle_fp4_decode(int(code)))
+
+
+def fp4_max() -> float:
+    return float(lib().oracle_fp4_max())
+
+
+def fp4_encode(v) -> int:
+    return int(lib().oracle_fp4_encode(np.float32(v)))
+
+
+def fp4_encode_array(v) -> np.ndarray:
+    v = np.ascontiguousarray(v, dtype=np.float32)
+    out = np.empty(v.shape, dtype=np.uint8)
+    lib().oracle_fp4_encode_array(v.ctypes.data, v.size, out.ctypes.data)
+    return out
+
+
+def fp4_scale_from_amax(amax):
+    s, si = C.c_float(), C.c_float()
+    lib().oracle_fp4_scale_from_amax(np.float32(amax), C.byref(s), C.byref(si))
+    return np.float32(s.value), np.float32(si.value)
+
+
+def fp4_quantize_bf16(x_bits, scale):
+    """Returns (codes uint8 with x's shape, one E2M1 code per byte; packed uint8 [(n + 1) // 2], two per byte)."""
+    x = _u16(x_bits)
+    codes = np.empty(x.shape, dtype=np.uint8)
+    packed = np.empty(((x.size + 1) // 2,), dtype=np.uint8)
+    lib().oracle_fp4_quantize_bf16(x.ctypes.data, x.size, np.float32(scale), codes.ctypes.data, packed.ctypes.data)
+    return codes, packed
+
+
+def fp4_quantize_per_tensor_current(x_bits):
+    amax = amax_bf16(x_bits)
+    scale, scale_inv = fp4_scale_from_amax(amax)
+    codes, packed = fp4_quantize_bf16(x_bits, scale)
+    return {"amax": amax, "scale": scale, "scale_inv": scale_inv, "codes": codes, "packed": packed}
