@@ -523,6 +523,57 @@ def streaming_bench(torch, tw, peaks):
     return rows
 
 
+def fp4_bench(torch, tw, peaks, reps=10):
+    """FP4 (E2M1, per-tensor scale): the cast (2 B read; 0.5 B packed codes + 1 B E4M3 carriers written per element;
+    current scaling reads the tensor twice) and the unpack of packed weights over rotating buffers, and the static
+    W4A4 linear (bf16 activations cast inside the call) at the config-5 shapes."""
+    side = torch.cuda.Stream()
+    out = {"cast": [], "w4a4_static_gemm": []}
+    sc = torch.full((1,), 2.0, dtype=torch.float32, device="cuda")
+    for name, n in (("cfg4 X [16384x2048]", 16384 * 2048), ("cfg5 W [11008x4096]", 11008 * 4096)):
+        def make_set(i):
+            x = torch.randn(n, device="cuda").to(torch.bfloat16)
+            return x, tw.fp4_quantize(x)
+        us, k = rotating_us(torch, side, make_set, lambda st: tw.fp4_quantize(st[0], out=st[1]), 3.5 * n)
+        out["cast"].append(_hbm_row(peaks, us, 5.5 * n, op="quantize_current packed+carriers", tensor=name, buffer_sets=k))
+
+        def make_given(i):
+            x = torch.randn(n, device="cuda").to(torch.bfloat16)
+            return x, tw.fp4_quantize(x, tw.SCALE_GIVEN, scale=sc, packed=False)
+        us, k = rotating_us(torch, side, make_given, lambda st: tw.fp4_quantize(st[0], tw.SCALE_GIVEN, out=st[1]), 3.0 * n)
+        out["cast"].append(_hbm_row(peaks, us, 3.0 * n, op="quantize_given carriers", tensor=name, buffer_sets=k))
+
+        def make_packed(i):
+            q4 = torch.randint(0, 256, (n // 2,), dtype=torch.uint8, device="cuda")
+            return q4, torch.empty(n, dtype=torch.uint8, device="cuda")
+        us, k = rotating_us(torch, side, make_packed, lambda st: tw.fp4_unpack(st[0], (n,), q8=st[1]), 1.5 * n)
+        out["cast"].append(_hbm_row(peaks, us, 1.5 * n, op="unpack", tensor=name, buffer_sets=k))
+        torch.cuda.empty_cache()
+    for K, N in ((4096, 4096), (4096, 11008)):
+        w = (0.02 * torch.randn((N, K), device="cuda")).to(torch.bfloat16)
+        wq = tw.fp4_quantize(w, packed=False)
+        del w
+        for M in (16, 1024, 8192):
+            x = torch.randn((M, K), device="cuda").to(torch.bfloat16)
+            y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            ws = tw.new_workspace(tw.OP_W8A8, M, N, K)
+            fn = lambda: [tw.w4a4_static_gemm(x, sc, wq.q8, wq.scale_inv, y=y, ws=ws) for _ in range(reps)]
+            fn()
+            torch.cuda.synchronize()
+            us = 1e3 * _time_replays(torch, _graph_of(torch, side, fn), 5) / reps
+            flops = 2.0 * M * K * N
+            nbytes = float(3 * M * K + M * K + K * N + 2 * M * N)   # the cast's 2 + 1, then the GEMM's operands and output
+            hbm_us, tc_us = nbytes / peaks["hbm"] / 1e3, flops / (2.0 * peaks["bf16"]) / 1e6
+            out["w4a4_static_gemm"].append({"M": M, "K": K, "N": N, "us": us, "tflops": flops / us / 1e6,
+                                            "bound": "hbm" if hbm_us > tc_us else "tensor", "includes": "activation cast",
+                                            "l2_resident": nbytes < L2_BYTES,
+                                            "frac_of_roofline": max(hbm_us, tc_us) / us})
+            del x, y, ws
+        del wq
+        torch.cuda.empty_cache()
+    return out
+
+
 def block_output_bench(torch, tw, peaks):
     """The fused block-output pass (x + f -> a, TWEO loss and gradient, amax, E4M3 copy with a given
     scale) at the block-output sizes of configs 2 and 4: 4 B read + 5 B written per element."""
@@ -902,7 +953,7 @@ def run_cuda(args):
                 fractions[name]["fused_gemm_frac_of_2x_bf16_burst"] = entry["fused"]["gemm_frac_of_2x_bf16_burst"]
             del ohost
 
-    w8a8, stream_rows, block_rows, int8_rows, act_rows, res8_rows, vendor_rows = (None,) * 7
+    w8a8, stream_rows, block_rows, int8_rows, act_rows, res8_rows, vendor_rows, fp4_rows = (None,) * 8
     if world == 1 and not args.no_w8a8:
         w8a8 = w8a8_sweep(torch, tw, peaks)
         stream_rows = streaming_bench(torch, tw, peaks)
@@ -910,6 +961,7 @@ def run_cuda(args):
         int8_rows = int8_bench(torch, tw, peaks)
         act_rows = act_norm_bench(torch, tw, peaks)
         res8_rows = residual8_bench(torch, tw, peaks)
+        fp4_rows = fp4_bench(torch, tw, peaks)
         vendor_rows = vendor_fp8_context(torch, tw)
         if tw.read_device_status() != 0:
             raise SystemExit("device status reports an expired wait")
@@ -959,6 +1011,8 @@ def run_cuda(args):
             line["act_norm_path"] = act_rows
         if res8_rows:
             line["residual_stream_8bit"] = res8_rows
+        if fp4_rows:
+            line["fp4_e2m1_per_tensor"] = fp4_rows
         if vendor_rows:
             line["context_vendor_fp8_gemm"] = vendor_rows
         if world == 1 and not args.no_cpu_baseline:

@@ -409,6 +409,50 @@ TWEO_API tweo_status_t tweo_w8a8_static_gemm(const void* x, int32_t x_dtype, int
                                     size_t ws_bytes, void* stream);
 
 /*
+ * FP4 (E2M1) with one scale per tensor -- the number format the paper's conclusion names as the step
+ * after FP8 (it fixes no format; taken here: the 4-bit floating-point element of the OCP
+ * Microscaling formats, 1 sign / 2 exponent (bias 1) / 1 mantissa bit, values +-{0, 0.5, 1, 1.5, 2,
+ * 3, 4, 6}, no infinity, no NaN) with the per-tensor scaling of Sec. 4.3: scale = fl32(6 / amax).
+ *
+ * tweo_fp4_quantize -- code_i = rne_sat(fl32(x_i * scale)): one binary32 multiply, one saturating
+ * round-to-nearest-even onto the E2M1 grid (ties to the even code; |v| >= 6 and infinities -> +-6;
+ * NaN -> +6, the format having no NaN; zero and values that round to zero keep their sign).
+ *   x: bf16 [n], 16-byte aligned.  mode CURRENT: amax = max|x| (NaN skipped), scale = 6 / amax
+ *   (1 when amax is 0 or not finite, clamped to FLT_MAX), scale_inv = 1 / scale are written;
+ *   mode GIVEN: *scale is read, *scale_inv and *amax (of this tensor) are written.
+ *   q4 (optional): packed codes, (n + 1) / 2 bytes, element 2i in the low nibble and element 2i + 1
+ *   in the high nibble of byte i (an odd n leaves the last high nibble 0); 8-byte aligned.
+ *   q8 (optional): "carriers", n bytes, the E4M3 code of every ROUNDED value (each E2M1 value is an
+ *   E4M3 value), 16-byte aligned: the operand form the FP8 GEMM entry points take, which then compute
+ *   the FP4 product exactly (pass fmt TWEO_E4M3 and this tensor's scale_inv).  At least one of q4, q8.
+ * All scalars are device pointers; nothing is read back by the host.
+ * Errors: TWEO_ERR_INVALID_ARG, TWEO_ERR_ALIGNMENT.
+ */
+TWEO_API tweo_status_t tweo_fp4_quantize(const uint16_t* x, int64_t n, int32_t mode, float* scale, float* scale_inv,
+                                float* amax, uint8_t* q4, uint8_t* q8, void* stream);
+
+/*
+ * tweo_fp4_unpack -- packed E2M1 codes (as tweo_fp4_quantize writes them) -> carriers: q8[i] = E4M3
+ * code of the value of code i.  For weights kept packed at rest and expanded once when loaded.
+ *   q4: (n + 1) / 2 bytes, 16-byte aligned; q8: n bytes, 16-byte aligned.
+ */
+TWEO_API tweo_status_t tweo_fp4_unpack(const uint8_t* q4, int64_t n, uint8_t* q8, void* stream);
+
+/*
+ * tweo_w4a4_static_gemm -- inference linear with static per-tensor scales and both operands on the
+ * E2M1 grid (the W4A4 setting the paper's conclusion points to, in its floating-point form):
+ *   Y[M,N] = (Xq . Wq^T) * (1 / *sx) * (*sw_inv) -> bf16,  Xq = tweo_fp4_quantize(x, GIVEN *sx).
+ *   x: bf16 [M,K], dense (ldx == K); sx: device const float*, the calibrated scale (6 / amax_cal).
+ *   wq8 [N,K]: carriers of the weight codes (tweo_fp4_quantize's q8, or tweo_fp4_unpack of the
+ *   packed codes), row pitch ldw; sw_inv: device const float*.
+ *   ws: tweo_workspace_bytes(TWEO_OP_W8A8, M, N, K) bytes (holds the activation carriers).
+ *   Shapes and routes as tweo_w8a8_static_gemm: N % 16 == 0, K % 16 == 0, any M >= 1.
+ */
+TWEO_API tweo_status_t tweo_w4a4_static_gemm(const uint16_t* x, int64_t ldx, const float* sx, const uint8_t* wq8,
+                                    int64_t ldw, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
+                                    int64_t N, int64_t K, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * tweo_absmax_quantize -- symmetric AbsMax b-bit quantisation (Sec. 4.4, Eq. 4):
  *   s = max|X| + eps,  X_q = round(X / s * Q_b),  Q_b = 2^(b-1) - 1   (Q_8 = 127, Q_6 = 31),
  * with one s for the whole tensor (TWEO_GRAN_TENSOR: the paper's "T") or one per row

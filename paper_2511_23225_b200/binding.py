@@ -29,6 +29,7 @@ EXPORTS = [
     "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_fwd_act",
     "tweo_layernorm_fp8", "tweo_fp8_linear_bwd_dgrad",
     "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_fp8_linear_group", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
+    "tweo_fp4_quantize", "tweo_fp4_unpack", "tweo_w4a4_static_gemm",
     "tweo_block_output_fused", "tweo_delayed_scaling_update", "tweo_absmax_quantize", "tweo_int8_linear", "tweo_int8_linear_q8", "tweo_residual_add_q8", "tweo_residual_add_q8_rows",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status", "tweo_selftest_bounded_wait",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
@@ -108,6 +109,9 @@ def lib() -> C.CDLL:
         L.tweo_residual_add_q8.argtypes = [vp, vp, vp, vp, i64, i32, vp, vp, vp]
         L.tweo_residual_add_q8_rows.argtypes = [vp, vp, vp, vp, i64, i64, i32, f32, vp, vp, vp]
         L.tweo_w8a8_static_gemm.argtypes = [vp, i32, i64, vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, sz, vp]
+        L.tweo_fp4_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp, vp, vp]
+        L.tweo_fp4_unpack.argtypes = [vp, i64, vp, vp]
+        L.tweo_w4a4_static_gemm.argtypes = [vp, i64, vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, sz, vp]
         L.tweo_workspace_bytes.argtypes = [i32, i64, i64, i64]
         L.tweo_workspace_bytes.restype = sz
         L.tweo_workspace_init.argtypes = [vp, sz, vp]
@@ -522,6 +526,69 @@ def w8a8_static_gemm(x, sx, wq, sw_inv, y=None, ws=None) -> torch.Tensor:
                                        _dev(wq, U8, "wq"), _rows(wq, "wq"), _dev(sw_inv, torch.float32),
                                        _dev(y, torch.bfloat16, "y"), _rows(y, "y"), M, N, K, ws.data_ptr(),
                                        ws.numel(), _stream()), "tweo_w8a8_static_gemm")
+    return y
+
+
+@dataclass
+class QuantizedFP4:
+    q4: torch.Tensor | None  # uint8 [(n + 1) // 2], two E2M1 codes per byte (element 2i in the low nibble)
+    q8: torch.Tensor | None  # uint8, x's shape: the E4M3 code of every rounded value (operand form of the FP8 GEMMs)
+    scale: torch.Tensor      # float32 [1]
+    scale_inv: torch.Tensor  # float32 [1]
+    amax: torch.Tensor       # float32 [1]
+
+
+def fp4_quantize(x: torch.Tensor, mode: int = SCALE_CURRENT, scale: torch.Tensor | None = None, packed: bool = True,
+                 carriers: bool = True, out: QuantizedFP4 | None = None) -> QuantizedFP4:
+    """tweo_fp4_quantize: amax -> scale -> E2M1 codes of a bf16 tensor (packed and / or as E4M3 carriers)."""
+    if not x.is_contiguous():
+        raise ValueError("x must be contiguous")
+    n = x.numel()
+    if out is None:
+        st = torch.zeros(3, dtype=torch.float32, device=x.device)
+        if mode == SCALE_GIVEN:
+            if scale is None:
+                raise ValueError("SCALE_GIVEN needs a scale")
+            st[0:1].copy_(scale)
+        out = QuantizedFP4(torch.empty((n + 1) // 2, dtype=torch.uint8, device=x.device) if packed else None,
+                           torch.empty(x.shape, dtype=torch.uint8, device=x.device) if carriers else None,
+                           st[0:1], st[1:2], st[2:3])
+    _check(lib().tweo_fp4_quantize(_dev(x, torch.bfloat16, "x"), n, mode, _dev(out.scale, torch.float32, "scale"),
+                                   _dev(out.scale_inv, torch.float32, "scale_inv"), _dev(out.amax, torch.float32, "amax"),
+                                   _dev(out.q4, U8, "q4") if out.q4 is not None else None,
+                                   _dev(out.q8, U8, "q8") if out.q8 is not None else None, _stream()),
+           "tweo_fp4_quantize")
+    return out
+
+
+def fp4_unpack(q4: torch.Tensor, shape, q8: torch.Tensor | None = None) -> torch.Tensor:
+    """tweo_fp4_unpack: packed E2M1 codes -> E4M3 carriers of the given shape."""
+    n = 1
+    for d in shape:
+        n *= int(d)
+    if q4.numel() != (n + 1) // 2:
+        raise ValueError("q4 holds (n + 1) // 2 bytes")
+    if q8 is None:
+        q8 = torch.empty(tuple(shape), dtype=torch.uint8, device=q4.device)
+    _check(lib().tweo_fp4_unpack(_dev(q4, U8, "q4"), n, _dev(q8, U8, "q8"), _stream()), "tweo_fp4_unpack")
+    return q8
+
+
+def w4a4_static_gemm(x, sx, wq8, sw_inv, y=None, ws=None) -> torch.Tensor:
+    """tweo_w4a4_static_gemm: static per-tensor linear with both operands on the E2M1 grid; bf16 activations,
+    weight carriers."""
+    M, K = x.shape
+    N, K2 = wq8.shape
+    if K != K2:
+        raise ValueError("inner dimensions differ")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    if ws is None:
+        ws = new_workspace(OP_W8A8, M, N, K)
+    _check(lib().tweo_w4a4_static_gemm(_dev(x, torch.bfloat16, "x"), _rows(x, "x"), _dev(sx, torch.float32, "sx"),
+                                       _dev(wq8, U8, "wq8"), _rows(wq8, "wq8"), _dev(sw_inv, torch.float32),
+                                       _dev(y, torch.bfloat16, "y"), _rows(y, "y"), M, N, K, ws.data_ptr(),
+                                       ws.numel(), _stream()), "tweo_w4a4_static_gemm")
     return y
 
 

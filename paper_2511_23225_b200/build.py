@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libtweo_b200.so")
-SOURCES = ["api.cu", "loss.cu", "block.cu", "absmax.cu", "norm.cu", "quantize.cu", "gemm.cu", "w8a8.cu"]
+SOURCES = ["api.cu", "loss.cu", "block.cu", "absmax.cu", "norm.cu", "quantize.cu", "gemm.cu", "w8a8.cu", "fp4.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fvisibility=hidden", "--expt-relaxed-constexpr"]
 

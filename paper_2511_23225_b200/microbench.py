@@ -79,6 +79,17 @@ def make(op, M, K, N):
         x = _bf16((M, K), 1.0, 1)
         out = tw.quantize_per_tensor(x, tw.E4M3, tw.SCALE_GIVEN, scale=_scalar(64.0))
         return (lambda: tw.quantize_per_tensor(x, tw.E4M3, tw.SCALE_GIVEN, out=out)), 3.0 * M * K, "GB/s"
+    if op == "fp4_quantize":   # one tensor [M, K] to E2M1, current scaling, packed codes and E4M3 carriers
+        x = _bf16((M, K), 1.0, 1)
+        out = tw.fp4_quantize(x)
+        return (lambda: tw.fp4_quantize(x, out=out)), 5.5 * M * K, "GB/s"
+    if op == "w4a4":           # static W4A4 linear: given-scale E2M1 cast of the activations, then the GEMM on carriers
+        x, w = _bf16((M, K), 1.0, 1), _bf16((N, K), 0.02, 2)
+        wq = tw.fp4_quantize(w, packed=False)
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        ws = tw.new_workspace(tw.OP_W8A8, M, N, K)
+        sx = _scalar(2.0)
+        return (lambda: tw.w4a4_static_gemm(x, sx, wq.q8, wq.scale_inv, y=y, ws=ws)), 2.0 * M * K * N, "TFLOP/s"
     if op == "loss":          # TWEO loss and bf16 gradient of one [M, K] block output
         a = [_bf16((M, K), 1.0, 1)]
         g = [torch.empty_like(a[0])]
@@ -132,7 +143,7 @@ def make(op, M, K, N):
 
 
 OPS = ("quantize", "quantize_given", "linear", "linear_fused", "linear_group", "loss", "block_output", "layernorm", "fwd_gelu", "fwd_swiglu", "absmax", "int8_linear_q8",
-       "residual_add_q8", "w8a8")
+       "residual_add_q8", "w8a8", "fp4_quantize", "w4a4")
 
 
 def main():

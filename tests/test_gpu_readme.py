@@ -47,5 +47,9 @@ def test_readme_call_sequences():
     sf, sy = torch.full((1,), 2.0, device="cuda"), torch.full((1,), 8.0, device="cuda")
     fq = tw.int8_linear_q8(xq, sx, wq8, sw, sf)
     yq = tw.residual_add_q8(xq, sx, fq, sf, sy)
+    wq4 = tw.fp4_quantize(w, carriers=False)
+    w8 = tw.fp4_unpack(wq4.q4, w.shape)
+    y4 = tw.w4a4_static_gemm(x, torch.full((1,), 6.0 / 4.0, device="cuda"), w8, wq4.scale_inv)
     torch.cuda.synchronize()
+    assert y4.shape == (M, N) and wq4.q4.numel() == N * K // 2
     assert yq.dtype == torch.int8 and yq.shape == (M, K) and tw.read_device_status() == 0
