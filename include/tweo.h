@@ -273,7 +273,9 @@ TWEO_API tweo_status_t tweo_fp8_linear_bwd(const uint8_t* dyq, int64_t lddy, int
  *   TWEO_PRODUCT_FWD    out = Y [M,N]  = tweo_fp8_linear_fwd       (xq, wq;  sx_inv, sw_inv)
  *   TWEO_PRODUCT_DGRAD  out = dX [M,K] = tweo_fp8_linear_bwd_dgrad (dyq, wq; sdy_inv, sw_inv)
  *   TWEO_PRODUCT_WGRAD  out = dW [N,K] = tweo_fp8_linear_bwd_wgrad (xq, dyq; sx_inv, sdy_inv; bf16, overwrite)
- * without fused epilogue outputs and without a workspace; results are bit-identical to those calls.  A launch costs
+ * without a workspace; results are bit-identical to those calls.  A FWD or DGRAD problem may carry the fused
+ * epilogue of the single call (`epi`: amax of the bf16 output, which the call resets first, and / or its FP8 copy
+ * with a given scale; the descriptor is read during the call); a WGRAD problem may not.  A launch costs
  * a fixed few microseconds (set-up, first loads, last epilogue) and leaves SMs idle at its ragged end; the tiles of
  * all problems of a group form one list, longest first, dealt to the CTA pairs so that each gets about the same
  * work, with one ramp-up and one tail for the whole group.
@@ -300,6 +302,7 @@ typedef struct tweo_linear_problem_t {
   uint16_t* out;                        /* bf16: Y [M,N], dX [M,K] or dW [N,K] */
   int64_t ldo;
   int64_t M, N, K;
+  const tweo_epilogue_t* epi;           /* optional fused outputs of Y (FWD) or dX (DGRAD); NULL: none */
 } tweo_linear_problem_t;
 TWEO_API tweo_status_t tweo_fp8_linear_group(const tweo_linear_problem_t* problems, int32_t count, void* stream);
 

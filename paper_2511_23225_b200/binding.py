@@ -62,7 +62,7 @@ class _LinearProblem(C.Structure):
                 ("xq", C.c_void_p), ("ldx", C.c_int64), ("wq", C.c_void_p), ("ldw", C.c_int64),
                 ("dyq", C.c_void_p), ("lddy", C.c_int64), ("sx_inv", C.c_void_p), ("sw_inv", C.c_void_p),
                 ("sdy_inv", C.c_void_p), ("out", C.c_void_p), ("ldo", C.c_int64),
-                ("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64)]
+                ("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64), ("epi", C.c_void_p)]
 
 
 class _Epilogue(C.Structure):
@@ -252,6 +252,11 @@ def quantize_per_tensor_batch(xs, outs, modes=None, ws: torch.Tensor | None = No
 
 
 def _epilogue(amax, q, q_fmt, q_scale):
+    e = _epilogue_struct(amax, q, q_fmt, q_scale)
+    return None if e is None else C.byref(e)
+
+
+def _epilogue_struct(amax, q, q_fmt, q_scale):
     if amax is None and q is None:
         return None
     e = _Epilogue()
@@ -261,7 +266,7 @@ def _epilogue(amax, q, q_fmt, q_scale):
         e.ldq = _rows(q, "out_q")
         e.q_fmt = q_fmt
         e.q_scale = _dev(q_scale, torch.float32, "q_scale")
-    return C.byref(e)
+    return e
 
 
 def _ws(ws):
@@ -408,12 +413,18 @@ def fp8_linear_group(problems):
     """tweo_fp8_linear_group: independent linear-layer products in one launch.  `problems` is a list of dicts:
     {"product": PRODUCT_FWD, "xq", "wq", "sx_inv", "sw_inv", "out" [M,N]}, {"product": PRODUCT_DGRAD, "dyq", "wq",
     "sdy_inv", "sw_inv", "out" [M,K]} or {"product": PRODUCT_WGRAD, "xq", "dyq", "sx_inv", "sdy_inv", "out" [N,K]},
-    each optionally with "fmt_x", "fmt_w", "fmt_dy" (defaults E4M3, E4M3, E5M2).  Outputs are bf16 tensors."""
+    each optionally with "fmt_x", "fmt_w", "fmt_dy" (defaults E4M3, E4M3, E5M2).  Outputs are bf16 tensors.  A FWD or
+    DGRAD problem may add the fused epilogue: "out_amax" and / or "out_q" with "q_fmt" and "q_scale"."""
     n = len(problems)
     if not 1 <= n <= MAX_GROUP:
         raise ValueError("need 1..MAX_GROUP problems")
     arr = (_LinearProblem * n)()
+    epis = []   # keeps the epilogue descriptors alive until the call returns
     for q, d in zip(arr, problems):
+        e = _epilogue_struct(d.get("out_amax"), d.get("out_q"), d.get("q_fmt", E4M3), d.get("q_scale"))
+        if e is not None:
+            epis.append(e)
+            q.epi = C.addressof(e)
         q.product = d["product"]
         q.fmt_x, q.fmt_w, q.fmt_dy = d.get("fmt_x", E4M3), d.get("fmt_w", E4M3), d.get("fmt_dy", E5M2)
         xq, wq, dyq = d.get("xq"), d.get("wq"), d.get("dyq")

@@ -725,13 +725,35 @@ struct GroupDesc {
   uint16_t* d;
   int64_t ldd;
   const float *sa, *sb;
+  // fused epilogue (all optional): amax of the bf16 output, its FP8 copy with the scale *q_scale
+  float* out_amax = nullptr;
+  uint8_t* out_q = nullptr;
+  int64_t ldq = 0;
+  int q_fmt = TWEO_E4M3;
+  const float* q_scale = nullptr;
 };
 
-template <int LIST>
+struct FloatPtrs {
+  float* p[kGroupMaxProblems];
+  int n;
+};
+// Clears the amax cells of a group's fused epilogues (in the chain, like zero_float_kernel).
+__global__ void zero_floats_kernel(const FloatPtrs f) {
+  chain_release();
+  chain_wait();
+  if ((int)threadIdx.x < f.n) *f.p[threadIdx.x] = 0.0f;
+}
+
+// QST: fused epilogue outputs (amax, FP8 copy) on some products.  EPIW / EBUF as in the kernel; the operand ring
+// takes what the staging buffers leave of the shared memory.
+template <int LIST, bool QST, int EPIW, int EBUF>
 tweo_status_t run_group_list(GroupDesc* d, int n, cudaStream_t st) {
-  constexpr int STAGES = 6;
-  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + 4 * 2 * 32 * 128 + 1024 + 256;
-  auto kern = gemm_fp8_pair_group_kernel<STAGES, LIST>;
+  constexpr size_t staging = (size_t)EPIW * EBUF * (32 * 128 + (QST ? 32 * 64 : 0));
+  constexpr int STAGES = (int)((227 * 1024 - 1024 - 256 - staging) / (BM * BK + 128 * BK)) > 6
+                             ? 6 : (int)((227 * 1024 - 1024 - 256 - staging) / (BM * BK + 128 * BK));
+  static_assert(STAGES >= 4, "operand ring too short");
+  constexpr size_t smem = (size_t)STAGES * (BM * BK + 128 * BK) + staging + 1024 + 256;
+  auto kern = gemm_fp8_pair_group_kernel<STAGES, LIST, QST, EPIW, EBUF>;
   static std::atomic<uint64_t> attr_done{0};  // per device
   int attr_dev = 0;
   if (device_once_pending(attr_done, &attr_dev)) {
@@ -756,9 +778,15 @@ tweo_status_t run_group_list(GroupDesc* d, int n, cudaStream_t st) {
     q.idesc = make_idesc(d[i].fa, d[i].fb, d[i].a_mn, d[i].b_mn, 256, 256);
     q.sa_inv = d[i].sa;
     q.sb_inv = d[i].sb;
+    q.out_amax = d[i].out_amax;
+    q.q_scale = d[i].out_q ? d[i].q_scale : nullptr;
+    q.q_fmt = d[i].q_fmt;
+    q.pad = 0;
     g.tile_start[i + 1] = g.tile_start[i] + q.tiles_m * q.tiles_n;
     cost[i] = (q.k_blocks < 8 ? 8 : q.k_blocks) + 2;  // k-blocks, with a floor for the epilogue of short tiles
     bool ok = make_out_map(&g.md[i], d[i].d, d[i].Nd, d[i].Md, d[i].ldd, false);
+    if (QST && d[i].out_q) ok = ok && make_q_map(&g.mq[i], d[i].out_q, d[i].Nd, d[i].Md, d[i].ldq);
+    else g.mq[i] = g.md[i];
     if (d[i].a_mn) ok = ok && make_map(&g.ma[i], d[i].a, d[i].Md, d[i].Kc, d[i].lda, BK);
     else ok = ok && make_map(&g.ma[i], d[i].a, d[i].Kc, d[i].Md, d[i].lda, BM);
     if (d[i].b_mn) ok = ok && make_map(&g.mb[i], d[i].b, d[i].Nd, d[i].Kc, d[i].ldb, BK);
@@ -798,7 +826,17 @@ tweo_status_t run_group_list(GroupDesc* d, int n, cudaStream_t st) {
     }
     for (int t = 0; t < g.total_tiles; ++t) g.list[fill[owner[t]]++] = (uint16_t)t;  // ascending t within a pair
   }
-  TWEO_CUDA_TRY(launch_chain(kern, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, st, 2, g));
+  if (QST) {
+    FloatPtrs z;
+    z.n = 0;
+    for (int i = 0; i < n; ++i)
+      if (d[i].out_amax) z.p[z.n++] = d[i].out_amax;
+    if (z.n) {
+      TWEO_CUDA_TRY(launch_chain(zero_floats_kernel, dim3(1), dim3(32), 0, st, 0, z));
+      count_launch();
+    }
+  }
+  TWEO_CUDA_TRY(launch_chain(kern, dim3((unsigned)(2 * pairs)), dim3(64 + 32 * EPIW), smem, st, 2, g));
   count_launch();
   return check_launch("gemm_fp8_pair_group_kernel");
 }
@@ -811,7 +849,21 @@ tweo_status_t run_group(GroupDesc* d, int n, cudaStream_t st) {
   });
   int64_t tiles = 0;
   for (int i = 0; i < n; ++i) tiles += ((d[i].Md + 2 * BM - 1) / (2 * BM)) * ((d[i].Nd + 255) / 256);
-  return tiles <= kGroupListSmall ? run_group_list<kGroupListSmall>(d, n, st) : run_group_list<kGroupListLarge>(d, n, st);
+  bool fused = false;
+  int64_t fused_kb_min = INT64_MAX;
+  for (int i = 0; i < n; ++i)
+    if (d[i].out_amax || d[i].out_q) {
+      fused = true;
+      fused_kb_min = std::min(fused_kb_min, (d[i].Kc + BK - 1) / BK);
+    }
+  const bool small = tiles <= kGroupListSmall;
+  if (!fused)
+    return small ? run_group_list<kGroupListSmall, false, 4, 2>(d, n, st) : run_group_list<kGroupListLarge, false, 4, 2>(d, n, st);
+  // the fused epilogue computes per element: at short contractions it outlasts the tile's main loop unless eight
+  // warps share it (the rule of the single fused products)
+  if (fused_kb_min < 16)
+    return small ? run_group_list<kGroupListSmall, true, 8, 1>(d, n, st) : run_group_list<kGroupListLarge, true, 8, 1>(d, n, st);
+  return small ? run_group_list<kGroupListSmall, true, 4, 1>(d, n, st) : run_group_list<kGroupListLarge, true, 4, 1>(d, n, st);
 }
 
 // dX and dW of one linear layer as a group of two products.
@@ -1117,6 +1169,18 @@ tweo_status_t tweo_fp8_linear_group(const tweo_linear_problem_t* problems, int32
         break;
       default:
         return TWEO_ERR_INVALID_ARG;
+    }
+    if (q.epi && (q.epi->out_amax || q.epi->out_q)) {
+      if (q.product == TWEO_PRODUCT_WGRAD) return TWEO_ERR_INVALID_ARG;   // the fused outputs feed the next linear: Y and dX only
+      d[i].out_amax = q.epi->out_amax;
+      if (q.epi->out_q) {
+        if (!q.epi->q_scale || !fmt_ok(q.epi->q_fmt)) return TWEO_ERR_INVALID_ARG;
+        if (!tweo_detail::aligned16(q.epi->out_q) || (q.epi->ldq & 15)) return TWEO_ERR_ALIGNMENT;
+        d[i].out_q = q.epi->out_q;
+        d[i].ldq = q.epi->ldq;
+        d[i].q_fmt = q.epi->q_fmt;
+        d[i].q_scale = q.epi->q_scale;
+      }
     }
     if (d[i].Md <= 128 || d[i].Nd <= 128) return TWEO_ERR_UNSUPPORTED_SHAPE;   // the pair kernel's 256 x 256 tiles
     if (!tweo_detail::aligned16(d[i].a) || !tweo_detail::aligned16(d[i].b) || (d[i].lda & 15) || (d[i].ldb & 15))

@@ -12,8 +12,10 @@
 //
 // The kernel is the CTA-pair kernel of gemm_pair.cuh (256 x 256 tiles, tcgen05 cta_group::2,
 // TMA-fed ring, two accumulators in tensor memory, staged TMA-store epilogue) with the operand
-// layouts taken at run time per product, bf16 outputs only, no fused epilogue and no splitting
-// along the contraction.  Every wait is bounded.
+// layouts taken at run time per product, bf16 outputs only and no splitting along the contraction.
+// The QST instantiation also carries the fused epilogue of the training step per product: the maximum
+// of |output| and the FP8 copy of the output with a given scale, staged in shared memory and stored by
+// TMA like the bf16 tile (one operand stage less).  Every wait is bounded.
 #pragma once
 
 #include <cuda.h>
@@ -35,11 +37,17 @@ struct GroupProblem {
   uint32_t idesc;
   const float* sa_inv;
   const float* sb_inv;
+  // fused epilogue (QST instantiation only)
+  float* out_amax;        // nullptr: none
+  const float* q_scale;   // nullptr: no FP8 copy
+  int32_t q_fmt;
+  int32_t pad;
 };
 
 template <int LIST>
 struct alignas(64) PairGroupParams {
   CUtensorMap ma[kGroupMaxProblems], mb[kGroupMaxProblems], md[kGroupMaxProblems];
+  CUtensorMap mq[kGroupMaxProblems];  // FP8 copies of the outputs (QST instantiation)
   GroupProblem pr[kGroupMaxProblems];
   int32_t n_problems;
   int32_t tile_start[kGroupMaxProblems + 1];  // product i owns the tile numbers [tile_start[i], tile_start[i + 1])
@@ -83,8 +91,12 @@ __device__ __forceinline__ void group_tile_coords(const GroupProblem& q, int til
   tm = first + in - tn * rows;
 }
 
-template <int STAGES, int LIST>
-__global__ void __launch_bounds__(kThreads, 1)
+// EPIW: epilogue warps per CTA (4 or 8; with 8, two warps share each quarter of the tensor-memory lanes and take
+// half of a tile's columns each -- the fused epilogue of a short contraction is bound by the issue rate of one
+// warp per scheduler).  EBUF: staging buffers per epilogue warp (2: a chunk is staged while the store of the
+// one before it drains; 1: half the staging memory, which buys an operand stage).
+template <int STAGES, int LIST, bool QST = false, int EPIW = 4, int EBUF = 2>
+__global__ void __launch_bounds__(64 + 32 * EPIW, 1)
 gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams<LIST> g) {
   constexpr int BN = 256;                 // tile columns of the pair
   constexpr uint32_t A_BYTES = BM * BK;   // this CTA's 128 rows of A
@@ -96,9 +108,13 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams<LIST> g) {
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   constexpr uint32_t EPI_BUF = 32 * 128;
-  constexpr uint32_t EPI_BYTES = 4 * 2 * EPI_BUF;
+  static_assert(EPIW == 4 || EPIW == 8, "epilogue warps per CTA");
+  static_assert(EBUF == 1 || EBUF == 2, "staging buffers per epilogue warp");
+  constexpr uint32_t EPI_BYTES = EPIW * EBUF * EPI_BUF;
+  constexpr uint32_t Q_BUF = 32 * 64;  // 32 rows x 64 one-byte codes
+  constexpr uint32_t Q_BYTES = QST ? EPIW * EBUF * Q_BUF : 0;
   uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(epi_smem + EPI_BYTES + Q_BYTES);
   // bars: [0,STAGES) full, [STAGES,2*STAGES) empty, then tfull[2], tempty[2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -121,7 +137,7 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams<LIST> g) {
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 8);  // four epilogue warps of each CTA of the pair
+      mbar_init(tempty_bar(a), 2 * EPIW);  // the epilogue warps of both CTAs of the pair
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -219,17 +235,33 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams<LIST> g) {
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    // ------------------------------------------------------------ epilogue (warps 2.., both CTAs)
     chain_wait();
-    const int quarter = warp & 3;
-    const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * 2u * EPI_BUF;
+    const int quarter = warp & 3;  // the tensor-memory lanes a warp may read: (warp index mod 4) * 32 ...
+    const uint32_t epi_base = smem_u32(epi_smem) + (uint32_t)(warp - 2) * (uint32_t)EBUF * EPI_BUF;
     const uint32_t row_off = (uint32_t)lane * 128u;
     const uint32_t swz = (uint32_t)(lane & 7);
     const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
+    const uint32_t q_base = smem_u32(epi_smem) + EPI_BYTES + (uint32_t)(warp - 2) * (uint32_t)EBUF * Q_BUF;
+    // with 8 epilogue warps, warps 2-5 take the first half of a tile's chunks and warps 6-9 the second
+    constexpr int NC_W = (BN / CH) / (EPIW / 4);
+    const int c_first = ((warp - 2) >> 2) * NC_W;
     uint32_t it = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
+    // fused amax: the running maximum of |accumulator| of the product this warp is working on; written out
+    // (scaled and rounded like the stored values) when the list moves on to another product and at the end
+    float run_max = 0.0f, max_alpha = 0.0f;
+    float* max_dst = nullptr;
+    auto flush_max = [&]() {
+      if (QST && max_dst) {
+        float m = __uint_as_float(f32_to_bf16_bits(__fmul_rn(run_max, fabsf(max_alpha))) << 16);
+        m = warp_max(m);
+        if (lane == 0 && m > 0.0f) atomicMax(reinterpret_cast<unsigned int*>(max_dst), __float_as_uint(m));
+      }
+      run_max = 0.0f;
+    };
     GroupSched sched(g, pair, num_pairs);
     int prob, tile;
     while (ok && sched.next(g, prob, tile)) {
@@ -237,6 +269,15 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams<LIST> g) {
       const CUtensorMap* md = &g.md[prob];
       const float alpha = __fmul_rn(__ldg(q.sa_inv), __ldg(q.sb_inv));
       const int Md = q.Md, Nd = q.Nd;
+      float qs = 0.0f;
+      if (QST) {
+        if (q.out_amax != max_dst) {
+          flush_max();
+          max_dst = q.out_amax;
+        }
+        max_alpha = alpha;
+        if (q.q_scale) qs = __ldg(q.q_scale);
+      }
       int tm, tn;
       group_tile_coords(q, tile, tm, tn);
       const int m0 = tm * (2 * BM) + (int)rank * BM;
@@ -245,7 +286,7 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams<LIST> g) {
       tc_fence_after();
       const int row0 = m0 + quarter * 32;
 #pragma unroll 1
-      for (int c = 0; c < BN / CH; ++c) {
+      for (int c = c_first; c < c_first + NC_W; ++c) {
         const int col0 = n0 + c * CH;
         if (col0 >= Nd) break;
         uint32_t r[CH];
@@ -254,9 +295,15 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams<LIST> g) {
         tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
         tmem_ld_wait();
         if (row0 >= Md) continue;
-        const uint32_t buf = epi_base + (it & 1u) * EPI_BUF;
-        if (lane == 0) bulk_wait_read<1>();
+        const uint32_t ebuf = EBUF == 2 ? (it & 1u) : 0u;
+        const uint32_t buf = epi_base + ebuf * EPI_BUF;
+        if (lane == 0) bulk_wait_read<EBUF - 1>();
         __syncwarp();
+        if (QST && max_dst) {
+          // rows and columns beyond the output hold exact zeros (the loads fill them), so they do not count
+#pragma unroll
+          for (int j = 0; j < CH; ++j) run_max = fmaxf(run_max, fabsf(__uint_as_float(r[j])));
+        }
         uint32_t packed[CH / 2];
 #pragma unroll
         for (int j = 0; j < CH / 2; ++j)
@@ -266,10 +313,27 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams<LIST> g) {
         for (int j = 0; j < 8; ++j)
           st_shared_v4(buf + row_off + (((uint32_t)j ^ swz) << 4), packed[4 * j], packed[4 * j + 1], packed[4 * j + 2],
                        packed[4 * j + 3]);
+        const uint32_t qbuf = q_base + ebuf * Q_BUF;
+        if (QST && q.q_scale) {
+          // 64 codes per row -> 32 rows x 64 B, 16-byte pieces XOR-swizzled with row bits 1-2
+          const uint32_t qrow = qbuf + (uint32_t)lane * 64u;
+          const uint32_t qswz = ((uint32_t)lane >> 1) & 3u;
+#pragma unroll
+          for (int g4 = 0; g4 < 4; ++g4) {
+            uint32_t qq[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t w0 = packed[8 * g4 + 2 * j], w1 = packed[8 * g4 + 2 * j + 1];
+              qq[j] = q.q_fmt == TWEO_E4M3 ? quant_words<TWEO_E4M3>(w0, w1, qs) : quant_words<TWEO_E5M2>(w0, w1, qs);
+            }
+            st_shared_v4(qrow + (((uint32_t)g4 ^ qswz) << 4), qq[0], qq[1], qq[2], qq[3]);
+          }
+        }
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
           tma_store_2d(md, col0, row0, buf);
+          if (QST && q.q_scale) tma_store_2d(&g.mq[prob], col0, row0, qbuf);
           bulk_commit();
         }
         ++it;
@@ -280,6 +344,7 @@ gemm_fp8_pair_group_kernel(const __grid_constant__ PairGroupParams<LIST> g) {
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
+    flush_max();
     if (lane == 0) bulk_wait_all();
   }
 

@@ -152,10 +152,15 @@ class BlockStep:
         modes = None if self.variant == "plain" else [tw.SCALE_GIVEN] * len(xs)
         tw.quantize_per_tensor_batch(xs, qs, modes, ws=self.quant_ws)
 
-    def cast_batches(self):
-        """The linears in cast order: the first alone (the first GEMM waits for it), then two per batch call."""
+    def batches(self):
+        """The linears two by two (a batch call casts two linears' tensors, a grouped launch runs their six products);
+        an odd count puts the single one first, so that the first GEMM launch waits for one linear's casts only."""
         idx = list(range(len(self.linears)))
-        return [idx[:1]] + [idx[i:i + 2] for i in range(1, len(idx), 2)]
+        head = len(idx) % 2
+        return ([idx[:1]] if head else []) + [idx[i:i + 2] for i in range(head, len(idx), 2)]
+
+    def cast_batches(self):
+        return self.batches()
 
     def gemms(self, lb: LinearBuffers, i: int = 0):
         if self.variant == "fused":
@@ -189,31 +194,36 @@ class BlockStep:
 
     def group_ok(self, lb: LinearBuffers) -> bool:
         """Whether all three products of this linear can go into a grouped launch (outputs wider and taller than 128)."""
-        return self.variant != "fused" and min(self.M, lb.lin.K, lb.lin.N) > 128
+        return min(self.M, lb.lin.K, lb.lin.N) > 128
 
     def gemms_grouped(self, lbs):
         """Forward, data-gradient and weight-gradient product of each of the given linears in ONE launch."""
         probs = []
-        for lb in lbs:
-            probs += [dict(product=tw.PRODUCT_FWD, xq=lb.qx.q, wq=lb.qw.q, sx_inv=lb.qx.scale_inv, sw_inv=lb.qw.scale_inv, out=lb.y),
+        for i, lb in lbs:
+            fwd_epi, dgrad_epi = {}, {}
+            if self.variant == "fused":   # amax and the FP8 copy of Y and dX from the epilogue, delayed scales
+                fwd_epi = dict(out_amax=self.amax_y[i:i + 1], out_q=lb.yq, q_fmt=tw.E4M3, q_scale=self.scale_y[i:i + 1])
+                dgrad_epi = dict(out_amax=self.amax_dx[i:i + 1], out_q=lb.dxq, q_fmt=self.grad_fmt,
+                                 q_scale=self.scale_dx[i:i + 1])
+            probs += [dict(product=tw.PRODUCT_FWD, xq=lb.qx.q, wq=lb.qw.q, sx_inv=lb.qx.scale_inv, sw_inv=lb.qw.scale_inv, out=lb.y,
+                           **fwd_epi),
                       dict(product=tw.PRODUCT_DGRAD, dyq=lb.qdy.q, wq=lb.qw.q, sdy_inv=lb.qdy.scale_inv, sw_inv=lb.qw.scale_inv,
-                           fmt_dy=self.grad_fmt, out=lb.dx),
+                           fmt_dy=self.grad_fmt, out=lb.dx, **dgrad_epi),
                       dict(product=tw.PRODUCT_WGRAD, xq=lb.qx.q, dyq=lb.qdy.q, sx_inv=lb.qx.scale_inv, sdy_inv=lb.qdy.scale_inv,
                            fmt_dy=self.grad_fmt, out=lb.dw)]
         tw.fp8_linear_group(probs)
 
     def gemm_batches(self):
-        """The linears in launch order: pairs that share a grouped launch (plain variant), else one by one."""
-        idx = list(range(len(self.linears)))
+        """The linears in launch order: the cast batches where every product can share a grouped launch, else one by one."""
         if not all(self.group_ok(lb) for lb in self.linears):
-            return [[i] for i in idx]
-        return [idx[i:i + 2] for i in range(0, len(idx), 2)]
+            return [[i] for i in range(len(self.linears))]
+        return self.batches()
 
     def run_gemm_batch(self, batch):
         if len(batch) == 1 and not self.group_ok(self.linears[batch[0]]):
             self.gemms(self.linears[batch[0]], batch[0])
         else:
-            self.gemms_grouped([self.linears[i] for i in batch])
+            self.gemms_grouped([(i, self.linears[i]) for i in batch])
             if self.variant == "unfused":
                 self.cast_outputs(batch)
 

@@ -80,3 +80,70 @@ def test_group_rejects_what_it_cannot_tile(tw):
     with pytest.raises(tw.TweoError) as e:      # a product whose operands were not given
         tw.fp8_linear_group([dict(product=tw.PRODUCT_DGRAD, dyq=dyq.new_zeros((256, 256)), wq=wq, sw_inv=sw, out=big)])
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("fmt_g", [E5M2, E4M3], ids=["e5m2grad", "e4m3grad"])
+def test_group_with_fused_epilogues_equals_the_single_calls_and_the_oracle(tw, fmt_g):
+    """The training step's fused outputs from a grouped launch: amax and the FP8 copy of Y (E4M3) and dX (gradient
+    format) per product, mixed with products that have none, only an amax, or only a copy.  Bit-identical to the
+    single calls; amax and codes also against the oracle (amax of the bf16 output, codes of the bf16 output under
+    the given scale).  Twice in a row: the amax cells are reset by the call."""
+    lins = [make_linear(640, 300, 400, 272, fmt_g), make_linear(650, 1024, 768, 2304, fmt_g),
+            make_linear(660, 2048, 256, 384, fmt_g)]
+    problems, singles, oracle_checks = [], [], []
+    u8 = lambda r, c: torch.zeros((r, c), dtype=torch.uint8, device="cuda")
+    bf = lambda r, c: torch.zeros((r, c), dtype=torch.bfloat16, device="cuda")
+    for li, (q, (xq, wq, dyq), (sx, sw, sd)) in enumerate(lins):
+        M, K = xq.shape
+        N = wq.shape[0]
+        sy, sdx = dev_scalar(37.0 + li), dev_scalar(2.9e4 if fmt_g == E5M2 else 310.0)
+        want = [dict(amax=True, q=True), dict(amax=True, q=False), dict(amax=False, q=True)][li]
+        def epi(rows, cols, fmt, scale):
+            d = {}
+            if want["amax"]:
+                d["out_amax"] = torch.full((1,), 123.0, dtype=torch.float32, device="cuda")   # stale value
+            if want["q"]:
+                d.update(out_q=u8(rows, cols), q_fmt=fmt, q_scale=scale)
+            return d
+        pf = dict(product=tw.PRODUCT_FWD, xq=xq, wq=wq, sx_inv=sx, sw_inv=sw, out=bf(M, N), **epi(M, N, E4M3, sy))
+        pd = dict(product=tw.PRODUCT_DGRAD, dyq=dyq, wq=wq, sdy_inv=sd, sw_inv=sw, fmt_dy=fmt_g, out=bf(M, K),
+                  **epi(M, K, fmt_g, sdx))
+        pw = dict(product=tw.PRODUCT_WGRAD, xq=xq, dyq=dyq, sx_inv=sx, sdy_inv=sd, fmt_dy=fmt_g, out=bf(N, K))
+        problems += [pf, pd, pw]
+        # the single calls with the same fused outputs
+        sf = dict(amax=torch.zeros(1, device="cuda") if want["amax"] else None, q=u8(M, N) if want["q"] else None)
+        sdg = dict(amax=torch.zeros(1, device="cuda") if want["amax"] else None, q=u8(M, K) if want["q"] else None)
+        yf = tw.fp8_linear_fwd(xq, wq, sx, sw, out_amax=sf["amax"], out_q=sf["q"], q_fmt=E4M3, q_scale=sy)
+        yd = tw.fp8_linear_bwd_dgrad(dyq, wq, sd, sw, fmt_dy=fmt_g, out_amax=sdg["amax"], out_q=sdg["q"], q_fmt=fmt_g,
+                                     q_scale=sdx)
+        yw = tw.fp8_linear_bwd_wgrad(xq, dyq, sx, sd, fmt_dy=fmt_g)
+        singles += [(yf, sf), (yd, sdg), (yw, dict(amax=None, q=None))]
+        oracle_checks += [(E4M3, float(sy.item())), (fmt_g, float(sdx.item())), None]
+    problems, singles, oracle_checks = problems[:8], singles[:8], oracle_checks[:8]      # eight products per launch
+    for rep in range(2):
+        tw.fp8_linear_group(problems)
+        torch.cuda.synchronize()
+        assert tw.read_device_status() == 0
+        for prob, (one, fused), chk in zip(problems, singles, oracle_checks):
+            assert torch.equal(prob["out"].view(torch.int16), one.view(torch.int16))
+            out_bits = prob["out"].view(torch.int16).cpu().numpy().view(np.uint16)
+            if fused["amax"] is not None:
+                assert torch.equal(prob["out_amax"], fused["amax"])
+                assert float(prob["out_amax"].item()) == float(orc.amax_bf16(out_bits))
+            if fused["q"] is not None:
+                assert torch.equal(prob["out_q"], fused["q"])
+                q_ref, _ = orc.quantize_bf16(out_bits, chk[0], np.float32(chk[1]))
+                assert np.array_equal(prob["out_q"].cpu().numpy(), q_ref)
+
+
+def test_group_rejects_fused_outputs_on_a_weight_gradient(tw):
+    q, (xq, wq, dyq), (sx, sw, sd) = make_linear(670, 256, 256, 384)
+    out = torch.empty((384, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(tw.TweoError) as e:
+        tw.fp8_linear_group([dict(product=tw.PRODUCT_WGRAD, xq=xq, dyq=dyq, sx_inv=sx, sdy_inv=sd, out=out,
+                                  out_amax=torch.zeros(1, device="cuda"))])
+    assert e.value.status == 1
+    y = torch.empty((256, 384), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises((tw.TweoError, TypeError)):   # an FP8 copy without its scale
+        tw.fp8_linear_group([dict(product=tw.PRODUCT_FWD, xq=xq, wq=wq, sx_inv=sx, sw_inv=sw, out=y,
+                                  out_q=torch.empty((256, 384), dtype=torch.uint8, device="cuda"))])
