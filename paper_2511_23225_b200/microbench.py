@@ -75,6 +75,28 @@ def make(op, M, K, N):
                  dict(product=tw.PRODUCT_DGRAD, dyq=dyq, wq=wq, sdy_inv=s, sw_inv=s, out=dx),
                  dict(product=tw.PRODUCT_WGRAD, xq=xq, dyq=dyq, sx_inv=s, sdy_inv=s, out=dw)]
         return (lambda: tw.fp8_linear_group(probs)), 6.0 * M * K * N, "TFLOP/s"
+    if op == "linear_group_fused":  # the three products of one linear in one launch, Y and dX with the fused epilogue
+        xq, wq, dyq = _codes((M, K), 1), _codes((N, K), 2), _codes((M, N), 3)
+        s, qs = _scalar(1e-3), _scalar(4.0)
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+        dw = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
+        yq = torch.empty((M, N), dtype=torch.uint8, device="cuda")
+        dxq = torch.empty((M, K), dtype=torch.uint8, device="cuda")
+        am = torch.zeros(2, dtype=torch.float32, device="cuda")
+        probs = [dict(product=tw.PRODUCT_FWD, xq=xq, wq=wq, sx_inv=s, sw_inv=s, out=y, out_amax=am[0:1], out_q=yq,
+                      q_fmt=tw.E4M3, q_scale=qs),
+                 dict(product=tw.PRODUCT_DGRAD, dyq=dyq, wq=wq, sdy_inv=s, sw_inv=s, out=dx, out_amax=am[1:2], out_q=dxq,
+                      q_fmt=tw.E5M2, q_scale=qs),
+                 dict(product=tw.PRODUCT_WGRAD, xq=xq, dyq=dyq, sx_inv=s, sdy_inv=s, out=dw)]
+        return (lambda: tw.fp8_linear_group(probs)), 6.0 * M * K * N, "TFLOP/s"
+    if op == "quantize_given_batch":  # the three casts of one linear with given (delayed) scales: one pass per format
+        xs = [_bf16((M, K), 1.0, 1), _bf16((N, K), 0.02, 2), _bf16((M, N), 1e-3, 3)]
+        outs = [tw.quantize_per_tensor(x, f, tw.SCALE_GIVEN, scale=_scalar(sc))
+                for x, f, sc in zip(xs, (tw.E4M3, tw.E4M3, tw.E5M2), (64.0, 4000.0, 1e6))]
+        modes = [tw.SCALE_GIVEN] * 3
+        ws = tw.new_workspace(tw.OP_QUANTIZE)
+        return (lambda: tw.quantize_per_tensor_batch(xs, outs, modes, ws=ws)), 3.0 * sum(x.numel() for x in xs), "GB/s"
     if op == "quantize_given":  # one tensor [M, K], given (delayed / static) scale: single pass, amax as by-product
         x = _bf16((M, K), 1.0, 1)
         out = tw.quantize_per_tensor(x, tw.E4M3, tw.SCALE_GIVEN, scale=_scalar(64.0))
@@ -142,7 +164,7 @@ def make(op, M, K, N):
     raise SystemExit(f"unknown --op {op}")
 
 
-OPS = ("quantize", "quantize_given", "linear", "linear_fused", "linear_group", "loss", "block_output", "layernorm", "fwd_gelu", "fwd_swiglu", "absmax", "int8_linear_q8",
+OPS = ("quantize", "quantize_given", "linear", "linear_fused", "linear_group", "linear_group_fused", "quantize_given_batch", "loss", "block_output", "layernorm", "fwd_gelu", "fwd_swiglu", "absmax", "int8_linear_q8",
        "residual_add_q8", "w8a8", "fp4_quantize", "w4a4")
 
 
