@@ -899,12 +899,13 @@ def run_cuda(args):
         for v in VARIANT_ORDER:
             if v == args.variant:
                 continue
-            o = measure_workload(torch, tw, cfg_idx, v, args.also_steps, 3, barrier, local, host=host, overlap=overlap,
+            # as many steps as the headline, so that the variants meet the same power / clock regime
+            o = measure_workload(torch, tw, cfg_idx, v, args.steps, 3, barrier, local, host=host, overlap=overlap,
                                  peaks=peaks)
             k = o["kernels"]
             variants[v] = {"ms_per_step": o["ms_per_step"], "value": flops_per_step / (o["ms_per_step"] * 1e-3) / 1e12,
                            "unit": UNIT, "launches_per_step": o["launches_per_step"], **gemm_summary(k, fp8_burst),
-                           "gemm_ms": k["gemm"]["ms_per_step"], "clocks": o["clocks"]}
+                           "gemm_ms": k["gemm"]["ms_per_step"], "steps": args.steps, "clocks": o["clocks"]}
             del o
             torch.cuda.empty_cache()
         fractions[args.workload]["step_tflops_by_variant"] = {args.variant: value / world,
