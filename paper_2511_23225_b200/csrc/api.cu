@@ -63,7 +63,7 @@ const char* tweo_status_string(tweo_status_t s) {
 
 const char* tweo_last_cuda_error(void) { return g_err; }
 
-int32_t tweo_version(void) { return 300; }
+int32_t tweo_version(void) { return 301; }
 
 uint64_t tweo_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
