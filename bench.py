@@ -52,7 +52,7 @@ UNIT = "TFLOP/s"
 FP8_DATASHEET_TFLOPS = 4500.0
 # DRAM traffic of the dominant kernel family (the GEMM launches of a step), per launch, from the ncu captures of
 # single launches summarised under profiles/; reported only while the GEMM sources are the ones profiled.
-GEMM_TRAFFIC = {"sources": "0912f393552f3652", "workload": "cfg4", "variant": "fused", "dram_over_algorithmic": 1.09,
+GEMM_TRAFFIC = {"sources": "91273a37be8bd483", "workload": "cfg4", "variant": "fused", "dram_over_algorithmic": 1.09,
                 "from": "profiles/gemm_pair_group_kernel_fused_epilogue_cfg2_qkv_cfg4_qkv.md (one linear's grouped launch, "
                         "scaled by the algorithmic bytes of the family)"}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, FALLBACK_BF16_SUSTAINED = 6650.0, 1590.0, 1400.0
@@ -548,6 +548,24 @@ def fp4_bench(torch, tw, peaks, reps=10):
             return q4, torch.empty(n, dtype=torch.uint8, device="cuda")
         us, k = rotating_us(torch, side, make_packed, lambda st: tw.fp4_unpack(st[0], (n,), q8=st[1]), 1.5 * n)
         out["cast"].append(_hbm_row(peaks, us, 1.5 * n, op="unpack", tensor=name, buffer_sets=k))
+        torch.cuda.empty_cache()
+    # few tokens on PACKED weights: the weight stream that bounds the call is half that of 8-bit weights (cold W:
+    # rotating weight buffers, as in the config-5 sweep)
+    out["packed_weight_linear_few_tokens"] = []
+    one = torch.ones(1, dtype=torch.float32, device="cuda")
+    for K, N in ((4096, 11008), (11008, 4096)):
+        Kp = (K + 127) // 128 * 128          # the packed route wants K % 128 == 0 (11008 = 86 * 128)
+        w4 = torch.randint(0, 256, (N, Kp // 2), dtype=torch.uint8, device="cuda")
+        for M in (1, 16, 128):
+            xq = torch.randint(0, 256, (M, Kp), dtype=torch.uint8, device="cuda") & 0xBF
+            y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            nbytes = float(M * Kp + Kp * N // 2 + 2 * M * N)
+            us, k = rotating_us(torch, side, lambda i: w4.clone(), lambda w: tw.fp4_weight_linear(xq, one, w, one, y=y), nbytes)
+            out["packed_weight_linear_few_tokens"].append(
+                {"M": M, "K": Kp, "N": N, "us": us, "weight_buffers": k, "l2_resident": False, "gbs": nbytes / us / 1e3,
+                 "frac_of_hbm_roofline": nbytes / peaks["hbm"] / 1e3 / us})
+            del xq, y
+        del w4
         torch.cuda.empty_cache()
     for K, N in ((4096, 4096), (4096, 11008)):
         w = (0.02 * torch.randn((N, K), device="cuda")).to(torch.bfloat16)

@@ -456,6 +456,23 @@ TWEO_API tweo_status_t tweo_w4a4_static_gemm(const uint16_t* x, int64_t ldx, con
                                     int64_t N, int64_t K, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * tweo_fp4_weight_linear -- the few-token inference linear with the weights kept PACKED in memory (two E2M1 codes
+ * per byte): Y[M,N] = (Xq . Wq^T) * (*sx_inv) * (*sw_inv) -> bf16 for M <= 128, where streaming W once bounds the
+ * call -- packed weights halve that stream.  The loads expand the codes on their way into shared memory and the
+ * tensor core reads them as E2M1 operands beside the 8-bit activations, so the result equals
+ * tweo_fp8_linear_fwd on the carriers of the same codes.
+ *   xq [M,K]: E4M3 or E5M2 codes (fmt_x), or E2M1 carriers (fmt_x = TWEO_E4M3; then the product is W4A4), row
+ *   pitch ldx; w4 [N, K/2 bytes]: tweo_fp4_quantize's packed codes of a [N,K] weight, row pitch ldw_bytes;
+ *   sx_inv, sw_inv: device scalars (reciprocal scales).
+ *   Shapes: 1 <= M <= 128 (else TWEO_ERR_UNSUPPORTED_SHAPE: expand the weights once with tweo_fp4_unpack and use
+ *   the FP8 entry points, which are bound by the tensor core there, not by the weight stream), N % 16 == 0,
+ *   K % 128 == 0.  w4 32-byte aligned, ldw_bytes % 32 == 0, xq 16-byte aligned, ldx % 16 == 0.
+ */
+TWEO_API tweo_status_t tweo_fp4_weight_linear(const uint8_t* xq, int64_t ldx, int32_t fmt_x, const float* sx_inv,
+                                     const uint8_t* w4, int64_t ldw_bytes, const float* sw_inv, uint16_t* y,
+                                     int64_t ldy, int64_t M, int64_t N, int64_t K, void* stream);
+
+/*
  * tweo_absmax_quantize -- symmetric AbsMax b-bit quantisation (Sec. 4.4, Eq. 4):
  *   s = max|X| + eps,  X_q = round(X / s * Q_b),  Q_b = 2^(b-1) - 1   (Q_8 = 127, Q_6 = 31),
  * with one s for the whole tensor (TWEO_GRAN_TENSOR: the paper's "T") or one per row

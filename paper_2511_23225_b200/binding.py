@@ -29,7 +29,7 @@ EXPORTS = [
     "tweo_quantize_per_tensor", "tweo_quantize_per_tensor_batch", "tweo_fp8_linear_fwd", "tweo_fp8_linear_fwd_act",
     "tweo_layernorm_fp8", "tweo_fp8_linear_bwd_dgrad",
     "tweo_fp8_linear_bwd_wgrad", "tweo_fp8_linear_bwd", "tweo_fp8_linear_group", "tweo_loss_fwd_bwd", "tweo_loss_fwd_bwd_static", "tweo_w8a8_static_gemm",
-    "tweo_fp4_quantize", "tweo_fp4_unpack", "tweo_w4a4_static_gemm",
+    "tweo_fp4_quantize", "tweo_fp4_unpack", "tweo_w4a4_static_gemm", "tweo_fp4_weight_linear",
     "tweo_block_output_fused", "tweo_delayed_scaling_update", "tweo_absmax_quantize", "tweo_int8_linear", "tweo_int8_linear_q8", "tweo_residual_add_q8", "tweo_residual_add_q8_rows",
     "tweo_workspace_bytes", "tweo_workspace_init", "tweo_read_device_status", "tweo_selftest_bounded_wait",
     "tweo_status_string", "tweo_last_cuda_error", "tweo_version", "tweo_launch_count",
@@ -112,6 +112,7 @@ def lib() -> C.CDLL:
         L.tweo_fp4_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp, vp, vp]
         L.tweo_fp4_unpack.argtypes = [vp, i64, vp, vp]
         L.tweo_w4a4_static_gemm.argtypes = [vp, i64, vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, sz, vp]
+        L.tweo_fp4_weight_linear.argtypes = [vp, i64, i32, vp, vp, i64, vp, vp, i64, i64, i64, i64, vp]
         L.tweo_workspace_bytes.argtypes = [i32, i64, i64, i64]
         L.tweo_workspace_bytes.restype = sz
         L.tweo_workspace_init.argtypes = [vp, sz, vp]
@@ -583,6 +584,22 @@ def fp4_unpack(q4: torch.Tensor, shape, q8: torch.Tensor | None = None) -> torch
         q8 = torch.empty(tuple(shape), dtype=torch.uint8, device=q4.device)
     _check(lib().tweo_fp4_unpack(_dev(q4, U8, "q4"), n, _dev(q8, U8, "q8"), _stream()), "tweo_fp4_unpack")
     return q8
+
+
+def fp4_weight_linear(xq, sx_inv, w4, sw_inv, fmt_x=E4M3, y=None) -> torch.Tensor:
+    """tweo_fp4_weight_linear: few-token (M <= 128) linear on PACKED E2M1 weights w4 [N, K // 2]; xq [M, K] holds
+    FP8 codes (W4A8) or E2M1 carriers (W4A4)."""
+    M, K = xq.shape
+    N, Kb = w4.shape
+    if 2 * Kb != K:
+        raise ValueError("w4 must be [N, K // 2]")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=xq.device)
+    _check(lib().tweo_fp4_weight_linear(_dev(xq, U8, "xq"), _rows(xq, "xq"), fmt_x, _dev(sx_inv, torch.float32, "sx_inv"),
+                                        _dev(w4, U8, "w4"), _rows(w4, "w4"), _dev(sw_inv, torch.float32, "sw_inv"),
+                                        _dev(y, torch.bfloat16, "y"), _rows(y, "y"), M, N, K, _stream()),
+           "tweo_fp4_weight_linear")
+    return y
 
 
 def w4a4_static_gemm(x, sx, wq8, sw_inv, y=None, ws=None) -> torch.Tensor:

@@ -368,6 +368,23 @@ bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, 
 }
 
 // 2-D output tensor [rows, cols] of bf16 or fp32, boxes of {128 bytes, 32 rows}, 128-byte swizzle.
+// Packed 4-bit elements, two per byte, [outer rows] x [inner elements], row pitch ld_bytes: the load expands every 16
+// elements (8 bytes) to a 16-byte group in shared memory, so a box of 128 elements fills the same 128-byte swizzled
+// row as 128 one-byte elements and the kernels' stage layout and descriptors stay as they are.
+bool make_map_packed4(CUtensorMap* map, const void* base, int64_t inner_elems, int64_t outer, int64_t ld_bytes,
+                      int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner_elems, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)ld_bytes};
+  cuuint32_t box[2] = {128u, (cuuint32_t)box_outer};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 bool make_out_map(CUtensorMap* map, void* base, int64_t cols, int64_t rows, int64_t ld, bool f32) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
@@ -395,13 +412,19 @@ bool make_q_map(CUtensorMap* map, void* base, int64_t cols, int64_t rows, int64_
   return r == CUDA_SUCCESS;
 }
 
+// Operand format beyond the public FP8 enum: 4-bit E2M1 elements, which kind::f8f6f4 reads from shared memory in
+// 16-byte groups of 16 elements (8 bytes of codes, 8 of padding) -- the form a tensor map of the packed 4-bit type
+// expands them to on the way in.
+constexpr int kFmtE2M1 = 2;
+
 uint32_t make_idesc(int fmt_a, int fmt_b, bool a_mn, bool b_mn, int n, int m = BM) {
-  // [4,6) accumulator format (1 = fp32)   [7,10) A format   [10,13) B format (0 = E4M3, 1 = E5M2)
+  // [4,6) accumulator format (1 = fp32)   [7,10) A format   [10,13) B format (0 = E4M3, 1 = E5M2, 5 = E2M1)
   // [15] A major (1 = MN)   [16] B major   [17,23) N >> 3   [24,29) M >> 4
+  auto code = [](int f) { return f == TWEO_E5M2 ? 1u : (f == kFmtE2M1 ? 5u : 0u); };
   uint32_t d = 0;
   d |= 1u << 4;
-  d |= (uint32_t)(fmt_a == TWEO_E5M2 ? 1 : 0) << 7;
-  d |= (uint32_t)(fmt_b == TWEO_E5M2 ? 1 : 0) << 10;
+  d |= code(fmt_a) << 7;
+  d |= code(fmt_b) << 10;
   d |= (uint32_t)(a_mn ? 1 : 0) << 15;
   d |= (uint32_t)(b_mn ? 1 : 0) << 16;
   d |= (uint32_t)(n >> 3) << 17;
@@ -660,16 +683,20 @@ tweo_status_t run_fwd_act(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8
 
 // Forward product for M <= 128 (see gemm_skinny.cuh): W is streamed once, K is sliced over CTAs.  The caller has
 // filled the scale fields of `p`; this fills the shape, the ring and the slicing, and launches.
+// w_packed4: W holds packed E2M1 codes (two per byte, ldw in BYTES); the ring and the kernel are the same, only the
+// tensor map of W differs (and the operand format in p.idesc, set by the caller).
 template <bool I8>
 tweo_status_t launch_skinny(SkinnyParams& p, const void* xq, int64_t ldx, const void* wq, int64_t ldw, int64_t M, int64_t N,
-                            int64_t K, cudaStream_t st) {
+                            int64_t K, cudaStream_t st, bool w_packed4 = false) {
   if (N > INT32_MAX || K > INT32_MAX) return TWEO_ERR_UNSUPPORTED_SHAPE;
   if (!aligned16(xq) || !aligned16(wq) || (ldx & 15) || (ldw & 15)) return TWEO_ERR_ALIGNMENT;
+  if (w_packed4 && ((reinterpret_cast<uintptr_t>(wq) & 31u) || (ldw & 31) || (K & 127))) return TWEO_ERR_ALIGNMENT;
   p.M = (int32_t)M;
   p.N = (int32_t)N;
   p.Mpad = (int32_t)((M + 15) / 16 * 16);
   p.k_blocks = (int32_t)((K + BK - 1) / BK);
   p.stage_bytes = (uint32_t)((BM * BK + p.Mpad * 128 + 1023) / 1024 * 1024);
+  p.w_tx_bytes = (uint32_t)(w_packed4 ? BM * BK / 2 : BM * BK);
   // A ring of at most 100 KB, so that two CTAs fit an SM: the CTAs of the next kernel of a launch chain become
   // resident (and fetch their first ring of W) while this kernel's are still reducing and writing.
   p.stages = (int32_t)((100 * 1024) / p.stage_bytes);
@@ -684,7 +711,8 @@ tweo_status_t launch_skinny(SkinnyParams& p, const void* xq, int64_t ldx, const 
   for (int sl = 2; sl <= 8; ++sl)
     if (slabs * sl <= 2 * sms && p.k_blocks / sl >= 4) p.slices = sl;
   CUtensorMap mw, mx;
-  if (!make_map(&mw, wq, K, N, ldw, BM) || !make_map(&mx, xq, K, M, ldx, p.Mpad)) {
+  const bool w_ok = w_packed4 ? make_map_packed4(&mw, wq, K, N, ldw, BM) : make_map(&mw, wq, K, N, ldw, BM);
+  if (!w_ok || !make_map(&mx, xq, K, M, ldx, p.Mpad)) {
     cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
     return TWEO_ERR_CUDA;
   }
@@ -713,6 +741,20 @@ tweo_status_t run_skinny(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_
   p.sw_inv = sw_inv;
   p.sx_is_scale = sx_is_scale ? 1 : 0;
   return launch_skinny<false>(p, xq, ldx, wq, ldw, M, N, K, st);
+}
+
+// The same with W as packed E2M1 codes: half the bytes of the stream that bounds the call.
+tweo_status_t run_skinny_w4(const uint8_t* xq, int64_t ldx, int fmt_x, const uint8_t* w4, int64_t ldw_bytes,
+                            const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M, int64_t N,
+                            int64_t K, cudaStream_t st) {
+  SkinnyParams p{};
+  p.y = y;
+  p.ldy = ldy;
+  p.idesc = make_idesc(kFmtE2M1, fmt_x, false, false, (int)((M + 15) / 16 * 16), BM);
+  p.sx_inv = sx_inv;
+  p.sw_inv = sw_inv;
+  p.sx_is_scale = 0;
+  return launch_skinny<false>(p, xq, ldx, w4, ldw_bytes, M, N, K, st, true);
 }
 
 // Up to kGroupMaxProblems independent products in ONE launch of the CTA-pair kernel (see gemm_pair_group.cuh).
@@ -1187,6 +1229,16 @@ tweo_status_t tweo_fp8_linear_group(const tweo_linear_problem_t* problems, int32
       return TWEO_ERR_ALIGNMENT;
   }
   return run_group(d, count, (cudaStream_t)stream);
+}
+
+tweo_status_t tweo_fp4_weight_linear(const uint8_t* xq, int64_t ldx, int32_t fmt_x, const float* sx_inv, const uint8_t* w4,
+                                     int64_t ldw_bytes, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M, int64_t N,
+                                     int64_t K, void* stream) {
+  if (!xq || !sx_inv || !w4 || !sw_inv || !y || !fmt_ok(fmt_x)) return TWEO_ERR_INVALID_ARG;
+  if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
+  if (M > 128 || (N & 15) || (K & 127)) return TWEO_ERR_UNSUPPORTED_SHAPE;
+  if (!tweo_detail::aligned16(y) || (ldy & 7)) return TWEO_ERR_ALIGNMENT;
+  return run_skinny_w4(xq, ldx, fmt_x, w4, ldw_bytes, sx_inv, sw_inv, y, ldy, M, N, K, (cudaStream_t)stream);
 }
 
 tweo_status_t tweo_selftest_bounded_wait(uint64_t limit_ns, uint32_t* gave_up, void* stream) {

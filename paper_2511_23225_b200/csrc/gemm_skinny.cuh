@@ -35,6 +35,8 @@ struct SkinnyParams {
   int32_t slices;          // slices of K = CTAs per cluster (1, 2, 4 or 8)
   int32_t stages;          // TMA ring depth (<= kSkinnyMaxStages)
   uint32_t stage_bytes;    // 16 KB of W + Mpad * 128 B of X, rounded up to 1 KB
+  uint32_t w_tx_bytes;     // bytes one W load reports to its barrier: the 16 KB it writes, or 8 KB for packed 4-bit
+                           // codes (the load counts the bytes it fetched, not the padded groups it writes)
   uint32_t tmem_cols;      // power of two >= max(32, Mpad)
   uint32_t idesc;
   const float* sx_inv;
@@ -127,7 +129,7 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
     if (lane == 0) {
       const int pre = min(p.stages, kb1 - kb0);   // the ring is empty: these stages need no wait
       for (int i = 0; i < pre; ++i) {
-        mbar_expect_tx(full_bar(i), BM * BK + x_bytes);
+        mbar_expect_tx(full_bar(i), p.w_tx_bytes + x_bytes);
         tma_load_2d(smem_base + i * p.stage_bytes, &tmap_w, (kb0 + i) * BK, n0, full_bar(i));
       }
       chain_wait();
@@ -138,7 +140,7 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
       for (int kb = kb0 + pre; kb < kb1; ++kb) {
         if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) break;
         const uint32_t fb = full_bar(stage);
-        mbar_expect_tx(fb, BM * BK + x_bytes);
+        mbar_expect_tx(fb, p.w_tx_bytes + x_bytes);
         const uint32_t sw = smem_base + stage * p.stage_bytes;
         tma_load_2d(sw, &tmap_w, kb * BK, n0, fb);
         tma_load_2d(sw + BM * BK, &tmap_x, kb * BK, 0, fb);

@@ -125,3 +125,45 @@ def test_w4a4_static_gemm_matches_oracle(tw, M, N, K):
     got = y.float().cpu().numpy().astype(np.float64)[rows, cols]
     # exact accumulation of exact products; two binary32 roundings of the factor, one bf16 rounding of the output
     assert np.all(np.abs(got - want) <= np.abs(want) * (2.0 ** -8 + 2.0 ** -21) + 1e-30)
+
+
+@pytest.mark.parametrize("M,N,K,a4", [(16, 256, 512, False), (1, 512, 4096, False), (128, 1024, 2048, True),
+                                      (37, 528, 1152, True)],
+                         ids=["w4a8_small", "w4a8_one_token", "w4a4_128_tokens", "w4a4_ragged"])
+def test_packed_weight_linear_equals_the_carrier_product_and_the_oracle(tw, M, N, K, a4):
+    """Few tokens on PACKED E2M1 weights (the loads expand the codes, the tensor core reads 4-bit operands): bit for
+    bit what the FP8 forward product gives on the carriers of the same codes, and the FP64 sum over decoded codes."""
+    x = synth.normal_bf16(60, (M, K), 1.0)
+    w = synth.normal_bf16(61, (N, K), 0.02)
+    wr = orc.fp4_quantize_per_tensor_current(w)
+    wq = tw.fp4_quantize(to_gpu_bf16(w))
+    w4 = wq.q4.view(N, K // 2)
+    if a4:
+        xr = orc.fp4_quantize_per_tensor_current(x)
+        xq_dev = tw.fp4_quantize(to_gpu_bf16(x), packed=False)
+        xq, sx_inv, x_codes, x_fmt = xq_dev.q8, xq_dev.scale_inv, xr["codes"], orc.E2M1
+    else:
+        xr = orc.quantize_per_tensor_current(x, orc.E4M3)
+        xq_dev = tw.quantize_per_tensor(to_gpu_bf16(x), tw.E4M3)
+        xq, sx_inv, x_codes, x_fmt = xq_dev.q, xq_dev.scale_inv, xr["q"], orc.E4M3
+    y = tw.fp4_weight_linear(xq, sx_inv, w4, wq.scale_inv)
+    y_ref = tw.fp8_linear_fwd(xq, wq.q8, sx_inv, wq.scale_inv)
+    torch.cuda.synchronize()
+    assert tw.read_device_status() == 0
+    assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16))
+    rows, cols = np.repeat(np.arange(M), 8)[:256], np.tile(np.arange(0, N, max(1, N // 8))[:8], M)[:256]
+    want = orc.gemm_fwd_at(x_codes, x_fmt, wr["codes"], orc.E2M1, float(xr["scale_inv"]), float(wr["scale_inv"]), rows, cols)
+    got = y.float().cpu().numpy().astype(np.float64)[rows, cols]
+    assert np.all(np.abs(got - want) <= np.abs(want) * (2.0 ** -8 + 2.0 ** -21) + 1e-30)
+
+
+def test_packed_weight_linear_rejects_what_it_cannot_do(tw):
+    xq = torch.zeros((256, 512), dtype=torch.uint8, device="cuda")
+    w4 = torch.zeros((256, 256), dtype=torch.uint8, device="cuda")
+    one = torch.ones(1, dtype=torch.float32, device="cuda")
+    with pytest.raises(tw.TweoError) as e:
+        tw.fp4_weight_linear(xq, one, w4, one)                       # 256 tokens: not the weight-streaming case
+    assert e.value.status == 2
+    with pytest.raises(tw.TweoError) as e:
+        tw.fp4_weight_linear(xq[:16, :320], one, w4[:, :160], one)   # K = 320 is not a multiple of 128
+    assert e.value.status == 2

@@ -50,6 +50,8 @@ def test_readme_call_sequences():
     wq4 = tw.fp4_quantize(w, carriers=False)
     w8 = tw.fp4_unpack(wq4.q4, w.shape)
     y4 = tw.w4a4_static_gemm(x, torch.full((1,), 6.0 / 4.0, device="cuda"), w8, wq4.scale_inv)
+    y1 = tw.fp4_weight_linear(qx.q[:16], qx.scale_inv, wq4.q4.view(N, K // 2), wq4.scale_inv)
     torch.cuda.synchronize()
+    assert y1.shape == (16, N)
     assert y4.shape == (M, N) and wq4.q4.numel() == N * K // 2
     assert yq.dtype == torch.int8 and yq.shape == (M, K) and tw.read_device_status() == 0
