@@ -76,6 +76,46 @@ __device__ __forceinline__ float skinny_out(const SkinnyParams& p, uint32_t acc,
   return __fmul_rn(__fmul_rn(__int2float_rn((int)acc), ar), alpha);
 }
 
+// The cluster's reduction for one output column (this thread's): CTA `slice` of the cluster sums tokens slice,
+// slice + S, ... over all S slices in slice order, reading the partial sums the CTAs parked in their shared memory
+// ([token][128 columns] fp32) through distributed shared memory, TOK tokens at a time (TOK * SL loads in flight).
+// SL: the slice count rounded up to 2, 4 or 8.
+template <bool I8, int TOK, int SL>
+__device__ __forceinline__ void skinny_reduce(const SkinnyParams& p, uint32_t mine, int slice, int n, float alpha) {
+  uint32_t peer[SL];
+#pragma unroll
+  for (int sl = 0; sl < SL; ++sl) peer[sl] = map_to_cta(mine, (uint32_t)(sl < p.slices ? sl : 0));
+  for (int t0 = slice; t0 < p.M; t0 += TOK * p.slices) {
+    uint32_t v[TOK][SL];
+#pragma unroll
+    for (int u = 0; u < TOK; ++u) {
+      const int t = t0 + u * p.slices;
+#pragma unroll
+      for (int sl = 0; sl < SL; ++sl)
+        v[u][sl] = (sl < p.slices && t < p.M) ? ld_shared_cluster_b32(peer[sl] + (uint32_t)t * 512u) : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < TOK; ++u) {
+      const int t = t0 + u * p.slices;
+      uint32_t acc;
+      if (I8) {
+        int a = (int)v[u][0];
+#pragma unroll
+        for (int sl = 1; sl < SL; ++sl)
+          if (sl < p.slices) a += (int)v[u][sl];   // exact
+        acc = (uint32_t)a;
+      } else {
+        float a = __uint_as_float(v[u][0]);
+#pragma unroll
+        for (int sl = 1; sl < SL; ++sl)
+          if (sl < p.slices) a += __uint_as_float(v[u][sl]);  // slice order
+        acc = __float_as_uint(a);
+      }
+      if (t < p.M && n < p.N) p.y[(int64_t)t * p.ldy + n] = (uint16_t)f32_to_bf16_bits(skinny_out<I8>(p, acc, t, alpha));
+    }
+  }
+}
+
 // I8: signed 8-bit operands (tcgen05 kind::i8, int32 accumulators: partial sums of K slices add exactly) with the
 // Eq. 4 dequantisation in the epilogue, per tensor or per token (activation rows) / per channel (weight rows).
 template <bool I8>
@@ -218,39 +258,10 @@ gemm_fp8_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_
       const float alpha = I8 ? __ldg(p.col_scale + (p.col_scale_per_col ? min(n, p.N - 1) : 0))
                              : dequant_alpha(p.sx_inv, p.sw_inv, p.sx_is_scale);
       const uint32_t mine = smem_base + (uint32_t)col * 4u;
-      uint32_t peer[8];
-#pragma unroll
-      for (int sl = 0; sl < 8; ++sl) peer[sl] = map_to_cta(mine, (uint32_t)(sl < p.slices ? sl : 0));
-      // eight tokens at a time, so up to 64 remote loads are in flight per thread
-      for (int t0 = slice; t0 < p.M; t0 += 8 * p.slices) {
-        uint32_t v[8][8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int t = t0 + u * p.slices;
-#pragma unroll
-          for (int sl = 0; sl < 8; ++sl)
-            v[u][sl] = (sl < p.slices && t < p.M) ? ld_shared_cluster_b32(peer[sl] + (uint32_t)t * 512u) : 0u;
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int t = t0 + u * p.slices;
-          uint32_t acc;
-          if (I8) {
-            int a = (int)v[u][0];
-#pragma unroll
-            for (int sl = 1; sl < 8; ++sl)
-              if (sl < p.slices) a += (int)v[u][sl];   // exact
-            acc = (uint32_t)a;
-          } else {
-            float a = __uint_as_float(v[u][0]);
-#pragma unroll
-            for (int sl = 1; sl < 8; ++sl)
-              if (sl < p.slices) a += __uint_as_float(v[u][sl]);  // slice order
-            acc = __float_as_uint(a);
-          }
-          if (t < p.M && n < p.N) p.y[(int64_t)t * p.ldy + n] = (uint16_t)f32_to_bf16_bits(skinny_out<I8>(p, acc, t, alpha));
-        }
-      }
+      // 64 remote loads in flight per thread whatever the slice count: 8, 16 or 32 tokens at a time
+      if (p.slices > 4) skinny_reduce<I8, 8, 8>(p, mine, slice, n, alpha);
+      else if (p.slices > 2) skinny_reduce<I8, 16, 4>(p, mine, slice, n, alpha);
+      else skinny_reduce<I8, 32, 2>(p, mine, slice, n, alpha);
     }
     cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
   }

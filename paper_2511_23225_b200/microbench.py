@@ -112,6 +112,12 @@ def make(op, M, K, N):
         ws = tw.new_workspace(tw.OP_W8A8, M, N, K)
         sx = _scalar(2.0)
         return (lambda: tw.w4a4_static_gemm(x, sx, wq.q8, wq.scale_inv, y=y, ws=ws)), 2.0 * M * K * N, "TFLOP/s"
+    if op == "w4_few_tokens":  # M <= 128 tokens of FP8 codes against PACKED E2M1 weights [N, K/2]
+        xq = _codes((M, K), 1)
+        w4 = torch.randint(0, 256, (N, K // 2), dtype=torch.uint8, device="cuda")
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        s = _scalar(1e-3)
+        return (lambda: tw.fp4_weight_linear(xq, s, w4, s, y=y)), float(M * K + K * N // 2 + 2 * M * N), "GB/s"
     if op == "loss":          # TWEO loss and bf16 gradient of one [M, K] block output
         a = [_bf16((M, K), 1.0, 1)]
         g = [torch.empty_like(a[0])]
@@ -165,7 +171,7 @@ def make(op, M, K, N):
 
 
 OPS = ("quantize", "quantize_given", "linear", "linear_fused", "linear_group", "linear_group_fused", "quantize_given_batch", "loss", "block_output", "layernorm", "fwd_gelu", "fwd_swiglu", "absmax", "int8_linear_q8",
-       "residual_add_q8", "w8a8", "fp4_quantize", "w4a4")
+       "residual_add_q8", "w8a8", "fp4_quantize", "w4a4", "w4_few_tokens")
 
 
 def main():
