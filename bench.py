@@ -52,7 +52,7 @@ UNIT = "TFLOP/s"
 FP8_DATASHEET_TFLOPS = 4500.0
 # DRAM traffic of the dominant kernel family (the GEMM launches of a step), per launch, from the ncu captures of
 # single launches summarised under profiles/; reported only while the GEMM sources are the ones profiled.
-GEMM_TRAFFIC = {"sources": "91273a37be8bd483", "workload": "cfg4", "variant": "fused", "dram_over_algorithmic": 1.09,
+GEMM_TRAFFIC = {"sources": "599990533a70756d", "workload": "cfg4", "variant": "fused", "dram_over_algorithmic": 1.09,
                 "from": "profiles/gemm_pair_group_kernel_fused_epilogue_cfg2_qkv_cfg4_qkv.md (one linear's grouped launch, "
                         "scaled by the algorithmic bytes of the family)"}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, FALLBACK_BF16_SUSTAINED = 6650.0, 1590.0, 1400.0

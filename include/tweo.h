@@ -567,6 +567,12 @@ TWEO_API tweo_status_t tweo_read_device_status(void* stream);
  */
 TWEO_API tweo_status_t tweo_selftest_bounded_wait(uint64_t limit_ns, uint32_t* gave_up, void* stream);
 
+/*
+ * Diagnostics.  With TWEO_LOG=1 in the environment (read once per process) every entry point prints one line to
+ * stderr before anything else: its name, shapes, formats, pitches and which optional pointers are set.  Nothing is
+ * read from the device and nothing is synchronised.  Device-side by-products that serve as metrics are ordinary
+ * outputs: amax of every cast and fused epilogue, the optional saturation counter, the loss scalars.
+ */
 TWEO_API const char* tweo_status_string(tweo_status_t s);
 TWEO_API const char* tweo_last_cuda_error(void); /* text of the last failing CUDA call in this thread */
 TWEO_API int32_t tweo_version(void);             /* major * 10000 + minor * 100 + patch */

@@ -151,6 +151,7 @@ size_t absmax_workspace_bytes() { return (size_t)kMaxSlots * sizeof(uint32_t); }
 extern "C" tweo_status_t tweo_absmax_quantize(const uint16_t* x, int64_t rows, int64_t cols, int64_t ldx, int32_t bits,
                                               int32_t granularity, int32_t mode, float eps, float* s, int8_t* q,
                                               int64_t ldq, void* ws, size_t ws_bytes, void* stream) {
+  TWEO_LOG_CALL("tweo_absmax_quantize " "rows=%lld cols=%lld ldx=%lld bits=%d", (long long)rows,(long long)cols,(long long)ldx,bits);
   if (rows < 0 || cols < 0 || !s) return TWEO_ERR_INVALID_ARG;
   if (bits < 2 || bits > 8) return TWEO_ERR_INVALID_ARG;
   if (granularity != TWEO_GRAN_TENSOR && granularity != TWEO_GRAN_ROW) return TWEO_ERR_INVALID_ARG;
@@ -247,6 +248,7 @@ __global__ void __launch_bounds__(256) residual_add_q8_kernel(const int8_t* xq, 
 
 extern "C" tweo_status_t tweo_residual_add_q8(const int8_t* xq, const float* sx, const int8_t* fq, const float* sf,
                                               int64_t n, int32_t bits, const float* sy, int8_t* yq, void* stream) {
+  TWEO_LOG_CALL("tweo_residual_add_q8 " "n=%lld bits=%d", (long long)n,bits);
   if (n < 0 || bits < 2 || bits > 8 || !sx || !sf || !sy) return TWEO_ERR_INVALID_ARG;
   if (n == 0) return TWEO_OK;
   if (!xq || !fq || !yq) return TWEO_ERR_INVALID_ARG;
@@ -353,6 +355,7 @@ cudaError_t launch_row_add(const RowAddArgs& a, cudaStream_t st) {
 extern "C" tweo_status_t tweo_residual_add_q8_rows(const int8_t* xq, const float* sx, const int8_t* fq, const float* sf,
                                                    int64_t rows, int64_t cols, int32_t bits, float eps, int8_t* yq,
                                                    float* sy, void* stream) {
+  TWEO_LOG_CALL("tweo_residual_add_q8_rows " "rows=%lld cols=%lld bits=%d eps=%g", (long long)rows,(long long)cols,bits,(double)eps);
   if (rows < 0 || cols < 1 || bits < 2 || bits > 8 || !(eps >= 0.0f)) return TWEO_ERR_INVALID_ARG;
   if ((cols & 15) || cols > 8192) return TWEO_ERR_UNSUPPORTED_SHAPE;
   if (rows == 0) return TWEO_OK;

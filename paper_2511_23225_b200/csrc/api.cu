@@ -1,5 +1,6 @@
 // Library-wide helpers: status strings, error text, launch counter, workspace sizing.
 #include <atomic>
+#include <cstdarg>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -23,6 +24,23 @@ int sm_count() {
     cached[dev] = n;
   }
   return cached[dev];
+}
+
+bool log_enabled() {
+  static const bool on = [] {
+    const char* v = getenv("TWEO_LOG");
+    return v && *v && strcmp(v, "0") != 0;
+  }();
+  return on;
+}
+
+void log_call(const char* fmt, ...) {
+  char line[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(line, sizeof line, fmt, ap);
+  va_end(ap);
+  fprintf(stderr, "[tweo] %s\n", line);
 }
 
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }

@@ -261,6 +261,7 @@ extern "C" tweo_status_t tweo_block_output_fused(const uint16_t* x, const uint16
                                                  float p, float grad_coeff, uint16_t* a, uint16_t* grad, float* loss,
                                                  float* amax, uint8_t* aq, int32_t q_fmt, const float* q_scale,
                                                  void* ws, size_t ws_bytes, void* stream) {
+  TWEO_LOG_CALL("tweo_block_output_fused " "n=%lld tau=%g eps=%g p=%g c=%g grad=%p aq=%p q_fmt=%d ws_bytes=%zu", (long long)n,(double)tau,(double)eps,(double)p,(double)grad_coeff,(void*)grad,(void*)aq,q_fmt,ws_bytes);
   if (n < 0 || !loss || !amax) return TWEO_ERR_INVALID_ARG;
   if (n > 0 && (!x || !f || !a)) return TWEO_ERR_INVALID_ARG;
   if (!(p > 1.0f) || !(tau + eps > 0.0f)) return TWEO_ERR_INVALID_ARG;
@@ -306,6 +307,7 @@ extern "C" tweo_status_t tweo_block_output_fused(const uint16_t* x, const uint16
 extern "C" tweo_status_t tweo_delayed_scaling_update(float* amax_history, int32_t history_len, const float* amax_new,
                                                      float* scale, float* scale_inv, int32_t n_tensors, int32_t fmt,
                                                      void* stream) {
+  TWEO_LOG_CALL("tweo_delayed_scaling_update " "history_len=%d n_tensors=%d fmt=%d", history_len,n_tensors,fmt);
   if (n_tensors < 0 || history_len < 1) return TWEO_ERR_INVALID_ARG;
   if (fmt != TWEO_E4M3 && fmt != TWEO_E5M2) return TWEO_ERR_INVALID_ARG;
   if (n_tensors == 0) return TWEO_OK;

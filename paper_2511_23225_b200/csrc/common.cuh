@@ -18,6 +18,12 @@ void count_launch(int n = 1);
 tweo_status_t cuda_fail(cudaError_t e, const char* what);  // records text, returns TWEO_ERR_CUDA
 tweo_status_t check_launch(const char* what);              // cudaGetLastError after a launch
 
+// TWEO_LOG=1 in the environment (read once): every entry point prints its name and its scalar arguments to stderr
+// before it does anything else -- shapes, formats, pitches, which optional pointers are set.  Nothing is read from
+// the device and nothing is synchronised.
+bool log_enabled();
+void log_call(const char* fmt, ...) __attribute__((format(printf, 1, 2)));
+
 // Device status word (bounded waits that expired); lives with the GEMM kernels.
 tweo_status_t read_and_clear_device_status(cudaStream_t stream);
 unsigned int* device_status_word();  // its device address on the current device (nullptr on failure)
@@ -47,6 +53,11 @@ inline void device_once_done(std::atomic<uint64_t>& mask, int dev) {
 }
 
 }  // namespace tweo_detail
+
+#define TWEO_LOG_CALL(...)                                               \
+  do {                                                                   \
+    if (tweo_detail::log_enabled()) tweo_detail::log_call(__VA_ARGS__);  \
+  } while (0)
 
 #define TWEO_CUDA_TRY(expr)                                              \
   do {                                                                   \

@@ -253,6 +253,7 @@ int cast_grid(int64_t n16, int u) {
 
 extern "C" tweo_status_t tweo_fp4_quantize(const uint16_t* x, int64_t n, int32_t mode, float* scale, float* scale_inv,
                                            float* amax, uint8_t* q4, uint8_t* q8, void* stream) {
+  TWEO_LOG_CALL("tweo_fp4_quantize " "x=%p n=%lld mode=%d q4=%p q8=%p", (const void*)x,(long long)n,mode,(void*)q4,(void*)q8);
   if (n < 0 || !scale || !scale_inv || !amax) return TWEO_ERR_INVALID_ARG;
   if (mode != TWEO_SCALE_CURRENT && mode != TWEO_SCALE_GIVEN) return TWEO_ERR_INVALID_ARG;
   if (n > 0 && (!x || (!q4 && !q8))) return TWEO_ERR_INVALID_ARG;
@@ -283,6 +284,7 @@ extern "C" tweo_status_t tweo_fp4_quantize(const uint16_t* x, int64_t n, int32_t
 }
 
 extern "C" tweo_status_t tweo_fp4_unpack(const uint8_t* q4, int64_t n, uint8_t* q8, void* stream) {
+  TWEO_LOG_CALL("tweo_fp4_unpack " "q4=%p n=%lld q8=%p", (const void*)q4,(long long)n,(void*)q8);
   if (n < 0 || (n > 0 && (!q4 || !q8))) return TWEO_ERR_INVALID_ARG;
   if (!aligned16(q8) || !aligned16(q4)) return TWEO_ERR_ALIGNMENT;
   if (n == 0) return TWEO_OK;
@@ -295,6 +297,7 @@ extern "C" tweo_status_t tweo_fp4_unpack(const uint8_t* q4, int64_t n, uint8_t* 
 extern "C" tweo_status_t tweo_w4a4_static_gemm(const uint16_t* x, int64_t ldx, const float* sx, const uint8_t* wq8,
                                                int64_t ldw, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
                                                int64_t N, int64_t K, void* ws, size_t ws_bytes, void* stream) {
+  TWEO_LOG_CALL("tweo_w4a4_static_gemm " "M=%lld N=%lld K=%lld ldx=%lld ldw=%lld ws_bytes=%zu", (long long)M,(long long)N,(long long)K,(long long)ldx,(long long)ldw,ws_bytes);
   if (!x || !sx || !wq8 || !sw_inv || !y) return TWEO_ERR_INVALID_ARG;
   if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
   if ((N & 15) || (K & 15) || ldx != K) return TWEO_ERR_UNSUPPORTED_SHAPE;

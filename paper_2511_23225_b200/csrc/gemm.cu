@@ -1090,6 +1090,7 @@ tweo_status_t tweo_fp8_linear_fwd(const uint8_t* xq, int64_t ldx, const uint8_t*
                                   const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
                                   int64_t N, int64_t K, int32_t fmt_x, int32_t fmt_w, const tweo_epilogue_t* epi,
                                   void* ws, size_t ws_bytes, void* stream) {
+  TWEO_LOG_CALL("tweo_fp8_linear_fwd " "M=%lld N=%lld K=%lld fmt_x=%d fmt_w=%d ldx=%lld ldw=%lld ldy=%lld epi=%p ws=%p", (long long)M,(long long)N,(long long)K,fmt_x,fmt_w,(long long)ldx,(long long)ldw,(long long)ldy,(const void*)epi,ws);
   if (!xq || !wq || !sx_inv || !sw_inv || !y || !fmt_ok(fmt_x) || !fmt_ok(fmt_w)) return TWEO_ERR_INVALID_ARG;
   if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
   if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
@@ -1101,6 +1102,7 @@ tweo_status_t tweo_fp8_linear_fwd_act(const uint8_t* xq, int64_t ldx, const uint
                                       const float* sx_inv, const float* sw_inv, int32_t act, uint16_t* y, int64_t ldy,
                                       int64_t M, int64_t N, int64_t K, int32_t fmt_x, int32_t fmt_w,
                                       const tweo_epilogue_t* epi, void* stream) {
+  TWEO_LOG_CALL("tweo_fp8_linear_fwd_act " "M=%lld N=%lld K=%lld act=%d fmt_x=%d fmt_w=%d epi=%p", (long long)M,(long long)N,(long long)K,act,fmt_x,fmt_w,(const void*)epi);
   if (act == TWEO_ACT_NONE)
     return tweo_fp8_linear_fwd(xq, ldx, wq, ldw, sx_inv, sw_inv, y, ldy, M, N, K, fmt_x, fmt_w, epi, nullptr, 0, stream);
   if (act != TWEO_ACT_GELU && act != TWEO_ACT_GELU_TANH && act != TWEO_ACT_SWIGLU) return TWEO_ERR_INVALID_ARG;
@@ -1122,6 +1124,7 @@ tweo_status_t tweo_fp8_linear_bwd_dgrad(const uint8_t* dyq, int64_t lddy, int32_
                                         int64_t ldw, int32_t fmt_w, const float* sdy_inv, const float* sw_inv,
                                         uint16_t* dx, int64_t lddx, int64_t M, int64_t N, int64_t K,
                                         const tweo_epilogue_t* epi, void* ws, size_t ws_bytes, void* stream) {
+  TWEO_LOG_CALL("tweo_fp8_linear_bwd_dgrad " "M=%lld N=%lld K=%lld fmt_dy=%d fmt_w=%d epi=%p ws=%p", (long long)M,(long long)N,(long long)K,fmt_dy,fmt_w,(const void*)epi,ws);
   if (!dyq || !wq || !sdy_inv || !sw_inv || !dx || !fmt_ok(fmt_dy) || !fmt_ok(fmt_w)) return TWEO_ERR_INVALID_ARG;
   if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
   if ((N & 15) || (K & 15)) return TWEO_ERR_UNSUPPORTED_SHAPE;
@@ -1143,6 +1146,7 @@ tweo_status_t tweo_fp8_linear_bwd_wgrad(const uint8_t* xq, int64_t ldx, int32_t 
                                         int64_t lddy, int32_t fmt_dy, const float* sx_inv, const float* sdy_inv,
                                         void* dw, int64_t lddw, int32_t dw_dtype, int32_t accumulate, int64_t M,
                                         int64_t N, int64_t K, void* ws, size_t ws_bytes, void* stream) {
+  TWEO_LOG_CALL("tweo_fp8_linear_bwd_wgrad " "M=%lld N=%lld K=%lld fmt_x=%d fmt_dy=%d ws=%p", (long long)M,(long long)N,(long long)K,fmt_x,fmt_dy,ws);
   if (!xq || !dyq || !sx_inv || !sdy_inv || !dw || !fmt_ok(fmt_x) || !fmt_ok(fmt_dy)) return TWEO_ERR_INVALID_ARG;
   if (dw_dtype != TWEO_BF16 && dw_dtype != TWEO_F32) return TWEO_ERR_INVALID_ARG;
   if (accumulate && dw_dtype != TWEO_F32) return TWEO_ERR_INVALID_ARG;
@@ -1166,6 +1170,7 @@ tweo_status_t tweo_fp8_linear_bwd(const uint8_t* dyq, int64_t lddy, int32_t fmt_
                                   const float* sx_inv, const float* sw_inv, uint16_t* dx, int64_t lddx, uint16_t* dw,
                                   int64_t lddw, int64_t M, int64_t N, int64_t K, void* ws, size_t ws_bytes,
                                   void* stream) {
+  TWEO_LOG_CALL("tweo_fp8_linear_bwd " "M=%lld N=%lld K=%lld fmt_dy=%d fmt_x=%d fmt_w=%d ws=%p", (long long)M,(long long)N,(long long)K,fmt_dy,fmt_x,fmt_w,ws);
   if (!dyq || !xq || !wq || !sdy_inv || !sx_inv || !sw_inv || !dx || !dw) return TWEO_ERR_INVALID_ARG;
   if (!fmt_ok(fmt_dy) || !fmt_ok(fmt_x) || !fmt_ok(fmt_w)) return TWEO_ERR_INVALID_ARG;
   if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
@@ -1187,6 +1192,7 @@ tweo_status_t tweo_fp8_linear_bwd(const uint8_t* dyq, int64_t lddy, int32_t fmt_
 }
 
 tweo_status_t tweo_fp8_linear_group(const tweo_linear_problem_t* problems, int32_t count, void* stream) {
+  TWEO_LOG_CALL("tweo_fp8_linear_group " "problems=%p count=%d", (const void*)problems, count);
   if (!problems || count < 1 || count > TWEO_MAX_GROUP) return TWEO_ERR_INVALID_ARG;
   GroupDesc d[TWEO_MAX_GROUP];
   for (int i = 0; i < count; ++i) {
@@ -1234,6 +1240,7 @@ tweo_status_t tweo_fp8_linear_group(const tweo_linear_problem_t* problems, int32
 tweo_status_t tweo_fp4_weight_linear(const uint8_t* xq, int64_t ldx, int32_t fmt_x, const float* sx_inv, const uint8_t* w4,
                                      int64_t ldw_bytes, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M, int64_t N,
                                      int64_t K, void* stream) {
+  TWEO_LOG_CALL("tweo_fp4_weight_linear " "M=%lld N=%lld K=%lld fmt_x=%d ldx=%lld ldw_bytes=%lld", (long long)M,(long long)N,(long long)K,fmt_x,(long long)ldx,(long long)ldw_bytes);
   if (!xq || !sx_inv || !w4 || !sw_inv || !y || !fmt_ok(fmt_x)) return TWEO_ERR_INVALID_ARG;
   if (M < 1 || N < 1 || K < 1) return TWEO_ERR_INVALID_ARG;
   if (M > 128 || (N & 15) || (K & 127)) return TWEO_ERR_UNSUPPORTED_SHAPE;
@@ -1251,6 +1258,7 @@ tweo_status_t tweo_selftest_bounded_wait(uint64_t limit_ns, uint32_t* gave_up, v
 tweo_status_t tweo_int8_linear(const int8_t* xq, int64_t ldx, const float* sx, int32_t sx_per_row, const int8_t* wq,
                                int64_t ldw, const float* sw, int32_t sw_per_row, int32_t bits, uint16_t* y, int64_t ldy,
                                int64_t M, int64_t N, int64_t K, void* stream) {
+  TWEO_LOG_CALL("tweo_int8_linear " "M=%lld N=%lld K=%lld bits=%d sx_per_row=%d sw_per_row=%d", (long long)M,(long long)N,(long long)K,bits,sx_per_row,sw_per_row);
   if (!y) return TWEO_ERR_INVALID_ARG;
   return tweo_detail::run_int8_linear(xq, ldx, sx, sx_per_row, wq, ldw, sw, sw_per_row, bits, y, ldy, nullptr, 0,
                                       nullptr, M, N, K, (cudaStream_t)stream);
@@ -1259,6 +1267,7 @@ tweo_status_t tweo_int8_linear(const int8_t* xq, int64_t ldx, const float* sx, i
 tweo_status_t tweo_int8_linear_q8(const int8_t* xq, int64_t ldx, const float* sx, int32_t sx_per_row, const int8_t* wq,
                                   int64_t ldw, const float* sw, int32_t sw_per_row, int32_t bits, const float* sy,
                                   int8_t* yq, int64_t ldq, int64_t M, int64_t N, int64_t K, void* stream) {
+  TWEO_LOG_CALL("tweo_int8_linear_q8 " "M=%lld N=%lld K=%lld bits=%d sx_per_row=%d sw_per_row=%d ldq=%lld", (long long)M,(long long)N,(long long)K,bits,sx_per_row,sw_per_row,(long long)ldq);
   if (!yq || !sy) return TWEO_ERR_INVALID_ARG;
   return tweo_detail::run_int8_linear(xq, ldx, sx, sx_per_row, wq, ldw, sw, sw_per_row, bits, nullptr, 0, yq, ldq, sy,
                                       M, N, K, (cudaStream_t)stream);

@@ -308,6 +308,7 @@ extern "C" tweo_status_t tweo_loss_fwd_bwd(const uint16_t* const* a, int32_t L, 
                                            float eps, float p, float grad_coeff, float* loss,
                                            float* loss_per_block, void* const* grad, int32_t grad_dtype,
                                            void* ws, size_t ws_bytes, void* stream) {
+  TWEO_LOG_CALL("tweo_loss_fwd_bwd " "L=%d n=%lld tau=%g eps=%g p=%g c=%g grad=%p grad_dtype=%d ws_bytes=%zu", L,(long long)n_per_tensor,(double)tau,(double)eps,(double)p,(double)grad_coeff,(const void*)grad,grad_dtype,ws_bytes);
   tweo_status_t s = check_loss_args(a, L, n_per_tensor, tau, eps, p, loss, grad, grad_dtype);
   if (s != TWEO_OK) return s;
   const size_t need = tweo_workspace_bytes(TWEO_OP_LOSS, n_per_tensor, L, 0);

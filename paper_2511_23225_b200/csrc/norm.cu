@@ -201,6 +201,7 @@ extern "C" tweo_status_t tweo_layernorm_fp8(const uint16_t* x, int64_t ldx, int6
                                             int64_t ldy, uint8_t* yq, int64_t ldq, int32_t q_fmt,
                                             const float* q_scale, float* amax, float* mean, float* rstd,
                                             void* stream) {
+  TWEO_LOG_CALL("tweo_layernorm_fp8 " "rows=%lld d=%lld ldx=%lld kind=%d", (long long)rows,(long long)d,(long long)ldx,kind);
   if (rows < 0 || d < 1 || !gamma || (kind != TWEO_NORM_LAYER && kind != TWEO_NORM_RMS)) return TWEO_ERR_INVALID_ARG;
   if ((d & 7) || d > 8192) return TWEO_ERR_UNSUPPORTED_SHAPE;
   cudaStream_t st = (cudaStream_t)stream;

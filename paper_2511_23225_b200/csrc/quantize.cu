@@ -517,12 +517,14 @@ size_t quantize_workspace_bytes() { return kBatchWsBytes; }
 extern "C" tweo_status_t tweo_quantize_per_tensor(const uint16_t* x, int64_t n, int32_t fmt, int32_t mode,
                                                   float* scale, float* scale_inv, float* amax, uint8_t* q,
                                                   uint32_t* sat_count, void* ws, size_t ws_bytes, void* stream) {
+  TWEO_LOG_CALL("tweo_quantize_per_tensor " "x=%p n=%lld fmt=%d mode=%d q=%p ws=%p", (const void*)x, (long long)n, fmt, mode, (void*)q, ws);
   tweo_quant_desc_t d{x, n, fmt, mode, scale, scale_inv, amax, q, sat_count};
   return quantize_many(&d, 1, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 extern "C" tweo_status_t tweo_quantize_per_tensor_batch(const tweo_quant_desc_t* descs, int32_t count, void* ws,
                                                         size_t ws_bytes, void* stream) {
+  TWEO_LOG_CALL("tweo_quantize_per_tensor_batch " "descs=%p count=%d ws=%p ws_bytes=%zu", (const void*)descs, count, ws, ws_bytes);
   if (!descs || count < 1 || count > TWEO_MAX_QUANT_BATCH) return TWEO_ERR_INVALID_ARG;
   if (ws && !aligned16(ws)) return TWEO_ERR_ALIGNMENT;
   return quantize_many(descs, count, ws, ws_bytes, (cudaStream_t)stream);

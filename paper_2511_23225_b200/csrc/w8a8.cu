@@ -14,6 +14,7 @@ extern "C" tweo_status_t tweo_w8a8_static_gemm(const void* x, int32_t x_dtype, i
                                                const uint8_t* wq, int64_t ldw, const float* sw_inv, uint16_t* y,
                                                int64_t ldy, int64_t M, int64_t N, int64_t K, void* ws,
                                                size_t ws_bytes, void* stream) {
+  TWEO_LOG_CALL("tweo_w8a8_static_gemm " "M=%lld N=%lld K=%lld x_dtype=%d ldx=%lld ldw=%lld ws_bytes=%zu", (long long)M,(long long)N,(long long)K,x_dtype,(long long)ldx,(long long)ldw,ws_bytes);
   using namespace tweo_detail;
   if (!x || !sx || !wq || !sw_inv || !y) return TWEO_ERR_INVALID_ARG;
   if (x_dtype != TWEO_BF16 && x_dtype != TWEO_FP8_E4M3) return TWEO_ERR_INVALID_ARG;

@@ -43,3 +43,25 @@ def test_binding_refuses_cpu_tensors():
     from paper_2511_23225_b200 import binding
     with pytest.raises(TypeError):
         binding.quantize_per_tensor(torch.zeros(16, dtype=torch.bfloat16))
+
+
+def test_tweo_log_dumps_the_arguments_of_a_call():
+    """TWEO_LOG=1: every entry point prints its name and scalar arguments to stderr before anything else -- also for a
+    call that the argument check then rejects, which is what can run without a GPU."""
+    import subprocess
+    import sys
+    code = (
+        "from paper_2511_23225_b200 import binding\n"
+        "L = binding.lib()\n"
+        "print(L.tweo_fp8_linear_fwd(None, 768, None, 768, None, None, None, 2304, 8192, 2304, 768, 0, 1, None, None, 0, None))\n"
+        "print(L.tweo_fp4_unpack(None, 4096, None, None))\n")
+    for env_value, expect in (("1", True), ("0", False), (None, False)):
+        env = dict(os.environ)
+        env.pop("TWEO_LOG", None)
+        if env_value is not None:
+            env["TWEO_LOG"] = env_value
+        r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=env, capture_output=True, text=True, timeout=300)
+        assert r.returncode == 0 and r.stdout.split() == ["1", "1"]            # both rejected: NULL operands
+        logged = "[tweo] tweo_fp8_linear_fwd M=8192 N=2304 K=768 fmt_x=0 fmt_w=1 ldx=768 ldw=768 ldy=2304" in r.stderr
+        assert logged == expect
+        assert ("[tweo] tweo_fp4_unpack" in r.stderr and "n=4096" in r.stderr) == expect
