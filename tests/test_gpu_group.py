@@ -147,3 +147,42 @@ def test_group_rejects_fused_outputs_on_a_weight_gradient(tw):
     with pytest.raises((tw.TweoError, TypeError)):   # an FP8 copy without its scale
         tw.fp8_linear_group([dict(product=tw.PRODUCT_FWD, xq=xq, wq=wq, sx_inv=sx, sw_inv=sw, out=y,
                                   out_q=torch.empty((256, 384), dtype=torch.uint8, device="cuda"))])
+
+
+def test_group_beyond_the_tile_list_capacity_deals_tiles_round_robin(tw):
+    """More tiles than the largest per-pair tile list holds (8192): the kernel deals them round-robin instead.  One
+    wide forward product of 8320 tiles (contraction 128, so it stays cheap) with the fused epilogue, and a small data
+    gradient behind it in the same launch; bit-identical to the single calls, sampled against the oracle."""
+    M, K, N = 256 * 128, 128, 256 * 65
+    g = np.random.Generator(np.random.PCG64(700))
+    xq_h = (g.integers(0, 256, (M, K), dtype=np.uint8) & 0xBF)          # finite E4M3 codes
+    wq_h = (g.integers(0, 256, (N, K), dtype=np.uint8) & 0xBF)
+    xq, wq = torch.from_numpy(xq_h).cuda(), torch.from_numpy(wq_h).cuda()
+    sx, sw, qs = dev_scalar(2.0 ** -7), dev_scalar(2.0 ** -6), dev_scalar(0.37)
+    q2, (xq2, wq2, dyq2), (sx2, sw2, sd2) = make_linear(710, 300, 400, 272)
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    yq = torch.zeros((M, N), dtype=torch.uint8, device="cuda")
+    am = torch.full((1,), 9.0, dtype=torch.float32, device="cuda")
+    dx2 = torch.zeros((300, 400), dtype=torch.bfloat16, device="cuda")
+    tw.fp8_linear_group([
+        dict(product=tw.PRODUCT_FWD, xq=xq, wq=wq, sx_inv=sx, sw_inv=sw, out=y, out_amax=am, out_q=yq, q_fmt=E4M3, q_scale=qs),
+        dict(product=tw.PRODUCT_DGRAD, dyq=dyq2, wq=wq2, sdy_inv=sd2, sw_inv=sw2, out=dx2)])
+    y1 = torch.empty_like(y)
+    yq1 = torch.empty_like(yq)
+    am1 = torch.zeros(1, dtype=torch.float32, device="cuda")
+    tw.fp8_linear_fwd(xq, wq, sx, sw, y=y1, out_amax=am1, out_q=yq1, q_fmt=E4M3, q_scale=qs)
+    dx1 = tw.fp8_linear_bwd_dgrad(dyq2, wq2, sd2, sw2)
+    torch.cuda.synchronize()
+    assert tw.read_device_status() == 0
+    assert torch.equal(y.view(torch.int16), y1.view(torch.int16)) and torch.equal(yq, yq1) and torch.equal(am, am1)
+    assert torch.equal(dx2.view(torch.int16), dx1.view(torch.int16))
+    assert float(am.item()) == float(y.abs().max().item())
+    del y1, yq1
+    rows = np.concatenate([g.integers(0, M, 300), [0, M - 1, M - 1]])
+    cols = np.concatenate([g.integers(0, N, 300), [0, N - 1, 0]])
+    want = orc.gemm_fwd_at(xq_h, E4M3, wq_h, E4M3, 2.0 ** -7, 2.0 ** -6, rows, cols)
+    got = y[torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()].float().cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -8 + 1e-30)
+    out_bits = y[:512].contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+    q_ref, _ = orc.quantize_bf16(out_bits, E4M3, np.float32(0.37))
+    assert np.array_equal(yq[:512].cpu().numpy(), q_ref)
