@@ -50,6 +50,24 @@ def test_quantize_beyond_2_31_elements(tw, big, fmt, with_ws):
     del out, q
 
 
+def test_fp4_quantize_beyond_2_31_elements(tw, big):
+    x, idx, bits = big
+    ref = orc.fp4_quantize_per_tensor_current(bits)            # the planted values decide amax and scale
+    out = tw.fp4_quantize(x)
+    torch.cuda.synchronize()
+    assert np.float32(out.amax.item()) == ref["amax"] == np.float32(250.0)
+    assert np.float32(out.scale.item()) == ref["scale"]
+    lut = np.array([orc.fp8_encode(orc.fp4_decode(c), E4M3) for c in range(16)], dtype=np.uint8)
+    assert np.array_equal(out.q8[idx].cpu().numpy(), lut[ref["codes"]])
+    pos = np.array(list(PLANTED.keys()), dtype=np.int64)
+    packed = out.q4[torch.from_numpy(pos // 2).cuda()].cpu().numpy()
+    assert np.array_equal((packed >> (4 * (pos & 1))) & 0xF, ref["codes"])
+    # nothing but the planted values with a non-zero code (a negative zero included) is set, in either form
+    nonzero = int(np.count_nonzero(ref["codes"]))
+    assert int(torch.count_nonzero(out.q8).item()) == nonzero and int(torch.count_nonzero(out.q4).item()) == nonzero
+    del out
+
+
 def test_tweo_loss_and_gradient_beyond_2_31_elements(tw, big):
     x, idx, bits = big
     tau, eps, p, c = 3.0, 1e-6, 4.0, 0.01
