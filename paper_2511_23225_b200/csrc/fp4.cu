@@ -17,6 +17,9 @@ tweo_status_t gemm_fwd_codes(const uint8_t* xq, int64_t ldx, int fmt_x, const ui
                              const float* sx_inv, const float* sw_inv, uint16_t* y, int64_t ldy, int64_t M,
                              int64_t N, int64_t K, const tweo_epilogue_t* epi, void* ws, size_t ws_bytes,
                              cudaStream_t st, bool sx_is_scale);
+// amax reset (+ reciprocal of a given scale) and, for current scaling, the amax pass: shared with the FP8 casts
+tweo_status_t launch_amax_prologue(const uint16_t* x, int64_t n, float* amax, uint32_t* sat_count, const float* scale_in,
+                                   float* scale_inv, cudaStream_t st);
 }
 
 namespace {
@@ -71,52 +74,6 @@ __device__ __forceinline__ float e2m1_scale_from_amax(float amax) {
     if (s > 3.402823466e38f) s = 3.402823466e38f;
   }
   return s;
-}
-
-__global__ void fp4_init_kernel(float* amax, const float* scale_in, float* scale_inv) {
-  chain_release();
-  chain_wait();
-  *amax = 0.0f;
-  if (scale_in) *scale_inv = __fdiv_rn(1.0f, *scale_in);
-}
-
-__global__ void __launch_bounds__(kThreads) fp4_amax_kernel(const uint16_t* x, int64_t n, float* amax) {
-  chain_release();
-  chain_wait();
-  const int64_t nvec = n >> 3;
-  const uint4* xv = reinterpret_cast<const uint4*>(x);
-  const int64_t stride = (int64_t)gridDim.x * kThreads * 4;
-  uint32_t m = 0;
-  for (int64_t base = (int64_t)blockIdx.x * kThreads * 4 + threadIdx.x; base < nvec; base += stride) {
-    uint4 v[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      int64_t i = base + (int64_t)u * kThreads;
-      v[u] = i < nvec ? __ldg(xv + i) : make_uint4(0, 0, 0, 0);
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      m = absmax_bits(m, v[u].x);
-      m = absmax_bits(m, v[u].y);
-      m = absmax_bits(m, v[u].z);
-      m = absmax_bits(m, v[u].w);
-    }
-  }
-  if (blockIdx.x == 0 && threadIdx.x < 8) {
-    int64_t i = (nvec << 3) + threadIdx.x;
-    if (i < n) m = absmax_bits(m, (uint32_t)x[i]);
-  }
-  m = absmax_fold(m);
-  __shared__ uint32_t part[kThreads / 32];
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = m;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-#pragma unroll
-    for (int w = 1; w < kThreads / 32; ++w) m = max(m, part[w]);
-    if (m) atomicMax(reinterpret_cast<unsigned int*>(amax), m << 16);  // non-negative binary32 order like their bits
-  }
 }
 
 // 16 elements per thread and pass: two 16-byte loads -> 8 bytes of packed codes and / or 16 carrier bytes.
@@ -260,15 +217,8 @@ extern "C" tweo_status_t tweo_fp4_quantize(const uint16_t* x, int64_t n, int32_t
   if (!aligned16(x) || !aligned16(q8) || (reinterpret_cast<uintptr_t>(q4) & 7u)) return TWEO_ERR_ALIGNMENT;
   cudaStream_t st = (cudaStream_t)stream;
   const bool given = mode == TWEO_SCALE_GIVEN;
-  TWEO_CUDA_TRY(launch_chain(fp4_init_kernel, dim3(1), dim3(1), 0, st, 0, amax,
-                             given ? (const float*)scale : (const float*)nullptr, scale_inv));
-  count_launch();
-  if (!given) {
-    const int64_t it = ((n >> 3) + kThreads * 4 - 1) / (kThreads * 4);
-    TWEO_CUDA_TRY(launch_chain(fp4_amax_kernel, dim3(balanced_grid(it, (int64_t)sm_count() * 8)), dim3(kThreads), 0, st, 0,
-                               x, n, amax));
-    count_launch();
-  }
+  tweo_status_t ps = launch_amax_prologue(x, n, amax, nullptr, given ? (const float*)scale : (const float*)nullptr, scale_inv, st);
+  if (ps != TWEO_OK) return ps;
   const int64_t n16 = n >> 4;
   const bool deep = n16 >= (int64_t)sm_count() * 8 * kThreads * 8;
   const dim3 grid(cast_grid(n16, deep ? 4 : 2));

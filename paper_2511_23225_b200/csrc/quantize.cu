@@ -19,6 +19,11 @@
 
 #include "common.cuh"
 
+namespace tweo_detail {
+tweo_status_t launch_amax_prologue(const uint16_t* x, int64_t n, float* amax, uint32_t* sat_count, const float* scale_in,
+                                   float* scale_inv, cudaStream_t st);
+}
+
 namespace {
 
 using namespace tweo_detail;
@@ -456,14 +461,9 @@ cudaError_t launch_cast(const tweo_quant_desc_t& d, cudaStream_t st) {
 
 tweo_status_t launch_single(const tweo_quant_desc_t& d, cudaStream_t st) {
   const bool given = d.mode == TWEO_SCALE_GIVEN;
-  TWEO_CUDA_TRY(launch_chain(init_kernel, dim3(1), dim3(1), 0, st, 0, d.amax, d.sat_count,
-                             given ? (const float*)d.scale : (const float*)nullptr, d.scale_inv));
-  count_launch();
-  if (!given) {
-    TWEO_CUDA_TRY(launch_chain(amax_kernel, dim3(grid_for(d.n >> 3, kThreads * 4, 8)), dim3(kThreads), 0, st, 0, d.x, d.n,
-                               d.amax));
-    count_launch();
-  }
+  tweo_status_t ps = tweo_detail::launch_amax_prologue(d.x, d.n, d.amax, d.sat_count,
+                                                       given ? (const float*)d.scale : (const float*)nullptr, d.scale_inv, st);
+  if (ps != TWEO_OK) return ps;
   const bool sat = d.sat_count != nullptr;
   cudaError_t e;
   if (d.fmt == TWEO_E4M3) {
@@ -511,6 +511,19 @@ tweo_status_t quantize_many(const tweo_quant_desc_t* descs, int count, void* ws,
 }  // namespace
 
 namespace tweo_detail {
+// The first launches of every one-tensor cast (FP8 here, FP4 in fp4.cu): the reset of amax (and of the saturation
+// counter; with a given scale also its reciprocal), then, for current scaling (scale_in == nullptr), the amax pass.
+tweo_status_t launch_amax_prologue(const uint16_t* x, int64_t n, float* amax, uint32_t* sat_count, const float* scale_in,
+                                   float* scale_inv, cudaStream_t st) {
+  TWEO_CUDA_TRY(launch_chain(init_kernel, dim3(1), dim3(1), 0, st, 0, amax, sat_count, scale_in, scale_inv));
+  count_launch();
+  if (!scale_in) {
+    TWEO_CUDA_TRY(launch_chain(amax_kernel, dim3(grid_for(n >> 3, kThreads * 4, 8)), dim3(kThreads), 0, st, 0, x, n, amax));
+    count_launch();
+  }
+  return TWEO_OK;
+}
+
 size_t quantize_workspace_bytes() { return kBatchWsBytes; }
 }
 
